@@ -1,0 +1,271 @@
+/*
+ * scalify.h - C ABI of the B200 (sm_100a) scaled-array kernels.
+ *
+ * The operations are the scaled primitives of "Scalify: scale propagation for
+ * efficient low-precision LLM training" (arxiv 2407.17353).  A ScaledArray is
+ * a pair (data, scale) whose value is data * scale (Section 2).  Here `data`
+ * is a device buffer in a low-precision format and `scale` is ONE fp32 power
+ * of two kept in DEVICE memory (Section 2: E8M0 scale simulated in float32;
+ * Section 3.1: scalar scale per tensor).  Every scale this library writes is a
+ * power of two obtained by rounding DOWN (Section 3.2, last paragraph).
+ *
+ * General contract
+ *   - All `scalify_array.data`, `.scale`, workspace, statistic, mean/rinv
+ *     pointers are DEVICE pointers owned by the caller.  The library
+ *     allocates no device memory and frees nothing.  Descriptor structs and
+ *     the arrays of descriptors passed to the Adam call are HOST memory and
+ *     are read before the call returns.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *     Calls only enqueue work; they never synchronise, except
+ *     scalify_check_status.
+ *   - A NULL `scale` pointer on an INPUT means "unscaled array", scale 1
+ *     (Section 3.1, get_data_and_scale).  A NULL `scale` on an OUTPUT means
+ *     the propagated scale is not stored.
+ *   - Input scale words must be finite positive powers of two within
+ *     [2^-126, 2^126]; a violation detected on the device sets
+ *     SCALIFY_DEV_BAD_SCALE in the workspace status word where a workspace
+ *     is available.
+ *   - Layout: row-major, `shape[0..ndim-1]` outermost first, `stride[]` in
+ *     elements, innermost stride 1, data pointer 16-byte aligned and every
+ *     outer stride a multiple of 16 bytes.
+ *   - An output scale word must not alias an input scale word of the same
+ *     call unless a function says otherwise (SCALIFY_ERR_ALIAS).
+ *   - Return value: 0 on success, a negative scalify_error otherwise.  A call
+ *     that fails validation enqueues nothing.  No call aborts, throws, or
+ *     traps on the device; every device-side wait is bounded and reports
+ *     SCALIFY_DEV_TIMEOUT in the status word when it expires.
+ *   - Rounding: data are converted round-to-nearest-even; FP8 conversions
+ *     saturate to the largest finite value; subnormals are kept.
+ */
+#ifndef SCALIFY_H_
+#define SCALIFY_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  SCALIFY_E4M3 = 0, /* OCP FP8 E4M3 (finite only, max 448)  - forward operands (Section 1, Appendix A) */
+  SCALIFY_E5M2 = 1, /* OCP FP8 E5M2 (max 57344)             - backward gradients (Section 1, Appendix A) */
+  SCALIFY_F16 = 2,  /* IEEE binary16 */
+  SCALIFY_BF16 = 3, /* bfloat16 */
+  SCALIFY_F32 = 4   /* IEEE binary32 */
+} scalify_dtype;
+
+typedef enum {
+  SCALIFY_STAT_NONE = 0,
+  SCALIFY_STAT_AMAX = 1, /* max |data| */
+  SCALIFY_STAT_L2 = 2    /* sqrt(mean(data^2)), the "L2 moment" of Section 3.3 */
+} scalify_stat;
+
+typedef enum {
+  SCALIFY_OK = 0,
+  SCALIFY_ERR_NULL = -1,        /* a required pointer is NULL */
+  SCALIFY_ERR_DTYPE = -2,       /* dtype not valid for this argument */
+  SCALIFY_ERR_SHAPE = -3,       /* shapes inconsistent or out of range */
+  SCALIFY_ERR_ALIGNMENT = -4,   /* pointer or stride not 16-byte aligned, innermost stride not 1 */
+  SCALIFY_ERR_WORKSPACE = -5,   /* workspace missing or too small */
+  SCALIFY_ERR_UNSUPPORTED = -6, /* valid but not implemented combination */
+  SCALIFY_ERR_CUDA = -7,        /* a CUDA runtime/driver call failed (see scalify_last_cuda_error) */
+  SCALIFY_ERR_ALIAS = -8,       /* forbidden aliasing of scale words or buffers */
+  SCALIFY_ERR_VALUE = -9        /* scalar argument out of range */
+} scalify_error;
+
+/* Bits of the device status word (first 4 bytes of any workspace). */
+enum {
+  SCALIFY_DEV_TIMEOUT = 1u,        /* a bounded device-side wait expired; results of that call are invalid */
+  SCALIFY_DEV_BAD_SCALE = 2u,      /* an input scale word was not a finite positive power of two */
+  SCALIFY_DEV_NONFINITE_STAT = 4u  /* a statistic was NaN or Inf; the rescale used factor 1 */
+};
+
+typedef struct scalify_array {
+  void* data;        /* device pointer, 16-byte aligned */
+  int32_t dtype;     /* scalify_dtype */
+  int32_t ndim;      /* 1..3 */
+  int64_t shape[3];  /* outermost first; unused entries ignored */
+  int64_t stride[3]; /* in elements; stride[ndim-1] must be 1 */
+  float* scale;      /* device pointer to one fp32 power of two, or NULL */
+} scalify_array;
+
+/* Operation codes for scalify_workspace_bytes. */
+enum {
+  SCALIFY_OP_MATMUL = 0,        /* d0 = batch*M, d1 = N */
+  SCALIFY_OP_RESCALE = 1,       /* d0 = number of elements, d1 unused */
+  SCALIFY_OP_LAYERNORM_BWD = 2, /* d0 = rows, d1 = row length */
+  SCALIFY_OP_ADAM = 3,          /* d0 = number of tensors, d1 unused */
+  SCALIFY_OP_STATISTIC = 4      /* d0 = number of elements */
+};
+
+/* Bytes of workspace the given call needs (an upper bound; always >= 4096).
+ * The first 256 bytes of a workspace form a header (status word, statistic
+ * word, reduction tickets); scalify_workspace_init must have zeroed it once
+ * before first use.  One workspace may serve successive calls on one stream;
+ * two calls that may overlap on the GPU need separate workspaces. */
+size_t scalify_workspace_bytes(int op, int64_t d0, int64_t d1);
+
+/* Zero the workspace header (asynchronously, on `stream`). */
+int scalify_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
+
+/* Synchronise `stream`, read and clear the status word of `workspace`.
+ * Returns the SCALIFY_DEV_* bits (>= 0) or a negative scalify_error. */
+int scalify_check_status(void* workspace, void* stream);
+
+const char* scalify_status_string(int code);
+/* The cudaError_t value recorded by the last call that returned SCALIFY_ERR_CUDA (per host thread). */
+int scalify_last_cuda_error(void);
+int scalify_version(void);
+
+/*
+ * Scaled matrix multiply (Section 3.2, the matmul rule of Algorithm 3; the
+ * mixed-format FP8 operands and higher-precision output of Appendix A).
+ *
+ *   Y_s = A_s * B_s * kf(K),   Y_d = (op(A)_d . op(B)_d) / kf(K)
+ *
+ * with kf(K) = sqrt(K) rounded down to a power of two: under the paper's
+ * assumption of independent unit-variance operands the contraction has
+ * variance K, so dividing the data by kf(K) restores unit scale, and the
+ * output scale depends only on the operand scales and the shape.
+ *
+ *   A : FP8 (E4M3 or E5M2), [M,K] (or [K,M] when transA != 0), ndim 2, or
+ *       ndim 3 with a leading batch dimension.
+ *   B : FP8 (E4M3 or E5M2, may differ from A), [K,N] (or [N,K] when transB).
+ *       A 2-D B with a 3-D A is shared by all batches.
+ *   Y : BF16, F16 or F32, [M,N] (or [batch,M,N]); receives the fp32
+ *       accumulator times 1/kf(K), rounded once.  Y->scale receives Y_s.
+ *   stat: statistic of the STORED Y data gathered in the epilogue (Section
+ *       3.3).  SCALIFY_STAT_NONE: none.  Otherwise the statistic is left, as
+ *       one fp32, at byte offset 16 of the workspace.
+ *   Yq: optional (may be NULL; requires stat != NONE).  Receives the dynamic
+ *       rescale of Y: r = statistic rounded down to a power of two,
+ *       Yq_d = cast(Y_d / r), Yq_s = Y_s * r.  Any dtype; same shape as Y.
+ *
+ * Accumulation is fp32 on the tensor cores (tcgen05, kind::f8f6f4).  Row
+ * strides must be multiples of 16 bytes.  Errors: see scalify_error.
+ */
+int scalify_scaled_matmul(const scalify_array* A, int transA, const scalify_array* B, int transB,
+                          scalify_array* Y, int stat, scalify_array* Yq,
+                          void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Statistic of the data component of X (Section 3.3: "L2 moment (or any other
+ * statistic)"), written as one fp32 to `out_stat` (device) and to byte offset
+ * 16 of the workspace.  X may be any dtype, contiguous.
+ */
+int scalify_statistic(const scalify_array* X, int stat, float* out_stat,
+                      void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Rescaling family (Sections 3.1 and 3.3; Algorithm 4).  Y has the same shape
+ * as X, any dtype; both contiguous.  Y may alias X (same buffer) only when the
+ * two dtypes have the same size.
+ *
+ *   stat == AMAX or L2, new_scale == NULL, stat_in == NULL:
+ *       dynamic_rescale: s = statistic(X_d); r = s rounded down to a power of
+ *       two (r = 1 when s is zero, non-finite or below 2^-126);
+ *       Y_d = cast(X_d / r); Y_s = X_s * r.  Needs a workspace.
+ *   stat == AMAX or L2, stat_in != NULL (device fp32):
+ *       delayed rescale: as above with s read from *stat_in instead of being
+ *       computed (Section 3.3: statistic gathered elsewhere, kept in state).
+ *   stat == NONE, new_scale != NULL (device fp32):
+ *       set_scaling: s' = *new_scale rounded down to a power of two;
+ *       Y_d = cast(X_d * X_s / s'); Y_s = s'.  With X->scale == NULL this is
+ *       as_scaled_array of an unscaled input.  Y->scale must not alias X->scale.
+ *   stat == NONE, new_scale == NULL:
+ *       plain cast (cast_on_forward / cast_on_backward of Appendix A):
+ *       Y_d = cast(X_d); Y_s = X_s.
+ *
+ * Y->scale may alias X->scale for the dynamic and delayed forms (in-place
+ * rebalance of a state tensor).
+ */
+int scalify_rescale(const scalify_array* X, int stat, const float* new_scale, const float* stat_in,
+                    scalify_array* Y, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Scaled add / subtract (Section 3.2, the add rule of Algorithm 3):
+ *   Y_s = sqrt(A_s^2 + B_s^2) rounded down to a power of two (= max(A_s,B_s)),
+ *   Y_d = cast(A_d*(A_s/Y_s) +- B_d*(B_s/Y_s)).
+ * A: [M,N] (or any contiguous shape); B: same shape as A, or a vector [N]
+ * broadcast over the rows of A (bias).  A and B: F16, BF16 or F32, same
+ * dtype; Y any dtype.  Y may alias A's buffer when sizes match.
+ */
+int scalify_scaled_add(const scalify_array* A, const scalify_array* B, int subtract,
+                       scalify_array* Y, void* stream);
+
+/*
+ * Scaled LayerNorm forward (Section 3.2.1 and Appendix C.2): the data
+ * component is normalised and the result carries scale 1, whatever X_s is:
+ *   n = (x_d - mean) / (sqrt(var) + eps)        (eps_inside_sqrt == 0, as printed)
+ *   n = (x_d - mean) / sqrt(var + eps)          (eps_inside_sqrt != 0, textbook)
+ * followed by the affine part through the ordinary mul and add rules:
+ *   Y_s = max(gamma_s, beta_s),  Y_d = cast(n*gamma_d*(gamma_s/Y_s) + beta_d*(beta_s/Y_s)).
+ * X: [R,d] F16/BF16/F32, d*elem_size a multiple of 16 bytes, d <= 16384.
+ * gamma, beta: [d], same dtype as each other (F16/BF16/F32), or both NULL
+ * (then Y_d = n, Y_s = 1).  Y: [R,d], any dtype.  mean, rinv: optional device
+ * fp32 [R] outputs (row mean and 1/(sigma+eps) or 1/sqrt(var+eps)), needed by
+ * the backward call.
+ */
+int scalify_scaled_layernorm(const scalify_array* X, const scalify_array* gamma, const scalify_array* beta,
+                             float eps, int eps_inside_sqrt, scalify_array* Y,
+                             float* mean, float* rinv, void* stream);
+
+/*
+ * Scaled LayerNorm backward with dynamic rescale of the input gradient
+ * (Section 4 and Algorithm 5: one dynamic rescale per residual branch, placed
+ * on the gradient that leaves the LayerNorm).
+ *   ghat = G_d*gamma_d;  dx = LayerNorm'(ghat; x_d)  (exact derivative of the
+ *   forward above);  dX_s = G_s*gamma_s / X_s;
+ *   dgamma_d = sum_rows(G_d*n)/kf(R), dbeta_d = sum_rows(G_d)/kf(R), both with
+ *   scale G_s*kf(R) (reduction over R rows treated like a contraction of size R).
+ * G, X: [R,d], F16/BF16/F32 (same dtype); mean, rinv: from the forward call.
+ * dX: [R,d] BF16/F16/F32: the un-rebalanced gradient (always written).
+ * stat_dx: statistic of the stored dX data, left at workspace offset 16.
+ * dXq: optional rescaled gradient (any dtype), as Yq of the matmul.
+ * dgamma, dbeta: optional [d] outputs, F32/BF16/F16 (both or neither).
+ */
+int scalify_scaled_layernorm_bwd(const scalify_array* G, const scalify_array* X, const scalify_array* gamma,
+                                 const float* mean, const float* rinv, float eps, int eps_inside_sqrt,
+                                 int stat_dx, scalify_array* dX, scalify_array* dXq,
+                                 scalify_array* dgamma, scalify_array* dbeta,
+                                 void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Scaled GELU forward / backward (Section 3.2.1 and Appendix C.1):
+ *   forward  (X_d * g(X_d*X_s), X_s);   backward  dX_d = G_d * f'(X_d*X_s), dX_s = G_s.
+ * exact_erf == 0: tanh form; != 0: Gaussian-CDF form.  X, G: F16/BF16/F32
+ * (same dtype), Y/dX any dtype, contiguous, same shape.
+ */
+int scalify_scaled_gelu(const scalify_array* X, int exact_erf, scalify_array* Y, void* stream);
+int scalify_scaled_gelu_bwd(const scalify_array* G, const scalify_array* X, int exact_erf,
+                            scalify_array* dX, void* stream);
+
+/*
+ * Scaled Adam step over a list of tensors (Sections 1, 3 and 4; Table 3 row 4:
+ * FP8 gradients, FP16 scaled optimizer state and master weights).  In value
+ * space this is textbook Adam with bias correction:
+ *   m' = b1*m + (1-b1)*g;  v' = b2*v + (1-b2)*g^2;
+ *   w' = w - lr * (m'/(1-b1^t)) / (sqrt(v'/(1-b2^t)) + eps)
+ * and the new scales follow from tracing that expression with the static
+ * rules (mul: product; add: max; div: ratio; sqrt: sqrt rounded down; a scalar
+ * constant c carries the scale "|c| rounded down to a power of two",
+ * Section 3.4):
+ *   m'_s = max(p2(b1)*m_s, p2(1-b1)*g_s)
+ *   v'_s = max(p2(b2)*v_s, p2(1-b2)*g_s^2)
+ *   u_s  = p2(lr) * (m'_s/p2(1-b1^t)) / max(p2(sqrt(v'_s/p2(1-b2^t))), p2(eps))
+ *   w'_s = max(w_s, u_s)
+ * Each of m', v', w' is rounded once from fp32 arithmetic.
+ *   grads[i]: any dtype (E5M2 typical); m[i], v[i]: F16 or F32 (same);
+ *   w[i]: F16, BF16 or F32.  All four have the same element count, are
+ *   contiguous, and m, v, w (data and scale words) are updated in place.
+ *   step >= 1 is t.  Needs a workspace (SCALIFY_OP_ADAM, n_tensors).
+ */
+int scalify_scaled_adam_step(int n_tensors, const scalify_array* grads, scalify_array* m, scalify_array* v,
+                             scalify_array* w, float lr, float beta1, float beta2, float eps, int64_t step,
+                             void* workspace, size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SCALIFY_H_ */

@@ -1,0 +1,258 @@
+"""Python binding of the scalify C ABI (``include/scalify.h``).
+
+Argument marshalling only: every arithmetic step runs in the CUDA library
+``libscalify.so`` (hand-written sm_100a kernels).  PyTorch supplies device
+memory and streams.  There is no CPU or PyTorch fallback: if the library
+cannot be loaded, importing the symbols below raises.
+
+A :class:`ScaledTensor` is the paper's ScaledArray (Section 2): ``data`` in a
+low-precision dtype plus ONE fp32 power-of-two ``scale`` kept on the device,
+with value = data * scale.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional, Sequence
+
+import torch
+
+from . import _build
+
+E4M3, E5M2, F16, BF16, F32 = 0, 1, 2, 3, 4
+STAT_NONE, STAT_AMAX, STAT_L2 = 0, 1, 2
+OP_MATMUL, OP_RESCALE, OP_LAYERNORM_BWD, OP_ADAM, OP_STATISTIC = 0, 1, 2, 3, 4
+DEV_TIMEOUT, DEV_BAD_SCALE, DEV_NONFINITE_STAT = 1, 2, 4
+
+_DTYPE_CODE = {torch.float8_e4m3fn: E4M3, torch.float8_e5m2: E5M2, torch.float16: F16,
+               torch.bfloat16: BF16, torch.float32: F32}
+TORCH_DTYPE = {v: k for k, v in _DTYPE_CODE.items()}
+
+
+class ScalifyError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = lib().scalify_status_string(code).decode()
+        extra = f" (cudaError {lib().scalify_last_cuda_error()})" if code == -7 else ""
+        super().__init__(f"{where}: {msg}{extra} [code {code}]")
+
+
+class scalify_array(ctypes.Structure):
+    _fields_ = [("data", ctypes.c_void_p), ("dtype", ctypes.c_int32), ("ndim", ctypes.c_int32),
+                ("shape", ctypes.c_int64 * 3), ("stride", ctypes.c_int64 * 3), ("scale", ctypes.c_void_p)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load ``libscalify.so`` (building it with nvcc if it is not there).  Raises if neither works."""
+    global _lib
+    if _lib is None:
+        path = _build.LIB
+        if not os.path.exists(path):
+            path = _build.build()
+        L = ctypes.CDLL(path)
+        c = ctypes
+        P = c.POINTER(scalify_array)
+        vp, i32, i64, f32, sz = c.c_void_p, c.c_int, c.c_int64, c.c_float, c.c_size_t
+        L.scalify_version.restype = i32
+        L.scalify_last_cuda_error.restype = i32
+        L.scalify_status_string.restype = c.c_char_p
+        L.scalify_status_string.argtypes = [i32]
+        L.scalify_workspace_bytes.restype = sz
+        L.scalify_workspace_bytes.argtypes = [i32, i64, i64]
+        L.scalify_workspace_init.argtypes = [vp, sz, vp]
+        L.scalify_check_status.argtypes = [vp, vp]
+        L.scalify_scaled_matmul.argtypes = [P, i32, P, i32, P, i32, P, vp, sz, vp]
+        L.scalify_statistic.argtypes = [P, i32, vp, vp, sz, vp]
+        L.scalify_rescale.argtypes = [P, i32, vp, vp, P, vp, sz, vp]
+        L.scalify_scaled_add.argtypes = [P, P, i32, P, vp]
+        L.scalify_scaled_layernorm.argtypes = [P, P, P, f32, i32, P, vp, vp, vp]
+        L.scalify_scaled_layernorm_bwd.argtypes = [P, P, P, vp, vp, f32, i32, i32, P, P, P, P, vp, sz, vp]
+        L.scalify_scaled_gelu.argtypes = [P, i32, P, vp]
+        L.scalify_scaled_gelu_bwd.argtypes = [P, P, i32, P, vp]
+        L.scalify_scaled_adam_step.argtypes = [i32, P, P, P, P, f32, f32, f32, f32, i64, vp, sz, vp]
+        for name in ("scalify_workspace_init", "scalify_check_status", "scalify_scaled_matmul", "scalify_statistic",
+                     "scalify_rescale", "scalify_scaled_add", "scalify_scaled_layernorm",
+                     "scalify_scaled_layernorm_bwd", "scalify_scaled_gelu", "scalify_scaled_gelu_bwd",
+                     "scalify_scaled_adam_step"):
+            getattr(L, name).restype = i32
+        _lib = L
+    return _lib
+
+
+@dataclass
+class ScaledTensor:
+    """ScaledArray (Section 2): value = data * scale.  ``scale`` is a 1-element fp32 CUDA tensor or None
+    (unscaled: scale 1)."""
+    data: torch.Tensor
+    scale: Optional[torch.Tensor] = None
+
+    @staticmethod
+    def empty(shape, dtype, device="cuda") -> "ScaledTensor":
+        return ScaledTensor(torch.empty(shape, dtype=dtype, device=device),
+                            torch.empty(1, dtype=torch.float32, device=device))
+
+    @staticmethod
+    def make(data: torch.Tensor, scale: float) -> "ScaledTensor":
+        return ScaledTensor(data, torch.full((1,), float(scale), dtype=torch.float32, device=data.device))
+
+    def scale_value(self) -> float:
+        return 1.0 if self.scale is None else float(self.scale.item())
+
+
+def _desc(t: Optional[ScaledTensor]):
+    """ctypes descriptor of a ScaledTensor (None -> NULL)."""
+    if t is None:
+        return None
+    d = t.data
+    if d.dim() < 1 or d.dim() > 3:
+        raise ValueError("scalify arrays have 1 to 3 dimensions")
+    a = scalify_array()
+    a.data = d.data_ptr()
+    a.dtype = _DTYPE_CODE[d.dtype]
+    a.ndim = d.dim()
+    for i in range(d.dim()):
+        a.shape[i] = d.shape[i]
+        a.stride[i] = d.stride(i)
+    if t.scale is not None:
+        if t.scale.dtype != torch.float32 or t.scale.numel() != 1 or t.scale.device != d.device:
+            raise ValueError("scale must be a 1-element fp32 tensor on the data's device")
+        a.scale = t.scale.data_ptr()
+    else:
+        a.scale = None
+    return a
+
+
+def _ref(a):
+    return None if a is None else ctypes.byref(a)
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else t.data_ptr()
+
+
+def _check(code: int, where: str) -> None:
+    if code != 0:
+        raise ScalifyError(code, where)
+
+
+class Workspace:
+    """Caller-owned scratch buffer with the zeroed 256-byte header the library expects."""
+
+    def __init__(self, nbytes: int, device="cuda", stream=None):
+        nbytes = max(int(nbytes), 4096)
+        self.buf = torch.empty(nbytes, dtype=torch.uint8, device=device)
+        self.nbytes = nbytes
+        _check(lib().scalify_workspace_init(self.buf.data_ptr(), nbytes, _stream(stream)), "scalify_workspace_init")
+
+    @property
+    def ptr(self) -> int:
+        return self.buf.data_ptr()
+
+    def statistic(self) -> torch.Tensor:
+        """The fp32 statistic word (byte offset 16) as a 1-element tensor view."""
+        return self.buf[16:20].view(torch.float32)
+
+    def check_status(self, stream=None) -> int:
+        return scalify_check_status(self, stream)
+
+
+def scalify_workspace_bytes(op: int, d0: int = 0, d1: int = 0) -> int:
+    return int(lib().scalify_workspace_bytes(op, int(d0), int(d1)))
+
+
+def scalify_check_status(ws: Workspace, stream=None) -> int:
+    rc = lib().scalify_check_status(ws.ptr, _stream(stream))
+    if rc < 0:
+        raise ScalifyError(rc, "scalify_check_status")
+    return rc
+
+
+def scalify_scaled_matmul(A: ScaledTensor, B: ScaledTensor, Y: ScaledTensor, ws: Workspace, *, transA=False,
+                          transB=False, stat: int = STAT_NONE, Yq: Optional[ScaledTensor] = None, stream=None) -> None:
+    a, b, y, yq = _desc(A), _desc(B), _desc(Y), _desc(Yq)
+    _check(lib().scalify_scaled_matmul(_ref(a), int(transA), _ref(b), int(transB), _ref(y), stat, _ref(yq),
+                                       ws.ptr, ws.nbytes, _stream(stream)), "scalify_scaled_matmul")
+
+
+def scalify_statistic(X: ScaledTensor, stat: int, ws: Workspace, out: Optional[torch.Tensor] = None, stream=None) -> None:
+    x = _desc(X)
+    _check(lib().scalify_statistic(_ref(x), stat, _ptr(out), ws.ptr, ws.nbytes, _stream(stream)), "scalify_statistic")
+
+
+def scalify_rescale(X: ScaledTensor, Y: ScaledTensor, *, stat: int = STAT_NONE, new_scale: Optional[torch.Tensor] = None,
+                    stat_in: Optional[torch.Tensor] = None, ws: Optional[Workspace] = None, stream=None) -> None:
+    x, y = _desc(X), _desc(Y)
+    _check(lib().scalify_rescale(_ref(x), stat, _ptr(new_scale), _ptr(stat_in), _ref(y),
+                                 None if ws is None else ws.ptr, 0 if ws is None else ws.nbytes, _stream(stream)),
+           "scalify_rescale")
+
+
+def scalify_scaled_add(A: ScaledTensor, B: ScaledTensor, Y: ScaledTensor, *, subtract=False, stream=None) -> None:
+    a, b, y = _desc(A), _desc(B), _desc(Y)
+    _check(lib().scalify_scaled_add(_ref(a), _ref(b), int(subtract), _ref(y), _stream(stream)), "scalify_scaled_add")
+
+
+def scalify_scaled_layernorm(X: ScaledTensor, gamma: Optional[ScaledTensor], beta: Optional[ScaledTensor],
+                             Y: ScaledTensor, *, eps: float = 1e-5, eps_inside_sqrt=False,
+                             mean: Optional[torch.Tensor] = None, rinv: Optional[torch.Tensor] = None,
+                             stream=None) -> None:
+    x, g, b, y = _desc(X), _desc(gamma), _desc(beta), _desc(Y)
+    _check(lib().scalify_scaled_layernorm(_ref(x), _ref(g), _ref(b), float(eps), int(eps_inside_sqrt), _ref(y),
+                                          _ptr(mean), _ptr(rinv), _stream(stream)), "scalify_scaled_layernorm")
+
+
+def scalify_scaled_layernorm_bwd(G: ScaledTensor, X: ScaledTensor, gamma: Optional[ScaledTensor], mean: torch.Tensor,
+                                 rinv: torch.Tensor, dX: ScaledTensor, ws: Workspace, *, eps: float = 1e-5,
+                                 eps_inside_sqrt=False, stat_dx: int = STAT_NONE, dXq: Optional[ScaledTensor] = None,
+                                 dgamma: Optional[ScaledTensor] = None, dbeta: Optional[ScaledTensor] = None,
+                                 stream=None) -> None:
+    g, x, gm, dx, dxq, dg, db = (_desc(G), _desc(X), _desc(gamma), _desc(dX), _desc(dXq), _desc(dgamma), _desc(dbeta))
+    _check(lib().scalify_scaled_layernorm_bwd(_ref(g), _ref(x), _ref(gm), _ptr(mean), _ptr(rinv), float(eps),
+                                              int(eps_inside_sqrt), stat_dx, _ref(dx), _ref(dxq), _ref(dg), _ref(db),
+                                              ws.ptr, ws.nbytes, _stream(stream)), "scalify_scaled_layernorm_bwd")
+
+
+def scalify_scaled_gelu(X: ScaledTensor, Y: ScaledTensor, *, exact_erf=False, stream=None) -> None:
+    x, y = _desc(X), _desc(Y)
+    _check(lib().scalify_scaled_gelu(_ref(x), int(exact_erf), _ref(y), _stream(stream)), "scalify_scaled_gelu")
+
+
+def scalify_scaled_gelu_bwd(G: ScaledTensor, X: ScaledTensor, dX: ScaledTensor, *, exact_erf=False, stream=None) -> None:
+    g, x, dx = _desc(G), _desc(X), _desc(dX)
+    _check(lib().scalify_scaled_gelu_bwd(_ref(g), _ref(x), int(exact_erf), _ref(dx), _stream(stream)),
+           "scalify_scaled_gelu_bwd")
+
+
+def _desc_array(ts: Sequence[ScaledTensor]):
+    arr = (scalify_array * len(ts))()
+    for i, t in enumerate(ts):
+        arr[i] = _desc(t)
+    return arr
+
+
+class AdamTensors:
+    """Marshalled descriptor arrays of a fixed parameter list (built once, reused every step)."""
+
+    def __init__(self, grads: Sequence[ScaledTensor], m: Sequence[ScaledTensor], v: Sequence[ScaledTensor],
+                 w: Sequence[ScaledTensor]):
+        assert len(grads) == len(m) == len(v) == len(w)
+        self.n = len(grads)
+        self.keep = (list(grads), list(m), list(v), list(w))
+        self.g, self.m, self.v, self.w = (_desc_array(grads), _desc_array(m), _desc_array(v), _desc_array(w))
+
+
+def scalify_scaled_adam_step(tensors: AdamTensors, ws: Workspace, *, lr: float, beta1: float, beta2: float, eps: float,
+                             step: int, stream=None) -> None:
+    _check(lib().scalify_scaled_adam_step(tensors.n, tensors.g, tensors.m, tensors.v, tensors.w, float(lr),
+                                          float(beta1), float(beta2), float(eps), int(step), ws.ptr, ws.nbytes,
+                                          _stream(stream)), "scalify_scaled_adam_step")

@@ -1,0 +1,402 @@
+// HBM-bound scaled elementwise kernels: statistic, rebalance / set_scaling /
+// cast, scaled add, scaled GELU.  Every kernel moves 16-byte vectors of its
+// widest operand per thread access, coalesced across the warp, with several
+// independent accesses in flight per thread; the grid is a multiple of the SM
+// count and strides over the array.
+#include "scalify_common.cuh"
+#include "scalify_launch.h"
+
+namespace scalify {
+
+constexpr int kThreads = 256;
+constexpr int kUnroll = 4;
+
+template <int A, int B> struct VecElems {
+  static constexpr int big = ElemBytes<A>::v > ElemBytes<B>::v ? ElemBytes<A>::v : ElemBytes<B>::v;
+  static constexpr int v = 16 / big;
+};
+
+static int grid_for(int64_t n_vec, int blocks_per_sm) {
+  int64_t tiles = (n_vec + int64_t(kThreads) * kUnroll - 1) / (int64_t(kThreads) * kUnroll);
+  int64_t cap = int64_t(sm_count()) * blocks_per_sm;
+  if (tiles < 1) tiles = 1;
+  return static_cast<int>(tiles < cap ? tiles : cap);
+}
+
+// ---------------------------------------------------------------------------------------------
+// statistic of the data component (Section 3.3): AMAX or root mean square
+// ---------------------------------------------------------------------------------------------
+// Each block leaves one partial (AMAX: bit pattern of max|x|; L2: fp64 sum of squares) in
+// `partials`; the block that draws the last ticket combines them in index order, so the result
+// does not depend on scheduling.
+template <int DT>
+__global__ void __launch_bounds__(kThreads) statistic_kernel(const void* __restrict__ x, int64_t n, int stat,
+                                                             double* __restrict__ partials, uint32_t* ticket,
+                                                             float* stat_word, float* out_stat) {
+  constexpr int VEC = 16 / ElemBytes<DT>::v;
+  constexpr int WORDS = 4;
+  const int64_t n_vec = n / VEC;
+  uint32_t amax = 0u;
+  float ssq = 0.f;
+  const int64_t stride = int64_t(gridDim.x) * kThreads * kUnroll;
+  for (int64_t base = int64_t(blockIdx.x) * kThreads * kUnroll; base < n_vec; base += stride) {
+    uint32_t w[kUnroll][WORDS];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      int64_t i = base + u * kThreads + threadIdx.x;
+      if (i < n_vec) ld_raw_stream<16>(static_cast<const char*>(x) + i * 16, w[u]);
+      else { w[u][0] = w[u][1] = w[u][2] = w[u][3] = 0u; }
+    }
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      float f[VEC];
+      decode_vec<DT, VEC>(w[u], f);
+#pragma unroll
+      for (int e = 0; e < VEC; ++e) {
+        amax = max(amax, abs_bits(f[e]));
+        ssq = fmaf(f[e], f[e], ssq);
+      }
+    }
+  }
+  if (blockIdx.x == 0 && threadIdx.x < static_cast<int>(n - n_vec * VEC)) {
+    float f = load_elem<DT>(x, n_vec * VEC + threadIdx.x);
+    amax = max(amax, abs_bits(f));
+    ssq = fmaf(f, f, ssq);
+  }
+  __shared__ double s_part[kThreads / 32];
+  __shared__ bool s_last;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  double mine;
+  if (stat == SCALIFY_STAT_AMAX) {
+    amax = warp_max_u32(amax);
+    mine = static_cast<double>(amax);
+  } else {
+    mine = warp_sum_f64(static_cast<double>(ssq));
+  }
+  if (lane == 0) s_part[warp] = mine;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double tot;
+    if (stat == SCALIFY_STAT_AMAX) {
+      uint32_t m = 0u;
+      for (int i = 0; i < kThreads / 32; ++i) m = max(m, static_cast<uint32_t>(s_part[i]));
+      tot = static_cast<double>(m);
+    } else {
+      tot = 0.0;
+      for (int i = 0; i < kThreads / 32; ++i) tot += s_part[i];
+    }
+    partials[blockIdx.x] = tot;
+    __threadfence();
+    uint32_t t = atomicAdd(ticket, 1u);
+    s_last = (t == gridDim.x - 1);
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  // fixed-order combination of the per-block partials
+  double acc = 0.0;
+  uint32_t accm = 0u;
+  for (int i = threadIdx.x; i < static_cast<int>(gridDim.x); i += kThreads) {
+    double p = __ldcg(&partials[i]);
+    if (stat == SCALIFY_STAT_AMAX) accm = max(accm, static_cast<uint32_t>(p));
+    else acc += p;
+  }
+  if (stat == SCALIFY_STAT_AMAX) {
+    accm = warp_max_u32(accm);
+    acc = static_cast<double>(accm);
+  } else {
+    acc = warp_sum_f64(acc);
+  }
+  __syncthreads();
+  if (lane == 0) s_part[warp] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float result;
+    if (stat == SCALIFY_STAT_AMAX) {
+      uint32_t m = 0u;
+      for (int i = 0; i < kThreads / 32; ++i) m = max(m, static_cast<uint32_t>(s_part[i]));
+      result = __uint_as_float(m);
+    } else {
+      double tot = 0.0;
+      for (int i = 0; i < kThreads / 32; ++i) tot += s_part[i];
+      result = static_cast<float>(sqrt(tot / static_cast<double>(n)));
+    }
+    *stat_word = result;
+    if (out_stat) *out_stat = result;
+    *ticket = 0u;
+  }
+}
+
+int launch_statistic(const void* x, int dtype, int64_t n, int stat, void* ws, float* out_stat, cudaStream_t st) {
+  WsView v = ws_view(ws);
+  constexpr int VECB = 16;
+  int64_t n_vec = n * elem_size(dtype) / VECB;
+  int grid = grid_for(n_vec, 8);
+  SCALIFY_DISPATCH_DTYPE(dtype, DT,
+      statistic_kernel<DT><<<grid, kThreads, 0, st>>>(x, n, stat, static_cast<double*>(v.area), v.ticket, v.stat,
+                                                      out_stat));
+  SCALIFY_CUDA_TRY(cudaGetLastError());
+  return SCALIFY_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// rebalance / set_scaling / cast (Sections 3.1, 3.3; Algorithm 4; Appendix A casts)
+// ---------------------------------------------------------------------------------------------
+
+template <int IN, int OUT>
+__global__ void __launch_bounds__(kThreads) rebalance_kernel(const void* __restrict__ x, void* __restrict__ y,
+                                                             int64_t n, const float* x_scale, float* y_scale,
+                                                             const float* stat, const float* new_scale, int mode,
+                                                             uint32_t* status) {
+  constexpr int VEC = VecElems<IN, OUT>::v;
+  constexpr int IB = VEC * ElemBytes<IN>::v, OB = VEC * ElemBytes<OUT>::v;
+  const float xs = load_scale(x_scale);
+  float factor = 1.0f, out_scale = xs;
+  uint32_t flags = is_pow2_scale(xs) ? 0u : SCALIFY_DEV_BAD_SCALE;
+  if (mode == kModeDynamic) {
+    bool nonfinite;
+    float r = rescale_factor(__ldg(stat), &nonfinite);
+    factor = 1.0f / r;  // exact: r is a power of two
+    out_scale = xs * r;
+    if (nonfinite) flags |= SCALIFY_DEV_NONFINITE_STAT;
+  } else if (mode == kModeSet) {
+    float req = __ldg(new_scale);
+    float ns = p2_floor(req);
+    if (!(req > 0.f) || !is_pow2_scale(ns)) { flags |= SCALIFY_DEV_BAD_SCALE; ns = 1.0f; }
+    factor = xs / ns;
+    out_scale = ns;
+  }
+  const int64_t n_vec = n / VEC;
+  const int64_t stride = int64_t(gridDim.x) * kThreads * kUnroll;
+  for (int64_t base = int64_t(blockIdx.x) * kThreads * kUnroll; base < n_vec; base += stride) {
+    uint32_t w[kUnroll][IB / 4];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      int64_t i = base + u * kThreads + threadIdx.x;
+      if (i < n_vec) ld_raw_stream<IB>(static_cast<const char*>(x) + i * IB, w[u]);
+    }
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      int64_t i = base + u * kThreads + threadIdx.x;
+      if (i < n_vec) {
+        float f[VEC];
+        decode_vec<IN, VEC>(w[u], f);
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) f[e] *= factor;
+        uint32_t o[OB / 4];
+        encode_vec<OUT, VEC>(f, o);
+        st_raw<OB>(static_cast<char*>(y) + i * OB, o);
+      }
+    }
+  }
+  if (blockIdx.x == 0) {
+    int tail = static_cast<int>(n - n_vec * VEC);
+    if (threadIdx.x < tail) {
+      int64_t i = n_vec * VEC + threadIdx.x;
+      store_elem<OUT>(y, i, load_elem<IN>(x, i) * factor);
+    }
+    if (threadIdx.x == 0) {
+      if (y_scale) *y_scale = out_scale;
+      if (flags && status) atomicOr(status, flags);
+    }
+  }
+}
+
+int launch_rebalance(const void* x, int in_dt, void* y, int out_dt, int64_t n, const float* x_scale, float* y_scale,
+                     const float* stat, const float* new_scale, int mode, uint32_t* status, cudaStream_t st) {
+  int big = elem_size(in_dt) > elem_size(out_dt) ? elem_size(in_dt) : elem_size(out_dt);
+  int64_t n_vec = n / (16 / big);
+  int grid = grid_for(n_vec, 8);
+  SCALIFY_DISPATCH_DTYPE(in_dt, IN, SCALIFY_DISPATCH_DTYPE(out_dt, OUT,
+      rebalance_kernel<IN, OUT><<<grid, kThreads, 0, st>>>(x, y, n, x_scale, y_scale, stat, new_scale, mode, status)));
+  SCALIFY_CUDA_TRY(cudaGetLastError());
+  return SCALIFY_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// scaled add / subtract (Section 3.2, add rule)
+// ---------------------------------------------------------------------------------------------
+struct FastDiv {
+  uint32_t d, magic, shift;
+};
+static FastDiv make_fastdiv(uint32_t d) {
+  FastDiv f;
+  f.d = d;
+  if (d == 1) { f.magic = 0; f.shift = 0; return f; }
+  uint32_t l = 0;
+  while ((1ull << l) < d) ++l;  // ceil(log2 d)
+  uint64_t m = ((1ull << 32) * ((1ull << l) - d)) / d + 1;
+  f.magic = static_cast<uint32_t>(m);
+  f.shift = l;
+  return f;
+}
+__device__ __forceinline__ uint32_t fastdiv(uint32_t n, FastDiv f) {
+  if (f.d == 1) return n;
+  uint32_t t = __umulhi(n, f.magic);
+  return (t + ((n - t) >> 1)) >> (f.shift - 1);
+}
+
+template <int AB, int OUT>
+__global__ void __launch_bounds__(kThreads) add_kernel(const void* __restrict__ a, const void* __restrict__ b,
+                                                       void* __restrict__ y, int64_t n, int64_t row_len,
+                                                       FastDiv row_vecs, int broadcast, const float* a_scale,
+                                                       const float* b_scale, float* y_scale, float sign) {
+  constexpr int VEC = VecElems<AB, OUT>::v;
+  constexpr int IB = VEC * ElemBytes<AB>::v, OB = VEC * ElemBytes<OUT>::v;
+  const float as = load_scale(a_scale), bs = load_scale(b_scale);
+  // sqrt(as^2+bs^2) rounded down to a power of two is max(as,bs) for power-of-two operands
+  const float ys = fmaxf(as, bs);
+  const float fa = as / ys, fb = sign * (bs / ys);
+  const int64_t n_vec = n / VEC;
+  const int64_t stride = int64_t(gridDim.x) * kThreads * kUnroll;
+  for (int64_t base = int64_t(blockIdx.x) * kThreads * kUnroll; base < n_vec; base += stride) {
+    uint32_t wa[kUnroll][IB / 4], wb[kUnroll][IB / 4];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      int64_t i = base + u * kThreads + threadIdx.x;
+      if (i < n_vec) {
+        ld_raw_stream<IB>(static_cast<const char*>(a) + i * IB, wa[u]);
+        if (broadcast) {
+          uint32_t iv = static_cast<uint32_t>(i);
+          uint32_t r = fastdiv(iv, row_vecs);
+          uint32_t c = iv - r * row_vecs.d;
+          ld_raw<IB>(static_cast<const char*>(b) + int64_t(c) * IB, wb[u]);
+        } else {
+          ld_raw_stream<IB>(static_cast<const char*>(b) + i * IB, wb[u]);
+        }
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      int64_t i = base + u * kThreads + threadIdx.x;
+      if (i < n_vec) {
+        float fa_[VEC], fb_[VEC];
+        decode_vec<AB, VEC>(wa[u], fa_);
+        decode_vec<AB, VEC>(wb[u], fb_);
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) fa_[e] = fmaf(fb_[e], fb, fa_[e] * fa);
+        uint32_t o[OB / 4];
+        encode_vec<OUT, VEC>(fa_, o);
+        st_raw<OB>(static_cast<char*>(y) + i * OB, o);
+      }
+    }
+  }
+  if (blockIdx.x == 0) {
+    int tail = static_cast<int>(n - n_vec * VEC);
+    if (threadIdx.x < tail) {
+      int64_t i = n_vec * VEC + threadIdx.x;
+      float av = load_elem<AB>(a, i);
+      float bv = load_elem<AB>(b, broadcast ? (i % row_len) : i);
+      store_elem<OUT>(y, i, fmaf(bv, fb, av * fa));
+    }
+    if (threadIdx.x == 0 && y_scale) *y_scale = ys;
+  }
+}
+
+int launch_add(const void* a, const void* b, int ab_dt, void* y, int out_dt, int64_t n, int64_t row_len, int broadcast,
+               const float* a_scale, const float* b_scale, float* y_scale, int subtract, cudaStream_t st) {
+  int big = elem_size(ab_dt) > elem_size(out_dt) ? elem_size(ab_dt) : elem_size(out_dt);
+  int vec = 16 / big;
+  int64_t n_vec = n / vec;
+  if (broadcast && (row_len % vec != 0 || n_vec >= (int64_t(1) << 31))) return SCALIFY_ERR_UNSUPPORTED;
+  FastDiv fd = make_fastdiv(static_cast<uint32_t>(broadcast ? row_len / vec : 1));
+  int grid = grid_for(n_vec, 8);
+  float sign = subtract ? -1.0f : 1.0f;
+  SCALIFY_DISPATCH_WIDE(ab_dt, AB, SCALIFY_DISPATCH_DTYPE(out_dt, OUT,
+      add_kernel<AB, OUT><<<grid, kThreads, 0, st>>>(a, b, y, n, row_len, fd, broadcast, a_scale, b_scale, y_scale,
+                                                     sign)));
+  SCALIFY_CUDA_TRY(cudaGetLastError());
+  return SCALIFY_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// scaled GELU (Appendix C.1): f(x) = x*g(x)
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ float gelu_u(float x) { return 0.7978845608028654f * fmaf(0.044715f * x * x, x, x); }
+
+// gate g(x): tanh form written as a logistic, 0.5*(1+tanh(u)) = 1/(1+exp(-2u)), which keeps
+// full relative accuracy where the gate is tiny
+template <int EXACT>
+__device__ __forceinline__ float gelu_gate(float x) {
+  if constexpr (EXACT) return 0.5f * (1.0f + erff(x * 0.7071067811865476f));
+  else return 1.0f / (1.0f + __expf(-2.0f * gelu_u(x)));
+}
+
+template <int EXACT>
+__device__ __forceinline__ float gelu_deriv(float x) {  // f'(x) = g + x*g'
+  if constexpr (EXACT) {
+    float g = 0.5f * (1.0f + erff(x * 0.7071067811865476f));
+    return fmaf(x, 0.3989422804014327f * __expf(-0.5f * x * x), g);
+  } else {
+    float g = 1.0f / (1.0f + __expf(-2.0f * gelu_u(x)));
+    float du = 0.7978845608028654f * fmaf(3.0f * 0.044715f * x, x, 1.0f);
+    return fmaf(x, 2.0f * g * (1.0f - g) * du, g);
+  }
+}
+
+template <int IN, int OUT, int EXACT, int BWD>
+__global__ void __launch_bounds__(kThreads) gelu_kernel(const void* __restrict__ x, const void* __restrict__ g,
+                                                        void* __restrict__ y, int64_t n, const float* x_scale,
+                                                        const float* g_scale, float* y_scale) {
+  constexpr int VEC = VecElems<IN, OUT>::v;
+  constexpr int IB = VEC * ElemBytes<IN>::v, OB = VEC * ElemBytes<OUT>::v;
+  const float xs = load_scale(x_scale);
+  const int64_t n_vec = n / VEC;
+  const int64_t stride = int64_t(gridDim.x) * kThreads * kUnroll;
+  for (int64_t base = int64_t(blockIdx.x) * kThreads * kUnroll; base < n_vec; base += stride) {
+    uint32_t wx[kUnroll][IB / 4], wg[kUnroll][IB / 4];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      int64_t i = base + u * kThreads + threadIdx.x;
+      if (i < n_vec) {
+        ld_raw_stream<IB>(static_cast<const char*>(x) + i * IB, wx[u]);
+        if (BWD) ld_raw_stream<IB>(static_cast<const char*>(g) + i * IB, wg[u]);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      int64_t i = base + u * kThreads + threadIdx.x;
+      if (i < n_vec) {
+        float fx[VEC], fg[VEC];
+        decode_vec<IN, VEC>(wx[u], fx);
+        if (BWD) decode_vec<IN, VEC>(wg[u], fg);
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) {
+          float v = fx[e] * xs;
+          fx[e] = BWD ? fg[e] * gelu_deriv<EXACT>(v) : fx[e] * gelu_gate<EXACT>(v);
+        }
+        uint32_t o[OB / 4];
+        encode_vec<OUT, VEC>(fx, o);
+        st_raw<OB>(static_cast<char*>(y) + i * OB, o);
+      }
+    }
+  }
+  if (blockIdx.x == 0) {
+    int tail = static_cast<int>(n - n_vec * VEC);
+    if (threadIdx.x < tail) {
+      int64_t i = n_vec * VEC + threadIdx.x;
+      float xd = load_elem<IN>(x, i);
+      float v = xd * xs;
+      store_elem<OUT>(y, i, BWD ? load_elem<IN>(g, i) * gelu_deriv<EXACT>(v) : xd * gelu_gate<EXACT>(v));
+    }
+    if (threadIdx.x == 0 && y_scale) *y_scale = BWD ? load_scale(g_scale) : xs;
+  }
+}
+
+int launch_gelu(const void* x, const void* g, int in_dt, void* y, int out_dt, int64_t n, const float* x_scale,
+                const float* g_scale, float* y_scale, int exact, int bwd, cudaStream_t st) {
+  int big = elem_size(in_dt) > elem_size(out_dt) ? elem_size(in_dt) : elem_size(out_dt);
+  int64_t n_vec = n / (16 / big);
+  int grid = grid_for(n_vec, 8);
+#define SCALIFY_GELU_LAUNCH(EX, BW) \
+  gelu_kernel<IN, OUT, EX, BW><<<grid, kThreads, 0, st>>>(x, g, y, n, x_scale, g_scale, y_scale)
+  SCALIFY_DISPATCH_WIDE(in_dt, IN, SCALIFY_DISPATCH_DTYPE(out_dt, OUT, {
+    if (exact) { if (bwd) SCALIFY_GELU_LAUNCH(1, 1); else SCALIFY_GELU_LAUNCH(1, 0); }
+    else { if (bwd) SCALIFY_GELU_LAUNCH(0, 1); else SCALIFY_GELU_LAUNCH(0, 0); }
+  }));
+#undef SCALIFY_GELU_LAUNCH
+  SCALIFY_CUDA_TRY(cudaGetLastError());
+  return SCALIFY_OK;
+}
+
+}  // namespace scalify

@@ -1,0 +1,480 @@
+// Scaled FP8 matmul for sm_100a (Section 3.2 matmul rule; Appendix A mixed E4M3/E5M2 operands,
+// higher-precision output):  Y_d = (op(A)_d . op(B)_d) / kf(K),  Y_s = A_s * B_s * kf(K).
+//
+// Persistent, warp-specialised kernel, one CTA per SM:
+//   warp 0      TMA producer: cp.async.bulk.tensor tiles of A and B into a kStages-deep ring of
+//               128-byte-swizzled shared-memory buffers, completion on mbarriers
+//   warp 1      MMA issuer: one thread issues tcgen05.mma (kind::f8f6f4, fp32 accumulate) from
+//               shared-memory descriptors into a TMEM accumulator; tcgen05.commit releases ring
+//               slots and publishes finished accumulators
+//   warps 2-5   epilogue: tcgen05.ld of the accumulator (two accumulators of 256 TMEM columns, so
+//               the epilogue of tile i overlaps the main loop of tile i+1), multiply by the exact
+//               power of two 1/kf(K), round once to the output type, 16-byte stores, and the
+//               statistic of the stored values (AMAX: warp-shuffle max + one atomicMax on the
+//               fp32 bit pattern per warp and tile; L2: per-warp partial sums in fixed slots)
+// Tile 128 x 256 x 128 (one 128-byte swizzle row of FP8 per K block, four K=32 MMAs per block).
+// Operands may be K-major (row-major [rows, K]) or MN-major (row-major [K, rows]); the layout is
+// expressed in the shared-memory descriptors and the instruction descriptor, not by copying.
+// Every wait on an mbarrier is bounded; on expiry the CTA records SCALIFY_DEV_TIMEOUT, drains
+// its own copies in flight, frees its TMEM and returns.
+#include <cuda.h>
+
+#include "scalify_common.cuh"
+#include "scalify_launch.h"
+
+namespace scalify {
+
+constexpr int kBM = 128;
+constexpr int kBN = 256;
+constexpr int kBK = 128;  // FP8 elements = bytes
+constexpr int kUmmaK = 32;
+constexpr int kStages = 4;
+constexpr int kAccStages = 2;
+constexpr int kGemmThreads = 192;
+constexpr int kABytes = kBM * kBK;           // 16 KB
+constexpr int kBBytes = kBN * kBK;           // 32 KB
+constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kTmemCols = kAccStages * kBN;  // 512
+constexpr int kGroupM = 16;                  // m-tiles per rasterisation group
+constexpr size_t kGemmSmem = size_t(kStages) * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
+
+struct GemmParams {
+  int M, N, K, batch;
+  int tiles_m, tiles_n;
+  int a_mn_major, b_mn_major;  // 0: K-major (row-major [rows,K]); 1: MN-major (row-major [K,rows])
+  uint32_t idesc;
+  float alpha;                 // 1/kf(K)
+  float kf;
+  void* Y;
+  long long ldy, y_batch_stride;  // elements
+  const float* a_scale;
+  const float* b_scale;
+  float* y_scale;
+  int stat;
+  uint32_t* stat_word;   // AMAX: atomicMax target
+  double* l2_partials;   // L2: [tiles][4]
+  uint32_t* status;
+};
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait: false when the limit expired or another role of this CTA has given up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_timer_ns();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 0xFFu) == 0u) {
+      if (*abort_flag) return false;
+      if (global_timer_ns() - t0 > kWaitLimitNs) {
+        *abort_flag = 1u;
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y), "r"(z)
+      : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_f8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1 (sm_100).
+//   bits [0,14)  start address >> 4      bits [16,30) leading-dimension byte offset >> 4
+//   bits [32,46) stride-dimension byte offset >> 4      bits [46,48) version = 1
+//   bits [61,64) layout type: 2 = SWIZZLE_128B
+// K-major tile ([rows][128 B of K]): 8-row swizzle atoms 1024 B apart (stride offset); the
+// leading offset is not used.  MN-major tile ([K rows][128 B of MN]): atoms of 8 K-rows are
+// 1024 B apart (stride offset) and successive 128-element MN chunks are `lbo` bytes apart.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);
+  d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= 1ull << 46;
+  d |= 2ull << 61;
+  return d;
+}
+
+__device__ __forceinline__ void tile_coords(const GemmParams& p, int tile, int& b, int& mt, int& nt) {
+  const int per_batch = p.tiles_m * p.tiles_n;
+  b = tile / per_batch;
+  const int t = tile - b * per_batch;
+  const int group_sz = kGroupM * p.tiles_n;
+  const int group = t / group_sz;
+  const int first_m = group * kGroupM;
+  const int gm = min(p.tiles_m - first_m, kGroupM);
+  const int r = t - group * group_sz;
+  mt = first_m + r % gm;
+  nt = r / gm;
+}
+
+template <int OUT>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                     const GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (base - raw);
+  const uint32_t smem_a = base;
+  const uint32_t smem_b = base + kStages * kABytes;
+  uint8_t* bar_mem = smem + kStages * kStageBytes;
+  const uint32_t bars = base + kStages * kStageBytes;
+  const uint32_t full_bar = bars;                         // kStages x 8 B
+  const uint32_t empty_bar = bars + 8 * kStages;          // kStages x 8 B
+  const uint32_t acc_full_bar = bars + 16 * kStages;      // kAccStages x 8 B
+  const uint32_t acc_empty_bar = acc_full_bar + 8 * kAccStages;
+  const uint32_t drain_bar = acc_empty_bar + 8 * kAccStages;
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bar_mem + 16 * kStages + 16 * kAccStages + 8);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int num_kb = (p.K + kBK - 1) / kBK;
+  const int num_tiles = p.tiles_m * p.tiles_n * p.batch;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(full_bar + 8 * s, 1); mbar_init(empty_bar + 8 * s, 1); }
+    for (int s = 0; s < kAccStages; ++s) { mbar_init(acc_full_bar + 8 * s, 1); mbar_init(acc_empty_bar + 8 * s, 4); }
+    mbar_init(drain_bar, 1);
+    *abort_flag = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (blockIdx.x == 0 && p.y_scale) *p.y_scale = load_scale(p.a_scale) * load_scale(p.b_scale) * p.kf;
+    if (blockIdx.x == 0 && p.status) {
+      if (!is_pow2_scale(load_scale(p.a_scale)) || !is_pow2_scale(load_scale(p.b_scale)))
+        atomicOr(p.status, static_cast<uint32_t>(SCALIFY_DEV_BAD_SCALE));
+    }
+  }
+  if (warp == 1) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  bool timed_out = false;
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_b)) : "memory");
+      uint32_t stage = 0, phase = 0;
+      long long issued = 0;
+      for (int tile = blockIdx.x; tile < num_tiles && !timed_out; tile += gridDim.x) {
+        int b, mt, nt;
+        tile_coords(p, tile, b, mt, nt);
+        const int m0 = mt * kBM, n0 = nt * kBN;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag)) { timed_out = true; break; }
+          const uint32_t fb = full_bar + 8 * stage;
+          mbar_expect_tx(fb, kStageBytes);
+          const int k0 = kb * kBK;
+          const uint32_t sa = smem_a + stage * kABytes, sb = smem_b + stage * kBBytes;
+          if (p.a_mn_major) tma_load_3d(sa, &map_a, fb, m0, k0, b);
+          else tma_load_3d(sa, &map_a, fb, k0, m0, b);
+          if (p.b_mn_major) {
+            tma_load_3d(sb, &map_b, fb, n0, k0, b);
+            tma_load_3d(sb + kBK * 128, &map_b, fb, n0 + 128, k0, b);
+          } else {
+            tma_load_3d(sb, &map_b, fb, k0, n0, b);
+          }
+          ++issued;
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (timed_out || *abort_flag) {
+        // drain: every copy this thread issued signals its full barrier; wait (bounded) for the
+        // most recent use of each ring slot so that no copy is in flight when the CTA exits
+        const int pending = issued < kStages ? static_cast<int>(issued) : kStages;
+        uint32_t s = stage, ph = phase;
+        for (int i = 0; i < pending; ++i) {
+          if (s == 0) { s = kStages - 1; ph ^= 1u; } else { --s; }
+          const unsigned long long t0 = global_timer_ns();
+          while (!mbar_try_wait(full_bar + 8 * s, ph) && global_timer_ns() - t0 < kWaitLimitNs) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
+      const uint32_t a_lbo = 0u, a_sbo = 1024u;
+      const uint32_t b_lbo = p.b_mn_major ? kBK * 128u : 0u, b_sbo = 1024u;
+      const uint32_t a_step = p.a_mn_major ? (kUmmaK * 128u) : kUmmaK;  // bytes per K=32 step
+      const uint32_t b_step = p.b_mn_major ? (kUmmaK * 128u) : kUmmaK;
+      for (int tile = blockIdx.x; tile < num_tiles && !timed_out; tile += gridDim.x) {
+        if (!mbar_wait(acc_empty_bar + 8 * acc, acc_phase ^ 1u, abort_flag)) { timed_out = true; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * kBN;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(full_bar + 8 * stage, phase, abort_flag)) { timed_out = true; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_a + stage * kABytes, sb = smem_b + stage * kBBytes;
+#pragma unroll
+          for (int k = 0; k < kBK / kUmmaK; ++k) {
+            const uint64_t ad = make_smem_desc(sa + k * a_step, a_lbo, a_sbo);
+            const uint64_t bd = make_smem_desc(sb + k * b_step, b_lbo, b_sbo);
+            umma_f8(d_tmem, ad, bd, p.idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          umma_commit(empty_bar + 8 * stage);  // slot free once these MMAs have read it
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (timed_out) break;
+        umma_commit(acc_full_bar + 8 * acc);  // accumulator complete
+        if (++acc == kAccStages) { acc = 0; acc_phase ^= 1u; }
+      }
+      if (timed_out || *abort_flag) {
+        // all MMAs issued so far must retire before TMEM is freed
+        umma_commit(drain_bar);
+        const unsigned long long t0 = global_timer_ns();
+        while (!mbar_try_wait(drain_bar, 0u) && global_timer_ns() - t0 < kWaitLimitNs) {}
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------- epilogue (warps 2..5)
+    const int q = warp & 3;  // TMEM lane quarter this warp may read
+    uint32_t acc = 0, acc_phase = 0;
+    uint32_t amax_bits = 0u;
+    char* const Yb = static_cast<char*>(p.Y);
+    constexpr int OSZ = ElemBytes<OUT>::v;
+    for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
+      int b, mt, nt;
+      tile_coords(p, tile, b, mt, nt);
+      if (!mbar_wait(acc_full_bar + 8 * acc, acc_phase, abort_flag)) { timed_out = true; break; }
+      tc_fence_after();
+      const int row = mt * kBM + q * 32 + lane;
+      const int n0 = nt * kBN;
+      const bool row_ok = row < p.M;
+      char* yrow = Yb + (static_cast<long long>(b) * p.y_batch_stride + static_cast<long long>(row) * p.ldy) * OSZ;
+      float ssq = 0.f;
+#pragma unroll 1
+      for (int c = 0; c < kBN / 32; ++c) {
+        const int col0 = n0 + c * 32;
+        if (col0 >= p.N) break;  // warp-uniform
+        uint32_t r[32];
+        tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kBN + c * 32, r);
+        tmem_ld_wait();
+        float v[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          v[i] = __uint_as_float(r[i]) * p.alpha;
+          amax_bits = max(amax_bits, abs_bits(v[i]));
+        }
+        if (p.stat == SCALIFY_STAT_L2) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) { const float s = round_through<OUT>(v[i]); ssq = fmaf(s, s, ssq); }
+        }
+        if (row_ok) {
+          if (col0 + 32 <= p.N) {
+            uint32_t o[32 * OSZ / 4];
+            encode_vec<OUT, 32>(v, o);
+#pragma unroll
+            for (int j = 0; j < 32 * OSZ / 16; ++j) st_raw<16>(yrow + static_cast<long long>(col0) * OSZ + j * 16, o + 4 * j);
+          } else {
+            for (int i = 0; i < 32 && col0 + i < p.N; ++i) store_elem<OUT>(yrow, col0 + i, v[i]);
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acc_empty_bar + 8 * acc);
+      if (p.stat == SCALIFY_STAT_L2) {
+        const double s = warp_sum_f64(static_cast<double>(ssq));
+        if (lane == 0) p.l2_partials[static_cast<long long>(tile) * 4 + q] = s;
+      }
+      if (++acc == kAccStages) { acc = 0; acc_phase ^= 1u; }
+    }
+    if (p.stat == SCALIFY_STAT_AMAX) {
+      // rounding is monotonic, so the max of the stored values is the stored value of the max
+      amax_bits = abs_bits(round_through<OUT>(__uint_as_float(amax_bits)));
+      amax_bits = warp_max_u32(amax_bits);
+      if (lane == 0 && amax_bits != 0u) atomicMax(p.stat_word, amax_bits);
+    }
+  }
+
+  if (timed_out && p.status) atomicOr(p.status, static_cast<uint32_t>(SCALIFY_DEV_TIMEOUT));
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// Sums the per-warp partial sums of squares in slot order and leaves sqrt(mean) in the statistic word.
+__global__ void __launch_bounds__(256) gemm_l2_finalize_kernel(const double* __restrict__ partials, int n_slots,
+                                                               double count, float* stat_word) {
+  __shared__ double s[8];
+  double acc = 0.0;
+  for (int i = threadIdx.x; i < n_slots; i += 256) acc += partials[i];
+  acc = warp_sum_f64(acc);
+  if ((threadIdx.x & 31) == 0) s[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double tot = 0.0;
+    for (int i = 0; i < 8; ++i) tot += s[i];
+    *stat_word = static_cast<float>(sqrt(tot / count));
+  }
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// Tensor map over a row-major byte matrix [batch][rows][inner] with row stride ld and batch
+// stride bs (bytes); box = [1][box_rows][128].
+static int make_map(CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t rows, uint64_t batch, uint64_t ld,
+                    uint64_t bs, uint32_t box_rows) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return SCALIFY_ERR_CUDA;
+  cuuint64_t dims[3] = {inner, rows, batch};
+  cuuint64_t strides[2] = {ld, bs ? bs : ld * rows};
+  cuuint32_t box[3] = {128u, box_rows, 1u};
+  cuuint32_t estr[3] = {1u, 1u, 1u};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    set_last_cuda_error(static_cast<int>(r));
+    return SCALIFY_ERR_CUDA;
+  }
+  return SCALIFY_OK;
+}
+
+size_t matmul_ws_bytes(int64_t rows, int64_t cols) {
+  int64_t tiles = ((rows + kBM - 1) / kBM + 8) * ((cols + kBN - 1) / kBN);
+  return kWsHeader + size_t(tiles) * 4 * sizeof(double) + 256;
+}
+
+int launch_scaled_matmul(const MatmulArgs& a, void* ws, cudaStream_t st) {
+  static bool attr_done = false;
+  WsView v = ws_view(ws);
+  CUtensorMap map_a, map_b;
+  // A is logically [M,K]; stored [M,K] (K-major) or, with transA, [K,M] (MN-major).
+  int rc;
+  if (!a.transA) rc = make_map(&map_a, a.A, a.K, a.M, a.batch, a.lda, a.a_bs, kBM);
+  else rc = make_map(&map_a, a.A, a.M, a.K, a.batch, a.lda, a.a_bs, kBK);
+  if (rc) return rc;
+  // B is logically [K,N]; stored [K,N] (MN-major) or, with transB, [N,K] (K-major).
+  if (a.transB) rc = make_map(&map_b, a.B, a.K, a.N, a.batch, a.ldb, a.b_bs, kBN);
+  else rc = make_map(&map_b, a.B, a.N, a.K, a.batch, a.ldb, a.b_bs, kBK);
+  if (rc) return rc;
+
+  GemmParams p;
+  p.M = a.M; p.N = a.N; p.K = a.K; p.batch = a.batch;
+  p.tiles_m = (a.M + kBM - 1) / kBM;
+  p.tiles_n = (a.N + kBN - 1) / kBN;
+  p.a_mn_major = a.transA ? 1 : 0;
+  p.b_mn_major = a.transB ? 0 : 1;
+  // instruction descriptor (kind::f8f6f4): D fp32, A/B formats (0 = E4M3, 1 = E5M2), operand
+  // majorness (0 = K-major), N >> 3, M >> 4
+  p.idesc = (1u << 4) | (uint32_t(a.a_dt == SCALIFY_E5M2) << 7) | (uint32_t(a.b_dt == SCALIFY_E5M2) << 10) |
+            (uint32_t(p.a_mn_major) << 15) | (uint32_t(p.b_mn_major) << 16) | (uint32_t(kBN >> 3) << 17) |
+            (uint32_t(kBM >> 4) << 24);
+  p.kf = kfactor(a.K);
+  p.alpha = 1.0f / p.kf;
+  p.Y = a.Y; p.ldy = a.ldy; p.y_batch_stride = a.y_bs;
+  p.a_scale = a.a_scale; p.b_scale = a.b_scale; p.y_scale = a.y_scale;
+  p.stat = a.stat;
+  p.stat_word = reinterpret_cast<uint32_t*>(v.stat);
+  p.l2_partials = static_cast<double*>(v.area);
+  p.status = v.status;
+  const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n * p.batch;
+  if (tiles > (1ll << 30)) return SCALIFY_ERR_SHAPE;
+  const int grid = static_cast<int>(tiles < sm_count() ? tiles : sm_count());
+  if (a.stat == SCALIFY_STAT_AMAX) SCALIFY_CUDA_TRY(cudaMemsetAsync(v.stat, 0, sizeof(float), st));
+  if (!attr_done) {
+    SCALIFY_CUDA_TRY(cudaFuncSetAttribute(scaled_matmul_kernel<SCALIFY_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kGemmSmem)));
+    SCALIFY_CUDA_TRY(cudaFuncSetAttribute(scaled_matmul_kernel<SCALIFY_F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kGemmSmem)));
+    SCALIFY_CUDA_TRY(cudaFuncSetAttribute(scaled_matmul_kernel<SCALIFY_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kGemmSmem)));
+    attr_done = true;
+  }
+  SCALIFY_DISPATCH_WIDE(a.y_dt, OUT,
+      scaled_matmul_kernel<OUT><<<grid, kGemmThreads, kGemmSmem, st>>>(map_a, map_b, p));
+  SCALIFY_CUDA_TRY(cudaGetLastError());
+  if (a.stat == SCALIFY_STAT_L2) {
+    gemm_l2_finalize_kernel<<<1, 256, 0, st>>>(p.l2_partials, static_cast<int>(tiles * 4),
+                                               double(a.M) * double(a.N) * double(a.batch), v.stat);
+    SCALIFY_CUDA_TRY(cudaGetLastError());
+  }
+  return SCALIFY_OK;
+}
+
+}  // namespace scalify

@@ -1,0 +1,444 @@
+// C ABI entry points: argument validation and dispatch to the kernel launchers.
+// Every check happens on the host before anything is enqueued.
+#include <math.h>
+#include <string.h>
+
+#include "scalify_common.cuh"
+#include "scalify_launch.h"
+#include <new>
+
+namespace scalify {
+
+static thread_local int g_last_cuda_error = 0;
+void set_last_cuda_error(int e) { g_last_cuda_error = e; }
+int cuda_fail(cudaError_t e) {
+  g_last_cuda_error = static_cast<int>(e);
+  return SCALIFY_ERR_CUDA;
+}
+
+int sm_count() {
+  static int cached[64] = {0};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+
+int check_array(const scalify_array* a) {
+  if (!a || !a->data) return SCALIFY_ERR_NULL;
+  if (!valid_dtype(a->dtype)) return SCALIFY_ERR_DTYPE;
+  if (a->ndim < 1 || a->ndim > 3) return SCALIFY_ERR_SHAPE;
+  for (int i = 0; i < a->ndim; ++i)
+    if (a->shape[i] < 0 || a->shape[i] > (int64_t(1) << 40)) return SCALIFY_ERR_SHAPE;
+  if (a->stride[a->ndim - 1] != 1) return SCALIFY_ERR_ALIGNMENT;
+  if (reinterpret_cast<uintptr_t>(a->data) % 16 != 0) return SCALIFY_ERR_ALIGNMENT;
+  const int es = elem_size(a->dtype);
+  for (int i = 0; i < a->ndim - 1; ++i) {
+    if (a->stride[i] < 0) return SCALIFY_ERR_ALIGNMENT;
+    if (a->shape[i] > 1 && (a->stride[i] * es) % 16 != 0) return SCALIFY_ERR_ALIGNMENT;
+  }
+  return SCALIFY_OK;
+}
+
+int64_t contiguous_numel(const scalify_array* a) {
+  int64_t n = 1;
+  for (int i = a->ndim - 1; i >= 0; --i) {
+    if (a->shape[i] != 1 && a->stride[i] != n) return -1;
+    n *= a->shape[i];
+  }
+  return n;
+}
+
+static bool same_shape(const scalify_array* a, const scalify_array* b) {
+  if (a->ndim != b->ndim) return false;
+  for (int i = 0; i < a->ndim; ++i)
+    if (a->shape[i] != b->shape[i]) return false;
+  return true;
+}
+
+static bool valid_stat(int s) { return s == SCALIFY_STAT_NONE || s == SCALIFY_STAT_AMAX || s == SCALIFY_STAT_L2; }
+
+// rows x cols view of a 2-D array (or 1-D as one row); row stride in elements
+static int as_rows(const scalify_array* a, int64_t* rows, int64_t* cols, int64_t* ld) {
+  if (a->ndim == 1) { *rows = 1; *cols = a->shape[0]; *ld = a->shape[0]; return SCALIFY_OK; }
+  if (a->ndim == 2) { *rows = a->shape[0]; *cols = a->shape[1]; *ld = a->stride[0]; return SCALIFY_OK; }
+  if (a->ndim == 3 && a->stride[0] == a->shape[1] * a->stride[1]) {
+    *rows = a->shape[0] * a->shape[1]; *cols = a->shape[2]; *ld = a->stride[1];
+    return SCALIFY_OK;
+  }
+  return SCALIFY_ERR_SHAPE;
+}
+
+}  // namespace scalify
+
+using namespace scalify;
+
+extern "C" {
+
+int scalify_version(void) { return 100; }
+
+int scalify_last_cuda_error(void) { return g_last_cuda_error; }
+
+const char* scalify_status_string(int code) {
+  switch (code) {
+    case SCALIFY_OK: return "ok";
+    case SCALIFY_ERR_NULL: return "a required pointer is NULL";
+    case SCALIFY_ERR_DTYPE: return "dtype not valid for this argument";
+    case SCALIFY_ERR_SHAPE: return "shapes inconsistent or out of range";
+    case SCALIFY_ERR_ALIGNMENT: return "pointer or stride not 16-byte aligned, or innermost stride not 1";
+    case SCALIFY_ERR_WORKSPACE: return "workspace missing or too small";
+    case SCALIFY_ERR_UNSUPPORTED: return "combination not supported";
+    case SCALIFY_ERR_CUDA: return "CUDA call failed (see scalify_last_cuda_error)";
+    case SCALIFY_ERR_ALIAS: return "forbidden aliasing of scale words or buffers";
+    case SCALIFY_ERR_VALUE: return "scalar argument out of range";
+    default: return code > 0 ? "device status bits set" : "unknown error";
+  }
+}
+
+size_t scalify_workspace_bytes(int op, int64_t d0, int64_t d1) {
+  size_t n = kWsMin;
+  const size_t stat_bytes = kWsHeader + size_t(sm_count()) * 8 * sizeof(double) + 256;
+  switch (op) {
+    case SCALIFY_OP_MATMUL: n = matmul_ws_bytes(d0, d1); break;
+    case SCALIFY_OP_RESCALE:
+    case SCALIFY_OP_STATISTIC: n = stat_bytes; break;
+    case SCALIFY_OP_LAYERNORM_BWD: n = layernorm_bwd_ws_bytes(d0, d1); break;
+    case SCALIFY_OP_ADAM: n = adam_ws_bytes(d0); break;
+    default: break;
+  }
+  if (n < stat_bytes) n = stat_bytes;
+  return n < kWsMin ? kWsMin : n;
+}
+
+int scalify_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
+  if (!workspace) return SCALIFY_ERR_NULL;
+  if (workspace_bytes < kWsMin || reinterpret_cast<uintptr_t>(workspace) % 256 != 0) return SCALIFY_ERR_WORKSPACE;
+  SCALIFY_CUDA_TRY(cudaMemsetAsync(workspace, 0, kWsHeader, static_cast<cudaStream_t>(stream)));
+  return SCALIFY_OK;
+}
+
+int scalify_check_status(void* workspace, void* stream) {
+  if (!workspace) return SCALIFY_ERR_NULL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint32_t bits = 0;
+  SCALIFY_CUDA_TRY(cudaMemcpyAsync(&bits, workspace, sizeof(bits), cudaMemcpyDeviceToHost, st));
+  SCALIFY_CUDA_TRY(cudaStreamSynchronize(st));
+  if (bits) {
+    SCALIFY_CUDA_TRY(cudaMemsetAsync(workspace, 0, sizeof(bits), st));
+    SCALIFY_CUDA_TRY(cudaStreamSynchronize(st));
+  }
+  return static_cast<int>(bits & 0x7FFFFFFFu);
+}
+
+static int check_ws(void* ws, size_t bytes, size_t need) {
+  if (!ws) return SCALIFY_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(ws) % 256 != 0) return SCALIFY_ERR_WORKSPACE;
+  if (bytes < need) return SCALIFY_ERR_WORKSPACE;
+  return SCALIFY_OK;
+}
+
+int scalify_statistic(const scalify_array* X, int stat, float* out_stat, void* workspace, size_t workspace_bytes,
+                      void* stream) {
+  int rc = check_array(X);
+  if (rc) return rc;
+  if (stat != SCALIFY_STAT_AMAX && stat != SCALIFY_STAT_L2) return SCALIFY_ERR_VALUE;
+  const int64_t n = contiguous_numel(X);
+  if (n < 0) return SCALIFY_ERR_SHAPE;
+  rc = check_ws(workspace, workspace_bytes, scalify_workspace_bytes(SCALIFY_OP_STATISTIC, n, 0));
+  if (rc) return rc;
+  return launch_statistic(X->data, X->dtype, n, stat, workspace, out_stat, static_cast<cudaStream_t>(stream));
+}
+
+int scalify_rescale(const scalify_array* X, int stat, const float* new_scale, const float* stat_in, scalify_array* Y,
+                    void* workspace, size_t workspace_bytes, void* stream) {
+  int rc = check_array(X);
+  if (rc) return rc;
+  rc = check_array(Y);
+  if (rc) return rc;
+  if (!valid_stat(stat)) return SCALIFY_ERR_VALUE;
+  if (stat != SCALIFY_STAT_NONE && new_scale) return SCALIFY_ERR_VALUE;
+  if (stat == SCALIFY_STAT_NONE && stat_in) return SCALIFY_ERR_VALUE;
+  const int64_t n = contiguous_numel(X);
+  if (n < 0 || contiguous_numel(Y) != n) return SCALIFY_ERR_SHAPE;
+  if (Y->data == X->data && elem_size(X->dtype) != elem_size(Y->dtype)) return SCALIFY_ERR_ALIAS;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint32_t* status = workspace ? ws_view(workspace).status : nullptr;
+  if (workspace && check_ws(workspace, workspace_bytes, kWsMin)) return SCALIFY_ERR_WORKSPACE;
+  if (stat == SCALIFY_STAT_NONE) {
+    if (new_scale) {
+      if (Y->scale && Y->scale == X->scale) return SCALIFY_ERR_ALIAS;
+      return launch_rebalance(X->data, X->dtype, Y->data, Y->dtype, n, X->scale, Y->scale, nullptr, new_scale,
+                              kModeSet, status, st);
+    }
+    return launch_rebalance(X->data, X->dtype, Y->data, Y->dtype, n, X->scale, Y->scale, nullptr, nullptr, kModeCast,
+                            status, st);
+  }
+  if (stat_in) {
+    return launch_rebalance(X->data, X->dtype, Y->data, Y->dtype, n, X->scale, Y->scale, stat_in, nullptr,
+                            kModeDynamic, status, st);
+  }
+  rc = check_ws(workspace, workspace_bytes, scalify_workspace_bytes(SCALIFY_OP_RESCALE, n, 0));
+  if (rc) return rc;
+  rc = launch_statistic(X->data, X->dtype, n, stat, workspace, nullptr, st);
+  if (rc) return rc;
+  return launch_rebalance(X->data, X->dtype, Y->data, Y->dtype, n, X->scale, Y->scale, ws_view(workspace).stat,
+                          nullptr, kModeDynamic, status, st);
+}
+
+int scalify_scaled_add(const scalify_array* A, const scalify_array* B, int subtract, scalify_array* Y, void* stream) {
+  int rc = check_array(A);
+  if (rc) return rc;
+  rc = check_array(B);
+  if (rc) return rc;
+  rc = check_array(Y);
+  if (rc) return rc;
+  if (!is_wide(A->dtype) || B->dtype != A->dtype) return SCALIFY_ERR_DTYPE;
+  const int64_t n = contiguous_numel(A);
+  if (n < 0 || !same_shape(A, Y) || contiguous_numel(Y) != n) return SCALIFY_ERR_SHAPE;
+  int broadcast = 0;
+  const int64_t row_len = A->shape[A->ndim - 1];
+  if (!same_shape(A, B)) {
+    if (B->ndim == 1 && B->shape[0] == row_len) broadcast = 1;
+    else return SCALIFY_ERR_SHAPE;
+  } else if (contiguous_numel(B) != n) {
+    return SCALIFY_ERR_SHAPE;
+  }
+  if (Y->scale && (Y->scale == A->scale || Y->scale == B->scale)) return SCALIFY_ERR_ALIAS;
+  if (Y->data == A->data && elem_size(A->dtype) != elem_size(Y->dtype)) return SCALIFY_ERR_ALIAS;
+  if (Y->data == B->data) return SCALIFY_ERR_ALIAS;
+  return launch_add(A->data, B->data, A->dtype, Y->data, Y->dtype, n, row_len, broadcast, A->scale, B->scale, Y->scale,
+                    subtract, static_cast<cudaStream_t>(stream));
+}
+
+int scalify_scaled_gelu(const scalify_array* X, int exact_erf, scalify_array* Y, void* stream) {
+  int rc = check_array(X);
+  if (rc) return rc;
+  rc = check_array(Y);
+  if (rc) return rc;
+  if (!is_wide(X->dtype)) return SCALIFY_ERR_DTYPE;
+  const int64_t n = contiguous_numel(X);
+  if (n < 0 || contiguous_numel(Y) != n) return SCALIFY_ERR_SHAPE;
+  if (Y->scale && Y->scale == X->scale) return SCALIFY_ERR_ALIAS;
+  return launch_gelu(X->data, nullptr, X->dtype, Y->data, Y->dtype, n, X->scale, nullptr, Y->scale, exact_erf ? 1 : 0, 0,
+                     static_cast<cudaStream_t>(stream));
+}
+
+int scalify_scaled_gelu_bwd(const scalify_array* G, const scalify_array* X, int exact_erf, scalify_array* dX,
+                            void* stream) {
+  int rc = check_array(G);
+  if (rc) return rc;
+  rc = check_array(X);
+  if (rc) return rc;
+  rc = check_array(dX);
+  if (rc) return rc;
+  if (!is_wide(X->dtype) || G->dtype != X->dtype) return SCALIFY_ERR_DTYPE;
+  const int64_t n = contiguous_numel(X);
+  if (n < 0 || contiguous_numel(G) != n || contiguous_numel(dX) != n) return SCALIFY_ERR_SHAPE;
+  if (dX->scale && (dX->scale == X->scale || dX->scale == G->scale)) return SCALIFY_ERR_ALIAS;
+  return launch_gelu(X->data, G->data, X->dtype, dX->data, dX->dtype, n, X->scale, G->scale, dX->scale,
+                     exact_erf ? 1 : 0, 1, static_cast<cudaStream_t>(stream));
+}
+
+int scalify_scaled_layernorm(const scalify_array* X, const scalify_array* gamma, const scalify_array* beta, float eps,
+                             int eps_inside_sqrt, scalify_array* Y, float* mean, float* rinv, void* stream) {
+  int rc = check_array(X);
+  if (rc) return rc;
+  rc = check_array(Y);
+  if (rc) return rc;
+  if (!is_wide(X->dtype)) return SCALIFY_ERR_DTYPE;
+  int64_t R, d, x_ld, Ry, dy, y_ld;
+  if (as_rows(X, &R, &d, &x_ld) || as_rows(Y, &Ry, &dy, &y_ld) || R != Ry || d != dy) return SCALIFY_ERR_SHAPE;
+  if (d < 1 || R > 0x7FFFFFFF || (d * elem_size(X->dtype)) % 16 != 0) return SCALIFY_ERR_SHAPE;
+  if (!(eps >= 0.f)) return SCALIFY_ERR_VALUE;
+  int gb_dt = SCALIFY_F32;
+  if (gamma) {
+    rc = check_array(gamma);
+    if (rc) return rc;
+    if (!is_wide(gamma->dtype) || gamma->ndim != 1 || gamma->shape[0] != d) return SCALIFY_ERR_SHAPE;
+    gb_dt = gamma->dtype;
+    if (beta) {
+      rc = check_array(beta);
+      if (rc) return rc;
+      if (beta->dtype != gb_dt || beta->ndim != 1 || beta->shape[0] != d) return SCALIFY_ERR_SHAPE;
+    }
+  } else if (beta) {
+    return SCALIFY_ERR_NULL;
+  }
+  if (R == 0) return SCALIFY_OK;
+  return launch_layernorm_fwd(X->data, X->dtype, x_ld, Y->data, Y->dtype, y_ld, static_cast<int>(R), static_cast<int>(d),
+                              gamma ? gamma->data : nullptr, beta ? beta->data : nullptr, gb_dt,
+                              gamma ? gamma->scale : nullptr, beta ? beta->scale : nullptr, Y->scale, eps,
+                              eps_inside_sqrt ? 1 : 0, mean, rinv, static_cast<cudaStream_t>(stream));
+}
+
+int scalify_scaled_layernorm_bwd(const scalify_array* G, const scalify_array* X, const scalify_array* gamma,
+                                 const float* mean, const float* rinv, float eps, int eps_inside_sqrt, int stat_dx,
+                                 scalify_array* dX, scalify_array* dXq, scalify_array* dgamma, scalify_array* dbeta,
+                                 void* workspace, size_t workspace_bytes, void* stream) {
+  int rc = check_array(G);
+  if (rc) return rc;
+  rc = check_array(X);
+  if (rc) return rc;
+  rc = check_array(dX);
+  if (rc) return rc;
+  if (!mean || !rinv) return SCALIFY_ERR_NULL;
+  if (!is_wide(X->dtype) || G->dtype != X->dtype || !is_wide(dX->dtype)) return SCALIFY_ERR_DTYPE;
+  if (!valid_stat(stat_dx)) return SCALIFY_ERR_VALUE;
+  int64_t R, d, x_ld, Rg, dg, g_ld, Rd, dd, dx_ld;
+  if (as_rows(X, &R, &d, &x_ld) || as_rows(G, &Rg, &dg, &g_ld) || as_rows(dX, &Rd, &dd, &dx_ld)) return SCALIFY_ERR_SHAPE;
+  if (R != Rg || d != dg || R != Rd || d != dd) return SCALIFY_ERR_SHAPE;
+  if (d < 1 || R < 1 || R > 0x7FFFFFFF || (d * elem_size(X->dtype)) % 16 != 0) return SCALIFY_ERR_SHAPE;
+  int gb_dt = SCALIFY_F32;
+  if (gamma) {
+    rc = check_array(gamma);
+    if (rc) return rc;
+    if (!is_wide(gamma->dtype) || gamma->ndim != 1 || gamma->shape[0] != d) return SCALIFY_ERR_SHAPE;
+    gb_dt = gamma->dtype;
+  }
+  int dg_dt = SCALIFY_F32;
+  if ((dgamma != nullptr) != (dbeta != nullptr)) return SCALIFY_ERR_NULL;
+  if (dgamma) {
+    rc = check_array(dgamma);
+    if (rc) return rc;
+    rc = check_array(dbeta);
+    if (rc) return rc;
+    if (!is_wide(dgamma->dtype) || dbeta->dtype != dgamma->dtype) return SCALIFY_ERR_DTYPE;
+    if (dgamma->ndim != 1 || dgamma->shape[0] != d || dbeta->ndim != 1 || dbeta->shape[0] != d) return SCALIFY_ERR_SHAPE;
+    dg_dt = dgamma->dtype;
+  }
+  if (dXq) {
+    rc = check_array(dXq);
+    if (rc) return rc;
+    if (stat_dx == SCALIFY_STAT_NONE) return SCALIFY_ERR_VALUE;
+    if (contiguous_numel(dX) != R * d || contiguous_numel(dXq) != R * d) return SCALIFY_ERR_SHAPE;
+    if (dXq->data == dX->data && elem_size(dXq->dtype) != elem_size(dX->dtype)) return SCALIFY_ERR_ALIAS;
+  }
+  if (dX->scale && (dX->scale == G->scale || dX->scale == X->scale || (gamma && dX->scale == gamma->scale)))
+    return SCALIFY_ERR_ALIAS;
+  rc = check_ws(workspace, workspace_bytes, scalify_workspace_bytes(SCALIFY_OP_LAYERNORM_BWD, R, d));
+  if (rc) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // the un-rebalanced gradient needs a scale word for the rebalance pass; use a workspace slot if the caller has none
+  float* dx_scale = dX->scale ? dX->scale : reinterpret_cast<float*>(static_cast<char*>(workspace) + 48);
+  rc = launch_layernorm_bwd(G->data, g_ld, X->data, X->dtype, x_ld, dX->data, dX->dtype, dx_ld, static_cast<int>(R),
+                            static_cast<int>(d), gamma ? gamma->data : nullptr, gb_dt, mean, rinv, eps,
+                            eps_inside_sqrt ? 1 : 0, stat_dx, dgamma ? dgamma->data : nullptr,
+                            dbeta ? dbeta->data : nullptr, dg_dt, G->scale, X->scale, gamma ? gamma->scale : nullptr,
+                            dx_scale, dgamma ? dgamma->scale : nullptr, dbeta ? dbeta->scale : nullptr, workspace, st);
+  if (rc) return rc;
+  if (dXq) {
+    WsView v = ws_view(workspace);
+    rc = launch_rebalance(dX->data, dX->dtype, dXq->data, dXq->dtype, R * d, dx_scale, dXq->scale, v.stat, nullptr,
+                          kModeDynamic, v.status, st);
+  }
+  return rc;
+}
+
+int scalify_scaled_adam_step(int n_tensors, const scalify_array* grads, scalify_array* m, scalify_array* v,
+                             scalify_array* w, float lr, float beta1, float beta2, float eps, int64_t step,
+                             void* workspace, size_t workspace_bytes, void* stream) {
+  if (n_tensors < 0) return SCALIFY_ERR_VALUE;
+  if (n_tensors == 0) return SCALIFY_OK;
+  if (!grads || !m || !v || !w) return SCALIFY_ERR_NULL;
+  if (step < 1 || !(beta1 >= 0.f && beta1 < 1.f) || !(beta2 >= 0.f && beta2 < 1.f) || !(eps >= 0.f) || !isfinite(lr))
+    return SCALIFY_ERR_VALUE;
+  int rc = check_ws(workspace, workspace_bytes, scalify_workspace_bytes(SCALIFY_OP_ADAM, n_tensors, 0));
+  if (rc) return rc;
+  int64_t stack_numel[64];
+  int64_t* numel = stack_numel;
+  int64_t* heap = nullptr;
+  if (n_tensors > 64) {
+    heap = new (std::nothrow) int64_t[n_tensors];
+    if (!heap) return SCALIFY_ERR_VALUE;
+    numel = heap;
+  }
+  rc = SCALIFY_OK;
+  for (int i = 0; i < n_tensors && rc == SCALIFY_OK; ++i) {
+    if ((rc = check_array(&grads[i])) || (rc = check_array(&m[i])) || (rc = check_array(&v[i])) ||
+        (rc = check_array(&w[i])))
+      break;
+    if (!m[i].scale || !v[i].scale || !w[i].scale) { rc = SCALIFY_ERR_NULL; break; }
+    if (grads[i].dtype != grads[0].dtype || m[i].dtype != m[0].dtype || v[i].dtype != m[0].dtype ||
+        w[i].dtype != w[0].dtype) { rc = SCALIFY_ERR_DTYPE; break; }
+    if (!(m[i].dtype == SCALIFY_F16 || m[i].dtype == SCALIFY_F32) || !is_wide(w[i].dtype)) { rc = SCALIFY_ERR_DTYPE; break; }
+    const int64_t n = contiguous_numel(&grads[i]);
+    if (n < 0 || contiguous_numel(&m[i]) != n || contiguous_numel(&v[i]) != n || contiguous_numel(&w[i]) != n) {
+      rc = SCALIFY_ERR_SHAPE;
+      break;
+    }
+    if (m[i].scale == v[i].scale || m[i].scale == w[i].scale || v[i].scale == w[i].scale ||
+        grads[i].scale == m[i].scale || grads[i].scale == v[i].scale || grads[i].scale == w[i].scale) {
+      rc = SCALIFY_ERR_ALIAS;
+      break;
+    }
+    numel[i] = n;
+  }
+  if (rc == SCALIFY_OK)
+    rc = launch_adam(n_tensors, grads, m, v, w, numel, lr, beta1, beta2, eps, step, workspace,
+                     static_cast<cudaStream_t>(stream));
+  delete[] heap;
+  return rc;
+}
+
+int scalify_scaled_matmul(const scalify_array* A, int transA, const scalify_array* B, int transB, scalify_array* Y,
+                          int stat, scalify_array* Yq, void* workspace, size_t workspace_bytes, void* stream) {
+  int rc = check_array(A);
+  if (rc) return rc;
+  rc = check_array(B);
+  if (rc) return rc;
+  rc = check_array(Y);
+  if (rc) return rc;
+  if (!is_fp8(A->dtype) || !is_fp8(B->dtype) || !is_wide(Y->dtype)) return SCALIFY_ERR_DTYPE;
+  if (!valid_stat(stat)) return SCALIFY_ERR_VALUE;
+  if (A->ndim < 2 || B->ndim < 2 || Y->ndim != A->ndim || B->ndim > A->ndim) return SCALIFY_ERR_SHAPE;
+  const int an = A->ndim, bn = B->ndim, yn = Y->ndim;
+  const int64_t batch = an == 3 ? A->shape[0] : 1;
+  const int64_t M = transA ? A->shape[an - 1] : A->shape[an - 2];
+  const int64_t K = transA ? A->shape[an - 2] : A->shape[an - 1];
+  const int64_t Kb = transB ? B->shape[bn - 1] : B->shape[bn - 2];
+  const int64_t N = transB ? B->shape[bn - 2] : B->shape[bn - 1];
+  if (K != Kb || K < 1 || M < 1 || N < 1 || batch < 1) return SCALIFY_ERR_SHAPE;
+  if (Y->shape[yn - 2] != M || Y->shape[yn - 1] != N) return SCALIFY_ERR_SHAPE;
+  if (an == 3 && (Y->shape[0] != batch || (bn == 3 && B->shape[0] != batch))) return SCALIFY_ERR_SHAPE;
+  if (M > 0x7FFFFFFF || N > 0x7FFFFFFF || K > 0x7FFFFFFF || batch > 0x7FFFFFFF) return SCALIFY_ERR_SHAPE;
+  if (Y->scale && (Y->scale == A->scale || Y->scale == B->scale)) return SCALIFY_ERR_ALIAS;
+  rc = check_ws(workspace, workspace_bytes, scalify_workspace_bytes(SCALIFY_OP_MATMUL, batch * M, N));
+  if (rc) return rc;
+  if (Yq) {
+    rc = check_array(Yq);
+    if (rc) return rc;
+    if (stat == SCALIFY_STAT_NONE) return SCALIFY_ERR_VALUE;
+    if (!same_shape(Y, Yq) || contiguous_numel(Y) != batch * M * N || contiguous_numel(Yq) != batch * M * N)
+      return SCALIFY_ERR_SHAPE;
+    if (Yq->data == Y->data && elem_size(Yq->dtype) != elem_size(Y->dtype)) return SCALIFY_ERR_ALIAS;
+    if (Yq->scale && (Yq->scale == A->scale || Yq->scale == B->scale)) return SCALIFY_ERR_ALIAS;
+  }
+  MatmulArgs a;
+  a.A = A->data; a.a_dt = A->dtype; a.transA = transA ? 1 : 0; a.lda = A->stride[an - 2];
+  a.a_bs = an == 3 ? A->stride[0] : 0;
+  a.B = B->data; a.b_dt = B->dtype; a.transB = transB ? 1 : 0; a.ldb = B->stride[bn - 2];
+  a.b_bs = bn == 3 ? B->stride[0] : 0;
+  a.Y = Y->data; a.y_dt = Y->dtype; a.ldy = Y->stride[yn - 2]; a.y_bs = yn == 3 ? Y->stride[0] : 0;
+  a.M = static_cast<int>(M); a.N = static_cast<int>(N); a.K = static_cast<int>(K); a.batch = static_cast<int>(batch);
+  a.a_scale = A->scale; a.b_scale = B->scale;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // the intermediate needs a scale word for the rebalance pass; use a workspace slot if the caller has none
+  float* y_scale = Y->scale ? Y->scale : reinterpret_cast<float*>(static_cast<char*>(workspace) + 48);
+  a.y_scale = y_scale;
+  a.stat = stat;
+  if (a.lda < (transA ? M : K) || a.ldb < (transB ? K : N) || a.ldy < N) return SCALIFY_ERR_SHAPE;
+  rc = launch_scaled_matmul(a, workspace, st);
+  if (rc) return rc;
+  if (Yq) {
+    WsView v = ws_view(workspace);
+    rc = launch_rebalance(Y->data, Y->dtype, Yq->data, Yq->dtype, batch * M * N, y_scale, Yq->scale, v.stat, nullptr,
+                          kModeDynamic, v.status, st);
+  }
+  return rc;
+}
+
+}  // extern "C"

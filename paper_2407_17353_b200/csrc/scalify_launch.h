@@ -1,0 +1,47 @@
+// Host-side launcher interfaces between the C ABI layer and the kernel translation units.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "scalify.h"
+
+namespace scalify {
+
+enum { kModeCast = 0, kModeDynamic = 1, kModeSet = 2 };
+
+int launch_statistic(const void* x, int dtype, int64_t n, int stat, void* ws, float* out_stat, cudaStream_t st);
+int launch_rebalance(const void* x, int in_dt, void* y, int out_dt, int64_t n, const float* x_scale, float* y_scale,
+                     const float* stat, const float* new_scale, int mode, uint32_t* status, cudaStream_t st);
+int launch_add(const void* a, const void* b, int ab_dt, void* y, int out_dt, int64_t n, int64_t row_len, int broadcast,
+               const float* a_scale, const float* b_scale, float* y_scale, int subtract, cudaStream_t st);
+int launch_gelu(const void* x, const void* g, int in_dt, void* y, int out_dt, int64_t n, const float* x_scale,
+                const float* g_scale, float* y_scale, int exact, int bwd, cudaStream_t st);
+int launch_layernorm_fwd(const void* X, int x_dt, int64_t x_ld, void* Y, int y_dt, int64_t y_ld, int R, int d,
+                         const void* gamma, const void* beta, int gb_dt, const float* gamma_scale,
+                         const float* beta_scale, float* y_scale, float eps, int eps_inside, float* mean,
+                         float* rinv, cudaStream_t st);
+size_t layernorm_bwd_ws_bytes(int64_t R, int64_t d);
+int launch_layernorm_bwd(const void* G, int64_t g_ld, const void* X, int x_dt, int64_t x_ld, void* dX, int dx_dt,
+                         int64_t dx_ld, int R, int d, const void* gamma, int gb_dt, const float* mean,
+                         const float* rinv, float eps, int eps_inside, int stat, void* dgamma, void* dbeta, int dg_dt,
+                         const float* g_scale, const float* x_scale, const float* gamma_scale, float* dx_scale,
+                         float* dgamma_scale, float* dbeta_scale, void* ws, cudaStream_t st);
+size_t adam_ws_bytes(int64_t n_tensors);
+int launch_adam(int n_tensors, const scalify_array* grads, scalify_array* m, scalify_array* v, scalify_array* w,
+                const int64_t* numel, float lr, float beta1, float beta2, float eps, int64_t step, void* ws,
+                cudaStream_t st);
+
+struct MatmulArgs {
+  const void* A; int a_dt; int transA; int64_t lda, a_bs;
+  const void* B; int b_dt; int transB; int64_t ldb, b_bs;
+  void* Y; int y_dt; int64_t ldy, y_bs;
+  int M, N, K, batch;
+  const float* a_scale; const float* b_scale; float* y_scale;
+  int stat;
+};
+size_t matmul_ws_bytes(int64_t rows, int64_t cols);
+int launch_scaled_matmul(const MatmulArgs& a, void* ws, cudaStream_t st);
+
+}  // namespace scalify

@@ -1,0 +1,49 @@
+"""Shared helpers of the GPU parity tests: bit-pattern transport between numpy
+(oracle side) and torch CUDA tensors (library side), and ulp distances."""
+import numpy as np
+import torch
+
+import oracle as orc
+
+TORCH_DT = {orc.E4M3: torch.float8_e4m3fn, orc.E5M2: torch.float8_e5m2, orc.F16: torch.float16,
+            orc.BF16: torch.bfloat16, orc.F32: torch.float32}
+NP_BITS = {orc.E4M3: np.uint8, orc.E5M2: np.uint8, orc.F16: np.uint16, orc.BF16: np.uint16, orc.F32: np.uint32}
+_SIGNED = {1: np.int8, 2: np.int16, 4: np.int32}
+_TSIGNED = {1: torch.int8, 2: torch.int16, 4: torch.int32}
+NBITS = {orc.E4M3: 8, orc.E5M2: 8, orc.F16: 16, orc.BF16: 16, orc.F32: 32}
+
+
+def to_dev(bits: np.ndarray, dtype: int, device="cuda") -> torch.Tensor:
+    """numpy bit patterns -> CUDA tensor of the matching torch dtype (no value conversion)."""
+    b = np.ascontiguousarray(bits)
+    t = torch.from_numpy(b.view(_SIGNED[b.dtype.itemsize])).to(device)
+    return t.view(TORCH_DT[dtype])
+
+
+def to_bits(t: torch.Tensor, dtype: int) -> np.ndarray:
+    """CUDA tensor -> numpy bit patterns."""
+    c = t.detach().contiguous().view(_TSIGNED[t.element_size()]).cpu().numpy()
+    return c.view(NP_BITS[dtype])
+
+
+def ordered(bits: np.ndarray, dtype: int) -> np.ndarray:
+    """Monotone integer image of sign-magnitude bit patterns (+0 and -0 both map to 0)."""
+    n = NBITS[dtype]
+    b = bits.astype(np.int64)
+    mag = b & ((1 << (n - 1)) - 1)
+    return np.where((b >> (n - 1)) & 1, -mag, mag)
+
+
+def ulp_diff(a: np.ndarray, b: np.ndarray, dtype: int) -> np.ndarray:
+    """Distance in representable values; NaN vs NaN counts as 0, NaN vs number as a huge distance."""
+    va, vb = orc.decode(a, dtype), orc.decode(b, dtype)
+    d = np.abs(ordered(a, dtype) - ordered(b, dtype))
+    both_nan = np.isnan(va) & np.isnan(vb)
+    one_nan = np.isnan(va) ^ np.isnan(vb)
+    d = np.where(both_nan, 0, d)
+    d = np.where(one_nan, 1 << 40, d)
+    return d
+
+
+def scale_of(t) -> float:
+    return float(t.scale.item())

@@ -1,0 +1,94 @@
+"""CPU-side checks of the C ABI: the shared library builds, loads and exports
+every function the public header declares; argument validation rejects bad
+calls on the host before anything is enqueued (no GPU needed: a call that
+fails validation launches nothing)."""
+import ctypes
+import os
+import re
+
+import paper_2407_17353_b200 as sc
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "scalify.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(scalify_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_function():
+    L = sc.lib()
+    names = declared_functions()
+    assert len(names) >= 14
+    for n in names:
+        assert hasattr(L, n), n
+    assert L.scalify_version() >= 100
+
+
+def test_status_strings_and_workspace_sizes():
+    L = sc.lib()
+    assert L.scalify_status_string(0) == b"ok"
+    for code in range(-9, 0):
+        assert len(L.scalify_status_string(code)) > 3
+    for op in range(5):
+        assert sc.scalify_workspace_bytes(op, 8192, 8192) >= 4096
+    assert sc.scalify_workspace_bytes(sc.OP_ADAM, 1000) >= 1000 * 32
+
+
+def _arr(ptr, dtype, shape, stride=None, scale=None):
+    a = sc.scalify_array()
+    a.data = ptr
+    a.dtype = dtype
+    a.ndim = len(shape)
+    st = stride
+    if st is None:
+        st, n = [], 1
+        for s in reversed(shape):
+            st.insert(0, n)
+            n *= s
+    for i, (s, t) in enumerate(zip(shape, st)):
+        a.shape[i] = s
+        a.stride[i] = t
+    a.scale = scale
+    return a
+
+
+def test_validation_rejects_bad_arguments_on_the_host():
+    L = sc.lib()
+    R = ctypes.byref
+    good = _arr(4096, sc.BF16, (4, 64))
+    out = _arr(8192, sc.BF16, (4, 64))
+    assert L.scalify_scaled_add(None, R(good), 0, R(out), None) == -1                      # NULL
+    assert L.scalify_scaled_add(R(_arr(0, sc.BF16, (4, 64))), R(good), 0, R(out), None) == -1
+    assert L.scalify_scaled_add(R(_arr(4096, 9, (4, 64))), R(good), 0, R(out), None) == -2  # dtype
+    assert L.scalify_scaled_add(R(_arr(4096, sc.E4M3, (4, 64))), R(_arr(4096, sc.E4M3, (4, 64))), 0, R(out), None) == -2
+    assert L.scalify_scaled_add(R(good), R(_arr(4096, sc.BF16, (4, 32))), 0, R(out), None) == -3  # shape
+    assert L.scalify_scaled_add(R(_arr(4098, sc.BF16, (4, 64))), R(good), 0, R(out), None) == -4  # alignment
+    assert L.scalify_scaled_add(R(_arr(4096, sc.BF16, (4, 64), (64, 2))), R(good), 0, R(out), None) == -4
+    assert L.scalify_scaled_add(R(_arr(4096, sc.BF16, (4, 64), scale=512)), R(good), 0,
+                                R(_arr(8192, sc.BF16, (4, 64), scale=512)), None) == -8           # alias
+    # matmul: dtype, shape and workspace checks
+    A = _arr(4096, sc.E4M3, (128, 64))
+    B = _arr(65536, sc.E4M3, (64, 256))
+    Y = _arr(1 << 20, sc.BF16, (128, 256))
+    assert L.scalify_scaled_matmul(R(A), 0, R(B), 0, R(Y), 0, None, None, 0, None) == -5          # workspace
+    assert L.scalify_scaled_matmul(R(good), 0, R(B), 0, R(Y), 0, None, 1 << 21, 1 << 20, None) == -2
+    assert L.scalify_scaled_matmul(R(A), 0, R(_arr(65536, sc.E4M3, (32, 256))), 0, R(Y), 0, None, 1 << 21, 1 << 20,
+                                   None) == -3
+    assert L.scalify_scaled_matmul(R(A), 0, R(B), 0, R(Y), 7, None, 1 << 21, 1 << 20, None) == -9
+    Yq = _arr(1 << 22, sc.E4M3, (128, 256))
+    assert L.scalify_scaled_matmul(R(A), 0, R(B), 0, R(Y), 0, R(Yq), 1 << 21, 1 << 20, None) == -9  # Yq needs a statistic
+    # rescale argument combinations
+    X = _arr(4096, sc.BF16, (256,))
+    Z = _arr(8192, sc.E4M3, (256,))
+    assert L.scalify_rescale(R(X), sc.STAT_AMAX, 64, None, R(Z), None, 0, None) == -9
+    assert L.scalify_rescale(R(X), sc.STAT_AMAX, None, None, R(Z), None, 0, None) == -5
+    assert L.scalify_rescale(R(X), sc.STAT_NONE, None, None, R(_arr(4096, sc.E4M3, (256,))), None, 0, None) == -8
+    # adam scalar ranges
+    assert L.scalify_scaled_adam_step(1, R(X), R(X), R(X), R(X), 1e-3, 1.5, 0.9, 1e-8, 1, 1 << 21, 1 << 20, None) == -9
+    assert L.scalify_scaled_adam_step(1, R(X), R(X), R(X), R(X), 1e-3, 0.9, 0.9, 1e-8, 0, 1 << 21, 1 << 20, None) == -9
+    assert L.scalify_scaled_adam_step(0, None, None, None, None, 1e-3, 0.9, 0.9, 1e-8, 1, None, 0, None) == 0
+    # layernorm row length must be a multiple of 16 bytes
+    assert L.scalify_scaled_layernorm(R(_arr(4096, sc.BF16, (4, 60), (64, 1))), None, None, 1e-5, 0,
+                                      R(_arr(8192, sc.BF16, (4, 60), (64, 1))), None, None, None) == -3

@@ -1,0 +1,85 @@
+"""GPU parity of the scaled Adam step against the oracle: scale words bit-exact
+(closed form of the static rules), FP16 / FP32 / BF16 outputs within 1 ulp."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as orc
+import paper_2407_17353_b200 as sc
+import scalify_inputs as si
+from helpers import to_dev, to_bits, ulp_diff
+
+pytestmark = pytest.mark.gpu
+
+
+def run_case(sizes, w_dt, mv_dt=orc.F16, g_dt=orc.E5M2, step=1000, seed=51, scales=None):
+    cases = []
+    G, M, V, W = [], [], [], []
+    for i, n in enumerate(sizes):
+        c = si.adam_case(n, seed=seed + i, w_dtype=w_dt if w_dt != orc.BF16 else orc.F16)
+        if w_dt == orc.BF16:
+            c["w"] = si.to_bits(si.normal(seed + i, 1, (n,), 0.02 * 64.0), orc.BF16)
+            c["w_dtype"] = orc.BF16
+        if mv_dt == orc.F32:
+            c["m"] = orc.encode(orc.decode(c["m"], orc.F16), orc.F32)
+            c["v"] = orc.encode(orc.decode(c["v"], orc.F16), orc.F32)
+            c["mv_dtype"] = orc.F32
+        if g_dt != orc.E5M2:
+            c["g"] = orc.encode(orc.decode(c["g"], orc.E5M2), g_dt)
+            c["g_dtype"] = g_dt
+        if scales:
+            c.update(scales)
+        cases.append(c)
+        G.append(sc.ScaledTensor.make(to_dev(c["g"], c["g_dtype"]), c["g_scale"]))
+        M.append(sc.ScaledTensor.make(to_dev(c["m"], c["mv_dtype"]), c["m_scale"]))
+        V.append(sc.ScaledTensor.make(to_dev(c["v"], c["mv_dtype"]), c["v_scale"]))
+        W.append(sc.ScaledTensor.make(to_dev(c["w"], c["w_dtype"]), c["w_scale"]))
+    ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_ADAM, len(sizes)))
+    tens = sc.AdamTensors(G, M, V, W)
+    c0 = cases[0]
+    sc.scalify_scaled_adam_step(tens, ws, lr=c0["lr"], beta1=c0["beta1"], beta2=c0["beta2"], eps=c0["eps"], step=step)
+    assert ws.check_status() == 0
+    for c, g, m, v, w in zip(cases, G, M, V, W):
+        mo, vo, wo, ms, vs, wsc = orc.adam_step(c["g"], c["g_dtype"], c["g_scale"], c["m"], c["v"], c["mv_dtype"],
+                                                c["m_scale"], c["v_scale"], c["w"], c["w_dtype"], c["w_scale"],
+                                                c["lr"], c["beta1"], c["beta2"], c["eps"], step)
+        assert (m.scale_value(), v.scale_value(), w.scale_value()) == (ms, vs, wsc)
+        assert ulp_diff(to_bits(m.data, c["mv_dtype"]), mo, c["mv_dtype"]).max() <= (1 if mv_dt != orc.F32 else 4)
+        assert ulp_diff(to_bits(v.data, c["mv_dtype"]), vo, c["mv_dtype"]).max() <= (1 if mv_dt != orc.F32 else 4)
+        assert ulp_diff(to_bits(w.data, c["w_dtype"]), wo, c["w_dtype"]).max() <= 1
+        # gradients are read-only
+        assert np.array_equal(to_bits(g.data, c["g_dtype"]), c["g"])
+
+
+@pytest.mark.parametrize("w_dt", [orc.F16, orc.F32, orc.BF16])
+def test_single_tensor_ragged_sizes(w_dt):
+    for n in (1, 7, 8, 1000, 8192 + 3, 256 * 8 * 4 * 3 + 9):
+        run_case([n], w_dt)
+
+
+@pytest.mark.parametrize("w_dt,mv_dt", [(orc.F16, orc.F16), (orc.F32, orc.F32)])
+def test_multi_tensor_list(w_dt, mv_dt):
+    sizes = [768, 2304, 768 * 64, 5, 8193, 3072, 1, 50257 * 8]
+    run_case(sizes, w_dt, mv_dt=mv_dt)
+
+
+def test_more_tensors_than_one_launch_holds():
+    run_case([64 + (i % 7) for i in range(170)], orc.F16)
+
+
+@pytest.mark.parametrize("step", [1, 2, 100000])
+def test_bias_correction_steps(step):
+    run_case([4096], orc.F16, step=step)
+
+
+def test_bf16_gradients_and_other_scales():
+    run_case([10000], orc.F32, g_dt=orc.BF16, scales=dict(g_scale=2.0 ** -3, m_scale=2.0 ** -2, v_scale=2.0 ** -9,
+                                                           w_scale=2.0 ** 1))
+
+
+def test_gpt2_small_parameter_list_shapes():
+    # the 148 tensors of the GPT-2-small-shaped list, scaled down 16x in the large dimensions to stay quick
+    shapes = si.gpt2_small_param_shapes()
+    sizes = [max(1, int(np.prod(s)) // 16) for s in shapes]
+    assert len(sizes) == 148
+    run_case(sizes, orc.F16)

@@ -1,0 +1,130 @@
+"""GPU parity of the scaled LayerNorm forward / backward kernels against the oracle.
+
+Forward outputs: within 1 ulp of the output format (fp32 arithmetic on the GPU,
+fp64 in the oracle).  Backward: dx is a difference of terms of size |ghat|*rinv,
+so its fp32 error is bounded relative to that magnitude, not to the (possibly
+tiny) result: |gpu - oracle| <= 1 ulp(result) or <= 2^-18 * max|ghat|*rinv of
+the row.  The fused statistic and the rescaled gradient are checked
+stage-isolated against the oracle's rescale of the library's own dX.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle as orc
+import paper_2407_17353_b200 as sc
+import scalify_inputs as si
+from helpers import to_dev, to_bits, ulp_diff
+
+pytestmark = pytest.mark.gpu
+
+
+def st(bits, dt, scale=None):
+    t = to_dev(bits, dt)
+    return sc.ScaledTensor.make(t, scale) if scale is not None else sc.ScaledTensor(t, None)
+
+
+SHAPES = [(1, 8), (37, 768), (300, 1024), (5, 4096), (129, 2048), (64, 72)]
+
+
+@pytest.mark.parametrize("R,d", SHAPES)
+@pytest.mark.parametrize("x_dt,y_dt", [(orc.BF16, orc.BF16), (orc.BF16, orc.E4M3), (orc.F16, orc.F16),
+                                       (orc.F32, orc.F32), (orc.F32, orc.BF16)])
+@pytest.mark.parametrize("eps_inside", [False, True])
+def test_layernorm_forward(R, d, x_dt, y_dt, eps_inside):
+    if x_dt == orc.F32 and d > 2048:
+        pytest.skip("row longer than the supported 8 KiB")
+    c = si.layernorm_case(R, d, seed=41, x_dtype=x_dt)
+    gs, bs = 2.0 ** -1, 2.0 ** 1
+    Y = sc.ScaledTensor.empty((R, d), sc.TORCH_DTYPE[y_dt])
+    mean = torch.empty(R, dtype=torch.float32, device="cuda")
+    rinv = torch.empty(R, dtype=torch.float32, device="cuda")
+    sc.scalify_scaled_layernorm(st(c["X"], x_dt, 2.0 ** 4), st(c["gamma"], orc.BF16, gs), st(c["beta"], orc.BF16, bs),
+                                Y, eps=1e-5, eps_inside_sqrt=eps_inside, mean=mean, rinv=rinv)
+    yo, ys, mo, ro = orc.layernorm_fwd(c["X"], x_dt, c["gamma"], orc.BF16, gs, c["beta"], orc.BF16, bs, 1e-5,
+                                       eps_inside, y_dt)
+    assert Y.scale_value() == ys == 2.0
+    got = to_bits(Y.data, y_dt)
+    if y_dt == orc.F32:
+        g, w = orc.decode(got, y_dt), orc.decode(yo, y_dt)
+        assert np.all(np.abs(g - w) <= 2e-6 * (np.abs(w) + 1.0))
+    else:
+        assert ulp_diff(got, yo, y_dt).max() <= 1
+    assert np.allclose(mean.cpu().numpy(), mo, rtol=0, atol=2e-6)
+    assert np.allclose(rinv.cpu().numpy(), ro, rtol=2e-6)
+
+
+def test_layernorm_forward_without_affine_constant_rows_and_strided_input():
+    R, d = 50, 256
+    x = si.scaled_normal(42, 1, (R, d), orc.BF16)
+    x[7, :] = si.to_bits(np.full(d, 3.0, dtype=np.float32), orc.BF16)  # zero-variance row
+    buf = torch.zeros((R, d + 64), dtype=torch.bfloat16, device="cuda")
+    buf[:, :d].copy_(to_dev(x, orc.BF16))
+    X = sc.ScaledTensor(buf[:, :d], None)
+    Y = sc.ScaledTensor.empty((R, d), torch.bfloat16)
+    sc.scalify_scaled_layernorm(X, None, None, Y, eps=1e-5)
+    yo, ys, _, _ = orc.layernorm_fwd(x, orc.BF16, None, 0, 1.0, None, 0, 1.0, 1e-5, False, orc.BF16)
+    assert Y.scale_value() == 1.0
+    got = to_bits(Y.data, orc.BF16)
+    assert ulp_diff(got, yo, orc.BF16).max() <= 1
+    assert np.all(orc.decode(got[7], orc.BF16) == 0.0)
+
+
+@pytest.mark.parametrize("R,d", [(1, 8), (37, 768), (300, 1024), (5, 4096), (1000, 768), (64, 72)])
+@pytest.mark.parametrize("eps_inside", [False, True])
+@pytest.mark.parametrize("stat", [sc.STAT_L2, sc.STAT_AMAX])
+def test_layernorm_backward_with_gradient_rescale(R, d, eps_inside, stat):
+    c = si.layernorm_case(R, d, seed=43)
+    x_s, g_s, gam_s = 2.0 ** 2, 2.0 ** -10, 2.0 ** -1
+    X, G, gamma = st(c["X"], orc.BF16, x_s), st(c["G"], orc.BF16, g_s), st(c["gamma"], orc.BF16, gam_s)
+    Y = sc.ScaledTensor.empty((R, d), torch.bfloat16)
+    mean = torch.empty(R, dtype=torch.float32, device="cuda")
+    rinv = torch.empty(R, dtype=torch.float32, device="cuda")
+    sc.scalify_scaled_layernorm(X, gamma, st(c["beta"], orc.BF16, 1.0), Y, eps=1e-5, eps_inside_sqrt=eps_inside,
+                                mean=mean, rinv=rinv)
+    dX = sc.ScaledTensor.empty((R, d), torch.bfloat16)
+    dXq = sc.ScaledTensor.empty((R, d), torch.float8_e5m2)
+    dg = sc.ScaledTensor.empty((d,), torch.float32)
+    db = sc.ScaledTensor.empty((d,), torch.float32)
+    ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_LAYERNORM_BWD, R, d))
+    sc.scalify_scaled_layernorm_bwd(G, X, gamma, mean, rinv, dX, ws, eps=1e-5, eps_inside_sqrt=eps_inside,
+                                    stat_dx=stat, dXq=dXq, dgamma=dg, dbeta=db)
+    assert ws.check_status() == 0
+    o = orc.layernorm_bwd(c["G"], orc.BF16, g_s, c["X"], orc.BF16, x_s, c["gamma"], orc.BF16, gam_s, 1e-5,
+                          eps_inside, orc.BF16, orc.F32, want_f64=True)
+    assert dX.scale_value() == o["dX_scale"]
+    assert dg.scale_value() == o["dgamma_scale"] and db.scale_value() == o["dbeta_scale"]
+    got = to_bits(dX.data, orc.BF16)
+    dists = ulp_diff(got, o["dX"], orc.BF16)
+    gv = orc.decode(c["G"], orc.BF16) * orc.decode(c["gamma"], orc.BF16)[None, :]
+    _, _, _, ro = orc.layernorm_fwd(c["X"], orc.BF16, None, 0, 1.0, None, 0, 1.0, 1e-5, eps_inside, orc.BF16)
+    row_mag = np.abs(gv).max(axis=1) * ro
+    abs_err = np.abs(orc.decode(got, orc.BF16) - o["dx_f64"])
+    ulp_of = np.abs(o["dx_f64"]) * 2.0 ** -8
+    ok = (dists <= 1) | (abs_err <= 0.5 * ulp_of + 2.0 ** -18 * row_mag[:, None])
+    assert ok.all(), int((~ok).sum())
+    # dgamma / dbeta: fp32 column sums, error relative to the sum of magnitudes
+    n, _, _, _ = orc.layernorm_fwd(c["X"], orc.BF16, None, 0, 1.0, None, 0, 1.0, 1e-5, eps_inside, orc.F32)
+    nv = orc.decode(n, orc.F32)
+    Gd = orc.decode(c["G"], orc.BF16)
+    f = orc.kf(R)
+    mag_g = np.abs(Gd * nv).sum(axis=0) / f
+    mag_b = np.abs(Gd).sum(axis=0) / f
+    got_dg = orc.decode(to_bits(dg.data, orc.F32), orc.F32)
+    got_db = orc.decode(to_bits(db.data, orc.F32), orc.F32)
+    assert np.all(np.abs(got_dg - (Gd * nv).sum(axis=0) / f) <= 2e-5 * mag_g + 1e-30)
+    assert np.all(np.abs(got_db - Gd.sum(axis=0) / f) <= 2e-5 * mag_b + 1e-30)
+    # statistic and rescaled gradient, stage-isolated on the library's own dX
+    so = orc.statistic(got, orc.BF16, stat)
+    gstat = float(ws.statistic().item())
+    if stat == sc.STAT_AMAX:
+        assert gstat == so
+    else:
+        assert abs(gstat - so) <= 2e-6 * so
+        if abs(math.log2(so) - round(math.log2(so))) < 1e-5:
+            return
+    qo, qs, _ = orc.rescale(got, orc.BF16, o["dX_scale"], stat, orc.E5M2)
+    assert dXq.scale_value() == qs
+    assert np.array_equal(to_bits(dXq.data, orc.E5M2), qo)

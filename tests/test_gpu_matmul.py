@@ -1,0 +1,207 @@
+"""GPU parity of the scaled FP8 matmul (tcgen05 kernel) against the fp64 oracle.
+
+Bars (stated by the benchmark contract): the propagated scale and every FP8 /
+scale word bit-exact; the fp32 pre-cast values within 1e-5 * sum|a*b| per
+element; BF16/F16 outputs within 1 ulp; the fused statistic equal to the
+statistic of the stored output; the rescaled output bit-exact against the
+oracle's rescale of the library's own intermediate (stage-isolated), because a
+power-of-two rescale of identical BF16 input has exactly one correct answer.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle as orc
+import paper_2407_17353_b200 as sc
+import scalify_inputs as si
+from helpers import to_dev, to_bits, ulp_diff
+
+pytestmark = pytest.mark.gpu
+
+
+def run_matmul(A, a_dt, a_s, B, b_dt, b_s, y_dt, transA=False, transB=False, stat=sc.STAT_NONE, q_dt=None,
+               lda_pad=0, ldb_pad=0):
+    """A, B: numpy bit arrays as stored (2-D or 3-D). Returns dict of numpy results."""
+    def dev(x, dt, pad):
+        if pad == 0:
+            return to_dev(x, dt)
+        shp = list(x.shape)
+        shp[-1] += pad
+        buf = torch.zeros(shp, dtype=torch.uint8, device="cuda").view(sc.TORCH_DTYPE[dt])
+        view = buf[..., : x.shape[-1]]
+        view.copy_(to_dev(x, dt))
+        return view
+    Ad, Bd = dev(A, a_dt, lda_pad), dev(B, b_dt, ldb_pad)
+    M = A.shape[-1] if transA else A.shape[-2]
+    N = B.shape[-2] if transB else B.shape[-1]
+    shape = (M, N) if A.ndim == 2 else (A.shape[0], M, N)
+    Y = sc.ScaledTensor.empty(shape, sc.TORCH_DTYPE[y_dt])
+    Yq = sc.ScaledTensor.empty(shape, sc.TORCH_DTYPE[q_dt]) if q_dt is not None else None
+    rows = M * (A.shape[0] if A.ndim == 3 else 1)
+    ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_MATMUL, rows, N))
+    sc.scalify_scaled_matmul(sc.ScaledTensor.make(Ad, a_s), sc.ScaledTensor.make(Bd, b_s), Y, ws, transA=transA,
+                             transB=transB, stat=stat, Yq=Yq)
+    status = ws.check_status()
+    out = dict(Y=to_bits(Y.data, y_dt), y_scale=Y.scale_value(), status=status,
+               stat=float(ws.statistic().item()))
+    if Yq is not None:
+        out["Yq"] = to_bits(Yq.data, q_dt)
+        out["yq_scale"] = Yq.scale_value()
+    return out
+
+
+def check_against_oracle(A, a_dt, a_s, B, b_dt, b_s, transA, transB, **kw):
+    # fp32 dump: accumulator error bar
+    g32 = run_matmul(A, a_dt, a_s, B, b_dt, b_s, orc.F32, transA, transB, **kw)
+    assert g32["status"] == 0
+    gb = run_matmul(A, a_dt, a_s, B, b_dt, b_s, orc.BF16, transA, transB, **kw)
+    assert gb["status"] == 0
+    if A.ndim == 2:
+        A3, B3 = A[None], B[None]
+    else:
+        A3, B3 = A, (B if B.ndim == 3 else np.broadcast_to(B, (A.shape[0],) + B.shape))
+    for b in range(A3.shape[0]):
+        Yo, ys, acc, sab = orc.scaled_matmul(A3[b], a_dt, a_s, B3[b], b_dt, b_s, orc.BF16, transA=transA,
+                                             transB=transB, want_acc=True)
+        g = g32["Y"].reshape((-1,) + Yo.shape)[b].view(np.float32).astype(np.float64)
+        assert g32["y_scale"] == ys and gb["y_scale"] == ys
+        err = np.abs(g - acc)
+        bound = 1e-5 * sab + 1e-30
+        assert np.all(err <= bound), (float((err / bound).max()), np.unravel_index(np.argmax(err / bound), err.shape))
+        d = ulp_diff(gb["Y"].reshape((-1,) + Yo.shape)[b], Yo, orc.BF16)
+        assert d.max() <= 1, int(d.max())
+        # bit-exact whenever the pre-cast fp32 value is identical: encode the library's own fp32 dump
+        assert np.array_equal(gb["Y"].reshape((-1,) + Yo.shape)[b], orc.encode(g, orc.BF16))
+
+
+def test_config1_256_cubed_with_dynamic_rescale():
+    c = si.config1()
+    Bt = np.ascontiguousarray(c["B"].T)
+    for transB, Bmat in [(True, Bt), (False, c["B"])]:
+        check_against_oracle(c["A"], orc.E4M3, c["a_scale"], Bmat, orc.E4M3, c["b_scale"], False, transB)
+        g = run_matmul(c["A"], orc.E4M3, c["a_scale"], Bmat, orc.E4M3, c["b_scale"], orc.BF16, False, transB,
+                       stat=sc.STAT_AMAX, q_dt=orc.BF16)
+        assert g["status"] == 0 and g["y_scale"] == 8.0
+        # the fused statistic is the AMAX of the stored intermediate
+        assert g["stat"] == orc.statistic(g["Y"], orc.BF16, orc.STAT_AMAX)
+        yq, yqs, _ = orc.rescale(g["Y"], orc.BF16, g["y_scale"], orc.STAT_AMAX, orc.BF16)
+        assert np.array_equal(g["Yq"], yq) and g["yq_scale"] == yqs
+        # end to end against the oracle chain
+        Yo, ys, _, _ = orc.scaled_matmul(c["A"], orc.E4M3, c["a_scale"], c["B"], orc.E4M3, c["b_scale"], orc.BF16)
+        yo, yos, so = orc.rescale(Yo, orc.BF16, ys, orc.STAT_AMAX, orc.BF16)
+        assert abs(so / orc.p2f(so) - 1.5) < 0.49  # this seed is not a binade-edge case
+        assert g["yq_scale"] == yos
+        assert ulp_diff(g["Yq"], yo, orc.BF16).max() <= 1
+
+
+@pytest.mark.parametrize("transA,transB", [(False, True), (False, False), (True, True), (True, False)])
+@pytest.mark.parametrize("a_dt,b_dt", [(orc.E4M3, orc.E4M3), (orc.E5M2, orc.E4M3), (orc.E4M3, orc.E5M2)])
+def test_ragged_shapes_all_layouts_and_formats(transA, transB, a_dt, b_dt):
+    M, N, K = 200, 304, 176  # ragged in every tile dimension; strides stay multiples of 16 bytes
+    A = si.scaled_normal(21, 1, (K, M) if transA else (M, K), a_dt)
+    B = si.scaled_normal(21, 2, (N, K) if transB else (K, N), b_dt)
+    check_against_oracle(A, a_dt, 2.0 ** -10, B, b_dt, 2.0 ** -6, transA, transB)
+
+
+def test_several_tiles_long_k_and_padded_leading_dimensions():
+    M, N, K = 384, 528, 1040
+    A = si.scaled_normal(22, 1, (M, K), orc.E5M2)
+    Bt = si.scaled_normal(22, 2, (N, K), orc.E4M3)
+    check_against_oracle(A, orc.E5M2, 1.0, Bt, orc.E4M3, 2.0 ** -6, False, True, lda_pad=48, ldb_pad=16)
+    B = np.ascontiguousarray(Bt.T)
+    check_against_oracle(A, orc.E5M2, 1.0, B, orc.E4M3, 2.0 ** -6, False, False, lda_pad=16, ldb_pad=32)
+
+
+def test_tiny_and_degenerate_shapes():
+    for (M, N, K) in [(1, 16, 16), (16, 16, 16), (129, 257, 144), (128, 256, 128)]:
+        A = si.scaled_normal(23, M, (M, K), orc.E4M3)
+        Bt = si.scaled_normal(23, 1000 + N, (N, K), orc.E4M3)
+        check_against_oracle(A, orc.E4M3, 1.0, Bt, orc.E4M3, 1.0, False, True)
+    # identity operand: exact copy of A (power-of-two rescale only)
+    K = 256
+    A = si.scaled_normal(23, 7, (128, K), orc.E4M3)
+    eye = si.to_bits(np.eye(K, dtype=np.float32) * 16.0, orc.E4M3)
+    g = run_matmul(A, orc.E4M3, 1.0, eye, orc.E4M3, 1.0, orc.BF16, False, False)
+    assert np.array_equal(orc.decode(g["Y"], orc.BF16), orc.decode(A, orc.E4M3))
+    assert g["y_scale"] == 16.0
+
+
+def test_batched_attention_like_shapes():
+    # QK^T-like: [b, T, 64] x [b, T, 64]^T ; PV-like: [b, T, T] x [b, T, 64]
+    b, T, hd = 3, 160, 64
+    Q = si.scaled_normal(24, 1, (b, T, hd), orc.E4M3)
+    Kt = si.scaled_normal(24, 2, (b, T, hd), orc.E4M3)
+    check_against_oracle(Q, orc.E4M3, 1.0, Kt, orc.E4M3, 1.0, False, True)
+    P = si.scaled_normal(24, 3, (b, T, T), orc.E4M3, 0.25)
+    V = si.scaled_normal(24, 4, (b, T, hd), orc.E4M3)
+    check_against_oracle(P, orc.E4M3, 1.0, V, orc.E4M3, 1.0, False, False)
+    # shared 2-D weight for every batch
+    W = si.scaled_normal(24, 5, (hd, 96), orc.E4M3)
+    check_against_oracle(Q, orc.E4M3, 1.0, W, orc.E4M3, 2.0 ** -6, False, False)
+
+
+@pytest.mark.parametrize("kind", ["fwd", "grad"])
+def test_config2_1024_full_compare_with_fused_amax_rescale_to_e4m3(kind):
+    c = si.gemm_case(1024, kind, seed=1)
+    check_against_oracle(c["A"], c["a_dtype"], c["a_scale"], c["Bt"], c["b_dtype"], c["b_scale"], False, True)
+    for stat in (sc.STAT_AMAX, sc.STAT_L2):
+        g = run_matmul(c["A"], c["a_dtype"], c["a_scale"], c["Bt"], c["b_dtype"], c["b_scale"], orc.BF16, False, True,
+                       stat=stat, q_dt=orc.E4M3)
+        assert g["status"] == 0
+        so = orc.statistic(g["Y"], orc.BF16, stat)
+        if stat == sc.STAT_AMAX:
+            assert g["stat"] == so
+        else:
+            assert abs(g["stat"] - so) <= 2e-6 * so
+            assert abs(so / orc.p2f(so) - 1.5) < 0.499  # not at a binade edge
+        yq, yqs, _ = orc.rescale(g["Y"], orc.BF16, g["y_scale"], stat, orc.E4M3)
+        assert g["yq_scale"] == yqs
+        assert np.array_equal(g["Yq"], yq)
+
+
+@pytest.mark.parametrize("n,kind", [(4096, "fwd"), (8192, "fwd"), (8192, "grad")])
+def test_config2_full_size_sampled_outputs_and_properties(n, kind):
+    c = si.gemm_case(n, kind, seed=2)
+    g = run_matmul(c["A"], c["a_dtype"], c["a_scale"], c["Bt"], c["b_dtype"], c["b_scale"], orc.BF16, False, True,
+                   stat=sc.STAT_AMAX, q_dt=orc.E4M3)
+    assert g["status"] == 0
+    assert g["y_scale"] == c["a_scale"] * c["b_scale"] * orc.kf(n)
+    rng = np.random.default_rng(5)
+    rows = np.concatenate([rng.integers(0, n, 2000), [0, n - 1, 127, 128, n - 129]])
+    cols = np.concatenate([rng.integers(0, n, 2000), [0, n - 1, 255, 256, n - 257]])
+    acc, sab = orc.scaled_matmul_samples(c["A"], c["a_dtype"], c["Bt"], c["b_dtype"], rows, cols, transB=True)
+    want = orc.encode(acc, orc.BF16)
+    got = g["Y"][rows, cols]
+    assert ulp_diff(got, want, orc.BF16).max() <= 1
+    # properties that hold at any size: statistic word = AMAX of the stored output; the rescaled
+    # output is the exact power-of-two rebalance of the stored intermediate
+    yv = torch.from_numpy(g["Y"].view(np.int16)).view(torch.bfloat16).float()
+    amax = float(yv.abs().max())
+    assert g["stat"] == amax
+    r = orc.p2f(amax)
+    assert g["yq_scale"] == g["y_scale"] * r
+    want_q = (yv / r).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    assert np.array_equal(g["Yq"], want_q)
+    assert 1.0 <= float(torch.from_numpy(g["Yq"]).view(torch.float8_e4m3fn).float().abs().max()) <= 2.0
+
+
+def test_accumulator_precision_with_adversarial_magnitudes():
+    # one large product followed by many small ones of the same sign: a narrow accumulator would
+    # lose the small terms.  Bound: 1e-5 * sum|a*b|.
+    M, N, K = 128, 256, 8192
+    a = np.full((M, K), 2.0 ** -3, dtype=np.float32)
+    a[:, 0] = 256.0
+    b = np.full((N, K), 2.0 ** -3, dtype=np.float32)
+    b[:, 0] = 256.0
+    A, Bt = si.to_bits(a, orc.E4M3), si.to_bits(b, orc.E4M3)
+    g = run_matmul(A, orc.E4M3, 1.0, Bt, orc.E4M3, 1.0, orc.F32, False, True)
+    exact = (65536.0 + (K - 1) * 2.0 ** -6) / orc.kf(K)
+    got = g["Y"].view(np.float32).astype(np.float64)
+    assert np.all(np.abs(got - exact) <= 1e-5 * exact), float(np.abs(got - exact).max() / exact)
+
+
+def test_bad_scale_is_reported_in_status_word():
+    A = si.scaled_normal(25, 1, (128, 128), orc.E4M3)
+    Bt = si.scaled_normal(25, 2, (256, 128), orc.E4M3)
+    g = run_matmul(A, orc.E4M3, 3.0, Bt, orc.E4M3, 1.0, orc.BF16, False, True)
+    assert g["status"] & sc.DEV_BAD_SCALE
