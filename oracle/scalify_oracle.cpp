@@ -210,18 +210,21 @@ double statistic(const std::vector<double>& x, int stat) {
 }
 
 double gelu_gate(double x, int exact_erf) {
-  // f(x) = x * g(x); tanh form is GPT-2's, erf form is the exact Gaussian CDF
-  if (exact_erf) return 0.5 * (1.0 + std::erf(x / std::sqrt(2.0)));
+  // f(x) = x * g(x).  Both gates are written in the form that keeps relative accuracy where the
+  // gate is tiny (x << 0): 0.5*(1+erf(x/sqrt2)) = 0.5*erfc(-x/sqrt2) (exact Gaussian CDF) and
+  // 0.5*(1+tanh(u)) = 1/(1+exp(-2u)) (GPT-2's tanh form); the left-hand forms cancel to 0 there.
+  if (exact_erf) return 0.5 * std::erfc(-x / std::sqrt(2.0));
   const double c = std::sqrt(2.0 / M_PI);
-  return 0.5 * (1.0 + std::tanh(c * (x + 0.044715 * x * x * x)));
+  const double u = c * (x + 0.044715 * x * x * x);
+  return 1.0 / (1.0 + std::exp(-2.0 * u));
 }
 
 double gelu_gate_deriv(double x, int exact_erf) {
   if (exact_erf) return std::exp(-0.5 * x * x) / std::sqrt(2.0 * M_PI);
   const double c = std::sqrt(2.0 / M_PI);
-  double u = c * (x + 0.044715 * x * x * x);
-  double t = std::tanh(u);
-  return 0.5 * (1.0 - t * t) * c * (1.0 + 3.0 * 0.044715 * x * x);
+  const double g = gelu_gate(x, 0);
+  // d/dx sigma(2u) = 2*sigma*(1-sigma)*u'
+  return 2.0 * g * (1.0 - g) * c * (1.0 + 3.0 * 0.044715 * x * x);
 }
 
 }  // namespace

@@ -314,21 +314,27 @@ int launch_add(const void* a, const void* b, int ab_dt, void* y, int out_dt, int
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ float gelu_u(float x) { return 0.7978845608028654f * fmaf(0.044715f * x * x, x, x); }
 
-// gate g(x): tanh form written as a logistic, 0.5*(1+tanh(u)) = 1/(1+exp(-2u)), which keeps
-// full relative accuracy where the gate is tiny
+// gate g(x): tanh form written as a logistic, 0.5*(1+tanh(u)) = 1/(1+exp(-2u)), and the erf form as
+// 0.5*erfc(-x/sqrt2); both keep full relative accuracy where the gate is tiny
 template <int EXACT>
 __device__ __forceinline__ float gelu_gate(float x) {
-  if constexpr (EXACT) return 0.5f * (1.0f + erff(x * 0.7071067811865476f));
-  else return 1.0f / (1.0f + __expf(-2.0f * gelu_u(x)));
+  if constexpr (EXACT) return 0.5f * erfcf(-x * 0.7071067811865476f);
+  else {
+    // logistic of 2u through t = exp(-2|u|) in (0,1]: never overflows, and underflows gradually
+    const float u = gelu_u(x);
+    const float t = __expf(-2.0f * fabsf(u));
+    const float r = 1.0f / (1.0f + t);
+    return u >= 0.f ? r : t * r;
+  }
 }
 
 template <int EXACT>
 __device__ __forceinline__ float gelu_deriv(float x) {  // f'(x) = g + x*g'
   if constexpr (EXACT) {
-    float g = 0.5f * (1.0f + erff(x * 0.7071067811865476f));
+    float g = 0.5f * erfcf(-x * 0.7071067811865476f);
     return fmaf(x, 0.3989422804014327f * __expf(-0.5f * x * x), g);
   } else {
-    float g = 1.0f / (1.0f + __expf(-2.0f * gelu_u(x)));
+    float g = gelu_gate<0>(x);
     float du = 0.7978845608028654f * fmaf(3.0f * 0.044715f * x, x, 1.0f);
     return fmaf(x, 2.0f * g * (1.0f - g) * du, g);
   }

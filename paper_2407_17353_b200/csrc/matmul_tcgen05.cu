@@ -43,6 +43,7 @@ struct GemmParams {
   int M, N, K, batch;
   int tiles_m, tiles_n;
   int a_mn_major, b_mn_major;  // 0: K-major (row-major [rows,K]); 1: MN-major (row-major [K,rows])
+  int b_batched;               // 0: one 2-D B shared by every batch
   uint32_t idesc;
   float alpha;                 // 1/kf(K)
   float kf;
@@ -236,11 +237,12 @@ scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
           const uint32_t sa = smem_a + stage * kABytes, sb = smem_b + stage * kBBytes;
           if (p.a_mn_major) tma_load_3d(sa, &map_a, fb, m0, k0, b);
           else tma_load_3d(sa, &map_a, fb, k0, m0, b);
+          const int bb = p.b_batched ? b : 0;
           if (p.b_mn_major) {
-            tma_load_3d(sb, &map_b, fb, n0, k0, b);
-            tma_load_3d(sb + kBK * 128, &map_b, fb, n0 + 128, k0, b);
+            tma_load_3d(sb, &map_b, fb, n0, k0, bb);
+            tma_load_3d(sb + kBK * 128, &map_b, fb, n0 + 128, k0, bb);
           } else {
-            tma_load_3d(sb, &map_b, fb, k0, n0, b);
+            tma_load_3d(sb, &map_b, fb, k0, n0, bb);
           }
           ++issued;
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
@@ -433,8 +435,10 @@ int launch_scaled_matmul(const MatmulArgs& a, void* ws, cudaStream_t st) {
   else rc = make_map(&map_a, a.A, a.M, a.K, a.batch, a.lda, a.a_bs, kBK);
   if (rc) return rc;
   // B is logically [K,N]; stored [K,N] (MN-major) or, with transB, [N,K] (K-major).
-  if (a.transB) rc = make_map(&map_b, a.B, a.K, a.N, a.batch, a.ldb, a.b_bs, kBN);
-  else rc = make_map(&map_b, a.B, a.N, a.K, a.batch, a.ldb, a.b_bs, kBK);
+  const int b_batched = a.b_bs != 0 ? 1 : 0;
+  const int b_batch = b_batched ? a.batch : 1;
+  if (a.transB) rc = make_map(&map_b, a.B, a.K, a.N, b_batch, a.ldb, a.b_bs, kBN);
+  else rc = make_map(&map_b, a.B, a.N, a.K, b_batch, a.ldb, a.b_bs, kBK);
   if (rc) return rc;
 
   GemmParams p;
@@ -443,6 +447,7 @@ int launch_scaled_matmul(const MatmulArgs& a, void* ws, cudaStream_t st) {
   p.tiles_n = (a.N + kBN - 1) / kBN;
   p.a_mn_major = a.transA ? 1 : 0;
   p.b_mn_major = a.transB ? 0 : 1;
+  p.b_batched = b_batched;
   // instruction descriptor (kind::f8f6f4): D fp32, A/B formats (0 = E4M3, 1 = E5M2), operand
   // majorness (0 = K-major), N >> 3, M >> 4
   p.idesc = (1u << 4) | (uint32_t(a.a_dt == SCALIFY_E5M2) << 7) | (uint32_t(a.b_dt == SCALIFY_E5M2) << 10) |

@@ -47,3 +47,27 @@ def ulp_diff(a: np.ndarray, b: np.ndarray, dtype: int) -> np.ndarray:
 
 def scale_of(t) -> float:
     return float(t.scale.item())
+
+
+_MBITS = {orc.E4M3: 3, orc.E5M2: 2, orc.F16: 10, orc.BF16: 7, orc.F32: 23}
+_EMIN = {orc.E4M3: -6, orc.E5M2: -14, orc.F16: -14, orc.BF16: -126, orc.F32: -126}
+
+
+def ulp_of(x: np.ndarray, dtype: int) -> np.ndarray:
+    """Spacing of the format `dtype` at magnitude |x| (the subnormal quantum below the smallest normal)."""
+    ax = np.abs(np.asarray(x, dtype=np.float64))
+    with np.errstate(divide="ignore"):
+        e = np.floor(np.log2(np.where(ax > 0, ax, 1.0)))
+    e = np.maximum(np.where(ax > 0, e, _EMIN[dtype]), _EMIN[dtype])
+    return np.exp2(e - _MBITS[dtype])
+
+
+def within(got_bits, want_bits, dtype, exact, err_mag, c):
+    """Mask of acceptable outputs for a result computed in fp32 and rounded once to `dtype`:
+    within 1 ulp of the oracle's encoding, or |value - exact| <= ulp(exact)/2 + c * err_mag, where
+    err_mag is the magnitude of the terms that were added (a sum that cancels has an error
+    relative to its terms, not to its result)."""
+    d = ulp_diff(got_bits, want_bits, dtype)
+    err = np.abs(orc.decode(got_bits, dtype) - exact)
+    with np.errstate(invalid="ignore"):
+        return (d <= 1) | (err <= 0.5 * ulp_of(exact, dtype) + c * err_mag)
