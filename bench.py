@@ -158,6 +158,92 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def run_profile_row(args):
+    """One row of the hot path alone, on a case that holds well under 2 GB on the device but is larger than
+    L2, launched `--steps` times after `--warmup` launches.  Meant to be run under ncu."""
+    import torch
+
+    import paper_2407_17353_b200 as sc
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+
+    def rnd(shape, dtype, tid, std=1.0):
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(tid)
+        return (torch.randn(shape, device=dev, dtype=torch.float32, generator=gen) * std).to(dtype)
+
+    row = args.profile_row
+    if row == "matmul":
+        n = N_GEMM
+        A = sc.ScaledTensor.make(rnd((n, n), torch.float8_e4m3fn, 1), 1.0)
+        Bt = sc.ScaledTensor.make(rnd((n, n), torch.float8_e4m3fn, 2), 2.0 ** -6)
+        Y = sc.ScaledTensor.empty((n, n), torch.bfloat16, dev)
+        ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_MATMUL, n, n), dev)
+        fn = lambda t: sc.scalify_scaled_matmul(A, Bt, Y, ws, transB=True, stat=sc.STAT_AMAX)
+        work = {"flop": 2.0 * n ** 3}
+    elif row == "rescale":
+        n = 8192 * 8192
+        X = sc.ScaledTensor.make(rnd((n,), torch.bfloat16, 1, 37.0), 1.0)
+        Yq = sc.ScaledTensor.empty((n,), torch.float8_e4m3fn, dev)
+        ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_RESCALE, n), dev)
+        fn = lambda t: sc.scalify_rescale(X, Yq, stat=sc.STAT_AMAX, ws=ws)
+        work = {"bytes": 5.0 * n}
+    elif row == "add":
+        n = 8192 * 8192
+        P = sc.ScaledTensor.make(rnd((n,), torch.bfloat16, 1), 1.0)
+        Q = sc.ScaledTensor.make(rnd((n,), torch.bfloat16, 2), 0.25)
+        S = sc.ScaledTensor.empty((n,), torch.bfloat16, dev)
+        fn = lambda t: sc.scalify_scaled_add(P, Q, S)
+        work = {"bytes": 6.0 * n}
+    elif row == "layernorm":
+        R, d = 65536, 1024
+        X = sc.ScaledTensor.make(rnd((R, d), torch.bfloat16, 3), 1.0)
+        G = sc.ScaledTensor.make(rnd((R, d), torch.bfloat16, 4), 2.0 ** -10)
+        gamma = sc.ScaledTensor.make((1.0 + 0.1 * rnd((d,), torch.float32, 5)).to(torch.bfloat16), 1.0)
+        beta = sc.ScaledTensor.make(rnd((d,), torch.bfloat16, 6, 0.1), 1.0)
+        LY = sc.ScaledTensor.empty((R, d), torch.bfloat16, dev)
+        mean = torch.empty(R, dtype=torch.float32, device=dev)
+        rinv = torch.empty(R, dtype=torch.float32, device=dev)
+        dX = sc.ScaledTensor.empty((R, d), torch.bfloat16, dev)
+        dXq = sc.ScaledTensor.empty((R, d), torch.float8_e5m2, dev)
+        dg = sc.ScaledTensor.empty((d,), torch.float32, dev)
+        db = sc.ScaledTensor.empty((d,), torch.float32, dev)
+        ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_LAYERNORM_BWD, R, d), dev)
+
+        def fn(t):
+            sc.scalify_scaled_layernorm(X, gamma, beta, LY, eps=1e-5, mean=mean, rinv=rinv)
+            sc.scalify_scaled_layernorm_bwd(G, X, gamma, mean, rinv, dX, ws, eps=1e-5, stat_dx=sc.STAT_L2, dXq=dXq,
+                                            dgamma=dg, dbeta=db)
+        work = {"bytes": 13.0 * R * d}
+    else:
+        n = 64 * 1024 * 1024
+        ag = sc.ScaledTensor.make(rnd((n,), torch.float8_e5m2, 7), 2.0 ** -12)
+        am = sc.ScaledTensor.make(rnd((n,), torch.float16, 8, 1.6), 2.0 ** -16)
+        av = sc.ScaledTensor.make((rnd((n,), torch.float32, 9) ** 2).to(torch.float16), 2.0 ** -24)
+        aw = sc.ScaledTensor.make(rnd((n,), torch.float16, 10, 1.28), 2.0 ** -6)
+        adam = sc.AdamTensors([ag], [am], [av], [aw])
+        ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_ADAM, 1), dev)
+        fn = lambda t: sc.scalify_scaled_adam_step(adam, ws, lr=3e-4, beta1=0.9, beta2=0.999, eps=1e-8,
+                                                   step=1000 + (t % 2))
+        work = {"bytes": 13.0 * n}
+    for t in range(args.warmup):
+        fn(t)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for t in range(args.steps):
+        fn(t)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / max(args.steps, 1)
+    out = {"profile_row": row, "ms_per_launch_group": ms}
+    if "flop" in work:
+        out["TFLOP/s"] = work["flop"] / (ms * 1e-3) / 1e12
+    else:
+        out["GB/s"] = work["bytes"] / (ms * 1e-3) / 1e9
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -165,9 +251,14 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--profile-row", default=None, choices=["matmul", "rescale", "add", "layernorm", "adam"],
+                    help="run only this row on a reduced, still larger-than-L2 case (for ncu captures)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.profile_row:
+        run_profile_row(args)
         return
 
     import numpy as np

@@ -24,20 +24,30 @@
 
 namespace scalify {
 
-constexpr int kBM = 128;
-constexpr int kBN = 256;
-constexpr int kBK = 128;  // FP8 elements = bytes
+constexpr int kBM = 128;   // rows of the output tile per CTA
+constexpr int kBN = 256;   // columns of the output tile
+constexpr int kBK = 128;   // FP8 elements = bytes per K block (one 128-byte swizzle row)
 constexpr int kUmmaK = 32;
-constexpr int kStages = 4;
 constexpr int kAccStages = 2;
 constexpr int kGemmThreads = 192;
-constexpr int kABytes = kBM * kBK;           // 16 KB
-constexpr int kBBytes = kBN * kBK;           // 32 KB
-constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kTmemCols = kAccStages * kBN;  // 512
-constexpr int kGroupM = 16;                  // m-tiles per rasterisation group
-constexpr size_t kGemmSmem = size_t(kStages) * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kGroupM = 8;                   // m-tiles per rasterisation group
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
+
+// NCTA = 1: one CTA computes a 128 x 256 tile (tcgen05 cta_group::1).
+// NCTA = 2: a cluster of two CTAs on an SM pair computes a 256 x 256 tile (cta_group::2): each
+//           CTA stages its own 128 rows of A and its own 128-column half of B, the leader CTA
+//           issues the MMAs, which read both CTAs' shared memory and write both CTAs' TMEM.
+//           Per SM this halves the shared-memory traffic of B, the limiter of the 1-CTA form.
+template <int NCTA> struct GemmCfg {
+  static constexpr int kTileM = kBM * NCTA;
+  static constexpr int kBRows = kBN / NCTA;          // B rows (columns of the output) staged per CTA
+  static constexpr int kABytes = kBM * kBK;          // 16 KB
+  static constexpr int kBBytes = kBRows * kBK;       // 32 KB / 16 KB
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kStages = NCTA == 1 ? 4 : 6;
+  static constexpr size_t kSmem = size_t(kStages) * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
 
 struct GemmParams {
   int M, N, K, batch;
@@ -145,6 +155,49 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// ---- cta_group::2 forms (cluster of two CTAs on an SM pair)
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// shared::cluster address of the same shared-memory offset in CTA `rank` of this cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA load whose completion bytes are counted on an mbarrier that may live in the peer CTA
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster_addr, int x,
+                                                 int y, int z) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar_cluster_addr), "r"(x), "r"(y), "r"(z)
+      : "memory");
+}
+__device__ __forceinline__ void umma_f8_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                             uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// arrives on the barrier at this shared-memory offset in BOTH CTAs of the pair
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  const uint16_t mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(mask) : "memory");
+}
+
 // Shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1 (sm_100).
 //   bits [0,14)  start address >> 4      bits [16,30) leading-dimension byte offset >> 4
 //   bits [32,46) stride-dimension byte offset >> 4      bits [46,48) version = 1
@@ -175,18 +228,20 @@ __device__ __forceinline__ void tile_coords(const GemmParams& p, int tile, int& 
   nt = r / gm;
 }
 
-template <int OUT>
+template <int OUT, int NCTA>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                      const GemmParams p) {
+  using C = GemmCfg<NCTA>;
+  constexpr int kStages = C::kStages;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (base - raw);
   const uint32_t smem_a = base;
-  const uint32_t smem_b = base + kStages * kABytes;
-  uint8_t* bar_mem = smem + kStages * kStageBytes;
-  const uint32_t bars = base + kStages * kStageBytes;
+  const uint32_t smem_b = base + kStages * C::kABytes;
+  uint8_t* bar_mem = smem + kStages * C::kStageBytes;
+  const uint32_t bars = base + kStages * C::kStageBytes;
   const uint32_t full_bar = bars;                         // kStages x 8 B
   const uint32_t empty_bar = bars + 8 * kStages;          // kStages x 8 B
   const uint32_t acc_full_bar = bars + 16 * kStages;      // kAccStages x 8 B
@@ -196,12 +251,18 @@ scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = (NCTA == 2) ? cluster_ctarank() : 0u;  // position in the CTA pair; 0 = leader
+  const int unit = blockIdx.x / NCTA;                          // CTA (NCTA=1) or cluster (NCTA=2) index
+  const int num_units = gridDim.x / NCTA;
   const int num_kb = (p.K + kBK - 1) / kBK;
   const int num_tiles = p.tiles_m * p.tiles_n * p.batch;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(full_bar + 8 * s, 1); mbar_init(empty_bar + 8 * s, 1); }
-    for (int s = 0; s < kAccStages; ++s) { mbar_init(acc_full_bar + 8 * s, 1); mbar_init(acc_empty_bar + 8 * s, 4); }
+    for (int s = 0; s < kAccStages; ++s) {
+      mbar_init(acc_full_bar + 8 * s, 1);
+      mbar_init(acc_empty_bar + 8 * s, 4 * NCTA);  // one arrival per epilogue warp of every CTA of the pair
+    }
     mbar_init(drain_bar, 1);
     *abort_flag = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -214,6 +275,7 @@ scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
   if (warp == 1) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
   tc_fence_before();
   __syncthreads();
+  if constexpr (NCTA == 2) cluster_sync_all();  // the peer's barriers exist before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   bool timed_out = false;
@@ -225,32 +287,43 @@ scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
       asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_b)) : "memory");
       uint32_t stage = 0, phase = 0;
       long long issued = 0;
-      for (int tile = blockIdx.x; tile < num_tiles && !timed_out; tile += gridDim.x) {
+      for (int tile = unit; tile < num_tiles && !timed_out; tile += num_units) {
         int b, mt, nt;
         tile_coords(p, tile, b, mt, nt);
-        const int m0 = mt * kBM, n0 = nt * kBN;
+        const int m0 = mt * C::kTileM + static_cast<int>(rank) * kBM;
+        const int n0 = nt * kBN + static_cast<int>(rank) * C::kBRows * (NCTA - 1);
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag)) { timed_out = true; break; }
-          const uint32_t fb = full_bar + 8 * stage;
-          mbar_expect_tx(fb, kStageBytes);
           const int k0 = kb * kBK;
-          const uint32_t sa = smem_a + stage * kABytes, sb = smem_b + stage * kBBytes;
-          if (p.a_mn_major) tma_load_3d(sa, &map_a, fb, m0, k0, b);
-          else tma_load_3d(sa, &map_a, fb, k0, m0, b);
+          const uint32_t sa = smem_a + stage * C::kABytes, sb = smem_b + stage * C::kBBytes;
           const int bb = p.b_batched ? b : 0;
-          if (p.b_mn_major) {
-            tma_load_3d(sb, &map_b, fb, n0, k0, bb);
-            tma_load_3d(sb + kBK * 128, &map_b, fb, n0 + 128, k0, bb);
+          if constexpr (NCTA == 1) {
+            const uint32_t fb = full_bar + 8 * stage;
+            mbar_expect_tx(fb, C::kStageBytes);
+            if (p.a_mn_major) tma_load_3d(sa, &map_a, fb, m0, k0, b);
+            else tma_load_3d(sa, &map_a, fb, k0, m0, b);
+            if (p.b_mn_major) {
+              tma_load_3d(sb, &map_b, fb, n0, k0, bb);
+              tma_load_3d(sb + kBK * 128, &map_b, fb, n0 + 128, k0, bb);
+            } else {
+              tma_load_3d(sb, &map_b, fb, k0, n0, bb);
+            }
           } else {
-            tma_load_3d(sb, &map_b, fb, k0, n0, bb);
+            // both CTAs' copies are counted on the LEADER's full barrier, which expects the bytes of the pair
+            const uint32_t fb = map_to_cta(full_bar + 8 * stage, 0u);
+            if (rank == 0u) mbar_expect_tx(full_bar + 8 * stage, 2 * C::kStageBytes);
+            if (p.a_mn_major) tma_load_3d_pair(sa, &map_a, fb, m0, k0, b);
+            else tma_load_3d_pair(sa, &map_a, fb, k0, m0, b);
+            if (p.b_mn_major) tma_load_3d_pair(sb, &map_b, fb, n0, k0, bb);
+            else tma_load_3d_pair(sb, &map_b, fb, k0, n0, bb);
           }
           ++issued;
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
-      if (timed_out || *abort_flag) {
-        // drain: every copy this thread issued signals its full barrier; wait (bounded) for the
-        // most recent use of each ring slot so that no copy is in flight when the CTA exits
+      if ((timed_out || *abort_flag) && rank == 0u) {
+        // drain: every copy signals a full barrier of this CTA; wait (bounded) for the most recent use of
+        // each ring slot so that no copy is in flight when the CTA (pair) exits
         const int pending = issued < kStages ? static_cast<int>(issued) : kStages;
         uint32_t s = stage, ph = phase;
         for (int i = 0; i < pending; ++i) {
@@ -261,37 +334,43 @@ scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
       }
     }
   } else if (warp == 1) {
-    // ---------------------------------------------------------------- MMA issuer
-    if (lane == 0) {
+    // ---------------------------------------------------------------- MMA issuer (leader CTA only)
+    if (lane == 0 && rank == 0u) {
       uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
       const uint32_t a_lbo = 0u, a_sbo = 1024u;
-      const uint32_t b_lbo = p.b_mn_major ? kBK * 128u : 0u, b_sbo = 1024u;
+      const uint32_t b_lbo = (p.b_mn_major && NCTA == 1) ? kBK * 128u : 0u, b_sbo = 1024u;
       const uint32_t a_step = p.a_mn_major ? (kUmmaK * 128u) : kUmmaK;  // bytes per K=32 step
       const uint32_t b_step = p.b_mn_major ? (kUmmaK * 128u) : kUmmaK;
-      for (int tile = blockIdx.x; tile < num_tiles && !timed_out; tile += gridDim.x) {
+      for (int tile = unit; tile < num_tiles && !timed_out; tile += num_units) {
         if (!mbar_wait(acc_empty_bar + 8 * acc, acc_phase ^ 1u, abort_flag)) { timed_out = true; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * kBN;
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(full_bar + 8 * stage, phase, abort_flag)) { timed_out = true; break; }
           tc_fence_after();
-          const uint32_t sa = smem_a + stage * kABytes, sb = smem_b + stage * kBBytes;
+          const uint32_t sa = smem_a + stage * C::kABytes, sb = smem_b + stage * C::kBBytes;
 #pragma unroll
           for (int k = 0; k < kBK / kUmmaK; ++k) {
             const uint64_t ad = make_smem_desc(sa + k * a_step, a_lbo, a_sbo);
             const uint64_t bd = make_smem_desc(sb + k * b_step, b_lbo, b_sbo);
-            umma_f8(d_tmem, ad, bd, p.idesc, (kb | k) != 0 ? 1u : 0u);
+            if constexpr (NCTA == 1) umma_f8(d_tmem, ad, bd, p.idesc, (kb | k) != 0 ? 1u : 0u);
+            else umma_f8_pair(d_tmem, ad, bd, p.idesc, (kb | k) != 0 ? 1u : 0u);
           }
-          umma_commit(empty_bar + 8 * stage);  // slot free once these MMAs have read it
+          // slot free (in both CTAs) once these MMAs have read it
+          if constexpr (NCTA == 1) umma_commit(empty_bar + 8 * stage);
+          else umma_commit_pair(empty_bar + 8 * stage);
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
         if (timed_out) break;
-        umma_commit(acc_full_bar + 8 * acc);  // accumulator complete
+        // accumulator complete (in both CTAs)
+        if constexpr (NCTA == 1) umma_commit(acc_full_bar + 8 * acc);
+        else umma_commit_pair(acc_full_bar + 8 * acc);
         if (++acc == kAccStages) { acc = 0; acc_phase ^= 1u; }
       }
       if (timed_out || *abort_flag) {
         // all MMAs issued so far must retire before TMEM is freed
-        umma_commit(drain_bar);
+        if constexpr (NCTA == 1) umma_commit(drain_bar);
+        else umma_commit_pair(drain_bar);
         const unsigned long long t0 = global_timer_ns();
         while (!mbar_try_wait(drain_bar, 0u) && global_timer_ns() - t0 < kWaitLimitNs) {}
       }
@@ -303,12 +382,12 @@ scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     uint32_t amax_bits = 0u;
     char* const Yb = static_cast<char*>(p.Y);
     constexpr int OSZ = ElemBytes<OUT>::v;
-    for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
+    for (int tile = unit; tile < num_tiles; tile += num_units) {
       int b, mt, nt;
       tile_coords(p, tile, b, mt, nt);
       if (!mbar_wait(acc_full_bar + 8 * acc, acc_phase, abort_flag)) { timed_out = true; break; }
       tc_fence_after();
-      const int row = mt * kBM + q * 32 + lane;
+      const int row = mt * C::kTileM + static_cast<int>(rank) * kBM + q * 32 + lane;
       const int n0 = nt * kBN;
       const bool row_ok = row < p.M;
       char* yrow = Yb + (static_cast<long long>(b) * p.y_batch_stride + static_cast<long long>(row) * p.ldy) * OSZ;
@@ -337,16 +416,21 @@ scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
 #pragma unroll
             for (int j = 0; j < 32 * OSZ / 16; ++j) st_raw<16>(yrow + static_cast<long long>(col0) * OSZ + j * 16, o + 4 * j);
           } else {
-            for (int i = 0; i < 32 && col0 + i < p.N; ++i) store_elem<OUT>(yrow, col0 + i, v[i]);
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (col0 + i < p.N) store_elem<OUT>(yrow, col0 + i, v[i]);
           }
         }
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(acc_empty_bar + 8 * acc);
+      if (lane == 0) {
+        if constexpr (NCTA == 1) mbar_arrive(acc_empty_bar + 8 * acc);
+        else mbar_arrive_cluster(map_to_cta(acc_empty_bar + 8 * acc, 0u));  // the leader issues the next MMAs
+      }
       if (p.stat == SCALIFY_STAT_L2) {
         const double s = warp_sum_f64(static_cast<double>(ssq));
-        if (lane == 0) p.l2_partials[static_cast<long long>(tile) * 4 + q] = s;
+        if (lane == 0) p.l2_partials[(static_cast<long long>(tile) * NCTA + rank) * 4 + q] = s;
       }
       if (++acc == kAccStages) { acc = 0; acc_phase ^= 1u; }
     }
@@ -361,6 +445,7 @@ scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
   if (timed_out && p.status) atomicOr(p.status, static_cast<uint32_t>(SCALIFY_DEV_TIMEOUT));
   tc_fence_before();
   __syncthreads();
+  if constexpr (NCTA == 2) cluster_sync_all();  // neither CTA leaves while the other may still touch its memory
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);
@@ -425,9 +510,59 @@ size_t matmul_ws_bytes(int64_t rows, int64_t cols) {
   return kWsHeader + size_t(tiles) * 4 * sizeof(double) + 256;
 }
 
-int launch_scaled_matmul(const MatmulArgs& a, void* ws, cudaStream_t st) {
+template <int OUT, int NCTA>
+static int launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, const GemmParams& p, long long tiles,
+                          cudaStream_t st) {
+  using C = GemmCfg<NCTA>;
+  auto kernel = scaled_matmul_kernel<OUT, NCTA>;
   static bool attr_done = false;
+  static int max_clusters = 0;
+  if (!attr_done) {
+    SCALIFY_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(C::kSmem)));
+    if (NCTA == 2) {
+      cudaLaunchConfig_t qc = {};
+      qc.gridDim = dim3(unsigned(sm_count() / 2 * 2));
+      qc.blockDim = dim3(kGemmThreads);
+      qc.dynamicSmemBytes = C::kSmem;
+      cudaLaunchAttribute qa[1];
+      qa[0].id = cudaLaunchAttributeClusterDimension;
+      qa[0].val.clusterDim.x = 2; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
+      qc.attrs = qa;
+      qc.numAttrs = 1;
+      int n = 0;
+      SCALIFY_CUDA_TRY(cudaOccupancyMaxActiveClusters(&n, kernel, &qc));
+      if (n < 1) return SCALIFY_ERR_UNSUPPORTED;
+      max_clusters = n;
+    }
+    attr_done = true;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attrs[1];
+  if (NCTA == 2) {
+    const long long units = tiles < max_clusters ? tiles : max_clusters;
+    cfg.gridDim = dim3(unsigned(units * 2));
+    attrs[0].id = cudaLaunchAttributeClusterDimension;
+    attrs[0].val.clusterDim.x = 2; attrs[0].val.clusterDim.y = 1; attrs[0].val.clusterDim.z = 1;
+    cfg.attrs = attrs;
+    cfg.numAttrs = 1;
+  } else {
+    cfg.gridDim = dim3(unsigned(tiles < sm_count() ? tiles : sm_count()));
+    cfg.attrs = nullptr;
+    cfg.numAttrs = 0;
+  }
+  cfg.blockDim = dim3(kGemmThreads);
+  cfg.dynamicSmemBytes = C::kSmem;
+  cfg.stream = st;
+  SCALIFY_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, map_a, map_b, p));
+  return SCALIFY_OK;
+}
+
+int launch_scaled_matmul(const MatmulArgs& a, void* ws, cudaStream_t st) {
   WsView v = ws_view(ws);
+  // two-CTA tiles (256 rows) whenever there is more than one 128-row tile of output
+  const int ncta = (a.M > kBM && a.force_ncta != 1) ? 2 : 1;
+  const int tile_m = kBM * ncta;
+  const uint32_t b_box_rows = ncta == 2 ? kBN / 2 : kBN;
   CUtensorMap map_a, map_b;
   // A is logically [M,K]; stored [M,K] (K-major) or, with transA, [K,M] (MN-major).
   int rc;
@@ -437,22 +572,22 @@ int launch_scaled_matmul(const MatmulArgs& a, void* ws, cudaStream_t st) {
   // B is logically [K,N]; stored [K,N] (MN-major) or, with transB, [N,K] (K-major).
   const int b_batched = a.b_bs != 0 ? 1 : 0;
   const int b_batch = b_batched ? a.batch : 1;
-  if (a.transB) rc = make_map(&map_b, a.B, a.K, a.N, b_batch, a.ldb, a.b_bs, kBN);
+  if (a.transB) rc = make_map(&map_b, a.B, a.K, a.N, b_batch, a.ldb, a.b_bs, b_box_rows);
   else rc = make_map(&map_b, a.B, a.N, a.K, b_batch, a.ldb, a.b_bs, kBK);
   if (rc) return rc;
 
   GemmParams p;
   p.M = a.M; p.N = a.N; p.K = a.K; p.batch = a.batch;
-  p.tiles_m = (a.M + kBM - 1) / kBM;
+  p.tiles_m = (a.M + tile_m - 1) / tile_m;
   p.tiles_n = (a.N + kBN - 1) / kBN;
   p.a_mn_major = a.transA ? 1 : 0;
   p.b_mn_major = a.transB ? 0 : 1;
   p.b_batched = b_batched;
   // instruction descriptor (kind::f8f6f4): D fp32, A/B formats (0 = E4M3, 1 = E5M2), operand
-  // majorness (0 = K-major), N >> 3, M >> 4
+  // majorness (0 = K-major), N >> 3, M >> 4 (M counts the rows of the whole CTA pair)
   p.idesc = (1u << 4) | (uint32_t(a.a_dt == SCALIFY_E5M2) << 7) | (uint32_t(a.b_dt == SCALIFY_E5M2) << 10) |
             (uint32_t(p.a_mn_major) << 15) | (uint32_t(p.b_mn_major) << 16) | (uint32_t(kBN >> 3) << 17) |
-            (uint32_t(kBM >> 4) << 24);
+            (uint32_t(tile_m >> 4) << 24);
   p.kf = kfactor(a.K);
   p.alpha = 1.0f / p.kf;
   p.Y = a.Y; p.ldy = a.ldy; p.y_batch_stride = a.y_bs;
@@ -463,19 +598,14 @@ int launch_scaled_matmul(const MatmulArgs& a, void* ws, cudaStream_t st) {
   p.status = v.status;
   const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n * p.batch;
   if (tiles > (1ll << 30)) return SCALIFY_ERR_SHAPE;
-  const int grid = static_cast<int>(tiles < sm_count() ? tiles : sm_count());
   if (a.stat == SCALIFY_STAT_AMAX) SCALIFY_CUDA_TRY(cudaMemsetAsync(v.stat, 0, sizeof(float), st));
-  if (!attr_done) {
-    SCALIFY_CUDA_TRY(cudaFuncSetAttribute(scaled_matmul_kernel<SCALIFY_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kGemmSmem)));
-    SCALIFY_CUDA_TRY(cudaFuncSetAttribute(scaled_matmul_kernel<SCALIFY_F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kGemmSmem)));
-    SCALIFY_CUDA_TRY(cudaFuncSetAttribute(scaled_matmul_kernel<SCALIFY_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kGemmSmem)));
-    attr_done = true;
-  }
-  SCALIFY_DISPATCH_WIDE(a.y_dt, OUT,
-      scaled_matmul_kernel<OUT><<<grid, kGemmThreads, kGemmSmem, st>>>(map_a, map_b, p));
-  SCALIFY_CUDA_TRY(cudaGetLastError());
+  SCALIFY_DISPATCH_WIDE(a.y_dt, OUT, {
+    if (ncta == 2) rc = launch_variant<OUT, 2>(map_a, map_b, p, tiles, st);
+    else rc = launch_variant<OUT, 1>(map_a, map_b, p, tiles, st);
+  });
+  if (rc) return rc;
   if (a.stat == SCALIFY_STAT_L2) {
-    gemm_l2_finalize_kernel<<<1, 256, 0, st>>>(p.l2_partials, static_cast<int>(tiles * 4),
+    gemm_l2_finalize_kernel<<<1, 256, 0, st>>>(p.l2_partials, static_cast<int>(tiles * ncta * 4),
                                                double(a.M) * double(a.N) * double(a.batch), v.stat);
     SCALIFY_CUDA_TRY(cudaGetLastError());
   }

@@ -430,6 +430,7 @@ int scalify_scaled_matmul(const scalify_array* A, int transA, const scalify_arra
   float* y_scale = Y->scale ? Y->scale : reinterpret_cast<float*>(static_cast<char*>(workspace) + 48);
   a.y_scale = y_scale;
   a.stat = stat;
+  a.force_ncta = 0;
   if (a.lda < (transA ? M : K) || a.ldb < (transB ? K : N) || a.ldy < N) return SCALIFY_ERR_SHAPE;
   rc = launch_scaled_matmul(a, workspace, st);
   if (rc) return rc;
