@@ -265,6 +265,34 @@ int scalify_scaled_adam_step(int n_tensors, const scalify_array* grads, scalify_
                              scalify_array* w, float lr, float beta1, float beta2, float eps, int64_t step,
                              void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * Scaled Adam step without a workspace.  (No counterpart in the paper: this entry point exists
+ * for the integration, not for the method.)
+ *
+ * Same operation, arguments and results as scalify_scaled_adam_step, for callers that cannot
+ * allocate the workspace that call needs: code running after the application's own memory
+ * pool has taken all device memory (a further cudaMalloc would fail), code on a path where
+ * the device-wide synchronisation of cudaMalloc is not acceptable, and integrations that are
+ * handed nothing but the tensors.  The scratch (old scale words and new reciprocals per
+ * tensor, and the status word) is a fixed 33 KB array inside the library image; every GPU
+ * that loads the library holds it until the process exits.  The call allocates nothing and
+ * frees nothing.
+ *
+ *   n_tensors   at most 1024; more returns SCALIFY_ERR_WORKSPACE and enqueues nothing.
+ *   status_out  optional DEVICE pointer to one uint32: receives the SCALIFY_DEV_* bits of this
+ *               call (0 if none), written in stream order.  May be NULL.
+ *
+ * The first call on each device looks up the array's device address (with that device
+ * current); make that first call before starting any stream capture.  All calls on a device
+ * share the one array, which keeps the previous call's contents (the call clears what it
+ * needs to start from zero): two calls that may overlap on the GPU - different streams
+ * without an ordering between them - race on it; order them or use
+ * scalify_scaled_adam_step with separate workspaces.
+ */
+int scalify_scaled_adam_step_static(int n_tensors, const scalify_array* grads, scalify_array* m, scalify_array* v,
+                                    scalify_array* w, float lr, float beta1, float beta2, float eps, int64_t step,
+                                    uint32_t* status_out, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -74,10 +74,11 @@ def lib() -> ctypes.CDLL:
         L.scalify_scaled_gelu.argtypes = [P, i32, P, vp]
         L.scalify_scaled_gelu_bwd.argtypes = [P, P, i32, P, vp]
         L.scalify_scaled_adam_step.argtypes = [i32, P, P, P, P, f32, f32, f32, f32, i64, vp, sz, vp]
+        L.scalify_scaled_adam_step_static.argtypes = [i32, P, P, P, P, f32, f32, f32, f32, i64, vp, vp]
         for name in ("scalify_workspace_init", "scalify_check_status", "scalify_scaled_matmul", "scalify_statistic",
                      "scalify_rescale", "scalify_scaled_add", "scalify_scaled_layernorm",
                      "scalify_scaled_layernorm_bwd", "scalify_scaled_gelu", "scalify_scaled_gelu_bwd",
-                     "scalify_scaled_adam_step"):
+                     "scalify_scaled_adam_step", "scalify_scaled_adam_step_static"):
             getattr(L, name).restype = i32
         _lib = L
     return _lib
@@ -256,3 +257,16 @@ def scalify_scaled_adam_step(tensors: AdamTensors, ws: Workspace, *, lr: float, 
     _check(lib().scalify_scaled_adam_step(tensors.n, tensors.g, tensors.m, tensors.v, tensors.w, float(lr),
                                           float(beta1), float(beta2), float(eps), int(step), ws.ptr, ws.nbytes,
                                           _stream(stream)), "scalify_scaled_adam_step")
+
+
+def scalify_scaled_adam_step_static(tensors: AdamTensors, *, lr: float, beta1: float, beta2: float, eps: float,
+                                    step: int, status_out: Optional[torch.Tensor] = None, stream=None) -> None:
+    """Adam step for callers that cannot allocate a workspace (their memory pool already owns the device,
+    or they must not trigger cudaMalloc's synchronisation): the scratch is a fixed array inside the library.
+    At most 1024 tensors.  `status_out`: optional 1-element int32/uint32 CUDA tensor that receives the device
+    status bits.  Calls on one device share that array: do not let two of them overlap on the GPU, and make
+    the first call on a device outside stream capture."""
+    _check(lib().scalify_scaled_adam_step_static(tensors.n, tensors.g, tensors.m, tensors.v, tensors.w, float(lr),
+                                                 float(beta1), float(beta2), float(eps), int(step),
+                                                 _ptr(status_out), _stream(stream)),
+           "scalify_scaled_adam_step_static")
