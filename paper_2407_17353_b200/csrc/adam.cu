@@ -41,10 +41,17 @@ struct AdamScalePtrs {
   int count;
 };
 
-// per tensor, in the workspace: old scales and reciprocals of the new ones
+// per tensor, in the workspace: the old scales folded with the step's constants, and the
+// reciprocals of the new scales (all scale factors are powers of two, so folding them is exact)
 struct AdamFactors {
-  float g_s, m_s, v_s, w_s;
-  float inv_m2, inv_v2, inv_w2, pad;
+  float cm;      // b1 * m_s            m' = cm*m_d + cg*g_d          (value space)
+  float cg;      // (1-b1) * g_s
+  float cv;      // b2 * v_s            v' = cv*v_d + cg2*g_d^2
+  float cg2;     // (1-b2) * g_s^2
+  float inv_m2;  // 1 / m'_s
+  float inv_v2;  // 1 / v'_s
+  float cw;      // w_s / w'_s          w'_d = cw*w_d - cu * m' / (sqrt(v'/bc2) + eps)
+  float cu;      // lr / bc1 / w'_s
 };
 
 struct AdamHyper {
@@ -67,12 +74,33 @@ __global__ void adam_scales_kernel(AdamScalePtrs sp, AdamHyper h, AdamFactors* _
   const float us = h.p_lr * (ms2 / h.p_bc1) / den;
   const float ws2 = fmaxf(ws, us);
   AdamFactors f;
-  f.g_s = gs; f.m_s = ms; f.v_s = vs; f.w_s = ws;
-  f.inv_m2 = 1.0f / ms2; f.inv_v2 = 1.0f / vs2; f.inv_w2 = 1.0f / ws2; f.pad = 0.f;
+  f.cm = h.b1 * ms;
+  f.cg = h.one_m_b1 * gs;
+  f.cv = h.b2 * vs;
+  f.cg2 = h.one_m_b2 * gs * gs;
+  f.inv_m2 = 1.0f / ms2;
+  f.inv_v2 = 1.0f / vs2;
+  f.cw = ws / ws2;
+  f.cu = h.lr * h.inv_bc1 / ws2;
   fac[i] = f;
   *sp.m[i] = ms2;
   *sp.v[i] = vs2;
   *sp.w[i] = ws2;
+}
+
+// One element.  sqrt and the division use the hardware approximations (each within 2 ulp of fp32),
+// far below the resolution of the FP16 / BF16 outputs and of the fp32 weight, whose update is a
+// small correction; the kernel is otherwise limited by instruction issue, not by HBM.
+__device__ __forceinline__ void adam_elem(float g, float& m, float& v, float& w, const AdamFactors& f,
+                                          const AdamHyper& h) {
+  const float m2 = fmaf(f.cm, m, f.cg * g);
+  const float v2 = fmaf(f.cv, v, f.cg2 * (g * g));
+  float root;
+  asm("sqrt.approx.f32 %0, %1;" : "=f"(root) : "f"(v2 * h.inv_bc2));
+  const float upd = f.cu * __fdividef(m2, root + h.eps);
+  w = fmaf(f.cw, w, -upd);
+  m = m2 * f.inv_m2;
+  v = v2 * f.inv_v2;
 }
 
 template <int GDT, int MVDT, int WDT>
@@ -84,17 +112,7 @@ __device__ __forceinline__ void adam_vec(const uint32_t* wg, uint32_t* wm, uint3
   decode_vec<MVDT, kAdamVec>(wv, v);
   decode_vec<WDT, kAdamVec>(ww, w);
 #pragma unroll
-  for (int e = 0; e < kAdamVec; ++e) {
-    const float gv = g[e] * f.g_s;
-    const float m2 = fmaf(h.b1, m[e] * f.m_s, h.one_m_b1 * gv);
-    const float v2 = fmaf(h.b2, v[e] * f.v_s, h.one_m_b2 * gv * gv);
-    const float mhat = m2 * h.inv_bc1;
-    const float vhat = v2 * h.inv_bc2;
-    const float w2 = w[e] * f.w_s - h.lr * mhat / (sqrtf(vhat) + h.eps);
-    m[e] = m2 * f.inv_m2;
-    v[e] = v2 * f.inv_v2;
-    w[e] = w2 * f.inv_w2;
-  }
+  for (int e = 0; e < kAdamVec; ++e) adam_elem(g[e], m[e], v[e], w[e], f, h);
   encode_vec<MVDT, kAdamVec>(m, wm);
   encode_vec<MVDT, kAdamVec>(v, wv);
   encode_vec<WDT, kAdamVec>(w, ww);
@@ -148,14 +166,11 @@ __global__ void __launch_bounds__(kAdamThreads) adam_update_kernel(const __grid_
     if (chunk == tab.chunk_start[ti + 1] - 1) {
       const long long i = n_vec * kAdamVec + threadIdx.x;
       if (i < n) {
-        const float gv = load_elem<GDT>(gp, i) * f.g_s;
-        const float m2 = fmaf(h.b1, load_elem<MVDT>(mp, i) * f.m_s, h.one_m_b1 * gv);
-        const float v2 = fmaf(h.b2, load_elem<MVDT>(vp, i) * f.v_s, h.one_m_b2 * gv * gv);
-        const float w2 = load_elem<WDT>(wp, i) * f.w_s -
-                         h.lr * (m2 * h.inv_bc1) / (sqrtf(v2 * h.inv_bc2) + h.eps);
-        store_elem<MVDT>(mp, i, m2 * f.inv_m2);
-        store_elem<MVDT>(vp, i, v2 * f.inv_v2);
-        store_elem<WDT>(wp, i, w2 * f.inv_w2);
+        float mm = load_elem<MVDT>(mp, i), vv = load_elem<MVDT>(vp, i), ww = load_elem<WDT>(wp, i);
+        adam_elem(load_elem<GDT>(gp, i), mm, vv, ww, f, h);
+        store_elem<MVDT>(mp, i, mm);
+        store_elem<MVDT>(vp, i, vv);
+        store_elem<WDT>(wp, i, ww);
       }
     }
   }

@@ -167,8 +167,12 @@ __global__ void __launch_bounds__(kThreads) rebalance_kernel(const void* __restr
     out_scale = ns;
   }
   const int64_t n_vec = n / VEC;
-  const int64_t stride = int64_t(gridDim.x) * kThreads * kUnroll;
-  for (int64_t base = int64_t(blockIdx.x) * kThreads * kUnroll; base < n_vec; base += stride) {
+  const int64_t n_tiles = (n_vec + kThreads * kUnroll - 1) / (kThreads * kUnroll);
+  // A dynamic rescale runs right after the kernel that produced (or measured) the data, whose most
+  // recently touched part - the end of the array - is still in L2: walk the array from the end.
+  const bool reverse = (mode == kModeDynamic);
+  for (int64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+    const int64_t base = (reverse ? n_tiles - 1 - tile : tile) * (kThreads * kUnroll);
     uint32_t w[kUnroll][IB / 4];
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {

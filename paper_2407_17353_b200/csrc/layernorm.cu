@@ -1,30 +1,42 @@
 // Scaled LayerNorm forward and backward (Section 3.2.1, Appendix C.2, Algorithm 5).
 //
-// HBM-bound: every element of X (and G) is read once and every output written once.  A row
-// is owned by a team of WARPS warps; each thread keeps up to kMaxVpt 16-byte vectors of the
-// row in registers, so mean, variance and the normalised values come from one read.  gamma
-// and beta are re-read per row through L1 (they are a few KB).  Blocks stride over rows with
-// a grid that is a multiple of the SM count.
+// HBM-bound: every element of X (and G) is read once and every output written once.  A row is
+// owned by a team of TW warps (TW = 1, 2, 4 or 8, chosen so that a thread holds at most two
+// 16-byte vectors of the row); the row stays in registers, so mean, variance and the normalised
+// values come from one read.  Blocks of 256 threads hold 8/TW teams and stride over the rows with
+// a grid that is a multiple of the SM count.  The raw words of a team's NEXT row are fetched
+// before the current row is processed, which doubles the bytes in flight per thread.  gamma and
+// beta for a thread's fixed columns are converted once and kept in registers.
 #include "scalify_common.cuh"
 #include "scalify_launch.h"
 
 namespace scalify {
 
-constexpr int kLnThreads = 128;  // 4 warps per block
-constexpr int kMaxVpt = 4;       // 16-byte vectors per thread and row
+constexpr int kLnThreads = 256;
+constexpr int kLnVpt = 2;  // 16-byte vectors per thread and row
 
-template <int WARPS>
-__device__ __forceinline__ void team_sum2(float& a, float& b, float* smem) {
+template <int TW>
+__device__ __forceinline__ void team_barrier(int team) {
+  if constexpr (TW == 8) __syncthreads();
+  else if constexpr (TW > 1) asm volatile("bar.sync %0, %1;" ::"r"(team + 1), "r"(TW * 32) : "memory");
+}
+
+// Sum of (a, b) over the team.  `buf` alternates between two shared arrays from call to call, so a
+// single barrier per call is enough (a warp can only overwrite an array after every warp of the
+// team has passed the barrier of the following call, i.e. after they have read it).
+template <int TW>
+__device__ __forceinline__ void team_sum2(float& a, float& b, float (*smem)[8][2], int team, int& buf) {
   a = warp_sum_f32(a);
   b = warp_sum_f32(b);
-  if constexpr (WARPS > 1) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    __syncthreads();  // previous use of smem is over
-    if (lane == 0) { smem[2 * warp] = a; smem[2 * warp + 1] = b; }
-    __syncthreads();
+  if constexpr (TW > 1) {
+    const int lane = threadIdx.x & 31, wit = (threadIdx.x >> 5) % TW;
+    float(*s)[2] = smem[buf] + team * TW;
+    if (lane == 0) { s[wit][0] = a; s[wit][1] = b; }
+    team_barrier<TW>(team);
     a = 0.f; b = 0.f;
 #pragma unroll
-    for (int w = 0; w < WARPS; ++w) { a += smem[2 * w]; b += smem[2 * w + 1]; }
+    for (int w = 0; w < TW; ++w) { a += s[w][0]; b += s[w][1]; }
+    buf ^= 1;
   }
 }
 
@@ -46,7 +58,7 @@ __device__ __forceinline__ void load_param_vec(const void* p, int dt, int c, flo
 // ---------------------------------------------------------------------------------------------
 // forward
 // ---------------------------------------------------------------------------------------------
-template <int XDT, int YDT, int WARPS>
+template <int XDT, int YDT, int TW>
 __global__ void __launch_bounds__(kLnThreads) layernorm_fwd_kernel(
     const void* __restrict__ X, int64_t x_ld, void* __restrict__ Y, int64_t y_ld, int R, int d,
     const void* __restrict__ gamma, const void* __restrict__ beta, int gb_dt, const float* gamma_scale,
@@ -54,9 +66,9 @@ __global__ void __launch_bounds__(kLnThreads) layernorm_fwd_kernel(
     float* __restrict__ rinv_out) {
   constexpr int VEC = 16 / ElemBytes<XDT>::v;
   constexpr int OB = VEC * ElemBytes<YDT>::v;
-  constexpr int TEAM = 32 * WARPS;
-  constexpr int TEAMS_PER_BLOCK = kLnThreads / TEAM;
-  __shared__ float smem[2 * (kLnThreads / 32)];
+  constexpr int TEAM = 32 * TW;
+  constexpr int TPB = kLnThreads / TEAM;  // teams per block
+  __shared__ float smem[2][8][2];
   const int n_vec = d / VEC;
   const int t = threadIdx.x % TEAM;
   const int team = threadIdx.x / TEAM;
@@ -67,39 +79,63 @@ __global__ void __launch_bounds__(kLnThreads) layernorm_fwd_kernel(
     fg = gs / ys;
     fb = bs / ys;
   }
-  const float inv_d = 1.0f / static_cast<float>(d);
-  const int rows_per_iter = gridDim.x * TEAMS_PER_BLOCK;
-  const int iters = (R + rows_per_iter - 1) / rows_per_iter;
-  for (int it = 0; it < iters; ++it) {
-    const int row = it * rows_per_iter + blockIdx.x * TEAMS_PER_BLOCK + team;
-    const bool live = row < R;
-    float x[kMaxVpt][VEC];
-    const char* xrow = static_cast<const char*>(X) + int64_t(live ? row : 0) * x_ld * ElemBytes<XDT>::v;
+  // this thread's columns: vectors t and t + TEAM
+  bool has[kLnVpt];
+  float gam[kLnVpt][VEC], bet[kLnVpt][VEC];
 #pragma unroll
-    for (int v = 0; v < kMaxVpt; ++v) {
-      const int vi = t + v * TEAM;
-      uint32_t w[4] = {0u, 0u, 0u, 0u};
-      if (live && vi < n_vec) ld_raw_stream<16>(xrow + int64_t(vi) * 16, w);
-      decode_vec<XDT, VEC>(w, x[v]);
+  for (int v = 0; v < kLnVpt; ++v) {
+    const int vi = t + v * TEAM;
+    has[v] = vi < n_vec;
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) { gam[v][e] = 1.0f; bet[v][e] = 0.0f; }
+    if (has[v] && gamma) {
+      load_param_vec<VEC>(gamma, gb_dt, vi * VEC, gam[v]);
+      if (beta) {
+        load_param_vec<VEC>(beta, gb_dt, vi * VEC, bet[v]);
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) bet[v][e] *= fb;  // exact: fb is a power of two
+      }
     }
+  }
+  const float inv_d = 1.0f / static_cast<float>(d);
+  const int rows_per_iter = gridDim.x * TPB;
+  const int iters = (R + rows_per_iter - 1) / rows_per_iter;
+  int buf = 0;
+  uint32_t nxt[kLnVpt][4];
+  auto fetch = [&](int row) {
+#pragma unroll
+    for (int v = 0; v < kLnVpt; ++v) {
+      nxt[v][0] = nxt[v][1] = nxt[v][2] = nxt[v][3] = 0u;
+      if (has[v] && row < R)
+        ld_raw_stream<16>(static_cast<const char*>(X) + (int64_t(row) * x_ld) * ElemBytes<XDT>::v +
+                              int64_t(t + v * TEAM) * 16, nxt[v]);
+    }
+  };
+  fetch(blockIdx.x * TPB + team);
+  for (int it = 0; it < iters; ++it) {
+    const int row = it * rows_per_iter + blockIdx.x * TPB + team;
+    const bool live = row < R;
+    float x[kLnVpt][VEC];
+#pragma unroll
+    for (int v = 0; v < kLnVpt; ++v) decode_vec<XDT, VEC>(nxt[v], x[v]);
+    fetch(row + rows_per_iter);  // raw words of this team's next row
     float s = 0.f, dummy = 0.f;
 #pragma unroll
-    for (int v = 0; v < kMaxVpt; ++v)
+    for (int v = 0; v < kLnVpt; ++v)
 #pragma unroll
-      for (int e = 0; e < VEC; ++e) s += x[v][e];
-    team_sum2<WARPS>(s, dummy, smem);
+      for (int e = 0; e < VEC; ++e) s += x[v][e];  // absent vectors hold zeros
+    team_sum2<TW>(s, dummy, smem, team, buf);
     const float mu = s * inv_d;
     float q = 0.f;
     dummy = 0.f;
 #pragma unroll
-    for (int v = 0; v < kMaxVpt; ++v) {
-      const int vi = t + v * TEAM;
-      if (vi < n_vec) {
+    for (int v = 0; v < kLnVpt; ++v) {
+      if (has[v]) {
 #pragma unroll
-        for (int e = 0; e < VEC; ++e) { float c = x[v][e] - mu; q = fmaf(c, c, q); }
+        for (int e = 0; e < VEC; ++e) { x[v][e] -= mu; q = fmaf(x[v][e], x[v][e], q); }
       }
     }
-    team_sum2<WARPS>(q, dummy, smem);
+    team_sum2<TW>(q, dummy, smem, team, buf);
     const float var = q * inv_d;
     const float rinv = eps_inside ? 1.0f / sqrtf(var + eps) : 1.0f / (sqrtf(var) + eps);
     if (live) {
@@ -107,28 +143,17 @@ __global__ void __launch_bounds__(kLnThreads) layernorm_fwd_kernel(
         if (mean_out) mean_out[row] = mu;
         if (rinv_out) rinv_out[row] = rinv;
       }
+      const float rg = rinv * fg;  // exact: fg is a power of two
       char* yrow = static_cast<char*>(Y) + int64_t(row) * y_ld * ElemBytes<YDT>::v;
 #pragma unroll
-      for (int v = 0; v < kMaxVpt; ++v) {
-        const int vi = t + v * TEAM;
-        if (vi < n_vec) {
+      for (int v = 0; v < kLnVpt; ++v) {
+        if (has[v]) {
           float o[VEC];
 #pragma unroll
-          for (int e = 0; e < VEC; ++e) o[e] = (x[v][e] - mu) * rinv;
-          if (gamma) {
-            float g[VEC];
-            load_param_vec<VEC>(gamma, gb_dt, vi * VEC, g);
-#pragma unroll
-            for (int e = 0; e < VEC; ++e) o[e] = o[e] * g[e] * fg;
-            if (beta) {
-              load_param_vec<VEC>(beta, gb_dt, vi * VEC, g);
-#pragma unroll
-              for (int e = 0; e < VEC; ++e) o[e] = fmaf(g[e], fb, o[e]);
-            }
-          }
+          for (int e = 0; e < VEC; ++e) o[e] = fmaf(x[v][e] * rg, gam[v][e], bet[v][e]);
           uint32_t ow[OB / 4];
           encode_vec<YDT, VEC>(o, ow);
-          st_raw<OB>(yrow + int64_t(vi) * OB, ow);
+          st_raw<OB>(yrow + int64_t(t + v * TEAM) * OB, ow);
         }
       }
     }
@@ -136,18 +161,18 @@ __global__ void __launch_bounds__(kLnThreads) layernorm_fwd_kernel(
   if (blockIdx.x == 0 && threadIdx.x == 0 && y_scale) *y_scale = ys;
 }
 
-int ln_grid(int R, int teams_per_block, int blocks_per_sm) {
+static int ln_grid(int R, int teams_per_block, int blocks_per_sm) {
   int64_t need = (int64_t(R) + teams_per_block - 1) / teams_per_block;
   int64_t cap = int64_t(sm_count()) * blocks_per_sm;
   if (need < 1) need = 1;
   return static_cast<int>(need < cap ? need : cap);
 }
 
-// chooses the team width; returns 0 if the row is too long for the register budget
-static int ln_warps(int d, int x_dt) {
-  int n_vec = d * elem_size(x_dt) / 16;
-  if (n_vec <= 32 * kMaxVpt) return 1;
-  if (n_vec <= 128 * kMaxVpt) return 4;
+// team width in warps so that a thread holds at most kLnVpt vectors; 0 if the row is too long
+static int ln_team_warps(int d, int x_dt) {
+  const int n_vec = d * elem_size(x_dt) / 16;
+  for (int tw = 1; tw <= 8; tw *= 2)
+    if (n_vec <= 32 * tw * kLnVpt) return tw;
   return 0;
 }
 
@@ -155,15 +180,20 @@ int launch_layernorm_fwd(const void* X, int x_dt, int64_t x_ld, void* Y, int y_d
                          const void* gamma, const void* beta, int gb_dt, const float* gamma_scale,
                          const float* beta_scale, float* y_scale, float eps, int eps_inside, float* mean,
                          float* rinv, cudaStream_t st) {
-  const int warps = ln_warps(d, x_dt);
-  if (warps == 0) return SCALIFY_ERR_UNSUPPORTED;
-  const int grid = ln_grid(R, 4 / warps, 12);
+  const int tw = ln_team_warps(d, x_dt);
+  if (tw == 0) return SCALIFY_ERR_UNSUPPORTED;
+  const int grid = ln_grid(R, 8 / tw, 3);
 #define SCALIFY_LN_FWD(W)                                                                                      \
   layernorm_fwd_kernel<XDT, YDT, W><<<grid, kLnThreads, 0, st>>>(X, x_ld, Y, y_ld, R, d, gamma, beta, gb_dt,    \
                                                                  gamma_scale, beta_scale, y_scale, eps,         \
                                                                  eps_inside, mean, rinv)
   SCALIFY_DISPATCH_WIDE(x_dt, XDT, SCALIFY_DISPATCH_DTYPE(y_dt, YDT, {
-    if (warps == 1) SCALIFY_LN_FWD(1); else SCALIFY_LN_FWD(4);
+    switch (tw) {
+      case 1: SCALIFY_LN_FWD(1); break;
+      case 2: SCALIFY_LN_FWD(2); break;
+      case 4: SCALIFY_LN_FWD(4); break;
+      default: SCALIFY_LN_FWD(8); break;
+    }
   }));
 #undef SCALIFY_LN_FWD
   SCALIFY_CUDA_TRY(cudaGetLastError());
@@ -175,69 +205,73 @@ int launch_layernorm_fwd(const void* X, int x_dt, int64_t x_ld, void* Y, int y_d
 // ---------------------------------------------------------------------------------------------
 // ws layout (after the header): float dgamma_part[grid][d]; float dbeta_part[grid][d];
 // double stat_part[grid].
-template <int WARPS> struct BwdCfg {
-  static constexpr int threads = WARPS == 1 ? 256 : 128;  // WARPS == 1: eight one-warp teams per block
-  static constexpr int min_blocks = WARPS == 1 ? 2 : 3;
-};
-
-template <int XDT, int DXDT, int WARPS>
-__global__ void __launch_bounds__(BwdCfg<WARPS>::threads, BwdCfg<WARPS>::min_blocks) layernorm_bwd_kernel(
+template <int XDT, int DXDT, int TW>
+__global__ void __launch_bounds__(kLnThreads, 2) layernorm_bwd_kernel(
     const void* __restrict__ G, int64_t g_ld, const void* __restrict__ X, int64_t x_ld, void* __restrict__ dX,
     int64_t dx_ld, int R, int d, const void* __restrict__ gamma, int gb_dt, const float* __restrict__ mean,
     const float* __restrict__ rinv_in, float eps, int eps_inside, int stat, float* __restrict__ dgamma_part,
     float* __restrict__ dbeta_part, double* __restrict__ stat_part) {
   constexpr int VEC = 16 / ElemBytes<XDT>::v;
   constexpr int OB = VEC * ElemBytes<DXDT>::v;
-  constexpr int TEAM = 32 * WARPS;
-  constexpr int THREADS = BwdCfg<WARPS>::threads;
-  constexpr int TEAMS_PER_BLOCK = THREADS / TEAM;
-  __shared__ float smem[2 * (THREADS / 32)];
+  constexpr int TEAM = 32 * TW;
+  constexpr int TPB = kLnThreads / TEAM;
+  __shared__ float smem[2][8][2];
   const int n_vec = d / VEC;
   const int t = threadIdx.x % TEAM;
   const int team = threadIdx.x / TEAM;
   const float inv_d = 1.0f / static_cast<float>(d);
-  float acc_dg[kMaxVpt][VEC], acc_db[kMaxVpt][VEC];
+  bool has[kLnVpt];
+  float gam[kLnVpt][VEC], acc_dg[kLnVpt][VEC], acc_db[kLnVpt][VEC];
 #pragma unroll
-  for (int v = 0; v < kMaxVpt; ++v)
+  for (int v = 0; v < kLnVpt; ++v) {
+    has[v] = (t + v * TEAM) < n_vec;
 #pragma unroll
-    for (int e = 0; e < VEC; ++e) { acc_dg[v][e] = 0.f; acc_db[v][e] = 0.f; }
+    for (int e = 0; e < VEC; ++e) { gam[v][e] = 1.0f; acc_dg[v][e] = 0.f; acc_db[v][e] = 0.f; }
+    if (has[v] && gamma) load_param_vec<VEC>(gamma, gb_dt, (t + v * TEAM) * VEC, gam[v]);
+  }
   uint32_t amax = 0u;
   float ssq = 0.f;
-  const int rows_per_iter = gridDim.x * TEAMS_PER_BLOCK;
+  const int rows_per_iter = gridDim.x * TPB;
   const int iters = (R + rows_per_iter - 1) / rows_per_iter;
-  for (int it = 0; it < iters; ++it) {
-    const int row = it * rows_per_iter + blockIdx.x * TEAMS_PER_BLOCK + team;
-    const bool live = row < R;
-    const int srow = live ? row : 0;
-    float x[kMaxVpt][VEC], g[kMaxVpt][VEC];
-    const char* xrow = static_cast<const char*>(X) + int64_t(srow) * x_ld * ElemBytes<XDT>::v;
-    const char* grow = static_cast<const char*>(G) + int64_t(srow) * g_ld * ElemBytes<XDT>::v;
+  int buf = 0;
+  uint32_t nx[kLnVpt][4], ng[kLnVpt][4];
+  float nmu = 0.f, nrinv = 0.f;
+  auto fetch = [&](int row) {
 #pragma unroll
-    for (int v = 0; v < kMaxVpt; ++v) {
-      const int vi = t + v * TEAM;
-      uint32_t wx[4] = {0u, 0u, 0u, 0u}, wg[4] = {0u, 0u, 0u, 0u};
-      if (live && vi < n_vec) {
-        ld_raw_stream<16>(xrow + int64_t(vi) * 16, wx);
-        ld_raw_stream<16>(grow + int64_t(vi) * 16, wg);
+    for (int v = 0; v < kLnVpt; ++v) {
+      nx[v][0] = nx[v][1] = nx[v][2] = nx[v][3] = 0u;
+      ng[v][0] = ng[v][1] = ng[v][2] = ng[v][3] = 0u;
+      if (has[v] && row < R) {
+        ld_raw_stream<16>(static_cast<const char*>(X) + (int64_t(row) * x_ld) * ElemBytes<XDT>::v +
+                              int64_t(t + v * TEAM) * 16, nx[v]);
+        ld_raw_stream<16>(static_cast<const char*>(G) + (int64_t(row) * g_ld) * ElemBytes<XDT>::v +
+                              int64_t(t + v * TEAM) * 16, ng[v]);
       }
-      decode_vec<XDT, VEC>(wx, x[v]);
-      decode_vec<XDT, VEC>(wg, g[v]);
     }
-    const float mu = __ldg(&mean[srow]);
-    const float rinv = __ldg(&rinv_in[srow]);
+    if (row < R) { nmu = __ldg(&mean[row]); nrinv = __ldg(&rinv_in[row]); }
+  };
+  fetch(blockIdx.x * TPB + team);
+  for (int it = 0; it < iters; ++it) {
+    const int row = it * rows_per_iter + blockIdx.x * TPB + team;
+    const bool live = row < R;
+    float x[kLnVpt][VEC], g[kLnVpt][VEC];
+#pragma unroll
+    for (int v = 0; v < kLnVpt; ++v) {
+      decode_vec<XDT, VEC>(nx[v], x[v]);
+      decode_vec<XDT, VEC>(ng[v], g[v]);
+    }
+    const float mu = nmu, rinv = nrinv;
+    fetch(row + rows_per_iter);
     float m1 = 0.f, m2 = 0.f;
 #pragma unroll
-    for (int v = 0; v < kMaxVpt; ++v) {
-      const int vi = t + v * TEAM;
-      if (live && vi < n_vec) {
-        float gam[VEC];
-        if (gamma) load_param_vec<VEC>(gamma, gb_dt, vi * VEC, gam);
+    for (int v = 0; v < kLnVpt; ++v) {
+      if (has[v] && live) {
 #pragma unroll
         for (int e = 0; e < VEC; ++e) {
           const float n = (x[v][e] - mu) * rinv;
           acc_dg[v][e] = fmaf(g[v][e], n, acc_dg[v][e]);
           acc_db[v][e] += g[v][e];
-          const float gh = gamma ? g[v][e] * gam[e] : g[v][e];
+          const float gh = g[v][e] * gam[v][e];
           x[v][e] = n;   // keep n
           g[v][e] = gh;  // keep ghat
           m1 += gh;
@@ -245,7 +279,7 @@ __global__ void __launch_bounds__(BwdCfg<WARPS>::threads, BwdCfg<WARPS>::min_blo
         }
       }
     }
-    team_sum2<WARPS>(m1, m2, smem);
+    team_sum2<TW>(m1, m2, smem, team, buf);
     m1 *= inv_d;
     m2 *= inv_d;
     // eps outside the root: dx = (ghat-m1)*rinv - n*m2/s with s = 1/rinv - eps (0 if s == 0)
@@ -260,9 +294,8 @@ __global__ void __launch_bounds__(BwdCfg<WARPS>::threads, BwdCfg<WARPS>::min_blo
     if (live) {
       char* orow = static_cast<char*>(dX) + int64_t(row) * dx_ld * ElemBytes<DXDT>::v;
 #pragma unroll
-      for (int v = 0; v < kMaxVpt; ++v) {
-        const int vi = t + v * TEAM;
-        if (vi < n_vec) {
+      for (int v = 0; v < kLnVpt; ++v) {
+        if (has[v]) {
           float o[VEC];
 #pragma unroll
           for (int e = 0; e < VEC; ++e) {
@@ -273,32 +306,30 @@ __global__ void __launch_bounds__(BwdCfg<WARPS>::threads, BwdCfg<WARPS>::min_blo
           }
           uint32_t ow[OB / 4];
           encode_vec<DXDT, VEC>(o, ow);
-          st_raw<OB>(orow + int64_t(vi) * OB, ow);
+          st_raw<OB>(orow + int64_t(t + v * TEAM) * OB, ow);
         }
       }
     }
   }
-  // per-block column partials of dgamma / dbeta
+  // per-block column partials of dgamma / dbeta: teams of a block own the same columns
   if (dgamma_part) {
-    if constexpr (WARPS == 1) {
-      // the teams of a block own the same columns: combine them through shared memory in team order
-      __shared__ float s_col[TEAMS_PER_BLOCK][32][VEC + 1];
+    if constexpr (TPB > 1) {
+      __shared__ float s_col[TPB][TEAM][VEC + 1];
 #pragma unroll
       for (int pass = 0; pass < 2; ++pass) {
 #pragma unroll
-        for (int v = 0; v < kMaxVpt; ++v) {
-          const int vi = t + v * TEAM;
+        for (int v = 0; v < kLnVpt; ++v) {
           __syncthreads();
 #pragma unroll
           for (int e = 0; e < VEC; ++e) s_col[team][t][e] = pass ? acc_db[v][e] : acc_dg[v][e];
           __syncthreads();
-          if (team == 0 && vi < n_vec) {
-            float* dst = (pass ? dbeta_part : dgamma_part) + int64_t(blockIdx.x) * d + vi * VEC;
+          if (team == 0 && has[v]) {
+            float* dst = (pass ? dbeta_part : dgamma_part) + int64_t(blockIdx.x) * d + (t + v * TEAM) * VEC;
 #pragma unroll
             for (int e = 0; e < VEC; ++e) {
               float sum = s_col[0][t][e];
 #pragma unroll
-              for (int tm = 1; tm < TEAMS_PER_BLOCK; ++tm) sum += s_col[tm][t][e];
+              for (int tm = 1; tm < TPB; ++tm) sum += s_col[tm][t][e];
               dst[e] = sum;
             }
           }
@@ -306,11 +337,10 @@ __global__ void __launch_bounds__(BwdCfg<WARPS>::threads, BwdCfg<WARPS>::min_blo
       }
     } else {
 #pragma unroll
-      for (int v = 0; v < kMaxVpt; ++v) {
-        const int vi = t + v * TEAM;
-        if (vi < n_vec) {
-          float* dg = dgamma_part + int64_t(blockIdx.x) * d + vi * VEC;
-          float* db = dbeta_part + int64_t(blockIdx.x) * d + vi * VEC;
+      for (int v = 0; v < kLnVpt; ++v) {
+        if (has[v]) {
+          float* dg = dgamma_part + int64_t(blockIdx.x) * d + (t + v * TEAM) * VEC;
+          float* db = dbeta_part + int64_t(blockIdx.x) * d + (t + v * TEAM) * VEC;
 #pragma unroll
           for (int e = 0; e < VEC; ++e) { dg[e] = acc_dg[v][e]; db[e] = acc_db[v][e]; }
         }
@@ -318,7 +348,7 @@ __global__ void __launch_bounds__(BwdCfg<WARPS>::threads, BwdCfg<WARPS>::min_blo
     }
   }
   if (stat != SCALIFY_STAT_NONE) {
-    __shared__ double s_stat[THREADS / 32];
+    __shared__ double s_stat[kLnThreads / 32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     double mine = (stat == SCALIFY_STAT_AMAX) ? static_cast<double>(warp_max_u32(amax))
                                               : warp_sum_f64(static_cast<double>(ssq));
@@ -326,7 +356,7 @@ __global__ void __launch_bounds__(BwdCfg<WARPS>::threads, BwdCfg<WARPS>::min_blo
     __syncthreads();
     if (threadIdx.x == 0) {
       double tot = s_stat[0];
-      for (int i = 1; i < THREADS / 32; ++i)
+      for (int i = 1; i < kLnThreads / 32; ++i)
         tot = (stat == SCALIFY_STAT_AMAX) ? fmax(tot, s_stat[i]) : tot + s_stat[i];
       stat_part[blockIdx.x] = tot;
     }
@@ -393,8 +423,10 @@ __global__ void __launch_bounds__(256) layernorm_bwd_finalize_kernel(
   }
 }
 
+constexpr int kLnBwdBlocksPerSm = 2;
+
 size_t layernorm_bwd_ws_bytes(int64_t R, int64_t d) {
-  int64_t grid = int64_t(sm_count()) * 3;
+  int64_t grid = int64_t(sm_count()) * kLnBwdBlocksPerSm;
   (void)R;
   return kWsHeader + size_t(grid) * size_t(d) * 8 + size_t(grid) * 8 + 256;
 }
@@ -404,21 +436,26 @@ int launch_layernorm_bwd(const void* G, int64_t g_ld, const void* X, int x_dt, i
                          const float* rinv, float eps, int eps_inside, int stat, void* dgamma, void* dbeta, int dg_dt,
                          const float* g_scale, const float* x_scale, const float* gamma_scale, float* dx_scale,
                          float* dgamma_scale, float* dbeta_scale, void* ws, cudaStream_t st) {
-  const int warps = ln_warps(d, x_dt);
-  if (warps == 0) return SCALIFY_ERR_UNSUPPORTED;
-  const int grid = (warps == 1) ? ln_grid(R, 8, 2) : ln_grid(R, 1, 3);
+  const int tw = ln_team_warps(d, x_dt);
+  if (tw == 0) return SCALIFY_ERR_UNSUPPORTED;
+  const int grid = ln_grid(R, 8 / tw, kLnBwdBlocksPerSm);
   WsView v = ws_view(ws);
   float* dg_part = static_cast<float*>(v.area);
   float* db_part = dg_part + size_t(grid) * d;
   double* st_part = reinterpret_cast<double*>(db_part + size_t(grid) * d);
   float* dgp = dgamma ? dg_part : nullptr;
   float* dbp = dgamma ? db_part : nullptr;
-#define SCALIFY_LN_BWD(W)                                                                                          \
-  layernorm_bwd_kernel<XDT, DXDT, W><<<grid, BwdCfg<W>::threads, 0, st>>>(G, g_ld, X, x_ld, dX, dx_ld, R, d, gamma, gb_dt,  \
-                                                                  mean, rinv, eps, eps_inside, stat, dgp, dbp,      \
+#define SCALIFY_LN_BWD(W)                                                                                        \
+  layernorm_bwd_kernel<XDT, DXDT, W><<<grid, kLnThreads, 0, st>>>(G, g_ld, X, x_ld, dX, dx_ld, R, d, gamma, gb_dt, \
+                                                                  mean, rinv, eps, eps_inside, stat, dgp, dbp,    \
                                                                   st_part)
   SCALIFY_DISPATCH_WIDE(x_dt, XDT, SCALIFY_DISPATCH_WIDE(dx_dt, DXDT, {
-    if (warps == 1) SCALIFY_LN_BWD(1); else SCALIFY_LN_BWD(4);
+    switch (tw) {
+      case 1: SCALIFY_LN_BWD(1); break;
+      case 2: SCALIFY_LN_BWD(2); break;
+      case 4: SCALIFY_LN_BWD(4); break;
+      default: SCALIFY_LN_BWD(8); break;
+    }
   }));
 #undef SCALIFY_LN_BWD
   SCALIFY_CUDA_TRY(cudaGetLastError());

@@ -54,7 +54,7 @@ def run_case(sizes, w_dt, mv_dt=orc.F16, g_dt=orc.E5M2, step=1000, seed=51, scal
                                                                                 orc.F32), orc.F32, c["w_scale"],
                                          c["lr"], c["beta1"], c["beta2"], c["eps"], step)[2], orc.F32)
         mag = (np.abs(wv) + np.abs(w_new * wsc - wv)) / wsc
-        ok = within(to_bits(w.data, c["w_dtype"]), wo, c["w_dtype"], w_new, mag, 4 * 2.0 ** -24)
+        ok = within(to_bits(w.data, c["w_dtype"]), wo, c["w_dtype"], w_new, mag, 8 * 2.0 ** -24)
         assert ok.all(), int((~ok).sum())
         # gradients are read-only
         assert np.array_equal(to_bits(g.data, c["g_dtype"]), c["g"])
