@@ -92,3 +92,55 @@ def test_gpt2_small_parameter_list_shapes():
     sizes = [max(1, int(np.prod(s)) // 16) for s in shapes]
     assert len(sizes) == 148
     run_case(sizes, orc.F16)
+
+
+def _sampled_adam_parity(tensors_np, G, M, V, W, hyper, step, rng, n_samples):
+    """Adam is elementwise: gather a sample of elements of each tensor, run the oracle on the sample with
+    the tensor's scales and compare with the library's result at the same positions."""
+    for c, g, m, v, w in zip(tensors_np, G, M, V, W):
+        n = c["g"].size
+        idx = np.unique(np.concatenate([rng.integers(0, n, min(n_samples, n)), [0, n - 1]]))
+        mo, vo, wo, ms, vs, wsc = orc.adam_step(c["g"][idx], orc.E5M2, c["g_scale"], c["m"][idx], c["v"][idx], orc.F16,
+                                                c["m_scale"], c["v_scale"], c["w"][idx], orc.F16, c["w_scale"],
+                                                hyper["lr"], hyper["beta1"], hyper["beta2"], hyper["eps"], step)
+        assert (m.scale_value(), v.scale_value(), w.scale_value()) == (ms, vs, wsc)
+        tidx = torch.from_numpy(idx).cuda()
+        assert ulp_diff(to_bits(m.data[tidx], orc.F16), mo, orc.F16).max() <= 1
+        assert ulp_diff(to_bits(v.data[tidx], orc.F16), vo, orc.F16).max() <= 1
+        assert ulp_diff(to_bits(w.data[tidx], orc.F16), wo, orc.F16).max() <= 1
+
+
+def test_config4_flat_125m_parameters_sampled():
+    """Full benchmark size, in the launch configuration the benchmark times: one flat tensor of 125M
+    parameters; 200k sampled elements against the oracle."""
+    n = 125_000_000
+    c = si.adam_case(n, seed=4)
+    G = [sc.ScaledTensor.make(to_dev(c["g"], orc.E5M2), c["g_scale"])]
+    M = [sc.ScaledTensor.make(to_dev(c["m"], orc.F16), c["m_scale"])]
+    V = [sc.ScaledTensor.make(to_dev(c["v"], orc.F16), c["v_scale"])]
+    W = [sc.ScaledTensor.make(to_dev(c["w"], orc.F16), c["w_scale"])]
+    ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_ADAM, 1))
+    hyper = dict(lr=c["lr"], beta1=c["beta1"], beta2=c["beta2"], eps=c["eps"])
+    sc.scalify_scaled_adam_step(sc.AdamTensors(G, M, V, W), ws, step=c["step"], **hyper)
+    assert ws.check_status() == 0
+    _sampled_adam_parity([c], G, M, V, W, hyper, c["step"], np.random.default_rng(7), 200_000)
+
+
+def test_config4_gpt2_small_parameter_list_full_size_sampled():
+    """The 148 tensors (124,439,808 parameters) of the GPT-2-small-shaped list in one call."""
+    shapes = si.gpt2_small_param_shapes()
+    sizes = [int(np.prod(s)) for s in shapes]
+    assert len(sizes) == 148 and sum(sizes) == 124_439_808
+    cases, G, M, V, W = [], [], [], [], []
+    for i, n in enumerate(sizes):
+        c = si.adam_case(n, seed=400 + i)
+        cases.append(c)
+        G.append(sc.ScaledTensor.make(to_dev(c["g"], orc.E5M2), c["g_scale"]))
+        M.append(sc.ScaledTensor.make(to_dev(c["m"], orc.F16), c["m_scale"]))
+        V.append(sc.ScaledTensor.make(to_dev(c["v"], orc.F16), c["v_scale"]))
+        W.append(sc.ScaledTensor.make(to_dev(c["w"], orc.F16), c["w_scale"]))
+    ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_ADAM, len(sizes)))
+    hyper = dict(lr=3e-4, beta1=0.9, beta2=0.999, eps=1e-8)
+    sc.scalify_scaled_adam_step(sc.AdamTensors(G, M, V, W), ws, step=1000, **hyper)
+    assert ws.check_status() == 0
+    _sampled_adam_parity(cases, G, M, V, W, hyper, 1000, np.random.default_rng(8), 2000)
