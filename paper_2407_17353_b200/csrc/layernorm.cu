@@ -4,9 +4,10 @@
 // owned by a team of TW warps (TW = 1, 2, 4 or 8, chosen so that a thread holds at most two
 // 16-byte vectors of the row); the row stays in registers, so mean, variance and the normalised
 // values come from one read.  Blocks of 256 threads hold 8/TW teams and stride over the rows with
-// a grid that is a multiple of the SM count.  The raw words of a team's NEXT row are fetched
-// before the current row is processed, which doubles the bytes in flight per thread.  gamma and
-// beta for a thread's fixed columns are converted once and kept in registers.
+// a grid that is a multiple of the SM count.  Rows are fetched ahead of use: the forward kernel
+// stages each thread's vectors of the next four rows in shared memory with cp.async, the backward
+// kernel keeps the raw words of the next row in registers.  gamma and beta for a thread's fixed
+// columns are converted once and kept in registers.
 #include "scalify_common.cuh"
 #include "scalify_launch.h"
 
@@ -14,6 +15,19 @@ namespace scalify {
 
 constexpr int kLnThreads = 256;
 constexpr int kLnVpt = 2;  // 16-byte vectors per thread and row
+constexpr int kLnFwdStages = 4;  // rows in flight per thread, forward
+
+// Per-thread asynchronous 16-byte copies into shared memory: a thread stages the vectors of its own
+// columns for the next kLnStages rows and later reads back only what it copied itself, so no
+// barrier is involved; cp.async.wait_group is a hardware wait, not a spin.  This keeps several rows
+// per thread in flight without holding them in registers.
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst))),
+               "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 template <int TW>
 __device__ __forceinline__ void team_barrier(int team) {
@@ -38,6 +52,36 @@ __device__ __forceinline__ void team_sum2(float& a, float& b, float (*smem)[8][2
     for (int w = 0; w < TW; ++w) { a += s[w][0]; b += s[w][1]; }
     buf ^= 1;
   }
+}
+
+template <int TW>
+__device__ __forceinline__ float team_sum1(float a, float (*smem)[8][2], int team, int& buf) {
+  a = warp_sum_f32(a);
+  if constexpr (TW > 1) {
+    const int lane = threadIdx.x & 31, wit = (threadIdx.x >> 5) % TW;
+    float(*s)[2] = smem[buf] + team * TW;
+    if (lane == 0) s[wit][0] = a;
+    team_barrier<TW>(team);
+    a = 0.f;
+#pragma unroll
+    for (int w = 0; w < TW; ++w) a += s[w][0];
+    buf ^= 1;
+  }
+  return a;
+}
+
+// 1/(sqrt(var)+eps) or 1/sqrt(var+eps) with the hardware approximations (each within 2 ulp of
+// fp32, far below the resolution of the 16-bit and 8-bit outputs)
+__device__ __forceinline__ float inv_sigma(float var, float eps, int eps_inside) {
+  float r;
+  if (eps_inside) {
+    asm("rsqrt.approx.f32 %0, %1;" : "=f"(r) : "f"(var + eps));
+  } else {
+    float sroot;
+    asm("sqrt.approx.f32 %0, %1;" : "=f"(sroot) : "f"(var));
+    r = __fdividef(1.0f, sroot + eps);
+  }
+  return r;
 }
 
 // gamma / beta vector of VEC elements starting at column c, as fp32 (dtype chosen at run time)
@@ -101,33 +145,43 @@ __global__ void __launch_bounds__(kLnThreads) layernorm_fwd_kernel(
   const int rows_per_iter = gridDim.x * TPB;
   const int iters = (R + rows_per_iter - 1) / rows_per_iter;
   int buf = 0;
-  uint32_t nxt[kLnVpt][4];
-  auto fetch = [&](int row) {
+  extern __shared__ uint4 ln_stage[];  // [stage][v][thread]
+  auto issue = [&](int row, int slot) {
 #pragma unroll
     for (int v = 0; v < kLnVpt; ++v) {
-      nxt[v][0] = nxt[v][1] = nxt[v][2] = nxt[v][3] = 0u;
       if (has[v] && row < R)
-        ld_raw_stream<16>(static_cast<const char*>(X) + (int64_t(row) * x_ld) * ElemBytes<XDT>::v +
-                              int64_t(t + v * TEAM) * 16, nxt[v]);
+        cp_async16(&ln_stage[(slot * kLnVpt + v) * kLnThreads + threadIdx.x],
+                   static_cast<const char*>(X) + (int64_t(row) * x_ld) * ElemBytes<XDT>::v + int64_t(t + v * TEAM) * 16);
     }
+    cp_async_commit();  // one group per row, even when empty, so that the group count stays uniform
   };
-  fetch(blockIdx.x * TPB + team);
+  const int first_row = blockIdx.x * TPB + team;
+#pragma unroll
+  for (int st = 0; st < kLnFwdStages; ++st) issue(first_row + st * rows_per_iter, st);
+  int slot = 0;
   for (int it = 0; it < iters; ++it) {
-    const int row = it * rows_per_iter + blockIdx.x * TPB + team;
+    const int row = it * rows_per_iter + first_row;
     const bool live = row < R;
     float x[kLnVpt][VEC];
+    cp_async_wait<kLnFwdStages - 1>();  // the oldest row in flight has landed
 #pragma unroll
-    for (int v = 0; v < kLnVpt; ++v) decode_vec<XDT, VEC>(nxt[v], x[v]);
-    fetch(row + rows_per_iter);  // raw words of this team's next row
-    float s = 0.f, dummy = 0.f;
+    for (int v = 0; v < kLnVpt; ++v) {
+      uint32_t w[4] = {0u, 0u, 0u, 0u};
+      if (has[v] && live) {
+        const uint4 q4 = ln_stage[(slot * kLnVpt + v) * kLnThreads + threadIdx.x];
+        w[0] = q4.x; w[1] = q4.y; w[2] = q4.z; w[3] = q4.w;
+      }
+      decode_vec<XDT, VEC>(w, x[v]);
+    }
+    issue(row + kLnFwdStages * rows_per_iter, slot);  // refill the slot just read
+    if (++slot == kLnFwdStages) slot = 0;
+    float s = 0.f;
 #pragma unroll
     for (int v = 0; v < kLnVpt; ++v)
 #pragma unroll
       for (int e = 0; e < VEC; ++e) s += x[v][e];  // absent vectors hold zeros
-    team_sum2<TW>(s, dummy, smem, team, buf);
-    const float mu = s * inv_d;
+    const float mu = team_sum1<TW>(s, smem, team, buf) * inv_d;
     float q = 0.f;
-    dummy = 0.f;
 #pragma unroll
     for (int v = 0; v < kLnVpt; ++v) {
       if (has[v]) {
@@ -135,9 +189,8 @@ __global__ void __launch_bounds__(kLnThreads) layernorm_fwd_kernel(
         for (int e = 0; e < VEC; ++e) { x[v][e] -= mu; q = fmaf(x[v][e], x[v][e], q); }
       }
     }
-    team_sum2<TW>(q, dummy, smem, team, buf);
-    const float var = q * inv_d;
-    const float rinv = eps_inside ? 1.0f / sqrtf(var + eps) : 1.0f / (sqrtf(var) + eps);
+    const float var = team_sum1<TW>(q, smem, team, buf) * inv_d;
+    const float rinv = inv_sigma(var, eps, eps_inside);
     if (live) {
       if (t == 0) {
         if (mean_out) mean_out[row] = mu;
@@ -184,7 +237,7 @@ int launch_layernorm_fwd(const void* X, int x_dt, int64_t x_ld, void* Y, int y_d
   if (tw == 0) return SCALIFY_ERR_UNSUPPORTED;
   const int grid = ln_grid(R, 8 / tw, 3);
 #define SCALIFY_LN_FWD(W)                                                                                      \
-  layernorm_fwd_kernel<XDT, YDT, W><<<grid, kLnThreads, 0, st>>>(X, x_ld, Y, y_ld, R, d, gamma, beta, gb_dt,    \
+  layernorm_fwd_kernel<XDT, YDT, W><<<grid, kLnThreads, kLnFwdStages * kLnVpt * kLnThreads * 16, st>>>(X, x_ld, Y, y_ld, R, d, gamma, beta, gb_dt,    \
                                                                  gamma_scale, beta_scale, y_scale, eps,         \
                                                                  eps_inside, mean, rinv)
   SCALIFY_DISPATCH_WIDE(x_dt, XDT, SCALIFY_DISPATCH_DTYPE(y_dt, YDT, {
@@ -234,6 +287,7 @@ __global__ void __launch_bounds__(kLnThreads, 2) layernorm_bwd_kernel(
   const int rows_per_iter = gridDim.x * TPB;
   const int iters = (R + rows_per_iter - 1) / rows_per_iter;
   int buf = 0;
+  // the raw words of the team's next row are fetched before the current row is processed
   uint32_t nx[kLnVpt][4], ng[kLnVpt][4];
   float nmu = 0.f, nrinv = 0.f;
   auto fetch = [&](int row) {
@@ -288,8 +342,8 @@ __global__ void __launch_bounds__(kLnThreads, 2) layernorm_bwd_kernel(
     if (eps_inside) {
       c2 = rinv * m2;
     } else {
-      const float s = 1.0f / rinv - eps;
-      c2 = (s > 0.f) ? m2 / s : 0.f;
+      const float s = __fdividef(1.0f, rinv) - eps;
+      c2 = (s > 0.f) ? __fdividef(m2, s) : 0.f;
     }
     if (live) {
       char* orow = static_cast<char*>(dX) + int64_t(row) * dx_ld * ElemBytes<DXDT>::v;
@@ -298,15 +352,20 @@ __global__ void __launch_bounds__(kLnThreads, 2) layernorm_bwd_kernel(
         if (has[v]) {
           float o[VEC];
 #pragma unroll
-          for (int e = 0; e < VEC; ++e) {
-            o[e] = fmaf(-x[v][e], c2, (g[v][e] - m1) * rinv);
-            const float stored = round_through<DXDT>(o[e]);
-            amax = max(amax, abs_bits(stored));
-            ssq = fmaf(stored, stored, ssq);
-          }
+          for (int e = 0; e < VEC; ++e) o[e] = fmaf(-x[v][e], c2, (g[v][e] - m1) * rinv);
           uint32_t ow[OB / 4];
           encode_vec<DXDT, VEC>(o, ow);
           st_raw<OB>(orow + int64_t(t + v * TEAM) * OB, ow);
+          if (stat == SCALIFY_STAT_AMAX) {
+            // rounding is monotonic: the max of the stored values is the stored value of the max
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) amax = max(amax, abs_bits(o[e]));
+          } else if (stat == SCALIFY_STAT_L2) {
+            float sv[VEC];
+            decode_vec<DXDT, VEC>(ow, sv);  // the values as stored
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) ssq = fmaf(sv[e], sv[e], ssq);
+          }
         }
       }
     }
@@ -350,6 +409,7 @@ __global__ void __launch_bounds__(kLnThreads, 2) layernorm_bwd_kernel(
   if (stat != SCALIFY_STAT_NONE) {
     __shared__ double s_stat[kLnThreads / 32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (stat == SCALIFY_STAT_AMAX) amax = abs_bits(round_through<DXDT>(__uint_as_float(amax)));
     double mine = (stat == SCALIFY_STAT_AMAX) ? static_cast<double>(warp_max_u32(amax))
                                               : warp_sum_f64(static_cast<double>(ssq));
     if (lane == 0) s_stat[warp] = mine;
@@ -363,22 +423,22 @@ __global__ void __launch_bounds__(kLnThreads, 2) layernorm_bwd_kernel(
   }
 }
 
-// Combines the per-block partials in block order: dgamma/dbeta columns (scaled by 1/kf(R)), the
-// statistic word, and the propagated scale words.  Block = 32 columns x 8 slices of the block list.
+// Combines the per-block partials in a fixed order: dgamma/dbeta columns (scaled by 1/kf(R)), the
+// statistic word, and the propagated scale words.  Block = 32 columns x 32 slices of the block list.
 template <int DGDT>
-__global__ void __launch_bounds__(256) layernorm_bwd_finalize_kernel(
+__global__ void __launch_bounds__(1024) layernorm_bwd_finalize_kernel(
     int nblocks, int R, int d, const float* __restrict__ dgamma_part, const float* __restrict__ dbeta_part,
     const double* __restrict__ stat_part, int stat, float* stat_word, void* __restrict__ dgamma,
     void* __restrict__ dbeta, const float* g_scale, const float* x_scale, const float* gamma_scale,
     float* dx_scale, float* dgamma_scale, float* dbeta_scale, uint32_t* status) {
-  __shared__ float s_a[8][33], s_b[8][33];
+  __shared__ float s_a[32][33], s_b[32][33];
   const float inv_kf = 1.0f / kfactor(R);
   const int cx = threadIdx.x & 31, slice = threadIdx.x >> 5;
   const int col = blockIdx.x * 32 + cx;
   if (dgamma_part) {
     float a = 0.f, b = 0.f;
     if (col < d) {
-      for (int i = slice; i < nblocks; i += 8) {
+      for (int i = slice; i < nblocks; i += 32) {
         a += dgamma_part[int64_t(i) * d + col];
         b += dbeta_part[int64_t(i) * d + col];
       }
@@ -387,7 +447,7 @@ __global__ void __launch_bounds__(256) layernorm_bwd_finalize_kernel(
     s_b[slice][cx] = b;
     __syncthreads();
     if (slice == 0 && col < d) {
-      for (int k = 1; k < 8; ++k) { a += s_a[k][cx]; b += s_b[k][cx]; }
+      for (int k = 1; k < 32; ++k) { a += s_a[k][cx]; b += s_b[k][cx]; }
       store_elem<DGDT>(dgamma, col, a * inv_kf);
       store_elem<DGDT>(dbeta, col, b * inv_kf);
     }
@@ -461,7 +521,7 @@ int launch_layernorm_bwd(const void* G, int64_t g_ld, const void* X, int x_dt, i
   SCALIFY_CUDA_TRY(cudaGetLastError());
   const int fgrid = dgamma ? (d + 31) / 32 : 1;
   SCALIFY_DISPATCH_WIDE(dg_dt, DGDT,
-      layernorm_bwd_finalize_kernel<DGDT><<<fgrid, 256, 0, st>>>(grid, R, d, dgp, dbp, st_part, stat, v.stat, dgamma,
+      layernorm_bwd_finalize_kernel<DGDT><<<fgrid, 1024, 0, st>>>(grid, R, d, dgp, dbp, st_part, stat, v.stat, dgamma,
                                                                  dbeta, g_scale, x_scale, gamma_scale, dx_scale,
                                                                  dgamma_scale, dbeta_scale, v.status));
   SCALIFY_CUDA_TRY(cudaGetLastError());
