@@ -158,6 +158,20 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def aggregate_over_ranks(dist, device, world, flops_per_rank, ms_per_step, head_ms, e2e_ms):
+    """Replicas-only scaling: every rank runs the same step on its own GPU.  The job's time is the MAX over
+    ranks of the device-measured times; the job's throughput is the work of all ranks over that time.
+    `dist` is torch.distributed (initialised) or None for one process."""
+    import torch
+    if dist is not None:
+        tt = torch.tensor([ms_per_step, head_ms, e2e_ms], device=device, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms_per_step, head_ms, e2e_ms = [float(x) for x in tt]
+    value = world * flops_per_rank / (head_ms * 1e-3) / 1e12
+    e2e_value = world * flops_per_rank / (e2e_ms * 1e-3) / 1e12 if e2e_ms == e2e_ms else float("nan")
+    return ms_per_step, head_ms, e2e_ms, value, e2e_value
+
+
 def run_profile_row(args):
     """One row of the hot path alone, on a case that holds well under 2 GB on the device but is larger than
     L2, launched `--steps` times after `--warmup` launches.  Meant to be run under ncu."""
@@ -425,14 +439,8 @@ def main():
     e2e_local = flops / (e2e_ms * 1e-3) / 1e12
 
     # ------------------------------------------------------------------ reduce over ranks (max time)
-    if dist is not None:
-        tt = torch.tensor([ms_per_step, head_ms, e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms_per_step, head_ms_max, e2e_ms_max = [float(x) for x in tt]
-    else:
-        head_ms_max, e2e_ms_max = head_ms, e2e_ms
-    value = world * flops / (head_ms_max * 1e-3) / 1e12
-    e2e_value = world * flops / (e2e_ms_max * 1e-3) / 1e12
+    ms_per_step, head_ms_max, e2e_ms_max, value, e2e_value = aggregate_over_ranks(
+        dist, dev, world, flops, ms_per_step, head_ms, e2e_ms)
 
     if rank != 0:
         if dist is not None:
