@@ -61,6 +61,9 @@ def lib() -> ctypes.CDLL:
         L.orc_statistic.argtypes = [vp, i32, i64, i32]
         L.orc_scaled_matmul.argtypes = [vp, i32, i64, i32, f32, vp, i32, i64, i32, f32, i64, i64, i64,
                                         i32, vp, i64, pf32, vp, vp]
+        L.orc_scaled_matmul_delayed.restype = f64
+        L.orc_scaled_matmul_delayed.argtypes = [vp, i32, i64, i32, f32, vp, i32, i64, i32, f32, i64, i64, i64, f64, i32,
+                                                i32, vp, i64, pf32]
         L.orc_scaled_matmul_samples.argtypes = [vp, i32, i64, i32, vp, i32, i64, i32, i64, i64, vp, vp, vp, vp]
         L.orc_rescale.restype = f64
         L.orc_rescale.argtypes = [vp, i32, i64, f32, i32, f64, i32, vp, pf32]
@@ -150,6 +153,21 @@ def scaled_matmul(A, a_dtype, a_scale, B, b_dtype, b_scale, y_dtype, transA=Fals
                             _ptr(B), b_dtype, B.shape[1], int(transB), float(b_scale),
                             M, N, K, y_dtype, _ptr(Y), N, ctypes.byref(ys), _ptr(acc), _ptr(sab))
     return Y, float(ys.value), acc, sab
+
+
+def scaled_matmul_delayed(A, a_dtype, a_scale, B, b_dtype, b_scale, stat_in, stat, y_dtype, transA=False, transB=False):
+    """Matmul whose output is rebalanced by p2f(stat_in) while this step's statistic is gathered.
+    Returns (Y bits, Y scale, statistic of the un-rebalanced data)."""
+    A = _bits(A, a_dtype)
+    B = _bits(B, b_dtype)
+    M, K = (A.shape[1], A.shape[0]) if transA else A.shape
+    N = B.shape[0] if transB else B.shape[1]
+    Y = np.empty((M, N), dtype=_BITS_NP[y_dtype])
+    ys = ctypes.c_float(0)
+    s = lib().orc_scaled_matmul_delayed(_ptr(A), a_dtype, A.shape[1], int(transA), float(a_scale), _ptr(B), b_dtype,
+                                        B.shape[1], int(transB), float(b_scale), M, N, K, float(stat_in), stat,
+                                        y_dtype, _ptr(Y), N, ctypes.byref(ys))
+    return Y, float(ys.value), float(s)
 
 
 def scaled_matmul_samples(A, a_dtype, B, b_dtype, rows, cols, transA=False, transB=False):

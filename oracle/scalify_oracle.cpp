@@ -303,6 +303,27 @@ void orc_scaled_matmul(const void* A, int a_dtype, int64_t lda, int transA, floa
   }
 }
 
+// Scaled matmul with DELAYED rescaling (Section 3.3: the statistic and the rebalancing are
+// decoupled, the statistic of an earlier step is kept in the state).  The output is written
+// already rebalanced by r = p2f(stat_in) (r = 1 when stat_in cannot define a scale):
+//   Y_d = encode((A_d . B_d) / kf(K) / r),  Y_s = A_s * B_s * kf(K) * r,
+// and the statistic of THIS step's un-rebalanced data (A_d . B_d)/kf(K), taken before any
+// rounding, is returned for the next step.
+double orc_scaled_matmul_delayed(const void* A, int a_dtype, int64_t lda, int transA, float a_scale,
+                                 const void* B, int b_dtype, int64_t ldb, int transB, float b_scale,
+                                 int64_t M, int64_t N, int64_t K, double stat_in, int stat,
+                                 int y_dtype, void* Y, int64_t ldy, float* y_scale) {
+  std::vector<double> acc(static_cast<size_t>(M * N));
+  float ys0 = 0.f;
+  orc_scaled_matmul(A, a_dtype, lda, transA, a_scale, B, b_dtype, ldb, transB, b_scale, M, N, K, F32, nullptr, N, &ys0,
+                    acc.data(), nullptr);
+  const double r = usable_stat(stat_in) ? p2f(stat_in) : 1.0;
+  for (int64_t i = 0; i < M; ++i)
+    for (int64_t j = 0; j < N; ++j) store_bits(Y, y_dtype, i * ldy + j, encode(acc[i * N + j] / r, y_dtype));
+  if (y_scale) *y_scale = static_cast<float>(static_cast<double>(ys0) * r);
+  return statistic(acc, stat);
+}
+
 // The same rule evaluated for a list of output positions only (full-size
 // parity checks on sampled outputs).
 void orc_scaled_matmul_samples(const void* A, int a_dtype, int64_t lda, int transA,

@@ -402,3 +402,22 @@ def test_adam_scale_words_golden_cfg4():
         d = vals(got, orc.F16)
         q = exact / s
         assert np.all(np.abs(d - q) <= np.maximum(np.abs(q) * 2.0 ** -11, 2.0 ** -25) * 1.0000001)
+
+
+# ---------------------------------------------------------------- delayed rescaling (Section 3.3)
+
+def test_delayed_matmul_equals_matmul_followed_by_rescale_with_the_old_statistic():
+    M, N, K = 24, 40, 64
+    A = si.scaled_normal(19, 1, (M, K), orc.E4M3)
+    B = si.scaled_normal(19, 2, (K, N), orc.E4M3)
+    # E4M3 products summed over K=64 are exact in fp32, so the fp32 intermediate loses nothing
+    Y32, ys, acc, _ = orc.scaled_matmul(A, orc.E4M3, 0.5, B, orc.E4M3, 2.0, orc.F32, want_acc=True)
+    assert np.array_equal(orc.decode(Y32, orc.F32), acc)
+    for stat_in in (9.0, 0.3, 0.0, float("inf")):
+        Yd, yds, s_now = orc.scaled_matmul_delayed(A, orc.E4M3, 0.5, B, orc.E4M3, 2.0, stat_in, orc.STAT_AMAX, orc.E4M3)
+        want, ws, _ = orc.rescale(Y32, orc.F32, ys, orc.STAT_AMAX, orc.E4M3,
+                                  stat_override=stat_in if np.isfinite(stat_in) and stat_in > 0 else 1.0)
+        assert np.array_equal(Yd, want) and yds == ws
+        assert s_now == np.abs(acc).max()
+    _, _, s_l2 = orc.scaled_matmul_delayed(A, orc.E4M3, 0.5, B, orc.E4M3, 2.0, 1.0, orc.STAT_L2, orc.BF16)
+    assert abs(s_l2 - np.sqrt(np.mean(acc ** 2))) < 1e-12
