@@ -10,6 +10,9 @@ shaped like GPT-style training tensors:
   5. scaled LayerNorm forward  [131072, 1024] BF16
   6. scaled LayerNorm backward + L2 dynamic rescale of the input gradient to E5M2
   7. scaled Adam step over 125M parameters (E5M2 grads, FP16 scaled m/v/w)
+Outside the step (own timed loop) the next-row variant is reported too: the same GEMM with delayed
+rescaling - one kernel, E4M3 written directly with the previous step's statistic while this step's AMAX
+is gathered, no BF16 intermediate, no pass 2.
 `value` is the headline metric: 2*M*N*K / (time of rows 1+2), measured with CUDA events inside
 the step.  Rows 3-7 are reported as GB/s of algorithmic bytes in `rows`.
 
@@ -349,6 +352,9 @@ def main():
     ws_ad = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_ADAM, 1), dev)
     del am0, av0, aw0
 
+    Yd = sc.ScaledTensor.empty((N_GEMM, N_GEMM), torch.float8_e4m3fn, dev)
+    stat_state = torch.full((1,), 4.0, dtype=torch.float32, device=dev)
+
     n_ev = 8
     launches_per_step = 2 + 2 + 1 + 1 + 3 + 2  # kernels of this library per step (memsets are not kernels)
 
@@ -410,6 +416,22 @@ def main():
     value_local = flops / (head_ms * 1e-3) / 1e12
     ms_per_step = total_ms / K
 
+    # ------------------------------------------------------------------ next-row variant, timed on its own
+    def delayed_step():
+        sc.scalify_scaled_matmul_delayed(A, Bt, stat_state, Yd, ws_mm, transB=True, stat=sc.STAT_AMAX,
+                                         stat_out=stat_state)
+    for _ in range(3):
+        delayed_step()
+    barrier()
+    d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    d_iters = max(3, min(K, 20))
+    d0.record()
+    for _ in range(d_iters):
+        delayed_step()
+    d1.record()
+    barrier()
+    delayed_ms = d0.elapsed_time(d1) / d_iters
+
     # ------------------------------------------------------------------ end to end through host buffers
     hY = torch.empty((N_GEMM, N_GEMM), dtype=torch.int8).pin_memory()
     hscale = torch.empty(1, dtype=torch.float32).pin_memory()
@@ -464,6 +486,9 @@ def main():
         row("a5 scaled LayerNorm fwd BF16->BF16 (4 B/elem + 8 B/row)", seg_ms[4], 4 * n_ln + 8 * LN_R),
         row("a6 scaled LayerNorm bwd + L2 rescale to E5M2 (9 B/elem + 8 B/row)", seg_ms[5], 9 * n_ln + 8 * LN_R),
         row("a7 scaled Adam, E5M2 grads, FP16 m/v/w (13 B/param)", seg_ms[6], 13 * ADAM_N),
+        {"row": "f1 (next, timed outside the step, back to back) delayed-rescale GEMM 8192^3: E4M3 out in one "
+                "kernel, no BF16 intermediate, no pass 2", "ms": round(float(delayed_ms), 4),
+         "TFLOP/s": round(flops / (delayed_ms * 1e-3) / 1e12, 1)},
     ]
     fp8_peak = 2.0 * peaks["bf16_sustained"]
     gemm_tflops = flops / (float(seg_ms[0]) * 1e-3) / 1e12

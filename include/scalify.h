@@ -150,6 +150,25 @@ int scalify_scaled_matmul(const scalify_array* A, int transA, const scalify_arra
                           void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Scaled matrix multiply with DELAYED rescaling (Section 3.3: "Delayed rescaling can be
+ * similarly implemented by decoupling the compute of statistics and rebalancing ..., keeping
+ * track of the first one in the model state").  One kernel, no intermediate, no second pass:
+ *
+ *   r   = *stat_in rounded down to a power of two (1 if *stat_in is zero, below 2^-126 or
+ *         non-finite): the statistic of an EARLIER step, kept by the caller on the device;
+ *   Y_d = cast((op(A)_d . op(B)_d) / kf(K) / r),   Y_s = A_s * B_s * kf(K) * r;
+ *   *stat_out (and workspace offset 16) = statistic `stat` of THIS step's un-rebalanced fp32
+ *         values (op(A)_d . op(B)_d)/kf(K), for the next step.
+ *
+ * Y may be FP8 (E4M3 / E5M2) as well as BF16 / F16 / F32.  stat_out may be NULL, and may be the
+ * same word as stat_in (it is written after the kernel has finished).  stat = SCALIFY_STAT_NONE
+ * gathers nothing (stat_out must then be NULL).  Other arguments as scalify_scaled_matmul.
+ */
+int scalify_scaled_matmul_delayed(const scalify_array* A, int transA, const scalify_array* B, int transB,
+                                  const float* stat_in, scalify_array* Y, int stat, float* stat_out,
+                                  void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Statistic of the data component of X (Section 3.3: "L2 moment (or any other
  * statistic)"), written as one fp32 to `out_stat` (device) and to byte offset
  * 16 of the workspace.  X may be any dtype, contiguous.

@@ -67,6 +67,7 @@ def lib() -> ctypes.CDLL:
         L.scalify_check_status.argtypes = [vp, vp]
         L.scalify_scaled_matmul.argtypes = [P, i32, P, i32, P, i32, P, vp, sz, vp]
         L.scalify_statistic.argtypes = [P, i32, vp, vp, sz, vp]
+        L.scalify_scaled_matmul_delayed.argtypes = [P, i32, P, i32, vp, P, i32, vp, vp, sz, vp]
         L.scalify_rescale.argtypes = [P, i32, vp, vp, P, vp, sz, vp]
         L.scalify_scaled_add.argtypes = [P, P, i32, P, vp]
         L.scalify_scaled_layernorm.argtypes = [P, P, P, f32, i32, P, vp, vp, vp]
@@ -75,7 +76,8 @@ def lib() -> ctypes.CDLL:
         L.scalify_scaled_gelu_bwd.argtypes = [P, P, i32, P, vp]
         L.scalify_scaled_adam_step.argtypes = [i32, P, P, P, P, f32, f32, f32, f32, i64, vp, sz, vp]
         L.scalify_scaled_adam_step_static.argtypes = [i32, P, P, P, P, f32, f32, f32, f32, i64, vp, vp]
-        for name in ("scalify_workspace_init", "scalify_check_status", "scalify_scaled_matmul", "scalify_statistic",
+        for name in ("scalify_workspace_init", "scalify_check_status", "scalify_scaled_matmul", "scalify_scaled_matmul_delayed",
+                     "scalify_statistic",
                      "scalify_rescale", "scalify_scaled_add", "scalify_scaled_layernorm",
                      "scalify_scaled_layernorm_bwd", "scalify_scaled_gelu", "scalify_scaled_gelu_bwd",
                      "scalify_scaled_adam_step", "scalify_scaled_adam_step_static"):
@@ -183,6 +185,15 @@ def scalify_scaled_matmul(A: ScaledTensor, B: ScaledTensor, Y: ScaledTensor, ws:
     a, b, y, yq = _desc(A), _desc(B), _desc(Y), _desc(Yq)
     _check(lib().scalify_scaled_matmul(_ref(a), int(transA), _ref(b), int(transB), _ref(y), stat, _ref(yq),
                                        ws.ptr, ws.nbytes, _stream(stream)), "scalify_scaled_matmul")
+
+
+def scalify_scaled_matmul_delayed(A: ScaledTensor, B: ScaledTensor, stat_in: torch.Tensor, Y: ScaledTensor,
+                                  ws: Workspace, *, transA=False, transB=False, stat: int = STAT_AMAX,
+                                  stat_out: Optional[torch.Tensor] = None, stream=None) -> None:
+    a, b, y = _desc(A), _desc(B), _desc(Y)
+    _check(lib().scalify_scaled_matmul_delayed(_ref(a), int(transA), _ref(b), int(transB), _ptr(stat_in), _ref(y),
+                                               stat, _ptr(stat_out), ws.ptr, ws.nbytes, _stream(stream)),
+           "scalify_scaled_matmul_delayed")
 
 
 def scalify_statistic(X: ScaledTensor, stat: int, ws: Workspace, out: Optional[torch.Tensor] = None, stream=None) -> None:

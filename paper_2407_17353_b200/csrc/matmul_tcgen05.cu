@@ -63,6 +63,7 @@ struct GemmParams {
   const float* b_scale;
   float* y_scale;
   int stat;
+  const float* stat_in;  // delayed rescale: statistic of an earlier step (device), or NULL
   uint32_t* stat_word;   // AMAX: atomicMax target
   double* l2_partials;   // L2: [tiles][4]
   uint32_t* status;
@@ -266,7 +267,13 @@ scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     mbar_init(drain_bar, 1);
     *abort_flag = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    if (blockIdx.x == 0 && p.y_scale) *p.y_scale = load_scale(p.a_scale) * load_scale(p.b_scale) * p.kf;
+    if (blockIdx.x == 0) {
+      float r = 1.0f;
+      bool nf = false;
+      if (p.stat_in) r = rescale_factor(__ldg(p.stat_in), &nf);
+      if (p.y_scale) *p.y_scale = load_scale(p.a_scale) * load_scale(p.b_scale) * p.kf * r;
+      if (nf && p.status) atomicOr(p.status, static_cast<uint32_t>(SCALIFY_DEV_NONFINITE_STAT));
+    }
     if (blockIdx.x == 0 && p.status) {
       if (!is_pow2_scale(load_scale(p.a_scale)) || !is_pow2_scale(load_scale(p.b_scale)))
         atomicOr(p.status, static_cast<uint32_t>(SCALIFY_DEV_BAD_SCALE));
@@ -382,6 +389,11 @@ scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     uint32_t amax_bits = 0u;
     char* const Yb = static_cast<char*>(p.Y);
     constexpr int OSZ = ElemBytes<OUT>::v;
+    // delayed rescale (Section 3.3): the data are written already divided by r = p2_floor(earlier
+    // statistic); this step's statistic is taken on the un-rebalanced fp32 values
+    float r_prev = 1.0f;
+    if (p.stat_in) { bool nf; r_prev = rescale_factor(__ldg(p.stat_in), &nf); }
+    const float alpha = p.alpha * (1.0f / r_prev);  // exact: both are powers of two
     for (int tile = unit; tile < num_tiles; tile += num_units) {
       int b, mt, nt;
       tile_coords(p, tile, b, mt, nt);
@@ -402,12 +414,15 @@ scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         float v[32];
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
-          v[i] = __uint_as_float(r[i]) * p.alpha;
+          v[i] = __uint_as_float(r[i]) * alpha;
           amax_bits = max(amax_bits, abs_bits(v[i]));
         }
         if (p.stat == SCALIFY_STAT_L2) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) { const float s = round_through<OUT>(v[i]); ssq = fmaf(s, s, ssq); }
+          for (int i = 0; i < 32; ++i) {
+            const float s = p.stat_in ? v[i] : round_through<OUT>(v[i]);
+            ssq = fmaf(s, s, ssq);
+          }
         }
         if (row_ok) {
           if (col0 + 32 <= p.N) {
@@ -429,14 +444,15 @@ scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         else mbar_arrive_cluster(map_to_cta(acc_empty_bar + 8 * acc, 0u));  // the leader issues the next MMAs
       }
       if (p.stat == SCALIFY_STAT_L2) {
-        const double s = warp_sum_f64(static_cast<double>(ssq));
+        const double s = warp_sum_f64(static_cast<double>(ssq)) * (double(r_prev) * double(r_prev));
         if (lane == 0) p.l2_partials[(static_cast<long long>(tile) * NCTA + rank) * 4 + q] = s;
       }
       if (++acc == kAccStages) { acc = 0; acc_phase ^= 1u; }
     }
     if (p.stat == SCALIFY_STAT_AMAX) {
       // rounding is monotonic, so the max of the stored values is the stored value of the max
-      amax_bits = abs_bits(round_through<OUT>(__uint_as_float(amax_bits)));
+      if (p.stat_in) amax_bits = abs_bits(__uint_as_float(amax_bits) * r_prev);  // un-rebalanced, unrounded
+      else amax_bits = abs_bits(round_through<OUT>(__uint_as_float(amax_bits)));
       amax_bits = warp_max_u32(amax_bits);
       if (lane == 0 && amax_bits != 0u) atomicMax(p.stat_word, amax_bits);
     }
@@ -593,13 +609,14 @@ int launch_scaled_matmul(const MatmulArgs& a, void* ws, cudaStream_t st) {
   p.Y = a.Y; p.ldy = a.ldy; p.y_batch_stride = a.y_bs;
   p.a_scale = a.a_scale; p.b_scale = a.b_scale; p.y_scale = a.y_scale;
   p.stat = a.stat;
+  p.stat_in = a.stat_in;
   p.stat_word = reinterpret_cast<uint32_t*>(v.stat);
   p.l2_partials = static_cast<double*>(v.area);
   p.status = v.status;
   const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n * p.batch;
   if (tiles > (1ll << 30)) return SCALIFY_ERR_SHAPE;
   if (a.stat == SCALIFY_STAT_AMAX) SCALIFY_CUDA_TRY(cudaMemsetAsync(v.stat, 0, sizeof(float), st));
-  SCALIFY_DISPATCH_WIDE(a.y_dt, OUT, {
+  SCALIFY_DISPATCH_DTYPE(a.y_dt, OUT, {
     if (ncta == 2) rc = launch_variant<OUT, 2>(map_a, map_b, p, tiles, st);
     else rc = launch_variant<OUT, 1>(map_a, map_b, p, tiles, st);
   });

@@ -430,6 +430,7 @@ int scalify_scaled_matmul(const scalify_array* A, int transA, const scalify_arra
   float* y_scale = Y->scale ? Y->scale : reinterpret_cast<float*>(static_cast<char*>(workspace) + 48);
   a.y_scale = y_scale;
   a.stat = stat;
+  a.stat_in = nullptr;
   a.force_ncta = 0;
   if (a.lda < (transA ? M : K) || a.ldb < (transB ? K : N) || a.ldy < N) return SCALIFY_ERR_SHAPE;
   rc = launch_scaled_matmul(a, workspace, st);
@@ -440,6 +441,54 @@ int scalify_scaled_matmul(const scalify_array* A, int transA, const scalify_arra
                           kModeDynamic, v.status, st);
   }
   return rc;
+}
+
+int scalify_scaled_matmul_delayed(const scalify_array* A, int transA, const scalify_array* B, int transB,
+                                  const float* stat_in, scalify_array* Y, int stat, float* stat_out, void* workspace,
+                                  size_t workspace_bytes, void* stream) {
+  int rc = check_array(A);
+  if (rc) return rc;
+  rc = check_array(B);
+  if (rc) return rc;
+  rc = check_array(Y);
+  if (rc) return rc;
+  if (!stat_in) return SCALIFY_ERR_NULL;
+  if (!is_fp8(A->dtype) || !is_fp8(B->dtype)) return SCALIFY_ERR_DTYPE;
+  if (!valid_stat(stat)) return SCALIFY_ERR_VALUE;
+  if (stat == SCALIFY_STAT_NONE && stat_out) return SCALIFY_ERR_VALUE;
+  if (A->ndim < 2 || B->ndim < 2 || Y->ndim != A->ndim || B->ndim > A->ndim) return SCALIFY_ERR_SHAPE;
+  const int an = A->ndim, bn = B->ndim, yn = Y->ndim;
+  const int64_t batch = an == 3 ? A->shape[0] : 1;
+  const int64_t M = transA ? A->shape[an - 1] : A->shape[an - 2];
+  const int64_t K = transA ? A->shape[an - 2] : A->shape[an - 1];
+  const int64_t Kb = transB ? B->shape[bn - 1] : B->shape[bn - 2];
+  const int64_t N = transB ? B->shape[bn - 2] : B->shape[bn - 1];
+  if (K != Kb || K < 1 || M < 1 || N < 1 || batch < 1) return SCALIFY_ERR_SHAPE;
+  if (Y->shape[yn - 2] != M || Y->shape[yn - 1] != N) return SCALIFY_ERR_SHAPE;
+  if (an == 3 && (Y->shape[0] != batch || (bn == 3 && B->shape[0] != batch))) return SCALIFY_ERR_SHAPE;
+  if (M > 0x7FFFFFFF || N > 0x7FFFFFFF || K > 0x7FFFFFFF || batch > 0x7FFFFFFF) return SCALIFY_ERR_SHAPE;
+  if (Y->scale && (Y->scale == A->scale || Y->scale == B->scale)) return SCALIFY_ERR_ALIAS;
+  rc = check_ws(workspace, workspace_bytes, scalify_workspace_bytes(SCALIFY_OP_MATMUL, batch * M, N));
+  if (rc) return rc;
+  MatmulArgs a;
+  a.A = A->data; a.a_dt = A->dtype; a.transA = transA ? 1 : 0; a.lda = A->stride[an - 2];
+  a.a_bs = an == 3 ? A->stride[0] : 0;
+  a.B = B->data; a.b_dt = B->dtype; a.transB = transB ? 1 : 0; a.ldb = B->stride[bn - 2];
+  a.b_bs = bn == 3 ? B->stride[0] : 0;
+  a.Y = Y->data; a.y_dt = Y->dtype; a.ldy = Y->stride[yn - 2]; a.y_bs = yn == 3 ? Y->stride[0] : 0;
+  a.M = static_cast<int>(M); a.N = static_cast<int>(N); a.K = static_cast<int>(K); a.batch = static_cast<int>(batch);
+  a.a_scale = A->scale; a.b_scale = B->scale; a.y_scale = Y->scale;
+  a.stat = stat;
+  a.stat_in = stat_in;
+  a.force_ncta = 0;
+  if (a.lda < (transA ? M : K) || a.ldb < (transB ? K : N) || a.ldy < N) return SCALIFY_ERR_SHAPE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  rc = launch_scaled_matmul(a, workspace, st);
+  if (rc) return rc;
+  // published only after the kernel has finished, so stat_out may be the word stat_in points to
+  if (stat_out)
+    SCALIFY_CUDA_TRY(cudaMemcpyAsync(stat_out, ws_view(workspace).stat, sizeof(float), cudaMemcpyDeviceToDevice, st));
+  return SCALIFY_OK;
 }
 
 }  // extern "C"

@@ -40,6 +40,7 @@ struct MatmulArgs {
   int M, N, K, batch;
   const float* a_scale; const float* b_scale; float* y_scale;
   int stat;
+  const float* stat_in;  // delayed rescale: earlier statistic (device) or NULL
   int force_ncta;  // 0: choose; 1: force the one-CTA kernel
 };
 size_t matmul_ws_bytes(int64_t rows, int64_t cols);

@@ -206,3 +206,84 @@ def test_bad_scale_is_reported_in_status_word():
     Bt = si.scaled_normal(25, 2, (256, 128), orc.E4M3)
     g = run_matmul(A, orc.E4M3, 3.0, Bt, orc.E4M3, 1.0, orc.BF16, False, True)
     assert g["status"] & sc.DEV_BAD_SCALE
+
+
+# ---------------------------------------------------------------- delayed rescaling: one kernel, FP8 out
+
+def run_delayed(A, a_dt, a_s, B, b_dt, b_s, stat_in, y_dt, transB=True, stat=sc.STAT_AMAX, state=None):
+    M = A.shape[0]
+    N = B.shape[0] if transB else B.shape[1]
+    Y = sc.ScaledTensor.empty((M, N), sc.TORCH_DTYPE[y_dt])
+    ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_MATMUL, M, N))
+    st_in = state if state is not None else torch.tensor([stat_in], dtype=torch.float32, device="cuda")
+    st_out = state if state is not None else torch.zeros(1, dtype=torch.float32, device="cuda")
+    sc.scalify_scaled_matmul_delayed(sc.ScaledTensor.make(to_dev(A, a_dt), a_s), sc.ScaledTensor.make(to_dev(B, b_dt), b_s),
+                                     st_in, Y, ws, transB=transB, stat=stat, stat_out=st_out)
+    status = ws.check_status()
+    return to_bits(Y.data, y_dt), Y.scale_value(), float(st_out.item()), status
+
+
+@pytest.mark.parametrize("a_dt,y_dt", [(orc.E4M3, orc.E4M3), (orc.E5M2, orc.E5M2), (orc.E4M3, orc.BF16)])
+@pytest.mark.parametrize("stat", [sc.STAT_AMAX, sc.STAT_L2])
+def test_delayed_rescale_matmul_single_pass_fp8_output(a_dt, y_dt, stat):
+    M, N, K = 384, 528, 1040
+    A = si.scaled_normal(26, 1, (M, K), a_dt)
+    Bt = si.scaled_normal(26, 2, (N, K), orc.E4M3)
+    for stat_in in (5.3, 0.07, 0.0):
+        got, gs, gstat, status = run_delayed(A, a_dt, 2.0 ** -10, Bt, orc.E4M3, 2.0 ** -6, stat_in, y_dt, stat=stat)
+        assert status == 0
+        Yo, ys, so = orc.scaled_matmul_delayed(A, a_dt, 2.0 ** -10, Bt, orc.E4M3, 2.0 ** -6, stat_in, stat, y_dt,
+                                               transB=True)
+        assert gs == ys
+        assert abs(gstat - so) <= 2e-5 * so
+        _, _, acc, sab = orc.scaled_matmul(A, a_dt, 2.0 ** -10, Bt, orc.E4M3, 2.0 ** -6, orc.F32, transB=True,
+                                           want_acc=True)
+        r = orc.p2f(stat_in) if stat_in >= 2.0 ** -126 else 1.0
+        assert within(got, Yo, y_dt, acc / r, sab / r, 1e-5).all()
+        # bit-exact against the encoding of the library's own fp32 values
+        g32, _, _, _ = run_delayed(A, a_dt, 2.0 ** -10, Bt, orc.E4M3, 2.0 ** -6, stat_in, orc.F32, stat=stat)
+        assert np.array_equal(got, orc.encode(orc.decode(g32, orc.F32), y_dt))
+
+
+def test_delayed_rescale_state_word_updated_in_place_over_steps():
+    M, N, K = 256, 256, 512
+    state = torch.tensor([1.0], dtype=torch.float32, device="cuda")  # initial guess of the statistic
+    prev = 1.0
+    for step in range(3):
+        A = si.scaled_normal(27, 10 + step, (M, K), orc.E4M3, 1.0 + step)  # the data grow from step to step
+        Bt = si.scaled_normal(27, 20 + step, (N, K), orc.E4M3)
+        got, gs, gstat, status = run_delayed(A, orc.E4M3, 1.0, Bt, orc.E4M3, 1.0, None, orc.E4M3, state=state)
+        Yo, ys, so = orc.scaled_matmul_delayed(A, orc.E4M3, 1.0, Bt, orc.E4M3, 1.0, prev, orc.STAT_AMAX, orc.E4M3,
+                                               transB=True)
+        assert status == 0 and gs == ys and abs(gstat - so) <= 2e-5 * so
+        assert ulp_diff(got, Yo, orc.E4M3).max() <= 1
+        prev = gstat  # the library's own statistic drives the next step on both sides
+
+
+def test_delayed_rescale_nonfinite_statistic_is_flagged_and_ignored():
+    A = si.scaled_normal(28, 1, (128, 128), orc.E4M3)
+    Bt = si.scaled_normal(28, 2, (256, 128), orc.E4M3)
+    got, gs, gstat, status = run_delayed(A, orc.E4M3, 1.0, Bt, orc.E4M3, 1.0, float("inf"), orc.BF16)
+    assert status == sc.DEV_NONFINITE_STAT
+    Yo, ys, _ = orc.scaled_matmul_delayed(A, orc.E4M3, 1.0, Bt, orc.E4M3, 1.0, float("inf"), orc.STAT_AMAX, orc.BF16,
+                                          transB=True)
+    assert gs == ys and ulp_diff(got, Yo, orc.BF16).max() <= 1
+
+
+def test_delayed_rescale_full_size_8192_sampled():
+    n = 8192
+    c = si.gemm_case(n, "fwd", seed=2)
+    stat_in = 6.0
+    got, gs, gstat, status = run_delayed(c["A"], orc.E4M3, c["a_scale"], c["Bt"], orc.E4M3, c["b_scale"], stat_in, orc.E4M3)
+    assert status == 0 and gs == c["a_scale"] * c["b_scale"] * orc.kf(n) * 4.0
+    rng = np.random.default_rng(6)
+    rows = np.concatenate([rng.integers(0, n, 2000), [0, n - 1, 255, 256]])
+    cols = np.concatenate([rng.integers(0, n, 2000), [0, n - 1, 255, 256]])
+    acc, sab = orc.scaled_matmul_samples(c["A"], orc.E4M3, c["Bt"], orc.E4M3, rows, cols, transB=True)
+    want = orc.encode(acc / 4.0, orc.E4M3)
+    assert within(got[rows, cols], want, orc.E4M3, acc / 4.0, sab / 4.0, 1e-5).all()
+    # the statistic is the AMAX of the un-rebalanced values: at least the max over the sample, and
+    # consistent with the stored FP8 data (|data| * r <= stat rounded up by one FP8 ulp)
+    assert gstat >= np.abs(acc).max() * (1 - 1e-5)
+    stored_max = float(torch.from_numpy(got).view(torch.float8_e4m3fn).float().abs().max()) * 4.0
+    assert stored_max * (1 - 2.0 ** -4) <= gstat <= stored_max * (1 + 2.0 ** -4)
