@@ -75,6 +75,12 @@ def lib() -> ctypes.CDLL:
                                         i32, vp, pf32, i32, vp, pf32, vp, pf32, vp]
         L.orc_gelu_fwd.argtypes = [vp, i32, f32, i64, i32, i32, vp, pf32]
         L.orc_gelu_bwd.argtypes = [vp, i32, f32, vp, i32, f32, i64, i32, i32, vp, pf32]
+        L.orc_embedding_fwd.argtypes = [vp, i64, i64, i64, vp, i32, f32, vp, i32, f32, i32, vp, pf32]
+        L.orc_embedding_bwd.argtypes = [vp, i64, i64, i64, i64, vp, i32, f32, i32, vp, pf32, vp, pf32]
+        L.orc_softmax_fwd.argtypes = [vp, i32, f32, i64, i64, i64, i32, i32, vp, pf32]
+        L.orc_softmax_bwd.argtypes = [vp, i32, f32, vp, i32, f32, i64, i64, i32, vp, pf32]
+        L.orc_cross_entropy.restype = f64
+        L.orc_cross_entropy.argtypes = [vp, i32, f32, i64, i64, i64, vp, i32, vp, pf32]
         L.orc_adam_step.argtypes = [i64, vp, i32, f32, vp, vp, i32, pf32, pf32, vp, i32, pf32,
                                     f32, f32, f32, f32, i64]
         _lib = L
@@ -285,3 +291,61 @@ def adam_step(g, g_dtype, g_scale, m, v, mv_dtype, m_scale, v_scale, w, w_dtype,
                         ctypes.byref(ms), ctypes.byref(vs), _ptr(w2), w_dtype, ctypes.byref(ws),
                         float(lr), float(beta1), float(beta2), float(eps), int(step))
     return m2, v2, w2, float(ms.value), float(vs.value), float(ws.value)
+
+
+def embedding_fwd(ids, seq_len, wte, wte_dtype, wte_scale, wpe, wpe_dtype, wpe_scale, y_dtype):
+    ids = np.ascontiguousarray(ids, dtype=np.int64)
+    wte = _bits(wte, wte_dtype)
+    wpe = None if wpe is None else _bits(wpe, wpe_dtype)
+    d = wte.shape[1]
+    Y = np.empty((ids.size, d), dtype=_BITS_NP[y_dtype])
+    ys = ctypes.c_float(0)
+    lib().orc_embedding_fwd(_ptr(ids), ids.size, int(seq_len), d, _ptr(wte), wte_dtype, float(wte_scale), _ptr(wpe),
+                            wpe_dtype, float(wpe_scale), y_dtype, _ptr(Y), ctypes.byref(ys))
+    return Y, float(ys.value)
+
+
+def embedding_bwd(ids, seq_len, vocab, dY, dy_dtype, dy_scale, out_dtype, want_wpe=True):
+    ids = np.ascontiguousarray(ids, dtype=np.int64)
+    dY = _bits(dY, dy_dtype)
+    d = dY.shape[1]
+    dwte = np.empty((vocab, d), dtype=_BITS_NP[out_dtype])
+    dwpe = np.empty((seq_len, d), dtype=_BITS_NP[out_dtype]) if want_wpe else None
+    s1, s2 = ctypes.c_float(0), ctypes.c_float(0)
+    lib().orc_embedding_bwd(_ptr(ids), ids.size, int(seq_len), d, int(vocab), _ptr(dY), dy_dtype, float(dy_scale),
+                            out_dtype, _ptr(dwte), ctypes.byref(s1), _ptr(dwpe), ctypes.byref(s2))
+    return dwte, float(s1.value), dwpe, float(s2.value)
+
+
+def softmax_fwd(S, s_dtype, s_scale, causal, p_dtype):
+    S = _bits(S, s_dtype)
+    Tq, Tk = S.shape[-2], S.shape[-1]
+    batch = S.size // (Tq * Tk)
+    P = np.empty(S.shape, dtype=_BITS_NP[p_dtype])
+    ps = ctypes.c_float(0)
+    lib().orc_softmax_fwd(_ptr(S), s_dtype, float(s_scale), batch, Tq, Tk, int(causal), p_dtype, _ptr(P),
+                          ctypes.byref(ps))
+    return P, float(ps.value)
+
+
+def softmax_bwd(dP, dp_dtype, dp_scale, P, p_dtype, p_scale, ds_dtype):
+    dP = _bits(dP, dp_dtype)
+    P = _bits(P, p_dtype)
+    Tk = P.shape[-1]
+    dS = np.empty(P.shape, dtype=_BITS_NP[ds_dtype])
+    ss = ctypes.c_float(0)
+    lib().orc_softmax_bwd(_ptr(dP), dp_dtype, float(dp_scale), _ptr(P), p_dtype, float(p_scale), P.size // Tk, Tk,
+                          ds_dtype, _ptr(dS), ctypes.byref(ss))
+    return dS, float(ss.value)
+
+
+def cross_entropy(logits, l_dtype, l_scale, n_classes, targets, g_dtype=None):
+    """Returns (mean loss, dlogits bits or None, dlogits scale)."""
+    logits = _bits(logits, l_dtype)
+    n, ld = logits.shape
+    targets = np.ascontiguousarray(targets, dtype=np.int64)
+    g = None if g_dtype is None else np.empty((n, ld), dtype=_BITS_NP[g_dtype])
+    gs = ctypes.c_float(0)
+    loss = lib().orc_cross_entropy(_ptr(logits), l_dtype, float(l_scale), n, int(n_classes), ld, _ptr(targets),
+                                   0 if g_dtype is None else g_dtype, _ptr(g), ctypes.byref(gs))
+    return float(loss), g, float(gs.value)

@@ -24,9 +24,10 @@
 // Parity pins: every function below is pinned by tests/test_oracle_*.py
 // (exhaustive codec round trips, comparison of the codecs with an independent
 // library cast, brute force on tiny matrices, closed forms, invariants,
-// finite differences, textbook Adam / LayerNorm).  The rules for attention /
-// softmax / cross-entropy are not part of this file.
+// finite differences, textbook Adam / LayerNorm; tests/test_oracle_support_ops.py pins
+// the embedding / softmax / cross-entropy readings against torch in fp64).
 
+#include <algorithm>
 #include <cmath>
 #include <cstdint>
 #include <cstring>
@@ -521,6 +522,123 @@ void orc_gelu_bwd(const void* G, int g_dtype, float g_scale, const void* X, int 
     store_bits(dX, y_dtype, i, encode(gd * fp, y_dtype));
   }
   if (dx_scale) *dx_scale = g_scale;
+}
+
+// ---- support operations of a GPT-style training step.  The paper gives no rule for attention,
+// softmax or the loss (Section 3.2.1 only says custom rules are possible there); these are the
+// readings this repository takes, stated in value space so that model invariance (Section 1) can
+// be checked against a plain unscaled implementation.
+
+// Embedding lookup: Y = wte[ids] + wpe[pos], pos = i mod seq_len, through the add rule.
+void orc_embedding_fwd(const int64_t* ids, int64_t n, int64_t seq_len, int64_t d,
+                       const void* wte, int wte_dtype, float wte_scale, const void* wpe, int wpe_dtype, float wpe_scale,
+                       int y_dtype, void* Y, float* y_scale) {
+  const double ts = wte_scale, ps = wpe ? static_cast<double>(wpe_scale) : 0.0;
+  const double ys = p2f(std::sqrt(ts * ts + ps * ps));
+  for (int64_t i = 0; i < n; ++i)
+    for (int64_t j = 0; j < d; ++j) {
+      double v = decode(load_bits(wte, wte_dtype, ids[i] * d + j), wte_dtype) * (ts / ys);
+      if (wpe) v += decode(load_bits(wpe, wpe_dtype, (i % seq_len) * d + j), wpe_dtype) * (ps / ys);
+      store_bits(Y, y_dtype, i * d + j, encode(v, y_dtype));
+    }
+  if (y_scale) *y_scale = static_cast<float>(ys);
+}
+
+// Embedding backward: dwte[v] = sum of the gradient rows whose token is v (scale unchanged: the
+// number of addends per row is data dependent, so no static factor is applied and the sum is kept in
+// a wide output format); dwpe[p] = sum over the n/seq_len sequences, a reduction of known size B,
+// divided by kf(B) with scale dY_s*kf(B).
+void orc_embedding_bwd(const int64_t* ids, int64_t n, int64_t seq_len, int64_t d, int64_t vocab,
+                       const void* dY, int dy_dtype, float dy_scale, int out_dtype,
+                       void* dwte, float* dwte_scale, void* dwpe, float* dwpe_scale) {
+  std::vector<double> te(static_cast<size_t>(vocab * d), 0.0), pe(static_cast<size_t>(seq_len * d), 0.0);
+  for (int64_t i = 0; i < n; ++i)
+    for (int64_t j = 0; j < d; ++j) {
+      const double g = decode(load_bits(dY, dy_dtype, i * d + j), dy_dtype);
+      te[ids[i] * d + j] += g;
+      pe[(i % seq_len) * d + j] += g;
+    }
+  const double f = kf(n / seq_len);
+  for (int64_t k = 0; k < vocab * d; ++k) store_bits(dwte, out_dtype, k, encode(te[k], out_dtype));
+  if (dwpe)
+    for (int64_t k = 0; k < seq_len * d; ++k) store_bits(dwpe, out_dtype, k, encode(pe[k] / f, out_dtype));
+  if (dwte_scale) *dwte_scale = dy_scale;
+  if (dwpe_scale) *dwpe_scale = static_cast<float>(static_cast<double>(dy_scale) * f);
+}
+
+// Row softmax of the VALUES S_d*S_s with an optional causal mask (row i of each [Tq,Tk] matrix sees
+// columns j <= i + Tk - Tq); the probabilities are bounded in [0,1] and carry scale 1, like the gate
+// of an activation (Appendix C.1).  Masked positions are exactly 0.
+void orc_softmax_fwd(const void* S, int s_dtype, float s_scale, int64_t batch, int64_t Tq, int64_t Tk, int causal,
+                     int p_dtype, void* P, float* p_scale) {
+  for (int64_t b = 0; b < batch; ++b)
+    for (int64_t i = 0; i < Tq; ++i) {
+      const int64_t lim = causal ? std::min<int64_t>(Tk, i + Tk - Tq + 1) : Tk;
+      const int64_t off = (b * Tq + i) * Tk;
+      double mx = -std::numeric_limits<double>::infinity();
+      for (int64_t j = 0; j < lim; ++j)
+        mx = std::max(mx, decode(load_bits(S, s_dtype, off + j), s_dtype) * static_cast<double>(s_scale));
+      double sum = 0.0;
+      for (int64_t j = 0; j < lim; ++j)
+        sum += std::exp(decode(load_bits(S, s_dtype, off + j), s_dtype) * static_cast<double>(s_scale) - mx);
+      for (int64_t j = 0; j < Tk; ++j) {
+        double p = 0.0;
+        if (j < lim) p = std::exp(decode(load_bits(S, s_dtype, off + j), s_dtype) * static_cast<double>(s_scale) - mx) / sum;
+        store_bits(P, p_dtype, off + j, encode(p, p_dtype));
+      }
+    }
+  if (p_scale) *p_scale = 1.0f;
+}
+
+// Softmax backward in value space: dS = P * (dP - sum_j dP_j P_j); the Jacobian is bounded by 1, so
+// the gradient scale passes through unchanged (dS_s = dP_s * P_s), as for activations.
+void orc_softmax_bwd(const void* dP, int dp_dtype, float dp_scale, const void* P, int p_dtype, float p_scale,
+                     int64_t rows, int64_t Tk, int ds_dtype, void* dS, float* ds_scale) {
+  for (int64_t r = 0; r < rows; ++r) {
+    double dot = 0.0;
+    for (int64_t j = 0; j < Tk; ++j)
+      dot += decode(load_bits(dP, dp_dtype, r * Tk + j), dp_dtype) * decode(load_bits(P, p_dtype, r * Tk + j), p_dtype);
+    for (int64_t j = 0; j < Tk; ++j) {
+      const double p = decode(load_bits(P, p_dtype, r * Tk + j), p_dtype);
+      const double g = decode(load_bits(dP, dp_dtype, r * Tk + j), dp_dtype);
+      store_bits(dS, ds_dtype, r * Tk + j, encode(p * (g - dot), ds_dtype));
+    }
+  }
+  if (ds_scale) *ds_scale = static_cast<float>(static_cast<double>(dp_scale) * static_cast<double>(p_scale));
+}
+
+// Mean cross-entropy of the VALUES z = logits_d*logits_s over n rows and the first n_classes columns
+// (row stride ld >= n_classes; padding columns are ignored and receive zero gradient), through
+// logsumexp (Appendix B).  Gradient w.r.t. the logits' values: (softmax(z) - onehot)/n, written as
+// data softmax - onehot in [-1,1] with scale 1/n rounded down to a power of two times the remainder
+// folded into the data.  Returns the loss.
+double orc_cross_entropy(const void* logits, int l_dtype, float l_scale, int64_t n, int64_t n_classes, int64_t ld,
+                         const int64_t* targets, int g_dtype, void* dlogits, float* g_scale) {
+  const double inv_n = 1.0 / static_cast<double>(n);
+  const double gs = p2f(inv_n);
+  const double rem = inv_n / gs;  // in [1,2): kept in the data
+  double loss = 0.0;
+  for (int64_t i = 0; i < n; ++i) {
+    double mx = -std::numeric_limits<double>::infinity();
+    for (int64_t j = 0; j < n_classes; ++j)
+      mx = std::max(mx, decode(load_bits(logits, l_dtype, i * ld + j), l_dtype) * static_cast<double>(l_scale));
+    double sum = 0.0;
+    for (int64_t j = 0; j < n_classes; ++j)
+      sum += std::exp(decode(load_bits(logits, l_dtype, i * ld + j), l_dtype) * static_cast<double>(l_scale) - mx);
+    const double zt = decode(load_bits(logits, l_dtype, i * ld + targets[i]), l_dtype) * static_cast<double>(l_scale);
+    loss += (mx + std::log(sum)) - zt;
+    if (dlogits)
+      for (int64_t j = 0; j < ld; ++j) {
+        double g = 0.0;
+        if (j < n_classes) {
+          g = std::exp(decode(load_bits(logits, l_dtype, i * ld + j), l_dtype) * static_cast<double>(l_scale) - mx) / sum;
+          if (j == targets[i]) g -= 1.0;
+        }
+        store_bits(dlogits, g_dtype, i * ld + j, encode(g * rem, g_dtype));
+      }
+  }
+  if (g_scale) *g_scale = static_cast<float>(gs);
+  return loss * inv_n;
 }
 
 // Scaled Adam step.  The paper states only that the optimizer update is traced
