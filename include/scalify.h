@@ -78,7 +78,8 @@ typedef enum {
 enum {
   SCALIFY_DEV_TIMEOUT = 1u,        /* a bounded device-side wait expired; results of that call are invalid */
   SCALIFY_DEV_BAD_SCALE = 2u,      /* an input scale word was not a finite positive power of two */
-  SCALIFY_DEV_NONFINITE_STAT = 4u  /* a statistic was NaN or Inf; the rescale used factor 1 */
+  SCALIFY_DEV_NONFINITE_STAT = 4u, /* a statistic was NaN or Inf; the rescale used factor 1 */
+  SCALIFY_DEV_BAD_INDEX = 8u       /* a token id or target was out of range (treated as 0) */
 };
 
 typedef struct scalify_array {
@@ -96,7 +97,8 @@ enum {
   SCALIFY_OP_RESCALE = 1,       /* d0 = number of elements, d1 unused */
   SCALIFY_OP_LAYERNORM_BWD = 2, /* d0 = rows, d1 = row length */
   SCALIFY_OP_ADAM = 3,          /* d0 = number of tensors, d1 unused */
-  SCALIFY_OP_STATISTIC = 4      /* d0 = number of elements */
+  SCALIFY_OP_STATISTIC = 4,     /* d0 = number of elements */
+  SCALIFY_OP_CROSS_ENTROPY = 5  /* d0 = number of rows */
 };
 
 /* Bytes of workspace the given call needs (an upper bound; always >= 4096).
@@ -259,6 +261,49 @@ int scalify_scaled_layernorm_bwd(const scalify_array* G, const scalify_array* X,
 int scalify_scaled_gelu(const scalify_array* X, int exact_erf, scalify_array* Y, void* stream);
 int scalify_scaled_gelu_bwd(const scalify_array* G, const scalify_array* X, int exact_erf,
                             scalify_array* dX, void* stream);
+
+/*
+ * Support operations of a GPT-style training step.  The paper states no scale rule for these
+ * (Section 3.2.1 only says that custom rules suit attention layers); the rules below are this
+ * library's readings, chosen so that values follow the unscaled network exactly (model invariance,
+ * Section 1) and bounded quantities carry scale 1 (as the gate of an activation, Appendix C.1).
+ *
+ * Embedding lookup through the add rule:  Y[i] = wte[ids[i]] + wpe[i mod seq_len],
+ *   Y_s = max(wte_s, wpe_s).  ids: DEVICE int64 [n]; wte [vocab,d], wpe [>=seq_len,d] or NULL, same
+ *   16/32-bit dtype; Y [n,d] any dtype; d*elem_size a multiple of 16 bytes.  An id outside
+ *   [0,vocab) sets SCALIFY_DEV_BAD_INDEX in *status (optional device word) and reads row 0.
+ * Backward: dwte[v] = sum of the rows of dY whose id is v, scale dY_s (the number of addends is data
+ *   dependent, so no static factor; fp32 atomics, order not fixed); dwpe[p] = sum over the
+ *   n/seq_len sequences divided by kf(n/seq_len), scale dY_s*kf(n/seq_len).  dwte [vocab,d] and
+ *   dwpe [seq_len,d] (or NULL) are F32 and fully overwritten.
+ */
+int scalify_scaled_embedding(const int64_t* ids, int64_t n, int64_t seq_len, const scalify_array* wte,
+                             const scalify_array* wpe, scalify_array* Y, uint32_t* status, void* stream);
+int scalify_scaled_embedding_bwd(const int64_t* ids, int64_t n, int64_t seq_len, const scalify_array* dY,
+                                 scalify_array* dwte, scalify_array* dwpe, void* stream);
+
+/*
+ * Row softmax of the VALUES S_d*S_s over the last dimension, optionally causal (row i of each
+ * [Tq,Tk] matrix attends to columns j <= i + Tk - Tq; requires Tk >= Tq); P_d in [0,1], P_s = 1,
+ * masked entries exactly 0.  S: [Tq,Tk] or [batch,Tq,Tk], F16/BF16/F32, contiguous, Tk*elem_size a
+ * multiple of 16 bytes and at most 4096 bytes; P: same shape, any dtype.
+ * Backward: dS_d = P_d*(dP_d - sum_j dP_d[j] P_d[j]), dS_s = dP_s*P_s (the Jacobian is bounded by 1,
+ * so the gradient scale passes through).  dP: F16/BF16/F32; P: E4M3/F16/BF16/F32; dS any dtype.
+ */
+int scalify_scaled_softmax(const scalify_array* S, int causal, scalify_array* P, void* stream);
+int scalify_scaled_softmax_bwd(const scalify_array* dP, const scalify_array* P, scalify_array* dS, void* stream);
+
+/*
+ * Mean cross-entropy of the values z = logits_d*logits_s through logsumexp (Appendix B) over the
+ * first n_classes columns of logits [n, ld>=n_classes] (padding columns ignored), and its gradient
+ * w.r.t. the values: dlogits_d = (softmax(z) - onehot(target)) * rem, dlogits_s = 1/n rounded down
+ * to a power of two, rem = (1/n)/dlogits_s in [1,2); padding columns receive 0.
+ * logits: F16/BF16/F32 (row stride = shape[1]); targets: DEVICE int64 [n]; loss: DEVICE fp32;
+ * dlogits: same shape as logits, any dtype, or NULL.  A target outside [0,n_classes) sets
+ * SCALIFY_DEV_BAD_INDEX in the workspace status word.  Workspace: SCALIFY_OP_CROSS_ENTROPY, n.
+ */
+int scalify_scaled_cross_entropy(const scalify_array* logits, int64_t n_classes, const int64_t* targets, float* loss,
+                                 scalify_array* dlogits, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * Scaled Adam step over a list of tensors (Sections 1, 3 and 4; Table 3 row 4:

@@ -22,8 +22,8 @@ from . import _build
 
 E4M3, E5M2, F16, BF16, F32 = 0, 1, 2, 3, 4
 STAT_NONE, STAT_AMAX, STAT_L2 = 0, 1, 2
-OP_MATMUL, OP_RESCALE, OP_LAYERNORM_BWD, OP_ADAM, OP_STATISTIC = 0, 1, 2, 3, 4
-DEV_TIMEOUT, DEV_BAD_SCALE, DEV_NONFINITE_STAT = 1, 2, 4
+OP_MATMUL, OP_RESCALE, OP_LAYERNORM_BWD, OP_ADAM, OP_STATISTIC, OP_CROSS_ENTROPY = 0, 1, 2, 3, 4, 5
+DEV_TIMEOUT, DEV_BAD_SCALE, DEV_NONFINITE_STAT, DEV_BAD_INDEX = 1, 2, 4, 8
 
 _DTYPE_CODE = {torch.float8_e4m3fn: E4M3, torch.float8_e5m2: E5M2, torch.float16: F16,
                torch.bfloat16: BF16, torch.float32: F32}
@@ -75,12 +75,19 @@ def lib() -> ctypes.CDLL:
         L.scalify_scaled_gelu.argtypes = [P, i32, P, vp]
         L.scalify_scaled_gelu_bwd.argtypes = [P, P, i32, P, vp]
         L.scalify_scaled_adam_step.argtypes = [i32, P, P, P, P, f32, f32, f32, f32, i64, vp, sz, vp]
+        L.scalify_scaled_embedding.argtypes = [vp, i64, i64, P, P, P, vp, vp]
+        L.scalify_scaled_embedding_bwd.argtypes = [vp, i64, i64, P, P, P, vp]
+        L.scalify_scaled_softmax.argtypes = [P, i32, P, vp]
+        L.scalify_scaled_softmax_bwd.argtypes = [P, P, P, vp]
+        L.scalify_scaled_cross_entropy.argtypes = [P, i64, vp, vp, P, vp, sz, vp]
         L.scalify_scaled_adam_step_static.argtypes = [i32, P, P, P, P, f32, f32, f32, f32, i64, vp, vp]
         for name in ("scalify_workspace_init", "scalify_check_status", "scalify_scaled_matmul", "scalify_scaled_matmul_delayed",
                      "scalify_statistic",
                      "scalify_rescale", "scalify_scaled_add", "scalify_scaled_layernorm",
                      "scalify_scaled_layernorm_bwd", "scalify_scaled_gelu", "scalify_scaled_gelu_bwd",
-                     "scalify_scaled_adam_step", "scalify_scaled_adam_step_static"):
+                     "scalify_scaled_adam_step", "scalify_scaled_adam_step_static", "scalify_scaled_embedding",
+                     "scalify_scaled_embedding_bwd", "scalify_scaled_softmax", "scalify_scaled_softmax_bwd",
+                     "scalify_scaled_cross_entropy"):
             getattr(L, name).restype = i32
         _lib = L
     return _lib
@@ -281,3 +288,37 @@ def scalify_scaled_adam_step_static(tensors: AdamTensors, *, lr: float, beta1: f
                                                  float(beta1), float(beta2), float(eps), int(step),
                                                  _ptr(status_out), _stream(stream)),
            "scalify_scaled_adam_step_static")
+
+
+def scalify_scaled_embedding(ids: torch.Tensor, seq_len: int, wte: ScaledTensor, wpe: Optional[ScaledTensor],
+                             Y: ScaledTensor, *, status: Optional[torch.Tensor] = None, stream=None) -> None:
+    assert ids.dtype == torch.int64 and ids.is_contiguous()
+    a, b, y = _desc(wte), _desc(wpe), _desc(Y)
+    _check(lib().scalify_scaled_embedding(ids.data_ptr(), ids.numel(), int(seq_len), _ref(a), _ref(b), _ref(y),
+                                          _ptr(status), _stream(stream)), "scalify_scaled_embedding")
+
+
+def scalify_scaled_embedding_bwd(ids: torch.Tensor, seq_len: int, dY: ScaledTensor, dwte: ScaledTensor,
+                                 dwpe: Optional[ScaledTensor], *, stream=None) -> None:
+    assert ids.dtype == torch.int64 and ids.is_contiguous()
+    g, a, b = _desc(dY), _desc(dwte), _desc(dwpe)
+    _check(lib().scalify_scaled_embedding_bwd(ids.data_ptr(), ids.numel(), int(seq_len), _ref(g), _ref(a), _ref(b),
+                                              _stream(stream)), "scalify_scaled_embedding_bwd")
+
+
+def scalify_scaled_softmax(S: ScaledTensor, P: ScaledTensor, *, causal=False, stream=None) -> None:
+    s, p = _desc(S), _desc(P)
+    _check(lib().scalify_scaled_softmax(_ref(s), int(causal), _ref(p), _stream(stream)), "scalify_scaled_softmax")
+
+
+def scalify_scaled_softmax_bwd(dP: ScaledTensor, P: ScaledTensor, dS: ScaledTensor, *, stream=None) -> None:
+    g, p, o = _desc(dP), _desc(P), _desc(dS)
+    _check(lib().scalify_scaled_softmax_bwd(_ref(g), _ref(p), _ref(o), _stream(stream)), "scalify_scaled_softmax_bwd")
+
+
+def scalify_scaled_cross_entropy(logits: ScaledTensor, n_classes: int, targets: torch.Tensor, loss: torch.Tensor,
+                                 dlogits: Optional[ScaledTensor], ws: Workspace, *, stream=None) -> None:
+    assert targets.dtype == torch.int64 and targets.is_contiguous() and loss.dtype == torch.float32
+    l, g = _desc(logits), _desc(dlogits)
+    _check(lib().scalify_scaled_cross_entropy(_ref(l), int(n_classes), targets.data_ptr(), loss.data_ptr(), _ref(g),
+                                              ws.ptr, ws.nbytes, _stream(stream)), "scalify_scaled_cross_entropy")

@@ -108,6 +108,7 @@ size_t scalify_workspace_bytes(int op, int64_t d0, int64_t d1) {
     case SCALIFY_OP_STATISTIC: n = stat_bytes; break;
     case SCALIFY_OP_LAYERNORM_BWD: n = layernorm_bwd_ws_bytes(d0, d1); break;
     case SCALIFY_OP_ADAM: n = adam_ws_bytes(d0); break;
+    case SCALIFY_OP_CROSS_ENTROPY: n = cross_entropy_ws_bytes(d0); break;
     default: break;
   }
   if (n < stat_bytes) n = stat_bytes;
@@ -489,6 +490,116 @@ int scalify_scaled_matmul_delayed(const scalify_array* A, int transA, const scal
   if (stat_out)
     SCALIFY_CUDA_TRY(cudaMemcpyAsync(stat_out, ws_view(workspace).stat, sizeof(float), cudaMemcpyDeviceToDevice, st));
   return SCALIFY_OK;
+}
+
+int scalify_scaled_embedding(const int64_t* ids, int64_t n, int64_t seq_len, const scalify_array* wte,
+                             const scalify_array* wpe, scalify_array* Y, uint32_t* status, void* stream) {
+  if (!ids) return SCALIFY_ERR_NULL;
+  int rc = check_array(wte);
+  if (rc) return rc;
+  rc = check_array(Y);
+  if (rc) return rc;
+  if (!is_wide(wte->dtype) || wte->ndim != 2 || Y->ndim != 2) return SCALIFY_ERR_DTYPE;
+  const int64_t vocab = wte->shape[0], d = wte->shape[1];
+  if (n < 1 || seq_len < 1 || n % seq_len != 0 || d < 1 || d > 0x7FFFFFFF || seq_len > 0x7FFFFFFF) return SCALIFY_ERR_SHAPE;
+  if (Y->shape[0] != n || Y->shape[1] != d || contiguous_numel(wte) != vocab * d || contiguous_numel(Y) != n * d)
+    return SCALIFY_ERR_SHAPE;
+  if ((d * elem_size(wte->dtype)) % 16 != 0) return SCALIFY_ERR_SHAPE;
+  if (wpe) {
+    rc = check_array(wpe);
+    if (rc) return rc;
+    if (wpe->dtype != wte->dtype) return SCALIFY_ERR_DTYPE;
+    if (wpe->ndim != 2 || wpe->shape[0] < seq_len || wpe->shape[1] != d || wpe->stride[0] != d) return SCALIFY_ERR_SHAPE;
+  }
+  if (Y->scale && (Y->scale == wte->scale || (wpe && Y->scale == wpe->scale))) return SCALIFY_ERR_ALIAS;
+  return launch_embedding_fwd(reinterpret_cast<const long long*>(ids), n, static_cast<int>(seq_len), static_cast<int>(d),
+                              vocab, wte->data, wpe ? wpe->data : nullptr, wte->dtype, wte->scale,
+                              wpe ? wpe->scale : nullptr, Y->data, Y->dtype, Y->scale, status,
+                              static_cast<cudaStream_t>(stream));
+}
+
+int scalify_scaled_embedding_bwd(const int64_t* ids, int64_t n, int64_t seq_len, const scalify_array* dY,
+                                 scalify_array* dwte, scalify_array* dwpe, void* stream) {
+  if (!ids) return SCALIFY_ERR_NULL;
+  int rc = check_array(dY);
+  if (rc) return rc;
+  rc = check_array(dwte);
+  if (rc) return rc;
+  if (!is_wide(dY->dtype) || dwte->dtype != SCALIFY_F32) return SCALIFY_ERR_DTYPE;
+  if (dY->ndim != 2 || dwte->ndim != 2) return SCALIFY_ERR_SHAPE;
+  const int64_t d = dY->shape[1], vocab = dwte->shape[0];
+  if (n < 1 || seq_len < 1 || n % seq_len != 0 || dY->shape[0] != n || dwte->shape[1] != d || d > 0x7FFFFFFF ||
+      seq_len > 0x7FFFFFFF)
+    return SCALIFY_ERR_SHAPE;
+  if (contiguous_numel(dY) != n * d || contiguous_numel(dwte) != vocab * d) return SCALIFY_ERR_SHAPE;
+  if ((d * elem_size(dY->dtype)) % 16 != 0) return SCALIFY_ERR_SHAPE;
+  if (dwpe) {
+    rc = check_array(dwpe);
+    if (rc) return rc;
+    if (dwpe->dtype != SCALIFY_F32) return SCALIFY_ERR_DTYPE;
+    if (dwpe->ndim != 2 || dwpe->shape[0] != seq_len || dwpe->shape[1] != d || contiguous_numel(dwpe) != seq_len * d)
+      return SCALIFY_ERR_SHAPE;
+  }
+  return launch_embedding_bwd(reinterpret_cast<const long long*>(ids), n, static_cast<int>(seq_len), static_cast<int>(d),
+                              vocab, dY->data, dY->dtype, dY->scale, static_cast<float*>(dwte->data), dwte->scale,
+                              dwpe ? static_cast<float*>(dwpe->data) : nullptr, dwpe ? dwpe->scale : nullptr,
+                              static_cast<cudaStream_t>(stream));
+}
+
+int scalify_scaled_softmax(const scalify_array* S, int causal, scalify_array* P, void* stream) {
+  int rc = check_array(S);
+  if (rc) return rc;
+  rc = check_array(P);
+  if (rc) return rc;
+  if (!is_wide(S->dtype)) return SCALIFY_ERR_DTYPE;
+  if (S->ndim < 2 || !same_shape(S, P)) return SCALIFY_ERR_SHAPE;
+  const int64_t Tq = S->shape[S->ndim - 2], Tk = S->shape[S->ndim - 1];
+  const int64_t total = contiguous_numel(S);
+  if (total < 1 || contiguous_numel(P) != total || Tk > 0x7FFFFFFF || Tq > 0x7FFFFFFF) return SCALIFY_ERR_SHAPE;
+  if ((Tk * elem_size(S->dtype)) % 16 != 0 || (causal && Tk < Tq)) return SCALIFY_ERR_SHAPE;
+  if (P->scale && P->scale == S->scale) return SCALIFY_ERR_ALIAS;
+  return launch_softmax_fwd(S->data, S->dtype, P->data, P->dtype, total / Tk, static_cast<int>(Tq), static_cast<int>(Tk),
+                            causal ? 1 : 0, S->scale, P->scale, static_cast<cudaStream_t>(stream));
+}
+
+int scalify_scaled_softmax_bwd(const scalify_array* dP, const scalify_array* P, scalify_array* dS, void* stream) {
+  int rc = check_array(dP);
+  if (rc) return rc;
+  rc = check_array(P);
+  if (rc) return rc;
+  rc = check_array(dS);
+  if (rc) return rc;
+  if (!is_wide(dP->dtype)) return SCALIFY_ERR_DTYPE;
+  if (dP->ndim < 2 || !same_shape(dP, P) || !same_shape(dP, dS)) return SCALIFY_ERR_SHAPE;
+  const int64_t Tk = dP->shape[dP->ndim - 1];
+  const int64_t total = contiguous_numel(dP);
+  if (total < 1 || contiguous_numel(P) != total || contiguous_numel(dS) != total || Tk > 0x7FFFFFFF) return SCALIFY_ERR_SHAPE;
+  if ((Tk * elem_size(dP->dtype)) % 16 != 0) return SCALIFY_ERR_SHAPE;
+  if (dS->scale && (dS->scale == dP->scale || dS->scale == P->scale)) return SCALIFY_ERR_ALIAS;
+  return launch_softmax_bwd(dP->data, dP->dtype, P->data, P->dtype, dS->data, dS->dtype, total / Tk, static_cast<int>(Tk),
+                            dP->scale, P->scale, dS->scale, static_cast<cudaStream_t>(stream));
+}
+
+int scalify_scaled_cross_entropy(const scalify_array* logits, int64_t n_classes, const int64_t* targets, float* loss,
+                                 scalify_array* dlogits, void* workspace, size_t workspace_bytes, void* stream) {
+  int rc = check_array(logits);
+  if (rc) return rc;
+  if (!targets || !loss) return SCALIFY_ERR_NULL;
+  if (!is_wide(logits->dtype) || logits->ndim != 2) return SCALIFY_ERR_DTYPE;
+  const int64_t n = logits->shape[0], ld = logits->shape[1];
+  if (n < 1 || n_classes < 1 || n_classes > ld || n_classes > 0x7FFFFFFF || logits->stride[0] != ld) return SCALIFY_ERR_SHAPE;
+  if (dlogits) {
+    rc = check_array(dlogits);
+    if (rc) return rc;
+    if (!same_shape(logits, dlogits) || dlogits->stride[0] != ld) return SCALIFY_ERR_SHAPE;
+    if (dlogits->scale && dlogits->scale == logits->scale) return SCALIFY_ERR_ALIAS;
+  }
+  rc = check_ws(workspace, workspace_bytes, scalify_workspace_bytes(SCALIFY_OP_CROSS_ENTROPY, n, 0));
+  if (rc) return rc;
+  return launch_cross_entropy(logits->data, logits->dtype, ld, static_cast<int>(n_classes),
+                              reinterpret_cast<const long long*>(targets), n, logits->scale, loss,
+                              dlogits ? dlogits->data : nullptr, dlogits ? dlogits->dtype : SCALIFY_F32,
+                              dlogits ? dlogits->scale : nullptr, workspace, static_cast<cudaStream_t>(stream));
 }
 
 }  // extern "C"

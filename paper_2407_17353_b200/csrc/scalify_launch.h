@@ -33,6 +33,21 @@ int launch_adam(int n_tensors, const scalify_array* grads, scalify_array* m, sca
                 const int64_t* numel, float lr, float beta1, float beta2, float eps, int64_t step, void* ws,
                 cudaStream_t st);
 
+int launch_embedding_fwd(const long long* ids, long long n, int seq_len, int d, long long vocab, const void* wte,
+                         const void* wpe, int w_dt, const float* wte_scale, const float* wpe_scale, void* Y, int y_dt,
+                         float* y_scale, uint32_t* status, cudaStream_t st);
+int launch_embedding_bwd(const long long* ids, long long n, int seq_len, int d, long long vocab, const void* dY, int g_dt,
+                         const float* dy_scale, float* dwte, float* dwte_scale, float* dwpe, float* dwpe_scale,
+                         cudaStream_t st);
+int launch_softmax_fwd(const void* S, int s_dt, void* P, int p_dt, long long rows, int Tq, int Tk, int causal,
+                       const float* s_scale, float* p_scale, cudaStream_t st);
+int launch_softmax_bwd(const void* dP, int g_dt, const void* P, int p_dt, void* dS, int o_dt, long long rows, int Tk,
+                       const float* dp_scale, const float* p_scale, float* ds_scale, cudaStream_t st);
+size_t cross_entropy_ws_bytes(int64_t n);
+int launch_cross_entropy(const void* logits, int l_dt, long long ld, int n_classes, const long long* targets, long long n,
+                         const float* l_scale, float* loss, void* dlogits, int g_dt, float* g_scale, void* ws,
+                         cudaStream_t st);
+
 struct MatmulArgs {
   const void* A; int a_dt; int transA; int64_t lda, a_bs;
   const void* B; int b_dt; int transB; int64_t ldb, b_bs;

@@ -1,0 +1,400 @@
+// Support kernels of a GPT-style training step around the scaled matmuls: embedding lookup and
+// its gradient, causal row softmax forward / backward, mean cross-entropy with its gradient.
+// The paper gives no scale rule for these (Section 3.2.1 only says custom rules are possible for
+// attention); the rules taken are stated with each kernel.  All arithmetic is fp32, every row is
+// read once from HBM (cross-entropy re-reads its row from L1/L2).
+#include "scalify_common.cuh"
+#include "scalify_launch.h"
+
+namespace scalify {
+
+// ---------------------------------------------------------------------------------------------
+// embedding: Y = wte[ids] + wpe[pos] through the add rule (Y_s = max of the two scales)
+// ---------------------------------------------------------------------------------------------
+template <int WDT, int YDT>
+__global__ void __launch_bounds__(256) embedding_fwd_kernel(const long long* __restrict__ ids, long long n, int seq_len,
+                                                            int d, long long vocab, const void* __restrict__ wte,
+                                                            const void* __restrict__ wpe, const float* wte_scale,
+                                                            const float* wpe_scale, void* __restrict__ Y, float* y_scale,
+                                                            uint32_t* bad_index) {
+  constexpr int VEC = 16 / ElemBytes<WDT>::v;
+  constexpr int OB = VEC * ElemBytes<YDT>::v;
+  const float ts = load_scale(wte_scale), ps = wpe ? load_scale(wpe_scale) : 0.f;
+  const float ys = fmaxf(ts, ps);
+  const float ft = ts / ys, fp = ps / ys;
+  const int n_vec = d / VEC;
+  const long long total = n * n_vec;
+  for (long long i = blockIdx.x * 256ll + threadIdx.x; i < total; i += 256ll * gridDim.x) {
+    const long long row = i / n_vec;
+    const int c = static_cast<int>(i - row * n_vec);
+    long long id = ids[row];
+    if (id < 0 || id >= vocab) {  // out-of-range token: recorded, row of zeros from the table
+      if (bad_index) atomicOr(bad_index, static_cast<uint32_t>(SCALIFY_DEV_BAD_INDEX));
+      id = 0;
+    }
+    uint32_t w[4];
+    float a[VEC], b[VEC];
+    ld_raw<16>(static_cast<const char*>(wte) + (id * d) * ElemBytes<WDT>::v + c * 16ll, w);
+    decode_vec<WDT, VEC>(w, a);
+    if (wpe) {
+      const int pos = static_cast<int>(row % seq_len);
+      ld_raw<16>(static_cast<const char*>(wpe) + (static_cast<long long>(pos) * d) * ElemBytes<WDT>::v + c * 16ll, w);
+      decode_vec<WDT, VEC>(w, b);
+#pragma unroll
+      for (int e = 0; e < VEC; ++e) a[e] = fmaf(b[e], fp, a[e] * ft);
+    } else {
+#pragma unroll
+      for (int e = 0; e < VEC; ++e) a[e] *= ft;
+    }
+    uint32_t o[OB / 4];
+    encode_vec<YDT, VEC>(a, o);
+    st_raw<OB>(static_cast<char*>(Y) + (row * d) * ElemBytes<YDT>::v + static_cast<long long>(c) * OB, o);
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0 && y_scale) *y_scale = ys;
+}
+
+// dwte[v] += rows of dY with token v (fp32 atomics; the table must have been zeroed); scale unchanged
+template <int GDT>
+__global__ void __launch_bounds__(256) embedding_bwd_scatter_kernel(const long long* __restrict__ ids, long long n, int d,
+                                                                    long long vocab, const void* __restrict__ dY,
+                                                                    float* __restrict__ dwte) {
+  constexpr int VEC = 16 / ElemBytes<GDT>::v;
+  const int n_vec = d / VEC;
+  const long long total = n * n_vec;
+  for (long long i = blockIdx.x * 256ll + threadIdx.x; i < total; i += 256ll * gridDim.x) {
+    const long long row = i / n_vec;
+    const int c = static_cast<int>(i - row * n_vec);
+    const long long id = ids[row];
+    if (id < 0 || id >= vocab) continue;
+    uint32_t w[4];
+    float g[VEC];
+    ld_raw_stream<16>(static_cast<const char*>(dY) + (row * d) * ElemBytes<GDT>::v + c * 16ll, w);
+    decode_vec<GDT, VEC>(w, g);
+    float* dst = dwte + id * d + static_cast<long long>(c) * VEC;
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) atomicAdd(dst + e, g[e]);
+  }
+}
+
+// dwpe[p] = sum over the B sequences of dY[b*T + p], divided by kf(B), scale dY_s*kf(B): fixed order
+template <int GDT>
+__global__ void __launch_bounds__(256) embedding_bwd_pos_kernel(long long n, int seq_len, int d,
+                                                                const void* __restrict__ dY, float* __restrict__ dwpe,
+                                                                const float* dy_scale, float* dwte_scale,
+                                                                float* dwpe_scale) {
+  constexpr int VEC = 16 / ElemBytes<GDT>::v;
+  const int n_vec = d / VEC;
+  const int B = static_cast<int>(n / seq_len);
+  const float f = kfactor(B);
+  const long long total = static_cast<long long>(seq_len) * n_vec;
+  if (dwpe) {
+    for (long long i = blockIdx.x * 256ll + threadIdx.x; i < total; i += 256ll * gridDim.x) {
+      const int pos = static_cast<int>(i / n_vec);
+      const int c = static_cast<int>(i - static_cast<long long>(pos) * n_vec);
+      float acc[VEC];
+#pragma unroll
+      for (int e = 0; e < VEC; ++e) acc[e] = 0.f;
+      for (int b = 0; b < B; ++b) {
+        uint32_t w[4];
+        float g[VEC];
+        ld_raw<16>(static_cast<const char*>(dY) + ((static_cast<long long>(b) * seq_len + pos) * d) * ElemBytes<GDT>::v + c * 16ll, w);
+        decode_vec<GDT, VEC>(w, g);
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) acc[e] += g[e];
+      }
+      float* dst = dwpe + static_cast<long long>(pos) * d + c * VEC;
+#pragma unroll
+      for (int e = 0; e < VEC; ++e) dst[e] = acc[e] / f;
+    }
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    const float gs = load_scale(dy_scale);
+    if (dwte_scale) *dwte_scale = gs;
+    if (dwpe_scale) *dwpe_scale = gs * f;
+  }
+}
+
+int launch_embedding_fwd(const long long* ids, long long n, int seq_len, int d, long long vocab, const void* wte,
+                         const void* wpe, int w_dt, const float* wte_scale, const float* wpe_scale, void* Y, int y_dt,
+                         float* y_scale, uint32_t* status, cudaStream_t st) {
+  const long long total = n * (d * elem_size(w_dt) / 16);
+  long long blocks = (total + 255) / 256;
+  const long long cap = static_cast<long long>(sm_count()) * 8;
+  const int grid = static_cast<int>(blocks < cap ? (blocks < 1 ? 1 : blocks) : cap);
+  SCALIFY_DISPATCH_WIDE(w_dt, WDT, SCALIFY_DISPATCH_DTYPE(y_dt, YDT,
+      embedding_fwd_kernel<WDT, YDT><<<grid, 256, 0, st>>>(ids, n, seq_len, d, vocab, wte, wpe, wte_scale, wpe_scale, Y,
+                                                           y_scale, status)));
+  SCALIFY_CUDA_TRY(cudaGetLastError());
+  return SCALIFY_OK;
+}
+
+int launch_embedding_bwd(const long long* ids, long long n, int seq_len, int d, long long vocab, const void* dY, int g_dt,
+                         const float* dy_scale, float* dwte, float* dwte_scale, float* dwpe, float* dwpe_scale,
+                         cudaStream_t st) {
+  SCALIFY_CUDA_TRY(cudaMemsetAsync(dwte, 0, static_cast<size_t>(vocab) * d * sizeof(float), st));
+  const long long total = n * (d * elem_size(g_dt) / 16);
+  long long blocks = (total + 255) / 256;
+  const long long cap = static_cast<long long>(sm_count()) * 8;
+  const int grid = static_cast<int>(blocks < cap ? (blocks < 1 ? 1 : blocks) : cap);
+  SCALIFY_DISPATCH_WIDE(g_dt, GDT, {
+    embedding_bwd_scatter_kernel<GDT><<<grid, 256, 0, st>>>(ids, n, d, vocab, dY, dwte);
+    embedding_bwd_pos_kernel<GDT><<<grid, 256, 0, st>>>(n, seq_len, d, dY, dwpe, dy_scale, dwte_scale, dwpe_scale);
+  });
+  SCALIFY_CUDA_TRY(cudaGetLastError());
+  return SCALIFY_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// row softmax of the values S_d*S_s with optional causal mask; probabilities carry scale 1
+// ---------------------------------------------------------------------------------------------
+constexpr int kSmVpt = 8;  // 16-byte vectors per lane: rows up to 256 vectors (2048 16-bit elements)
+
+template <int SDT, int PDT>
+__global__ void __launch_bounds__(128) softmax_fwd_kernel(const void* __restrict__ S, void* __restrict__ P,
+                                                          long long rows, int Tq, int Tk, int causal,
+                                                          const float* s_scale, float* p_scale) {
+  constexpr int VEC = 16 / ElemBytes<SDT>::v;
+  constexpr int OB = VEC * ElemBytes<PDT>::v;
+  const int lane = threadIdx.x & 31;
+  const long long warp = (blockIdx.x * 128ll + threadIdx.x) >> 5, n_warps = (gridDim.x * 128ll) >> 5;
+  const int n_vec = Tk / VEC;
+  const float sc2 = load_scale(s_scale) * 1.4426950408889634f;  // values in units of log2(e)
+  for (long long row = warp; row < rows; row += n_warps) {
+    const int i = static_cast<int>(row % Tq);
+    const int lim = causal ? min(Tk, i + Tk - Tq + 1) : Tk;
+    float x[kSmVpt][VEC];
+    float mx = -INFINITY;
+    const char* srow = static_cast<const char*>(S) + row * Tk * ElemBytes<SDT>::v;
+#pragma unroll
+    for (int v = 0; v < kSmVpt; ++v) {
+      const int vi = lane + v * 32;
+      if (vi < n_vec && vi * VEC < lim) {
+        uint32_t w[4];
+        ld_raw_stream<16>(srow + vi * 16ll, w);
+        decode_vec<SDT, VEC>(w, x[v]);
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) {
+          x[v][e] = (vi * VEC + e < lim) ? x[v][e] * sc2 : -INFINITY;
+          mx = fmaxf(mx, x[v][e]);
+        }
+      } else {
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) x[v][e] = -INFINITY;
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+    float sum = 0.f;
+#pragma unroll
+    for (int v = 0; v < kSmVpt; ++v)
+#pragma unroll
+      for (int e = 0; e < VEC; ++e) {
+        x[v][e] = exp2f(x[v][e] - mx);  // exp2f(-inf) = 0 for masked positions
+        sum += x[v][e];
+      }
+    sum = warp_sum_f32(sum);
+    const float inv = 1.0f / sum;
+    char* prow = static_cast<char*>(P) + row * Tk * ElemBytes<PDT>::v;
+#pragma unroll
+    for (int v = 0; v < kSmVpt; ++v) {
+      const int vi = lane + v * 32;
+      if (vi < n_vec) {
+        float o[VEC];
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) o[e] = x[v][e] * inv;
+        uint32_t ow[OB / 4];
+        encode_vec<PDT, VEC>(o, ow);
+        st_raw<OB>(prow + static_cast<long long>(vi) * OB, ow);
+      }
+    }
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0 && p_scale) *p_scale = 1.0f;
+}
+
+// dS = P*(dP - sum_j dP_j P_j), dS_s = dP_s * P_s
+template <int GDT, int PDT, int ODT>
+__global__ void __launch_bounds__(128) softmax_bwd_kernel(const void* __restrict__ dP, const void* __restrict__ P,
+                                                          void* __restrict__ dS, long long rows, int Tk,
+                                                          const float* dp_scale, const float* p_scale, float* ds_scale) {
+  constexpr int VEC = 16 / ElemBytes<GDT>::v;            // vector of the gradient dtype
+  constexpr int PB = VEC * ElemBytes<PDT>::v, OB = VEC * ElemBytes<ODT>::v;
+  const int lane = threadIdx.x & 31;
+  const long long warp = (blockIdx.x * 128ll + threadIdx.x) >> 5, n_warps = (gridDim.x * 128ll) >> 5;
+  const int n_vec = Tk / VEC;
+  for (long long row = warp; row < rows; row += n_warps) {
+    float g[kSmVpt][VEC], p[kSmVpt][VEC];
+    float dot = 0.f;
+    const char* grow = static_cast<const char*>(dP) + row * Tk * ElemBytes<GDT>::v;
+    const char* prow = static_cast<const char*>(P) + row * Tk * ElemBytes<PDT>::v;
+#pragma unroll
+    for (int v = 0; v < kSmVpt; ++v) {
+      const int vi = lane + v * 32;
+      if (vi < n_vec) {
+        uint32_t wg[4], wp[PB / 4];
+        ld_raw_stream<16>(grow + vi * 16ll, wg);
+        ld_raw_stream<PB>(prow + static_cast<long long>(vi) * PB, wp);
+        decode_vec<GDT, VEC>(wg, g[v]);
+        decode_vec<PDT, VEC>(wp, p[v]);
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) dot = fmaf(g[v][e], p[v][e], dot);
+      }
+    }
+    dot = warp_sum_f32(dot);
+    char* orow = static_cast<char*>(dS) + row * Tk * ElemBytes<ODT>::v;
+#pragma unroll
+    for (int v = 0; v < kSmVpt; ++v) {
+      const int vi = lane + v * 32;
+      if (vi < n_vec) {
+        float o[VEC];
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) o[e] = p[v][e] * (g[v][e] - dot);
+        uint32_t ow[OB / 4];
+        encode_vec<ODT, VEC>(o, ow);
+        st_raw<OB>(orow + static_cast<long long>(vi) * OB, ow);
+      }
+    }
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0 && ds_scale) *ds_scale = load_scale(dp_scale) * load_scale(p_scale);
+}
+
+static int rows_grid(long long rows, int rows_per_block) {
+  long long need = (rows + rows_per_block - 1) / rows_per_block;
+  const long long cap = static_cast<long long>(sm_count()) * 16;
+  if (need < 1) need = 1;
+  return static_cast<int>(need < cap ? need : cap);
+}
+
+int launch_softmax_fwd(const void* S, int s_dt, void* P, int p_dt, long long rows, int Tq, int Tk, int causal,
+                       const float* s_scale, float* p_scale, cudaStream_t st) {
+  if (Tk * elem_size(s_dt) / 16 > 32 * kSmVpt) return SCALIFY_ERR_UNSUPPORTED;
+  const int grid = rows_grid(rows, 4);
+  SCALIFY_DISPATCH_WIDE(s_dt, SDT, SCALIFY_DISPATCH_DTYPE(p_dt, PDT,
+      softmax_fwd_kernel<SDT, PDT><<<grid, 128, 0, st>>>(S, P, rows, Tq, Tk, causal, s_scale, p_scale)));
+  SCALIFY_CUDA_TRY(cudaGetLastError());
+  return SCALIFY_OK;
+}
+
+int launch_softmax_bwd(const void* dP, int g_dt, const void* P, int p_dt, void* dS, int o_dt, long long rows, int Tk,
+                       const float* dp_scale, const float* p_scale, float* ds_scale, cudaStream_t st) {
+  if (Tk * elem_size(g_dt) / 16 > 32 * kSmVpt) return SCALIFY_ERR_UNSUPPORTED;
+  const int grid = rows_grid(rows, 4);
+  // P: the probabilities as used in the forward (E4M3 matmul operand) or a 16-bit copy; dS: 16-bit or FP8
+  if (!(p_dt == SCALIFY_E4M3 || p_dt == SCALIFY_BF16 || p_dt == SCALIFY_F16 || p_dt == SCALIFY_F32))
+    return SCALIFY_ERR_UNSUPPORTED;
+#define SCALIFY_SM_BWD(PD)                                                                                   \
+  SCALIFY_DISPATCH_DTYPE(o_dt, ODT, softmax_bwd_kernel<GDT, PD, ODT><<<grid, 128, 0, st>>>(dP, P, dS, rows, Tk, \
+                                                                                          dp_scale, p_scale, ds_scale))
+  SCALIFY_DISPATCH_WIDE(g_dt, GDT, {
+    if (p_dt == SCALIFY_E4M3) { SCALIFY_SM_BWD(SCALIFY_E4M3); }
+    else if (p_dt == SCALIFY_BF16) { SCALIFY_SM_BWD(SCALIFY_BF16); }
+    else if (p_dt == SCALIFY_F16) { SCALIFY_SM_BWD(SCALIFY_F16); }
+    else { SCALIFY_SM_BWD(SCALIFY_F32); }
+  });
+#undef SCALIFY_SM_BWD
+  SCALIFY_CUDA_TRY(cudaGetLastError());
+  return SCALIFY_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// mean cross-entropy over n rows (logsumexp, Appendix B) and its gradient
+// ---------------------------------------------------------------------------------------------
+// One block per row; three sweeps over the row (max, sum of exponentials, gradient), the second and
+// third served by L1/L2.  Per-row losses go to the workspace and are summed in row order.
+template <int LDT, int GDT>
+__global__ void __launch_bounds__(256) cross_entropy_kernel(const void* __restrict__ logits, long long ld, int n_classes,
+                                                            const long long* __restrict__ targets, long long n,
+                                                            const float* l_scale, void* __restrict__ dlogits,
+                                                            float rem, float* __restrict__ row_loss,
+                                                            uint32_t* bad_index) {
+  __shared__ float s_red[8];
+  __shared__ float s_bcast;
+  const float ls = load_scale(l_scale) * 1.4426950408889634f;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (long long row = blockIdx.x; row < n; row += gridDim.x) {
+    const char* lrow = static_cast<const char*>(logits) + row * ld * ElemBytes<LDT>::v;
+    float mx = -INFINITY;
+    for (int j = threadIdx.x; j < n_classes; j += 256) mx = fmaxf(mx, load_elem<LDT>(lrow, j) * ls);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+    __syncthreads();
+    if (lane == 0) s_red[warp] = mx;
+    __syncthreads();
+    mx = s_red[0];
+#pragma unroll
+    for (int k = 1; k < 8; ++k) mx = fmaxf(mx, s_red[k]);
+    float sum = 0.f;
+    for (int j = threadIdx.x; j < n_classes; j += 256) sum += exp2f(load_elem<LDT>(lrow, j) * ls - mx);
+    sum = warp_sum_f32(sum);
+    __syncthreads();
+    if (lane == 0) s_red[warp] = sum;
+    __syncthreads();
+    sum = 0.f;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) sum += s_red[k];
+    long long t = targets[row];
+    if (t < 0 || t >= n_classes) {
+      if (threadIdx.x == 0 && bad_index) atomicOr(bad_index, static_cast<uint32_t>(SCALIFY_DEV_BAD_INDEX));
+      t = 0;
+    }
+    if (threadIdx.x == 0) {
+      const float zt = load_elem<LDT>(lrow, t) * ls;
+      // loss in natural-log units: ln(sum) + (mx - zt)*ln2
+      row_loss[row] = logf(sum) + (mx - zt) * 0.6931471805599453f;
+      s_bcast = rem / sum;
+    }
+    __syncthreads();
+    if (dlogits) {
+      const float k = s_bcast;
+      char* grow = static_cast<char*>(dlogits) + row * ld * ElemBytes<GDT>::v;
+      for (long long j = threadIdx.x; j < ld; j += 256) {
+        float g = 0.f;
+        if (j < n_classes) {
+          g = exp2f(load_elem<LDT>(lrow, j) * ls - mx) * k;
+          if (j == t) g -= rem;
+        }
+        store_elem<GDT>(grow, j, g);
+      }
+    }
+  }
+}
+
+__global__ void __launch_bounds__(256) cross_entropy_finalize_kernel(const float* __restrict__ row_loss, long long n,
+                                                                     float* loss, float* g_scale, float gs) {
+  __shared__ double s[8];
+  double acc = 0.0;
+  for (long long i = threadIdx.x; i < n; i += 256) acc += static_cast<double>(row_loss[i]);
+  acc = warp_sum_f64(acc);
+  if ((threadIdx.x & 31) == 0) s[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double tot = 0.0;
+    for (int i = 0; i < 8; ++i) tot += s[i];
+    *loss = static_cast<float>(tot / static_cast<double>(n));
+    if (g_scale) *g_scale = gs;
+  }
+}
+
+size_t cross_entropy_ws_bytes(int64_t n) { return kWsHeader + static_cast<size_t>(n) * sizeof(float) + 256; }
+
+int launch_cross_entropy(const void* logits, int l_dt, long long ld, int n_classes, const long long* targets, long long n,
+                         const float* l_scale, float* loss, void* dlogits, int g_dt, float* g_scale, void* ws,
+                         cudaStream_t st) {
+  WsView v = ws_view(ws);
+  float* row_loss = static_cast<float*>(v.area);
+  // 1/n = gs * rem with gs a power of two (rounded down) and rem in [1,2) kept in the data
+  int ex;
+  frexp(1.0 / static_cast<double>(n), &ex);
+  const double gs = ldexp(1.0, ex - 1);
+  const float rem = static_cast<float>((1.0 / static_cast<double>(n)) / gs);
+  const long long cap = static_cast<long long>(sm_count()) * 8;
+  const int grid = static_cast<int>(n < cap ? n : cap);
+  SCALIFY_DISPATCH_WIDE(l_dt, LDT, SCALIFY_DISPATCH_DTYPE(g_dt, GDT,
+      cross_entropy_kernel<LDT, GDT><<<grid, 256, 0, st>>>(logits, ld, n_classes, targets, n, l_scale, dlogits, rem,
+                                                           row_loss, v.status)));
+  SCALIFY_CUDA_TRY(cudaGetLastError());
+  cross_entropy_finalize_kernel<<<1, 256, 0, st>>>(row_loss, n, loss, g_scale, static_cast<float>(gs));
+  SCALIFY_CUDA_TRY(cudaGetLastError());
+  return SCALIFY_OK;
+}
+
+}  // namespace scalify
