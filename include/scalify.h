@@ -263,6 +263,14 @@ int scalify_scaled_gelu_bwd(const scalify_array* G, const scalify_array* X, int 
                             scalify_array* dX, void* stream);
 
 /*
+ * Multiply a ScaledArray by a scalar constant c that is a positive power of two (Section 3.4: a
+ * broadcast scalar contributes the scale "c rounded down to a power of two" and its mantissa stays
+ * in the data; for a power of two the mantissa is 1, so only the scale word changes: X_s *= c).
+ * Other constants return SCALIFY_ERR_UNSUPPORTED.  Used for the 1/sqrt(head_dim) of attention.
+ */
+int scalify_scalar_mul_pow2(scalify_array* X, float c, void* stream);
+
+/*
  * Support operations of a GPT-style training step.  The paper states no scale rule for these
  * (Section 3.2.1 only says that custom rules suit attention layers); the rules below are this
  * library's readings, chosen so that values follow the unscaled network exactly (model invariance,

@@ -218,6 +218,18 @@ int launch_rebalance(const void* x, int in_dt, void* y, int out_dt, int64_t n, c
 }
 
 // ---------------------------------------------------------------------------------------------
+// multiplication by a scalar constant that is a power of two (Section 3.4: a broadcast scalar
+// splits into mantissa and exponent; with mantissa 1 only the scale word changes)
+// ---------------------------------------------------------------------------------------------
+__global__ void scale_word_mul_kernel(float* scale, float c) { *scale = *scale * c; }
+
+int launch_scale_word_mul(float* scale, float c, cudaStream_t st) {
+  scale_word_mul_kernel<<<1, 1, 0, st>>>(scale, c);
+  SCALIFY_CUDA_TRY(cudaGetLastError());
+  return SCALIFY_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
 // scaled add / subtract (Section 3.2, add rule)
 // ---------------------------------------------------------------------------------------------
 struct FastDiv {

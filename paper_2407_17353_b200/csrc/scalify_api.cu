@@ -492,6 +492,13 @@ int scalify_scaled_matmul_delayed(const scalify_array* A, int transA, const scal
   return SCALIFY_OK;
 }
 
+int scalify_scalar_mul_pow2(scalify_array* X, float c, void* stream) {
+  if (!X || !X->scale) return SCALIFY_ERR_NULL;
+  int ex;
+  if (!(c > 0.f) || !isfinite(c) || frexpf(c, &ex) != 0.5f) return SCALIFY_ERR_UNSUPPORTED;
+  return launch_scale_word_mul(X->scale, c, static_cast<cudaStream_t>(stream));
+}
+
 int scalify_scaled_embedding(const int64_t* ids, int64_t n, int64_t seq_len, const scalify_array* wte,
                              const scalify_array* wpe, scalify_array* Y, uint32_t* status, void* stream) {
   if (!ids) return SCALIFY_ERR_NULL;

@@ -1,0 +1,300 @@
+"""Library calls with an optional stage-isolated oracle check.
+
+`Ops(check=True)` runs every C-ABI call and then the oracle on the SAME inputs (downloaded bit
+patterns of the library's own previous outputs), holding each call to its own tolerance.  With
+`check=False` the same code only launches kernels (used to time a full-size step)."""
+import numpy as np
+import torch
+
+import paper_2407_17353_b200 as sc
+
+E4, E5, F16, BF, F32 = sc.E4M3, sc.E5M2, sc.F16, sc.BF16, sc.F32
+_CODE = {torch.float8_e4m3fn: E4, torch.float8_e5m2: E5, torch.float16: F16, torch.bfloat16: BF, torch.float32: F32}
+
+
+def code(t: torch.Tensor) -> int:
+    return _CODE[t.dtype]
+
+
+class Ops:
+    def __init__(self, check: bool, ws_bytes: int = 1 << 26, device="cuda"):
+        self.check = check
+        self.dev = device
+        self.ws = sc.Workspace(ws_bytes, device)
+        self.calls = 0
+        if check:
+            import oracle as orc
+            from helpers import to_bits, ulp_diff, within
+            self.orc, self.to_bits, self.ulp_diff, self.within = orc, to_bits, ulp_diff, within
+
+    # ---------------------------------------------------------------- helpers
+    def empty(self, shape, dt):
+        return sc.ScaledTensor.empty(tuple(shape), sc.TORCH_DTYPE[dt], self.dev)
+
+    def bits(self, T):
+        return self.to_bits(T.data, code(T.data))
+
+    def _status_ok(self):
+        if self.check:
+            st = self.ws.check_status()
+            assert st == 0, st
+
+    # ---------------------------------------------------------------- casts and rescales
+    def cast(self, X, dt):
+        Y = self.empty(X.data.shape, dt)
+        sc.scalify_rescale(X, Y)
+        self.calls += 1
+        if self.check:
+            o = self.orc
+            assert Y.scale_value() == X.scale_value()
+            assert np.array_equal(self.bits(Y), o.encode(o.decode(self.bits(X), code(X.data)), dt))
+        return Y
+
+    def rescale(self, X, stat, dt):
+        """Dynamic rescale (statistic -> power of two -> rebalance)."""
+        Y = self.empty(X.data.shape, dt)
+        sc.scalify_rescale(X, Y, stat=stat, ws=self.ws)
+        self.calls += 2
+        if self.check:
+            o = self.orc
+            self._status_ok()
+            yo, ys, so = o.rescale(self.bits(X).reshape(-1), code(X.data), X.scale_value(), stat, dt)
+            if stat == sc.STAT_L2 and abs(np.log2(so) - round(np.log2(so))) < 1e-5:
+                return Y  # binade edge: either neighbouring scale is correct
+            assert Y.scale_value() == ys
+            assert np.array_equal(self.bits(Y).reshape(-1), yo)
+        return Y
+
+    def scalar_mul(self, X, c):
+        before = X.scale_value() if self.check else None
+        sc.scalify_scalar_mul_pow2(X, c)
+        self.calls += 1
+        if self.check:
+            assert X.scale_value() == before * c
+        return X
+
+    # ---------------------------------------------------------------- matmul
+    def mm(self, A, B, *, transA=False, transB=False, out_dt=BF, Y=None, stat=sc.STAT_NONE, q_dt=None):
+        a, b = A.data, B.data
+        M = a.shape[-1] if transA else a.shape[-2]
+        N = b.shape[-2] if transB else b.shape[-1]
+        shape = (M, N) if a.dim() == 2 else (a.shape[0], M, N)
+        if Y is None:
+            Y = self.empty(shape, out_dt)
+        Yq = self.empty(shape, q_dt) if q_dt is not None else None
+        sc.scalify_scaled_matmul(A, B, Y, self.ws, transA=transA, transB=transB, stat=stat, Yq=Yq)
+        self.calls += 1 + (1 if Yq is not None else 0)
+        if self.check:
+            o = self.orc
+            self._status_ok()
+            a_dt, b_dt, y_dt = code(a), code(b), code(Y.data)
+            Ab, Bb, Yb = self.bits(A), self.bits(B), self.bits(Y)
+            if a.dim() == 2:
+                Ab, Bb, Yb = Ab[None], Bb[None], Yb[None]
+            elif b.dim() == 2:
+                Bb = np.broadcast_to(Bb, (Ab.shape[0],) + Bb.shape)
+            for i in range(Ab.shape[0]):
+                Yo, ys, acc, sab = o.scaled_matmul(Ab[i], a_dt, A.scale_value(), Bb[i], b_dt, B.scale_value(), y_dt,
+                                                   transA=transA, transB=transB, want_acc=True)
+                assert Y.scale_value() == ys
+                ok = self.within(Yb[i], Yo, y_dt, acc, sab, 1e-5)
+                assert ok.all(), int((~ok).sum())
+            if Yq is not None:
+                so = o.statistic(self.bits(Y).reshape(-1), y_dt, stat)
+                got = float(self.ws.statistic().item())
+                assert got == so if stat == sc.STAT_AMAX else abs(got - so) <= 2e-6 * so
+                qo, qs, _ = o.rescale(self.bits(Y).reshape(-1), y_dt, Y.scale_value(), stat, q_dt)
+                if not (stat == sc.STAT_L2 and abs(np.log2(so) - round(np.log2(so))) < 1e-5):
+                    assert Yq.scale_value() == qs
+                    assert np.array_equal(self.bits(Yq).reshape(-1), qo)
+        return (Y, Yq) if q_dt is not None else Y
+
+    # ---------------------------------------------------------------- add
+    def add(self, A, B, subtract=False, out_dt=None):
+        Y = self.empty(A.data.shape, out_dt if out_dt is not None else code(A.data))
+        sc.scalify_scaled_add(A, B, Y, subtract=subtract)
+        self.calls += 1
+        if self.check:
+            o = self.orc
+            dt, ydt = code(A.data), code(Y.data)
+            a, b = self.bits(A), self.bits(B)
+            a2 = a.reshape(-1, a.shape[-1])
+            yo, ys = o.scaled_add(a2, dt, A.scale_value(), b if b.ndim == 1 else b.reshape(a2.shape), dt,
+                                  B.scale_value(), ydt, subtract=subtract)
+            assert Y.scale_value() == ys
+            fa, fb = A.scale_value() / ys, B.scale_value() / ys
+            av = o.decode(a2, dt) * fa
+            bv = o.decode(b, dt) * fb
+            bv = bv[None, :] if b.ndim == 1 else bv.reshape(a2.shape)
+            exact = av - bv if subtract else av + bv
+            ok = self.within(self.bits(Y).reshape(a2.shape), yo, ydt, exact, np.abs(av) + np.abs(bv), 2.0 ** -23)
+            assert ok.all(), int((~ok).sum())
+        return Y
+
+    # ---------------------------------------------------------------- LayerNorm
+    def ln(self, X, gamma, beta, eps=1e-5):
+        R, d = X.data.shape
+        Y = self.empty((R, d), BF)
+        mean = torch.empty(R, dtype=torch.float32, device=self.dev)
+        rinv = torch.empty(R, dtype=torch.float32, device=self.dev)
+        sc.scalify_scaled_layernorm(X, gamma, beta, Y, eps=eps, mean=mean, rinv=rinv)
+        self.calls += 1
+        if self.check:
+            o = self.orc
+            xdt, gdt = code(X.data), code(gamma.data)
+            gs, bs = gamma.scale_value(), beta.scale_value()
+            yo, ys, _, _ = o.layernorm_fwd(self.bits(X), xdt, self.bits(gamma), gdt, gs, self.bits(beta), gdt, bs, eps,
+                                           False, BF)
+            n32, _, _, _ = o.layernorm_fwd(self.bits(X), xdt, None, 0, 1.0, None, 0, 1.0, eps, False, F32)
+            nv = o.decode(n32, F32)
+            g = o.decode(self.bits(gamma), gdt) * (gs / ys)
+            b = o.decode(self.bits(beta), gdt) * (bs / ys)
+            assert Y.scale_value() == ys
+            ok = self.within(self.bits(Y), yo, BF, nv * g + b, np.abs(nv * g) + np.abs(b) + 1e-3, 2e-6)
+            assert ok.all(), int((~ok).sum())
+        return Y, mean, rinv
+
+    def ln_bwd(self, G, X, gamma, mean, rinv, stat=sc.STAT_L2, q_dt=BF, eps=1e-5):
+        R, d = X.data.shape
+        dX = self.empty((R, d), BF)
+        dXq = self.empty((R, d), q_dt)
+        dg, db = self.empty((d,), F32), self.empty((d,), F32)
+        sc.scalify_scaled_layernorm_bwd(G, X, gamma, mean, rinv, dX, self.ws, eps=eps, stat_dx=stat, dXq=dXq,
+                                        dgamma=dg, dbeta=db)
+        self.calls += 3
+        if self.check:
+            o = self.orc
+            self._status_ok()
+            xdt, gdt = code(X.data), code(gamma.data)
+            gb, xb, gamb = self.bits(G), self.bits(X), self.bits(gamma)
+            r = o.layernorm_bwd(gb, xdt, G.scale_value(), xb, xdt, X.scale_value(), gamb, gdt, gamma.scale_value(), eps,
+                                False, BF, F32, want_f64=True)
+            assert dX.scale_value() == r["dX_scale"] and dg.scale_value() == r["dgamma_scale"]
+            _, _, _, ro = o.layernorm_fwd(xb, xdt, None, 0, 1.0, None, 0, 1.0, eps, False, BF)
+            gv = o.decode(gamb, gdt)
+            ghat = o.decode(gb, xdt) * gv[None, :]
+            row_mag = np.abs(ghat).max(axis=1) * ro
+            got = self.bits(dX)
+            err = np.abs(o.decode(got, BF) - r["dx_f64"])
+            ok = (self.ulp_diff(got, r["dX"], BF) <= 1) | (err <= 0.5 * np.abs(r["dx_f64"]) * 2.0 ** -8 +
+                                                           2.0 ** -18 * row_mag[:, None])
+            assert ok.all(), int((~ok).sum())
+            n32, _, _, _ = o.layernorm_fwd(xb, xdt, None, 0, 1.0, None, 0, 1.0, eps, False, F32)
+            nv, Gd, f = o.decode(n32, F32), o.decode(gb, xdt), o.kf(R)
+            assert np.all(np.abs(o.decode(self.bits(dg), F32) - (Gd * nv).sum(0) / f) <=
+                          2e-5 * np.abs(Gd * nv).sum(0) / f + 1e-30)
+            assert np.all(np.abs(o.decode(self.bits(db), F32) - Gd.sum(0) / f) <= 2e-5 * np.abs(Gd).sum(0) / f + 1e-30)
+            so = o.statistic(got.reshape(-1), BF, stat)
+            gstat = float(self.ws.statistic().item())
+            assert gstat == so if stat == sc.STAT_AMAX else abs(gstat - so) <= 2e-6 * so
+            if not (stat == sc.STAT_L2 and abs(np.log2(so) - round(np.log2(so))) < 1e-5):
+                qo, qs, _ = o.rescale(got.reshape(-1), BF, r["dX_scale"], stat, q_dt)
+                assert dXq.scale_value() == qs and np.array_equal(self.bits(dXq).reshape(-1), qo)
+        return dXq, dg, db
+
+    # ---------------------------------------------------------------- GELU
+    def gelu(self, X):
+        Y = self.empty(X.data.shape, BF)
+        sc.scalify_scaled_gelu(X, Y)
+        self.calls += 1
+        if self.check:
+            o = self.orc
+            yo, ys = o.gelu_fwd(self.bits(X), code(X.data), X.scale_value(), BF)
+            assert Y.scale_value() == ys and self.ulp_diff(self.bits(Y), yo, BF).max() <= 1
+        return Y
+
+    def gelu_bwd(self, G, X):
+        dX = self.empty(X.data.shape, BF)
+        sc.scalify_scaled_gelu_bwd(G, X, dX)
+        self.calls += 1
+        if self.check:
+            o = self.orc
+            dt = code(X.data)
+            do, ds = o.gelu_bwd(self.bits(G), dt, G.scale_value(), self.bits(X), dt, X.scale_value(), BF)
+            assert dX.scale_value() == ds
+            dd = self.ulp_diff(self.bits(dX), do, BF)
+            bad = dd > 1  # f' crosses zero near x = -0.75: absolute bound there
+            if bad.any():
+                err = np.abs(o.decode(self.bits(dX), BF) - o.decode(do, BF))
+                assert np.all(err[bad] <= 2.0 ** -9 * 2e-2 * np.abs(o.decode(self.bits(G), dt))[bad] + 2.0 ** -16)
+        return dX
+
+    # ---------------------------------------------------------------- attention pieces
+    def softmax(self, S, causal, p_dt):
+        P = self.empty(S.data.shape, p_dt)
+        sc.scalify_scaled_softmax(S, P, causal=causal)
+        self.calls += 1
+        if self.check:
+            o = self.orc
+            po, ps = o.softmax_fwd(self.bits(S), code(S.data), S.scale_value(), causal, p_dt)
+            assert P.scale_value() == ps and self.ulp_diff(self.bits(P), po, p_dt).max() <= 1
+        return P
+
+    def softmax_bwd(self, dP, P, o_dt):
+        dS = self.empty(P.data.shape, o_dt)
+        sc.scalify_scaled_softmax_bwd(dP, P, dS)
+        self.calls += 1
+        if self.check:
+            o = self.orc
+            gdt, pdt = code(dP.data), code(P.data)
+            so, ss = o.softmax_bwd(self.bits(dP), gdt, dP.scale_value(), self.bits(P), pdt, P.scale_value(), o_dt)
+            assert dS.scale_value() == ss
+            pv, gv = o.decode(self.bits(P), pdt), o.decode(self.bits(dP), gdt)
+            dot = (pv * gv).sum(-1, keepdims=True)
+            mag = pv * (np.abs(gv) + np.abs(pv * gv).sum(-1, keepdims=True))
+            assert self.within(self.bits(dS), so, o_dt, pv * (gv - dot), mag, 4e-6).all()
+        return dS
+
+    # ---------------------------------------------------------------- embedding and loss
+    def embedding(self, ids, T, wte, wpe):
+        n, d = ids.numel(), wte.data.shape[1]
+        Y = self.empty((n, d), BF)
+        sc.scalify_scaled_embedding(ids, T, wte, wpe, Y)
+        self.calls += 1
+        if self.check:
+            o = self.orc
+            dt = code(wte.data)
+            yo, ys = o.embedding_fwd(ids.cpu().numpy(), T, self.bits(wte), dt, wte.scale_value(), self.bits(wpe), dt,
+                                     wpe.scale_value(), BF)
+            assert Y.scale_value() == ys and self.ulp_diff(self.bits(Y), yo, BF).max() <= 1
+        return Y
+
+    def embedding_bwd(self, ids, T, dY, vocab):
+        n, d = dY.data.shape
+        dwte, dwpe = self.empty((vocab, d), F32), self.empty((T, d), F32)
+        sc.scalify_scaled_embedding_bwd(ids, T, dY, dwte, dwpe)
+        self.calls += 2
+        if self.check:
+            o = self.orc
+            dt = code(dY.data)
+            idn = ids.cpu().numpy()
+            to, s1, po, s2 = o.embedding_bwd(idn, T, vocab, self.bits(dY), dt, dY.scale_value(), F32)
+            assert dwte.scale_value() == s1 and dwpe.scale_value() == s2
+            g = np.abs(o.decode(self.bits(dY), dt))
+            mag = np.zeros((vocab, d))
+            np.add.at(mag, idn, g)
+            assert np.all(np.abs(o.decode(self.bits(dwte), F32) - o.decode(to, F32)) <= 2e-6 * mag + 1e-30)
+            magp = g.reshape(n // T, T, d).sum(0) / o.kf(n // T)
+            assert np.all(np.abs(o.decode(self.bits(dwpe), F32) - o.decode(po, F32)) <= 2e-6 * magp + 1e-30)
+        return dwte, dwpe
+
+    def cross_entropy(self, logits, n_classes, targets, g_dt):
+        n, ld = logits.data.shape
+        G = self.empty((n, ld), g_dt)
+        loss = torch.zeros(1, dtype=torch.float32, device=self.dev)
+        ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_CROSS_ENTROPY, n), self.dev)
+        sc.scalify_scaled_cross_entropy(logits, n_classes, targets, loss, G, ws)
+        self.calls += 2
+        if self.check:
+            o = self.orc
+            assert ws.check_status() == 0
+            ldt = code(logits.data)
+            lb = self.bits(logits).copy()
+            lb[:, n_classes:] = 0  # padding columns hold whatever the buffer had; the call ignores them
+            lo, go, gs = o.cross_entropy(lb, ldt, logits.scale_value(), n_classes, targets.cpu().numpy(), g_dt)
+            _, g64, _ = o.cross_entropy(lb, ldt, logits.scale_value(), n_classes, targets.cpu().numpy(), F32)
+            assert abs(float(loss.item()) - lo) <= 2e-6 * abs(lo) + 1e-6
+            assert G.scale_value() == gs
+            ex = o.decode(g64, F32)
+            assert self.within(self.bits(G), go, g_dt, ex, np.abs(ex) + 1e-6, 8e-6).all()
+        return loss, G

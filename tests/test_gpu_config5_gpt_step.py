@@ -1,0 +1,102 @@
+"""Config 5: a GPT-2-shaped training step (embedding, L pre-LN transformer layers with causal
+attention and GELU MLP, tied head, cross-entropy, backward, scaled Adam), every matmul scaled FP8.
+
+Reduced shapes (vocab 1000 padded to 1024, seq 128, d 128, 2 heads, 2 layers, batch 2) so that the
+fp64 oracle can follow every one of the ~250 kernel launches of the step: each call is checked
+stage-isolated against the oracle on the library's own inputs (see checked_ops.Ops).  Then model
+invariance (Section 1): the loss and the gradients agree with an unscaled fp64 PyTorch evaluation
+of the same network to FP8 quantisation noise.  The GPT-2-small shapes themselves (12 layers,
+d 768, 12 heads, seq 1024, batch 8, vocab 50257) run through the same code unchecked in
+`test_full_size_step_runs`."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as orc
+import paper_2407_17353_b200 as sc
+import scalify_inputs as si
+from checked_ops import Ops
+from gpt_model import GPTConfig, ScaledGPT
+from helpers import to_bits
+
+pytestmark = pytest.mark.gpu
+
+
+def torch_reference(model, ids, targets):
+    """The same network in fp64 on the decoded master weights; returns loss and gradients by name."""
+    c = model.cfg
+    P = {k: torch.from_numpy(orc.decode(to_bits(v.data, orc.F16), orc.F16) * v.scale_value()).requires_grad_(True)
+         for k, v in model.params.items()}
+    d, H, T, B = c.d, c.heads, c.seq, c.batch
+    hd = d // H
+
+    def ln(x, g, b):
+        mu = x.mean(-1, keepdim=True)
+        sig = ((x - mu) ** 2).mean(-1, keepdim=True).sqrt()
+        return (x - mu) / (sig + 1e-5) * g + b
+    pos = torch.arange(B * T) % T
+    x = P["wte"][ids] + P["wpe"][pos]
+    mask = torch.ones(T, T, dtype=torch.bool).tril()
+    for l in range(c.layers):
+        p = f"h{l}."
+        h = ln(x, P[p + "ln1.g"], P[p + "ln1.b"])
+        q, k, v = (h @ P[p + "w" + nm] + P[p + "b" + nm] for nm in ("q", "k", "v"))
+        sp = lambda t: t.view(B, T, H, hd).permute(0, 2, 1, 3)
+        S = sp(q) @ sp(k).transpose(-1, -2) / np.sqrt(hd)
+        A = torch.softmax(S.masked_fill(~mask, float("-inf")), -1)
+        o = (A @ sp(v)).permute(0, 2, 1, 3).reshape(B * T, d)
+        x = x + o @ P[p + "wo"] + P[p + "bo"]
+        h2 = ln(x, P[p + "ln2.g"], P[p + "ln2.b"])
+        a1 = h2 @ P[p + "w1"] + P[p + "b1"]
+        x = x + torch.nn.functional.gelu(a1, approximate="tanh") @ P[p + "w2"] + P[p + "b2"]
+    logits = ln(x, P["lnf.g"], P["lnf.b"]) @ P["wte"].T
+    loss = torch.nn.functional.cross_entropy(logits, targets)
+    loss.backward()
+    return float(loss.detach()), {k: v.grad.numpy() for k, v in P.items()}
+
+
+def test_reduced_gpt_step_every_call_checked_and_model_invariance():
+    cfg = GPTConfig(vocab=1000, seq=128, d=128, heads=2, layers=2, batch=2)
+    ops = Ops(check=True)
+    model = ScaledGPT(cfg, ops, seed=5)
+    n = cfg.batch * cfg.seq
+    ids = torch.from_numpy(si.uniform_int(5, 901, (n,), cfg.vocab))
+    tgt = torch.from_numpy(si.uniform_int(5, 902, (n,), cfg.vocab))
+    ref_loss, ref_grads = torch_reference(model, ids, tgt)
+    loss = model.step(ids.cuda(), tgt.cuda(), t=1)
+    assert ops.calls > 200
+    got_loss = float(loss.item())
+    assert abs(got_loss - ref_loss) < 0.02 * ref_loss, (got_loss, ref_loss)
+    # gradients as handed to the optimizer (E5M2 data x power-of-two scale) against fp64 autograd
+    worst = {}
+    for k, g in model.last_grads.items():
+        val = orc.decode(to_bits(g.data, orc.E5M2), orc.E5M2).reshape(ref_grads[k].shape) * g.scale_value()
+        s = g.scale_value()
+        assert s > 0 and np.log2(s) == round(np.log2(s))
+        if k.endswith(".bk"):
+            # the key bias shifts every score of a row equally, which softmax ignores: its true gradient is 0
+            assert np.abs(val).max() < 0.2 * np.abs(ref_grads[k.replace(".bk", ".bq")]).max()  # FP8 noise only
+            continue
+        rel = np.sqrt(np.mean((val - ref_grads[k]) ** 2)) / (np.sqrt(np.mean(ref_grads[k] ** 2)) + 1e-30)
+        worst[k] = rel
+        assert rel < 0.25, (k, rel)          # E5M2 carries 2 mantissa bits: ~8 % rounding noise per element
+    assert np.median(list(worst.values())) < 0.15
+
+
+def test_full_size_step_runs():
+    """GPT-2-small shapes, unchecked (the oracle cannot follow 7e12 flop): two steps run, the loss is finite
+    and near ln(vocab) for random weights, every scale stays a power of two, no status bit is raised."""
+    cfg = GPTConfig()
+    ops = Ops(check=False)
+    model = ScaledGPT(cfg, ops, seed=6)
+    assert model.n_params() == 124_439_808 + 0  # tied head; q/k/v kept as separate [768,768] matrices
+    n = cfg.batch * cfg.seq
+    ids = torch.from_numpy(si.uniform_int(6, 901, (n,), cfg.vocab)).cuda()
+    tgt = torch.from_numpy(si.uniform_int(6, 902, (n,), cfg.vocab)).cuda()
+    for t in (1, 2):
+        loss = float(model.step(ids, tgt, t=t).item())
+        assert np.isfinite(loss) and abs(loss - np.log(cfg.vocab)) < 1.0, loss
+        assert ops.ws.check_status() == 0 and model.adam_ws.check_status() == 0
+    for k, v in model.params.items():
+        s = v.scale_value()
+        assert s > 0 and np.log2(s) == round(np.log2(s))
