@@ -263,6 +263,17 @@ int scalify_scaled_gelu_bwd(const scalify_array* G, const scalify_array* X, int 
                             scalify_array* dX, void* stream);
 
 /*
+ * Diagnostic for the bounded device-side waits (no counterpart in the paper).  Enqueues a one-thread
+ * kernel that waits, with the same routine and status path as the matmul pipeline, on a barrier that
+ * nothing signals; after `limit_us` microseconds (1..1e6) the wait gives up, sets
+ * SCALIFY_DEV_TIMEOUT in the workspace status word and the kernel ends normally.  `waited_us`
+ * (optional device word) receives the time actually spent.  Nothing faults and the context stays
+ * usable: this is how a lost copy or a lost MMA completion would surface.
+ */
+int scalify_debug_expire_wait(void* workspace, size_t workspace_bytes, uint32_t limit_us, uint32_t* waited_us,
+                              void* stream);
+
+/*
  * Multiply a ScaledArray by a scalar constant c that is a positive power of two (Section 3.4: a
  * broadcast scalar contributes the scale "c rounded down to a power of two" and its mantissa stays
  * in the data; for a power of two the mantissa is 1, so only the scale word changes: X_s *= c).

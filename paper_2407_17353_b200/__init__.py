@@ -75,6 +75,7 @@ def lib() -> ctypes.CDLL:
         L.scalify_scaled_gelu.argtypes = [P, i32, P, vp]
         L.scalify_scaled_gelu_bwd.argtypes = [P, P, i32, P, vp]
         L.scalify_scaled_adam_step.argtypes = [i32, P, P, P, P, f32, f32, f32, f32, i64, vp, sz, vp]
+        L.scalify_debug_expire_wait.argtypes = [vp, sz, c.c_uint32, vp, vp]
         L.scalify_scalar_mul_pow2.argtypes = [P, f32, vp]
         L.scalify_scaled_embedding.argtypes = [vp, i64, i64, P, P, P, vp, vp]
         L.scalify_scaled_embedding_bwd.argtypes = [vp, i64, i64, P, P, P, vp]
@@ -88,7 +89,7 @@ def lib() -> ctypes.CDLL:
                      "scalify_scaled_layernorm_bwd", "scalify_scaled_gelu", "scalify_scaled_gelu_bwd",
                      "scalify_scaled_adam_step", "scalify_scaled_adam_step_static", "scalify_scaled_embedding",
                      "scalify_scaled_embedding_bwd", "scalify_scaled_softmax", "scalify_scaled_softmax_bwd",
-                     "scalify_scaled_cross_entropy", "scalify_scalar_mul_pow2"):
+                     "scalify_scaled_cross_entropy", "scalify_scalar_mul_pow2", "scalify_debug_expire_wait"):
             getattr(L, name).restype = i32
         _lib = L
     return _lib
@@ -328,3 +329,8 @@ def scalify_scaled_cross_entropy(logits: ScaledTensor, n_classes: int, targets: 
 def scalify_scalar_mul_pow2(X: ScaledTensor, c: float, *, stream=None) -> None:
     x = _desc(X)
     _check(lib().scalify_scalar_mul_pow2(_ref(x), float(c), _stream(stream)), "scalify_scalar_mul_pow2")
+
+
+def scalify_debug_expire_wait(ws: Workspace, limit_us: int, waited_us: Optional[torch.Tensor] = None, *, stream=None) -> None:
+    _check(lib().scalify_debug_expire_wait(ws.ptr, ws.nbytes, int(limit_us), _ptr(waited_us), _stream(stream)),
+           "scalify_debug_expire_wait")

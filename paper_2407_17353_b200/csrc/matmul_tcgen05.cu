@@ -98,14 +98,15 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
   return t;
 }
 // Bounded wait: false when the limit expired or another role of this CTA has given up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          unsigned long long limit_ns = kWaitLimitNs) {
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = global_timer_ns();
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 0xFFu) == 0u) {
       if (*abort_flag) return false;
-      if (global_timer_ns() - t0 > kWaitLimitNs) {
+      if (global_timer_ns() - t0 > limit_ns) {
         *abort_flag = 1u;
         return false;
       }
@@ -466,6 +467,30 @@ scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);
   }
+}
+
+// Diagnostic: one thread waits, with the GEMM's bounded-wait routine and a short limit, on an
+// mbarrier that nothing ever arrives at; the wait must give up, record SCALIFY_DEV_TIMEOUT and let
+// the kernel finish normally (this is the path a lost copy or a lost MMA completion would take).
+__global__ void expire_wait_kernel(uint32_t* status, unsigned long long limit_ns, uint32_t* waited_us) {
+  __shared__ uint64_t bar;
+  __shared__ uint32_t abort_flag;
+  if (threadIdx.x == 0) {
+    const uint32_t b = smem_u32(&bar);
+    mbar_init(b, 1);
+    abort_flag = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    const unsigned long long t0 = global_timer_ns();
+    const bool ok = mbar_wait(b, 0u, &abort_flag, limit_ns);
+    if (waited_us) *waited_us = static_cast<uint32_t>((global_timer_ns() - t0) / 1000ull);
+    if (!ok && status) atomicOr(status, static_cast<uint32_t>(SCALIFY_DEV_TIMEOUT));
+  }
+}
+
+int launch_expire_wait(void* ws, unsigned long long limit_ns, uint32_t* waited_us, cudaStream_t st) {
+  expire_wait_kernel<<<1, 32, 0, st>>>(ws_view(ws).status, limit_ns, waited_us);
+  SCALIFY_CUDA_TRY(cudaGetLastError());
+  return SCALIFY_OK;
 }
 
 // Sums the per-warp partial sums of squares in slot order and leaves sqrt(mean) in the statistic word.

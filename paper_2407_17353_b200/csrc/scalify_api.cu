@@ -492,6 +492,15 @@ int scalify_scaled_matmul_delayed(const scalify_array* A, int transA, const scal
   return SCALIFY_OK;
 }
 
+int scalify_debug_expire_wait(void* workspace, size_t workspace_bytes, uint32_t limit_us, uint32_t* waited_us,
+                              void* stream) {
+  int rc = check_ws(workspace, workspace_bytes, kWsMin);
+  if (rc) return rc;
+  if (limit_us < 1 || limit_us > 1000000u) return SCALIFY_ERR_VALUE;
+  return launch_expire_wait(workspace, static_cast<unsigned long long>(limit_us) * 1000ull, waited_us,
+                            static_cast<cudaStream_t>(stream));
+}
+
 int scalify_scalar_mul_pow2(scalify_array* X, float c, void* stream) {
   if (!X || !X->scale) return SCALIFY_ERR_NULL;
   int ex;

@@ -60,6 +60,7 @@ struct MatmulArgs {
   int force_ncta;  // 0: choose; 1: force the one-CTA kernel
 };
 size_t matmul_ws_bytes(int64_t rows, int64_t cols);
+int launch_expire_wait(void* ws, unsigned long long limit_ns, uint32_t* waited_us, cudaStream_t st);
 int launch_scaled_matmul(const MatmulArgs& a, void* ws, cudaStream_t st);
 
 }  // namespace scalify

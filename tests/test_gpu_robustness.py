@@ -1,0 +1,135 @@
+"""Robustness on the GPU without faulting it: (1) a bounded device-side wait that runs out is
+reported through the status word and leaves the context usable; (2) no kernel writes outside its
+output: outputs are carved out of a larger buffer filled with a sentinel, ragged shapes are run,
+and the guard regions before, after and between rows must be untouched."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2407_17353_b200 as sc
+import scalify_inputs as si
+from helpers import to_dev
+
+pytestmark = pytest.mark.gpu
+SENT = 0x5A
+
+
+def test_expired_wait_sets_timeout_status_and_context_survives():
+    ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_RESCALE, 1024))
+    waited = torch.zeros(1, dtype=torch.int32, device="cuda")
+    sc.scalify_debug_expire_wait(ws, 1500, waited)
+    assert ws.check_status() == sc.DEV_TIMEOUT
+    assert 1500 <= int(waited.item()) < 200000
+    assert ws.check_status() == 0  # cleared by the read
+    # the context is alive: an ordinary call right after works
+    x = sc.ScaledTensor.make(torch.ones(1024, dtype=torch.bfloat16, device="cuda"), 1.0)
+    y = sc.ScaledTensor.empty((1024,), torch.float8_e4m3fn)
+    sc.scalify_rescale(x, y, stat=sc.STAT_AMAX, ws=ws)
+    assert ws.check_status() == 0 and float(y.data.float().abs().max()) == 1.0
+
+
+def guarded(shape, dtype, row_pad=0, guard=4096):
+    """A tensor view of `shape` inside a sentinel-filled byte buffer: guard bytes in front and behind,
+    and (for 2-D) row_pad elements of padding after each row."""
+    es = torch.empty(0, dtype=dtype).element_size()
+    rows = int(np.prod(shape[:-1])) if len(shape) > 1 else 1
+    cols = shape[-1]
+    ld = cols + row_pad
+    raw = torch.full((guard + rows * ld * es + guard,), SENT, dtype=torch.uint8, device="cuda")
+    body = raw[guard:guard + rows * ld * es].view(dtype).view(rows, ld)
+    view = body[:, :cols]
+    if len(shape) == 1:
+        view = view.reshape(cols) if row_pad == 0 else view[0]
+    return raw, view, (guard, rows, ld, cols, es)
+
+
+def assert_guards_intact(raw, meta):
+    guard, rows, ld, cols, es = meta
+    r = raw.cpu().numpy()
+    assert np.all(r[:guard] == SENT) and np.all(r[-guard:] == SENT)
+    if ld > cols:
+        body = r[guard:-guard].reshape(rows, ld * es)
+        assert np.all(body[:, cols * es:] == SENT)
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 16, 16), (130, 272, 144), (257, 528, 400)])
+@pytest.mark.parametrize("y_dt", [torch.bfloat16, torch.float32, torch.float8_e4m3fn])
+def test_matmul_writes_only_its_output(M, N, K, y_dt):
+    A = sc.ScaledTensor.make(to_dev(si.scaled_normal(81, 1, (M, K), si.E4M3), si.E4M3), 1.0)
+    Bt = sc.ScaledTensor.make(to_dev(si.scaled_normal(81, 2, (N, K), si.E4M3), si.E4M3), 1.0)
+    pad = 16 // torch.empty(0, dtype=y_dt).element_size() * 3
+    raw, view, meta = guarded((M, N), y_dt, row_pad=pad)
+    Y = sc.ScaledTensor(view, torch.empty(1, dtype=torch.float32, device="cuda"))
+    ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_MATMUL, M, N))
+    if y_dt == torch.float8_e4m3fn:
+        sc.scalify_scaled_matmul_delayed(A, Bt, torch.ones(1, device="cuda"), Y, ws, transB=True)
+    else:
+        sc.scalify_scaled_matmul(A, Bt, Y, ws, transB=True, stat=sc.STAT_AMAX)
+    assert ws.check_status() == 0
+    assert_guards_intact(raw, meta)
+    assert torch.isfinite(view.float()).all()
+
+
+@pytest.mark.parametrize("n", [1, 17, 4099, 256 * 32 + 3])
+def test_elementwise_kernels_write_only_their_output(n):
+    x = sc.ScaledTensor.make(torch.randn(n, device="cuda").to(torch.bfloat16), 1.0)
+    y = sc.ScaledTensor.make(torch.randn(n, device="cuda").to(torch.bfloat16), 0.5)
+    ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_RESCALE, n))
+    for dt in (torch.float8_e4m3fn, torch.bfloat16, torch.float32):
+        raw, view, meta = guarded((n,), dt)
+        out = sc.ScaledTensor(view, torch.empty(1, dtype=torch.float32, device="cuda"))
+        sc.scalify_rescale(x, out, stat=sc.STAT_AMAX, ws=ws)
+        assert_guards_intact(raw, meta)
+        raw, view, meta = guarded((n,), dt)
+        out = sc.ScaledTensor(view, torch.empty(1, dtype=torch.float32, device="cuda"))
+        sc.scalify_scaled_add(x, y, out)
+        assert_guards_intact(raw, meta)
+        raw, view, meta = guarded((n,), dt)
+        out = sc.ScaledTensor(view, torch.empty(1, dtype=torch.float32, device="cuda"))
+        sc.scalify_scaled_gelu(x, out)
+        assert_guards_intact(raw, meta)
+
+
+@pytest.mark.parametrize("R,d", [(1, 8), (37, 776), (5, 4096)])
+def test_layernorm_writes_only_its_outputs(R, d):
+    x = sc.ScaledTensor.make(torch.randn(R, d, device="cuda").to(torch.bfloat16), 1.0)
+    g = sc.ScaledTensor.make(torch.randn(R, d, device="cuda").to(torch.bfloat16), 2.0 ** -10)
+    gamma = sc.ScaledTensor.make(torch.ones(d, device="cuda", dtype=torch.bfloat16), 1.0)
+    beta = sc.ScaledTensor.make(torch.zeros(d, device="cuda", dtype=torch.bfloat16), 1.0)
+    raw, view, meta = guarded((R, d), torch.bfloat16, row_pad=8)
+    Y = sc.ScaledTensor(view, torch.empty(1, dtype=torch.float32, device="cuda"))
+    rawm, mean, mm = guarded((R,), torch.float32)
+    rawr, rinv, mr = guarded((R,), torch.float32)
+    sc.scalify_scaled_layernorm(x, gamma, beta, Y, mean=mean, rinv=rinv)
+    for r_, m_ in ((raw, meta), (rawm, mm), (rawr, mr)):
+        assert_guards_intact(r_, m_)
+    rawd, dview, md = guarded((R, d), torch.bfloat16, row_pad=8)
+    dX = sc.ScaledTensor(dview, torch.empty(1, dtype=torch.float32, device="cuda"))
+    rawg, gview, mg = guarded((d,), torch.float32)
+    rawb, bview, mb = guarded((d,), torch.float32)
+    dg = sc.ScaledTensor(gview, torch.empty(1, dtype=torch.float32, device="cuda"))
+    db = sc.ScaledTensor(bview, torch.empty(1, dtype=torch.float32, device="cuda"))
+    ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_LAYERNORM_BWD, R, d))
+    sc.scalify_scaled_layernorm_bwd(g, x, gamma, mean, rinv, dX, ws, stat_dx=sc.STAT_L2, dgamma=dg, dbeta=db)
+    assert ws.check_status() == 0
+    for r_, m_ in ((rawd, md), (rawg, mg), (rawb, mb)):
+        assert_guards_intact(r_, m_)
+
+
+@pytest.mark.parametrize("n", [1, 9, 8195])
+def test_adam_writes_only_its_state(n):
+    c = si.adam_case(n, seed=82)
+    bufs = {}
+    T = {}
+    for name, dt, code in (("m", torch.float16, si.F16), ("v", torch.float16, si.F16), ("w", torch.float16, si.F16)):
+        raw, view, meta = guarded((n,), dt)
+        view.copy_(to_dev(c[name], code))
+        bufs[name] = (raw, meta)
+        T[name] = sc.ScaledTensor.make(view, c[name + "_scale"])
+    G = sc.ScaledTensor.make(to_dev(c["g"], si.E5M2), c["g_scale"])
+    ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_ADAM, 1))
+    sc.scalify_scaled_adam_step(sc.AdamTensors([G], [T["m"]], [T["v"]], [T["w"]]), ws, lr=3e-4, beta1=0.9, beta2=0.999,
+                                eps=1e-8, step=10)
+    assert ws.check_status() == 0
+    for raw, meta in bufs.values():
+        assert_guards_intact(raw, meta)
