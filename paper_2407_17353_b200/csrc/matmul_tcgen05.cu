@@ -7,17 +7,19 @@
 //   warp 1      MMA issuer: one thread issues tcgen05.mma (kind::f8f6f4, fp32 accumulate) from
 //               shared-memory descriptors into a TMEM accumulator; tcgen05.commit releases ring
 //               slots and publishes finished accumulators
-//   warps 2-5   epilogue: tcgen05.ld of the accumulator (two accumulators of 256 TMEM columns, so
+//   warps 2-9   epilogue: tcgen05.ld of the accumulator (two accumulators of 256 TMEM columns, so
 //               the epilogue of tile i overlaps the main loop of tile i+1), multiply by the exact
 //               power of two 1/kf(K), round once to the output type, 16-byte stores, and the
 //               statistic of the stored values (AMAX: warp-shuffle max + one atomicMax on the
-//               fp32 bit pattern per warp and tile; L2: per-warp partial sums in fixed slots)
+//               fp32 bit pattern per warp; L2: per-warp partial sums in fixed slots)
 // Tile 128 x 256 x 128 (one 128-byte swizzle row of FP8 per K block, four K=32 MMAs per block).
 // Operands may be K-major (row-major [rows, K]) or MN-major (row-major [K, rows]); the layout is
 // expressed in the shared-memory descriptors and the instruction descriptor, not by copying.
 // Every wait on an mbarrier is bounded; on expiry the CTA records SCALIFY_DEV_TIMEOUT, drains
 // its own copies in flight, frees its TMEM and returns.
 #include <cuda.h>
+
+#include <atomic>
 
 #include "scalify_common.cuh"
 #include "scalify_launch.h"
@@ -29,7 +31,8 @@ constexpr int kBN = 256;   // columns of the output tile
 constexpr int kBK = 128;   // FP8 elements = bytes per K block (one 128-byte swizzle row)
 constexpr int kUmmaK = 32;
 constexpr int kAccStages = 2;
-constexpr int kGemmThreads = 192;
+constexpr int kEpiWarps = 8;                 // two warps per TMEM lane quarter, each taking half of the columns
+constexpr int kGemmThreads = 64 + 32 * kEpiWarps;
 constexpr int kTmemCols = kAccStages * kBN;  // 512
 constexpr int kGroupM = 8;                   // m-tiles per rasterisation group
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
@@ -46,7 +49,8 @@ template <int NCTA> struct GemmCfg {
   static constexpr int kBBytes = kBRows * kBK;       // 32 KB / 16 KB
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kStages = NCTA == 1 ? 4 : 6;
-  static constexpr size_t kSmem = size_t(kStages) * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static constexpr int kEpiBytes = kEpiWarps * 32 * 128;  // per-warp staging tile of the epilogue: 32 rows x up to 128 B
+  static constexpr size_t kSmem = size_t(kStages) * kStageBytes + kEpiBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
 struct GemmParams {
@@ -64,7 +68,8 @@ struct GemmParams {
   float* y_scale;
   int stat;
   const float* stat_in;  // delayed rescale: statistic of an earlier step (device), or NULL
-  uint32_t* stat_word;   // AMAX: atomicMax target
+  unsigned long long* stat_word;  // AMAX: 64-bit atomicMax target: {call generation : fp32 bit pattern}
+  uint32_t generation;   // tag of this call; a later call always overrides an earlier one, so no zeroing is needed
   double* l2_partials;   // L2: [tiles][4]
   uint32_t* status;
 };
@@ -157,6 +162,17 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// ---- TMA store of a shared-memory tile (epilogue)
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int x, int y, int z) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(x), "r"(y), "r"(z) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
 // ---- cta_group::2 forms (cluster of two CTAs on an SM pair)
 __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;
@@ -233,7 +249,7 @@ __device__ __forceinline__ void tile_coords(const GemmParams& p, int tile, int& 
 template <int OUT, int NCTA>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                     const GemmParams p) {
+                     const __grid_constant__ CUtensorMap map_y, const GemmParams p) {
   using C = GemmCfg<NCTA>;
   constexpr int kStages = C::kStages;
   extern __shared__ uint8_t smem_raw[];
@@ -242,8 +258,9 @@ scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
   uint8_t* smem = smem_raw + (base - raw);
   const uint32_t smem_a = base;
   const uint32_t smem_b = base + kStages * C::kABytes;
-  uint8_t* bar_mem = smem + kStages * C::kStageBytes;
-  const uint32_t bars = base + kStages * C::kStageBytes;
+  uint8_t* epi_mem = smem + kStages * C::kStageBytes;  // 16 KB, 1024-byte aligned
+  uint8_t* bar_mem = epi_mem + C::kEpiBytes;
+  const uint32_t bars = base + kStages * C::kStageBytes + C::kEpiBytes;
   const uint32_t full_bar = bars;                         // kStages x 8 B
   const uint32_t empty_bar = bars + 8 * kStages;          // kStages x 8 B
   const uint32_t acc_full_bar = bars + 16 * kStages;      // kAccStages x 8 B
@@ -263,7 +280,7 @@ scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     for (int s = 0; s < kStages; ++s) { mbar_init(full_bar + 8 * s, 1); mbar_init(empty_bar + 8 * s, 1); }
     for (int s = 0; s < kAccStages; ++s) {
       mbar_init(acc_full_bar + 8 * s, 1);
-      mbar_init(acc_empty_bar + 8 * s, 4 * NCTA);  // one arrival per epilogue warp of every CTA of the pair
+      mbar_init(acc_empty_bar + 8 * s, kEpiWarps * NCTA);  // one arrival per epilogue warp of every CTA of the pair
     }
     mbar_init(drain_bar, 1);
     *abort_flag = 0u;
@@ -293,6 +310,7 @@ scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     if (lane == 0) {
       asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
       asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_b)) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_y)) : "memory");
       uint32_t stage = 0, phase = 0;
       long long issued = 0;
       for (int tile = unit; tile < num_tiles && !timed_out; tile += num_units) {
@@ -385,10 +403,11 @@ scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     }
   } else {
     // ---------------------------------------------------------------- epilogue (warps 2..5)
-    const int q = warp & 3;  // TMEM lane quarter this warp may read
+    const int q = warp & 3;                       // TMEM lane quarter this warp may read
+    const int half = (warp - 2) / 4;              // which half of the tile's columns this warp handles
+    constexpr int kChunksPerWarp = (kBN / 32) / (kEpiWarps / 4);
     uint32_t acc = 0, acc_phase = 0;
     uint32_t amax_bits = 0u;
-    char* const Yb = static_cast<char*>(p.Y);
     constexpr int OSZ = ElemBytes<OUT>::v;
     // delayed rescale (Section 3.3): the data are written already divided by r = p2_floor(earlier
     // statistic); this step's statistic is taken on the un-rebalanced fp32 values
@@ -400,22 +419,19 @@ scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
       tile_coords(p, tile, b, mt, nt);
       if (!mbar_wait(acc_full_bar + 8 * acc, acc_phase, abort_flag)) { timed_out = true; break; }
       tc_fence_after();
-      const int row = mt * C::kTileM + static_cast<int>(rank) * kBM + q * 32 + lane;
       const int n0 = nt * kBN;
-      const bool row_ok = row < p.M;
-      char* yrow = Yb + (static_cast<long long>(b) * p.y_batch_stride + static_cast<long long>(row) * p.ldy) * OSZ;
       float ssq = 0.f;
-#pragma unroll 1
-      for (int c = 0; c < kBN / 32; ++c) {
-        const int col0 = n0 + c * 32;
-        if (col0 >= p.N) break;  // warp-uniform
-        uint32_t r[32];
-        tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kBN + c * 32, r);
-        tmem_ld_wait();
+      const int c_first = half * kChunksPerWarp;
+      const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kBN + c_first * 32;
+      // chunks of this warp that lie inside the matrix (warp-uniform)
+      const int n_chunks = max(0, min(kChunksPerWarp, (p.N - n0 + 31) / 32 - c_first));
+      // One 32-column chunk of this thread's row: scale, statistic, round, store.
+      auto process = [&](const uint32_t* acc_regs, int c) {
+        const int col0 = n0 + (c_first + c) * 32;
         float v[32];
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
-          v[i] = __uint_as_float(r[i]) * alpha;
+          v[i] = __uint_as_float(acc_regs[i]) * alpha;
           amax_bits = max(amax_bits, abs_bits(v[i]));
         }
         if (p.stat == SCALIFY_STAT_L2) {
@@ -425,17 +441,39 @@ scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             ssq = fmaf(s, s, ssq);
           }
         }
-        if (row_ok) {
-          if (col0 + 32 <= p.N) {
-            uint32_t o[32 * OSZ / 4];
-            encode_vec<OUT, 32>(v, o);
+        // Each lane holds 32 consecutive columns of ONE row.  The warp writes the chunk (32 rows x 32 columns)
+        // into a shared-memory tile in the swizzle pattern TMA uses for rows of this width, and one lane hands
+        // the tile to a TMA store, which writes whole row segments and clips rows >= M and columns >= N.
+        constexpr int CPR = 32 * OSZ / 16;              // 16-byte pieces per row: 2 (FP8), 4 (16-bit), 8 (F32)
+        constexpr int NBUF = OSZ == 4 ? 1 : 2;          // staging tiles per warp (4 KB per warp in all)
+        uint32_t o[32 * OSZ / 4];
+        encode_vec<OUT, 32>(v, o);
+        uint8_t* tile_b = epi_mem + (warp - 2) * (32 * 128) + (NBUF == 2 ? (c & 1) * 2048 : 0);
+        if (lane == 0) bulk_wait_read<NBUF - 1>();      // the tile's previous store has read it
+        __syncwarp();
+        uint4* tile = reinterpret_cast<uint4*>(tile_b);
 #pragma unroll
-            for (int j = 0; j < 32 * OSZ / 16; ++j) st_raw<16>(yrow + static_cast<long long>(col0) * OSZ + j * 16, o + 4 * j);
-          } else {
-#pragma unroll
-            for (int i = 0; i < 32; ++i)
-              if (col0 + i < p.N) store_elem<OUT>(yrow, col0 + i, v[i]);
-          }
+        for (int j = 0; j < CPR; ++j)
+          tile[lane * CPR + (j ^ ((lane / (8 / CPR)) % CPR))] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          tma_store_3d(&map_y, smem_u32(tile_b), col0, mt * C::kTileM + static_cast<int>(rank) * kBM + q * 32, b);
+          bulk_commit();
+        }
+      };
+      // The TMEM load of the next chunk is in flight while the current chunk is processed.
+      uint32_t ra[32], rb[32];
+      if (n_chunks > 0) tmem_ld32(t_addr, ra);
+#pragma unroll 1
+      for (int c = 0; c < n_chunks; c += 2) {
+        tmem_ld_wait();
+        if (c + 1 < n_chunks) tmem_ld32(t_addr + (c + 1) * 32, rb);
+        process(ra, c);
+        if (c + 1 < n_chunks) {
+          tmem_ld_wait();
+          if (c + 2 < n_chunks) tmem_ld32(t_addr + (c + 2) * 32, ra);
+          process(rb, c + 1);
         }
       }
       tc_fence_before();
@@ -446,16 +484,21 @@ scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
       }
       if (p.stat == SCALIFY_STAT_L2) {
         const double s = warp_sum_f64(static_cast<double>(ssq)) * (double(r_prev) * double(r_prev));
-        if (lane == 0) p.l2_partials[(static_cast<long long>(tile) * NCTA + rank) * 4 + q] = s;
+        if (lane == 0) p.l2_partials[((static_cast<long long>(tile) * NCTA + rank) * 4 + q) * 2 + half] = s;
       }
       if (++acc == kAccStages) { acc = 0; acc_phase ^= 1u; }
     }
+    if (lane == 0) bulk_wait_all();  // every store of this warp has completed
     if (p.stat == SCALIFY_STAT_AMAX) {
       // rounding is monotonic, so the max of the stored values is the stored value of the max
       if (p.stat_in) amax_bits = abs_bits(__uint_as_float(amax_bits) * r_prev);  // un-rebalanced, unrounded
       else amax_bits = abs_bits(round_through<OUT>(__uint_as_float(amax_bits)));
       amax_bits = warp_max_u32(amax_bits);
-      if (lane == 0 && amax_bits != 0u) atomicMax(p.stat_word, amax_bits);
+      // The statistic word is the low half of a 64-bit word whose high half is the generation of the call
+      // that wrote it: an atomicMax of {generation, bits} both resets an older call's value and takes the
+      // maximum within this call, so the word never has to be zeroed in-stream before the launch.
+      if (lane == 0 && (amax_bits != 0u || (blockIdx.x == 0 && warp == 2)))
+        atomicMax(p.stat_word, (static_cast<unsigned long long>(p.generation) << 32) | amax_bits);
     }
   }
 
@@ -546,13 +589,37 @@ static int make_map(CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t 
   return SCALIFY_OK;
 }
 
+// Tensor map of the output [batch][M][N] (row stride ld, batch stride bs, in elements of `es` bytes) for the
+// epilogue's stores: box 32 columns x 32 rows, swizzle equal to the width of a box row (32 / 64 / 128 bytes).
+static int make_map_y(CUtensorMap* map, const void* ptr, int es, uint64_t N, uint64_t M, uint64_t batch, uint64_t ld,
+                      uint64_t bs) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return SCALIFY_ERR_CUDA;
+  cuuint64_t dims[3] = {N, M, batch};
+  cuuint64_t strides[2] = {ld * es, (bs ? bs : ld * M) * es};
+  cuuint32_t box[3] = {32u, 32u, 1u};
+  cuuint32_t estr[3] = {1u, 1u, 1u};
+  const CUtensorMapDataType dt = es == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8
+                               : es == 2 ? CU_TENSOR_MAP_DATA_TYPE_UINT16 : CU_TENSOR_MAP_DATA_TYPE_UINT32;
+  const CUtensorMapSwizzle sw = es == 1 ? CU_TENSOR_MAP_SWIZZLE_32B
+                              : es == 2 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B;
+  CUresult r = fn(map, dt, 3, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+                  CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    set_last_cuda_error(static_cast<int>(r));
+    return SCALIFY_ERR_CUDA;
+  }
+  return SCALIFY_OK;
+}
+
 size_t matmul_ws_bytes(int64_t rows, int64_t cols) {
   int64_t tiles = ((rows + kBM - 1) / kBM + 8) * ((cols + kBN - 1) / kBN);
-  return kWsHeader + size_t(tiles) * 4 * sizeof(double) + 256;
+  return kWsHeader + size_t(tiles) * 8 * sizeof(double) + 256;
 }
 
 template <int OUT, int NCTA>
-static int launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, const GemmParams& p, long long tiles,
+static int launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_y,
+                          const GemmParams& p, long long tiles,
                           cudaStream_t st) {
   using C = GemmCfg<NCTA>;
   auto kernel = scaled_matmul_kernel<OUT, NCTA>;
@@ -594,7 +661,7 @@ static int launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, co
   cfg.blockDim = dim3(kGemmThreads);
   cfg.dynamicSmemBytes = C::kSmem;
   cfg.stream = st;
-  SCALIFY_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, map_a, map_b, p));
+  SCALIFY_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, map_a, map_b, map_y, p));
   return SCALIFY_OK;
 }
 
@@ -604,7 +671,7 @@ int launch_scaled_matmul(const MatmulArgs& a, void* ws, cudaStream_t st) {
   const int ncta = (a.M > kBM && a.force_ncta != 1) ? 2 : 1;
   const int tile_m = kBM * ncta;
   const uint32_t b_box_rows = ncta == 2 ? kBN / 2 : kBN;
-  CUtensorMap map_a, map_b;
+  CUtensorMap map_a, map_b, map_y;
   // A is logically [M,K]; stored [M,K] (K-major) or, with transA, [K,M] (MN-major).
   int rc;
   if (!a.transA) rc = make_map(&map_a, a.A, a.K, a.M, a.batch, a.lda, a.a_bs, kBM);
@@ -615,6 +682,9 @@ int launch_scaled_matmul(const MatmulArgs& a, void* ws, cudaStream_t st) {
   const int b_batch = b_batched ? a.batch : 1;
   if (a.transB) rc = make_map(&map_b, a.B, a.K, a.N, b_batch, a.ldb, a.b_bs, b_box_rows);
   else rc = make_map(&map_b, a.B, a.N, a.K, b_batch, a.ldb, a.b_bs, kBK);
+  if (rc) return rc;
+
+  rc = make_map_y(&map_y, a.Y, elem_size(a.y_dt), a.N, a.M, a.batch, a.ldy, a.y_bs);
   if (rc) return rc;
 
   GemmParams p;
@@ -635,19 +705,27 @@ int launch_scaled_matmul(const MatmulArgs& a, void* ws, cudaStream_t st) {
   p.a_scale = a.a_scale; p.b_scale = a.b_scale; p.y_scale = a.y_scale;
   p.stat = a.stat;
   p.stat_in = a.stat_in;
-  p.stat_word = reinterpret_cast<uint32_t*>(v.stat);
+  p.stat_word = reinterpret_cast<unsigned long long*>(v.stat);
   p.l2_partials = static_cast<double*>(v.area);
   p.status = v.status;
   const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n * p.batch;
   if (tiles > (1ll << 30)) return SCALIFY_ERR_SHAPE;
-  if (a.stat == SCALIFY_STAT_AMAX) SCALIFY_CUDA_TRY(cudaMemsetAsync(v.stat, 0, sizeof(float), st));
+  p.generation = 0;
+  if (a.stat == SCALIFY_STAT_AMAX) {
+    static std::atomic<uint32_t> next_generation{1};
+    p.generation = next_generation.fetch_add(1);
+    if (p.generation == 0) {  // the 32-bit tag wrapped: start over from a zeroed word
+      SCALIFY_CUDA_TRY(cudaMemsetAsync(v.stat, 0, 2 * sizeof(float), st));
+      p.generation = next_generation.fetch_add(1);
+    }
+  }
   SCALIFY_DISPATCH_DTYPE(a.y_dt, OUT, {
-    if (ncta == 2) rc = launch_variant<OUT, 2>(map_a, map_b, p, tiles, st);
-    else rc = launch_variant<OUT, 1>(map_a, map_b, p, tiles, st);
+    if (ncta == 2) rc = launch_variant<OUT, 2>(map_a, map_b, map_y, p, tiles, st);
+    else rc = launch_variant<OUT, 1>(map_a, map_b, map_y, p, tiles, st);
   });
   if (rc) return rc;
   if (a.stat == SCALIFY_STAT_L2) {
-    gemm_l2_finalize_kernel<<<1, 256, 0, st>>>(p.l2_partials, static_cast<int>(tiles * ncta * 4),
+    gemm_l2_finalize_kernel<<<1, 256, 0, st>>>(p.l2_partials, static_cast<int>(tiles * ncta * 8),
                                                double(a.M) * double(a.N) * double(a.batch), v.stat);
     SCALIFY_CUDA_TRY(cudaGetLastError());
   }
