@@ -34,7 +34,7 @@ constexpr int kAccStages = 2;
 constexpr int kEpiWarps = 8;                 // two warps per TMEM lane quarter, each taking half of the columns
 constexpr int kGemmThreads = 64 + 32 * kEpiWarps;
 constexpr int kTmemCols = kAccStages * kBN;  // 512
-constexpr int kGroupM = 8;                   // m-tiles per rasterisation group
+constexpr int kGroupM = 16;                  // m-tiles per rasterisation group
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
 
 // NCTA = 1: one CTA computes a 128 x 256 tile (tcgen05 cta_group::1).
