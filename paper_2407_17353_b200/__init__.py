@@ -116,10 +116,15 @@ class ScaledTensor:
 
 
 def _desc(t: Optional[ScaledTensor]):
-    """ctypes descriptor of a ScaledTensor (None -> NULL)."""
+    """ctypes descriptor of a ScaledTensor (None -> NULL); cached on the object while its buffers stay the same."""
     if t is None:
         return None
     d = t.data
+    sp = 0 if t.scale is None else t.scale.data_ptr()
+    key = (d.data_ptr(), d.dtype, tuple(d.shape), d.stride(), sp)
+    cached = t.__dict__.get("_desc_cache")
+    if cached is not None and cached[0] == key:
+        return cached[1]
     if d.dim() < 1 or d.dim() > 3:
         raise ValueError("scalify arrays have 1 to 3 dimensions")
     a = scalify_array()
@@ -132,9 +137,10 @@ def _desc(t: Optional[ScaledTensor]):
     if t.scale is not None:
         if t.scale.dtype != torch.float32 or t.scale.numel() != 1 or t.scale.device != d.device:
             raise ValueError("scale must be a 1-element fp32 tensor on the data's device")
-        a.scale = t.scale.data_ptr()
+        a.scale = sp
     else:
         a.scale = None
+    t.__dict__["_desc_cache"] = (key, a)
     return a
 
 
