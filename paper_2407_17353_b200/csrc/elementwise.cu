@@ -5,6 +5,8 @@
 // count and strides over the array.
 #include "scalify_common.cuh"
 #include "scalify_launch.h"
+#include <cooperative_groups.h>
+namespace cg = cooperative_groups;
 
 namespace scalify {
 
@@ -215,6 +217,176 @@ int launch_rebalance(const void* x, int in_dt, void* y, int out_dt, int64_t n, c
       rebalance_kernel<IN, OUT><<<grid, kThreads, 0, st>>>(x, y, n, x_scale, y_scale, stat, new_scale, mode, status)));
   SCALIFY_CUDA_TRY(cudaGetLastError());
   return SCALIFY_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// dynamic rescale in one cooperative launch (Section 3.3): statistic, grid barrier, rebalance
+// ---------------------------------------------------------------------------------------------
+// Every block owns one contiguous run of tiles.  Phase 1 reads the run front to back with the
+// default cache policy and leaves one partial per block; after the grid barrier every block
+// combines all partials in index order (so all blocks hold the same statistic, bit for bit) and
+// phase 2 walks its run back to front, so that what phase 1 touched last - still in L2 - is read
+// first.  For arrays up to about the L2 size the second read never reaches HBM.
+template <int IN, int OUT>
+__global__ void __launch_bounds__(kThreads) fused_rescale_kernel(const void* x, void* y, int64_t n, int stat,
+                                                                 const float* x_scale, float* y_scale,
+                                                                 double* partials, float* stat_word,
+                                                                 uint32_t* status) {
+  constexpr int VEC = VecElems<IN, OUT>::v;
+  constexpr int IB = VEC * ElemBytes<IN>::v, OB = VEC * ElemBytes<OUT>::v;
+  constexpr int kTile = kThreads * kUnroll;
+  cg::grid_group grid = cg::this_grid();
+  const int64_t n_vec = n / VEC;
+  const int64_t n_tiles = (n_vec + kTile - 1) / kTile;
+  const int64_t t0 = n_tiles * blockIdx.x / gridDim.x, t1 = n_tiles * (blockIdx.x + 1) / gridDim.x;
+  const int tail = static_cast<int>(n - n_vec * VEC);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  __shared__ double s_part[kThreads / 32];
+
+  uint32_t amax = 0u;
+  float ssq = 0.f;
+  for (int64_t tile = t0; tile < t1; ++tile) {
+    const int64_t base = tile * kTile;
+    uint32_t w[kUnroll][IB / 4];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      int64_t i = base + u * kThreads + threadIdx.x;
+      if (i < n_vec) {
+        ld_raw<IB>(static_cast<const char*>(x) + i * IB, w[u]);
+      } else {
+#pragma unroll
+        for (int q = 0; q < IB / 4; ++q) w[u][q] = 0u;
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      float f[VEC];
+      decode_vec<IN, VEC>(w[u], f);
+#pragma unroll
+      for (int e = 0; e < VEC; ++e) {
+        amax = max(amax, abs_bits(f[e]));
+        ssq = fmaf(f[e], f[e], ssq);
+      }
+    }
+  }
+  if (blockIdx.x == 0 && threadIdx.x < tail) {
+    float f = load_elem<IN>(x, n_vec * VEC + threadIdx.x);
+    amax = max(amax, abs_bits(f));
+    ssq = fmaf(f, f, ssq);
+  }
+  double mine = (stat == SCALIFY_STAT_AMAX) ? static_cast<double>(warp_max_u32(amax))
+                                            : warp_sum_f64(static_cast<double>(ssq));
+  if (lane == 0) s_part[warp] = mine;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double tot = 0.0;
+    if (stat == SCALIFY_STAT_AMAX) {
+      for (int i = 0; i < kThreads / 32; ++i) tot = fmax(tot, s_part[i]);
+    } else {
+      for (int i = 0; i < kThreads / 32; ++i) tot += s_part[i];
+    }
+    partials[blockIdx.x] = tot;
+  }
+  grid.sync();
+
+  // the same fixed-order combination in every block
+  double acc = 0.0;
+  for (int i = threadIdx.x; i < static_cast<int>(gridDim.x); i += kThreads) {
+    double p = __ldcg(&partials[i]);
+    acc = (stat == SCALIFY_STAT_AMAX) ? fmax(acc, p) : acc + p;
+  }
+  if (stat == SCALIFY_STAT_AMAX) acc = static_cast<double>(warp_max_u32(static_cast<uint32_t>(acc)));
+  else acc = warp_sum_f64(acc);
+  __syncthreads();
+  if (lane == 0) s_part[warp] = acc;
+  __syncthreads();
+  double tot = 0.0;
+  if (stat == SCALIFY_STAT_AMAX) {
+    for (int i = 0; i < kThreads / 32; ++i) tot = fmax(tot, s_part[i]);
+  } else {
+    for (int i = 0; i < kThreads / 32; ++i) tot += s_part[i];
+  }
+  const float statistic = (stat == SCALIFY_STAT_AMAX) ? __uint_as_float(static_cast<uint32_t>(tot))
+                                                      : static_cast<float>(sqrt(tot / static_cast<double>(n)));
+  const float xs = load_scale(x_scale);
+  bool nonfinite;
+  const float r = rescale_factor(statistic, &nonfinite);
+  const float factor = 1.0f / r;  // exact: r is a power of two
+
+  for (int64_t tile = t1 - 1; tile >= t0; --tile) {
+    const int64_t base = tile * kTile;
+    uint32_t w[kUnroll][IB / 4];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      int64_t i = base + u * kThreads + threadIdx.x;
+      if (i < n_vec) ld_raw_stream<IB>(static_cast<const char*>(x) + i * IB, w[u]);
+    }
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      int64_t i = base + u * kThreads + threadIdx.x;
+      if (i < n_vec) {
+        float f[VEC];
+        decode_vec<IN, VEC>(w[u], f);
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) f[e] *= factor;
+        uint32_t o[OB / 4];
+        encode_vec<OUT, VEC>(f, o);
+        st_raw_stream<OB>(static_cast<char*>(y) + i * OB, o);
+      }
+    }
+  }
+  if (blockIdx.x == 0) {
+    if (threadIdx.x < tail) {
+      int64_t i = n_vec * VEC + threadIdx.x;
+      store_elem<OUT>(y, i, load_elem<IN>(x, i) * factor);
+    }
+    if (threadIdx.x == 0) {
+      uint32_t flags = is_pow2_scale(xs) ? 0u : SCALIFY_DEV_BAD_SCALE;
+      if (nonfinite) flags |= SCALIFY_DEV_NONFINITE_STAT;
+      *stat_word = statistic;
+      if (y_scale) *y_scale = xs * r;
+      if (flags && status) atomicOr(status, flags);
+    }
+  }
+}
+
+template <int IN, int OUT>
+static int fused_rescale_blocks_per_sm() {
+  static int cached[64] = {0};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+  if (cached[dev] == 0) {
+    int b = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, fused_rescale_kernel<IN, OUT>, kThreads, 0) != cudaSuccess)
+      b = 0;
+    cached[dev] = b > 0 ? b : -1;
+  }
+  return cached[dev] > 0 ? cached[dev] : 0;
+}
+
+// Returns SCALIFY_OK after a cooperative launch, 1 if the device cannot run one (the caller then
+// takes the two-launch path), or an error code.
+int launch_fused_rescale(const void* x, int in_dt, void* y, int out_dt, int64_t n, int stat, const float* x_scale,
+                         float* y_scale, void* ws, cudaStream_t st) {
+  WsView v = ws_view(ws);
+  int big = elem_size(in_dt) > elem_size(out_dt) ? elem_size(in_dt) : elem_size(out_dt);
+  int64_t n_vec = n / (16 / big);
+  double* partials = static_cast<double*>(v.area);
+  float* stat_word = v.stat;
+  uint32_t* status = v.status;
+  void* args[] = {&x, &y, &n, &stat, &x_scale, &y_scale, &partials, &stat_word, &status};
+  int rc = 1;
+  SCALIFY_DISPATCH_DTYPE(in_dt, IN, SCALIFY_DISPATCH_DTYPE(out_dt, OUT, {
+    int per_sm = fused_rescale_blocks_per_sm<IN, OUT>();
+    if (per_sm > 0) {
+      int grid = grid_for(n_vec, per_sm < 8 ? per_sm : 8);
+      cudaError_t e = cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(fused_rescale_kernel<IN, OUT>),
+                                                  dim3(grid), dim3(kThreads), args, 0, st);
+      if (e == cudaSuccess) rc = SCALIFY_OK;
+      else (void)cudaGetLastError();
+    }
+  }));
+  return rc;
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -184,6 +184,10 @@ int scalify_rescale(const scalify_array* X, int stat, const float* new_scale, co
   }
   rc = check_ws(workspace, workspace_bytes, scalify_workspace_bytes(SCALIFY_OP_RESCALE, n, 0));
   if (rc) return rc;
+  // one cooperative launch (statistic, grid barrier, rebalance); two launches where the device
+  // cannot run a cooperative grid
+  rc = launch_fused_rescale(X->data, X->dtype, Y->data, Y->dtype, n, stat, X->scale, Y->scale, workspace, st);
+  if (rc <= 0) return rc;
   rc = launch_statistic(X->data, X->dtype, n, stat, workspace, nullptr, st);
   if (rc) return rc;
   return launch_rebalance(X->data, X->dtype, Y->data, Y->dtype, n, X->scale, Y->scale, ws_view(workspace).stat,

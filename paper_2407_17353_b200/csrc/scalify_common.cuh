@@ -164,6 +164,20 @@ __device__ __forceinline__ void ld_raw_stream(const void* p, uint32_t* w) {
   }
 }
 
+template <int BYTES>
+__device__ __forceinline__ void st_raw_stream(void* p, const uint32_t* w) {
+  if constexpr (BYTES == 16) {
+    __stcs(reinterpret_cast<uint4*>(p), make_uint4(w[0], w[1], w[2], w[3]));
+  } else if constexpr (BYTES == 32) {
+    __stcs(reinterpret_cast<uint4*>(p), make_uint4(w[0], w[1], w[2], w[3]));
+    __stcs(reinterpret_cast<uint4*>(p) + 1, make_uint4(w[4], w[5], w[6], w[7]));
+  } else if constexpr (BYTES == 8) {
+    __stcs(reinterpret_cast<uint2*>(p), make_uint2(w[0], w[1]));
+  } else {
+    __stcs(reinterpret_cast<uint32_t*>(p), w[0]);
+  }
+}
+
 // ---- element decode: raw words -> floats
 __device__ __forceinline__ float bf16_bits_to_float(uint32_t h) { return __uint_as_float(h << 16); }
 

@@ -55,6 +55,25 @@ def test_dynamic_rescale(n, in_dt, out_dt, stat):
     assert np.array_equal(to_bits(Y.data, out_dt), yo)
 
 
+@pytest.mark.parametrize("stat", [sc.STAT_AMAX, sc.STAT_L2])
+@pytest.mark.parametrize("in_dt,out_dt,in_place", [(orc.BF16, orc.E4M3, False), (orc.F16, orc.F16, True)])
+def test_dynamic_rescale_many_tiles_per_block(stat, in_dt, out_dt, in_place):
+    """Several tiles per block plus a ragged tail: every block of the one-launch rescale walks its
+    run of tiles forward for the statistic and backward for the rebalance."""
+    n = 8 * 1024 * 2700 + 13
+    x = si.to_bits(si.normal(35, n, (n,), 11.0), in_dt)
+    X = st(x, in_dt, 2.0 ** 3)
+    Y = X if in_place else sc.ScaledTensor.empty((n,), sc.TORCH_DTYPE[out_dt])
+    ws = new_ws()
+    sc.scalify_rescale(X, Y, stat=stat, ws=ws)
+    assert ws.check_status() == 0
+    yo, ys, so = orc.rescale(x, in_dt, 2.0 ** 3, stat, out_dt)
+    got_stat = float(ws.statistic().item())
+    assert got_stat == so if stat == sc.STAT_AMAX else abs(got_stat - so) <= 2e-6 * so
+    assert Y.scale_value() == ys
+    assert np.array_equal(to_bits(Y.data, out_dt), yo)
+
+
 @pytest.mark.parametrize("in_dt", [orc.E4M3, orc.E5M2, orc.F16, orc.BF16, orc.F32])
 def test_statistic_kernel(in_dt):
     n = 3 * 256 * 64 + 11
