@@ -225,8 +225,9 @@ int launch_adam(int n_tensors, const scalify_array* grads, scalify_array* m, sca
     adam_scales_kernel<<<(cnt + 127) / 128, 128, 0, st>>>(sp, h, fac, view.status);
     SCALIFY_CUDA_TRY(cudaGetLastError());
     const int total = tab.chunk_start[cnt];
-    const int cap = sm_count() * 8;
-    const int grid = total < cap ? total : cap;
+    // one chunk per block: the hardware scheduler balances the blocks over the SMs (measured
+    // faster on B200 than a grid of 8 blocks per SM striding over the chunks)
+    const int grid = total > 0 ? total : 1;
 #define SCALIFY_ADAM_LAUNCH(G, MV, W) \
   adam_update_kernel<G, MV, W><<<grid, kAdamThreads, 0, st>>>(tab, fac, h)
     SCALIFY_DISPATCH_DTYPE(g_dt, GDT, {

@@ -3,10 +3,9 @@
 // HBM-bound: every element of X (and G) is read once and every output written once.  A row is
 // owned by a team of TW warps (TW = 1, 2, 4 or 8, chosen so that a thread holds at most two
 // 16-byte vectors of the row); the row stays in registers, so mean, variance and the normalised
-// values come from one read.  Blocks of 256 threads hold 8/TW teams and stride over the rows with
-// a grid that is a multiple of the SM count.  Rows are fetched ahead of use: the forward kernel
-// stages each thread's vectors of the next four rows in shared memory with cp.async, the backward
-// kernel keeps the raw words of the next row in registers.  gamma and beta for a thread's fixed
+// values come from one read.  Blocks of 256 threads hold 8/TW teams.  Rows are fetched ahead of
+// use: the forward kernel stages each thread's vectors of the next four rows in shared memory
+// with cp.async, the backward kernel keeps the raw words of the next row in registers.  gamma and beta for a thread's fixed
 // columns are converted once and kept in registers.
 #include "scalify_common.cuh"
 #include "scalify_launch.h"
@@ -102,12 +101,12 @@ __device__ __forceinline__ void load_param_vec(const void* p, int dt, int c, flo
 // ---------------------------------------------------------------------------------------------
 // forward
 // ---------------------------------------------------------------------------------------------
-template <int XDT, int YDT, int TW>
+template <int XDT, int YDT, int TW, int VPT>
 __global__ void __launch_bounds__(kLnThreads) layernorm_fwd_kernel(
     const void* __restrict__ X, int64_t x_ld, void* __restrict__ Y, int64_t y_ld, int R, int d,
     const void* __restrict__ gamma, const void* __restrict__ beta, int gb_dt, const float* gamma_scale,
     const float* beta_scale, float* y_scale, float eps, int eps_inside, float* __restrict__ mean_out,
-    float* __restrict__ rinv_out) {
+    float* __restrict__ rinv_out, int rows_per_team) {
   constexpr int VEC = 16 / ElemBytes<XDT>::v;
   constexpr int OB = VEC * ElemBytes<YDT>::v;
   constexpr int TEAM = 32 * TW;
@@ -123,13 +122,33 @@ __global__ void __launch_bounds__(kLnThreads) layernorm_fwd_kernel(
     fg = gs / ys;
     fb = bs / ys;
   }
-  // this thread's columns: vectors t and t + TEAM
-  bool has[kLnVpt];
-  float gam[kLnVpt][VEC], bet[kLnVpt][VEC];
+  // this thread's columns: vectors t, t + TEAM, ...
+  bool has[VPT];
 #pragma unroll
-  for (int v = 0; v < kLnVpt; ++v) {
+  for (int v = 0; v < VPT; ++v) has[v] = (t + v * TEAM) < n_vec;
+  const float inv_d = 1.0f / static_cast<float>(d);
+  // a block owns TPB * rows_per_team consecutive rows; each iteration its teams take TPB adjacent rows
+  constexpr int rows_per_iter = TPB;
+  const int iters = rows_per_team;
+  int buf = 0;
+  extern __shared__ uint4 ln_stage[];  // [stage][v][thread]
+  auto issue = [&](int row, int slot) {
+#pragma unroll
+    for (int v = 0; v < VPT; ++v) {
+      if (has[v] && row < R)
+        cp_async16(&ln_stage[(slot * VPT + v) * kLnThreads + threadIdx.x],
+                   static_cast<const char*>(X) + (int64_t(row) * x_ld) * ElemBytes<XDT>::v + int64_t(t + v * TEAM) * 16);
+    }
+    cp_async_commit();  // one group per row, even when empty, so that the group count stays uniform
+  };
+  const int first_row = blockIdx.x * (TPB * rows_per_team) + team;
+#pragma unroll
+  for (int st = 0; st < kLnFwdStages; ++st) issue(first_row + st * rows_per_iter, st);
+  // gamma and beta of this thread's columns, requested after the first rows so that both are in flight together
+  float gam[VPT][VEC], bet[VPT][VEC];
+#pragma unroll
+  for (int v = 0; v < VPT; ++v) {
     const int vi = t + v * TEAM;
-    has[v] = vi < n_vec;
 #pragma unroll
     for (int e = 0; e < VEC; ++e) { gam[v][e] = 1.0f; bet[v][e] = 0.0f; }
     if (has[v] && gamma) {
@@ -141,34 +160,17 @@ __global__ void __launch_bounds__(kLnThreads) layernorm_fwd_kernel(
       }
     }
   }
-  const float inv_d = 1.0f / static_cast<float>(d);
-  const int rows_per_iter = gridDim.x * TPB;
-  const int iters = (R + rows_per_iter - 1) / rows_per_iter;
-  int buf = 0;
-  extern __shared__ uint4 ln_stage[];  // [stage][v][thread]
-  auto issue = [&](int row, int slot) {
-#pragma unroll
-    for (int v = 0; v < kLnVpt; ++v) {
-      if (has[v] && row < R)
-        cp_async16(&ln_stage[(slot * kLnVpt + v) * kLnThreads + threadIdx.x],
-                   static_cast<const char*>(X) + (int64_t(row) * x_ld) * ElemBytes<XDT>::v + int64_t(t + v * TEAM) * 16);
-    }
-    cp_async_commit();  // one group per row, even when empty, so that the group count stays uniform
-  };
-  const int first_row = blockIdx.x * TPB + team;
-#pragma unroll
-  for (int st = 0; st < kLnFwdStages; ++st) issue(first_row + st * rows_per_iter, st);
   int slot = 0;
   for (int it = 0; it < iters; ++it) {
     const int row = it * rows_per_iter + first_row;
     const bool live = row < R;
-    float x[kLnVpt][VEC];
+    float x[VPT][VEC];
     cp_async_wait<kLnFwdStages - 1>();  // the oldest row in flight has landed
 #pragma unroll
-    for (int v = 0; v < kLnVpt; ++v) {
+    for (int v = 0; v < VPT; ++v) {
       uint32_t w[4] = {0u, 0u, 0u, 0u};
       if (has[v] && live) {
-        const uint4 q4 = ln_stage[(slot * kLnVpt + v) * kLnThreads + threadIdx.x];
+        const uint4 q4 = ln_stage[(slot * VPT + v) * kLnThreads + threadIdx.x];
         w[0] = q4.x; w[1] = q4.y; w[2] = q4.z; w[3] = q4.w;
       }
       decode_vec<XDT, VEC>(w, x[v]);
@@ -177,13 +179,13 @@ __global__ void __launch_bounds__(kLnThreads) layernorm_fwd_kernel(
     if (++slot == kLnFwdStages) slot = 0;
     float s = 0.f;
 #pragma unroll
-    for (int v = 0; v < kLnVpt; ++v)
+    for (int v = 0; v < VPT; ++v)
 #pragma unroll
       for (int e = 0; e < VEC; ++e) s += x[v][e];  // absent vectors hold zeros
     const float mu = team_sum1<TW>(s, smem, team, buf) * inv_d;
     float q = 0.f;
 #pragma unroll
-    for (int v = 0; v < kLnVpt; ++v) {
+    for (int v = 0; v < VPT; ++v) {
       if (has[v]) {
 #pragma unroll
         for (int e = 0; e < VEC; ++e) { x[v][e] -= mu; q = fmaf(x[v][e], x[v][e], q); }
@@ -199,7 +201,7 @@ __global__ void __launch_bounds__(kLnThreads) layernorm_fwd_kernel(
       const float rg = rinv * fg;  // exact: fg is a power of two
       char* yrow = static_cast<char*>(Y) + int64_t(row) * y_ld * ElemBytes<YDT>::v;
 #pragma unroll
-      for (int v = 0; v < kLnVpt; ++v) {
+      for (int v = 0; v < VPT; ++v) {
         if (has[v]) {
           float o[VEC];
 #pragma unroll
@@ -233,19 +235,40 @@ int launch_layernorm_fwd(const void* X, int x_dt, int64_t x_ld, void* Y, int y_d
                          const void* gamma, const void* beta, int gb_dt, const float* gamma_scale,
                          const float* beta_scale, float* y_scale, float eps, int eps_inside, float* mean,
                          float* rinv, cudaStream_t st) {
-  const int tw = ln_team_warps(d, x_dt);
+  int tw = ln_team_warps(d, x_dt);
   if (tw == 0) return SCALIFY_ERR_UNSUPPORTED;
-  const int grid = ln_grid(R, 8 / tw, 3);
-#define SCALIFY_LN_FWD(W)                                                                                      \
-  layernorm_fwd_kernel<XDT, YDT, W><<<grid, kLnThreads, kLnFwdStages * kLnVpt * kLnThreads * 16, st>>>(X, x_ld, Y, y_ld, R, d, gamma, beta, gb_dt,    \
-                                                                 gamma_scale, beta_scale, y_scale, eps,         \
-                                                                 eps_inside, mean, rinv)
+  // rows of 65..128 vectors: one warp per row with four vectors per thread (no cross-warp step)
+  const int n_vec = d * elem_size(x_dt) / 16;
+  const bool wide = n_vec > 64 && n_vec <= 128;
+  if (wide) tw = 1;
+  // Blocks are not persistent: each owns a short run of consecutive rows (6 per team) and the
+  // hardware scheduler hands out the runs in address order.  Measured on B200 (131072 x 1024 BF16):
+  // 90 us, against 104 us for a grid of 3 blocks per SM striding over the rows, and 101 us with 16
+  // rows per team (fewer, longer blocks leave a larger partial last wave).
+  const int tpb = 8 / tw;
+  int rpt = 6;
+  while (rpt > 1 && (int64_t(R) + tpb * rpt - 1) / (tpb * rpt) < 4 * int64_t(sm_count())) --rpt;
+  const int grid = static_cast<int>((int64_t(R) + tpb * rpt - 1) / (tpb * rpt));
+#define SCALIFY_LN_FWD(W, V)                                                                                   \
+  do {                                                                                                         \
+    constexpr int kSmem = kLnFwdStages * V * kLnThreads * 16;                                                  \
+    if (kSmem > 48 * 1024)                                                                                     \
+      SCALIFY_CUDA_TRY(cudaFuncSetAttribute(layernorm_fwd_kernel<XDT, YDT, W, V>,                              \
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem));              \
+    layernorm_fwd_kernel<XDT, YDT, W, V><<<grid, kLnThreads, kSmem, st>>>(                                     \
+        X, x_ld, Y, y_ld, R, d, gamma, beta, gb_dt, gamma_scale, beta_scale, y_scale, eps, eps_inside, mean,   \
+        rinv, rpt);                                                                                                \
+  } while (0)
   SCALIFY_DISPATCH_WIDE(x_dt, XDT, SCALIFY_DISPATCH_DTYPE(y_dt, YDT, {
-    switch (tw) {
-      case 1: SCALIFY_LN_FWD(1); break;
-      case 2: SCALIFY_LN_FWD(2); break;
-      case 4: SCALIFY_LN_FWD(4); break;
-      default: SCALIFY_LN_FWD(8); break;
+    if (wide) {
+      SCALIFY_LN_FWD(1, 4);
+    } else {
+      switch (tw) {
+        case 1: SCALIFY_LN_FWD(1, 2); break;
+        case 2: SCALIFY_LN_FWD(2, 2); break;
+        case 4: SCALIFY_LN_FWD(4, 2); break;
+        default: SCALIFY_LN_FWD(8, 2); break;
+      }
     }
   }));
 #undef SCALIFY_LN_FWD
