@@ -105,7 +105,12 @@ enum {
  * The first 256 bytes of a workspace form a header (status word, statistic
  * word, reduction tickets); scalify_workspace_init must have zeroed it once
  * before first use.  One workspace may serve successive calls on one stream;
- * two calls that may overlap on the GPU need separate workspaces. */
+ * two calls that may overlap on the GPU need separate workspaces.
+ * For SCALIFY_OP_RESCALE and SCALIFY_OP_STATISTIC the figure grows with d0
+ * (one fp64 partial per block of the statistic pass, at most 512 KiB); those
+ * two calls also accept any smaller workspace of at least 4096 bytes and
+ * then run the statistic pass with fewer, longer blocks (same result for
+ * AMAX; for L2 the fp64 partial sums are combined in a different grouping). */
 size_t scalify_workspace_bytes(int op, int64_t d0, int64_t d1);
 
 /* Zero the workspace header (asynchronously, on `stream`). */

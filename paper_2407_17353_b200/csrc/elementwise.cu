@@ -57,7 +57,7 @@ __global__ void __launch_bounds__(kThreads) statistic_kernel(const void* __restr
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
       int64_t i = base + u * kThreads + threadIdx.x;
-      if (i < v1) ld_raw_stream<16>(static_cast<const char*>(x) + i * 16, w[u]);
+      if (i < v1) ld_raw<16>(static_cast<const char*>(x) + i * 16, w[u]);
       else { w[u][0] = w[u][1] = w[u][2] = w[u][3] = 0u; }
     }
 #pragma unroll
@@ -140,14 +140,27 @@ __global__ void __launch_bounds__(kThreads) statistic_kernel(const void* __restr
   }
 }
 
-int launch_statistic(const void* x, int dtype, int64_t n, int stat, void* ws, float* out_stat, cudaStream_t st) {
+// Blocks wanted for a statistic over n elements of at most 4 bytes: about four tiles each (many
+// more blocks than fit on the device at once, so the hardware scheduler balances them), at most 65536.
+int64_t statistic_blocks_wanted(int64_t n, int elem_bytes) {
+  const int64_t tiles = (n * elem_bytes / 16 + int64_t(kThreads) * kUnroll - 1) / (int64_t(kThreads) * kUnroll);
+  int64_t blocks = (tiles + 3) / 4;
+  const int64_t floor_blocks = int64_t(sm_count()) * 8;
+  if (blocks < floor_blocks) blocks = tiles < floor_blocks ? (tiles > 0 ? tiles : 1) : floor_blocks;
+  return blocks < 65536 ? blocks : 65536;
+}
+
+int launch_statistic(const void* x, int dtype, int64_t n, int stat, void* ws, size_t ws_bytes, float* out_stat,
+                     cudaStream_t st) {
   WsView v = ws_view(ws);
-  constexpr int VECB = 16;
-  int64_t n_vec = n * elem_size(dtype) / VECB;
-  int grid = grid_for(n_vec, 8);
+  // one partial per block: a workspace smaller than scalify_workspace_bytes() asks for gets fewer blocks
+  int64_t grid = statistic_blocks_wanted(n, elem_size(dtype));
+  const int64_t room = static_cast<int64_t>((ws_bytes - kWsHeader) / sizeof(double));
+  if (grid > room) grid = room;
+  if (grid < 1) grid = 1;
   SCALIFY_DISPATCH_DTYPE(dtype, DT,
-      statistic_kernel<DT><<<grid, kThreads, 0, st>>>(x, n, stat, static_cast<double*>(v.area), v.ticket, v.stat,
-                                                      out_stat));
+      statistic_kernel<DT><<<static_cast<int>(grid), kThreads, 0, st>>>(x, n, stat, static_cast<double*>(v.area),
+                                                                       v.ticket, v.stat, out_stat));
   SCALIFY_CUDA_TRY(cudaGetLastError());
   return SCALIFY_OK;
 }
@@ -380,8 +393,9 @@ static int fused_rescale_blocks_per_sm() {
 // Returns SCALIFY_OK after a cooperative launch, 1 if the device cannot run one (the caller then
 // takes the two-launch path), or an error code.
 int launch_fused_rescale(const void* x, int in_dt, void* y, int out_dt, int64_t n, int stat, const float* x_scale,
-                         float* y_scale, void* ws, cudaStream_t st) {
+                         float* y_scale, void* ws, size_t ws_bytes, cudaStream_t st) {
   WsView v = ws_view(ws);
+  const int64_t room = static_cast<int64_t>((ws_bytes - kWsHeader) / sizeof(double));
   int big = elem_size(in_dt) > elem_size(out_dt) ? elem_size(in_dt) : elem_size(out_dt);
   int64_t n_vec = n / (16 / big);
   double* partials = static_cast<double*>(v.area);
@@ -393,6 +407,7 @@ int launch_fused_rescale(const void* x, int in_dt, void* y, int out_dt, int64_t 
     int per_sm = fused_rescale_blocks_per_sm<IN, OUT>();
     if (per_sm > 0) {
       int grid = grid_for(n_vec, per_sm < 8 ? per_sm : 8);
+      if (grid > room) grid = static_cast<int>(room);
       cudaError_t e = cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(fused_rescale_kernel<IN, OUT>),
                                                   dim3(grid), dim3(kThreads), args, 0, st);
       if (e == cudaSuccess) rc = SCALIFY_OK;

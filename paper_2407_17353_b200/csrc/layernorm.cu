@@ -311,13 +311,12 @@ __global__ void __launch_bounds__(kLnThreads, 2) layernorm_bwd_kernel(
   const int iters = (R + rows_per_iter - 1) / rows_per_iter;
   int buf = 0;
   // the raw words of the team's next row are fetched before the current row is processed
-  uint32_t nx[kLnVpt][4], ng[kLnVpt][4];
+  // (zeroed once: words of absent vectors or rows past the end are decoded but never used)
+  uint32_t nx[kLnVpt][4] = {}, ng[kLnVpt][4] = {};
   float nmu = 0.f, nrinv = 0.f;
   auto fetch = [&](int row) {
 #pragma unroll
     for (int v = 0; v < kLnVpt; ++v) {
-      nx[v][0] = nx[v][1] = nx[v][2] = nx[v][3] = 0u;
-      ng[v][0] = ng[v][1] = ng[v][2] = ng[v][3] = 0u;
       if (has[v] && row < R) {
         ld_raw_stream<16>(static_cast<const char*>(X) + (int64_t(row) * x_ld) * ElemBytes<XDT>::v +
                               int64_t(t + v * TEAM) * 16, nx[v]);
@@ -368,6 +367,7 @@ __global__ void __launch_bounds__(kLnThreads, 2) layernorm_bwd_kernel(
       const float s = __fdividef(1.0f, rinv) - eps;
       c2 = (s > 0.f) ? __fdividef(m2, s) : 0.f;
     }
+    const float nm1r = -m1 * rinv;
     if (live) {
       char* orow = static_cast<char*>(dX) + int64_t(row) * dx_ld * ElemBytes<DXDT>::v;
 #pragma unroll
@@ -375,7 +375,7 @@ __global__ void __launch_bounds__(kLnThreads, 2) layernorm_bwd_kernel(
         if (has[v]) {
           float o[VEC];
 #pragma unroll
-          for (int e = 0; e < VEC; ++e) o[e] = fmaf(-x[v][e], c2, (g[v][e] - m1) * rinv);
+          for (int e = 0; e < VEC; ++e) o[e] = fmaf(g[v][e], rinv, fmaf(x[v][e], -c2, nm1r));
           uint32_t ow[OB / 4];
           encode_vec<DXDT, VEC>(o, ow);
           st_raw<OB>(orow + int64_t(t + v * TEAM) * OB, ow);

@@ -105,7 +105,10 @@ size_t scalify_workspace_bytes(int op, int64_t d0, int64_t d1) {
   switch (op) {
     case SCALIFY_OP_MATMUL: n = matmul_ws_bytes(d0, d1); break;
     case SCALIFY_OP_RESCALE:
-    case SCALIFY_OP_STATISTIC: n = stat_bytes; break;
+    case SCALIFY_OP_STATISTIC:
+      // one fp64 partial per block of the statistic pass over d0 elements (of at most 4 bytes)
+      n = kWsHeader + size_t(statistic_blocks_wanted(d0 > 0 ? d0 : 0, 4)) * sizeof(double) + 256;
+      break;
     case SCALIFY_OP_LAYERNORM_BWD: n = layernorm_bwd_ws_bytes(d0, d1); break;
     case SCALIFY_OP_ADAM: n = adam_ws_bytes(d0); break;
     case SCALIFY_OP_CROSS_ENTROPY: n = cross_entropy_ws_bytes(d0); break;
@@ -149,9 +152,10 @@ int scalify_statistic(const scalify_array* X, int stat, float* out_stat, void* w
   if (stat != SCALIFY_STAT_AMAX && stat != SCALIFY_STAT_L2) return SCALIFY_ERR_VALUE;
   const int64_t n = contiguous_numel(X);
   if (n < 0) return SCALIFY_ERR_SHAPE;
-  rc = check_ws(workspace, workspace_bytes, scalify_workspace_bytes(SCALIFY_OP_STATISTIC, n, 0));
+  rc = check_ws(workspace, workspace_bytes, kWsMin);
   if (rc) return rc;
-  return launch_statistic(X->data, X->dtype, n, stat, workspace, out_stat, static_cast<cudaStream_t>(stream));
+  return launch_statistic(X->data, X->dtype, n, stat, workspace, workspace_bytes, out_stat,
+                          static_cast<cudaStream_t>(stream));
 }
 
 int scalify_rescale(const scalify_array* X, int stat, const float* new_scale, const float* stat_in, scalify_array* Y,
@@ -182,13 +186,14 @@ int scalify_rescale(const scalify_array* X, int stat, const float* new_scale, co
     return launch_rebalance(X->data, X->dtype, Y->data, Y->dtype, n, X->scale, Y->scale, stat_in, nullptr,
                             kModeDynamic, status, st);
   }
-  rc = check_ws(workspace, workspace_bytes, scalify_workspace_bytes(SCALIFY_OP_RESCALE, n, 0));
+  rc = check_ws(workspace, workspace_bytes, kWsMin);
   if (rc) return rc;
   // one cooperative launch (statistic, grid barrier, rebalance); two launches where the device
   // cannot run a cooperative grid
-  rc = launch_fused_rescale(X->data, X->dtype, Y->data, Y->dtype, n, stat, X->scale, Y->scale, workspace, st);
+  rc = launch_fused_rescale(X->data, X->dtype, Y->data, Y->dtype, n, stat, X->scale, Y->scale, workspace,
+                            workspace_bytes, st);
   if (rc <= 0) return rc;
-  rc = launch_statistic(X->data, X->dtype, n, stat, workspace, nullptr, st);
+  rc = launch_statistic(X->data, X->dtype, n, stat, workspace, workspace_bytes, nullptr, st);
   if (rc) return rc;
   return launch_rebalance(X->data, X->dtype, Y->data, Y->dtype, n, X->scale, Y->scale, ws_view(workspace).stat,
                           nullptr, kModeDynamic, status, st);
