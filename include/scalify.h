@@ -354,6 +354,23 @@ int scalify_scaled_adam_step(int n_tensors, const scalify_array* grads, scalify_
                              void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The same step, which also writes the low-precision compute copy of every
+ * updated weight that the next forward pass multiplies with (the static cast
+ * on the forward path, Appendix A; Section 4: FP8 matmul operands, wider master
+ * weights): w_cast[i]_d = cast(stored w'[i]_d), w_cast[i]_s = w'[i]_s.  The
+ * cast starts from the value as stored in w[i] (already rounded to its dtype),
+ * so the copy is bit-identical to a separate scalify_rescale(STAT_NONE) of
+ * w[i], at one extra written byte per parameter instead of a 3-byte pass.
+ *   w_cast[i]: E4M3, E5M2, F16 or BF16 (all the same, narrower than w[i]),
+ *   contiguous, same element count as w[i], own scale word (no aliasing with
+ *   g, m, v, w scale words; data must not alias w[i]).
+ * Errors as scalify_scaled_adam_step; SCALIFY_ERR_NULL when w_cast is NULL.
+ */
+int scalify_scaled_adam_step_cast(int n_tensors, const scalify_array* grads, scalify_array* m, scalify_array* v,
+                                  scalify_array* w, scalify_array* w_cast, float lr, float beta1, float beta2,
+                                  float eps, int64_t step, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Scaled Adam step without a workspace.  (No counterpart in the paper: this entry point exists
  * for the integration, not for the method.)
  *

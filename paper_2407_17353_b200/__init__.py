@@ -75,6 +75,7 @@ def lib() -> ctypes.CDLL:
         L.scalify_scaled_gelu.argtypes = [P, i32, P, vp]
         L.scalify_scaled_gelu_bwd.argtypes = [P, P, i32, P, vp]
         L.scalify_scaled_adam_step.argtypes = [i32, P, P, P, P, f32, f32, f32, f32, i64, vp, sz, vp]
+        L.scalify_scaled_adam_step_cast.argtypes = [i32, P, P, P, P, P, f32, f32, f32, f32, i64, vp, sz, vp]
         L.scalify_debug_expire_wait.argtypes = [vp, sz, c.c_uint32, vp, vp]
         L.scalify_scalar_mul_pow2.argtypes = [P, f32, vp]
         L.scalify_scaled_embedding.argtypes = [vp, i64, i64, P, P, P, vp, vp]
@@ -87,7 +88,7 @@ def lib() -> ctypes.CDLL:
                      "scalify_statistic",
                      "scalify_rescale", "scalify_scaled_add", "scalify_scaled_layernorm",
                      "scalify_scaled_layernorm_bwd", "scalify_scaled_gelu", "scalify_scaled_gelu_bwd",
-                     "scalify_scaled_adam_step", "scalify_scaled_adam_step_static", "scalify_scaled_embedding",
+                     "scalify_scaled_adam_step", "scalify_scaled_adam_step_cast", "scalify_scaled_adam_step_static", "scalify_scaled_embedding",
                      "scalify_scaled_embedding_bwd", "scalify_scaled_softmax", "scalify_scaled_softmax_bwd",
                      "scalify_scaled_cross_entropy", "scalify_scalar_mul_pow2", "scalify_debug_expire_wait"):
             getattr(L, name).restype = i32
@@ -283,6 +284,19 @@ def scalify_scaled_adam_step(tensors: AdamTensors, ws: Workspace, *, lr: float, 
     _check(lib().scalify_scaled_adam_step(tensors.n, tensors.g, tensors.m, tensors.v, tensors.w, float(lr),
                                           float(beta1), float(beta2), float(eps), int(step), ws.ptr, ws.nbytes,
                                           _stream(stream)), "scalify_scaled_adam_step")
+
+
+def scalify_scaled_adam_step_cast(tensors: AdamTensors, w_cast: Sequence[ScaledTensor], ws: Workspace, *, lr: float,
+                                  beta1: float, beta2: float, eps: float, step: int, stream=None) -> None:
+    """Adam step that also writes the low-precision compute copy of every updated weight."""
+    assert len(w_cast) == tensors.n
+    wc = getattr(tensors, "_wc_cache", None)
+    if wc is None or wc[0] is not w_cast:
+        wc = (w_cast, _desc_array(w_cast))
+        tensors._wc_cache = wc
+    _check(lib().scalify_scaled_adam_step_cast(tensors.n, tensors.g, tensors.m, tensors.v, tensors.w, wc[1],
+                                               float(lr), float(beta1), float(beta2), float(eps), int(step), ws.ptr,
+                                               ws.nbytes, _stream(stream)), "scalify_scaled_adam_step_cast")
 
 
 def scalify_scaled_adam_step_static(tensors: AdamTensors, *, lr: float, beta1: float, beta2: float, eps: float,

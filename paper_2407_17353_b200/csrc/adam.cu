@@ -24,6 +24,7 @@ struct AdamTensorPtrs {
   void* m;
   void* v;
   void* w;
+  void* wc;  // optional compute copy of the updated weight (static cast of the stored value), or null
 };
 
 struct AdamTable {
@@ -31,6 +32,7 @@ struct AdamTable {
   long long n[kAdamMaxTensors];
   int chunk_start[kAdamMaxTensors + 1];  // prefix sum of ceil(n/kAdamChunk)
   int count;
+  int wc_dt;  // dtype of the compute copies
 };
 
 struct AdamScalePtrs {
@@ -38,6 +40,7 @@ struct AdamScalePtrs {
   float* m[kAdamMaxTensors];
   float* v[kAdamMaxTensors];
   float* w[kAdamMaxTensors];
+  float* wc[kAdamMaxTensors];  // scale word of the compute copy, or null
   int count;
 };
 
@@ -86,6 +89,7 @@ __global__ void adam_scales_kernel(AdamScalePtrs sp, AdamHyper h, AdamFactors* _
   *sp.m[i] = ms2;
   *sp.v[i] = vs2;
   *sp.w[i] = ws2;
+  if (sp.wc[i]) *sp.wc[i] = ws2;  // a static cast keeps the scale (Appendix A)
 }
 
 // One element.  sqrt and the division use the hardware approximations (each within 2 ulp of fp32),
@@ -118,6 +122,31 @@ __device__ __forceinline__ void adam_vec(const uint32_t* wg, uint32_t* wm, uint3
   encode_vec<WDT, kAdamVec>(w, ww);
 }
 
+// Compute copy of the updated weight: the STORED value (already rounded to WDT) converted to the
+// copy's dtype, 8 elements -> 8 bytes (FP8) or 16 bytes (FP16 / BF16).
+template <int WDT>
+__device__ __forceinline__ void adam_cast_store(const uint32_t* ww, int dt, char* wcp, long long i) {
+  float w[kAdamVec];
+  decode_vec<WDT, kAdamVec>(ww, w);
+  if (dt == SCALIFY_E4M3) {
+    uint32_t o[2];
+    encode_vec<SCALIFY_E4M3, kAdamVec>(w, o);
+    st_raw<8>(wcp + i * 8, o);
+  } else if (dt == SCALIFY_E5M2) {
+    uint32_t o[2];
+    encode_vec<SCALIFY_E5M2, kAdamVec>(w, o);
+    st_raw<8>(wcp + i * 8, o);
+  } else if (dt == SCALIFY_BF16) {
+    uint32_t o[4];
+    encode_vec<SCALIFY_BF16, kAdamVec>(w, o);
+    st_raw<16>(wcp + i * 16, o);
+  } else {
+    uint32_t o[4];
+    encode_vec<SCALIFY_F16, kAdamVec>(w, o);
+    st_raw<16>(wcp + i * 16, o);
+  }
+}
+
 template <int GDT, int MVDT, int WDT>
 __global__ void __launch_bounds__(kAdamThreads) adam_update_kernel(const __grid_constant__ AdamTable tab,
                                                                    const AdamFactors* __restrict__ fac,
@@ -141,6 +170,7 @@ __global__ void __launch_bounds__(kAdamThreads) adam_update_kernel(const __grid_
     char* mp = static_cast<char*>(tab.t[ti].m);
     char* vp = static_cast<char*>(tab.t[ti].v);
     char* wp = static_cast<char*>(tab.t[ti].w);
+    char* wcp = static_cast<char*>(tab.t[ti].wc);
     uint32_t wg[4][GB / 4 > 0 ? GB / 4 : 1], wm[4][MB / 4], wv[4][MB / 4], ww[4][WB / 4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
@@ -160,6 +190,7 @@ __global__ void __launch_bounds__(kAdamThreads) adam_update_kernel(const __grid_
         st_raw<MB>(mp + i * MB, wm[u]);
         st_raw<MB>(vp + i * MB, wv[u]);
         st_raw<WB>(wp + i * WB, ww[u]);
+        if (wcp) adam_cast_store<WDT>(ww[u], tab.wc_dt, wcp, i);
       }
     }
     // ragged tail of the tensor (fewer than kAdamVec elements), done by its last chunk
@@ -171,6 +202,13 @@ __global__ void __launch_bounds__(kAdamThreads) adam_update_kernel(const __grid_
         store_elem<MVDT>(mp, i, mm);
         store_elem<MVDT>(vp, i, vv);
         store_elem<WDT>(wp, i, ww);
+        if (wcp) {
+          const float stored = round_through<WDT>(ww);
+          if (tab.wc_dt == SCALIFY_E4M3) store_elem<SCALIFY_E4M3>(wcp, i, stored);
+          else if (tab.wc_dt == SCALIFY_E5M2) store_elem<SCALIFY_E5M2>(wcp, i, stored);
+          else if (tab.wc_dt == SCALIFY_BF16) store_elem<SCALIFY_BF16>(wcp, i, stored);
+          else store_elem<SCALIFY_F16>(wcp, i, stored);
+        }
       }
     }
   }
@@ -186,7 +224,7 @@ static float host_p2_floor_abs(double c) {
 size_t adam_ws_bytes(int64_t n_tensors) { return kWsHeader + size_t(n_tensors) * sizeof(AdamFactors) + 256; }
 
 int launch_adam(int n_tensors, const scalify_array* grads, scalify_array* m, scalify_array* v, scalify_array* w,
-                const int64_t* numel, float lr, float beta1, float beta2, float eps, int64_t step, void* ws,
+                const scalify_array* w_cast, const int64_t* numel, float lr, float beta1, float beta2, float eps, int64_t step, void* ws,
                 cudaStream_t st) {
   WsView view = ws_view(ws);
   AdamFactors* fac_all = static_cast<AdamFactors*>(view.area);
@@ -209,11 +247,14 @@ int launch_adam(int n_tensors, const scalify_array* grads, scalify_array* m, sca
     AdamTable tab;
     AdamScalePtrs sp;
     tab.count = cnt;
+    tab.wc_dt = w_cast ? w_cast[0].dtype : SCALIFY_E4M3;
     sp.count = cnt;
     tab.chunk_start[0] = 0;
     for (int i = 0; i < cnt; ++i) {
       const int k = base + i;
       tab.t[i].g = grads[k].data; tab.t[i].m = m[k].data; tab.t[i].v = v[k].data; tab.t[i].w = w[k].data;
+      tab.t[i].wc = w_cast ? w_cast[k].data : nullptr;
+      sp.wc[i] = w_cast ? w_cast[k].scale : nullptr;
       tab.n[i] = numel[k];
       int64_t chunks = (numel[k] + kAdamChunk - 1) / kAdamChunk;
       if (chunks < 1) chunks = 1;

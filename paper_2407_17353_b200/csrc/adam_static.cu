@@ -82,7 +82,7 @@ extern "C" int scalify_scaled_adam_step_static(int n_tensors, const scalify_arra
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // the array keeps whatever the previous call left: the status word has to start at zero
   SCALIFY_CUDA_TRY(cudaMemsetAsync(scratch, 0, kWsHeader, st));
-  rc = launch_adam(n_tensors, grads, m, v, w, numel, lr, beta1, beta2, eps, step, scratch, st);
+  rc = launch_adam(n_tensors, grads, m, v, w, nullptr, numel, lr, beta1, beta2, eps, step, scratch, st);
   if (rc) return rc;
   if (status_out)
     SCALIFY_CUDA_TRY(cudaMemcpyAsync(status_out, scratch, sizeof(uint32_t), cudaMemcpyDeviceToDevice, st));

@@ -348,9 +348,9 @@ int scalify_scaled_layernorm_bwd(const scalify_array* G, const scalify_array* X,
   return rc;
 }
 
-int scalify_scaled_adam_step(int n_tensors, const scalify_array* grads, scalify_array* m, scalify_array* v,
-                             scalify_array* w, float lr, float beta1, float beta2, float eps, int64_t step,
-                             void* workspace, size_t workspace_bytes, void* stream) {
+static int adam_step_impl(int n_tensors, const scalify_array* grads, scalify_array* m, scalify_array* v,
+                          scalify_array* w, const scalify_array* w_cast, float lr, float beta1, float beta2,
+                          float eps, int64_t step, void* workspace, size_t workspace_bytes, void* stream) {
   if (n_tensors < 0) return SCALIFY_ERR_VALUE;
   if (n_tensors == 0) return SCALIFY_OK;
   if (!grads || !m || !v || !w) return SCALIFY_ERR_NULL;
@@ -385,13 +385,43 @@ int scalify_scaled_adam_step(int n_tensors, const scalify_array* grads, scalify_
       rc = SCALIFY_ERR_ALIAS;
       break;
     }
+    if (w_cast) {
+      const scalify_array* c = &w_cast[i];
+      if ((rc = check_array(c))) break;
+      if (!c->scale) { rc = SCALIFY_ERR_NULL; break; }
+      if (c->dtype == SCALIFY_F32 || c->dtype != w_cast[0].dtype || elem_size(c->dtype) >= elem_size(w[i].dtype)) {
+        rc = SCALIFY_ERR_DTYPE;  // the copy is narrower than the weight it is cast from
+        break;
+      }
+      if (contiguous_numel(c) != n) { rc = SCALIFY_ERR_SHAPE; break; }
+      if (c->scale == m[i].scale || c->scale == v[i].scale || c->scale == w[i].scale || c->scale == grads[i].scale ||
+          c->data == w[i].data) {
+        rc = SCALIFY_ERR_ALIAS;
+        break;
+      }
+    }
     numel[i] = n;
   }
   if (rc == SCALIFY_OK)
-    rc = launch_adam(n_tensors, grads, m, v, w, numel, lr, beta1, beta2, eps, step, workspace,
+    rc = launch_adam(n_tensors, grads, m, v, w, w_cast, numel, lr, beta1, beta2, eps, step, workspace,
                      static_cast<cudaStream_t>(stream));
   delete[] heap;
   return rc;
+}
+
+int scalify_scaled_adam_step(int n_tensors, const scalify_array* grads, scalify_array* m, scalify_array* v,
+                             scalify_array* w, float lr, float beta1, float beta2, float eps, int64_t step,
+                             void* workspace, size_t workspace_bytes, void* stream) {
+  return adam_step_impl(n_tensors, grads, m, v, w, nullptr, lr, beta1, beta2, eps, step, workspace, workspace_bytes,
+                        stream);
+}
+
+int scalify_scaled_adam_step_cast(int n_tensors, const scalify_array* grads, scalify_array* m, scalify_array* v,
+                                  scalify_array* w, scalify_array* w_cast, float lr, float beta1, float beta2,
+                                  float eps, int64_t step, void* workspace, size_t workspace_bytes, void* stream) {
+  if (n_tensors > 0 && !w_cast) return SCALIFY_ERR_NULL;
+  return adam_step_impl(n_tensors, grads, m, v, w, w_cast, lr, beta1, beta2, eps, step, workspace, workspace_bytes,
+                        stream);
 }
 
 int scalify_scaled_matmul(const scalify_array* A, int transA, const scalify_array* B, int transB, scalify_array* Y,

@@ -35,6 +35,7 @@ int launch_layernorm_bwd(const void* G, int64_t g_ld, const void* X, int x_dt, i
                          float* dgamma_scale, float* dbeta_scale, void* ws, cudaStream_t st);
 size_t adam_ws_bytes(int64_t n_tensors);
 int launch_adam(int n_tensors, const scalify_array* grads, scalify_array* m, scalify_array* v, scalify_array* w,
+                const scalify_array* w_cast,
                 const int64_t* numel, float lr, float beta1, float beta2, float eps, int64_t step, void* ws,
                 cudaStream_t st);
 

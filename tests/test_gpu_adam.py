@@ -144,3 +144,66 @@ def test_config4_gpt2_small_parameter_list_full_size_sampled():
     sc.scalify_scaled_adam_step(sc.AdamTensors(G, M, V, W), ws, step=1000, **hyper)
     assert ws.check_status() == 0
     _sampled_adam_parity(cases, G, M, V, W, hyper, 1000, np.random.default_rng(8), 2000)
+
+
+@pytest.mark.parametrize("w_dt,c_dt", [(orc.F16, orc.E4M3), (orc.F32, orc.E4M3), (orc.F32, orc.BF16),
+                                       (orc.BF16, orc.E5M2), (orc.F32, orc.F16)])
+def test_adam_step_with_compute_copy(w_dt, c_dt):
+    """The step that also emits the low-precision compute copy: m, v, w and their scales are bit-identical
+    to the plain step, and the copy is the oracle's static cast of the weight as stored, with w's new scale."""
+    sizes = [1, 13, 4096, 8192 * 3 + 5, 777]
+    lists = []
+    for variant in range(2):
+        G, M, V, W, cases = [], [], [], [], []
+        for i, n in enumerate(sizes):
+            c = si.adam_case(n, seed=90 + i, w_dtype=w_dt if w_dt != orc.BF16 else orc.F16)
+            if w_dt == orc.BF16:
+                c["w"] = si.to_bits(si.normal(90 + i, 1, (n,), 0.02 * 64.0), orc.BF16)
+                c["w_dtype"] = orc.BF16
+            cases.append(c)
+            G.append(sc.ScaledTensor.make(to_dev(c["g"], c["g_dtype"]), c["g_scale"]))
+            M.append(sc.ScaledTensor.make(to_dev(c["m"], c["mv_dtype"]), c["m_scale"]))
+            V.append(sc.ScaledTensor.make(to_dev(c["v"], c["mv_dtype"]), c["v_scale"]))
+            W.append(sc.ScaledTensor.make(to_dev(c["w"], c["w_dtype"]), c["w_scale"]))
+        lists.append((G, M, V, W, cases))
+    c0 = lists[0][4][0]
+    hyper = dict(lr=c0["lr"], beta1=c0["beta1"], beta2=c0["beta2"], eps=c0["eps"], step=7)
+    ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_ADAM, len(sizes)))
+    sc.scalify_scaled_adam_step(sc.AdamTensors(*lists[0][:4]), ws, **hyper)
+    WC = [sc.ScaledTensor.make(torch.zeros(n, dtype=sc.TORCH_DTYPE[c_dt], device="cuda"), 123.0) for n in sizes]
+    sc.scalify_scaled_adam_step_cast(sc.AdamTensors(*lists[1][:4]), WC, ws, **hyper)
+    assert ws.check_status() == 0
+    for k in range(len(sizes)):
+        for a, b, dt in ((lists[0][1][k], lists[1][1][k], orc.F16), (lists[0][2][k], lists[1][2][k], orc.F16),
+                         (lists[0][3][k], lists[1][3][k], w_dt)):
+            assert a.scale_value() == b.scale_value()
+            assert np.array_equal(to_bits(a.data, dt), to_bits(b.data, dt))
+        w_bits = to_bits(lists[1][3][k].data, w_dt)
+        want = orc.encode(orc.decode(w_bits, w_dt), c_dt)
+        assert np.array_equal(to_bits(WC[k].data, c_dt), want)
+        assert WC[k].scale_value() == lists[1][3][k].scale_value()
+
+
+def test_adam_step_with_compute_copy_rejects_bad_arguments():
+    n = 64
+    c = si.adam_case(n, seed=5, w_dtype=orc.F16)
+    G = [sc.ScaledTensor.make(to_dev(c["g"], c["g_dtype"]), c["g_scale"])]
+    M = [sc.ScaledTensor.make(to_dev(c["m"], c["mv_dtype"]), c["m_scale"])]
+    V = [sc.ScaledTensor.make(to_dev(c["v"], c["mv_dtype"]), c["v_scale"])]
+    W = [sc.ScaledTensor.make(to_dev(c["w"], c["w_dtype"]), c["w_scale"])]
+    ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_ADAM, 1))
+    hyper = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, step=1)
+    before = to_bits(W[0].data, orc.F16).copy()
+    # a copy as wide as the weight is not a compute copy
+    with pytest.raises(sc.ScalifyError):
+        sc.scalify_scaled_adam_step_cast(sc.AdamTensors(G, M, V, W),
+                                         [sc.ScaledTensor.make(torch.zeros(n, dtype=torch.float16, device="cuda"), 1.0)],
+                                         ws, **hyper)
+    # wrong element count
+    with pytest.raises(sc.ScalifyError):
+        sc.scalify_scaled_adam_step_cast(sc.AdamTensors(G, M, V, W),
+                                         [sc.ScaledTensor.make(torch.zeros(n + 16, dtype=torch.float8_e4m3fn,
+                                                                           device="cuda"), 1.0)], ws, **hyper)
+    # a failed call launched nothing
+    torch.cuda.synchronize()
+    assert np.array_equal(to_bits(W[0].data, orc.F16), before)
