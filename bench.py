@@ -43,7 +43,7 @@ REFERENCE_ROWS_PER_STEP = 32  # --impl reference: rows per timed step
 
 # DRAM traffic of one 8192^3 GEMM launch (dram__bytes_read.sum + dram__bytes_write.sum), from the ncu
 # capture summarised in profiles/ (algorithmic bytes: 268 MB).
-GEMM_DRAM_TRAFFIC_BYTES = 460_373_504  # profiles/matmul_8192_e4m3_two_cta_ncu.md: 345.3 MB read + 115.1 MB written
+GEMM_DRAM_TRAFFIC_BYTES = 358_119_424  # profiles/matmul_8192_e4m3_two_cta_ncu.md: 240.0 MB read + 118.1 MB written
 
 
 def load_peaks():
@@ -269,6 +269,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (for ncu launch lists)")
+    ap.add_argument("--no-next", action="store_true",
+                    help="skip the separately timed next-row variants f1, f2 (for ncu launch lists of the step)")
     ap.add_argument("--profile-row", default=None, choices=["matmul", "rescale", "add", "layernorm", "adam"],
                     help="run only this row on a reduced, still larger-than-L2 case (for ncu captures)")
     args = ap.parse_args()
@@ -422,17 +424,17 @@ def main():
     def delayed_step():
         sc.scalify_scaled_matmul_delayed(A, Bt, stat_state, Yd, ws_mm, transB=True, stat=sc.STAT_AMAX,
                                          stat_out=stat_state)
-    for _ in range(3):
+    for _ in range(0 if args.no_next else 3):
         delayed_step()
     barrier()
     d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    d_iters = max(3, min(K, 20))
+    d_iters = 0 if args.no_next else max(3, min(K, 20))
     d0.record()
     for _ in range(d_iters):
         delayed_step()
     d1.record()
     barrier()
-    delayed_ms = d0.elapsed_time(d1) / d_iters
+    delayed_ms = d0.elapsed_time(d1) / d_iters if d_iters else float("nan")
 
     # Adam that also writes the E4M3 compute copy of the updated weight (1 more byte per parameter)
     awc = sc.ScaledTensor.make(torch.empty(ADAM_N, dtype=torch.float8_e4m3fn, device=dev), 1.0)
@@ -442,17 +444,17 @@ def main():
     def adam_cast_step(t):
         sc.scalify_scaled_adam_step_cast(adam, wc_list, ws_ad, lr=3e-4, beta1=0.9, beta2=0.999, eps=1e-8,
                                          step=2000 + t)
-    for t in range(3):
+    for t in range(0 if args.no_next else 3):
         adam_cast_step(t)
     barrier()
     c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    c_iters = max(3, min(K, 20))
+    c_iters = 0 if args.no_next else max(3, min(K, 20))
     c0.record()
     for t in range(c_iters):
         adam_cast_step(t)
     c1.record()
     barrier()
-    adam_cast_ms = c0.elapsed_time(c1) / c_iters
+    adam_cast_ms = c0.elapsed_time(c1) / c_iters if c_iters else float("nan")
 
     # ------------------------------------------------------------------ end to end through host buffers
     hY = torch.empty((N_GEMM, N_GEMM), dtype=torch.int8).pin_memory()
