@@ -83,6 +83,10 @@ def lib() -> ctypes.CDLL:
         L.orc_cross_entropy.argtypes = [vp, i32, f32, i64, i64, i64, vp, i32, vp, pf32]
         L.orc_adam_step.argtypes = [i64, vp, i32, f32, vp, vp, i32, pf32, pf32, vp, i32, pf32,
                                     f32, f32, f32, f32, i64]
+        L.orc_e8m0_decode.restype = f64
+        L.orc_e8m0_decode.argtypes = [c.c_uint32]
+        L.orc_mx_quantize.argtypes = [vp, i32, i64, i64, i32, vp, vp]
+        L.orc_mx_matmul.argtypes = [vp, i32, vp, f32, vp, i32, vp, f32, i64, i64, i64, i32, vp, i64, pf32, vp, vp]
         _lib = L
     return _lib
 
@@ -349,3 +353,38 @@ def cross_entropy(logits, l_dtype, l_scale, n_classes, targets, g_dtype=None):
     loss = lib().orc_cross_entropy(_ptr(logits), l_dtype, float(l_scale), n, int(n_classes), ld, _ptr(targets),
                                    0 if g_dtype is None else g_dtype, _ptr(g), ctypes.byref(gs))
     return float(loss), g, float(gs.value)
+
+
+def e8m0_decode(code: int) -> float:
+    return float(lib().orc_e8m0_decode(int(code)))
+
+
+def mx_quantize(X, x_dtype, elem_dtype):
+    """Block-scale quantisation of the data component of X [R,K] (K % 32 == 0) along K.
+    Returns (element bits [R,K] uint8, E8M0 codes [R,K/32] uint8)."""
+    X = _bits(X, x_dtype)
+    R, K = X.shape
+    assert K % 32 == 0
+    data = np.empty((R, K), dtype=np.uint8)
+    codes = np.empty((R, K // 32), dtype=np.uint8)
+    lib().orc_mx_quantize(_ptr(X), x_dtype, R, K, elem_dtype, _ptr(data), _ptr(codes))
+    return data, codes
+
+
+def mx_matmul(A, a_dtype, Ea, a_scale, B, b_dtype, Eb, b_scale, y_dtype, want_acc=False):
+    """A [M,K], B [N,K] FP8 bits, Ea [M,K/32], Eb [N,K/32] E8M0 codes.
+    Returns (Y bits [M,N], Y scale, acc or None, sabs or None)."""
+    A = _bits(A, a_dtype)
+    B = _bits(B, b_dtype)
+    Ea = np.ascontiguousarray(Ea, dtype=np.uint8)
+    Eb = np.ascontiguousarray(Eb, dtype=np.uint8)
+    M, K = A.shape
+    N, Kb = B.shape
+    assert K == Kb and K % 32 == 0 and Ea.shape == (M, K // 32) and Eb.shape == (N, K // 32)
+    Y = np.empty((M, N), dtype=_BITS_NP[y_dtype])
+    ys = ctypes.c_float(0)
+    acc = np.empty((M, N), dtype=np.float64) if want_acc else None
+    sab = np.empty((M, N), dtype=np.float64) if want_acc else None
+    lib().orc_mx_matmul(_ptr(A), a_dtype, _ptr(Ea), float(a_scale), _ptr(B), b_dtype, _ptr(Eb), float(b_scale),
+                        M, N, K, y_dtype, _ptr(Y), N, ctypes.byref(ys), _ptr(acc), _ptr(sab))
+    return Y, float(ys.value), acc, sab

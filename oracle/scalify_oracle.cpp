@@ -25,7 +25,8 @@
 // (exhaustive codec round trips, comparison of the codecs with an independent
 // library cast, brute force on tiny matrices, closed forms, invariants,
 // finite differences, textbook Adam / LayerNorm; tests/test_oracle_support_ops.py pins
-// the embedding / softmax / cross-entropy readings against torch in fp64).
+// the embedding / softmax / cross-entropy readings against torch in fp64;
+// tests/test_oracle_mx.py pins the block-scale functions).
 
 #include <algorithm>
 #include <cmath>
@@ -688,6 +689,94 @@ void orc_adam_step(int64_t n, const void* g, int g_dtype, float g_scale,
   *m_scale = static_cast<float>(ms2);
   *v_scale = static_cast<float>(vs2);
   *w_scale = static_cast<float>(ws2);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Block scales (Section 2: the scale component may be any array broadcastable to the data; the
+// paper names E8M0 and the OCP micro-scaling formats as the standard it follows).
+//
+// Reading used here: a block-scaled ScaledArray is (data, E, scale) with
+//   value[i,k] = data[i,k] * 2^(E[i, k/32] - 127) * scale,
+// E an E8M0 code (0..254; 255 is NaN) shared by 32 consecutive elements of a row, i.e. along
+// the contraction dimension (OCP MX).  The tensor-wide scale stays one fp32 power of two and is
+// the only thing the static rules see; the block exponents belong to the data component.
+// ---------------------------------------------------------------------------------------------
+
+double orc_e8m0_decode(uint32_t code) {
+  if (code >= 255u) return std::numeric_limits<double>::quiet_NaN();
+  return std::ldexp(1.0, static_cast<int>(code) - 127);
+}
+
+// Largest power-of-two exponent of a normal number of the element format (OCP MX: "emax").
+static int elem_emax(int dtype) { return dtype == 0 ? 8 : 15; }
+
+// Quantise the data component of X [R,K] (K a multiple of 32) to FP8 elements with one E8M0
+// exponent per 32 elements: per block, e = floor(log2(max|x|)) - emax(element format), clamped
+// to the E8M0 range, data = encode(x / 2^e) (saturating, round to nearest even).  A block whose
+// maximum is zero or not finite gets e = 0, like a dynamic rescale whose statistic cannot
+// define a scale (Section 3.3).  This is the dynamic rescale with the AMAX statistic applied per
+// block, the power of two rounded DOWN as everywhere else (Section 3.2).
+void orc_mx_quantize(const void* X, int x_dtype, int64_t R, int64_t K, int elem_dtype, void* data_out,
+                     uint8_t* e8m0_out) {
+  const int64_t nb = K / 32;
+#pragma omp parallel for schedule(static)
+  for (int64_t i = 0; i < R; ++i) {
+    for (int64_t b = 0; b < nb; ++b) {
+      double v[32], amax = 0.0;
+      bool finite = true;
+      for (int t = 0; t < 32; ++t) {
+        v[t] = decode(load_bits(X, x_dtype, i * K + b * 32 + t), x_dtype);
+        if (!std::isfinite(v[t])) finite = false;
+        amax = std::max(amax, std::fabs(v[t]));
+      }
+      int e = 0;
+      if (finite && amax > 0.0) {
+        int ex;
+        std::frexp(amax, &ex);  // amax = f * 2^ex, f in [0.5, 1)  =>  floor(log2 amax) = ex - 1
+        e = (ex - 1) - elem_emax(elem_dtype);
+        e = std::max(-127, std::min(127, e));
+      }
+      e8m0_out[i * nb + b] = static_cast<uint8_t>(e + 127);
+      for (int t = 0; t < 32; ++t)
+        store_bits(data_out, elem_dtype, i * K + b * 32 + t, encode(std::ldexp(v[t], -e), elem_dtype));
+    }
+  }
+}
+
+// Block-scaled matmul with the static matmul rule on the tensor scales:
+//   Y_s = A_s * B_s * kf(K),   Y_d = (sum_k a[i,k] * b[j,k]) / kf(K),
+// a[i,k] = A_d[i,k] * 2^(Ea[i,k/32]-127), b[j,k] = B_d[j,k] * 2^(Eb[j,k/32]-127).
+// A is [M,K], B is [N,K] (both with the contraction dimension innermost), Ea [M,K/32],
+// Eb [N,K/32].  Optional acc / sabs outputs as in orc_scaled_matmul.
+void orc_mx_matmul(const void* A, int a_dtype, const uint8_t* Ea, float a_scale,
+                   const void* B, int b_dtype, const uint8_t* Eb, float b_scale,
+                   int64_t M, int64_t N, int64_t K, int y_dtype, void* Y, int64_t ldy, float* y_scale,
+                   double* acc_out, double* sabs_out) {
+  const int64_t nb = K / 32;
+  std::vector<double> Ad(static_cast<size_t>(M * K)), Bd(static_cast<size_t>(N * K));
+  for (int64_t i = 0; i < M; ++i)
+    for (int64_t k = 0; k < K; ++k)
+      Ad[i * K + k] = decode(load_bits(A, a_dtype, i * K + k), a_dtype) * orc_e8m0_decode(Ea[i * nb + k / 32]);
+  for (int64_t j = 0; j < N; ++j)
+    for (int64_t k = 0; k < K; ++k)
+      Bd[j * K + k] = decode(load_bits(B, b_dtype, j * K + k), b_dtype) * orc_e8m0_decode(Eb[j * nb + k / 32]);
+  const double f = kf(K);
+  if (y_scale) *y_scale = static_cast<float>(static_cast<double>(a_scale) * static_cast<double>(b_scale) * f);
+#pragma omp parallel for schedule(static)
+  for (int64_t i = 0; i < M; ++i) {
+    for (int64_t j = 0; j < N; ++j) {
+      double acc = 0.0, sab = 0.0;
+      for (int64_t k = 0; k < K; ++k) {
+        const double p = Ad[i * K + k] * Bd[j * K + k];
+        acc += p;
+        sab += std::fabs(p);
+      }
+      const double yd = acc / f;
+      if (Y) store_bits(Y, y_dtype, i * ldy + j, encode(yd, y_dtype));
+      if (acc_out) acc_out[i * N + j] = yd;
+      if (sabs_out) sabs_out[i * N + j] = sab / f;
+    }
+  }
 }
 
 }  // extern "C"
