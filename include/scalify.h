@@ -371,6 +371,63 @@ int scalify_scaled_adam_step_cast(int n_tensors, const scalify_array* grads, sca
                                   float eps, int64_t step, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Block scales (Section 2: the scale component may be any array that broadcasts
+ * against the data; the paper names the E8M0 exponent byte and the OCP
+ * micro-scaling formats as the standard it follows, and works with one scalar
+ * scale per tensor; this is the block form of the same representation).
+ *
+ * A block-scaled array is FP8 data [rows, K] (row-major, dense, K innermost),
+ * one E8M0 exponent per 32 consecutive elements of a row, and the usual
+ * tensor-wide fp32 power-of-two scale:
+ *   value[i,k] = data[i,k] * 2^(exponent[i, k/32] - 127) * scale.
+ * Only the tensor-wide scale takes part in the static scale rules; the
+ * exponents belong to the data component.
+ * K must be a multiple of 128.  `sf` holds the exponents in the order the
+ * block-scaled tensor-core instruction consumes: tiles of 128 rows x 4 blocks
+ * (512 bytes), tile (r, k) at byte ((r * (K/128)) + k) * 512, and inside a tile
+ * row `row`, block `blk` at byte (row % 32) * 16 + (row / 32) * 4 + blk.  The
+ * row count is padded up to a multiple of 256: scalify_mx_sf_bytes(rows, K)
+ * bytes, 16-byte aligned; the exponents of the padding rows must be valid
+ * (scalify_mx_quantize writes 127 there).  All pointers are DEVICE pointers
+ * owned by the caller.
+ */
+typedef struct scalify_mx_array {
+  void* data;     /* FP8 elements [rows, K], 16-byte aligned */
+  int32_t dtype;  /* SCALIFY_E4M3 or SCALIFY_E5M2 */
+  int64_t rows;
+  int64_t K;
+  uint8_t* sf;    /* E8M0 exponents, tiled as described above */
+  float* scale;   /* one fp32 power of two, or NULL (scale 1) */
+} scalify_mx_array;
+
+size_t scalify_mx_sf_bytes(int64_t rows, int64_t K);
+
+/*
+ * Quantises the data component of X [rows, K] (F16, BF16 or F32; row stride
+ * stride[0]) into Y: per block of 32 elements, exponent e = floor(log2(max|x|))
+ * - emax (emax = 8 for E4M3, 15 for E5M2: the OCP MX rule, i.e. a dynamic
+ * rescale with the AMAX statistic per block, Section 3.3, the power of two
+ * rounded down), clamped to [-127, 127]; data = round-to-nearest-even of
+ * x * 2^-e, saturating.  A block whose maximum is zero, infinite or NaN gets
+ * e = 0.  Y_s = X_s.  `status`: optional DEVICE word that receives
+ * SCALIFY_DEV_BAD_SCALE.  Errors: NULL, DTYPE, SHAPE (K % 128), ALIGNMENT.
+ */
+int scalify_mx_quantize(const scalify_array* X, scalify_mx_array* Y, uint32_t* status, void* stream);
+
+/*
+ * Block-scaled matmul with the static matmul rule (Section 3.2) on the
+ * tensor-wide scales:  Y_s = A_s * B_s * kf(K),
+ *   Y_d[i,j] = (sum_k A_d[i,k] 2^(Ea[i,k/32]-127) * B_d[j,k] 2^(Eb[j,k/32]-127)) / kf(K)
+ * with fp32 accumulation on the tensor cores (tcgen05 kind::mxf8f6f4 with the
+ * exponents in tensor memory).  A is [M,K], B is [N,K]; Y [M,N] is F16, BF16
+ * or F32 (row stride stride[0]).  stat: NONE, AMAX or L2 of the stored Y, left
+ * in the workspace's statistic word as by scalify_scaled_matmul.  Workspace:
+ * SCALIFY_OP_MATMUL (M, N).
+ */
+int scalify_mx_matmul(const scalify_mx_array* A, const scalify_mx_array* B, scalify_array* Y, int stat,
+                      void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Scaled Adam step without a workspace.  (No counterpart in the paper: this entry point exists
  * for the integration, not for the method.)
  *

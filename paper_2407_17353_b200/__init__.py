@@ -43,6 +43,11 @@ class scalify_array(ctypes.Structure):
                 ("shape", ctypes.c_int64 * 3), ("stride", ctypes.c_int64 * 3), ("scale", ctypes.c_void_p)]
 
 
+class scalify_mx_array(ctypes.Structure):
+    _fields_ = [("data", ctypes.c_void_p), ("dtype", ctypes.c_int32), ("rows", ctypes.c_int64), ("K", ctypes.c_int64),
+                ("sf", ctypes.c_void_p), ("scale", ctypes.c_void_p)]
+
+
 _lib = None
 
 
@@ -75,6 +80,10 @@ def lib() -> ctypes.CDLL:
         L.scalify_scaled_gelu.argtypes = [P, i32, P, vp]
         L.scalify_scaled_gelu_bwd.argtypes = [P, P, i32, P, vp]
         L.scalify_scaled_adam_step.argtypes = [i32, P, P, P, P, f32, f32, f32, f32, i64, vp, sz, vp]
+        L.scalify_mx_sf_bytes.restype = sz
+        L.scalify_mx_sf_bytes.argtypes = [i64, i64]
+        L.scalify_mx_quantize.argtypes = [P, vp, vp, vp]
+        L.scalify_mx_matmul.argtypes = [vp, vp, P, i32, vp, sz, vp]
         L.scalify_scaled_adam_step_cast.argtypes = [i32, P, P, P, P, P, f32, f32, f32, f32, i64, vp, sz, vp]
         L.scalify_debug_expire_wait.argtypes = [vp, sz, c.c_uint32, vp, vp]
         L.scalify_scalar_mul_pow2.argtypes = [P, f32, vp]
@@ -90,7 +99,8 @@ def lib() -> ctypes.CDLL:
                      "scalify_scaled_layernorm_bwd", "scalify_scaled_gelu", "scalify_scaled_gelu_bwd",
                      "scalify_scaled_adam_step", "scalify_scaled_adam_step_cast", "scalify_scaled_adam_step_static", "scalify_scaled_embedding",
                      "scalify_scaled_embedding_bwd", "scalify_scaled_softmax", "scalify_scaled_softmax_bwd",
-                     "scalify_scaled_cross_entropy", "scalify_scalar_mul_pow2", "scalify_debug_expire_wait"):
+                     "scalify_scaled_cross_entropy", "scalify_scalar_mul_pow2", "scalify_debug_expire_wait",
+                     "scalify_mx_quantize", "scalify_mx_matmul"):
             getattr(L, name).restype = i32
         _lib = L
     return _lib
@@ -354,3 +364,54 @@ def scalify_scalar_mul_pow2(X: ScaledTensor, c: float, *, stream=None) -> None:
 def scalify_debug_expire_wait(ws: Workspace, limit_us: int, waited_us: Optional[torch.Tensor] = None, *, stream=None) -> None:
     _check(lib().scalify_debug_expire_wait(ws.ptr, ws.nbytes, int(limit_us), _ptr(waited_us), _stream(stream)),
            "scalify_debug_expire_wait")
+
+
+class MxTensor:
+    """Block-scaled array: FP8 data [rows, K], E8M0 exponents per 32 elements of K in the tile order the
+    tensor cores consume (see ``include/scalify.h``), and the tensor-wide fp32 power-of-two scale."""
+
+    def __init__(self, rows: int, K: int, dtype: torch.dtype = torch.float8_e4m3fn, device="cuda"):
+        assert dtype in (torch.float8_e4m3fn, torch.float8_e5m2) and K % 128 == 0 and rows >= 1
+        self.rows, self.K = int(rows), int(K)
+        self.data = torch.empty((rows, K), dtype=dtype, device=device)
+        self.sf = torch.empty(scalify_mx_sf_bytes(rows, K), dtype=torch.uint8, device=device)
+        self.scale = torch.ones(1, dtype=torch.float32, device=device)
+        self._d = scalify_mx_array(self.data.data_ptr(), _DTYPE_CODE[dtype], self.rows, self.K, self.sf.data_ptr(),
+                                   self.scale.data_ptr())
+
+    def scale_value(self) -> float:
+        return float(self.scale.item())
+
+    def exponents(self) -> torch.Tensor:
+        """The E8M0 codes as a plain [rows, K/32] uint8 tensor (un-tiled copy, for inspection)."""
+        kb = self.K // 32
+        pr = (self.rows + 255) // 256 * 256
+        t = self.sf.view(pr // 128, self.K // 128, 32, 4, 4)          # [row tile, k tile, row % 32, row / 32, blk]
+        t = t.permute(0, 3, 2, 1, 4).reshape(pr, kb)                   # row = tile*128 + (row/32)*32 + row%32
+        return t[: self.rows].contiguous()
+
+    def set_exponents(self, codes: torch.Tensor, pad: int = 127) -> None:
+        """Fill the tiled exponent buffer from plain [rows, K/32] codes (padding rows get `pad`)."""
+        kb = self.K // 32
+        pr = (self.rows + 255) // 256 * 256
+        full = torch.full((pr, kb), pad, dtype=torch.uint8, device=self.sf.device)
+        full[: self.rows] = codes.to(self.sf.device)
+        t = full.view(pr // 128, 4, 32, self.K // 128, 4).permute(0, 3, 2, 1, 4).contiguous()
+        self.sf.copy_(t.view(-1))
+
+
+def scalify_mx_sf_bytes(rows: int, K: int) -> int:
+    return int(lib().scalify_mx_sf_bytes(int(rows), int(K)))
+
+
+def scalify_mx_quantize(X: ScaledTensor, Y: MxTensor, *, status: Optional[torch.Tensor] = None, stream=None) -> None:
+    x = _desc(X)
+    _check(lib().scalify_mx_quantize(_ref(x), ctypes.addressof(Y._d), _ptr(status), _stream(stream)),
+           "scalify_mx_quantize")
+
+
+def scalify_mx_matmul(A: MxTensor, B: MxTensor, Y: ScaledTensor, ws: Workspace, *, stat: int = STAT_NONE,
+                      stream=None) -> None:
+    y = _desc(Y)
+    _check(lib().scalify_mx_matmul(ctypes.addressof(A._d), ctypes.addressof(B._d), _ref(y), int(stat), ws.ptr,
+                                   ws.nbytes, _stream(stream)), "scalify_mx_matmul")

@@ -42,16 +42,24 @@ constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
 //           CTA stages its own 128 rows of A and its own 128-column half of B, the leader CTA
 //           issues the MMAs, which read both CTAs' shared memory and write both CTAs' TMEM.
 //           Per SM this halves the shared-memory traffic of B, the limiter of the 1-CTA form.
-template <int NCTA> struct GemmCfg {
+// MX: block-scaled operands (one E8M0 exponent per 32 elements of K, Section 2's block-scale
+//     generalisation): each ring slot also holds the exponent tiles of its K block (512 B for the
+//     128 rows of A, 2 x 512 B for the 256 rows of B), which the MMA warp copies into TMEM before
+//     the block's four MMAs.  TMEM then holds ONE 256-column accumulator plus 12 exponent columns.
+template <int NCTA, bool MX = false> struct GemmCfg {
   static constexpr int kTileM = kBM * NCTA;
   static constexpr int kBRows = kBN / NCTA;          // B rows (columns of the output) staged per CTA
   static constexpr int kABytes = kBM * kBK;          // 16 KB
   static constexpr int kBBytes = kBRows * kBK;       // 32 KB / 16 KB
-  static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kStages = NCTA == 1 ? 4 : 6;
+  static constexpr int kSfBytes = MX ? 2048 : 0;     // exponent tiles of one K block (1536 B used)
+  static constexpr int kStageBytes = kABytes + kBBytes + kSfBytes;
+  static constexpr int kStages = MX ? 3 : (NCTA == 1 ? 4 : 6);
+  static constexpr int kAcc = MX ? 1 : kAccStages;   // accumulators in TMEM
   static constexpr int kEpiBytes = kEpiWarps * 32 * 128;  // per-warp staging tile of the epilogue: 32 rows x up to 128 B
   static constexpr size_t kSmem = size_t(kStages) * kStageBytes + kEpiBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
+constexpr uint32_t kSfaTmemCol = 256;  // MX: TMEM columns of the exponents of A (4) and of B (8)
+constexpr uint32_t kSfbTmemCol = 260;
 
 struct GemmParams {
   int M, N, K, batch;
@@ -72,6 +80,10 @@ struct GemmParams {
   uint32_t generation;   // tag of this call; a later call always overrides an earlier one, so no zeroing is needed
   double* l2_partials;   // L2: [tiles][4]
   uint32_t* status;
+  // MX only: block exponents in tiles of 128 rows x 4 K-blocks (512 B each), tile (r, k) at
+  // ((r * K/128) + k) * 512, byte (row % 32) * 16 + (row / 32 % 4) * 4 + (block % 4)
+  const uint8_t* sfa;
+  const uint8_t* sfb;
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -143,6 +155,26 @@ __device__ __forceinline__ void umma_f8(uint32_t d_tmem, uint64_t adesc, uint64_
       "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
+}
+// Block-scaled form: the exponents of A and B are read from TMEM (one byte per row and MMA, selected by
+// the scale-factor ids in the instruction descriptor).
+__device__ __forceinline__ void umma_mxf8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate, uint32_t sfa_tmem, uint32_t sfb_tmem) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::mxf8f6f4.block_scale [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
+      : "memory");
+}
+// 32 rows x 16 bytes of shared memory -> the same 4 TMEM columns in all four lane quarters
+__device__ __forceinline__ void tmem_cp_32x128b_warpx4(uint32_t taddr, uint64_t sdesc) {
+  asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+// plain (untiled) bulk copy global -> shared, completion counted on an mbarrier; 16-byte aligned, size % 16 == 0
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar) : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -233,6 +265,17 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_
   return d;
 }
 
+// Descriptor of an un-swizzled K-major block of 8-row x 16-byte core matrices `sbo_bytes` apart
+// (the source of the exponent copy: 32 rows x 16 B, four core matrices 128 B apart).
+__device__ __forceinline__ uint64_t make_smem_desc_noswizzle(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);
+  d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= 1ull << 46;
+  return d;
+}
+
 __device__ __forceinline__ void tile_coords(const GemmParams& p, int tile, int& b, int& mt, int& nt) {
   const int per_batch = p.tiles_m * p.tiles_n;
   b = tile / per_batch;
@@ -246,18 +289,20 @@ __device__ __forceinline__ void tile_coords(const GemmParams& p, int tile, int& 
   nt = r / gm;
 }
 
-template <int OUT, int NCTA>
-__global__ void __launch_bounds__(kGemmThreads, 1)
-scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                     const __grid_constant__ CUtensorMap map_y, const GemmParams p) {
-  using C = GemmCfg<NCTA>;
+template <int OUT, int NCTA, bool MX>
+__device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_y,
+                                          const GemmParams& p) {
+  static_assert(!MX || NCTA == 1, "the block-scaled form is built for one CTA per tile");
+  using C = GemmCfg<NCTA, MX>;
   constexpr int kStages = C::kStages;
+  constexpr int kAcc = C::kAcc;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (base - raw);
   const uint32_t smem_a = base;
   const uint32_t smem_b = base + kStages * C::kABytes;
+  const uint32_t smem_sf = smem_b + kStages * C::kBBytes;  // MX: [stage][A exponents 512 B | B exponents 2 x 512 B | pad]
   uint8_t* epi_mem = smem + kStages * C::kStageBytes;  // 16 KB, 1024-byte aligned
   uint8_t* bar_mem = epi_mem + C::kEpiBytes;
   const uint32_t bars = base + kStages * C::kStageBytes + C::kEpiBytes;
@@ -325,7 +370,13 @@ scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
           const int bb = p.b_batched ? b : 0;
           if constexpr (NCTA == 1) {
             const uint32_t fb = full_bar + 8 * stage;
-            mbar_expect_tx(fb, C::kStageBytes);
+            mbar_expect_tx(fb, C::kABytes + C::kBBytes + (MX ? 1536 : 0));
+            if constexpr (MX) {
+              const uint32_t ssf = smem_sf + stage * C::kSfBytes;
+              bulk_load(ssf, p.sfa + (static_cast<size_t>(mt) * num_kb + kb) * 512, 512, fb);
+              bulk_load(ssf + 512, p.sfb + (static_cast<size_t>(2 * nt) * num_kb + kb) * 512, 512, fb);
+              bulk_load(ssf + 1024, p.sfb + (static_cast<size_t>(2 * nt + 1) * num_kb + kb) * 512, 512, fb);
+            }
             if (p.a_mn_major) tma_load_3d(sa, &map_a, fb, m0, k0, b);
             else tma_load_3d(sa, &map_a, fb, k0, m0, b);
             if (p.b_mn_major) {
@@ -375,12 +426,26 @@ scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
           if (!mbar_wait(full_bar + 8 * stage, phase, abort_flag)) { timed_out = true; break; }
           tc_fence_after();
           const uint32_t sa = smem_a + stage * C::kABytes, sb = smem_b + stage * C::kBBytes;
+          if constexpr (MX) {
+            // this K block's exponents: shared memory -> TMEM (executes in order with the MMAs of this thread)
+            const uint32_t ssf = smem_sf + stage * C::kSfBytes;
+            tmem_cp_32x128b_warpx4(tmem_base + kSfaTmemCol, make_smem_desc_noswizzle(ssf, 512u, 128u));
+            tmem_cp_32x128b_warpx4(tmem_base + kSfbTmemCol, make_smem_desc_noswizzle(ssf + 512, 512u, 128u));
+            tmem_cp_32x128b_warpx4(tmem_base + kSfbTmemCol + 4, make_smem_desc_noswizzle(ssf + 1024, 512u, 128u));
+          }
 #pragma unroll
           for (int k = 0; k < kBK / kUmmaK; ++k) {
             const uint64_t ad = make_smem_desc(sa + k * a_step, a_lbo, a_sbo);
             const uint64_t bd = make_smem_desc(sb + k * b_step, b_lbo, b_sbo);
-            if constexpr (NCTA == 1) umma_f8(d_tmem, ad, bd, p.idesc, (kb | k) != 0 ? 1u : 0u);
-            else umma_f8_pair(d_tmem, ad, bd, p.idesc, (kb | k) != 0 ? 1u : 0u);
+            if constexpr (MX) {
+              // scale-factor ids: byte k of the 4-byte exponent word of each row (bits 29-30 for A, 4-5 for B)
+              umma_mxf8(d_tmem, ad, bd, p.idesc | (uint32_t(k) << 29) | (uint32_t(k) << 4), (kb | k) != 0 ? 1u : 0u,
+                        tmem_base + kSfaTmemCol, tmem_base + kSfbTmemCol);
+            } else if constexpr (NCTA == 1) {
+              umma_f8(d_tmem, ad, bd, p.idesc, (kb | k) != 0 ? 1u : 0u);
+            } else {
+              umma_f8_pair(d_tmem, ad, bd, p.idesc, (kb | k) != 0 ? 1u : 0u);
+            }
           }
           // slot free (in both CTAs) once these MMAs have read it
           if constexpr (NCTA == 1) umma_commit(empty_bar + 8 * stage);
@@ -391,7 +456,7 @@ scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         // accumulator complete (in both CTAs)
         if constexpr (NCTA == 1) umma_commit(acc_full_bar + 8 * acc);
         else umma_commit_pair(acc_full_bar + 8 * acc);
-        if (++acc == kAccStages) { acc = 0; acc_phase ^= 1u; }
+        if (++acc == kAcc) { acc = 0; acc_phase ^= 1u; }
       }
       if (timed_out || *abort_flag) {
         // all MMAs issued so far must retire before TMEM is freed
@@ -486,7 +551,7 @@ scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         const double s = warp_sum_f64(static_cast<double>(ssq)) * (double(r_prev) * double(r_prev));
         if (lane == 0) p.l2_partials[((static_cast<long long>(tile) * NCTA + rank) * 4 + q) * 2 + half] = s;
       }
-      if (++acc == kAccStages) { acc = 0; acc_phase ^= 1u; }
+      if (++acc == kAcc) { acc = 0; acc_phase ^= 1u; }
     }
     if (lane == 0) bulk_wait_all();  // every store of this warp has completed
     if (p.stat == SCALIFY_STAT_AMAX) {
@@ -510,6 +575,21 @@ scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);
   }
+}
+
+template <int OUT, int NCTA>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                     const __grid_constant__ CUtensorMap map_y, const GemmParams p) {
+  gemm_body<OUT, NCTA, false>(map_a, map_b, map_y, p);
+}
+
+// Block-scaled operands (E8M0 exponent per 32 elements of K), K-major A [M,K] and B [N,K].
+template <int OUT>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+mx_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                 const __grid_constant__ CUtensorMap map_y, const GemmParams p) {
+  gemm_body<OUT, 1, true>(map_a, map_b, map_y, p);
 }
 
 // Diagnostic: one thread waits, with the GEMM's bounded-wait routine and a short limit, on an
@@ -665,6 +745,12 @@ static int launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, co
   return SCALIFY_OK;
 }
 
+// tag of a call that gathers AMAX with the generation-tagged atomicMax (shared by all GEMM forms)
+static uint32_t next_stat_generation() {
+  static std::atomic<uint32_t> next_generation{1};
+  return next_generation.fetch_add(1);
+}
+
 int launch_scaled_matmul(const MatmulArgs& a, void* ws, cudaStream_t st) {
   WsView v = ws_view(ws);
   // two-CTA tiles (256 rows) whenever there is more than one 128-row tile of output
@@ -708,15 +794,16 @@ int launch_scaled_matmul(const MatmulArgs& a, void* ws, cudaStream_t st) {
   p.stat_word = reinterpret_cast<unsigned long long*>(v.stat);
   p.l2_partials = static_cast<double*>(v.area);
   p.status = v.status;
+  p.sfa = nullptr;
+  p.sfb = nullptr;
   const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n * p.batch;
   if (tiles > (1ll << 30)) return SCALIFY_ERR_SHAPE;
   p.generation = 0;
   if (a.stat == SCALIFY_STAT_AMAX) {
-    static std::atomic<uint32_t> next_generation{1};
-    p.generation = next_generation.fetch_add(1);
+    p.generation = next_stat_generation();
     if (p.generation == 0) {  // the 32-bit tag wrapped: start over from a zeroed word
       SCALIFY_CUDA_TRY(cudaMemsetAsync(v.stat, 0, 2 * sizeof(float), st));
-      p.generation = next_generation.fetch_add(1);
+      p.generation = next_stat_generation();
     }
   }
   SCALIFY_DISPATCH_DTYPE(a.y_dt, OUT, {
@@ -727,6 +814,70 @@ int launch_scaled_matmul(const MatmulArgs& a, void* ws, cudaStream_t st) {
   if (a.stat == SCALIFY_STAT_L2) {
     gemm_l2_finalize_kernel<<<1, 256, 0, st>>>(p.l2_partials, static_cast<int>(tiles * ncta * 8),
                                                double(a.M) * double(a.N) * double(a.batch), v.stat);
+    SCALIFY_CUDA_TRY(cudaGetLastError());
+  }
+  return SCALIFY_OK;
+}
+
+int launch_mx_matmul(const MxMatmulArgs& a, void* ws, cudaStream_t st) {
+  WsView v = ws_view(ws);
+  CUtensorMap map_a, map_b, map_y;
+  int rc = make_map(&map_a, a.A, a.K, a.M, 1, a.K, 0, kBM);
+  if (rc) return rc;
+  rc = make_map(&map_b, a.B, a.K, a.N, 1, a.K, 0, kBN);
+  if (rc) return rc;
+  rc = make_map_y(&map_y, a.Y, elem_size(a.y_dt), a.N, a.M, 1, a.ldy, 0);
+  if (rc) return rc;
+  GemmParams p;
+  p.M = a.M; p.N = a.N; p.K = a.K; p.batch = 1;
+  p.tiles_m = (a.M + kBM - 1) / kBM;
+  p.tiles_n = (a.N + kBN - 1) / kBN;
+  p.a_mn_major = 0;
+  p.b_mn_major = 0;
+  p.b_batched = 0;
+  // block-scaled instruction descriptor (kind::mxf8f6f4): scale-factor ids in bits 4-5 (B) and 29-30 (A)
+  // are filled in per MMA, A/B formats, K-major operands, N >> 3, E8M0 exponents (bit 23), M >> 4
+  p.idesc = (uint32_t(a.a_dt == SCALIFY_E5M2) << 7) | (uint32_t(a.b_dt == SCALIFY_E5M2) << 10) |
+            (uint32_t(kBN >> 3) << 17) | (1u << 23) | (uint32_t(kBM >> 4) << 24);
+  p.kf = kfactor(a.K);
+  p.alpha = 1.0f / p.kf;
+  p.Y = a.Y; p.ldy = a.ldy; p.y_batch_stride = 0;
+  p.a_scale = a.a_scale; p.b_scale = a.b_scale; p.y_scale = a.y_scale;
+  p.stat = a.stat;
+  p.stat_in = nullptr;
+  p.stat_word = reinterpret_cast<unsigned long long*>(v.stat);
+  p.l2_partials = static_cast<double*>(v.area);
+  p.status = v.status;
+  p.sfa = a.sfa;
+  p.sfb = a.sfb;
+  const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n;
+  if (tiles > (1ll << 30)) return SCALIFY_ERR_SHAPE;
+  p.generation = 0;
+  if (a.stat == SCALIFY_STAT_AMAX) {
+    p.generation = next_stat_generation();
+    if (p.generation == 0) {
+      SCALIFY_CUDA_TRY(cudaMemsetAsync(v.stat, 0, 2 * sizeof(float), st));
+      p.generation = next_stat_generation();
+    }
+  }
+  SCALIFY_DISPATCH_WIDE(a.y_dt, OUT, {
+    using C = GemmCfg<1, true>;
+    auto kernel = mx_matmul_kernel<OUT>;
+    static bool attr_done = false;
+    if (!attr_done) {
+      SCALIFY_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(C::kSmem)));
+      attr_done = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(unsigned(tiles < sm_count() ? tiles : sm_count()));
+    cfg.blockDim = dim3(kGemmThreads);
+    cfg.dynamicSmemBytes = C::kSmem;
+    cfg.stream = st;
+    SCALIFY_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, map_a, map_b, map_y, p));
+  });
+  if (a.stat == SCALIFY_STAT_L2) {
+    gemm_l2_finalize_kernel<<<1, 256, 0, st>>>(p.l2_partials, static_cast<int>(tiles * 8),
+                                               double(a.M) * double(a.N), v.stat);
     SCALIFY_CUDA_TRY(cudaGetLastError());
   }
   return SCALIFY_OK;

@@ -348,6 +348,57 @@ int scalify_scaled_layernorm_bwd(const scalify_array* G, const scalify_array* X,
   return rc;
 }
 
+static int check_mx(const scalify_mx_array* a) {
+  if (!a || !a->data || !a->sf) return SCALIFY_ERR_NULL;
+  if (a->dtype != SCALIFY_E4M3 && a->dtype != SCALIFY_E5M2) return SCALIFY_ERR_DTYPE;
+  if (a->rows < 1 || a->K < 128 || a->K % 128 != 0 || a->rows > 0x7FFFFFFF || a->K > 0x7FFFFFFF)
+    return SCALIFY_ERR_SHAPE;
+  if (reinterpret_cast<uintptr_t>(a->data) % 16 != 0 || reinterpret_cast<uintptr_t>(a->sf) % 16 != 0)
+    return SCALIFY_ERR_ALIGNMENT;
+  return SCALIFY_OK;
+}
+
+size_t scalify_mx_sf_bytes(int64_t rows, int64_t K) {
+  if (rows < 1 || K < 128 || K % 128 != 0) return 0;
+  return mx_sf_bytes(rows, K);
+}
+
+int scalify_mx_quantize(const scalify_array* X, scalify_mx_array* Y, uint32_t* status, void* stream) {
+  int rc = check_array(X);
+  if (rc) return rc;
+  rc = check_mx(Y);
+  if (rc) return rc;
+  if (!is_wide(X->dtype)) return SCALIFY_ERR_DTYPE;
+  if (X->ndim != 2 || X->shape[0] != Y->rows || X->shape[1] != Y->K) return SCALIFY_ERR_SHAPE;
+  if (Y->scale && Y->scale == X->scale) return SCALIFY_ERR_ALIAS;
+  return launch_mx_quantize(X->data, X->dtype, Y->rows, Y->K, X->stride[0], Y->data, Y->dtype, Y->sf, X->scale,
+                            Y->scale, status, static_cast<cudaStream_t>(stream));
+}
+
+int scalify_mx_matmul(const scalify_mx_array* A, const scalify_mx_array* B, scalify_array* Y, int stat,
+                      void* workspace, size_t workspace_bytes, void* stream) {
+  int rc = check_mx(A);
+  if (rc) return rc;
+  rc = check_mx(B);
+  if (rc) return rc;
+  rc = check_array(Y);
+  if (rc) return rc;
+  if (!valid_stat(stat)) return SCALIFY_ERR_VALUE;
+  if (!is_wide(Y->dtype)) return SCALIFY_ERR_DTYPE;
+  if (A->K != B->K || Y->ndim != 2 || Y->shape[0] != A->rows || Y->shape[1] != B->rows) return SCALIFY_ERR_SHAPE;
+  if (Y->scale && (Y->scale == A->scale || Y->scale == B->scale)) return SCALIFY_ERR_ALIAS;
+  rc = check_ws(workspace, workspace_bytes, scalify_workspace_bytes(SCALIFY_OP_MATMUL, A->rows, B->rows));
+  if (rc) return rc;
+  MxMatmulArgs a;
+  a.A = A->data; a.a_dt = A->dtype; a.sfa = A->sf;
+  a.B = B->data; a.b_dt = B->dtype; a.sfb = B->sf;
+  a.Y = Y->data; a.y_dt = Y->dtype; a.ldy = Y->stride[0];
+  a.M = static_cast<int>(A->rows); a.N = static_cast<int>(B->rows); a.K = static_cast<int>(A->K);
+  a.a_scale = A->scale; a.b_scale = B->scale; a.y_scale = Y->scale;
+  a.stat = stat;
+  return launch_mx_matmul(a, workspace, static_cast<cudaStream_t>(stream));
+}
+
 static int adam_step_impl(int n_tensors, const scalify_array* grads, scalify_array* m, scalify_array* v,
                           scalify_array* w, const scalify_array* w_cast, float lr, float beta1, float beta2,
                           float eps, int64_t step, void* workspace, size_t workspace_bytes, void* stream) {

@@ -67,5 +67,18 @@ struct MatmulArgs {
 size_t matmul_ws_bytes(int64_t rows, int64_t cols);
 int launch_expire_wait(void* ws, unsigned long long limit_ns, uint32_t* waited_us, cudaStream_t st);
 int launch_scaled_matmul(const MatmulArgs& a, void* ws, cudaStream_t st);
+// Block-scaled matmul: A [M,K], B [N,K] FP8 row-major (dense), exponents in 128-row x 4-block tiles.
+struct MxMatmulArgs {
+  const void* A; int a_dt; const uint8_t* sfa;
+  const void* B; int b_dt; const uint8_t* sfb;
+  void* Y; int y_dt; int64_t ldy;
+  int M, N, K;
+  const float* a_scale; const float* b_scale; float* y_scale;
+  int stat;
+};
+int launch_mx_matmul(const MxMatmulArgs& a, void* ws, cudaStream_t st);
+size_t mx_sf_bytes(int64_t rows, int64_t K);
+int launch_mx_quantize(const void* X, int x_dt, int64_t rows, int64_t K, int64_t ldx, void* data, int elem_dt,
+                       uint8_t* sf, const float* x_scale, float* y_scale, uint32_t* status, cudaStream_t st);
 
 }  // namespace scalify

@@ -1,0 +1,152 @@
+"""GPU parity of the block-scaled path (E8M0 exponent per 32 elements of K) against the fp64 oracle.
+
+Bars: quantised FP8 bytes, exponent bytes and scale words bit-exact; the matmul's fp32 output within
+1e-5 * sum|a*b| per element; BF16 / F16 outputs within 1 ulp (or half an ulp plus the accumulation bar
+where the dot product cancels); the fused AMAX equal to the maximum of the stored output."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as orc
+import paper_2407_17353_b200 as sc
+import scalify_inputs as si
+from helpers import to_dev, to_bits, within
+
+pytestmark = pytest.mark.gpu
+
+
+def wide_range_input(seed, rows, K, dt, spread=20):
+    x = si.normal(seed, 1, (rows, K), 1.0).astype(np.float64)
+    x *= np.exp2(np.random.default_rng(seed).integers(-spread, spread, size=(rows, K // 32))).repeat(32, axis=1)
+    return si.to_bits(x.astype(np.float32), dt)
+
+
+@pytest.mark.parametrize("rows,K", [(1, 128), (300, 256), (513, 1024), (128, 4096)])
+@pytest.mark.parametrize("x_dt", [orc.BF16, orc.F16, orc.F32])
+@pytest.mark.parametrize("elem", [orc.E4M3, orc.E5M2])
+def test_mx_quantize_bit_exact(rows, K, x_dt, elem):
+    xb = wide_range_input(100 + rows, rows, K, x_dt, spread=6 if x_dt == orc.F16 else 20)
+    X = sc.ScaledTensor.make(to_dev(xb, x_dt), 2.0 ** -4)
+    Y = sc.MxTensor(rows, K, sc.TORCH_DTYPE[elem])
+    Y.sf.fill_(0xFF)  # whatever was there, padding rows included, must be overwritten
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    sc.scalify_mx_quantize(X, Y, status=status)
+    assert int(status.item()) == 0
+    data, codes = orc.mx_quantize(xb, x_dt, elem)
+    assert np.array_equal(Y.exponents().cpu().numpy(), codes)
+    assert np.array_equal(to_bits(Y.data, elem), data)
+    assert Y.scale_value() == 2.0 ** -4
+    # every exponent byte of the padding rows is the neutral code
+    pr = (rows + 255) // 256 * 256
+    full = Y.sf.view(pr // 128, K // 128, 32, 4, 4).permute(0, 3, 2, 1, 4).reshape(pr, K // 32)
+    assert bool((full[rows:] == 127).all())
+
+
+def test_mx_quantize_degenerate_blocks_and_strided_input():
+    rows, K = 5, 256
+    x = np.zeros((rows, K + 64), dtype=np.float32)
+    x[:, :K] = si.normal(3, 1, (rows, K), 1.0)
+    x[0, :32] = 0.0                      # all-zero block
+    x[1, 40] = np.inf                    # a block that cannot define a scale
+    x[2, 70] = np.nan
+    x[3, 96:128] = 2.0 ** -140           # fp32 subnormals: exponent clamps at the bottom of E8M0
+    x[4, 128] = 500.0                    # saturates E4M3 after scaling
+    buf = torch.from_numpy(x).cuda()
+    X = sc.ScaledTensor.make(buf[:, :K], 1.0)
+    Y = sc.MxTensor(rows, K)
+    sc.scalify_mx_quantize(X, Y)
+    xb = np.ascontiguousarray(x[:, :K]).view(np.uint32)
+    data, codes = orc.mx_quantize(xb, orc.F32, orc.E4M3)
+    assert np.array_equal(Y.exponents().cpu().numpy(), codes)
+    got = to_bits(Y.data, orc.E4M3)
+    nan = (data & 0x7F) == 0x7F
+    assert np.array_equal(got[~nan], data[~nan]) and np.all((got[nan] & 0x7F) == 0x7F)
+    assert codes[0, 0] == 127 and codes[1, 1] == 127 and codes[2, 2] == 127 and codes[3, 3] == 0
+
+
+def run_mx_matmul(a, a_dt, ea, a_s, b, b_dt, eb, b_s, y_dt, stat=sc.STAT_NONE):
+    M, K = a.shape
+    N = b.shape[0]
+    A = sc.MxTensor(M, K, sc.TORCH_DTYPE[a_dt])
+    B = sc.MxTensor(N, K, sc.TORCH_DTYPE[b_dt])
+    A.data.copy_(to_dev(a, a_dt)); B.data.copy_(to_dev(b, b_dt))
+    A.set_exponents(torch.from_numpy(ea)); B.set_exponents(torch.from_numpy(eb))
+    A.scale.fill_(a_s); B.scale.fill_(b_s)
+    Y = sc.ScaledTensor.empty((M, N), sc.TORCH_DTYPE[y_dt])
+    ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_MATMUL, M, N))
+    sc.scalify_mx_matmul(A, B, Y, ws, stat=stat)
+    assert ws.check_status() == 0
+    return to_bits(Y.data, y_dt), Y.scale_value(), float(ws.statistic().item())
+
+
+@pytest.mark.parametrize("M,N,K", [(128, 256, 128), (64, 40, 256), (200, 304, 384), (257, 520, 1024)])
+@pytest.mark.parametrize("a_dt,b_dt", [(orc.E4M3, orc.E4M3), (orc.E5M2, orc.E4M3)])
+def test_mx_matmul_against_oracle(M, N, K, a_dt, b_dt):
+    a = si.to_bits(si.normal(21, M + K, (M, K), 1.0), a_dt)
+    b = si.to_bits(si.normal(22, N + K, (N, K), 1.0), b_dt)
+    rng = np.random.default_rng(M * 7 + N)
+    ea = rng.integers(117, 138, size=(M, K // 32)).astype(np.uint8)   # a different exponent for every block
+    eb = rng.integers(117, 138, size=(N, K // 32)).astype(np.uint8)
+    Yo, ys, acc, sab = orc.mx_matmul(a, a_dt, ea, 0.25, b, b_dt, eb, 8.0, orc.BF16, want_acc=True)
+    g32, s32, _ = run_mx_matmul(a, a_dt, ea, 0.25, b, b_dt, eb, 8.0, orc.F32)
+    assert s32 == ys
+    err = np.abs(orc.decode(g32, orc.F32).reshape(M, N) - acc)
+    assert np.all(err <= 1e-5 * sab + 1e-30), float((err / (sab + 1e-30)).max())
+    gb, sb, stat = run_mx_matmul(a, a_dt, ea, 0.25, b, b_dt, eb, 8.0, orc.BF16, stat=sc.STAT_AMAX)
+    assert sb == ys
+    ok = within(gb, Yo, orc.BF16, acc, sab, 1e-5)
+    assert ok.all(), int((~ok).sum())
+    assert stat == float(np.abs(orc.decode(gb, orc.BF16)).max())
+
+
+def test_mx_matmul_distinguishes_every_exponent_byte():
+    """One block of A and one block of B get a large exponent each, at every position in turn: a kernel
+    that picked the wrong exponent byte (wrong row group, wrong K block, wrong half of a 256-column tile)
+    would miss the product."""
+    M, N, K = 128, 256, 256
+    a = si.to_bits(np.ones((M, K), dtype=np.float32), orc.E4M3)
+    b = si.to_bits(np.ones((N, K), dtype=np.float32), orc.E4M3)
+    for (i, kb, j) in [(0, 0, 0), (31, 1, 33), (32, 2, 127), (64, 3, 128), (97, 4, 200), (127, 7, 255)]:
+        ea = np.full((M, K // 32), 127, dtype=np.uint8)
+        eb = np.full((N, K // 32), 127, dtype=np.uint8)
+        ea[i, kb] = 130
+        eb[j, kb] = 125
+        Yo, _, acc, _ = orc.mx_matmul(a, orc.E4M3, ea, 1.0, b, orc.E4M3, eb, 1.0, orc.F32, want_acc=True)
+        g, _, _ = run_mx_matmul(a, orc.E4M3, ea, 1.0, b, orc.E4M3, eb, 1.0, orc.F32)
+        assert np.array_equal(orc.decode(g, orc.F32).reshape(M, N), acc), (i, kb, j)
+
+
+def test_quantize_then_matmul_matches_the_oracle_pipeline():
+    M, N, K = 384, 512, 512
+    xa = wide_range_input(31, M, K, orc.BF16, spread=8)
+    xb = wide_range_input(32, N, K, orc.BF16, spread=8)
+    A, B = sc.MxTensor(M, K), sc.MxTensor(N, K)
+    sc.scalify_mx_quantize(sc.ScaledTensor.make(to_dev(xa, orc.BF16), 0.5), A)
+    sc.scalify_mx_quantize(sc.ScaledTensor.make(to_dev(xb, orc.BF16), 2.0), B)
+    Y = sc.ScaledTensor.empty((M, N), torch.float32)
+    ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_MATMUL, M, N))
+    sc.scalify_mx_matmul(A, B, Y, ws)
+    da, ea = orc.mx_quantize(xa, orc.BF16, orc.E4M3)
+    db, eb = orc.mx_quantize(xb, orc.BF16, orc.E4M3)
+    _, ys, acc, sab = orc.mx_matmul(da, orc.E4M3, ea, 0.5, db, orc.E4M3, eb, 2.0, orc.F32, want_acc=True)
+    assert Y.scale_value() == ys
+    err = np.abs(orc.decode(to_bits(Y.data, orc.F32), orc.F32).reshape(M, N) - acc)
+    assert np.all(err <= 1e-5 * sab)
+    # and the block-scaled product is close to the product of the un-quantised operands
+    va, vb = orc.decode(xa, orc.BF16).reshape(M, K), orc.decode(xb, orc.BF16).reshape(N, K)
+    exact = va @ vb.T / orc.kf(K)
+    rel = np.linalg.norm(acc - exact) / np.linalg.norm(exact)
+    assert rel < 0.05
+
+
+def test_mx_argument_checks():
+    A = sc.MxTensor(64, 128)
+    B = sc.MxTensor(32, 256)
+    Y = sc.ScaledTensor.empty((64, 32), torch.bfloat16)
+    ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_MATMUL, 64, 32))
+    with pytest.raises(sc.ScalifyError):
+        sc.scalify_mx_matmul(A, B, Y, ws)      # K differs
+    assert sc.scalify_mx_sf_bytes(64, 100) == 0  # K must be a multiple of 128
+    X = sc.ScaledTensor.make(torch.zeros((64, 256), dtype=torch.bfloat16, device="cuda"), 1.0)
+    with pytest.raises(sc.ScalifyError):
+        sc.scalify_mx_quantize(X, A)           # shape differs
