@@ -456,6 +456,36 @@ def main():
     barrier()
     adam_cast_ms = c0.elapsed_time(c1) / c_iters if c_iters else float("nan")
 
+    # Block-scaled variant (E8M0 exponent per 32 elements of K): quantise both BF16 operands, then the
+    # block-scaled GEMM with fused AMAX, BF16 out
+    mx_q_ms = mx_mm_ms = float("nan")
+    if not args.no_next:
+        Xa = sc.ScaledTensor.make(rnd((N_GEMM, N_GEMM), torch.bfloat16, 21), 1.0)
+        Xb = sc.ScaledTensor.make(rnd((N_GEMM, N_GEMM), torch.bfloat16, 22), 1.0)
+        Am, Bm = sc.MxTensor(N_GEMM, N_GEMM, device=dev), sc.MxTensor(N_GEMM, N_GEMM, device=dev)
+
+        def mx_quant():
+            sc.scalify_mx_quantize(Xa, Am)
+            sc.scalify_mx_quantize(Xb, Bm)
+
+        def mx_mm():
+            sc.scalify_mx_matmul(Am, Bm, Y, ws_mm, stat=sc.STAT_AMAX)
+        x_iters = max(3, min(K, 20))
+        times = []
+        for fn in (mx_quant, mx_mm):
+            for _ in range(3):
+                fn()
+            barrier()
+            x0, x1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            x0.record()
+            for _ in range(x_iters):
+                fn()
+            x1.record()
+            barrier()
+            times.append(x0.elapsed_time(x1) / x_iters)
+        mx_q_ms, mx_mm_ms = times
+        del Xa, Xb, Am, Bm
+
     # ------------------------------------------------------------------ end to end through host buffers
     hY = torch.empty((N_GEMM, N_GEMM), dtype=torch.int8).pin_memory()
     hscale = torch.empty(1, dtype=torch.float32).pin_memory()
@@ -551,6 +581,11 @@ def main():
          "TFLOP/s": round(flops / (delayed_ms * 1e-3) / 1e12, 1)},
         row("f2 (next, timed outside the step, back to back) scaled Adam that also writes the E4M3 compute copy "
             "of the weight (14 B/param)", adam_cast_ms, 14 * ADAM_N),
+        row("f3 (next, own loop) block-scale quantisation of two 8192^2 BF16 operands to E4M3 + E8M0 per 32 "
+            "elements (3.03 B/elem)", mx_q_ms, 2 * (3 * N_GEMM * N_GEMM + N_GEMM * N_GEMM // 32)),
+        {"row": "f3 (next, own loop) block-scaled GEMM 8192^3 (tcgen05 kind::mxf8f6f4.block_scale, two-CTA tiles), "
+                "BF16 out + fused AMAX", "ms": round(float(mx_mm_ms), 4),
+         "TFLOP/s": round(flops / (mx_mm_ms * 1e-3) / 1e12, 1)},
     ]
     fp8_peak = 2.0 * peaks["bf16_sustained"]
     gemm_tflops = flops / (float(seg_ms[0]) * 1e-3) / 1e12

@@ -46,6 +46,8 @@ constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
 //     generalisation): each ring slot also holds the exponent tiles of its K block (512 B for the
 //     128 rows of A, 2 x 512 B for the 256 rows of B), which the MMA warp copies into TMEM before
 //     the block's four MMAs.  TMEM then holds ONE 256-column accumulator plus 12 exponent columns.
+//     In the two-CTA form every CTA stages the exponents of its own 128 rows of A and of ALL 256
+//     rows of B (each CTA multiplies its rows of A with the whole B tile).
 template <int NCTA, bool MX = false> struct GemmCfg {
   static constexpr int kTileM = kBM * NCTA;
   static constexpr int kBRows = kBN / NCTA;          // B rows (columns of the output) staged per CTA
@@ -53,7 +55,7 @@ template <int NCTA, bool MX = false> struct GemmCfg {
   static constexpr int kBBytes = kBRows * kBK;       // 32 KB / 16 KB
   static constexpr int kSfBytes = MX ? 2048 : 0;     // exponent tiles of one K block (1536 B used)
   static constexpr int kStageBytes = kABytes + kBBytes + kSfBytes;
-  static constexpr int kStages = MX ? 3 : (NCTA == 1 ? 4 : 6);
+  static constexpr int kStages = MX ? (NCTA == 1 ? 3 : 5) : (NCTA == 1 ? 4 : 6);
   static constexpr int kAcc = MX ? 1 : kAccStages;   // accumulators in TMEM
   static constexpr int kEpiBytes = kEpiWarps * 32 * 128;  // per-warp staging tile of the epilogue: 32 rows x up to 128 B
   static constexpr size_t kSmem = size_t(kStages) * kStageBytes + kEpiBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
@@ -166,6 +168,19 @@ __device__ __forceinline__ void umma_mxf8(uint32_t d_tmem, uint64_t adesc, uint6
       "tcgen05.mma.cta_group::1.kind::mxf8f6f4.block_scale [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
       : "memory");
+}
+__device__ __forceinline__ void umma_mxf8_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                               uint32_t accumulate, uint32_t sfa_tmem, uint32_t sfb_tmem) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::mxf8f6f4.block_scale [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
+      : "memory");
+}
+// the same copy executed in both CTAs of the pair, each from its own shared memory into its own TMEM
+__device__ __forceinline__ void tmem_cp_32x128b_warpx4_pair(uint32_t taddr, uint64_t sdesc) {
+  asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
 }
 // 32 rows x 16 bytes of shared memory -> the same 4 TMEM columns in all four lane quarters
 __device__ __forceinline__ void tmem_cp_32x128b_warpx4(uint32_t taddr, uint64_t sdesc) {
@@ -291,8 +306,7 @@ __device__ __forceinline__ void tile_coords(const GemmParams& p, int tile, int& 
 
 template <int OUT, int NCTA, bool MX>
 __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_y,
-                                          const GemmParams& p) {
-  static_assert(!MX || NCTA == 1, "the block-scaled form is built for one CTA per tile");
+                                          const CUtensorMap& map_sfa, const CUtensorMap& map_sfb, const GemmParams& p) {
   using C = GemmCfg<NCTA, MX>;
   constexpr int kStages = C::kStages;
   constexpr int kAcc = C::kAcc;
@@ -388,11 +402,18 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
           } else {
             // both CTAs' copies are counted on the LEADER's full barrier, which expects the bytes of the pair
             const uint32_t fb = map_to_cta(full_bar + 8 * stage, 0u);
-            if (rank == 0u) mbar_expect_tx(full_bar + 8 * stage, 2 * C::kStageBytes);
+            if (rank == 0u) mbar_expect_tx(full_bar + 8 * stage, 2 * (C::kABytes + C::kBBytes + (MX ? 1536 : 0)));
             if (p.a_mn_major) tma_load_3d_pair(sa, &map_a, fb, m0, k0, b);
             else tma_load_3d_pair(sa, &map_a, fb, k0, m0, b);
             if (p.b_mn_major) tma_load_3d_pair(sb, &map_b, fb, n0, k0, bb);
             else tma_load_3d_pair(sb, &map_b, fb, k0, n0, bb);
+            if constexpr (MX) {
+              // exponent tiles (rows of 512 bytes in the tile list): own half of A, both halves of B
+              const uint32_t ssf = smem_sf + stage * C::kSfBytes;
+              tma_load_3d_pair(ssf, &map_sfa, fb, 0, (2 * mt + static_cast<int>(rank)) * num_kb + kb, 0);
+              tma_load_3d_pair(ssf + 512, &map_sfb, fb, 0, (2 * nt) * num_kb + kb, 0);
+              tma_load_3d_pair(ssf + 1024, &map_sfb, fb, 0, (2 * nt + 1) * num_kb + kb, 0);
+            }
           }
           ++issued;
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
@@ -429,9 +450,15 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
           if constexpr (MX) {
             // this K block's exponents: shared memory -> TMEM (executes in order with the MMAs of this thread)
             const uint32_t ssf = smem_sf + stage * C::kSfBytes;
-            tmem_cp_32x128b_warpx4(tmem_base + kSfaTmemCol, make_smem_desc_noswizzle(ssf, 512u, 128u));
-            tmem_cp_32x128b_warpx4(tmem_base + kSfbTmemCol, make_smem_desc_noswizzle(ssf + 512, 512u, 128u));
-            tmem_cp_32x128b_warpx4(tmem_base + kSfbTmemCol + 4, make_smem_desc_noswizzle(ssf + 1024, 512u, 128u));
+            if constexpr (NCTA == 1) {
+              tmem_cp_32x128b_warpx4(tmem_base + kSfaTmemCol, make_smem_desc_noswizzle(ssf, 512u, 128u));
+              tmem_cp_32x128b_warpx4(tmem_base + kSfbTmemCol, make_smem_desc_noswizzle(ssf + 512, 512u, 128u));
+              tmem_cp_32x128b_warpx4(tmem_base + kSfbTmemCol + 4, make_smem_desc_noswizzle(ssf + 1024, 512u, 128u));
+            } else {
+              tmem_cp_32x128b_warpx4_pair(tmem_base + kSfaTmemCol, make_smem_desc_noswizzle(ssf, 512u, 128u));
+              tmem_cp_32x128b_warpx4_pair(tmem_base + kSfbTmemCol, make_smem_desc_noswizzle(ssf + 512, 512u, 128u));
+              tmem_cp_32x128b_warpx4_pair(tmem_base + kSfbTmemCol + 4, make_smem_desc_noswizzle(ssf + 1024, 512u, 128u));
+            }
           }
 #pragma unroll
           for (int k = 0; k < kBK / kUmmaK; ++k) {
@@ -439,8 +466,12 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
             const uint64_t bd = make_smem_desc(sb + k * b_step, b_lbo, b_sbo);
             if constexpr (MX) {
               // scale-factor ids: byte k of the 4-byte exponent word of each row (bits 29-30 for A, 4-5 for B)
-              umma_mxf8(d_tmem, ad, bd, p.idesc | (uint32_t(k) << 29) | (uint32_t(k) << 4), (kb | k) != 0 ? 1u : 0u,
-                        tmem_base + kSfaTmemCol, tmem_base + kSfbTmemCol);
+              const uint32_t id = p.idesc | (uint32_t(k) << 29) | (uint32_t(k) << 4);
+              if constexpr (NCTA == 1)
+                umma_mxf8(d_tmem, ad, bd, id, (kb | k) != 0 ? 1u : 0u, tmem_base + kSfaTmemCol, tmem_base + kSfbTmemCol);
+              else
+                umma_mxf8_pair(d_tmem, ad, bd, id, (kb | k) != 0 ? 1u : 0u, tmem_base + kSfaTmemCol,
+                               tmem_base + kSfbTmemCol);
             } else if constexpr (NCTA == 1) {
               umma_f8(d_tmem, ad, bd, p.idesc, (kb | k) != 0 ? 1u : 0u);
             } else {
@@ -581,15 +612,16 @@ template <int OUT, int NCTA>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                      const __grid_constant__ CUtensorMap map_y, const GemmParams p) {
-  gemm_body<OUT, NCTA, false>(map_a, map_b, map_y, p);
+  gemm_body<OUT, NCTA, false>(map_a, map_b, map_y, map_a, map_a, p);
 }
 
 // Block-scaled operands (E8M0 exponent per 32 elements of K), K-major A [M,K] and B [N,K].
-template <int OUT>
+template <int OUT, int NCTA>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 mx_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                 const __grid_constant__ CUtensorMap map_y, const GemmParams p) {
-  gemm_body<OUT, 1, true>(map_a, map_b, map_y, p);
+                 const __grid_constant__ CUtensorMap map_y, const __grid_constant__ CUtensorMap map_sfa,
+                 const __grid_constant__ CUtensorMap map_sfb, const GemmParams p) {
+  gemm_body<OUT, NCTA, true>(map_a, map_b, map_y, map_sfa, map_sfb, p);
 }
 
 // Diagnostic: one thread waits, with the GEMM's bounded-wait routine and a short limit, on an
@@ -819,26 +851,95 @@ int launch_scaled_matmul(const MatmulArgs& a, void* ws, cudaStream_t st) {
   return SCALIFY_OK;
 }
 
+// Tensor map over the exponent tiles of a block-scaled operand: a list of 512-byte tiles, one per box.
+static int make_map_sf(CUtensorMap* map, const void* ptr, uint64_t n_tiles) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return SCALIFY_ERR_CUDA;
+  cuuint64_t dims[3] = {128, n_tiles, 1};  // 128 32-bit words = 512 bytes per tile
+  cuuint64_t strides[2] = {512, 512 * n_tiles};
+  cuuint32_t box[3] = {128u, 1u, 1u};
+  cuuint32_t estr[3] = {1u, 1u, 1u};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    set_last_cuda_error(static_cast<int>(r));
+    return SCALIFY_ERR_CUDA;
+  }
+  return SCALIFY_OK;
+}
+
+template <int OUT, int NCTA>
+static int launch_mx_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_y,
+                             const CUtensorMap& map_sfa, const CUtensorMap& map_sfb, const GemmParams& p,
+                             long long tiles, cudaStream_t st) {
+  using C = GemmCfg<NCTA, true>;
+  auto kernel = mx_matmul_kernel<OUT, NCTA>;
+  static bool attr_done = false;
+  static int max_clusters = 0;
+  cudaLaunchAttribute attrs[1];
+  attrs[0].id = cudaLaunchAttributeClusterDimension;
+  attrs[0].val.clusterDim.x = 2; attrs[0].val.clusterDim.y = 1; attrs[0].val.clusterDim.z = 1;
+  if (!attr_done) {
+    SCALIFY_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(C::kSmem)));
+    if (NCTA == 2) {
+      cudaLaunchConfig_t qc = {};
+      qc.gridDim = dim3(unsigned(sm_count() / 2 * 2));
+      qc.blockDim = dim3(kGemmThreads);
+      qc.dynamicSmemBytes = C::kSmem;
+      qc.attrs = attrs;
+      qc.numAttrs = 1;
+      int n = 0;
+      SCALIFY_CUDA_TRY(cudaOccupancyMaxActiveClusters(&n, kernel, &qc));
+      if (n < 1) return SCALIFY_ERR_UNSUPPORTED;
+      max_clusters = n;
+    }
+    attr_done = true;
+  }
+  cudaLaunchConfig_t cfg = {};
+  if (NCTA == 2) {
+    const long long units = tiles < max_clusters ? tiles : max_clusters;
+    cfg.gridDim = dim3(unsigned(units * 2));
+    cfg.attrs = attrs;
+    cfg.numAttrs = 1;
+  } else {
+    cfg.gridDim = dim3(unsigned(tiles < sm_count() ? tiles : sm_count()));
+  }
+  cfg.blockDim = dim3(kGemmThreads);
+  cfg.dynamicSmemBytes = C::kSmem;
+  cfg.stream = st;
+  SCALIFY_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, map_a, map_b, map_y, map_sfa, map_sfb, p));
+  return SCALIFY_OK;
+}
+
 int launch_mx_matmul(const MxMatmulArgs& a, void* ws, cudaStream_t st) {
   WsView v = ws_view(ws);
-  CUtensorMap map_a, map_b, map_y;
+  const int ncta = (a.M > kBM && a.force_ncta != 1) ? 2 : 1;
+  const int tile_m = kBM * ncta;
+  CUtensorMap map_a, map_b, map_y, map_sfa, map_sfb;
   int rc = make_map(&map_a, a.A, a.K, a.M, 1, a.K, 0, kBM);
   if (rc) return rc;
-  rc = make_map(&map_b, a.B, a.K, a.N, 1, a.K, 0, kBN);
+  rc = make_map(&map_b, a.B, a.K, a.N, 1, a.K, 0, ncta == 2 ? kBN / 2 : kBN);
   if (rc) return rc;
   rc = make_map_y(&map_y, a.Y, elem_size(a.y_dt), a.N, a.M, 1, a.ldy, 0);
   if (rc) return rc;
+  const uint64_t k_tiles = uint64_t(a.K) / 128;
+  rc = make_map_sf(&map_sfa, a.sfa, uint64_t((a.M + 255) / 256 * 2) * k_tiles);
+  if (rc) return rc;
+  rc = make_map_sf(&map_sfb, a.sfb, uint64_t((a.N + 255) / 256 * 2) * k_tiles);
+  if (rc) return rc;
   GemmParams p;
   p.M = a.M; p.N = a.N; p.K = a.K; p.batch = 1;
-  p.tiles_m = (a.M + kBM - 1) / kBM;
+  p.tiles_m = (a.M + tile_m - 1) / tile_m;
   p.tiles_n = (a.N + kBN - 1) / kBN;
   p.a_mn_major = 0;
   p.b_mn_major = 0;
   p.b_batched = 0;
   // block-scaled instruction descriptor (kind::mxf8f6f4): scale-factor ids in bits 4-5 (B) and 29-30 (A)
-  // are filled in per MMA, A/B formats, K-major operands, N >> 3, E8M0 exponents (bit 23), M >> 4
+  // are filled in per MMA; A/B formats, K-major operands, N >> 3, E8M0 exponents (bit 23), M >> 4 (M counts
+  // the rows of the whole CTA pair)
   p.idesc = (uint32_t(a.a_dt == SCALIFY_E5M2) << 7) | (uint32_t(a.b_dt == SCALIFY_E5M2) << 10) |
-            (uint32_t(kBN >> 3) << 17) | (1u << 23) | (uint32_t(kBM >> 4) << 24);
+            (uint32_t(kBN >> 3) << 17) | (1u << 23) | (uint32_t(tile_m >> 4) << 24);
   p.kf = kfactor(a.K);
   p.alpha = 1.0f / p.kf;
   p.Y = a.Y; p.ldy = a.ldy; p.y_batch_stride = 0;
@@ -861,22 +962,12 @@ int launch_mx_matmul(const MxMatmulArgs& a, void* ws, cudaStream_t st) {
     }
   }
   SCALIFY_DISPATCH_WIDE(a.y_dt, OUT, {
-    using C = GemmCfg<1, true>;
-    auto kernel = mx_matmul_kernel<OUT>;
-    static bool attr_done = false;
-    if (!attr_done) {
-      SCALIFY_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(C::kSmem)));
-      attr_done = true;
-    }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(unsigned(tiles < sm_count() ? tiles : sm_count()));
-    cfg.blockDim = dim3(kGemmThreads);
-    cfg.dynamicSmemBytes = C::kSmem;
-    cfg.stream = st;
-    SCALIFY_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, map_a, map_b, map_y, p));
+    if (ncta == 2) rc = launch_mx_variant<OUT, 2>(map_a, map_b, map_y, map_sfa, map_sfb, p, tiles, st);
+    else rc = launch_mx_variant<OUT, 1>(map_a, map_b, map_y, map_sfa, map_sfb, p, tiles, st);
   });
+  if (rc) return rc;
   if (a.stat == SCALIFY_STAT_L2) {
-    gemm_l2_finalize_kernel<<<1, 256, 0, st>>>(p.l2_partials, static_cast<int>(tiles * 8),
+    gemm_l2_finalize_kernel<<<1, 256, 0, st>>>(p.l2_partials, static_cast<int>(tiles * ncta * 8),
                                                double(a.M) * double(a.N), v.stat);
     SCALIFY_CUDA_TRY(cudaGetLastError());
   }

@@ -396,6 +396,7 @@ int scalify_mx_matmul(const scalify_mx_array* A, const scalify_mx_array* B, scal
   a.M = static_cast<int>(A->rows); a.N = static_cast<int>(B->rows); a.K = static_cast<int>(A->K);
   a.a_scale = A->scale; a.b_scale = B->scale; a.y_scale = Y->scale;
   a.stat = stat;
+  a.force_ncta = 0;
   return launch_mx_matmul(a, workspace, static_cast<cudaStream_t>(stream));
 }
 

@@ -75,6 +75,7 @@ struct MxMatmulArgs {
   int M, N, K;
   const float* a_scale; const float* b_scale; float* y_scale;
   int stat;
+  int force_ncta;  // 0: choose; 1: force the one-CTA kernel
 };
 int launch_mx_matmul(const MxMatmulArgs& a, void* ws, cudaStream_t st);
 size_t mx_sf_bytes(int64_t rows, int64_t K);

@@ -99,14 +99,16 @@ def test_mx_matmul_against_oracle(M, N, K, a_dt, b_dt):
     assert stat == float(np.abs(orc.decode(gb, orc.BF16)).max())
 
 
-def test_mx_matmul_distinguishes_every_exponent_byte():
+@pytest.mark.parametrize("M", [128, 256])
+def test_mx_matmul_distinguishes_every_exponent_byte(M):
     """One block of A and one block of B get a large exponent each, at every position in turn: a kernel
-    that picked the wrong exponent byte (wrong row group, wrong K block, wrong half of a 256-column tile)
-    would miss the product."""
-    M, N, K = 128, 256, 256
+    that picked the wrong exponent byte (wrong row group, wrong K block, wrong half of a 256-column tile,
+    wrong CTA of a pair: M = 256 runs the two-CTA form) would miss the product."""
+    N, K = 256, 256
     a = si.to_bits(np.ones((M, K), dtype=np.float32), orc.E4M3)
     b = si.to_bits(np.ones((N, K), dtype=np.float32), orc.E4M3)
-    for (i, kb, j) in [(0, 0, 0), (31, 1, 33), (32, 2, 127), (64, 3, 128), (97, 4, 200), (127, 7, 255)]:
+    for (i, kb, j) in [(0, 0, 0), (31, 1, 33), (32, 2, 127), (64, 3, 128), (97, 4, 200), (127, 7, 255),
+                       (M - 128, 5, 129), (M - 1, 6, 64), (M - 60, 0, 250)]:
         ea = np.full((M, K // 32), 127, dtype=np.uint8)
         eb = np.full((N, K // 32), 127, dtype=np.uint8)
         ea[i, kb] = 130
