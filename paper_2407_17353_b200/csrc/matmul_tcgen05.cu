@@ -60,8 +60,9 @@ template <int NCTA, bool MX = false> struct GemmCfg {
   static constexpr int kEpiBytes = kEpiWarps * 32 * 128;  // per-warp staging tile of the epilogue: 32 rows x up to 128 B
   static constexpr size_t kSmem = size_t(kStages) * kStageBytes + kEpiBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
-constexpr uint32_t kSfaTmemCol = 256;  // MX: TMEM columns of the exponents of A (4) and of B (8)
-constexpr uint32_t kSfbTmemCol = 260;
+// MX: TMEM columns of the exponents, two buffers of 16 columns (A: 4, B: 8) used by alternate K blocks so
+// that the copy for one block does not have to wait for the MMAs of the block before it
+constexpr uint32_t kSfaTmemCol = 256;
 
 struct GemmParams {
   int M, N, K, batch;
@@ -443,6 +444,7 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
         if (!mbar_wait(acc_empty_bar + 8 * acc, acc_phase ^ 1u, abort_flag)) { timed_out = true; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * kBN;
+        uint32_t sf_col = 0;
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(full_bar + 8 * stage, phase, abort_flag)) { timed_out = true; break; }
           tc_fence_after();
@@ -450,14 +452,15 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
           if constexpr (MX) {
             // this K block's exponents: shared memory -> TMEM (executes in order with the MMAs of this thread)
             const uint32_t ssf = smem_sf + stage * C::kSfBytes;
+            sf_col = tmem_base + kSfaTmemCol + static_cast<uint32_t>(kb & 1) * 16u;  // two exponent buffers in TMEM
             if constexpr (NCTA == 1) {
-              tmem_cp_32x128b_warpx4(tmem_base + kSfaTmemCol, make_smem_desc_noswizzle(ssf, 512u, 128u));
-              tmem_cp_32x128b_warpx4(tmem_base + kSfbTmemCol, make_smem_desc_noswizzle(ssf + 512, 512u, 128u));
-              tmem_cp_32x128b_warpx4(tmem_base + kSfbTmemCol + 4, make_smem_desc_noswizzle(ssf + 1024, 512u, 128u));
+              tmem_cp_32x128b_warpx4(sf_col, make_smem_desc_noswizzle(ssf, 512u, 128u));
+              tmem_cp_32x128b_warpx4(sf_col + 4, make_smem_desc_noswizzle(ssf + 512, 512u, 128u));
+              tmem_cp_32x128b_warpx4(sf_col + 8, make_smem_desc_noswizzle(ssf + 1024, 512u, 128u));
             } else {
-              tmem_cp_32x128b_warpx4_pair(tmem_base + kSfaTmemCol, make_smem_desc_noswizzle(ssf, 512u, 128u));
-              tmem_cp_32x128b_warpx4_pair(tmem_base + kSfbTmemCol, make_smem_desc_noswizzle(ssf + 512, 512u, 128u));
-              tmem_cp_32x128b_warpx4_pair(tmem_base + kSfbTmemCol + 4, make_smem_desc_noswizzle(ssf + 1024, 512u, 128u));
+              tmem_cp_32x128b_warpx4_pair(sf_col, make_smem_desc_noswizzle(ssf, 512u, 128u));
+              tmem_cp_32x128b_warpx4_pair(sf_col + 4, make_smem_desc_noswizzle(ssf + 512, 512u, 128u));
+              tmem_cp_32x128b_warpx4_pair(sf_col + 8, make_smem_desc_noswizzle(ssf + 1024, 512u, 128u));
             }
           }
 #pragma unroll
@@ -468,10 +471,9 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
               // scale-factor ids: byte k of the 4-byte exponent word of each row (bits 29-30 for A, 4-5 for B)
               const uint32_t id = p.idesc | (uint32_t(k) << 29) | (uint32_t(k) << 4);
               if constexpr (NCTA == 1)
-                umma_mxf8(d_tmem, ad, bd, id, (kb | k) != 0 ? 1u : 0u, tmem_base + kSfaTmemCol, tmem_base + kSfbTmemCol);
+                umma_mxf8(d_tmem, ad, bd, id, (kb | k) != 0 ? 1u : 0u, sf_col, sf_col + 4);
               else
-                umma_mxf8_pair(d_tmem, ad, bd, id, (kb | k) != 0 ? 1u : 0u, tmem_base + kSfaTmemCol,
-                               tmem_base + kSfbTmemCol);
+                umma_mxf8_pair(d_tmem, ad, bd, id, (kb | k) != 0 ? 1u : 0u, sf_col, sf_col + 4);
             } else if constexpr (NCTA == 1) {
               umma_f8(d_tmem, ad, bd, p.idesc, (kb | k) != 0 ? 1u : 0u);
             } else {
