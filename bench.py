@@ -198,6 +198,19 @@ def run_profile_row(args):
         ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_MATMUL, n, n), dev)
         fn = lambda t: sc.scalify_scaled_matmul(A, Bt, Y, ws, transB=True, stat=sc.STAT_AMAX)
         work = {"flop": 2.0 * n ** 3}
+    elif row == "mx":
+        n = N_GEMM
+        Xa = sc.ScaledTensor.make(rnd((n, n), torch.bfloat16, 1), 1.0)
+        Xb = sc.ScaledTensor.make(rnd((n, n), torch.bfloat16, 2), 1.0)
+        Am, Bm = sc.MxTensor(n, n, device=dev), sc.MxTensor(n, n, device=dev)
+        Y = sc.ScaledTensor.empty((n, n), torch.bfloat16, dev)
+        ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_MATMUL, n, n), dev)
+
+        def fn(t):
+            sc.scalify_mx_quantize(Xa, Am)
+            sc.scalify_mx_quantize(Xb, Bm)
+            sc.scalify_mx_matmul(Am, Bm, Y, ws, stat=sc.STAT_AMAX)
+        work = {"flop": 2.0 * n ** 3}
     elif row == "rescale":
         n = 8192 * 8192
         X = sc.ScaledTensor.make(rnd((n,), torch.bfloat16, 1, 37.0), 1.0)
@@ -271,7 +284,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (for ncu launch lists)")
     ap.add_argument("--no-next", action="store_true",
                     help="skip the separately timed next-row variants f1, f2 (for ncu launch lists of the step)")
-    ap.add_argument("--profile-row", default=None, choices=["matmul", "rescale", "add", "layernorm", "adam"],
+    ap.add_argument("--profile-row", default=None, choices=["matmul", "mx", "rescale", "add", "layernorm", "adam"],
                     help="run only this row on a reduced, still larger-than-L2 case (for ncu captures)")
     args = ap.parse_args()
     if args.impl == "reference":

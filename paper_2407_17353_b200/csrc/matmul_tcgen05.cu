@@ -55,13 +55,17 @@ template <int NCTA, bool MX = false> struct GemmCfg {
   static constexpr int kBBytes = kBRows * kBK;       // 32 KB / 16 KB
   static constexpr int kSfBytes = MX ? 2048 : 0;     // exponent tiles of one K block (1536 B used)
   static constexpr int kStageBytes = kABytes + kBBytes + kSfBytes;
-  static constexpr int kStages = MX ? (NCTA == 1 ? 3 : 5) : (NCTA == 1 ? 4 : 6);
+  static constexpr int kStages = MX ? (NCTA == 1 ? 3 : 4) : (NCTA == 1 ? 3 : 5);
   static constexpr int kAcc = MX ? 1 : kAccStages;   // accumulators in TMEM
-  static constexpr int kEpiBytes = kEpiWarps * 32 * 128;  // per-warp staging tile of the epilogue: 32 rows x up to 128 B
+  // Epilogue staging: 8 KB per warp = one tile (32 rows x 32 columns) per chunk of a 16-bit output, so that a
+  // warp never waits for the TMA store of an earlier chunk of the same accumulator (two tiles for fp32 output).
+  static constexpr int kEpiWarpBytes = 8192;
+  static constexpr int kEpiBytes = kEpiWarps * kEpiWarpBytes;
   static constexpr size_t kSmem = size_t(kStages) * kStageBytes + kEpiBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
-// MX: TMEM columns of the exponents, two buffers of 16 columns (A: 4, B: 8) used by alternate K blocks so
-// that the copy for one block does not have to wait for the MMAs of the block before it
+// MX: TMEM columns of the exponents, two buffers 64 columns apart (A: 4 columns at +0, B: 8 columns at +32)
+// used by alternate K blocks so that the copy for one block does not have to wait for the MMAs of the block
+// before it
 constexpr uint32_t kSfaTmemCol = 256;
 
 struct GemmParams {
@@ -318,7 +322,7 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
   const uint32_t smem_a = base;
   const uint32_t smem_b = base + kStages * C::kABytes;
   const uint32_t smem_sf = smem_b + kStages * C::kBBytes;  // MX: [stage][A exponents 512 B | B exponents 2 x 512 B | pad]
-  uint8_t* epi_mem = smem + kStages * C::kStageBytes;  // 16 KB, 1024-byte aligned
+  uint8_t* epi_mem = smem + kStages * C::kStageBytes;  // 8 KB per epilogue warp, 1024-byte aligned
   uint8_t* bar_mem = epi_mem + C::kEpiBytes;
   const uint32_t bars = base + kStages * C::kStageBytes + C::kEpiBytes;
   const uint32_t full_bar = bars;                         // kStages x 8 B
@@ -440,44 +444,55 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
       const uint32_t b_lbo = (p.b_mn_major && NCTA == 1) ? kBK * 128u : 0u, b_sbo = 1024u;
       const uint32_t a_step = p.a_mn_major ? (kUmmaK * 128u) : kUmmaK;  // bytes per K=32 step
       const uint32_t b_step = p.b_mn_major ? (kUmmaK * 128u) : kUmmaK;
+      // The issuing thread is alone on its scheduler slot and every instruction between two MMAs is exposed
+      // latency, so everything that does not change is computed once: descriptors of ring slot 0 (a later
+      // slot or K step only adds to the 14-bit address field, which cannot carry: shared memory ends below
+      // 2^18 bytes), and the four instruction descriptors of a K block.
+      const uint64_t a_desc0 = make_smem_desc(smem_a, a_lbo, a_sbo);
+      const uint64_t b_desc0 = make_smem_desc(smem_b, b_lbo, b_sbo);
+      const uint64_t sf_desc0 = make_smem_desc_noswizzle(smem_sf, 512u, 128u);
+      constexpr uint32_t kAStageInc = C::kABytes >> 4, kBStageInc = C::kBBytes >> 4, kSfStageInc = C::kSfBytes >> 4;
+      const uint32_t a_k_inc = a_step >> 4, b_k_inc = b_step >> 4;
+      uint32_t idesc_k[kBK / kUmmaK];
+#pragma unroll
+      for (int k = 0; k < kBK / kUmmaK; ++k)  // MX: scale-factor ids = exponent byte k of each row's word (bits 29-30: A, 4-5: B)
+        idesc_k[k] = MX ? (p.idesc | (uint32_t(k) << 29) | (uint32_t(k) << 4)) : p.idesc;
       for (int tile = unit; tile < num_tiles && !timed_out; tile += num_units) {
         if (!mbar_wait(acc_empty_bar + 8 * acc, acc_phase ^ 1u, abort_flag)) { timed_out = true; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * kBN;
-        uint32_t sf_col = 0;
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(full_bar + 8 * stage, phase, abort_flag)) { timed_out = true; break; }
           tc_fence_after();
-          const uint32_t sa = smem_a + stage * C::kABytes, sb = smem_b + stage * C::kBBytes;
+          const uint64_t ad0 = a_desc0 + static_cast<uint64_t>(stage * kAStageInc);
+          const uint64_t bd0 = b_desc0 + static_cast<uint64_t>(stage * kBStageInc);
+          const uint32_t sf_col = tmem_base + kSfaTmemCol + static_cast<uint32_t>(kb & 1) * 64u;
           if constexpr (MX) {
-            // this K block's exponents: shared memory -> TMEM (executes in order with the MMAs of this thread)
-            const uint32_t ssf = smem_sf + stage * C::kSfBytes;
-            sf_col = tmem_base + kSfaTmemCol + static_cast<uint32_t>(kb & 1) * 16u;  // two exponent buffers in TMEM
+            // this K block's exponents: shared memory -> TMEM (executes in order with the MMAs of this thread);
+            // A's tile, then the two tiles of B, 512 bytes apart in the slot
+            const uint64_t sfd = sf_desc0 + static_cast<uint64_t>(stage * kSfStageInc);
             if constexpr (NCTA == 1) {
-              tmem_cp_32x128b_warpx4(sf_col, make_smem_desc_noswizzle(ssf, 512u, 128u));
-              tmem_cp_32x128b_warpx4(sf_col + 4, make_smem_desc_noswizzle(ssf + 512, 512u, 128u));
-              tmem_cp_32x128b_warpx4(sf_col + 8, make_smem_desc_noswizzle(ssf + 1024, 512u, 128u));
+              tmem_cp_32x128b_warpx4(sf_col, sfd);
+              tmem_cp_32x128b_warpx4(sf_col + 32, sfd + 32);
+              tmem_cp_32x128b_warpx4(sf_col + 36, sfd + 64);
             } else {
-              tmem_cp_32x128b_warpx4_pair(sf_col, make_smem_desc_noswizzle(ssf, 512u, 128u));
-              tmem_cp_32x128b_warpx4_pair(sf_col + 4, make_smem_desc_noswizzle(ssf + 512, 512u, 128u));
-              tmem_cp_32x128b_warpx4_pair(sf_col + 8, make_smem_desc_noswizzle(ssf + 1024, 512u, 128u));
+              tmem_cp_32x128b_warpx4_pair(sf_col, sfd);
+              tmem_cp_32x128b_warpx4_pair(sf_col + 32, sfd + 32);
+              tmem_cp_32x128b_warpx4_pair(sf_col + 36, sfd + 64);
             }
           }
 #pragma unroll
           for (int k = 0; k < kBK / kUmmaK; ++k) {
-            const uint64_t ad = make_smem_desc(sa + k * a_step, a_lbo, a_sbo);
-            const uint64_t bd = make_smem_desc(sb + k * b_step, b_lbo, b_sbo);
+            const uint64_t ad = ad0 + static_cast<uint64_t>(k * a_k_inc);
+            const uint64_t bd = bd0 + static_cast<uint64_t>(k * b_k_inc);
+            const uint32_t accumulate = (kb | k) != 0 ? 1u : 0u;
             if constexpr (MX) {
-              // scale-factor ids: byte k of the 4-byte exponent word of each row (bits 29-30 for A, 4-5 for B)
-              const uint32_t id = p.idesc | (uint32_t(k) << 29) | (uint32_t(k) << 4);
-              if constexpr (NCTA == 1)
-                umma_mxf8(d_tmem, ad, bd, id, (kb | k) != 0 ? 1u : 0u, sf_col, sf_col + 4);
-              else
-                umma_mxf8_pair(d_tmem, ad, bd, id, (kb | k) != 0 ? 1u : 0u, sf_col, sf_col + 4);
+              if constexpr (NCTA == 1) umma_mxf8(d_tmem, ad, bd, idesc_k[k], accumulate, sf_col, sf_col + 32);
+              else umma_mxf8_pair(d_tmem, ad, bd, idesc_k[k], accumulate, sf_col, sf_col + 32);
             } else if constexpr (NCTA == 1) {
-              umma_f8(d_tmem, ad, bd, p.idesc, (kb | k) != 0 ? 1u : 0u);
+              umma_f8(d_tmem, ad, bd, idesc_k[k], accumulate);
             } else {
-              umma_f8_pair(d_tmem, ad, bd, p.idesc, (kb | k) != 0 ? 1u : 0u);
+              umma_f8_pair(d_tmem, ad, bd, idesc_k[k], accumulate);
             }
           }
           // slot free (in both CTAs) once these MMAs have read it
@@ -543,10 +558,11 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
         // into a shared-memory tile in the swizzle pattern TMA uses for rows of this width, and one lane hands
         // the tile to a TMA store, which writes whole row segments and clips rows >= M and columns >= N.
         constexpr int CPR = 32 * OSZ / 16;              // 16-byte pieces per row: 2 (FP8), 4 (16-bit), 8 (F32)
-        constexpr int NBUF = OSZ == 4 ? 1 : 2;          // staging tiles per warp (4 KB per warp in all)
+        constexpr int kTileBytes = 32 * 32 * OSZ;
+        constexpr int NBUF = C::kEpiWarpBytes / kTileBytes > 4 ? 4 : C::kEpiWarpBytes / kTileBytes;  // 4, 4 or 2
         uint32_t o[32 * OSZ / 4];
         encode_vec<OUT, 32>(v, o);
-        uint8_t* tile_b = epi_mem + (warp - 2) * (32 * 128) + (NBUF == 2 ? (c & 1) * 2048 : 0);
+        uint8_t* tile_b = epi_mem + (warp - 2) * C::kEpiWarpBytes + (c % NBUF) * kTileBytes;
         if (lane == 0) bulk_wait_read<NBUF - 1>();      // the tile's previous store has read it
         __syncwarp();
         uint4* tile = reinterpret_cast<uint4*>(tile_b);
