@@ -538,9 +538,11 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
       const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kBN + c_first * 32;
       // chunks of this warp that lie inside the matrix (warp-uniform)
       const int n_chunks = max(0, min(kChunksPerWarp, (p.N - n0 + 31) / 32 - c_first));
-      // One 32-column chunk of this thread's row: scale, statistic, round, store.
-      auto process = [&](const uint32_t* acc_regs, int c) {
-        const int col0 = n0 + (c_first + c) * 32;
+      // One 32-column chunk of this thread's row in two steps: scale + statistic + round (convert), then store.
+      constexpr int CPR = 32 * OSZ / 16;              // 16-byte pieces per row: 2 (FP8), 4 (16-bit), 8 (F32)
+      constexpr int kTileBytes = 32 * 32 * OSZ;
+      constexpr int NBUF = C::kEpiWarpBytes / kTileBytes > 4 ? 4 : C::kEpiWarpBytes / kTileBytes;  // 4, 4 or 2
+      auto convert = [&](const uint32_t* acc_regs, uint32_t* o) {
         float v[32];
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
@@ -554,14 +556,13 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
             ssq = fmaf(s, s, ssq);
           }
         }
-        // Each lane holds 32 consecutive columns of ONE row.  The warp writes the chunk (32 rows x 32 columns)
-        // into a shared-memory tile in the swizzle pattern TMA uses for rows of this width, and one lane hands
-        // the tile to a TMA store, which writes whole row segments and clips rows >= M and columns >= N.
-        constexpr int CPR = 32 * OSZ / 16;              // 16-byte pieces per row: 2 (FP8), 4 (16-bit), 8 (F32)
-        constexpr int kTileBytes = 32 * 32 * OSZ;
-        constexpr int NBUF = C::kEpiWarpBytes / kTileBytes > 4 ? 4 : C::kEpiWarpBytes / kTileBytes;  // 4, 4 or 2
-        uint32_t o[32 * OSZ / 4];
         encode_vec<OUT, 32>(v, o);
+      };
+      // Each lane holds 32 consecutive columns of ONE row.  The warp writes the chunk (32 rows x 32 columns)
+      // into a shared-memory tile in the swizzle pattern TMA uses for rows of this width, and one lane hands
+      // the tile to a TMA store, which writes whole row segments and clips rows >= M and columns >= N.
+      auto store = [&](const uint32_t* o, int c) {
+        const int col0 = n0 + (c_first + c) * 32;
         uint8_t* tile_b = epi_mem + (warp - 2) * C::kEpiWarpBytes + (c % NBUF) * kTileBytes;
         if (lane == 0) bulk_wait_read<NBUF - 1>();      // the tile's previous store has read it
         __syncwarp();
@@ -576,25 +577,50 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
           bulk_commit();
         }
       };
-      // The TMEM load of the next chunk is in flight while the current chunk is processed.
-      uint32_t ra[32], rb[32];
-      if (n_chunks > 0) tmem_ld32(t_addr, ra);
-#pragma unroll 1
-      for (int c = 0; c < n_chunks; c += 2) {
-        tmem_ld_wait();
-        if (c + 1 < n_chunks) tmem_ld32(t_addr + (c + 1) * 32, rb);
-        process(ra, c);
-        if (c + 1 < n_chunks) {
-          tmem_ld_wait();
-          if (c + 2 < n_chunks) tmem_ld32(t_addr + (c + 2) * 32, ra);
-          process(rb, c + 1);
+      auto release_accumulator = [&]() {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+          if constexpr (NCTA == 1) mbar_arrive(acc_empty_bar + 8 * acc);
+          else mbar_arrive_cluster(map_to_cta(acc_empty_bar + 8 * acc, 0u));  // the leader issues the next MMAs
         }
-      }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) {
-        if constexpr (NCTA == 1) mbar_arrive(acc_empty_bar + 8 * acc);
-        else mbar_arrive_cluster(map_to_cta(acc_empty_bar + 8 * acc, 0u));  // the leader issues the next MMAs
+      };
+      uint32_t ra[32], rb[32];
+      if constexpr (kAcc == 1 && OSZ <= 2) {
+        // A single accumulator: the next tile's MMAs wait for this read-out, so all chunks are read and
+        // converted first (kept as packed output words), the accumulator is handed back, then the stores follow.
+        uint32_t oc[kChunksPerWarp][32 * OSZ / 4];
+        if (n_chunks > 0) tmem_ld32(t_addr, ra);
+#pragma unroll
+        for (int c = 0; c < kChunksPerWarp; ++c) {
+          if (c < n_chunks) {
+            tmem_ld_wait();
+            if (c + 1 < n_chunks) tmem_ld32(t_addr + (c + 1) * 32, (c & 1) ? ra : rb);
+            convert((c & 1) ? rb : ra, oc[c]);
+          }
+        }
+        release_accumulator();
+#pragma unroll
+        for (int c = 0; c < kChunksPerWarp; ++c)
+          if (c < n_chunks) store(oc[c], c);
+      } else {
+        // The TMEM load of the next chunk is in flight while the current chunk is processed.
+        uint32_t o[32 * OSZ / 4];
+        if (n_chunks > 0) tmem_ld32(t_addr, ra);
+#pragma unroll 1
+        for (int c = 0; c < n_chunks; c += 2) {
+          tmem_ld_wait();
+          if (c + 1 < n_chunks) tmem_ld32(t_addr + (c + 1) * 32, rb);
+          convert(ra, o);
+          store(o, c);
+          if (c + 1 < n_chunks) {
+            tmem_ld_wait();
+            if (c + 2 < n_chunks) tmem_ld32(t_addr + (c + 2) * 32, ra);
+            convert(rb, o);
+            store(o, c + 1);
+          }
+        }
+        release_accumulator();
       }
       if (p.stat == SCALIFY_STAT_L2) {
         const double s = warp_sum_f64(static_cast<double>(ssq)) * (double(r_prev) * double(r_prev));
