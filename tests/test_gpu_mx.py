@@ -118,6 +118,22 @@ def test_mx_matmul_distinguishes_every_exponent_byte(M):
         assert np.array_equal(orc.decode(g, orc.F32).reshape(M, N), acc), (i, kb, j)
 
 
+def test_mx_matmul_f16_output_and_l2_statistic():
+    M, N, K = 320, 272, 256
+    a = si.to_bits(si.normal(41, 1, (M, K), 1.0), orc.E5M2)
+    b = si.to_bits(si.normal(41, 2, (N, K), 1.0), orc.E5M2)
+    rng = np.random.default_rng(11)
+    ea = rng.integers(122, 130, size=(M, K // 32)).astype(np.uint8)
+    eb = rng.integers(122, 130, size=(N, K // 32)).astype(np.uint8)
+    Yo, ys, acc, sab = orc.mx_matmul(a, orc.E5M2, ea, 1.0, b, orc.E5M2, eb, 2.0 ** -5, orc.F16, want_acc=True)
+    g, s, stat = run_mx_matmul(a, orc.E5M2, ea, 1.0, b, orc.E5M2, eb, 2.0 ** -5, orc.F16, stat=sc.STAT_L2)
+    assert s == ys
+    ok = within(g, Yo, orc.F16, acc, sab, 1e-5)
+    assert ok.all(), int((~ok).sum())
+    want = float(np.sqrt(np.mean(orc.decode(g, orc.F16).astype(np.float64) ** 2)))
+    assert abs(stat - want) <= 2e-6 * want
+
+
 def test_quantize_then_matmul_matches_the_oracle_pipeline():
     M, N, K = 384, 512, 512
     xa = wide_range_input(31, M, K, orc.BF16, spread=8)
