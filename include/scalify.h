@@ -428,6 +428,33 @@ int scalify_mx_matmul(const scalify_mx_array* A, const scalify_mx_array* B, scal
                       void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Fused scaled attention forward: S = Q K^T, P = softmax(S c), O = P V in one
+ * kernel per (head, 128 queries); the scores and the probabilities stay on chip.
+ * The paper names attention as a place for a custom scale rule (Section 3.2.1)
+ * and gives none; the rule here is the composition of the calls it replaces:
+ *   S_s = Q_s K_s kf(hd),  S_d = (Q_d K_d^T) / kf(hd) rounded to BF16      (matmul rule)
+ *   P   = softmax over the keys of the VALUES S_d S_s c, optionally causal
+ *         (query i sees keys j <= i + Tk - Tq); bounded in [0,1], scale 1, rounded to E4M3
+ *   O_s = V_s kf(Tk),      O_d = (P_d V_d) / kf(Tk)                          (matmul rule)
+ * i.e. scalify_scaled_matmul, scalify_scalar_mul_pow2, scalify_scaled_softmax,
+ * scalify_scaled_matmul.  The softmax is the exact two-sweep form (row maximum
+ * and sum first, then the normalised probabilities), not an online rescaling.
+ *   Q [heads, Tq, hd], K, V [heads, Tk, hd]: E4M3 or E5M2, hd = 64, 3-D views
+ *   (row and head strides in stride[1], stride[0]; 2-D arrays are one head);
+ *   O [heads, Tq, hd]: F16, BF16 or F32, same kind of view; c: any finite
+ *   scalar (a power of two only shifts the exponent; otherwise its mantissa is
+ *   applied in fp32).  causal needs Tk >= Tq.
+ *   S_dump (BF16) and P_dump (E4M3): optional dense [heads, Tq, Tk] DEVICE
+ *   copies of S_d and P for checking (Tk % 32 == 0), normally NULL.
+ *   status: optional DEVICE word (SCALIFY_DEV_TIMEOUT, SCALIFY_DEV_BAD_SCALE).
+ * Errors: NULL, DTYPE, SHAPE, ALIGNMENT, UNSUPPORTED (hd != 64, causal with
+ * Tk < Tq), ALIAS (O_s aliasing an input scale word).
+ */
+int scalify_scaled_attention(const scalify_array* Q, const scalify_array* K, const scalify_array* V, float sm_scale,
+                             int causal, scalify_array* O, scalify_array* S_dump, scalify_array* P_dump,
+                             uint32_t* status, void* stream);
+
+/*
  * Scaled Adam step without a workspace.  (No counterpart in the paper: this entry point exists
  * for the integration, not for the method.)
  *

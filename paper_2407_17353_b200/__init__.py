@@ -80,6 +80,7 @@ def lib() -> ctypes.CDLL:
         L.scalify_scaled_gelu.argtypes = [P, i32, P, vp]
         L.scalify_scaled_gelu_bwd.argtypes = [P, P, i32, P, vp]
         L.scalify_scaled_adam_step.argtypes = [i32, P, P, P, P, f32, f32, f32, f32, i64, vp, sz, vp]
+        L.scalify_scaled_attention.argtypes = [P, P, P, f32, i32, P, P, P, vp, vp]
         L.scalify_mx_sf_bytes.restype = sz
         L.scalify_mx_sf_bytes.argtypes = [i64, i64]
         L.scalify_mx_quantize.argtypes = [P, vp, vp, vp]
@@ -100,7 +101,7 @@ def lib() -> ctypes.CDLL:
                      "scalify_scaled_adam_step", "scalify_scaled_adam_step_cast", "scalify_scaled_adam_step_static", "scalify_scaled_embedding",
                      "scalify_scaled_embedding_bwd", "scalify_scaled_softmax", "scalify_scaled_softmax_bwd",
                      "scalify_scaled_cross_entropy", "scalify_scalar_mul_pow2", "scalify_debug_expire_wait",
-                     "scalify_mx_quantize", "scalify_mx_matmul"):
+                     "scalify_mx_quantize", "scalify_mx_matmul", "scalify_scaled_attention"):
             getattr(L, name).restype = i32
         _lib = L
     return _lib
@@ -415,3 +416,14 @@ def scalify_mx_matmul(A: MxTensor, B: MxTensor, Y: ScaledTensor, ws: Workspace, 
     y = _desc(Y)
     _check(lib().scalify_mx_matmul(ctypes.addressof(A._d), ctypes.addressof(B._d), _ref(y), int(stat), ws.ptr,
                                    ws.nbytes, _stream(stream)), "scalify_mx_matmul")
+
+
+def scalify_scaled_attention(Q: ScaledTensor, K: ScaledTensor, V: ScaledTensor, O: ScaledTensor, *, sm_scale: float,
+                             causal: bool = True, S_dump: Optional[ScaledTensor] = None,
+                             P_dump: Optional[ScaledTensor] = None, status: Optional[torch.Tensor] = None,
+                             stream=None) -> None:
+    """Fused attention forward over [heads, T, 64] FP8 views; S_dump / P_dump are optional debug copies."""
+    q, k, v, o, sd, pd = _desc(Q), _desc(K), _desc(V), _desc(O), _desc(S_dump), _desc(P_dump)
+    _check(lib().scalify_scaled_attention(_ref(q), _ref(k), _ref(v), float(sm_scale), int(bool(causal)), _ref(o),
+                                          _ref(sd), _ref(pd), _ptr(status), _stream(stream)),
+           "scalify_scaled_attention")

@@ -1,0 +1,345 @@
+// Fused scaled attention forward (Section 3.2.1: attention is a place for a custom scale rule;
+// the rule taken here is the composition the unfused path uses): for every head
+//   S = Q K^T            scaled FP8 matmul, static rule:  S_s = Q_s K_s kf(hd),  S_d = bf16(acc / kf(hd))
+//   P = softmax(S_d S_s c) on VALUES (c = 1/sqrt(hd) or any scalar), causal mask optional; the
+//                        probabilities are bounded, carry scale 1 and are rounded to E4M3
+//   O = P V              scaled FP8 matmul, static rule:  O_s = V_s kf(Tk),  O_d = acc / kf(Tk)
+// in ONE kernel: neither S nor P ever reaches HBM (unless the caller asks for debug copies).
+//
+// One CTA per (head, block of 128 queries); 160 threads:
+//   warps 0-3   one query row per thread (the TMEM lane of the row): read the score block from
+//               TMEM, softmax arithmetic, write the E4M3 probabilities as the A operand of the
+//               second matmul into shared memory (128-byte swizzle), final read-out of O
+//   warp 4      one thread: TMA loads of Q, K, V tiles (64-byte swizzle) and all tcgen05.mma
+// The softmax is the exact two-sweep form, not an online approximation of it: sweep A runs
+// Q K^T over the key blocks and keeps the row maximum m and the sum l = sum exp(s - m)
+// (rescaled when m grows); sweep B recomputes Q K^T, forms p = exp(s - m) / l, rounds it to
+// E4M3 and accumulates P V in TMEM.  The probabilities are therefore the same normalised values
+// the unfused path quantises, and O needs no rescaling.  Cost: the Q K^T work twice.
+// TMEM: 128 columns of scores + 64 columns of O (256 allocated, so two CTAs share an SM).
+// Every mbarrier wait is bounded; on expiry the CTA records SCALIFY_DEV_TIMEOUT and leaves.
+#include <cuda.h>
+
+#include "scalify_common.cuh"
+#include "scalify_launch.h"
+#include "tcgen05_ptx.cuh"
+
+namespace scalify {
+
+constexpr int kAttQ = 128;     // queries per CTA
+constexpr int kAttK = 128;     // keys per block
+constexpr int kAttHd = 64;     // head dimension (bytes per row of Q, K, V)
+constexpr int kAttThreads = 160;
+constexpr int kAttTmemCols = 256;
+constexpr uint32_t kAttOCol = 128;
+constexpr int kAttTileBytes = kAttK * kAttHd;  // 8 KB: a Q, K or V tile
+constexpr size_t kAttSmem = size_t(kAttTileBytes) * 5 /*Q, 2 x K, 2 x V*/ + kAttQ * kAttK /*P*/ + 1024 + 256;
+
+struct AttParams {
+  int heads, Tq, Tk, q_blocks;
+  int causal;
+  const float* q_scale; const float* k_scale;
+  float sc_const;   // kf(hd) c log2(e); times Q_s K_s: scores' data component -> exponent in base 2
+  float inv_kf_hd;  // 1 / kf(hd)
+  float inv_kf_tk;  // 1 / kf(Tk)
+  uint32_t idesc_s, idesc_pv;
+  void* O; long long o_ld, o_hs;
+  void* S_dump; void* P_dump;
+  const float* v_scale; float kf_tk; float* o_scale;
+  uint32_t* status;
+};
+
+// 64-byte-swizzle shared-memory matrix descriptor (layout type 4): K-major tile of 64-byte rows
+// (8-row atoms 512 B apart) or MN-major tile whose 64 MN-elements are one row (8 K-rows per atom).
+__device__ __forceinline__ uint64_t make_smem_desc_sw64(uint32_t saddr, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);
+  d |= static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= 1ull << 46;
+  d |= 4ull << 61;
+  return d;
+}
+
+template <int ODT>
+__global__ void __launch_bounds__(kAttThreads, 2)
+attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                     const __grid_constant__ CUtensorMap map_v, const AttParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (base - raw);
+  const uint32_t smem_q = base;
+  const uint32_t smem_k = base + kAttTileBytes;          // 2 slots
+  const uint32_t smem_v = base + 3 * kAttTileBytes;      // 2 slots
+  const uint32_t smem_p = base + 5 * kAttTileBytes;      // 16 KB, 1024-byte aligned
+  uint8_t* p_tile = smem + 5 * kAttTileBytes;
+  uint8_t* bar_mem = p_tile + kAttQ * kAttK;
+  const uint32_t bars = smem_p + kAttQ * kAttK;
+  const uint32_t q_full = bars, kv_full = bars + 8 /*2*/, kv_empty = bars + 24 /*2*/, s_full = bars + 40,
+                 s_empty = bars + 48, p_full = bars + 56, p_empty = bars + 64, o_full = bars + 72;
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bar_mem + 80);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int head = blockIdx.x / p.q_blocks, qb = blockIdx.x % p.q_blocks;
+  const int q0 = qb * kAttQ;
+  const int shift = p.Tk - p.Tq;  // causal: query i sees keys j <= i + shift
+  int n_kb = (p.Tk + kAttK - 1) / kAttK;
+  if (p.causal) n_kb = min(n_kb, (q0 + kAttQ - 1 + shift) / kAttK + 1);
+
+  if (threadIdx.x == 0) {
+    mbar_init(q_full, 1);
+    for (int s = 0; s < 2; ++s) { mbar_init(kv_full + 8 * s, 1); mbar_init(kv_empty + 8 * s, 1); }
+    mbar_init(s_full, 1);
+    mbar_init(s_empty, 4);
+    mbar_init(p_full, 4);
+    mbar_init(p_empty, 1);
+    mbar_init(o_full, 1);
+    *abort_flag = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (blockIdx.x == 0) {
+      const float vs = load_scale(p.v_scale);
+      if (p.o_scale) *p.o_scale = vs * p.kf_tk;  // P carries scale 1
+      if (!is_pow2_scale(vs) && p.status) atomicOr(p.status, static_cast<uint32_t>(SCALIFY_DEV_BAD_SCALE));
+    }
+  }
+  if (warp == 4) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kAttTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  bool timed_out = false;
+
+  if (warp == 4) {
+    // ------------------------------------------------------------ loads and MMAs (one thread)
+    if (lane == 0) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_q)) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_k)) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_v)) : "memory");
+      const int n_it = 2 * n_kb;  // sweep A (K only), sweep B (K and V)
+      auto issue_load = [&](int it) {
+        const int slot = it & 1, use = it >> 1;
+        if (use >= 1 && !mbar_wait(kv_empty + 8 * slot, (use - 1) & 1, abort_flag)) { timed_out = true; return; }
+        const bool sweep_b = it >= n_kb;
+        const int kb = sweep_b ? it - n_kb : it;
+        const uint32_t fb = kv_full + 8 * slot;
+        mbar_expect_tx(fb, sweep_b ? 2 * kAttTileBytes : kAttTileBytes);
+        tma_load_3d(smem_k + slot * kAttTileBytes, &map_k, fb, 0, kb * kAttK, head);
+        if (sweep_b) tma_load_3d(smem_v + slot * kAttTileBytes, &map_v, fb, 0, kb * kAttK, head);
+      };
+      mbar_expect_tx(q_full, kAttTileBytes);
+      tma_load_3d(smem_q, &map_q, q_full, 0, q0, head);
+      issue_load(0);
+      if (!timed_out && !mbar_wait(q_full, 0u, abort_flag)) timed_out = true;
+      const uint64_t q_desc = make_smem_desc_sw64(smem_q, 512u);
+      const uint64_t p_desc = make_smem_desc(smem_p, 0u, 1024u);
+      for (int it = 0; it < n_it && !timed_out; ++it) {
+        if (it + 1 < n_it) { issue_load(it + 1); if (timed_out) break; }
+        const int slot = it & 1;
+        if (!mbar_wait(kv_full + 8 * slot, (it >> 1) & 1, abort_flag)) { timed_out = true; break; }
+        // the score block in TMEM is free once the softmax threads have read the previous one
+        if (it >= 1 && !mbar_wait(s_empty, (it - 1) & 1, abort_flag)) { timed_out = true; break; }
+        tc_fence_after();
+        const uint64_t k_desc = make_smem_desc_sw64(smem_k + slot * kAttTileBytes, 512u);
+#pragma unroll
+        for (int k = 0; k < kAttHd / 32; ++k)  // K = 32 bytes per MMA: +32 B on both K-major operands
+          umma_f8(tmem_base, q_desc + static_cast<uint64_t>(k * 2), k_desc + static_cast<uint64_t>(k * 2), p.idesc_s,
+                  k != 0 ? 1u : 0u);
+        umma_commit(s_full);
+        if (it < n_kb) {
+          umma_commit(kv_empty + 8 * slot);  // sweep A: the K tile is free after Q K^T
+        } else {
+          const int b = it - n_kb;
+          if (!mbar_wait(p_full, b & 1, abort_flag)) { timed_out = true; break; }
+          tc_fence_after();
+          // V tile [128 keys][64 B]: the B operand in MN-major form, 8-key atoms 512 B apart, 32 keys per MMA
+          const uint64_t v_desc = make_smem_desc_sw64(smem_v + slot * kAttTileBytes, 512u);
+#pragma unroll
+          for (int k = 0; k < kAttK / 32; ++k)
+            umma_f8(tmem_base + kAttOCol, p_desc + static_cast<uint64_t>(k * 2),
+                    v_desc + static_cast<uint64_t>(k * (32 * kAttHd / 16)), p.idesc_pv, (b | k) != 0 ? 1u : 0u);
+          umma_commit(p_empty);
+          umma_commit(kv_empty + 8 * slot);
+        }
+      }
+      if (!timed_out) umma_commit(o_full);
+      if (timed_out || *abort_flag) {
+        // wait (bounded) for the copies still in flight before the CTA's shared memory goes away
+        const unsigned long long t0 = global_timer_ns();
+        while (global_timer_ns() - t0 < 2000000ull) {}
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ softmax rows (one row per thread)
+    const int r = warp * 32 + lane;
+    const int i = q0 + r;                     // query index
+    const int lim = p.causal ? min(p.Tk, i + shift + 1) : p.Tk;  // keys [0, lim) are visible
+    const uint32_t t_row = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
+    float m = -INFINITY, l = 0.f;
+    const float sc2 = load_scale(p.q_scale) * load_scale(p.k_scale) * p.sc_const;
+    long long dump_row = (static_cast<long long>(head) * p.Tq + i) * p.Tk;
+    // x = data component of the score (rounded to BF16 like the unfused intermediate) in units of log2(e)
+    auto score = [&](uint32_t acc_bits, int j) {
+      const float sd = round_through<SCALIFY_BF16>(__uint_as_float(acc_bits) * p.inv_kf_hd);
+      return j < lim ? sd * sc2 : -INFINITY;
+    };
+    int it = 0;
+    // sweep A: row maximum and sum of exponentials
+    for (int kb = 0; kb < n_kb; ++kb, ++it) {
+      if (!mbar_wait(s_full, it & 1, abort_flag)) { timed_out = true; break; }
+      tc_fence_after();
+      uint32_t acc[32];
+      float bm = -INFINITY;
+#pragma unroll 1
+      for (int c = 0; c < kAttK / 32; ++c) {
+        tmem_ld32(t_row + c * 32, acc);
+        tmem_ld_wait();
+#pragma unroll
+        for (int e = 0; e < 32; ++e) bm = fmaxf(bm, score(acc[e], kb * kAttK + c * 32 + e));
+        if (p.S_dump && i < p.Tq) {
+          const int j0 = kb * kAttK + c * 32;
+          if (j0 < p.Tk) {  // Tk is a multiple of 32 when a dump is requested
+            float v[32];
+#pragma unroll
+            for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(acc[e]) * p.inv_kf_hd;
+            uint32_t o[16];
+            encode_vec<SCALIFY_BF16, 32>(v, o);
+            uint4* dst = reinterpret_cast<uint4*>(static_cast<char*>(p.S_dump) + (dump_row + j0) * 2);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) dst[q] = make_uint4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
+          }
+        }
+      }
+      const float m_new = fmaxf(m, bm);
+      float add = 0.f;
+      if (m_new > -INFINITY) {
+#pragma unroll 1
+        for (int c = 0; c < kAttK / 32; ++c) {
+          tmem_ld32(t_row + c * 32, acc);
+          tmem_ld_wait();
+#pragma unroll
+          for (int e = 0; e < 32; ++e) add += exp2f(score(acc[e], kb * kAttK + c * 32 + e) - m_new);
+        }
+        l = l * exp2f(m - m_new) + add;  // exp2f(-inf) = 0 while nothing has been seen yet
+        m = m_new;
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(s_empty);
+    }
+    const float inv_l = 1.0f / l;
+    // sweep B: probabilities -> E4M3 -> shared memory (A operand of P V)
+    for (int kb = 0; kb < n_kb && !timed_out; ++kb, ++it) {
+      if (!mbar_wait(s_full, it & 1, abort_flag)) { timed_out = true; break; }
+      tc_fence_after();
+      // the previous block's P V must have read the tile before it is overwritten
+      if (kb >= 1 && !mbar_wait(p_empty, (kb - 1) & 1, abort_flag)) { timed_out = true; break; }
+      uint32_t acc[32];
+#pragma unroll 1
+      for (int c = 0; c < kAttK / 32; ++c) {
+        tmem_ld32(t_row + c * 32, acc);
+        tmem_ld_wait();
+        float pr[32];
+#pragma unroll
+        for (int e = 0; e < 32; ++e) pr[e] = exp2f(score(acc[e], kb * kAttK + c * 32 + e) - m) * inv_l;
+        uint32_t o[8];
+        encode_vec<SCALIFY_E4M3, 32>(pr, o);
+        // row r of the tile: 128 bytes = eight 16-byte pieces, piece index XOR (r % 8) (128-byte swizzle)
+        uint4* row = reinterpret_cast<uint4*>(p_tile + r * 128);
+        row[(2 * c) ^ (r & 7)] = make_uint4(o[0], o[1], o[2], o[3]);
+        row[(2 * c + 1) ^ (r & 7)] = make_uint4(o[4], o[5], o[6], o[7]);
+        if (p.P_dump && i < p.Tq) {
+          const int j0 = kb * kAttK + c * 32;
+          if (j0 < p.Tk) {
+            uint4* dst = reinterpret_cast<uint4*>(static_cast<char*>(p.P_dump) + dump_row + j0);
+            dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+            dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+          }
+        }
+      }
+      fence_async_smem();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) { mbar_arrive(s_empty); mbar_arrive(p_full); }
+    }
+    // O: 64 fp32 columns of this row
+    if (!timed_out && mbar_wait(o_full, 0u, abort_flag)) {
+      tc_fence_after();
+      constexpr int OSZ = ElemBytes<ODT>::v;
+#pragma unroll 1
+      for (int c = 0; c < kAttHd / 32; ++c) {
+        uint32_t acc[32];
+        tmem_ld32(t_row + kAttOCol + c * 32, acc);
+        tmem_ld_wait();
+        if (i < p.Tq) {
+          float v[32];
+#pragma unroll
+          for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(acc[e]) * p.inv_kf_tk;
+          uint32_t o[32 * OSZ / 4];
+          encode_vec<ODT, 32>(v, o);
+          uint4* dst = reinterpret_cast<uint4*>(static_cast<char*>(p.O) +
+                                                (static_cast<long long>(head) * p.o_hs + static_cast<long long>(i) * p.o_ld +
+                                                 c * 32) * OSZ);
+#pragma unroll
+          for (int q = 0; q < 32 * OSZ / 16; ++q) dst[q] = make_uint4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
+        }
+      }
+    } else {
+      timed_out = true;
+    }
+  }
+
+  if (timed_out && p.status) atomicOr(p.status, static_cast<uint32_t>(SCALIFY_DEV_TIMEOUT));
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 4) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kAttTmemCols);
+  }
+}
+
+int launch_attention(const AttentionArgs& a, cudaStream_t st) {
+  CUtensorMap map_q, map_k, map_v;
+  int rc = make_byte_map(&map_q, a.Q, a.hd, a.Tq, a.heads, a.q_ld, a.q_hs, kAttHd, kAttQ);
+  if (rc) return rc;
+  rc = make_byte_map(&map_k, a.K, a.hd, a.Tk, a.heads, a.k_ld, a.k_hs, kAttHd, kAttK);
+  if (rc) return rc;
+  rc = make_byte_map(&map_v, a.V, a.hd, a.Tk, a.heads, a.v_ld, a.v_hs, kAttHd, kAttK);
+  if (rc) return rc;
+  AttParams p;
+  p.heads = a.heads; p.Tq = a.Tq; p.Tk = a.Tk;
+  p.q_blocks = (a.Tq + kAttQ - 1) / kAttQ;
+  p.causal = a.causal;
+  p.inv_kf_hd = 1.0f / kfactor(a.hd);
+  p.kf_tk = kfactor(a.Tk);
+  p.inv_kf_tk = 1.0f / p.kf_tk;
+  p.O = a.O; p.o_ld = a.o_ld; p.o_hs = a.o_hs;
+  p.S_dump = a.S_dump; p.P_dump = a.P_dump;
+  p.v_scale = a.v_scale; p.o_scale = a.o_scale;
+  p.status = a.status;
+  // scores: D fp32, A = Q, B = K (both K-major), N = 128, M = 128
+  p.idesc_s = (1u << 4) | (uint32_t(a.q_dt == SCALIFY_E5M2) << 7) | (uint32_t(a.k_dt == SCALIFY_E5M2) << 10) |
+              (uint32_t(kAttK >> 3) << 17) | (uint32_t(kAttQ >> 4) << 24);
+  // P V: A = P (E4M3, K-major), B = V (MN-major: keys are the contraction), N = 64, M = 128
+  p.idesc_pv = (1u << 4) | (uint32_t(a.v_dt == SCALIFY_E5M2) << 10) | (1u << 16) | (uint32_t(kAttHd >> 3) << 17) |
+               (uint32_t(kAttQ >> 4) << 24);
+  p.q_scale = a.q_scale; p.k_scale = a.k_scale;
+  // kf(hd) and a power-of-two c only shift the exponent; the product with log2(e) rounds once, as in the
+  // stand-alone softmax kernel
+  p.sc_const = kfactor(a.hd) * a.sm_scale * 1.4426950408889634f;
+  const long long ctas = static_cast<long long>(a.heads) * p.q_blocks;
+  if (ctas > 0x7FFFFFFF) return SCALIFY_ERR_SHAPE;
+  SCALIFY_DISPATCH_WIDE(a.o_dt, ODT, {
+    auto kernel = attention_fwd_kernel<ODT>;
+    static bool attr_done = false;
+    if (!attr_done) {
+      SCALIFY_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kAttSmem)));
+      attr_done = true;
+    }
+    kernel<<<static_cast<unsigned>(ctas), kAttThreads, kAttSmem, st>>>(map_q, map_k, map_v, p);
+  });
+  SCALIFY_CUDA_TRY(cudaGetLastError());
+  return SCALIFY_OK;
+}
+
+}  // namespace scalify

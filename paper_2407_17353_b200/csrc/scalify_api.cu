@@ -400,6 +400,58 @@ int scalify_mx_matmul(const scalify_mx_array* A, const scalify_mx_array* B, scal
   return launch_mx_matmul(a, workspace, static_cast<cudaStream_t>(stream));
 }
 
+// [heads, T, hd] view of a 2-D or 3-D array: head count, rows, row and head strides (elements)
+static int as_heads(const scalify_array* a, int64_t* heads, int64_t* rows, int64_t* cols, int64_t* ld, int64_t* hs) {
+  if (a->ndim == 2) { *heads = 1; *rows = a->shape[0]; *cols = a->shape[1]; *ld = a->stride[0]; *hs = 0; return SCALIFY_OK; }
+  if (a->ndim == 3) {
+    *heads = a->shape[0]; *rows = a->shape[1]; *cols = a->shape[2]; *ld = a->stride[1]; *hs = a->stride[0];
+    return SCALIFY_OK;
+  }
+  return SCALIFY_ERR_SHAPE;
+}
+
+int scalify_scaled_attention(const scalify_array* Q, const scalify_array* K, const scalify_array* V, float sm_scale,
+                             int causal, scalify_array* O, scalify_array* S_dump, scalify_array* P_dump,
+                             uint32_t* status, void* stream) {
+  int rc;
+  if ((rc = check_array(Q)) || (rc = check_array(K)) || (rc = check_array(V)) || (rc = check_array(O))) return rc;
+  if (is_wide(Q->dtype) || is_wide(K->dtype) || is_wide(V->dtype) || !is_wide(O->dtype)) return SCALIFY_ERR_DTYPE;
+  if (!isfinite(sm_scale)) return SCALIFY_ERR_VALUE;
+  AttentionArgs a;
+  int64_t hq, hk, hv, ho, tq, tk, tv, to, dq, dk, dv, dout;
+  if ((rc = as_heads(Q, &hq, &tq, &dq, &a.q_ld, &a.q_hs)) || (rc = as_heads(K, &hk, &tk, &dk, &a.k_ld, &a.k_hs)) ||
+      (rc = as_heads(V, &hv, &tv, &dv, &a.v_ld, &a.v_hs)) || (rc = as_heads(O, &ho, &to, &dout, &a.o_ld, &a.o_hs)))
+    return rc;
+  if (hq != hk || hq != hv || hq != ho || tk != tv || tq != to || dq != dk || dq != dv || dq != dout)
+    return SCALIFY_ERR_SHAPE;
+  if (tq < 1 || tk < 1 || hq < 1 || tq > 0x7FFFFFFF || tk > 0x7FFFFFFF || hq > 0x7FFFFFFF) return SCALIFY_ERR_SHAPE;
+  if (dq != 64 || (causal && tk < tq)) return SCALIFY_ERR_UNSUPPORTED;
+  if (O->scale && (O->scale == Q->scale || O->scale == K->scale || O->scale == V->scale)) return SCALIFY_ERR_ALIAS;
+  a.S_dump = nullptr;
+  a.P_dump = nullptr;
+  if (S_dump) {
+    if ((rc = check_array(S_dump))) return rc;
+    if (S_dump->dtype != SCALIFY_BF16) return SCALIFY_ERR_DTYPE;
+    if (contiguous_numel(S_dump) != hq * tq * tk || tk % 32 != 0) return SCALIFY_ERR_SHAPE;
+    a.S_dump = S_dump->data;
+  }
+  if (P_dump) {
+    if ((rc = check_array(P_dump))) return rc;
+    if (P_dump->dtype != SCALIFY_E4M3) return SCALIFY_ERR_DTYPE;
+    if (contiguous_numel(P_dump) != hq * tq * tk || tk % 32 != 0) return SCALIFY_ERR_SHAPE;
+    a.P_dump = P_dump->data;
+  }
+  a.Q = Q->data; a.K = K->data; a.V = V->data;
+  a.q_dt = Q->dtype; a.k_dt = K->dtype; a.v_dt = V->dtype;
+  a.O = O->data; a.o_dt = O->dtype;
+  a.heads = static_cast<int>(hq); a.Tq = static_cast<int>(tq); a.Tk = static_cast<int>(tk); a.hd = 64;
+  a.causal = causal ? 1 : 0;
+  a.sm_scale = sm_scale;
+  a.q_scale = Q->scale; a.k_scale = K->scale; a.v_scale = V->scale; a.o_scale = O->scale;
+  a.status = status;
+  return launch_attention(a, static_cast<cudaStream_t>(stream));
+}
+
 static int adam_step_impl(int n_tensors, const scalify_array* grads, scalify_array* m, scalify_array* v,
                           scalify_array* w, const scalify_array* w_cast, float lr, float beta1, float beta2,
                           float eps, int64_t step, void* workspace, size_t workspace_bytes, void* stream) {

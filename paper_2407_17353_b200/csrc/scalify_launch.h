@@ -7,7 +7,12 @@
 
 #include "scalify.h"
 
+struct CUtensorMap_st;
+
 namespace scalify {
+
+int make_byte_map(CUtensorMap_st* map, const void* ptr, uint64_t inner, uint64_t rows, uint64_t batch, uint64_t ld,
+                  uint64_t bs, uint32_t box_inner, uint32_t box_rows);
 
 enum { kModeCast = 0, kModeDynamic = 1, kModeSet = 2 };
 
@@ -79,6 +84,19 @@ struct MxMatmulArgs {
 };
 int launch_mx_matmul(const MxMatmulArgs& a, void* ws, cudaStream_t st);
 size_t mx_sf_bytes(int64_t rows, int64_t K);
+struct AttentionArgs {
+  const void* Q; const void* K; const void* V; int q_dt, k_dt, v_dt;   // FP8 [heads, T, hd] views
+  int64_t q_ld, q_hs, k_ld, k_hs, v_ld, v_hs;                         // row and head strides in elements
+  void* O; int o_dt; int64_t o_ld, o_hs;                              // [heads, Tq, hd], F16 / BF16
+  int heads, Tq, Tk, hd;
+  int causal;
+  float sm_scale;
+  const float* q_scale; const float* k_scale; const float* v_scale; float* o_scale;
+  void* S_dump;  // optional BF16 [heads, Tq, Tk] dense: the scores' data component as rounded
+  void* P_dump;  // optional E4M3 [heads, Tq, Tk] dense: the probabilities as fed to the second matmul
+  uint32_t* status;
+};
+int launch_attention(const AttentionArgs& a, cudaStream_t st);
 int launch_mx_quantize(const void* X, int x_dt, int64_t rows, int64_t K, int64_t ldx, void* data, int elem_dt,
                        uint8_t* sf, const float* x_scale, float* y_scale, uint32_t* status, cudaStream_t st);
 

@@ -1,0 +1,115 @@
+"""GPU parity of the fused attention forward against the oracle's composition of the calls it replaces
+(scaled matmul -> softmax on values -> scaled matmul), stage by stage through the kernel's optional
+copies of the scores and the probabilities:
+  scores   within 1 ulp of BF16 (or the 1e-5 * sum|a*b| accumulation bar) of the oracle's Q K^T,
+  P        within 1 ulp of E4M3 of the oracle's softmax of the kernel's own scores (exactly 0 where masked),
+  O        within 1 ulp (or the accumulation bar) of the oracle's matmul of the kernel's own P with V,
+  O scale  bit-exact (V_s * kf(Tk))."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as orc
+import paper_2407_17353_b200 as sc
+import scalify_inputs as si
+from helpers import to_dev, to_bits, ulp_diff, within
+
+pytestmark = pytest.mark.gpu
+
+HD = 64
+
+
+def run_case(H, Tq, Tk, causal, merged_layout=False, q_dt=orc.E4M3, v_dt=orc.E4M3, o_dt=orc.BF16, seed=1):
+    qs, ks, vs, c = 2.0 ** -1, 2.0 ** 1, 2.0 ** -3, 0.125
+    q = si.to_bits(si.normal(seed, 1, (H, Tq, HD), 1.0), q_dt)
+    k = si.to_bits(si.normal(seed, 2, (H, Tk, HD), 1.0), orc.E4M3)
+    v = si.to_bits(si.normal(seed, 3, (H, Tk, HD), 1.0), v_dt)
+
+    def dev_heads(x, dt, T):
+        if not merged_layout:
+            return to_dev(x, dt)
+        buf = torch.zeros((T, H * HD), dtype=torch.uint8, device="cuda").view(sc.TORCH_DTYPE[dt])
+        view = buf.view(T, H, HD).permute(1, 0, 2)      # [H, T, HD] view of a [T, H*HD] buffer
+        view.copy_(to_dev(x, dt))
+        return view
+    Q = sc.ScaledTensor.make(dev_heads(q, q_dt, Tq), qs)
+    K = sc.ScaledTensor.make(dev_heads(k, orc.E4M3, Tk), ks)
+    V = sc.ScaledTensor.make(dev_heads(v, v_dt, Tk), vs)
+    if merged_layout:
+        obuf = torch.zeros((Tq, H * HD), dtype=sc.TORCH_DTYPE[o_dt], device="cuda")
+        O = sc.ScaledTensor(obuf.view(Tq, H, HD).permute(1, 0, 2), torch.zeros(1, device="cuda"))
+    else:
+        O = sc.ScaledTensor.empty((H, Tq, HD), sc.TORCH_DTYPE[o_dt])
+    Sd = sc.ScaledTensor(torch.zeros((H, Tq, Tk), dtype=torch.bfloat16, device="cuda"), None)
+    Pd = sc.ScaledTensor(torch.zeros((H, Tq, Tk), dtype=torch.uint8, device="cuda").view(torch.float8_e4m3fn), None)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    sc.scalify_scaled_attention(Q, K, V, O, sm_scale=c, causal=causal, S_dump=Sd, P_dump=Pd, status=status)
+    assert int(status.item()) == 0
+    kf_hd, kf_tk = orc.kf(HD), orc.kf(Tk)
+    assert O.scale_value() == vs * kf_tk
+    S_gpu = to_bits(Sd.data, orc.BF16)
+    P_gpu = to_bits(Pd.data, orc.E4M3)
+    O_gpu = to_bits(O.data.contiguous(), o_dt)
+    ii, jj = np.meshgrid(np.arange(Tq), np.arange(Tk), indexing="ij")
+    visible = (jj <= ii + (Tk - Tq)) if causal else np.ones((Tq, Tk), dtype=bool)
+    for h in range(H):
+        # scores
+        So, s_scale, acc, sab = orc.scaled_matmul(q[h], q_dt, qs, k[h], orc.E4M3, ks, orc.BF16, transB=True,
+                                                  want_acc=True)
+        assert s_scale == qs * ks * kf_hd
+        ok = within(S_gpu[h][visible], So[visible], orc.BF16, acc[visible], sab[visible], 1e-5)
+        assert ok.all(), (h, int((~ok).sum()))
+        # probabilities from the kernel's own scores
+        S_in = np.where(visible, S_gpu[h], 0).astype(np.uint16)
+        Po, ps = orc.softmax_fwd(S_in[None], orc.BF16, s_scale * c, causal, orc.E4M3)
+        assert ps == 1.0
+        assert ulp_diff(P_gpu[h][visible], Po[0][visible], orc.E4M3).max() <= 1, h
+        assert np.all(P_gpu[h][~visible] == 0)
+        # output from the kernel's own probabilities
+        Oo, o_scale, oacc, osab = orc.scaled_matmul(P_gpu[h], orc.E4M3, 1.0, v[h], v_dt, vs, o_dt, want_acc=True)
+        assert o_scale == vs * kf_tk
+        ok = within(O_gpu[h], Oo, o_dt, oacc, osab, 1e-5)
+        assert ok.all(), (h, int((~ok).sum()))
+    return O
+
+
+@pytest.mark.parametrize("H,T", [(2, 128), (3, 256), (2, 1024)])
+def test_causal_self_attention(H, T):
+    run_case(H, T, T, True)
+
+
+def test_full_attention_with_more_keys_than_queries():
+    run_case(2, 128, 384, False)
+
+
+def test_ragged_lengths_and_shifted_causal_mask():
+    run_case(2, 200, 224, True)
+
+
+def test_heads_inside_a_token_major_buffer_and_mixed_formats():
+    run_case(4, 256, 256, True, merged_layout=True, q_dt=orc.E5M2, v_dt=orc.E5M2, o_dt=orc.F16)
+
+
+def test_probabilities_sum_to_one_and_without_copies():
+    H, T = 2, 384
+    q = si.to_bits(si.normal(5, 1, (H, T, HD), 1.0), orc.E4M3)
+    k = si.to_bits(si.normal(5, 2, (H, T, HD), 1.0), orc.E4M3)
+    ones = si.to_bits(np.ones((H, T, HD), dtype=np.float32), orc.E4M3)
+    Q, K, V = (sc.ScaledTensor.make(to_dev(x, orc.E4M3), 1.0) for x in (q, k, ones))
+    O = sc.ScaledTensor.empty((H, T, HD), torch.float32)
+    sc.scalify_scaled_attention(Q, K, V, O, sm_scale=0.125, causal=True)
+    # V = 1 everywhere: O values = sum of the (E4M3-rounded) probabilities of each row, about 1
+    vals = O.data.float().cpu().numpy() * O.scale_value()
+    assert np.all(np.abs(vals - 1.0) < 0.08)
+
+
+def test_argument_checks():
+    Q = sc.ScaledTensor.make(torch.zeros((2, 128, 32), dtype=torch.uint8, device="cuda").view(torch.float8_e4m3fn), 1.0)
+    O = sc.ScaledTensor.empty((2, 128, 32), torch.bfloat16)
+    with pytest.raises(sc.ScalifyError):
+        sc.scalify_scaled_attention(Q, Q, Q, O, sm_scale=0.125)   # head dimension 32 is not built
+    Q = sc.ScaledTensor.make(torch.zeros((2, 256, 64), dtype=torch.uint8, device="cuda").view(torch.float8_e4m3fn), 1.0)
+    K = sc.ScaledTensor.make(torch.zeros((2, 128, 64), dtype=torch.uint8, device="cuda").view(torch.float8_e4m3fn), 1.0)
+    O = sc.ScaledTensor.empty((2, 256, 64), torch.bfloat16)
+    with pytest.raises(sc.ScalifyError):
+        sc.scalify_scaled_attention(Q, K, K, O, sm_scale=0.125, causal=True)   # causal with fewer keys than queries
