@@ -499,6 +499,26 @@ def main():
         mx_q_ms, mx_mm_ms = times
         del Xa, Xb, Am, Bm
 
+    # Fused attention forward on the config-5 shape: 8 sequences x 12 heads, 1024 tokens, head dimension 64
+    att_ms = float("nan")
+    ATT_H, ATT_T, ATT_HD = 96, 1024, 64
+    if not args.no_next:
+        Qa, Ka, Va = (sc.ScaledTensor.make(rnd((ATT_H, ATT_T, ATT_HD), torch.float8_e4m3fn, 30 + i), 1.0)
+                      for i in range(3))
+        Oa = sc.ScaledTensor.empty((ATT_H, ATT_T, ATT_HD), torch.bfloat16, dev)
+        for _ in range(3):
+            sc.scalify_scaled_attention(Qa, Ka, Va, Oa, sm_scale=0.125, causal=True)
+        barrier()
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a_iters = max(3, min(K, 20))
+        a0.record()
+        for _ in range(a_iters):
+            sc.scalify_scaled_attention(Qa, Ka, Va, Oa, sm_scale=0.125, causal=True)
+        a1.record()
+        barrier()
+        att_ms = a0.elapsed_time(a1) / a_iters
+        del Qa, Ka, Va, Oa
+
     # ------------------------------------------------------------------ end to end through host buffers
     hY = torch.empty((N_GEMM, N_GEMM), dtype=torch.int8).pin_memory()
     hscale = torch.empty(1, dtype=torch.float32).pin_memory()
@@ -599,6 +619,10 @@ def main():
         {"row": "f3 (next, own loop) block-scaled GEMM 8192^3 (tcgen05 kind::mxf8f6f4.block_scale, two-CTA tiles), "
                 "BF16 out + fused AMAX", "ms": round(float(mx_mm_ms), 4),
          "TFLOP/s": round(flops / (mx_mm_ms * 1e-3) / 1e12, 1)},
+        {"row": "f4 (next, own loop) fused causal attention forward, 96 heads x 1024 tokens x 64 (scores and "
+                "probabilities never leave the chip)", "ms": round(float(att_ms), 4),
+         "TFLOP/s": round(2.0 * ATT_H * ATT_T * ATT_T * ATT_HD / (att_ms * 1e-3) / 1e12, 1),
+         "note": "flop counted for the causal half of Q K^T and P V"},
     ]
     fp8_peak = 2.0 * peaks["bf16_sustained"]
     gemm_tflops = flops / (float(seg_ms[0]) * 1e-3) / 1e12

@@ -13,7 +13,7 @@
 //   warp 4      one thread: TMA loads of Q, K, V tiles (64-byte swizzle) and all tcgen05.mma
 // The softmax is the exact two-sweep form, not an online approximation of it: sweep A runs
 // Q K^T over the key blocks and keeps the row maximum m and the sum l = sum exp(s - m)
-// (rescaled when m grows); sweep B recomputes Q K^T, forms p = exp(s - m) / l, rounds it to
+// (moved to the new maximum whenever a 32-key chunk raises it); sweep B recomputes Q K^T, forms p = exp(s - m) / l, rounds it to
 // E4M3 and accumulates P V in TMEM.  The probabilities are therefore the same normalised values
 // the unfused path quantises, and O needs no rescaling.  Cost: the Q K^T work twice.
 // TMEM: 128 columns of scores + 64 columns of O (256 allocated, so two CTAs share an SM).
@@ -58,6 +58,14 @@ __device__ __forceinline__ uint64_t make_smem_desc_sw64(uint32_t saddr, uint32_t
   d |= 1ull << 46;
   d |= 4ull << 61;
   return d;
+}
+
+// 2^x for x <= 0 (and -inf): the hardware approximation (2 ulp of fp32, results below 2^-126 flush to 0),
+// far finer than the E4M3 probabilities it feeds
+__device__ __forceinline__ float exp2_neg(float x) {
+  float r;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+  return r;
 }
 
 template <int ODT>
@@ -189,16 +197,29 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       if (!mbar_wait(s_full, it & 1, abort_flag)) { timed_out = true; break; }
       tc_fence_after();
       uint32_t acc[32];
-      float bm = -INFINITY;
 #pragma unroll 1
       for (int c = 0; c < kAttK / 32; ++c) {
         tmem_ld32(t_row + c * 32, acc);
         tmem_ld_wait();
+        // one pass per 32-key chunk: chunk maximum, then the running sum is moved to the new maximum
+        float x[32];
+        float cm = -INFINITY;
 #pragma unroll
-        for (int e = 0; e < 32; ++e) bm = fmaxf(bm, score(acc[e], kb * kAttK + c * 32 + e));
+        for (int e = 0; e < 32; ++e) {
+          x[e] = score(acc[e], kb * kAttK + c * 32 + e);
+          cm = fmaxf(cm, x[e]);
+        }
+        const float m_new = fmaxf(m, cm);
+        if (m_new > -INFINITY) {
+          float add = 0.f;
+#pragma unroll
+          for (int e = 0; e < 32; ++e) add += exp2_neg(x[e] - m_new);  // exp2f(-inf) = 0 for masked keys
+          l = l * exp2_neg(m - m_new) + add;                          // and while nothing has been seen yet
+          m = m_new;
+        }
         if (p.S_dump && i < p.Tq) {
           const int j0 = kb * kAttK + c * 32;
-          if (j0 < p.Tk) {  // Tk is a multiple of 32 when a dump is requested
+          if (j0 < p.Tk) {  // Tk is a multiple of 32 when a copy is requested
             float v[32];
 #pragma unroll
             for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(acc[e]) * p.inv_kf_hd;
@@ -209,19 +230,6 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             for (int q = 0; q < 4; ++q) dst[q] = make_uint4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
           }
         }
-      }
-      const float m_new = fmaxf(m, bm);
-      float add = 0.f;
-      if (m_new > -INFINITY) {
-#pragma unroll 1
-        for (int c = 0; c < kAttK / 32; ++c) {
-          tmem_ld32(t_row + c * 32, acc);
-          tmem_ld_wait();
-#pragma unroll
-          for (int e = 0; e < 32; ++e) add += exp2f(score(acc[e], kb * kAttK + c * 32 + e) - m_new);
-        }
-        l = l * exp2f(m - m_new) + add;  // exp2f(-inf) = 0 while nothing has been seen yet
-        m = m_new;
       }
       tc_fence_before();
       __syncwarp();
@@ -241,7 +249,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         tmem_ld_wait();
         float pr[32];
 #pragma unroll
-        for (int e = 0; e < 32; ++e) pr[e] = exp2f(score(acc[e], kb * kAttK + c * 32 + e) - m) * inv_l;
+        for (int e = 0; e < 32; ++e) pr[e] = exp2_neg(score(acc[e], kb * kAttK + c * 32 + e) - m) * inv_l;
         uint32_t o[8];
         encode_vec<SCALIFY_E4M3, 32>(pr, o);
         // row r of the tile: 128 bytes = eight 16-byte pieces, piece index XOR (r % 8) (128-byte swizzle)
