@@ -6,11 +6,13 @@
 //   O = P V              scaled FP8 matmul, static rule:  O_s = V_s kf(Tk),  O_d = acc / kf(Tk)
 // in ONE kernel: neither S nor P ever reaches HBM (unless the caller asks for debug copies).
 //
-// One CTA per (head, block of 128 queries); 160 threads:
-//   warps 0-3   one query row per thread (the TMEM lane of the row): read the score block from
-//               TMEM, softmax arithmetic, write the E4M3 probabilities as the A operand of the
-//               second matmul into shared memory (128-byte swizzle), final read-out of O
-//   warp 4      one thread: TMA loads of Q, K, V tiles (64-byte swizzle) and all tcgen05.mma
+// One CTA per (head, block of 128 queries); 288 threads:
+//   warps 0-7   two threads per query row (the TMEM lane of the row; each takes 64 of a block's 128
+//               keys): read the score block from TMEM, softmax arithmetic, write the E4M3
+//               probabilities as the A operand of the second matmul into shared memory (128-byte
+//               swizzle), final read-out of O; the two partial (maximum, sum) pairs of a row are
+//               combined once, between the sweeps
+//   warp 8      one thread: TMA loads of Q, K, V tiles (64-byte swizzle) and all tcgen05.mma
 // The softmax is the exact two-sweep form, not an online approximation of it: sweep A runs
 // Q K^T over the key blocks and keeps the row maximum m and the sum l = sum exp(s - m)
 // (moved to the new maximum whenever a 32-key chunk raises it); sweep B recomputes Q K^T, forms p = exp(s - m) / l, rounds it to
@@ -29,7 +31,8 @@ namespace scalify {
 constexpr int kAttQ = 128;     // queries per CTA
 constexpr int kAttK = 128;     // keys per block
 constexpr int kAttHd = 64;     // head dimension (bytes per row of Q, K, V)
-constexpr int kAttThreads = 160;
+constexpr int kAttSmWarps = 8;   // softmax warps: two per TMEM lane quarter, each taking half of the key columns
+constexpr int kAttThreads = 32 * (kAttSmWarps + 1);
 constexpr int kAttTmemCols = 256;
 constexpr uint32_t kAttOCol = 128;
 constexpr int kAttTileBytes = kAttK * kAttHd;  // 8 KB: a Q, K or V tile
@@ -99,8 +102,8 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     mbar_init(q_full, 1);
     for (int s = 0; s < 2; ++s) { mbar_init(kv_full + 8 * s, 1); mbar_init(kv_empty + 8 * s, 1); }
     mbar_init(s_full, 1);
-    mbar_init(s_empty, 4);
-    mbar_init(p_full, 4);
+    mbar_init(s_empty, kAttSmWarps);
+    mbar_init(p_full, kAttSmWarps);
     mbar_init(p_empty, 1);
     mbar_init(o_full, 1);
     *abort_flag = 0u;
@@ -111,14 +114,14 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       if (!is_pow2_scale(vs) && p.status) atomicOr(p.status, static_cast<uint32_t>(SCALIFY_DEV_BAD_SCALE));
     }
   }
-  if (warp == 4) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kAttTmemCols);
+  if (warp == kAttSmWarps) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kAttTmemCols);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   bool timed_out = false;
 
-  if (warp == 4) {
+  if (warp == kAttSmWarps) {
     // ------------------------------------------------------------ loads and MMAs (one thread)
     if (lane == 0) {
       asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_q)) : "memory");
@@ -179,17 +182,28 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     }
   } else {
     // ------------------------------------------------------------ softmax rows (one row per thread)
-    const int r = warp * 32 + lane;
+    const int quarter = warp & 3, half = warp >> 2;   // TMEM lane quarter; which 64 of a block's 128 keys
+    const int r = quarter * 32 + lane;
     const int i = q0 + r;                     // query index
     const int lim = p.causal ? min(p.Tk, i + shift + 1) : p.Tk;  // keys [0, lim) are visible
-    const uint32_t t_row = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
+    const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+    constexpr int kChunks = kAttK / 32 / 2;   // 32-key chunks per thread and block
+    const int c_first = half * kChunks;
     float m = -INFINITY, l = 0.f;
     const float sc2 = load_scale(p.q_scale) * load_scale(p.k_scale) * p.sc_const;
     long long dump_row = (static_cast<long long>(head) * p.Tq + i) * p.Tk;
-    // x = data component of the score (rounded to BF16 like the unfused intermediate) in units of log2(e)
-    auto score = [&](uint32_t acc_bits, int j) {
-      const float sd = round_through<SCALIFY_BF16>(__uint_as_float(acc_bits) * p.inv_kf_hd);
-      return j < lim ? sd * sc2 : -INFINITY;
+    // x = data component of the score, rounded to BF16 like the unfused intermediate, in units of log2(e).
+    // Dividing by kf(hd) only shifts the exponent, so it commutes with the rounding and is folded into sc3.
+    const float sc3 = sc2 * p.inv_kf_hd;
+    auto chunk_scores = [&](const uint32_t* acc_bits, int j0, float* x) {
+      if (j0 + 32 <= lim) {  // every key of the chunk is visible to this row
+#pragma unroll
+        for (int e = 0; e < 32; ++e) x[e] = round_through<SCALIFY_BF16>(__uint_as_float(acc_bits[e])) * sc3;
+      } else {
+#pragma unroll
+        for (int e = 0; e < 32; ++e)
+          x[e] = (j0 + e < lim) ? round_through<SCALIFY_BF16>(__uint_as_float(acc_bits[e])) * sc3 : -INFINITY;
+      }
     };
     int it = 0;
     // sweep A: row maximum and sum of exponentials
@@ -198,23 +212,21 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       tc_fence_after();
       uint32_t acc[32];
 #pragma unroll 1
-      for (int c = 0; c < kAttK / 32; ++c) {
+      for (int c = c_first; c < c_first + kChunks; ++c) {
         tmem_ld32(t_row + c * 32, acc);
         tmem_ld_wait();
         // one pass per 32-key chunk: chunk maximum, then the running sum is moved to the new maximum
         float x[32];
-        float cm = -INFINITY;
+        chunk_scores(acc, kb * kAttK + c * 32, x);
+        float cm4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // four independent chains
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          x[e] = score(acc[e], kb * kAttK + c * 32 + e);
-          cm = fmaxf(cm, x[e]);
-        }
-        const float m_new = fmaxf(m, cm);
+        for (int e = 0; e < 32; ++e) cm4[e & 3] = fmaxf(cm4[e & 3], x[e]);
+        const float m_new = fmaxf(m, fmaxf(fmaxf(cm4[0], cm4[1]), fmaxf(cm4[2], cm4[3])));
         if (m_new > -INFINITY) {
-          float add = 0.f;
+          float add4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-          for (int e = 0; e < 32; ++e) add += exp2_neg(x[e] - m_new);  // exp2f(-inf) = 0 for masked keys
-          l = l * exp2_neg(m - m_new) + add;                          // and while nothing has been seen yet
+          for (int e = 0; e < 32; ++e) add4[e & 3] += exp2_neg(x[e] - m_new);  // 2^-inf = 0 for masked keys
+          l = l * exp2_neg(m - m_new) + ((add4[0] + add4[1]) + (add4[2] + add4[3]));  // and while nothing was seen
           m = m_new;
         }
         if (p.S_dump && i < p.Tq) {
@@ -235,6 +247,16 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       __syncwarp();
       if (lane == 0) mbar_arrive(s_empty);
     }
+    // the two threads of a row (one per half of the key columns) combine their maxima and sums
+    float2* part = reinterpret_cast<float2*>(p_tile);  // [2][128], the P tile is not in use yet
+    part[half * kAttQ + r] = make_float2(m, l);
+    asm volatile("bar.sync 1, %0;" ::"n"(32 * kAttSmWarps) : "memory");
+    {
+      const float2 a = part[r], b = part[kAttQ + r];
+      m = fmaxf(a.x, b.x);
+      l = (a.x > -INFINITY ? a.y * exp2_neg(a.x - m) : 0.f) + (b.x > -INFINITY ? b.y * exp2_neg(b.x - m) : 0.f);
+    }
+    asm volatile("bar.sync 1, %0;" ::"n"(32 * kAttSmWarps) : "memory");  // the tile may be overwritten from here on
     const float inv_l = 1.0f / l;
     // sweep B: probabilities -> E4M3 -> shared memory (A operand of P V)
     for (int kb = 0; kb < n_kb && !timed_out; ++kb, ++it) {
@@ -244,12 +266,13 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       if (kb >= 1 && !mbar_wait(p_empty, (kb - 1) & 1, abort_flag)) { timed_out = true; break; }
       uint32_t acc[32];
 #pragma unroll 1
-      for (int c = 0; c < kAttK / 32; ++c) {
+      for (int c = c_first; c < c_first + kChunks; ++c) {
         tmem_ld32(t_row + c * 32, acc);
         tmem_ld_wait();
         float pr[32];
+        chunk_scores(acc, kb * kAttK + c * 32, pr);
 #pragma unroll
-        for (int e = 0; e < 32; ++e) pr[e] = exp2_neg(score(acc[e], kb * kAttK + c * 32 + e) - m) * inv_l;
+        for (int e = 0; e < 32; ++e) pr[e] = exp2_neg(pr[e] - m) * inv_l;
         uint32_t o[8];
         encode_vec<SCALIFY_E4M3, 32>(pr, o);
         // row r of the tile: 128 bytes = eight 16-byte pieces, piece index XOR (r % 8) (128-byte swizzle)
@@ -275,7 +298,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       tc_fence_after();
       constexpr int OSZ = ElemBytes<ODT>::v;
 #pragma unroll 1
-      for (int c = 0; c < kAttHd / 32; ++c) {
+      for (int c = half; c < half + 1; ++c) {
         uint32_t acc[32];
         tmem_ld32(t_row + kAttOCol + c * 32, acc);
         tmem_ld_wait();
@@ -300,7 +323,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   if (timed_out && p.status) atomicOr(p.status, static_cast<uint32_t>(SCALIFY_DEV_TIMEOUT));
   tc_fence_before();
   __syncthreads();
-  if (warp == 4) {
+  if (warp == kAttSmWarps) {
     tc_fence_after();
     tmem_dealloc(tmem_base, kAttTmemCols);
   }
