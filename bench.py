@@ -211,6 +211,12 @@ def run_profile_row(args):
             sc.scalify_mx_quantize(Xb, Bm)
             sc.scalify_mx_matmul(Am, Bm, Y, ws, stat=sc.STAT_AMAX)
         work = {"flop": 2.0 * n ** 3}
+    elif row == "attention":
+        H, T, HD = 96, 1024, 64
+        Qa, Ka, Va = (sc.ScaledTensor.make(rnd((H, T, HD), torch.float8_e4m3fn, 30 + i), 1.0) for i in range(3))
+        Oa = sc.ScaledTensor.empty((H, T, HD), torch.bfloat16, dev)
+        fn = lambda t: sc.scalify_scaled_attention(Qa, Ka, Va, Oa, sm_scale=0.125, causal=True)
+        work = {"flop": 2.0 * H * T * T * HD}
     elif row == "rescale":
         n = 8192 * 8192
         X = sc.ScaledTensor.make(rnd((n,), torch.bfloat16, 1, 37.0), 1.0)
@@ -284,7 +290,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (for ncu launch lists)")
     ap.add_argument("--no-next", action="store_true",
                     help="skip the separately timed next-row variants f1, f2 (for ncu launch lists of the step)")
-    ap.add_argument("--profile-row", default=None, choices=["matmul", "mx", "rescale", "add", "layernorm", "adam"],
+    ap.add_argument("--profile-row", default=None, choices=["matmul", "mx", "attention", "rescale", "add", "layernorm", "adam"],
                     help="run only this row on a reduced, still larger-than-L2 case (for ncu captures)")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -195,14 +195,16 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     // x = data component of the score, rounded to BF16 like the unfused intermediate, in units of log2(e).
     // Dividing by kf(hd) only shifts the exponent, so it commutes with the rounding and is folded into sc3.
     const float sc3 = sc2 * p.inv_kf_hd;
+    // The BF16 rounding is done with integer arithmetic (round to nearest even on the upper 16 bits; the
+    // scores are finite): the conversion unit is shared with exp2 and is this kernel's busiest pipe.
+    auto bf16_rne = [](uint32_t b) { return __uint_as_float((b + 0x7FFFu + ((b >> 16) & 1u)) & 0xFFFF0000u); };
     auto chunk_scores = [&](const uint32_t* acc_bits, int j0, float* x) {
       if (j0 + 32 <= lim) {  // every key of the chunk is visible to this row
 #pragma unroll
-        for (int e = 0; e < 32; ++e) x[e] = round_through<SCALIFY_BF16>(__uint_as_float(acc_bits[e])) * sc3;
+        for (int e = 0; e < 32; ++e) x[e] = bf16_rne(acc_bits[e]) * sc3;
       } else {
 #pragma unroll
-        for (int e = 0; e < 32; ++e)
-          x[e] = (j0 + e < lim) ? round_through<SCALIFY_BF16>(__uint_as_float(acc_bits[e])) * sc3 : -INFINITY;
+        for (int e = 0; e < 32; ++e) x[e] = (j0 + e < lim) ? bf16_rne(acc_bits[e]) * sc3 : -INFINITY;
       }
     };
     int it = 0;
