@@ -19,8 +19,6 @@
 // its own copies in flight, frees its TMEM and returns.
 #include <cuda.h>
 
-#include <atomic>
-
 #include "scalify_common.cuh"
 #include "scalify_launch.h"
 #include "tcgen05_ptx.cuh"
@@ -83,8 +81,13 @@ struct GemmParams {
   float* y_scale;
   int stat;
   const float* stat_in;  // delayed rescale: statistic of an earlier step (device), or NULL
-  unsigned long long* stat_word;  // AMAX: 64-bit atomicMax target: {call generation : fp32 bit pattern}
-  uint32_t generation;   // tag of this call; a later call always overrides an earlier one, so no zeroing is needed
+  // AMAX: every epilogue warp takes an atomicMax of the fp32 bit pattern on a scratch word; the CTA that
+  // draws the last ticket moves the result to the statistic word and leaves scratch and ticket at zero for
+  // the next launch.  Nothing is zeroed from the host and nothing depends on the launch's position in a
+  // sequence, so a recorded launch can be replayed from a CUDA graph.
+  float* stat_word;
+  uint32_t* amax_scratch;
+  uint32_t* ticket;
   double* l2_partials;   // L2: [tiles][4]
   uint32_t* status;
   // MX only: block exponents in tiles of 128 rows x 4 K-blocks (512 B each), tile (r, k) at
@@ -431,17 +434,22 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
       if (p.stat_in) amax_bits = abs_bits(__uint_as_float(amax_bits) * r_prev);  // un-rebalanced, unrounded
       else amax_bits = abs_bits(round_through<OUT>(__uint_as_float(amax_bits)));
       amax_bits = warp_max_u32(amax_bits);
-      // The statistic word is the low half of a 64-bit word whose high half is the generation of the call
-      // that wrote it: an atomicMax of {generation, bits} both resets an older call's value and takes the
-      // maximum within this call, so the word never has to be zeroed in-stream before the launch.
-      if (lane == 0 && (amax_bits != 0u || (blockIdx.x == 0 && warp == 2)))
-        atomicMax(p.stat_word, (static_cast<unsigned long long>(p.generation) << 32) | amax_bits);
+      if (lane == 0 && amax_bits != 0u) atomicMax(p.amax_scratch, amax_bits);
     }
   }
 
   if (timed_out && p.status) atomicOr(p.status, static_cast<uint32_t>(SCALIFY_DEV_TIMEOUT));
   tc_fence_before();
   __syncthreads();
+  if (p.stat == SCALIFY_STAT_AMAX && threadIdx.x == 0) {
+    // publish: the last CTA to get here has everybody's maxima in the scratch word
+    __threadfence();
+    if (atomicAdd(p.ticket, 1u) == gridDim.x - 1) {
+      __threadfence();
+      *p.stat_word = __uint_as_float(atomicExch(p.amax_scratch, 0u));
+      *p.ticket = 0u;
+    }
+  }
   if constexpr (NCTA == 2) cluster_sync_all();  // neither CTA leaves while the other may still touch its memory
   if (warp == 1) {
     tc_fence_after();
@@ -640,12 +648,6 @@ static int launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, co
   return SCALIFY_OK;
 }
 
-// tag of a call that gathers AMAX with the generation-tagged atomicMax (shared by all GEMM forms)
-static uint32_t next_stat_generation() {
-  static std::atomic<uint32_t> next_generation{1};
-  return next_generation.fetch_add(1);
-}
-
 int launch_scaled_matmul(const MatmulArgs& a, void* ws, cudaStream_t st) {
   WsView v = ws_view(ws);
   // two-CTA tiles (256 rows) whenever there is more than one 128-row tile of output
@@ -686,21 +688,15 @@ int launch_scaled_matmul(const MatmulArgs& a, void* ws, cudaStream_t st) {
   p.a_scale = a.a_scale; p.b_scale = a.b_scale; p.y_scale = a.y_scale;
   p.stat = a.stat;
   p.stat_in = a.stat_in;
-  p.stat_word = reinterpret_cast<unsigned long long*>(v.stat);
+  p.stat_word = v.stat;
+  p.amax_scratch = reinterpret_cast<uint32_t*>(v.stat) + 1;
+  p.ticket = v.ticket;
   p.l2_partials = static_cast<double*>(v.area);
   p.status = v.status;
   p.sfa = nullptr;
   p.sfb = nullptr;
   const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n * p.batch;
   if (tiles > (1ll << 30)) return SCALIFY_ERR_SHAPE;
-  p.generation = 0;
-  if (a.stat == SCALIFY_STAT_AMAX) {
-    p.generation = next_stat_generation();
-    if (p.generation == 0) {  // the 32-bit tag wrapped: start over from a zeroed word
-      SCALIFY_CUDA_TRY(cudaMemsetAsync(v.stat, 0, 2 * sizeof(float), st));
-      p.generation = next_stat_generation();
-    }
-  }
   SCALIFY_DISPATCH_DTYPE(a.y_dt, OUT, {
     if (ncta == 2) rc = launch_variant<OUT, 2>(map_a, map_b, map_y, p, tiles, st);
     else rc = launch_variant<OUT, 1>(map_a, map_b, map_y, p, tiles, st);
@@ -809,21 +805,15 @@ int launch_mx_matmul(const MxMatmulArgs& a, void* ws, cudaStream_t st) {
   p.a_scale = a.a_scale; p.b_scale = a.b_scale; p.y_scale = a.y_scale;
   p.stat = a.stat;
   p.stat_in = nullptr;
-  p.stat_word = reinterpret_cast<unsigned long long*>(v.stat);
+  p.stat_word = v.stat;
+  p.amax_scratch = reinterpret_cast<uint32_t*>(v.stat) + 1;
+  p.ticket = v.ticket;
   p.l2_partials = static_cast<double*>(v.area);
   p.status = v.status;
   p.sfa = a.sfa;
   p.sfb = a.sfb;
   const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n;
   if (tiles > (1ll << 30)) return SCALIFY_ERR_SHAPE;
-  p.generation = 0;
-  if (a.stat == SCALIFY_STAT_AMAX) {
-    p.generation = next_stat_generation();
-    if (p.generation == 0) {
-      SCALIFY_CUDA_TRY(cudaMemsetAsync(v.stat, 0, 2 * sizeof(float), st));
-      p.generation = next_stat_generation();
-    }
-  }
   SCALIFY_DISPATCH_WIDE(a.y_dt, OUT, {
     if (ncta == 2) rc = launch_mx_variant<OUT, 2>(map_a, map_b, map_y, map_sfa, map_sfb, p, tiles, st);
     else rc = launch_mx_variant<OUT, 1>(map_a, map_b, map_y, map_sfa, map_sfb, p, tiles, st);

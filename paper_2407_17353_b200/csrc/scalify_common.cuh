@@ -16,7 +16,7 @@ namespace scalify {
 // ---------------------------------------------------------------- workspace header
 // byte 0   : uint32 status bits (SCALIFY_DEV_*)
 // byte 16  : fp32 statistic word (bit pattern is also used for atomicMax)
-// byte 20  : generation tag of the matmul call that last wrote the statistic word
+// byte 20  : scratch word of the matmul's fused AMAX (atomicMax target; zero between launches)
 // byte 32  : uint32 ticket of the "last block finishes" reductions (self-resetting)
 // byte 64  : (Adam) not used
 // byte 256 : operation-specific area
