@@ -87,3 +87,107 @@ def test_chain_of_calls_replays_from_a_cuda_graph():
     torch.cuda.synchronize()
     for g, w in zip(outputs(), want[0.25]):
         assert np.array_equal(g, w)
+
+
+def test_training_style_chain_with_state_replays_from_a_cuda_graph():
+    """Calls that carry state from one call to the next (the delayed-rescale statistic, Adam's moments and
+    weights with their scales) plus the backward and support kernels: two eager steps from a saved initial
+    state must equal two replays of one recorded step from the same state."""
+    dev = torch.device("cuda")
+    g = torch.Generator(device=dev).manual_seed(11)
+    rnd = lambda shape, dt, std=1.0: (torch.randn(shape, device=dev, generator=g) * std).to(dt)
+    R, D, V, T = 256, 512, 1000, 64
+    VP = 1008
+    ids = torch.randint(0, V, (R,), device=dev, generator=g, dtype=torch.int64)
+    targets = torch.randint(0, V, (R,), device=dev, generator=g, dtype=torch.int64)
+    wte = sc.ScaledTensor.make(rnd((VP, D), torch.bfloat16, 0.02 * 64), 2.0 ** -6)
+    wpe = sc.ScaledTensor.make(rnd((T, D), torch.bfloat16, 0.02 * 64), 2.0 ** -6)
+    X = sc.ScaledTensor.empty((R, D), torch.bfloat16)
+    gamma = sc.ScaledTensor.make(rnd((D,), torch.bfloat16) * 0.1 + 1.0, 1.0)
+    beta = sc.ScaledTensor.make(rnd((D,), torch.bfloat16, 0.1), 1.0)
+    H8 = sc.ScaledTensor.empty((R, D), torch.float8_e4m3fn)
+    mean = torch.empty(R, dtype=torch.float32, device=dev)
+    rinv = torch.empty(R, dtype=torch.float32, device=dev)
+    W8 = sc.ScaledTensor.make(rnd((VP, D), torch.float8_e4m3fn), 2.0 ** -6)
+    stat_state = torch.full((1,), 2.0, dtype=torch.float32, device=dev)
+    logits = sc.ScaledTensor.empty((R, VP), torch.bfloat16)
+    loss = torch.zeros(1, dtype=torch.float32, device=dev)
+    dlogits = sc.ScaledTensor.empty((R, VP), torch.float8_e5m2)
+    dH = sc.ScaledTensor.empty((R, D), torch.bfloat16)
+    Gx = sc.ScaledTensor.empty((R, D), torch.bfloat16)
+    Ga = sc.ScaledTensor.empty((R, D), torch.bfloat16)
+    act = sc.ScaledTensor.empty((R, D), torch.bfloat16)
+    dX = sc.ScaledTensor.empty((R, D), torch.bfloat16)
+    dXq = sc.ScaledTensor.empty((R, D), torch.float8_e5m2)
+    dgam = sc.ScaledTensor.empty((D,), torch.float32)
+    dbet = sc.ScaledTensor.empty((D,), torch.float32)
+    S = sc.ScaledTensor.make(rnd((4, T, T), torch.bfloat16, 2.0), 0.5)
+    P = sc.ScaledTensor.empty((4, T, T), torch.float8_e4m3fn)
+    dP = sc.ScaledTensor.make(rnd((4, T, T), torch.bfloat16), 2.0 ** -8)
+    dS = sc.ScaledTensor.empty((4, T, T), torch.bfloat16)
+    dwte = sc.ScaledTensor.empty((VP, D), torch.float32)
+    dwpe = sc.ScaledTensor.empty((T, D), torch.float32)
+    n = 4096 + 5
+    ag = sc.ScaledTensor.make(rnd((n,), torch.float8_e5m2), 2.0 ** -12)
+    am = sc.ScaledTensor.make(rnd((n,), torch.float16, 1.6), 2.0 ** -16)
+    av = sc.ScaledTensor.make((rnd((n,), torch.float32) ** 2).to(torch.float16), 2.0 ** -24)
+    aw = sc.ScaledTensor.make(rnd((n,), torch.float16, 1.28), 2.0 ** -6)
+    awc = sc.ScaledTensor.make(torch.zeros(n, dtype=torch.uint8, device=dev).view(torch.float8_e4m3fn), 1.0)
+    adam, wc = sc.AdamTensors([ag], [am], [av], [aw]), [awc]
+    ws_mm = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_MATMUL, R, VP))
+    ws_ln = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_LAYERNORM_BWD, R, D))
+    ws_ce = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_CROSS_ENTROPY, R))
+    ws_ad = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_ADAM, 1))
+    state = [stat_state, am.data, am.scale, av.data, av.scale, aw.data, aw.scale]
+    saved = [x.clone() for x in state]
+
+    def reset():
+        for x, s in zip(state, saved):
+            x.copy_(s)
+
+    def step():
+        sc.scalify_scaled_embedding(ids, T, wte, wpe, X)
+        sc.scalify_scaled_layernorm(X, gamma, beta, H8, eps=1e-5, mean=mean, rinv=rinv)
+        sc.scalify_scaled_matmul_delayed(H8, W8, stat_state, logits, ws_mm, transB=True, stat=sc.STAT_AMAX,
+                                         stat_out=stat_state)
+        sc.scalify_scaled_cross_entropy(logits, V, targets, loss, dlogits, ws_ce)
+        sc.scalify_scaled_matmul(dlogits, W8, dH, ws_mm)
+        sc.scalify_scaled_gelu(X, act)
+        sc.scalify_scaled_gelu_bwd(dH, X, Ga)
+        sc.scalify_scaled_layernorm_bwd(dH, X, gamma, mean, rinv, dX, ws_ln, eps=1e-5, stat_dx=sc.STAT_L2, dXq=dXq,
+                                        dgamma=dgam, dbeta=dbet)
+        sc.scalify_scaled_softmax(S, P, causal=True)
+        sc.scalify_scaled_softmax_bwd(dP, P, dS)
+        sc.scalify_scaled_embedding_bwd(ids, T, dX, dwte, dwpe)
+        sc.scalify_scaled_adam_step_cast(adam, wc, ws_ad, lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, step=3)
+
+    outs = [logits, dlogits, dH, act, Ga, dX, dXq, dgam, dbet, P, dS, am, av, aw, awc]
+    atomics = [dwte, dwpe]   # scatter-adds with fp32 atomics: the order of the addends is not fixed
+
+    def snapshot():
+        torch.cuda.synchronize()
+        return [x.data.contiguous().view(torch.uint8).cpu().numpy().copy() for x in outs] + \
+               [np.array([x.scale_value() for x in outs] + [float(loss.item()), float(stat_state.item())])]
+
+    reset()
+    step()
+    first = snapshot()
+    first_atomics = [x.data.float().cpu().numpy().copy() for x in atomics]
+    step()
+    second = snapshot()
+    assert not np.array_equal(first[-1], second[-1])     # the state did move between the steps
+    reset()
+    stream = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(graph, stream=stream):
+            step()
+    reset()
+    graph.replay()
+    for a, b in zip(snapshot(), first):
+        assert np.array_equal(a, b)
+    for x, w in zip(atomics, first_atomics):
+        assert np.allclose(x.data.float().cpu().numpy(), w, rtol=1e-5, atol=1e-6)
+    graph.replay()
+    for a, b in zip(snapshot(), second):
+        assert np.array_equal(a, b)
