@@ -100,3 +100,40 @@ def test_full_size_step_runs():
     for k, v in model.params.items():
         s = v.scale_value()
         assert s > 0 and np.log2(s) == round(np.log2(s))
+
+
+def test_full_size_step_replays_from_a_cuda_graph():
+    """The whole GPT-2-small-shaped step (about 2000 launches) is recorded once and replayed: starting from
+    the same parameters and optimizer state, a replay gives the loss and the weights of the eager step bit for
+    bit (the embedding gradient, a scatter-add with fp32 atomics, only to rounding)."""
+    cfg = GPTConfig()
+    n = cfg.batch * cfg.seq
+    ids = torch.from_numpy(si.uniform_int(6, 901, (n,), cfg.vocab)).cuda()
+    tgt = torch.from_numpy(si.uniform_int(6, 902, (n,), cfg.vocab)).cuda()
+
+    def fresh():
+        ops = Ops(check=False)
+        return ScaledGPT(cfg, ops, seed=6)
+    eager = fresh()
+    eager.step(ids, tgt, t=1)                 # also does the one-time host work of every kernel
+    loss_eager = float(eager.step(ids, tgt, t=2).item())
+    model = fresh()
+    model.step(ids, tgt, t=1)
+    stream = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(graph, stream=stream):
+            loss = model.step(ids, tgt, t=2)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert float(loss.item()) == loss_eager
+    exact = close = 0
+    for k, v in model.params.items():
+        w = eager.params[k]
+        assert v.scale_value() == w.scale_value(), k
+        if torch.equal(v.data, w.data):
+            exact += 1
+        else:   # tensors that receive the embedding's atomically accumulated gradient
+            assert torch.allclose(v.data.float(), w.data.float(), rtol=2e-3, atol=0), k
+            close += 1
+    assert exact >= len(model.params) - 2, (exact, close)
