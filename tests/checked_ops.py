@@ -230,6 +230,37 @@ class Ops:
             assert P.scale_value() == ps and self.ulp_diff(self.bits(P), po, p_dt).max() <= 1
         return P
 
+    def attention(self, Q, K, V, O, sm_scale, causal=True):
+        """Fused forward over [heads, T, 64] views; returns the E4M3 probabilities (kept for the backward).
+        Checked stage by stage through the kernel's own copies of the scores and probabilities."""
+        H, Tq, _ = Q.data.shape
+        Tk = K.data.shape[1]
+        P = sc.ScaledTensor(torch.zeros((H, Tq, Tk), dtype=torch.uint8, device=Q.data.device).view(torch.float8_e4m3fn),
+                            torch.ones(1, dtype=torch.float32, device=Q.data.device))
+        Sd = None
+        if self.check:
+            Sd = sc.ScaledTensor(torch.zeros((H, Tq, Tk), dtype=torch.bfloat16, device=Q.data.device), None)
+        sc.scalify_scaled_attention(Q, K, V, O, sm_scale=sm_scale, causal=causal, S_dump=Sd, P_dump=P)
+        self.calls += 1
+        if self.check:
+            o = self.orc
+            q_dt, k_dt, v_dt, o_dt = code(Q.data), code(K.data), code(V.data), code(O.data)
+            qb, kb, vb = self.bits(Q), self.bits(K), self.bits(V)
+            Sg, Pg, Og = self.bits(Sd), self.bits(P), self.bits(sc.ScaledTensor(O.data.contiguous(), None))
+            ii, jj = np.meshgrid(np.arange(Tq), np.arange(Tk), indexing="ij")
+            vis = (jj <= ii + (Tk - Tq)) if causal else np.ones((Tq, Tk), dtype=bool)
+            for h in range(H):
+                So, ss, acc, sab = o.scaled_matmul(qb[h], q_dt, Q.scale_value(), kb[h], k_dt, K.scale_value(), BF,
+                                                   transB=True, want_acc=True)
+                assert self.within(Sg[h][vis], So[vis], BF, acc[vis], sab[vis], 1e-5).all()
+                Sin = np.where(vis, Sg[h], 0).astype(np.uint16)
+                Po, ps = o.softmax_fwd(Sin[None], BF, ss * sm_scale, causal, E4)
+                assert self.ulp_diff(Pg[h][vis], Po[0][vis], E4).max() <= 1 and np.all(Pg[h][~vis] == 0)
+                Oo, os_, oacc, osab = o.scaled_matmul(Pg[h], E4, 1.0, vb[h], v_dt, V.scale_value(), o_dt, want_acc=True)
+                assert O.scale_value() == os_
+                assert self.within(Og[h], Oo, o_dt, oacc, osab, 1e-5).all()
+        return P
+
     def softmax_bwd(self, dP, P, o_dt):
         dS = self.empty(P.data.shape, o_dt)
         sc.scalify_scaled_softmax_bwd(dP, P, dS)

@@ -127,13 +127,19 @@ class ScaledGPT:
             s["P8"] = []
             att_scale = None
             for b in range(B):
-                S = o.mm(self._heads(q8, b), self._heads(k8, b), transB=True)        # [H, T, T]
-                o.scalar_mul(S, 1.0 / float(np.sqrt(hd)))                           # 1/sqrt(hd), a power of two here
-                Pb = o.softmax(S, True, E4)
-                s["P8"].append(Pb)
                 Ob = sc.ScaledTensor(self._heads(sc.ScaledTensor(att.data, None), b).data,
                                      torch.empty(1, dtype=torch.float32, device=self.dev))
-                o.mm(Pb, self._heads(v8, b), Y=Ob)                                   # written into the merged layout
+                if hd == 64:
+                    # Q K^T, 1/sqrt(hd), causal softmax and P V in one kernel; the probabilities it used are
+                    # kept for the backward pass
+                    Pb = o.attention(self._heads(q8, b), self._heads(k8, b), self._heads(v8, b), Ob,
+                                     1.0 / float(np.sqrt(hd)))
+                else:
+                    S = o.mm(self._heads(q8, b), self._heads(k8, b), transB=True)    # [H, T, T]
+                    o.scalar_mul(S, 1.0 / float(np.sqrt(hd)))                       # 1/sqrt(hd), a power of two here
+                    Pb = o.softmax(S, True, E4)
+                    o.mm(Pb, self._heads(v8, b), Y=Ob)                               # written into the merged layout
+                s["P8"].append(Pb)
                 att_scale = Ob.scale  # identical for every b: static rule
             att = sc.ScaledTensor(att.data, att_scale)
             s["o8"] = o8 = o.cast(att, E4)
