@@ -157,6 +157,25 @@ int scalify_scaled_matmul(const scalify_array* A, int transA, const scalify_arra
                           void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * scalify_scaled_matmul with stat = AMAX and a rebalanced FP8 output, made cheaper by a PREDICTION of the
+ * statistic (Section 3.3 observes that statistics change slowly, which is what delayed rescaling exploits;
+ * here the result stays that of the exact dynamic rescale).  *stat_hint (DEVICE) holds a predicted
+ * statistic, typically the one this call produced last step.  The GEMM writes the 16-bit intermediate Y
+ * and, in the same epilogue, Yq = fp8(stored Y / r_pred) with r_pred = the hint rounded down to a power of
+ * two (1 if the hint cannot define a scale).  A second, small launch compares r_pred with the power of two
+ * of the TRUE statistic of Y: if they agree (the common case) Yq is already the exact result and only its
+ * scale word is written; if not, Yq is rebuilt from Y as scalify_scaled_matmul would.  Either way Y, Yq,
+ * both scale words and the statistic word are bit-identical to scalify_scaled_matmul(..., AMAX, Yq), and
+ * *stat_hint is overwritten with this call's statistic.  In the common case the separate pass over Y
+ * (2 bytes read + 1 written per element) is replaced by 1 extra written byte per element in the GEMM.
+ *   Y: F16 or BF16, contiguous; Yq: E4M3 or E5M2, contiguous, same shape; other arguments and errors as
+ *   scalify_scaled_matmul; SCALIFY_ERR_NULL if stat_hint or Yq is NULL.
+ */
+int scalify_scaled_matmul_speculative(const scalify_array* A, int transA, const scalify_array* B, int transB,
+                                      scalify_array* Y, scalify_array* Yq, float* stat_hint, void* workspace,
+                                      size_t workspace_bytes, void* stream);
+
+/*
  * Scaled matrix multiply with DELAYED rescaling (Section 3.3: "Delayed rescaling can be
  * similarly implemented by decoupling the compute of statistics and rebalancing ..., keeping
  * track of the first one in the model state").  One kernel, no intermediate, no second pass:

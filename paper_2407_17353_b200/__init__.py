@@ -71,6 +71,7 @@ def lib() -> ctypes.CDLL:
         L.scalify_workspace_init.argtypes = [vp, sz, vp]
         L.scalify_check_status.argtypes = [vp, vp]
         L.scalify_scaled_matmul.argtypes = [P, i32, P, i32, P, i32, P, vp, sz, vp]
+        L.scalify_scaled_matmul_speculative.argtypes = [P, i32, P, i32, P, P, vp, vp, sz, vp]
         L.scalify_statistic.argtypes = [P, i32, vp, vp, sz, vp]
         L.scalify_scaled_matmul_delayed.argtypes = [P, i32, P, i32, vp, P, i32, vp, vp, sz, vp]
         L.scalify_rescale.argtypes = [P, i32, vp, vp, P, vp, sz, vp]
@@ -101,7 +102,8 @@ def lib() -> ctypes.CDLL:
                      "scalify_scaled_adam_step", "scalify_scaled_adam_step_cast", "scalify_scaled_adam_step_static", "scalify_scaled_embedding",
                      "scalify_scaled_embedding_bwd", "scalify_scaled_softmax", "scalify_scaled_softmax_bwd",
                      "scalify_scaled_cross_entropy", "scalify_scalar_mul_pow2", "scalify_debug_expire_wait",
-                     "scalify_mx_quantize", "scalify_mx_matmul", "scalify_scaled_attention"):
+                     "scalify_mx_quantize", "scalify_mx_matmul", "scalify_scaled_attention",
+                     "scalify_scaled_matmul_speculative"):
             getattr(L, name).restype = i32
         _lib = L
     return _lib
@@ -212,6 +214,17 @@ def scalify_scaled_matmul(A: ScaledTensor, B: ScaledTensor, Y: ScaledTensor, ws:
     a, b, y, yq = _desc(A), _desc(B), _desc(Y), _desc(Yq)
     _check(lib().scalify_scaled_matmul(_ref(a), int(transA), _ref(b), int(transB), _ref(y), stat, _ref(yq),
                                        ws.ptr, ws.nbytes, _stream(stream)), "scalify_scaled_matmul")
+
+
+def scalify_scaled_matmul_speculative(A: ScaledTensor, B: ScaledTensor, Y: ScaledTensor, Yq: ScaledTensor,
+                                      stat_hint: torch.Tensor, ws: Workspace, *, transA=False, transB=False,
+                                      stream=None) -> None:
+    """GEMM + exact AMAX rescale to FP8 where the GEMM already writes Yq with a predicted factor (stat_hint: a
+    1-element fp32 CUDA tensor, read as the prediction and overwritten with this call's statistic)."""
+    a, b, y, yq = _desc(A), _desc(B), _desc(Y), _desc(Yq)
+    _check(lib().scalify_scaled_matmul_speculative(_ref(a), int(transA), _ref(b), int(transB), _ref(y), _ref(yq),
+                                                   _ptr(stat_hint), ws.ptr, ws.nbytes, _stream(stream)),
+           "scalify_scaled_matmul_speculative")
 
 
 def scalify_scaled_matmul_delayed(A: ScaledTensor, B: ScaledTensor, stat_in: torch.Tensor, Y: ScaledTensor,

@@ -244,6 +244,83 @@ int launch_rebalance(const void* x, int in_dt, void* y, int out_dt, int64_t n, c
 }
 
 // ---------------------------------------------------------------------------------------------
+// check of a speculative rescale (Section 3.3: dynamic rescale; the producer already wrote the
+// rebalanced array with a PREDICTED power of two)
+// ---------------------------------------------------------------------------------------------
+// If the power of two of the true statistic equals the predicted one, y already holds the exact
+// result and only the scale word is written; otherwise the array is rebalanced from x as usual.
+template <int IN, int OUT>
+__global__ void __launch_bounds__(kThreads) rebalance_check_kernel(const void* __restrict__ x, void* __restrict__ y,
+                                                                   int64_t n, const float* x_scale, float* y_scale,
+                                                                   const float* stat, const float* r_pred,
+                                                                   float* hint_out, uint32_t* status) {
+  constexpr int VEC = VecElems<IN, OUT>::v;
+  constexpr int IB = VEC * ElemBytes<IN>::v, OB = VEC * ElemBytes<OUT>::v;
+  const float xs = load_scale(x_scale);
+  const float s = __ldg(stat);
+  bool nonfinite;
+  const float r = rescale_factor(s, &nonfinite);
+  const float rp = __ldg(r_pred);
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    uint32_t flags = is_pow2_scale(xs) ? 0u : SCALIFY_DEV_BAD_SCALE;
+    if (nonfinite) flags |= SCALIFY_DEV_NONFINITE_STAT;
+    if (y_scale) *y_scale = xs * r;
+    if (hint_out) *hint_out = s;  // the prediction for the next call
+    if (flags && status) atomicOr(status, flags);
+  }
+  if (r == rp) return;
+  const float factor = 1.0f / r;  // exact: r is a power of two
+  const int64_t n_vec = n / VEC;
+  const int64_t n_tiles = (n_vec + kThreads * kUnroll - 1) / (kThreads * kUnroll);
+  for (int64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+    const int64_t base = tile * (kThreads * kUnroll);
+    uint32_t w[kUnroll][IB / 4];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      int64_t i = base + u * kThreads + threadIdx.x;
+      if (i < n_vec) ld_raw_stream<IB>(static_cast<const char*>(x) + i * IB, w[u]);
+    }
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      int64_t i = base + u * kThreads + threadIdx.x;
+      if (i < n_vec) {
+        float f[VEC];
+        decode_vec<IN, VEC>(w[u], f);
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) f[e] *= factor;
+        uint32_t o[OB / 4];
+        encode_vec<OUT, VEC>(f, o);
+        st_raw<OB>(static_cast<char*>(y) + i * OB, o);
+      }
+    }
+  }
+  if (blockIdx.x == 0) {
+    const int tail = static_cast<int>(n - n_vec * VEC);
+    if (threadIdx.x < tail) {
+      int64_t i = n_vec * VEC + threadIdx.x;
+      store_elem<OUT>(y, i, load_elem<IN>(x, i) * factor);
+    }
+  }
+}
+
+int launch_rebalance_check(const void* x, int in_dt, void* y, int out_dt, int64_t n, const float* x_scale,
+                           float* y_scale, const float* stat, const float* r_pred, float* hint_out,
+                           uint32_t* status, cudaStream_t st) {
+  const int64_t n_vec = n / (16 / 2);
+  const int grid = grid_for(n_vec, 8);  // small grid: in the expected case every block returns at once
+#define SCALIFY_RBC(IN, OUT) \
+  rebalance_check_kernel<IN, OUT><<<grid, kThreads, 0, st>>>(x, y, n, x_scale, y_scale, stat, r_pred, hint_out, status)
+  if (in_dt == SCALIFY_BF16) {
+    if (out_dt == SCALIFY_E4M3) SCALIFY_RBC(SCALIFY_BF16, SCALIFY_E4M3); else SCALIFY_RBC(SCALIFY_BF16, SCALIFY_E5M2);
+  } else {
+    if (out_dt == SCALIFY_E4M3) SCALIFY_RBC(SCALIFY_F16, SCALIFY_E4M3); else SCALIFY_RBC(SCALIFY_F16, SCALIFY_E5M2);
+  }
+#undef SCALIFY_RBC
+  SCALIFY_CUDA_TRY(cudaGetLastError());
+  return SCALIFY_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
 // dynamic rescale in one cooperative launch (Section 3.3): statistic, grid barrier, rebalance
 // ---------------------------------------------------------------------------------------------
 // Every block owns one contiguous run of vectors.  Phase 1 reads the run front to back with the

@@ -90,6 +90,11 @@ struct GemmParams {
   uint32_t* ticket;
   double* l2_partials;   // L2: [tiles][4]
   uint32_t* status;
+  // Speculative rescale (SPEC kernels): besides Y, the epilogue writes Yq = fp8(stored Y / r_pred) with
+  // r_pred = p2_floor(*stat_hint); a later check compares r_pred with the power of two of the true statistic.
+  const float* stat_hint;
+  int q_dt;          // SCALIFY_E4M3 or SCALIFY_E5M2
+  float* r_pred_out; // the r_pred this launch used (read by the check kernel)
   // MX only: block exponents in tiles of 128 rows x 4 K-blocks (512 B each), tile (r, k) at
   // ((r * K/128) + k) * 512, byte (row % 32) * 16 + (row / 32 % 4) * 4 + (block % 4)
   const uint8_t* sfa;
@@ -109,9 +114,12 @@ __device__ __forceinline__ void tile_coords(const GemmParams& p, int tile, int& 
   nt = r / gm;
 }
 
-template <int OUT, int NCTA, bool MX>
+// map_sfa is the exponent map of A in the block-scaled form and the map of the speculative FP8 output in the
+// SPEC form (the two never occur together).
+template <int OUT, int NCTA, bool MX, bool SPEC = false>
 __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_y,
                                           const CUtensorMap& map_sfa, const CUtensorMap& map_sfb, const GemmParams& p) {
+  static_assert(!SPEC || (!MX && ElemBytes<OUT>::v == 2), "speculative FP8 output: per-tensor kernel, 16-bit Y");
   using C = GemmCfg<NCTA, MX>;
   constexpr int kStages = C::kStages;
   constexpr int kAcc = C::kAcc;
@@ -154,6 +162,10 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
       bool nf = false;
       if (p.stat_in) r = rescale_factor(__ldg(p.stat_in), &nf);
       if (p.y_scale) *p.y_scale = load_scale(p.a_scale) * load_scale(p.b_scale) * p.kf * r;
+      if constexpr (SPEC) {
+        bool nf2;
+        *p.r_pred_out = rescale_factor(__ldg(p.stat_hint), &nf2);
+      }
       if (nf && p.status) atomicOr(p.status, static_cast<uint32_t>(SCALIFY_DEV_NONFINITE_STAT));
     }
     if (blockIdx.x == 0 && p.status) {
@@ -341,7 +353,10 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
       // One 32-column chunk of this thread's row in two steps: scale + statistic + round (convert), then store.
       constexpr int CPR = 32 * OSZ / 16;              // 16-byte pieces per row: 2 (FP8), 4 (16-bit), 8 (F32)
       constexpr int kTileBytes = 32 * 32 * OSZ;
-      constexpr int NBUF = C::kEpiWarpBytes / kTileBytes > 4 ? 4 : C::kEpiWarpBytes / kTileBytes;  // 4, 4 or 2
+      // staging tiles per warp: 4, 4 or 2; with the speculative output 2 of Y (4 KB) and 2 FP8 tiles behind them
+      constexpr int NBUF = SPEC ? 2 : (C::kEpiWarpBytes / kTileBytes > 4 ? 4 : C::kEpiWarpBytes / kTileBytes);
+      float inv_r_pred = 1.0f;
+      if constexpr (SPEC) { bool nf2; inv_r_pred = 1.0f / rescale_factor(__ldg(p.stat_hint), &nf2); }
       auto convert = [&](const uint32_t* acc_regs, uint32_t* o) {
         float v[32];
 #pragma unroll
@@ -358,6 +373,15 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
         }
         encode_vec<OUT, 32>(v, o);
       };
+      // speculative FP8 copy of a chunk: the STORED 16-bit values divided by the predicted power of two
+      auto convert_q = [&](const uint32_t* o, uint32_t* oq) {
+        float vr[32];
+        decode_vec<OUT, 32>(o, vr);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) vr[i] *= inv_r_pred;
+        if (p.q_dt == SCALIFY_E4M3) encode_vec<SCALIFY_E4M3, 32>(vr, oq);
+        else encode_vec<SCALIFY_E5M2, 32>(vr, oq);
+      };
       // Each lane holds 32 consecutive columns of ONE row.  The warp writes the chunk (32 rows x 32 columns)
       // into a shared-memory tile in the swizzle pattern TMA uses for rows of this width, and one lane hands
       // the tile to a TMA store, which writes whole row segments and clips rows >= M and columns >= N.
@@ -370,10 +394,20 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
 #pragma unroll
         for (int j = 0; j < CPR; ++j)
           tile[lane * CPR + (j ^ ((lane / (8 / CPR)) % CPR))] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+        uint8_t* tile_q = epi_mem + (warp - 2) * C::kEpiWarpBytes + 4096 + (c % NBUF) * 1024;
+        if constexpr (SPEC) {
+          uint32_t oq[8];
+          convert_q(o, oq);
+          uint4* tq = reinterpret_cast<uint4*>(tile_q);  // 32 rows x 32 B, 32-byte swizzle: piece XOR (row / 4) % 2
+          tq[lane * 2 + (0 ^ ((lane >> 2) & 1))] = make_uint4(oq[0], oq[1], oq[2], oq[3]);
+          tq[lane * 2 + (1 ^ ((lane >> 2) & 1))] = make_uint4(oq[4], oq[5], oq[6], oq[7]);
+        }
         fence_async_smem();
         __syncwarp();
         if (lane == 0) {
-          tma_store_3d(&map_y, smem_u32(tile_b), col0, mt * C::kTileM + static_cast<int>(rank) * kBM + q * 32, b);
+          const int row0 = mt * C::kTileM + static_cast<int>(rank) * kBM + q * 32;
+          tma_store_3d(&map_y, smem_u32(tile_b), col0, row0, b);
+          if constexpr (SPEC) tma_store_3d(&map_sfa, smem_u32(tile_q), col0, row0, b);
           bulk_commit();
         }
       };
@@ -462,6 +496,15 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
 scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                      const __grid_constant__ CUtensorMap map_y, const GemmParams p) {
   gemm_body<OUT, NCTA, false>(map_a, map_b, map_y, map_a, map_a, p);
+}
+
+// The same kernel that also writes the FP8 output quantised with a PREDICTED rescale factor.
+template <int OUT, int NCTA>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+scaled_matmul_spec_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                          const __grid_constant__ CUtensorMap map_y, const __grid_constant__ CUtensorMap map_q,
+                          const GemmParams p) {
+  gemm_body<OUT, NCTA, false, true>(map_a, map_b, map_y, map_q, map_q, p);
 }
 
 // Block-scaled operands (E8M0 exponent per 32 elements of K), K-major A [M,K] and B [N,K].
@@ -600,12 +643,21 @@ size_t matmul_ws_bytes(int64_t rows, int64_t cols) {
   return kWsHeader + size_t(tiles) * 8 * sizeof(double) + 256;
 }
 
+template <int OUT, int NCTA, bool SPEC>
+struct GemmKernelOf {
+  static auto get() { return scaled_matmul_kernel<OUT, NCTA>; }
+};
 template <int OUT, int NCTA>
+struct GemmKernelOf<OUT, NCTA, true> {
+  static auto get() { return scaled_matmul_spec_kernel<OUT, NCTA>; }
+};
+
+template <int OUT, int NCTA, bool SPEC = false>
 static int launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_y,
-                          const GemmParams& p, long long tiles,
+                          const CUtensorMap& map_q, const GemmParams& p, long long tiles,
                           cudaStream_t st) {
   using C = GemmCfg<NCTA>;
-  auto kernel = scaled_matmul_kernel<OUT, NCTA>;
+  auto kernel = GemmKernelOf<OUT, NCTA, SPEC>::get();
   static bool attr_done = false;
   static int max_clusters = 0;
   if (!attr_done) {
@@ -644,7 +696,8 @@ static int launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, co
   cfg.blockDim = dim3(kGemmThreads);
   cfg.dynamicSmemBytes = C::kSmem;
   cfg.stream = st;
-  SCALIFY_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, map_a, map_b, map_y, p));
+  if constexpr (SPEC) SCALIFY_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, map_a, map_b, map_y, map_q, p));
+  else SCALIFY_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, map_a, map_b, map_y, p));
   return SCALIFY_OK;
 }
 
@@ -695,12 +748,29 @@ int launch_scaled_matmul(const MatmulArgs& a, void* ws, cudaStream_t st) {
   p.status = v.status;
   p.sfa = nullptr;
   p.sfb = nullptr;
+  p.stat_hint = a.stat_hint;
+  p.q_dt = a.q_dt;
+  p.r_pred_out = reinterpret_cast<float*>(static_cast<char*>(ws) + 52);  // header word read by the check kernel
   const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n * p.batch;
   if (tiles > (1ll << 30)) return SCALIFY_ERR_SHAPE;
-  SCALIFY_DISPATCH_DTYPE(a.y_dt, OUT, {
-    if (ncta == 2) rc = launch_variant<OUT, 2>(map_a, map_b, map_y, p, tiles, st);
-    else rc = launch_variant<OUT, 1>(map_a, map_b, map_y, p, tiles, st);
-  });
+  if (a.stat_hint) {
+    // speculative FP8 output next to the 16-bit intermediate
+    CUtensorMap map_q;
+    rc = make_map_y(&map_q, a.Yq, 1, a.N, a.M, a.batch, a.ldy, a.y_bs);
+    if (rc) return rc;
+    if (a.y_dt == SCALIFY_BF16) {
+      if (ncta == 2) rc = launch_variant<SCALIFY_BF16, 2, true>(map_a, map_b, map_y, map_q, p, tiles, st);
+      else rc = launch_variant<SCALIFY_BF16, 1, true>(map_a, map_b, map_y, map_q, p, tiles, st);
+    } else {
+      if (ncta == 2) rc = launch_variant<SCALIFY_F16, 2, true>(map_a, map_b, map_y, map_q, p, tiles, st);
+      else rc = launch_variant<SCALIFY_F16, 1, true>(map_a, map_b, map_y, map_q, p, tiles, st);
+    }
+  } else {
+    SCALIFY_DISPATCH_DTYPE(a.y_dt, OUT, {
+      if (ncta == 2) rc = launch_variant<OUT, 2>(map_a, map_b, map_y, map_a, p, tiles, st);
+      else rc = launch_variant<OUT, 1>(map_a, map_b, map_y, map_a, p, tiles, st);
+    });
+  }
   if (rc) return rc;
   if (a.stat == SCALIFY_STAT_L2) {
     gemm_l2_finalize_kernel<<<1, 256, 0, st>>>(p.l2_partials, static_cast<int>(tiles * ncta * 8),
@@ -812,6 +882,9 @@ int launch_mx_matmul(const MxMatmulArgs& a, void* ws, cudaStream_t st) {
   p.status = v.status;
   p.sfa = a.sfa;
   p.sfb = a.sfb;
+  p.stat_hint = nullptr;
+  p.q_dt = SCALIFY_E4M3;
+  p.r_pred_out = nullptr;
   const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n;
   if (tiles > (1ll << 30)) return SCALIFY_ERR_SHAPE;
   SCALIFY_DISPATCH_WIDE(a.y_dt, OUT, {

@@ -528,8 +528,9 @@ int scalify_scaled_adam_step_cast(int n_tensors, const scalify_array* grads, sca
                         stream);
 }
 
-int scalify_scaled_matmul(const scalify_array* A, int transA, const scalify_array* B, int transB, scalify_array* Y,
-                          int stat, scalify_array* Yq, void* workspace, size_t workspace_bytes, void* stream) {
+static int matmul_impl(const scalify_array* A, int transA, const scalify_array* B, int transB, scalify_array* Y,
+                       int stat, scalify_array* Yq, float* stat_hint, void* workspace, size_t workspace_bytes,
+                       void* stream) {
   int rc = check_array(A);
   if (rc) return rc;
   rc = check_array(B);
@@ -576,15 +577,44 @@ int scalify_scaled_matmul(const scalify_array* A, int transA, const scalify_arra
   a.stat = stat;
   a.stat_in = nullptr;
   a.force_ncta = 0;
+  a.stat_hint = nullptr;
+  a.Yq = nullptr;
+  a.q_dt = SCALIFY_E4M3;
+  if (stat_hint) {
+    // speculative rescale: 16-bit intermediate, FP8 result, AMAX (the statistic the GEMM gathers exactly)
+    if (!Yq || stat != SCALIFY_STAT_AMAX) return SCALIFY_ERR_VALUE;
+    if (!(Y->dtype == SCALIFY_BF16 || Y->dtype == SCALIFY_F16) || !is_fp8(Yq->dtype)) return SCALIFY_ERR_DTYPE;
+    if (Yq->data == Y->data) return SCALIFY_ERR_ALIAS;
+    a.stat_hint = stat_hint;
+    a.Yq = Yq->data;
+    a.q_dt = Yq->dtype;
+  }
   if (a.lda < (transA ? M : K) || a.ldb < (transB ? K : N) || a.ldy < N) return SCALIFY_ERR_SHAPE;
   rc = launch_scaled_matmul(a, workspace, st);
   if (rc) return rc;
   if (Yq) {
     WsView v = ws_view(workspace);
-    rc = launch_rebalance(Y->data, Y->dtype, Yq->data, Yq->dtype, batch * M * N, y_scale, Yq->scale, v.stat, nullptr,
-                          kModeDynamic, v.status, st);
+    if (stat_hint)
+      rc = launch_rebalance_check(Y->data, Y->dtype, Yq->data, Yq->dtype, batch * M * N, y_scale, Yq->scale, v.stat,
+                                  reinterpret_cast<const float*>(static_cast<char*>(workspace) + 52), stat_hint,
+                                  v.status, st);
+    else
+      rc = launch_rebalance(Y->data, Y->dtype, Yq->data, Yq->dtype, batch * M * N, y_scale, Yq->scale, v.stat, nullptr,
+                            kModeDynamic, v.status, st);
   }
   return rc;
+}
+
+int scalify_scaled_matmul(const scalify_array* A, int transA, const scalify_array* B, int transB, scalify_array* Y,
+                          int stat, scalify_array* Yq, void* workspace, size_t workspace_bytes, void* stream) {
+  return matmul_impl(A, transA, B, transB, Y, stat, Yq, nullptr, workspace, workspace_bytes, stream);
+}
+
+int scalify_scaled_matmul_speculative(const scalify_array* A, int transA, const scalify_array* B, int transB,
+                                      scalify_array* Y, scalify_array* Yq, float* stat_hint, void* workspace,
+                                      size_t workspace_bytes, void* stream) {
+  if (!stat_hint || !Yq) return SCALIFY_ERR_NULL;
+  return matmul_impl(A, transA, B, transB, Y, SCALIFY_STAT_AMAX, Yq, stat_hint, workspace, workspace_bytes, stream);
 }
 
 int scalify_scaled_matmul_delayed(const scalify_array* A, int transA, const scalify_array* B, int transB,
@@ -625,6 +655,9 @@ int scalify_scaled_matmul_delayed(const scalify_array* A, int transA, const scal
   a.stat = stat;
   a.stat_in = stat_in;
   a.force_ncta = 0;
+  a.stat_hint = nullptr;
+  a.Yq = nullptr;
+  a.q_dt = SCALIFY_E4M3;
   if (a.lda < (transA ? M : K) || a.ldb < (transB ? K : N) || a.ldy < N) return SCALIFY_ERR_SHAPE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   rc = launch_scaled_matmul(a, workspace, st);

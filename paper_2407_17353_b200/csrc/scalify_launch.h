@@ -23,6 +23,9 @@ int launch_fused_rescale(const void* x, int in_dt, void* y, int out_dt, int64_t 
                          float* y_scale, void* ws, size_t ws_bytes, cudaStream_t st);
 int launch_rebalance(const void* x, int in_dt, void* y, int out_dt, int64_t n, const float* x_scale, float* y_scale,
                      const float* stat, const float* new_scale, int mode, uint32_t* status, cudaStream_t st);
+int launch_rebalance_check(const void* x, int in_dt, void* y, int out_dt, int64_t n, const float* x_scale,
+                            float* y_scale, const float* stat, const float* r_pred, float* hint_out,
+                            uint32_t* status, cudaStream_t st);
 int launch_scale_word_mul(float* scale, float c, cudaStream_t st);
 int launch_add(const void* a, const void* b, int ab_dt, void* y, int out_dt, int64_t n, int64_t row_len, int broadcast,
                const float* a_scale, const float* b_scale, float* y_scale, int subtract, cudaStream_t st);
@@ -68,6 +71,9 @@ struct MatmulArgs {
   int stat;
   const float* stat_in;  // delayed rescale: earlier statistic (device) or NULL
   int force_ncta;  // 0: choose; 1: force the one-CTA kernel
+  // speculative rescale: predicted statistic (device) or NULL; then Yq (FP8, dense like Y) is written by the GEMM
+  const float* stat_hint;
+  void* Yq; int q_dt;
 };
 size_t matmul_ws_bytes(int64_t rows, int64_t cols);
 int launch_expire_wait(void* ws, unsigned long long limit_ns, uint32_t* waited_us, cudaStream_t st);

@@ -287,3 +287,33 @@ def test_delayed_rescale_full_size_8192_sampled():
     assert gstat >= np.abs(acc).max() * (1 - 1e-5)
     stored_max = float(torch.from_numpy(got).view(torch.float8_e4m3fn).float().abs().max()) * 4.0
     assert stored_max * (1 - 2.0 ** -4) <= gstat <= stored_max * (1 + 2.0 ** -4)
+
+
+@pytest.mark.parametrize("M,N,K", [(256, 256, 256), (520, 304, 384), (100, 48, 128)])
+@pytest.mark.parametrize("y_dt,q_dt", [(orc.BF16, orc.E4M3), (orc.F16, orc.E5M2)])
+def test_speculative_rescale_is_the_exact_dynamic_rescale(M, N, K, y_dt, q_dt):
+    """Whatever the predicted statistic is (right binade, wrong binade either way, zero, NaN), the intermediate,
+    the FP8 output, both scale words and the statistic equal those of the plain call bit for bit, and the hint
+    leaves as this call's statistic."""
+    A = si.to_bits(si.normal(81, M + K, (M, K), 1.0), orc.E4M3)
+    B = si.to_bits(si.normal(82, N + K, (N, K), 1.0), orc.E5M2)
+    plain = run_matmul(A, orc.E4M3, 2.0 ** -2, B, orc.E5M2, 2.0 ** 3, y_dt, transB=True, stat=sc.STAT_AMAX, q_dt=q_dt)
+    assert plain["status"] == 0
+    stat = plain["stat"]
+    # the plain path itself against the oracle's rescale of its own intermediate
+    qo, qs, _ = orc.rescale(plain["Y"].reshape(-1), y_dt, plain["y_scale"], orc.STAT_AMAX, q_dt)
+    assert plain["yq_scale"] == qs and np.array_equal(plain["Yq"].reshape(-1), qo)
+    Ad = sc.ScaledTensor.make(to_dev(A, orc.E4M3), 2.0 ** -2)
+    Bd = sc.ScaledTensor.make(to_dev(B, orc.E5M2), 2.0 ** 3)
+    ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_MATMUL, M, N))
+    for hint in (stat, stat * 1.3, stat / 1.3, stat * 64.0, stat / 1000.0, 0.0, float("nan"), float("inf")):
+        Y = sc.ScaledTensor.empty((M, N), sc.TORCH_DTYPE[y_dt])
+        Yq = sc.ScaledTensor.empty((M, N), sc.TORCH_DTYPE[q_dt])
+        Yq.data.view(torch.uint8).fill_(0x55)
+        h = torch.tensor([hint], dtype=torch.float32, device="cuda")
+        sc.scalify_scaled_matmul_speculative(Ad, Bd, Y, Yq, h, ws, transB=True)
+        assert ws.check_status() == 0
+        assert float(h.item()) == stat and float(ws.statistic().item()) == stat
+        assert Y.scale_value() == plain["y_scale"] and Yq.scale_value() == plain["yq_scale"]
+        assert np.array_equal(to_bits(Y.data, y_dt), plain["Y"])
+        assert np.array_equal(to_bits(Yq.data, q_dt), plain["Yq"]), hint
