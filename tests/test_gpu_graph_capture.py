@@ -22,6 +22,8 @@ def build_chain(seed_scale):
     B = sc.ScaledTensor.make(t["b"].to(torch.float8_e4m3fn), 2.0 ** -6)
     Y = sc.ScaledTensor.empty((M, N), torch.bfloat16)
     Yq = sc.ScaledTensor.empty((M, N), torch.float8_e4m3fn)
+    Yq2 = sc.ScaledTensor.empty((M, N), torch.float8_e4m3fn)
+    hint = torch.zeros(1, dtype=torch.float32, device=dev)   # carries over from call to call, whatever its value
     R = sc.ScaledTensor.make(torch.randn((M, N), device=dev, generator=g).to(torch.bfloat16), 1.0)
     S = sc.ScaledTensor.empty((M, N), torch.bfloat16)
     S8 = sc.ScaledTensor.empty((M, N), torch.float8_e4m3fn)
@@ -42,6 +44,7 @@ def build_chain(seed_scale):
 
     def chain():
         sc.scalify_scaled_matmul(A, B, Y, ws_mm, transB=True, stat=sc.STAT_AMAX, Yq=Yq)   # GEMM + pass 2
+        sc.scalify_scaled_matmul_speculative(A, B, Y, Yq2, hint, ws_mm, transB=True)       # predicted rescale
         sc.scalify_scaled_add(Y, R, S)
         sc.scalify_rescale(S, S8, stat=sc.STAT_AMAX, ws=ws_rs)                             # one-launch rescale
         sc.scalify_scaled_layernorm(S, gamma, beta, L, eps=1e-5, mean=mean, rinv=rinv)
@@ -50,8 +53,8 @@ def build_chain(seed_scale):
         sc.scalify_mx_matmul(Am, Bm, Y2, ws_mm)
         sc.scalify_scaled_attention(heads(L), heads(S8), heads(Yq), O, sm_scale=0.125, causal=True)
 
-    outputs = lambda: [x.data.contiguous().view(torch.uint8).cpu().numpy().copy() for x in (Yq, S8, L, Y2, O)] + \
-                      [np.array([x.scale_value() for x in (Yq, S8, L, Y2, O)])]
+    outputs = lambda: [x.data.contiguous().view(torch.uint8).cpu().numpy().copy() for x in (Yq, Yq2, S8, L, Y2, O)] + \
+                      [np.array([x.scale_value() for x in (Yq, Yq2, S8, L, Y2, O)])]
     return A, t, chain, outputs
 
 
