@@ -142,9 +142,23 @@ __global__ void __launch_bounds__(kLnThreads) layernorm_fwd_kernel(
     cp_async_commit();  // one group per row, even when empty, so that the group count stays uniform
   };
   const int first_row = blockIdx.x * (TPB * rows_per_team) + team;
+  // gamma and beta go through shared memory once per block (all teams of a block use the same columns): the
+  // whole block copies them as the oldest cp.async group, then the first rows follow
+  uint4* gb_stage = ln_stage + kLnFwdStages * VPT * kLnThreads;  // [gamma | beta], raw bytes
+  const int gb_bytes = d * (gb_dt == SCALIFY_F32 ? 4 : 2);
+  if (gamma) {
+    for (int idx = threadIdx.x; idx < gb_bytes / 16; idx += kLnThreads) {
+      cp_async16(&gb_stage[idx], static_cast<const char*>(gamma) + idx * 16);
+      if (beta) cp_async16(&gb_stage[gb_bytes / 16 + idx], static_cast<const char*>(beta) + idx * 16);
+    }
+  }
+  cp_async_commit();
 #pragma unroll
   for (int st = 0; st < kLnFwdStages; ++st) issue(first_row + st * rows_per_iter, st);
-  // gamma and beta of this thread's columns, requested after the first rows so that both are in flight together
+  cp_async_wait<kLnFwdStages>();  // the parameter group has landed (this thread's part) ...
+  __syncthreads();                // ... and everybody else's
+  const void* gamma_s = gb_stage;
+  const void* beta_s = reinterpret_cast<const char*>(gb_stage) + gb_bytes;
   float gam[VPT][VEC], bet[VPT][VEC];
 #pragma unroll
   for (int v = 0; v < VPT; ++v) {
@@ -152,9 +166,9 @@ __global__ void __launch_bounds__(kLnThreads) layernorm_fwd_kernel(
 #pragma unroll
     for (int e = 0; e < VEC; ++e) { gam[v][e] = 1.0f; bet[v][e] = 0.0f; }
     if (has[v] && gamma) {
-      load_param_vec<VEC>(gamma, gb_dt, vi * VEC, gam[v]);
+      load_param_vec<VEC>(gamma_s, gb_dt, vi * VEC, gam[v]);
       if (beta) {
-        load_param_vec<VEC>(beta, gb_dt, vi * VEC, bet[v]);
+        load_param_vec<VEC>(beta_s, gb_dt, vi * VEC, bet[v]);
 #pragma unroll
         for (int e = 0; e < VEC; ++e) bet[v][e] *= fb;  // exact: fb is a power of two
       }
@@ -251,11 +265,13 @@ int launch_layernorm_fwd(const void* X, int x_dt, int64_t x_ld, void* Y, int y_d
   const int grid = static_cast<int>((int64_t(R) + tpb * rpt - 1) / (tpb * rpt));
 #define SCALIFY_LN_FWD(W, V)                                                                                   \
   do {                                                                                                         \
-    constexpr int kSmem = kLnFwdStages * V * kLnThreads * 16;                                                  \
-    if (kSmem > 48 * 1024)                                                                                     \
+    /* row staging + gamma and beta (up to 4 bytes per element each) */                                       \
+    constexpr int kSmemMax = kLnFwdStages * V * kLnThreads * 16 + 2 * (32 * W * V * 16 / 2) * 4;               \
+    const int smem_bytes = kLnFwdStages * V * kLnThreads * 16 + 2 * d * 4;                                     \
+    if (kSmemMax > 40 * 1024) /* the kernel also has a little static shared memory */                         \
       SCALIFY_CUDA_TRY(cudaFuncSetAttribute(layernorm_fwd_kernel<XDT, YDT, W, V>,                              \
-                                            cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem));              \
-    layernorm_fwd_kernel<XDT, YDT, W, V><<<grid, kLnThreads, kSmem, st>>>(                                     \
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax));           \
+    layernorm_fwd_kernel<XDT, YDT, W, V><<<grid, kLnThreads, smem_bytes, st>>>(                                     \
         X, x_ld, Y, y_ld, R, d, gamma, beta, gb_dt, gamma_scale, beta_scale, y_scale, eps, eps_inside, mean,   \
         rinv, rpt);                                                                                                \
   } while (0)
