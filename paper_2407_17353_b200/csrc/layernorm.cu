@@ -463,35 +463,45 @@ __global__ void __launch_bounds__(kLnThreads, 2) layernorm_bwd_kernel(
 }
 
 // Combines the per-block partials in a fixed order: dgamma/dbeta columns (scaled by 1/kf(R)), the
-// statistic word, and the propagated scale words.  Block = 32 columns x 32 slices of the block list.
+// statistic word, and the propagated scale words.
 template <int DGDT>
 __global__ void __launch_bounds__(1024) layernorm_bwd_finalize_kernel(
     int nblocks, int R, int d, const float* __restrict__ dgamma_part, const float* __restrict__ dbeta_part,
     const double* __restrict__ stat_part, int stat, float* stat_word, void* __restrict__ dgamma,
     void* __restrict__ dbeta, const float* g_scale, const float* x_scale, const float* gamma_scale,
     float* dx_scale, float* dgamma_scale, float* dbeta_scale, uint32_t* status) {
-  __shared__ float s_a[32][33], s_b[32][33];
+  // block = 8 columns (one 32-byte sector of a partial row) x 128 slices of the block list: 4 x as many
+  // blocks as a 32-column layout, so the partials (a few MB in L2) are read by more SMs at once
+  __shared__ float s_a[128][9], s_b[128][9];
   const float inv_kf = 1.0f / kfactor(R);
-  const int cx = threadIdx.x & 31, slice = threadIdx.x >> 5;
-  const int col = blockIdx.x * 32 + cx;
+  const int pc = threadIdx.x & 7, slice = threadIdx.x >> 3;
+  const int col = blockIdx.x * 8 + pc;
+  const int cx = threadIdx.x & 31, warp = threadIdx.x >> 5;
   if (dgamma_part) {
     float a = 0.f, b = 0.f;
     if (col < d) {
-      for (int i = slice; i < nblocks; i += 32) {
+      for (int i = slice; i < nblocks; i += 128) {
         a += dgamma_part[int64_t(i) * d + col];
         b += dbeta_part[int64_t(i) * d + col];
       }
     }
-    s_a[slice][cx] = a;
-    s_b[slice][cx] = b;
+    s_a[slice][pc] = a;
+    s_b[slice][pc] = b;
     __syncthreads();
+#pragma unroll
+    for (int off = 64; off > 0; off >>= 1) {  // fixed tree over the slices
+      if (slice < off) {
+        s_a[slice][pc] += s_a[slice + off][pc];
+        s_b[slice][pc] += s_b[slice + off][pc];
+      }
+      __syncthreads();
+    }
     if (slice == 0 && col < d) {
-      for (int k = 1; k < 32; ++k) { a += s_a[k][cx]; b += s_b[k][cx]; }
-      store_elem<DGDT>(dgamma, col, a * inv_kf);
-      store_elem<DGDT>(dbeta, col, b * inv_kf);
+      store_elem<DGDT>(dgamma, col, s_a[0][pc] * inv_kf);
+      store_elem<DGDT>(dbeta, col, s_b[0][pc] * inv_kf);
     }
   }
-  if (blockIdx.x == 0 && slice == 1) {
+  if (blockIdx.x == 0 && warp == 1) {
     if (stat != SCALIFY_STAT_NONE) {
       double tot = 0.0;
       for (int i = cx; i < nblocks; i += 32) {
@@ -558,7 +568,7 @@ int launch_layernorm_bwd(const void* G, int64_t g_ld, const void* X, int x_dt, i
   }));
 #undef SCALIFY_LN_BWD
   SCALIFY_CUDA_TRY(cudaGetLastError());
-  const int fgrid = dgamma ? (d + 31) / 32 : 1;
+  const int fgrid = dgamma ? (d + 7) / 8 : 1;
   SCALIFY_DISPATCH_WIDE(dg_dt, DGDT,
       layernorm_bwd_finalize_kernel<DGDT><<<fgrid, 1024, 0, st>>>(grid, R, d, dgp, dbp, st_part, stat, v.stat, dgamma,
                                                                  dbeta, g_scale, x_scale, gamma_scale, dx_scale,
