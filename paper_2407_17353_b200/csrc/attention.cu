@@ -92,7 +92,9 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int head = blockIdx.x / p.q_blocks, qb = blockIdx.x % p.q_blocks;
+  // query blocks in descending order within the launch: with a causal mask the late blocks have the most key
+  // blocks, and starting them first leaves the short ones to fill the end of the launch
+  const int qb = p.q_blocks - 1 - static_cast<int>(blockIdx.x / p.heads), head = blockIdx.x % p.heads;
   const int q0 = qb * kAttQ;
   const int shift = p.Tk - p.Tq;  // causal: query i sees keys j <= i + shift
   int n_kb = (p.Tk + kAttK - 1) / kAttK;
