@@ -2,9 +2,9 @@
 // exponents as in the OCP micro-scaling formats): FP8 elements plus one E8M0 exponent per 32
 // consecutive elements of a row, written in the tile order the block-scaled MMA consumes.
 //
-// HBM-bound: four lanes share a block (8 elements = one 16-byte vector of 16-bit input per lane),
-// the block maximum comes from two shuffles, every lane rounds its 8 elements once and stores
-// 8 bytes, and one lane keeps the exponent byte.
+// HBM-bound: a thread holds 32 bytes of input (16 elements of a 16-bit format: two lanes share a
+// block; 8 fp32 elements: four lanes), the block maximum comes from one or two shuffles, every lane
+// rounds its elements once and stores them, and one lane keeps the exponent byte.
 #include "scalify_common.cuh"
 #include "scalify_launch.h"
 
@@ -12,8 +12,18 @@ namespace scalify {
 
 constexpr int kMxThreads = 256;
 constexpr int kMxBlock = 32;   // elements that share an exponent
-constexpr int kMxLaneElems = 8;
-constexpr int kMxUnroll = 4;   // loads in flight per thread
+constexpr int kMxUnroll = 4;   // loads in flight per thread (32 bytes each)
+
+// 32 bytes that are read once: one 256-bit load where the address allows it
+__device__ __forceinline__ void mx_load32(const void* p, bool aligned32, uint32_t* w) {
+  if (aligned32) {
+    asm volatile("ld.global.cs.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
+                 : "l"(p));
+  } else {
+    ld_raw_stream<32>(p, w);
+  }
+}
 
 // Exponent storage: tiles of 128 rows x 4 blocks (128 elements of K), 512 bytes each, tile (r, k)
 // at ((r * K/128) + k) * 512; inside a tile row `row`, block `blk` sit at byte
@@ -25,42 +35,61 @@ size_t mx_sf_bytes(int64_t rows, int64_t K) {
 }
 
 // One thread block quantises a tile of 128 rows x 128 elements of K: exactly one 512-byte exponent
-// tile, which is assembled in shared memory and written with 16-byte stores.  A warp covers two rows
-// (2 x 16 pieces of 8 elements) per step, the eight warps 16 rows, eight steps the tile; all of a
-// thread's loads of four steps are issued before their first use.
+// tile, which is assembled in shared memory and written with 16-byte stores.  With 16-bit input a
+// warp covers four rows (4 x 8 pieces of 16 elements) per step, the eight warps 32 rows, four steps the
+// tile; with fp32 input half as many.  All of a thread's loads of four steps are issued before their
+// first use.
 template <int IN, int ELEM>
 __global__ void __launch_bounds__(kMxThreads) mx_quantize_kernel(const void* __restrict__ X, int64_t ldx, int64_t rows,
                                                                  int64_t K, void* __restrict__ data,
                                                                  uint8_t* __restrict__ sf, const float* x_scale,
                                                                  float* y_scale, uint32_t* status) {
-  constexpr int IB = kMxLaneElems * ElemBytes<IN>::v;  // 16 (16-bit input) or 32 (fp32 input)
+  constexpr int LE = 32 / ElemBytes<IN>::v;       // elements per thread: 16 or 8
+  constexpr int kPieces = 128 / LE;               // threads per 128-element row segment: 8 or 16
+  constexpr int kLanesPerBlock = kMxBlock / LE;   // 2 or 4
+  constexpr int kRowsPerStep = kMxThreads / kPieces;
+  constexpr int kGroups = 128 / kRowsPerStep / kMxUnroll;
   constexpr int kEmax = ELEM == SCALIFY_E4M3 ? 8 : 15;
   __shared__ __align__(16) uint8_t s_sf[512];
   const int64_t k_tile = blockIdx.x, r_tile = blockIdx.y;
-  const int piece = threadIdx.x & 15;        // 8-element piece of the 128-element row segment
-  const int row_in_step = threadIdx.x >> 4;  // 0..15
-  const int64_t col0 = k_tile * 128 + piece * kMxLaneElems;
+  const int piece = threadIdx.x % kPieces;
+  const int row_in_step = threadIdx.x / kPieces;
+  const int64_t col0 = k_tile * 128 + piece * LE;
+  const bool aligned32 = ((reinterpret_cast<uintptr_t>(X) | static_cast<uintptr_t>(ldx * ElemBytes<IN>::v)) & 31) == 0;
 #pragma unroll
-  for (int half = 0; half < 2; ++half) {
-    uint32_t w[kMxUnroll][IB / 4];
+  for (int g = 0; g < kGroups; ++g) {
+    uint32_t w[kMxUnroll][8];
 #pragma unroll
     for (int u = 0; u < kMxUnroll; ++u) {
-      const int64_t row = r_tile * 128 + (half * kMxUnroll + u) * 16 + row_in_step;
+      const int64_t row = r_tile * 128 + (g * kMxUnroll + u) * kRowsPerStep + row_in_step;
 #pragma unroll
-      for (int q = 0; q < IB / 4; ++q) w[u][q] = 0u;
-      if (row < rows) ld_raw_stream<IB>(static_cast<const char*>(X) + (row * ldx + col0) * ElemBytes<IN>::v, w[u]);
+      for (int q = 0; q < 8; ++q) w[u][q] = 0u;
+      if (row < rows)
+        mx_load32(static_cast<const char*>(X) + (row * ldx + col0) * ElemBytes<IN>::v, aligned32, w[u]);
     }
 #pragma unroll
     for (int u = 0; u < kMxUnroll; ++u) {
-      const int lrow = (half * kMxUnroll + u) * 16 + row_in_step;  // row inside the tile
+      const int lrow = (g * kMxUnroll + u) * kRowsPerStep + row_in_step;  // row inside the tile
       const int64_t row = r_tile * 128 + lrow;
-      float f[kMxLaneElems];
-      decode_vec<IN, kMxLaneElems>(w[u], f);
+      float f[LE];
+      decode_vec<IN, LE>(w[u], f);
       uint32_t amax = 0u;
+      if constexpr (ElemBytes<IN>::v == 2) {
+        // the 15 magnitude bits of a 16-bit float order like the magnitudes: maximum on the packed halves,
+        // widened to the fp32 pattern afterwards (exact)
+        uint32_t m2 = 0u;
 #pragma unroll
-      for (int e = 0; e < kMxLaneElems; ++e) amax = max(amax, abs_bits(f[e]));
-      amax = max(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
-      amax = max(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 2));
+        for (int q = 0; q < 8; ++q) m2 = __vmaxu2(m2, w[u][q] & 0x7FFF7FFFu);
+        amax = max(m2 & 0xFFFFu, m2 >> 16);
+      } else {
+#pragma unroll
+        for (int e = 0; e < LE; ++e) amax = max(amax, abs_bits(f[e]));
+      }
+#pragma unroll
+      for (int m = 1; m < kLanesPerBlock; m <<= 1) amax = max(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, m));
+      if constexpr (IN == SCALIFY_BF16) amax <<= 16;
+      if constexpr (IN == SCALIFY_F16)
+        amax = __float_as_uint(__half2float(__ushort_as_half(static_cast<unsigned short>(amax))));
       // shared exponent: floor(log2(amax)) - emax of the element format; 0 for a block whose maximum is
       // zero, infinite or NaN (abs_bits orders NaN above infinity, so one comparison covers both)
       int e = 0;
@@ -71,17 +100,17 @@ __global__ void __launch_bounds__(kMxThreads) mx_quantize_kernel(const void* __r
         e = max(-127, min(127, e));
       }
       if (row < rows) {
-        // multiply by 2^-e exactly (two steps keep each factor a normal fp32 for every e in [-127, 127])
-        const int h = (-e) / 2;
-        const float s1 = __uint_as_float(static_cast<uint32_t>(h + 127) << 23);
-        const float s2 = __uint_as_float(static_cast<uint32_t>((-e - h) + 127) << 23);
+        // multiply by 2^-e, exactly: 2^-127 is the subnormal 0x00400000, every other factor is normal
+        const uint32_t field = static_cast<uint32_t>(127 - e);
+        const float s = __uint_as_float(field ? field << 23 : 0x00400000u);
 #pragma unroll
-        for (int t = 0; t < kMxLaneElems; ++t) f[t] = f[t] * s1 * s2;
-        uint32_t o[2];
-        encode_vec<ELEM, kMxLaneElems>(f, o);
-        st_raw<8>(static_cast<char*>(data) + row * K + col0, o);
+        for (int t = 0; t < LE; ++t) f[t] *= s;
+        uint32_t o[LE / 4];
+        encode_vec<ELEM, LE>(f, o);
+        st_raw<LE>(static_cast<char*>(data) + row * K + col0, o);
       }
-      if ((piece & 3) == 0) s_sf[(lrow & 31) * 16 + (lrow >> 5) * 4 + (piece >> 2)] = static_cast<uint8_t>(e + 127);
+      if (piece % kLanesPerBlock == 0)
+        s_sf[(lrow & 31) * 16 + (lrow >> 5) * 4 + piece / kLanesPerBlock] = static_cast<uint8_t>(e + 127);
     }
   }
   __syncthreads();

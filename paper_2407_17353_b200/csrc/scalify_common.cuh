@@ -18,6 +18,8 @@ namespace scalify {
 // byte 16  : fp32 statistic word (bit pattern is also used for atomicMax)
 // byte 20  : scratch word of the matmul's fused AMAX (atomicMax target; zero between launches)
 // byte 32  : uint32 ticket of the "last block finishes" reductions (self-resetting)
+// byte 48  : fp32 scale word of an output whose caller passed no scale pointer
+// byte 52  : fp32 rescale factor a speculative matmul predicted
 // byte 64  : (Adam) not used
 // byte 256 : operation-specific area
 constexpr size_t kWsStatus = 0;

@@ -64,6 +64,21 @@ def test_mx_quantize_degenerate_blocks_and_strided_input():
     assert codes[0, 0] == 127 and codes[1, 1] == 127 and codes[2, 2] == 127 and codes[3, 3] == 0
 
 
+@pytest.mark.parametrize("x_dt,lead,skip", [(orc.BF16, 16, 8), (orc.BF16, 8, 0), (orc.F32, 4, 4)])
+def test_mx_quantize_rows_aligned_to_16_bytes_only(x_dt, lead, skip):
+    # a window of a wider buffer whose first element, or whose row stride, is a multiple of 16 bytes
+    # but not of 32: the kernel's 32-byte loads must fall back to 16-byte ones
+    rows, K = 70, 256
+    xb = np.ascontiguousarray(wide_range_input(9, rows, K + 32, x_dt, spread=10)[:, :K + lead])
+    buf = to_dev(xb, x_dt)
+    X = sc.ScaledTensor.make(buf[:, skip:skip + K], 1.0)
+    Y = sc.MxTensor(rows, K)
+    sc.scalify_mx_quantize(X, Y)
+    data, codes = orc.mx_quantize(np.ascontiguousarray(xb[:, skip:skip + K]), x_dt, orc.E4M3)
+    assert np.array_equal(Y.exponents().cpu().numpy(), codes)
+    assert np.array_equal(to_bits(Y.data, orc.E4M3), data)
+
+
 def run_mx_matmul(a, a_dt, ea, a_s, b, b_dt, eb, b_s, y_dt, stat=sc.STAT_NONE):
     M, K = a.shape
     N = b.shape[0]
