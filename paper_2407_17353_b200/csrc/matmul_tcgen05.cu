@@ -385,29 +385,40 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
       // Each lane holds 32 consecutive columns of ONE row.  The warp writes the chunk (32 rows x 32 columns)
       // into a shared-memory tile in the swizzle pattern TMA uses for rows of this width, and one lane hands
       // the tile to a TMA store, which writes whole row segments and clips rows >= M and columns >= N.
-      auto store = [&](const uint32_t* o, int c) {
-        const int col0 = n0 + (c_first + c) * 32;
+      // (stage_chunk fills the tile; issue_chunk hands it to TMA)
+      auto stage_chunk = [&](const uint32_t* o, int c) {
         uint8_t* tile_b = epi_mem + (warp - 2) * C::kEpiWarpBytes + (c % NBUF) * kTileBytes;
-        if (lane == 0) bulk_wait_read<NBUF - 1>();      // the tile's previous store has read it
-        __syncwarp();
         uint4* tile = reinterpret_cast<uint4*>(tile_b);
 #pragma unroll
         for (int j = 0; j < CPR; ++j)
           tile[lane * CPR + (j ^ ((lane / (8 / CPR)) % CPR))] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
-        uint8_t* tile_q = epi_mem + (warp - 2) * C::kEpiWarpBytes + 4096 + (c % NBUF) * 1024;
         if constexpr (SPEC) {
+          uint8_t* tile_q = epi_mem + (warp - 2) * C::kEpiWarpBytes + 4096 + (c % NBUF) * 1024;
           uint32_t oq[8];
           convert_q(o, oq);
           uint4* tq = reinterpret_cast<uint4*>(tile_q);  // 32 rows x 32 B, 32-byte swizzle: piece XOR (row / 4) % 2
           tq[lane * 2 + (0 ^ ((lane >> 2) & 1))] = make_uint4(oq[0], oq[1], oq[2], oq[3]);
           tq[lane * 2 + (1 ^ ((lane >> 2) & 1))] = make_uint4(oq[4], oq[5], oq[6], oq[7]);
         }
+      };
+      auto issue_chunk = [&](int c) {  // lane 0, after fence_async_smem + __syncwarp
+        const int col0 = n0 + (c_first + c) * 32;
+        const int row0 = mt * C::kTileM + static_cast<int>(rank) * kBM + q * 32;
+        uint8_t* tile_b = epi_mem + (warp - 2) * C::kEpiWarpBytes + (c % NBUF) * kTileBytes;
+        tma_store_3d(&map_y, smem_u32(tile_b), col0, row0, b);
+        if constexpr (SPEC) {
+          uint8_t* tile_q = epi_mem + (warp - 2) * C::kEpiWarpBytes + 4096 + (c % NBUF) * 1024;
+          tma_store_3d(&map_sfa, smem_u32(tile_q), col0, row0, b);
+        }
+      };
+      auto store = [&](const uint32_t* o, int c) {
+        if (lane == 0) bulk_wait_read<NBUF - 1>();      // the tile's previous store has read it
+        __syncwarp();
+        stage_chunk(o, c);
         fence_async_smem();
         __syncwarp();
         if (lane == 0) {
-          const int row0 = mt * C::kTileM + static_cast<int>(rank) * kBM + q * 32;
-          tma_store_3d(&map_y, smem_u32(tile_b), col0, row0, b);
-          if constexpr (SPEC) tma_store_3d(&map_sfa, smem_u32(tile_q), col0, row0, b);
+          issue_chunk(c);
           bulk_commit();
         }
       };
@@ -421,22 +432,34 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
       };
       uint32_t ra[32], rb[32];
       if constexpr (kAcc == 1 && OSZ <= 2) {
-        // A single accumulator: the next tile's MMAs wait for this read-out, so all chunks are read and
-        // converted first (kept as packed output words), the accumulator is handed back, then the stores follow.
-        uint32_t oc[kChunksPerWarp][32 * OSZ / 4];
+        // A single accumulator: the next tile's MMAs wait for this read-out.  The staging area holds all of
+        // a warp's chunks (NBUF == kChunksPerWarp), so every chunk is converted straight into its tile, the
+        // accumulator is handed back, and only then the TMA stores are issued.
+        static_assert(NBUF >= kChunksPerWarp, "staging must hold every chunk of a warp");
+        uint32_t o[32 * OSZ / 4];
+        if (lane == 0) bulk_wait_read<0>();  // the previous tile's stores have read the staging area
+        __syncwarp();
         if (n_chunks > 0) tmem_ld32(t_addr, ra);
-#pragma unroll
-        for (int c = 0; c < kChunksPerWarp; ++c) {
-          if (c < n_chunks) {
+#pragma unroll 1
+        for (int c = 0; c < n_chunks; c += 2) {
+          tmem_ld_wait();
+          if (c + 1 < n_chunks) tmem_ld32(t_addr + (c + 1) * 32, rb);
+          convert(ra, o);
+          stage_chunk(o, c);
+          if (c + 1 < n_chunks) {
             tmem_ld_wait();
-            if (c + 1 < n_chunks) tmem_ld32(t_addr + (c + 1) * 32, (c & 1) ? ra : rb);
-            convert((c & 1) ? rb : ra, oc[c]);
+            if (c + 2 < n_chunks) tmem_ld32(t_addr + (c + 2) * 32, ra);
+            convert(rb, o);
+            stage_chunk(o, c + 1);
           }
         }
         release_accumulator();
-#pragma unroll
-        for (int c = 0; c < kChunksPerWarp; ++c)
-          if (c < n_chunks) store(oc[c], c);
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0 && n_chunks > 0) {
+          for (int c = 0; c < n_chunks; ++c) issue_chunk(c);
+          bulk_commit();
+        }
       } else {
         // The TMEM load of the next chunk is in flight while the current chunk is processed.
         uint32_t o[32 * OSZ / 4];
