@@ -474,6 +474,38 @@ int scalify_scaled_attention(const scalify_array* Q, const scalify_array* K, con
                              uint32_t* status, void* stream);
 
 /*
+ * Fused scaled attention backward: the gradients of scalify_scaled_attention with
+ * respect to Q, K and V, from the gradient dO of its output and the probabilities
+ * P it used (its P_dump).  Same custom rule (Section 3.2.1), i.e. the composition
+ * of the calls it replaces:
+ *   dP_s = dO_s V_s kf(hd),   dP_d = (dO_d V_d^T) / kf(hd) rounded to BF16       (matmul rule)
+ *   dS_d = P_d (dP_d - sum_j dP_d[i,j] P_d[i,j]) rounded to E5M2,
+ *   dS_s = dP_s P_s c                                  (softmax backward, scalar c)
+ *   dQ_s = dS_s K_s kf(Tk),   dQ_d = (dS_d K_d) / kf(Tk)                          (matmul rule)
+ *   dK_s = dS_s Q_s kf(Tq),   dK_d = (dS_d^T Q_d) / kf(Tq)
+ *   dV_s = P_s dO_s kf(Tq),   dV_d = (P_d^T dO_d) / kf(Tq)
+ * i.e. scalify_scaled_matmul, scalify_scaled_softmax_bwd, scalify_scalar_mul_pow2
+ * and three more scalify_scaled_matmul.  Two launches: one CTA per (head, 128
+ * queries) forms dP (twice, it never reaches memory), dS and dQ; one CTA per
+ * (head, 128 keys) contracts P and dS over the queries into dV and dK.
+ *   Q, dO [heads, Tq, hd], K, V [heads, Tk, hd]: E4M3 or E5M2, hd = 64, 3-D views
+ *   as for the forward call.  P: E4M3, dense [heads, Tq, Tk], exact zeros where
+ *   the mask hides a key.  dS (output): E5M2, dense [heads, Tq, Tk], scale word
+ *   required; with causal != 0 the 128 x 128 blocks wholly above the diagonal are
+ *   not written.  dQ [heads, Tq, hd], dK, dV [heads, Tk, hd]: F16, BF16 or F32
+ *   (one dtype), same kind of view.  c: the forward's scalar, a power of two.
+ *   Tk % 32 == 0.  dP_dump (BF16, dense [heads, Tq, Tk]): optional copy of dP_d
+ *   for checking, normally NULL.  status: optional DEVICE word.
+ * Errors: NULL (also: dS without a scale word), DTYPE, SHAPE, ALIGNMENT,
+ * UNSUPPORTED (hd != 64, causal with Tk < Tq, c not a power of two), ALIAS (an
+ * output scale word aliasing another scale word of the call).
+ */
+int scalify_scaled_attention_bwd(const scalify_array* Q, const scalify_array* K, const scalify_array* V,
+                                 const scalify_array* P, const scalify_array* dO, float sm_scale, int causal,
+                                 scalify_array* dS, scalify_array* dQ, scalify_array* dK, scalify_array* dV,
+                                 scalify_array* dP_dump, uint32_t* status, void* stream);
+
+/*
  * Scaled Adam step without a workspace.  (No counterpart in the paper: this entry point exists
  * for the integration, not for the method.)
  *

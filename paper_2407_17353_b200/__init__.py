@@ -82,6 +82,7 @@ def lib() -> ctypes.CDLL:
         L.scalify_scaled_gelu_bwd.argtypes = [P, P, i32, P, vp]
         L.scalify_scaled_adam_step.argtypes = [i32, P, P, P, P, f32, f32, f32, f32, i64, vp, sz, vp]
         L.scalify_scaled_attention.argtypes = [P, P, P, f32, i32, P, P, P, vp, vp]
+        L.scalify_scaled_attention_bwd.argtypes = [P, P, P, P, P, f32, i32, P, P, P, P, P, vp, vp]
         L.scalify_mx_sf_bytes.restype = sz
         L.scalify_mx_sf_bytes.argtypes = [i64, i64]
         L.scalify_mx_quantize.argtypes = [P, vp, vp, vp]
@@ -103,6 +104,7 @@ def lib() -> ctypes.CDLL:
                      "scalify_scaled_embedding_bwd", "scalify_scaled_softmax", "scalify_scaled_softmax_bwd",
                      "scalify_scaled_cross_entropy", "scalify_scalar_mul_pow2", "scalify_debug_expire_wait",
                      "scalify_mx_quantize", "scalify_mx_matmul", "scalify_scaled_attention",
+                     "scalify_scaled_attention_bwd",
                      "scalify_scaled_matmul_speculative"):
             getattr(L, name).restype = i32
         _lib = L
@@ -440,3 +442,16 @@ def scalify_scaled_attention(Q: ScaledTensor, K: ScaledTensor, V: ScaledTensor, 
     _check(lib().scalify_scaled_attention(_ref(q), _ref(k), _ref(v), float(sm_scale), int(bool(causal)), _ref(o),
                                           _ref(sd), _ref(pd), _ptr(status), _stream(stream)),
            "scalify_scaled_attention")
+
+
+def scalify_scaled_attention_bwd(Q: ScaledTensor, K: ScaledTensor, V: ScaledTensor, P: ScaledTensor, dO: ScaledTensor,
+                                 dS: ScaledTensor, dQ: ScaledTensor, dK: ScaledTensor, dV: ScaledTensor, *,
+                                 sm_scale: float, causal: bool = True, dP_dump: Optional[ScaledTensor] = None,
+                                 status: Optional[torch.Tensor] = None, stream=None) -> None:
+    """Fused attention backward: P is the forward's P_dump, dS (E5M2, dense [heads, Tq, Tk]) an output."""
+    q, k, v, pp, do = _desc(Q), _desc(K), _desc(V), _desc(P), _desc(dO)
+    ds, dq, dk, dv, dpd = _desc(dS), _desc(dQ), _desc(dK), _desc(dV), _desc(dP_dump)
+    _check(lib().scalify_scaled_attention_bwd(_ref(q), _ref(k), _ref(v), _ref(pp), _ref(do), float(sm_scale),
+                                              int(bool(causal)), _ref(ds), _ref(dq), _ref(dk), _ref(dv), _ref(dpd),
+                                              _ptr(status), _stream(stream)),
+           "scalify_scaled_attention_bwd")

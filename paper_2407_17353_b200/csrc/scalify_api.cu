@@ -452,6 +452,64 @@ int scalify_scaled_attention(const scalify_array* Q, const scalify_array* K, con
   return launch_attention(a, static_cast<cudaStream_t>(stream));
 }
 
+int scalify_scaled_attention_bwd(const scalify_array* Q, const scalify_array* K, const scalify_array* V,
+                                 const scalify_array* P, const scalify_array* dO, float sm_scale, int causal,
+                                 scalify_array* dS, scalify_array* dQ, scalify_array* dK, scalify_array* dV,
+                                 scalify_array* dP_dump, uint32_t* status, void* stream) {
+  int rc;
+  if ((rc = check_array(Q)) || (rc = check_array(K)) || (rc = check_array(V)) || (rc = check_array(P)) ||
+      (rc = check_array(dO)) || (rc = check_array(dS)) || (rc = check_array(dQ)) || (rc = check_array(dK)) ||
+      (rc = check_array(dV)))
+    return rc;
+  if (is_wide(Q->dtype) || is_wide(K->dtype) || is_wide(V->dtype) || is_wide(dO->dtype)) return SCALIFY_ERR_DTYPE;
+  if (P->dtype != SCALIFY_E4M3 || dS->dtype != SCALIFY_E5M2) return SCALIFY_ERR_DTYPE;
+  if (!is_wide(dQ->dtype) || dK->dtype != dQ->dtype || dV->dtype != dQ->dtype) return SCALIFY_ERR_DTYPE;
+  if (!dS->scale) return SCALIFY_ERR_NULL;  // the second launch reads dS_s from the device
+  int ex = 0;
+  if (!(sm_scale > 0.f) || !isfinite(sm_scale) || frexpf(sm_scale, &ex) != 0.5f) return SCALIFY_ERR_UNSUPPORTED;
+  AttentionBwdArgs a;
+  int64_t hq, hk, hv, hdo, h1, h2, h3, tq, tk, tv, tdo, t1, t2, t3, dq, dk, dv, ddo, d1, d2, d3;
+  if ((rc = as_heads(Q, &hq, &tq, &dq, &a.q_ld, &a.q_hs)) || (rc = as_heads(K, &hk, &tk, &dk, &a.k_ld, &a.k_hs)) ||
+      (rc = as_heads(V, &hv, &tv, &dv, &a.v_ld, &a.v_hs)) || (rc = as_heads(dO, &hdo, &tdo, &ddo, &a.do_ld, &a.do_hs)) ||
+      (rc = as_heads(dQ, &h1, &t1, &d1, &a.dq_ld, &a.dq_hs)) || (rc = as_heads(dK, &h2, &t2, &d2, &a.dk_ld, &a.dk_hs)) ||
+      (rc = as_heads(dV, &h3, &t3, &d3, &a.dv_ld, &a.dv_hs)))
+    return rc;
+  if (hq != hk || hq != hv || hq != hdo || hq != h1 || hq != h2 || hq != h3) return SCALIFY_ERR_SHAPE;
+  if (tk != tv || tq != tdo || tq != t1 || tk != t2 || tk != t3) return SCALIFY_ERR_SHAPE;
+  if (dq != dk || dq != dv || dq != ddo || dq != d1 || dq != d2 || dq != d3) return SCALIFY_ERR_SHAPE;
+  if (tq < 1 || tk < 1 || hq < 1 || tq > 0x7FFFFFFF || tk > 0x7FFFFFFF || hq > 0x7FFFFFFF) return SCALIFY_ERR_SHAPE;
+  if (dq != 64 || (causal && tk < tq)) return SCALIFY_ERR_UNSUPPORTED;
+  if (tk % 32 != 0) return SCALIFY_ERR_SHAPE;  // rows of P and dS are read and written in 32-byte pieces
+  if (contiguous_numel(P) != hq * tq * tk || contiguous_numel(dS) != hq * tq * tk) return SCALIFY_ERR_SHAPE;
+  const float* in_scales[5] = {Q->scale, K->scale, V->scale, P->scale, dO->scale};
+  float* out_scales[4] = {dS->scale, dQ->scale, dK->scale, dV->scale};
+  for (int o = 0; o < 4; ++o) {
+    if (!out_scales[o]) continue;
+    for (int i = 0; i < 5; ++i)
+      if (out_scales[o] == in_scales[i]) return SCALIFY_ERR_ALIAS;
+    for (int o2 = 0; o2 < o; ++o2)
+      if (out_scales[o] == out_scales[o2]) return SCALIFY_ERR_ALIAS;
+  }
+  a.dP_dump = nullptr;
+  if (dP_dump) {
+    if ((rc = check_array(dP_dump))) return rc;
+    if (dP_dump->dtype != SCALIFY_BF16) return SCALIFY_ERR_DTYPE;
+    if (contiguous_numel(dP_dump) != hq * tq * tk) return SCALIFY_ERR_SHAPE;
+    a.dP_dump = dP_dump->data;
+  }
+  a.Q = Q->data; a.K = K->data; a.V = V->data; a.dO = dO->data;
+  a.q_dt = Q->dtype; a.k_dt = K->dtype; a.v_dt = V->dtype; a.do_dt = dO->dtype;
+  a.P = P->data; a.dS = dS->data;
+  a.dQ = dQ->data; a.dK = dK->data; a.dV = dV->data; a.g_dt = dQ->dtype;
+  a.heads = static_cast<int>(hq); a.Tq = static_cast<int>(tq); a.Tk = static_cast<int>(tk); a.hd = 64;
+  a.causal = causal ? 1 : 0;
+  a.sm_scale = sm_scale;
+  a.q_scale = Q->scale; a.k_scale = K->scale; a.v_scale = V->scale; a.p_scale = P->scale; a.do_scale = dO->scale;
+  a.ds_scale = dS->scale; a.dq_scale = dQ->scale; a.dk_scale = dK->scale; a.dv_scale = dV->scale;
+  a.status = status;
+  return launch_attention_bwd(a, static_cast<cudaStream_t>(stream));
+}
+
 static int adam_step_impl(int n_tensors, const scalify_array* grads, scalify_array* m, scalify_array* v,
                           scalify_array* w, const scalify_array* w_cast, float lr, float beta1, float beta2,
                           float eps, int64_t step, void* workspace, size_t workspace_bytes, void* stream) {

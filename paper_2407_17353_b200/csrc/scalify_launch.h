@@ -103,6 +103,23 @@ struct AttentionArgs {
   uint32_t* status;
 };
 int launch_attention(const AttentionArgs& a, cudaStream_t st);
+
+struct AttentionBwdArgs {
+  const void* Q; const void* K; const void* V; const void* dO; int q_dt, k_dt, v_dt, do_dt;  // FP8 [heads, T, hd] views
+  int64_t q_ld, q_hs, k_ld, k_hs, v_ld, v_hs, do_ld, do_hs;                                  // strides in elements
+  const void* P;   // E4M3 [heads, Tq, Tk] dense: the probabilities the forward pass used
+  void* dS;        // E5M2 [heads, Tq, Tk] dense (output, and operand of the dK product)
+  void* dQ; void* dK; void* dV; int g_dt;   // F16 / BF16 / F32 [heads, T, hd] views
+  int64_t dq_ld, dq_hs, dk_ld, dk_hs, dv_ld, dv_hs;
+  int heads, Tq, Tk, hd;
+  int causal;
+  float sm_scale;  // a power of two
+  const float* q_scale; const float* k_scale; const float* v_scale; const float* p_scale; const float* do_scale;
+  float* ds_scale; float* dq_scale; float* dk_scale; float* dv_scale;
+  void* dP_dump;   // optional BF16 [heads, Tq, Tk] dense: dP's data component as rounded
+  uint32_t* status;
+};
+int launch_attention_bwd(const AttentionBwdArgs& a, cudaStream_t st);
 int launch_mx_quantize(const void* X, int x_dt, int64_t rows, int64_t K, int64_t ldx, void* data, int elem_dt,
                        uint8_t* sf, const float* x_scale, float* y_scale, uint32_t* status, cudaStream_t st);
 
