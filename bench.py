@@ -217,6 +217,19 @@ def run_profile_row(args):
         Oa = sc.ScaledTensor.empty((H, T, HD), torch.bfloat16, dev)
         fn = lambda t: sc.scalify_scaled_attention(Qa, Ka, Va, Oa, sm_scale=0.125, causal=True)
         work = {"flop": 2.0 * H * T * T * HD}
+    elif row == "attention_bwd":
+        H, T, HD = 96, 1024, 64
+        Qa, Ka, Va = (sc.ScaledTensor.make(rnd((H, T, HD), torch.float8_e4m3fn, 30 + i), 1.0) for i in range(3))
+        Oa = sc.ScaledTensor.empty((H, T, HD), torch.bfloat16, dev)
+        Pa = sc.ScaledTensor(torch.zeros((H, T, T), dtype=torch.uint8, device=dev).view(torch.float8_e4m3fn),
+                             torch.ones(1, dtype=torch.float32, device=dev))
+        sc.scalify_scaled_attention(Qa, Ka, Va, Oa, sm_scale=0.125, causal=True, P_dump=Pa)
+        dOa = sc.ScaledTensor.make(rnd((H, T, HD), torch.float8_e5m2, 34), 2.0 ** -9)
+        dSa = sc.ScaledTensor.empty((H, T, T), torch.float8_e5m2, dev)
+        dQa, dKa, dVa = (sc.ScaledTensor.empty((H, T, HD), torch.bfloat16, dev) for _ in range(3))
+        fn = lambda t: sc.scalify_scaled_attention_bwd(Qa, Ka, Va, Pa, dOa, dSa, dQa, dKa, dVa, sm_scale=0.125,
+                                                       causal=True)
+        work = {"flop": 4.0 * H * T * T * HD}
     elif row == "rescale":
         n = 8192 * 8192
         X = sc.ScaledTensor.make(rnd((n,), torch.bfloat16, 1, 37.0), 1.0)
@@ -293,7 +306,7 @@ def main():
                          "(scalify_scaled_matmul_speculative; same outputs bit for bit)")
     ap.add_argument("--no-next", action="store_true",
                     help="skip the separately timed next-row variants f1, f2 (for ncu launch lists of the step)")
-    ap.add_argument("--profile-row", default=None, choices=["matmul", "mx", "attention", "rescale", "add", "layernorm", "adam"],
+    ap.add_argument("--profile-row", default=None, choices=["matmul", "mx", "attention", "attention_bwd", "rescale", "add", "layernorm", "adam"],
                     help="run only this row on a reduced, still larger-than-L2 case (for ncu captures)")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -530,7 +543,7 @@ def main():
         del Xa, Xb, Am, Bm
 
     # Fused attention forward on the config-5 shape: 8 sequences x 12 heads, 1024 tokens, head dimension 64
-    att_ms = float("nan")
+    att_ms = att_bwd_ms = float("nan")
     ATT_H, ATT_T, ATT_HD = 96, 1024, 64
     if not args.no_next:
         Qa, Ka, Va = (sc.ScaledTensor.make(rnd((ATT_H, ATT_T, ATT_HD), torch.float8_e4m3fn, 30 + i), 1.0)
@@ -547,7 +560,25 @@ def main():
         a1.record()
         barrier()
         att_ms = a0.elapsed_time(a1) / a_iters
-        del Qa, Ka, Va, Oa
+        # ... and its backward (two launches): P from the forward's copy, dO as E5M2
+        Pa = sc.ScaledTensor(torch.zeros((ATT_H, ATT_T, ATT_T), dtype=torch.uint8, device=dev).view(torch.float8_e4m3fn),
+                             torch.ones(1, dtype=torch.float32, device=dev))
+        sc.scalify_scaled_attention(Qa, Ka, Va, Oa, sm_scale=0.125, causal=True, P_dump=Pa)
+        dOa = sc.ScaledTensor.make(rnd((ATT_H, ATT_T, ATT_HD), torch.float8_e5m2, 34), 2.0 ** -9)
+        dSa = sc.ScaledTensor.empty((ATT_H, ATT_T, ATT_T), torch.float8_e5m2, dev)
+        dQa, dKa, dVa = (sc.ScaledTensor.empty((ATT_H, ATT_T, ATT_HD), torch.bfloat16, dev) for _ in range(3))
+        att_bwd = lambda: sc.scalify_scaled_attention_bwd(Qa, Ka, Va, Pa, dOa, dSa, dQa, dKa, dVa, sm_scale=0.125,
+                                                          causal=True)
+        for _ in range(3):
+            att_bwd()
+        barrier()
+        a0.record()
+        for _ in range(a_iters):
+            att_bwd()
+        a1.record()
+        barrier()
+        att_bwd_ms = a0.elapsed_time(a1) / a_iters
+        del Qa, Ka, Va, Oa, Pa, dOa, dSa, dQa, dKa, dVa
 
     # ------------------------------------------------------------------ end to end through host buffers
     hY = torch.empty((N_GEMM, N_GEMM), dtype=torch.int8).pin_memory()
@@ -657,6 +688,11 @@ def main():
                 "probabilities never leave the chip)", "ms": round(float(att_ms), 4),
          "TFLOP/s": round(2.0 * ATT_H * ATT_T * ATT_T * ATT_HD / (att_ms * 1e-3) / 1e12, 1),
          "note": "flop counted for the causal half of Q K^T and P V"},
+        {"row": "f4 (next, own loop) fused causal attention backward, same shape: dQ, dK, dV from dO and the "
+                "forward's E4M3 probabilities in two launches (dP never leaves the chip, dS is written once)",
+         "ms": round(float(att_bwd_ms), 4),
+         "TFLOP/s": round(4.0 * ATT_H * ATT_T * ATT_T * ATT_HD / (att_bwd_ms * 1e-3) / 1e12, 1),
+         "note": "flop counted for the causal half of dO V^T, dS K, dS^T Q and P^T dO"},
     ]
     fp8_peak = 2.0 * peaks["bf16_sustained"]
     gemm_tflops = flops / (float(seg_ms[0]) * 1e-3) / 1e12

@@ -489,8 +489,8 @@ int scalify_scaled_attention(const scalify_array* Q, const scalify_array* K, con
  * queries) forms dP (twice, it never reaches memory), dS and dQ; one CTA per
  * (head, 128 keys) contracts P and dS over the queries into dV and dK.
  *   Q, dO [heads, Tq, hd], K, V [heads, Tk, hd]: E4M3 or E5M2, hd = 64, 3-D views
- *   as for the forward call.  P: E4M3, dense [heads, Tq, Tk], exact zeros where
- *   the mask hides a key.  dS (output): E5M2, dense [heads, Tq, Tk], scale word
+ *   as for the forward call.  P: E4M3, dense [heads, Tq, Tk], non-negative (the
+ *   sign bit is ignored), exact zeros where the mask hides a key.  dS (output): E5M2, dense [heads, Tq, Tk], scale word
  *   required; with causal != 0 the 128 x 128 blocks wholly above the diagonal are
  *   not written.  dQ [heads, Tq, hd], dK, dV [heads, Tk, hd]: F16, BF16 or F32
  *   (one dtype), same kind of view.  c: the forward's scalar, a power of two.

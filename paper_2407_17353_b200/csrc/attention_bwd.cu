@@ -16,8 +16,8 @@
 //               forms dS, rounds it to E5M2 and writes it as the A operand of dS K (128-byte swizzle) and to HBM
 //   warp 8      one thread: TMA loads (dO once; V, P and in sweep B also K per key block) and all tcgen05.mma
 //   TMEM: 128 columns of dP + 64 columns of dQ.
-// Launch 2, one CTA per (head, block of 128 keys), 192 threads: a two-stage TMA ring of (P, dS, dO, Q) tiles
-// over the query blocks that see the key block; P^T dO and dS^T Q read the P and dS tiles MN-major (the
+// Launch 2, one CTA per (head, block of 128 keys), 192 threads: a two-slot TMA ring of (P, dS, dO, Q) tiles,
+// 64 queries each, over the queries that see the key block; P^T dO and dS^T Q read the P and dS tiles MN-major (the
 // queries are the contraction), so no transposed copy exists; dV and dK accumulate in TMEM (64 columns
 // each) and are read out once.
 // Every mbarrier wait is bounded; on expiry the CTA records SCALIFY_DEV_TIMEOUT and leaves.
@@ -67,15 +67,25 @@ __device__ __forceinline__ uint64_t bw_desc_sw64(uint32_t saddr, uint32_t sbo_by
   return d;
 }
 
-// Four E4M3 bytes of a word -> fp32 with integer arithmetic: sign and the seven magnitude bits moved
-// to the fp32 fields, then the bias difference 2^(127-7) as one exact multiply (subnormals included).
+// Four E4M3 magnitudes of a word -> fp32 with integer arithmetic: the seven magnitude bits moved to the
+// top of the fp32 exponent/mantissa fields (one shift and one mask per element), then the bias
+// difference 2^(127-7) as one exact multiply (subnormals included).  The sign bit is ignored:
+// probabilities are never negative.
 __device__ __forceinline__ void e4m3x4_to_float(uint32_t w, float* f) {
-#pragma unroll
-  for (int k = 0; k < 4; ++k) {
-    const uint32_t t = __byte_perm(w, 0u, 0x0444u | (static_cast<uint32_t>(k) << 12));  // byte k in bits 24-31
-    const uint32_t bits = (t & 0x80000000u) | ((t & 0x7F000000u) >> 4);
-    f[k] = __uint_as_float(bits) * 1.329227995784916e36f;  // 2^120
-  }
+  const float k = 1.329227995784916e36f;  // 2^120
+  f[0] = __uint_as_float((w << 20) & 0x07F00000u) * k;
+  f[1] = __uint_as_float((w << 12) & 0x07F00000u) * k;
+  f[2] = __uint_as_float((w << 4) & 0x07F00000u) * k;
+  f[3] = __uint_as_float((w >> 4) & 0x07F00000u) * k;
+}
+
+// Two fp32 accumulators -> their BF16 roundings (round to nearest even, one conversion instruction for
+// the pair: that pipe is idle in these kernels), widened back to fp32
+__device__ __forceinline__ void bf16_round_pair(uint32_t a_bits, uint32_t b_bits, float& a, float& b) {
+  uint32_t packed;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(packed) : "f"(__uint_as_float(b_bits)), "f"(__uint_as_float(a_bits)));
+  a = __uint_as_float(packed << 16);
+  b = __uint_as_float(packed & 0xFFFF0000u);
 }
 
 template <int GDT>
@@ -206,9 +216,8 @@ attention_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_do, const __grid
     constexpr int kChunks = kBwK / 32 / 2;    // 32-key chunks per thread and block
     const int c_first = half * kChunks;
     const long long dump_row = (static_cast<long long>(head) * p.Tq + i) * p.Tk;
-    // dP's data component: the accumulator rounded to BF16 (integer round-to-nearest-even on the upper 16
-    // bits) and divided by kf(hd), a power of two, which commutes with the rounding
-    auto bf16_rne = [](uint32_t b) { return __uint_as_float((b + 0x7FFFu + ((b >> 16) & 1u)) & 0xFFFF0000u); };
+    // dP's data component: the accumulator rounded to BF16 and divided by kf(hd), a power of two, which
+    // commutes with the rounding
     // this thread's 32 probabilities of chunk c: two 16-byte pieces of row r of the 128-byte-swizzled tile
     auto load_p = [&](const uint8_t* p_tile, int c, float* pf) {
       const uint4* row = reinterpret_cast<const uint4*>(p_tile + r * 128);
@@ -234,7 +243,12 @@ attention_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_do, const __grid
         tmem_ld_wait();
         float d4[4] = {0.f, 0.f, 0.f, 0.f};  // four independent chains
 #pragma unroll
-        for (int e = 0; e < 32; ++e) d4[e & 3] = fmaf(bf16_rne(acc[e]) * p.inv_kf_hd, pf[e], d4[e & 3]);
+        for (int e = 0; e < 32; e += 2) {
+          float x0, x1;
+          bf16_round_pair(acc[e], acc[e + 1], x0, x1);
+          d4[e & 3] = fmaf(x0 * p.inv_kf_hd, pf[e], d4[e & 3]);
+          d4[(e + 1) & 3] = fmaf(x1 * p.inv_kf_hd, pf[e + 1], d4[(e + 1) & 3]);
+        }
         delta += (d4[0] + d4[1]) + (d4[2] + d4[3]);
         if (p.dP_dump && i < p.Tq) {
           const int j0 = kb * kBwK + c * 32;
@@ -277,7 +291,12 @@ attention_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_do, const __grid
         load_p(p_tile, c, pf);
         tmem_ld_wait();
 #pragma unroll
-        for (int e = 0; e < 32; ++e) pf[e] *= bf16_rne(acc[e]) * p.inv_kf_hd - delta;
+        for (int e = 0; e < 32; e += 2) {
+          float x0, x1;
+          bf16_round_pair(acc[e], acc[e + 1], x0, x1);
+          pf[e] *= x0 * p.inv_kf_hd - delta;
+          pf[e + 1] *= x1 * p.inv_kf_hd - delta;
+        }
         uint32_t o[8];
         encode_vec<SCALIFY_E5M2, 32>(pf, o);
         uint4* row = reinterpret_cast<uint4*>(ds_tile + r * 128);
@@ -335,12 +354,16 @@ attention_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_do, const __grid
 // ---------------------------------------------------------------------------------------------
 constexpr int kBw2Threads = 192;   // warp 0: TMA, warp 1: MMA, warps 2-5: read-out
 constexpr int kBw2Stages = 2;
-constexpr int kBw2Stage = 2 * kBwPTile + 2 * kBwTile;  // P, dS, dO, Q of one query block: 48 KB
+constexpr int kBw2Q = 64;          // queries per ring slot: short slots, so that four CTAs fit an SM and their
+                                   // prologues and read-outs overlap the others' loads
+constexpr int kBw2PTile = kBw2Q * kBwK;    // 8 KB: 64 queries x 128 keys of P or dS
+constexpr int kBw2Tile = kBw2Q * kBwHd;    // 4 KB: 64 rows of dO or Q
+constexpr int kBw2Stage = 2 * kBw2PTile + 2 * kBw2Tile;  // 24 KB
 constexpr size_t kBw2Smem = size_t(kBw2Stages) * kBw2Stage + 1024 + 256;
 constexpr int kBw2TmemCols = 128;  // dV: columns 0-63, dK: columns 64-127
 
 template <int GDT>
-__global__ void __launch_bounds__(kBw2Threads, 2)
+__global__ void __launch_bounds__(kBw2Threads, 4)
 attention_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_ds,
                          const __grid_constant__ CUtensorMap map_do, const __grid_constant__ CUtensorMap map_q,
                          const AttBwdParams p) {
@@ -358,8 +381,8 @@ attention_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
   // with a causal mask the early key blocks are seen by the most query blocks: they come first
   const int kb = static_cast<int>(blockIdx.x / p.heads), head = blockIdx.x % p.heads;
   const int shift = p.Tk - p.Tq;
-  const int i_min = p.causal ? max(0, kb * kBwK - shift) / kBwQ : 0;  // first query block that sees a key of this block
-  const int n_qb = p.q_blocks - i_min;
+  const int i_min = p.causal ? max(0, kb * kBwK - shift) / kBw2Q : 0;  // first 64-query step that sees a key of this block
+  const int n_qb = (p.Tq + kBw2Q - 1) / kBw2Q - i_min;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kBw2Stages; ++s) { mbar_init(full_bar + 8 * s, 1); mbar_init(empty_bar + 8 * s, 1); }
@@ -392,12 +415,12 @@ attention_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
         if (use >= 1 && !mbar_wait(empty_bar + 8 * stage, (use - 1) & 1, abort_flag)) { timed_out = true; break; }
         const uint32_t fb = full_bar + 8 * stage;
         const uint32_t s0 = base + stage * kBw2Stage;
-        const int q0 = (i_min + t) * kBwQ;
+        const int q0 = (i_min + t) * kBw2Q;
         mbar_expect_tx(fb, kBw2Stage);
         tma_load_3d(s0, &map_p, fb, kb * kBwK, q0, head);
-        tma_load_3d(s0 + kBwPTile, &map_ds, fb, kb * kBwK, q0, head);
-        tma_load_3d(s0 + 2 * kBwPTile, &map_do, fb, 0, q0, head);
-        tma_load_3d(s0 + 2 * kBwPTile + kBwTile, &map_q, fb, 0, q0, head);
+        tma_load_3d(s0 + kBw2PTile, &map_ds, fb, kb * kBwK, q0, head);
+        tma_load_3d(s0 + 2 * kBw2PTile, &map_do, fb, 0, q0, head);
+        tma_load_3d(s0 + 2 * kBw2PTile + kBw2Tile, &map_q, fb, 0, q0, head);
       }
     }
   } else if (warp == 1) {
@@ -407,19 +430,19 @@ attention_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
         if (!mbar_wait(full_bar + 8 * stage, use & 1, abort_flag)) { timed_out = true; break; }
         tc_fence_after();
         const uint32_t s0 = base + stage * kBw2Stage;
-        // P and dS tiles [128 queries][128 keys]: A operands in MN-major form (the keys are M, the queries the
-        // contraction): 8-query atoms 1024 B apart, 32 queries (4096 B) per MMA.  dO and Q tiles [128 queries][64 B]:
+        // P and dS tiles [64 queries][128 keys]: A operands in MN-major form (the keys are M, the queries the
+        // contraction): 8-query atoms 1024 B apart, 32 queries (4096 B) per MMA.  dO and Q tiles [64 queries][64 B]:
         // B operands in MN-major form, 8-query atoms 512 B apart, 32 queries (2048 B) per MMA.
         const uint64_t p_desc = make_smem_desc(s0, 0u, 1024u);
-        const uint64_t ds_desc = make_smem_desc(s0 + kBwPTile, 0u, 1024u);
-        const uint64_t do_desc = bw_desc_sw64(s0 + 2 * kBwPTile, 512u);
-        const uint64_t q_desc = bw_desc_sw64(s0 + 2 * kBwPTile + kBwTile, 512u);
+        const uint64_t ds_desc = make_smem_desc(s0 + kBw2PTile, 0u, 1024u);
+        const uint64_t do_desc = bw_desc_sw64(s0 + 2 * kBw2PTile, 512u);
+        const uint64_t q_desc = bw_desc_sw64(s0 + 2 * kBw2PTile + kBw2Tile, 512u);
 #pragma unroll
-        for (int k = 0; k < kBwQ / 32; ++k)
+        for (int k = 0; k < kBw2Q / 32; ++k)
           umma_f8(tmem_base, p_desc + static_cast<uint64_t>(k * (32 * 128 / 16)),
                   do_desc + static_cast<uint64_t>(k * (32 * kBwHd / 16)), p.idesc_dv, (t | k) != 0 ? 1u : 0u);
 #pragma unroll
-        for (int k = 0; k < kBwQ / 32; ++k)
+        for (int k = 0; k < kBw2Q / 32; ++k)
           umma_f8(tmem_base + 64, ds_desc + static_cast<uint64_t>(k * (32 * 128 / 16)),
                   q_desc + static_cast<uint64_t>(k * (32 * kBwHd / 16)), p.idesc_dk, (t | k) != 0 ? 1u : 0u);
         umma_commit(empty_bar + 8 * stage);
@@ -473,15 +496,19 @@ attention_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
 }
 
 int launch_attention_bwd(const AttentionBwdArgs& a, cudaStream_t st) {
-  CUtensorMap map_q, map_k, map_v, map_do, map_p, map_ds;
+  CUtensorMap map_k, map_v, map_do, map_p;
   int rc;
-  if ((rc = make_byte_map(&map_q, a.Q, a.hd, a.Tq, a.heads, a.q_ld, a.q_hs, kBwHd, kBwQ))) return rc;
   if ((rc = make_byte_map(&map_do, a.dO, a.hd, a.Tq, a.heads, a.do_ld, a.do_hs, kBwHd, kBwQ))) return rc;
   if ((rc = make_byte_map(&map_k, a.K, a.hd, a.Tk, a.heads, a.k_ld, a.k_hs, kBwHd, kBwK))) return rc;
   if ((rc = make_byte_map(&map_v, a.V, a.hd, a.Tk, a.heads, a.v_ld, a.v_hs, kBwHd, kBwK))) return rc;
   const uint64_t plane = static_cast<uint64_t>(a.Tq) * static_cast<uint64_t>(a.Tk);
   if ((rc = make_byte_map(&map_p, a.P, a.Tk, a.Tq, a.heads, a.Tk, plane, kBwK, kBwQ))) return rc;
-  if ((rc = make_byte_map(&map_ds, a.dS, a.Tk, a.Tq, a.heads, a.Tk, plane, kBwK, kBwQ))) return rc;
+  // launch 2 reads 64 queries per ring slot
+  CUtensorMap map_p2, map_ds2, map_do2, map_q2;
+  if ((rc = make_byte_map(&map_p2, a.P, a.Tk, a.Tq, a.heads, a.Tk, plane, kBwK, kBw2Q))) return rc;
+  if ((rc = make_byte_map(&map_ds2, a.dS, a.Tk, a.Tq, a.heads, a.Tk, plane, kBwK, kBw2Q))) return rc;
+  if ((rc = make_byte_map(&map_do2, a.dO, a.hd, a.Tq, a.heads, a.do_ld, a.do_hs, kBwHd, kBw2Q))) return rc;
+  if ((rc = make_byte_map(&map_q2, a.Q, a.hd, a.Tq, a.heads, a.q_ld, a.q_hs, kBwHd, kBw2Q))) return rc;
   AttBwdParams p;
   p.heads = a.heads; p.Tq = a.Tq; p.Tk = a.Tk;
   p.q_blocks = (a.Tq + kBwQ - 1) / kBwQ;
@@ -521,7 +548,7 @@ int launch_attention_bwd(const AttentionBwdArgs& a, cudaStream_t st) {
     }
     k1<<<static_cast<unsigned>(ctas1), kBw1Threads, kBw1Smem, st>>>(map_do, map_v, map_k, map_p, p);
     SCALIFY_CUDA_TRY(cudaGetLastError());
-    k2<<<static_cast<unsigned>(ctas2), kBw2Threads, kBw2Smem, st>>>(map_p, map_ds, map_do, map_q, p);
+    k2<<<static_cast<unsigned>(ctas2), kBw2Threads, kBw2Smem, st>>>(map_p2, map_ds2, map_do2, map_q2, p);
   });
   SCALIFY_CUDA_TRY(cudaGetLastError());
   return SCALIFY_OK;

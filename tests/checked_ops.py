@@ -261,6 +261,48 @@ class Ops:
                 assert self.within(Og[h], Oo, o_dt, oacc, osab, 1e-5).all()
         return P
 
+    def attention_bwd(self, Q, K, V, P, dO, dQ, dK, dV, sm_scale, causal=True):
+        """Fused backward over [heads, T, 64] views: dQ, dK, dV are written in place (their scale words too).
+        Checked stage by stage through the kernel's own dP copy and its dS output."""
+        H, Tq, _ = Q.data.shape
+        Tk = K.data.shape[1]
+        dev = Q.data.device
+        dS = sc.ScaledTensor(torch.zeros((H, Tq, Tk), dtype=torch.uint8, device=dev).view(torch.float8_e5m2),
+                             torch.zeros(1, dtype=torch.float32, device=dev))
+        dPd = None
+        if self.check:
+            dPd = sc.ScaledTensor(torch.zeros((H, Tq, Tk), dtype=torch.bfloat16, device=dev), None)
+        sc.scalify_scaled_attention_bwd(Q, K, V, P, dO, dS, dQ, dK, dV, sm_scale=sm_scale, causal=causal, dP_dump=dPd)
+        self.calls += 1
+        if self.check:
+            o = self.orc
+            q_dt, k_dt, v_dt, g_in, g_dt = code(Q.data), code(K.data), code(V.data), code(dO.data), code(dQ.data)
+            qb, kb, vb, gb, pb = self.bits(Q), self.bits(K), self.bits(V), self.bits(dO), self.bits(P)
+            dPg, dSg = self.bits(dPd), self.bits(dS)
+            dQg, dKg, dVg = (self.bits(sc.ScaledTensor(t.data.contiguous(), None)) for t in (dQ, dK, dV))
+            ii, jj = np.meshgrid(np.arange(Tq), np.arange(Tk), indexing="ij")
+            shift = Tk - Tq
+            vis = ((jj // 128) * 128 <= (ii // 128) * 128 + 127 + shift) if causal else np.ones((Tq, Tk), dtype=bool)
+            for h in range(H):
+                dPo, dps, acc, sab = o.scaled_matmul(gb[h], g_in, dO.scale_value(), vb[h], v_dt, V.scale_value(), BF,
+                                                     transB=True, want_acc=True)
+                assert self.within(dPg[h][vis], dPo[vis], BF, acc[vis], sab[vis], 1e-5).all()
+                dPin = np.where(vis, dPg[h], 0).astype(np.uint16)
+                dSo, dss = o.softmax_bwd(dPin, BF, dps, pb[h], E4, P.scale_value(), E5)
+                assert dS.scale_value() == dss * sm_scale
+                pv, gv = o.decode(pb[h], E4), o.decode(dPin, BF)
+                dot = (pv * gv).sum(-1, keepdims=True)
+                mag = pv * (np.abs(gv) + np.abs(pv * gv).sum(-1, keepdims=True))
+                assert self.within(dSg[h][vis], dSo[vis], E5, (pv * (gv - dot))[vis], mag[vis], 1e-5).all()
+                dSin = np.where(vis, dSg[h], 0).astype(np.uint8)
+                for got, (A, a_dt, a_s, B, b_dt, b_s, tA), out in (
+                        (dQg[h], (dSin, E5, dS.scale_value(), kb[h], k_dt, K.scale_value(), False), dQ),
+                        (dKg[h], (dSin, E5, dS.scale_value(), qb[h], q_dt, Q.scale_value(), True), dK),
+                        (dVg[h], (pb[h], E4, P.scale_value(), gb[h], g_in, dO.scale_value(), True), dV)):
+                    Yo, ys, a2, b2 = o.scaled_matmul(A, a_dt, a_s, B, b_dt, b_s, g_dt, transA=tA, want_acc=True)
+                    assert out.scale_value() == ys
+                    assert self.within(got, Yo, g_dt, a2, b2, 1e-5).all()
+
     def softmax_bwd(self, dP, P, o_dt):
         dS = self.empty(P.data.shape, o_dt)
         sc.scalify_scaled_softmax_bwd(dP, P, dS)

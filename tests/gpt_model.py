@@ -179,8 +179,13 @@ class ScaledGPT:
             for b in range(B):
                 Pb = s["P8"][b]
                 dOb = self._heads(datt8, b)
-                dPb = o.mm(dOb, self._heads(s["v8"], b), transB=True)                # dO V^T  [H, T, T]
                 view = lambda Tn: sc.ScaledTensor(self._heads(sc.ScaledTensor(Tn.data, None), b).data, Tn.scale)
+                if hd == 64:
+                    # dO V^T, the softmax backward, 1/sqrt(hd) and the three gradient products in two launches
+                    o.attention_bwd(self._heads(s["q8"], b), self._heads(s["k8"], b), self._heads(s["v8"], b), Pb, dOb,
+                                    view(dq), view(dk), view(dv), 1.0 / float(np.sqrt(hd)))
+                    continue
+                dPb = o.mm(dOb, self._heads(s["v8"], b), transB=True)                # dO V^T  [H, T, T]
                 o.mm(Pb, dOb, transA=True, Y=view(dv))                               # P^T dO  [H, T, hd]
                 dSb = o.softmax_bwd(dPb, Pb, E5)
                 o.scalar_mul(dSb, 1.0 / float(np.sqrt(hd)))

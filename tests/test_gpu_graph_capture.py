@@ -38,6 +38,12 @@ def build_chain(seed_scale):
     H = N // 64
     O = sc.ScaledTensor(torch.empty((M, N), dtype=torch.bfloat16, device=dev).view(M, H, 64).permute(1, 0, 2),
                         torch.zeros(1, device=dev))
+    Pd = sc.ScaledTensor(torch.zeros((H, M, M), dtype=torch.uint8, device=dev).view(torch.float8_e4m3fn),
+                         torch.ones(1, device=dev))
+    dO8 = sc.ScaledTensor.make(torch.randn((M, N), device=dev, generator=g).to(torch.float8_e5m2), 2.0 ** -9)
+    dS = sc.ScaledTensor.empty((H, M, M), torch.float8_e5m2)
+    dQ, dK, dV = (sc.ScaledTensor(torch.empty((M, N), dtype=torch.bfloat16, device=dev).view(M, H, 64).permute(1, 0, 2),
+                                  torch.zeros(1, device=dev)) for _ in range(3))
     ws_mm = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_MATMUL, M, N))
     ws_rs = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_RESCALE, M * N))
     heads = lambda X: sc.ScaledTensor(X.data.view(M, H, 64).permute(1, 0, 2), X.scale)
@@ -51,10 +57,13 @@ def build_chain(seed_scale):
         sc.scalify_mx_quantize(S, Am)
         sc.scalify_mx_quantize(W2, Bm)
         sc.scalify_mx_matmul(Am, Bm, Y2, ws_mm)
-        sc.scalify_scaled_attention(heads(L), heads(S8), heads(Yq), O, sm_scale=0.125, causal=True)
+        sc.scalify_scaled_attention(heads(L), heads(S8), heads(Yq), O, sm_scale=0.125, causal=True, P_dump=Pd)
+        sc.scalify_scaled_attention_bwd(heads(L), heads(S8), heads(Yq), Pd, heads(dO8), dS, dQ, dK, dV,
+                                        sm_scale=0.125, causal=True)
 
-    outputs = lambda: [x.data.contiguous().view(torch.uint8).cpu().numpy().copy() for x in (Yq, Yq2, S8, L, Y2, O)] + \
-                      [np.array([x.scale_value() for x in (Yq, Yq2, S8, L, Y2, O)])]
+    outs = (Yq, Yq2, S8, L, Y2, O, dQ, dK, dV)
+    outputs = lambda: [x.data.contiguous().view(torch.uint8).cpu().numpy().copy() for x in outs] + \
+                      [np.array([x.scale_value() for x in outs])]
     return A, t, chain, outputs
 
 
