@@ -136,6 +136,37 @@ def test_ragged_lengths_and_shifted_causal_mask_backward():
     run_case(2, 200, 224, True)
 
 
+@pytest.mark.parametrize("H,Tq,Tk,causal", [(1, 96, 32, False), (2, 320, 320, True), (1, 40, 2048, True),
+                                            (1, 2048, 2048, True), (3, 64, 64, True)])
+def test_backward_edge_shapes(H, Tq, Tk, causal):
+    # a single partial key block; a length that ends in the middle of a 128-query block (one 64-query ring
+    # slot of the dK/dV launch is empty past the end); few queries against many keys; 16 key blocks
+    run_case(H, Tq, Tk, causal, seed=7)
+
+
+def test_backward_of_a_single_head_given_as_2d_arrays():
+    T = 256
+    q = si.to_bits(si.normal(9, 1, (1, T, HD), 1.0), orc.E4M3)
+    k = si.to_bits(si.normal(9, 2, (1, T, HD), 1.0), orc.E4M3)
+    v = si.to_bits(si.normal(9, 3, (1, T, HD), 1.0), orc.E4M3)
+    do = si.to_bits(si.normal(9, 4, (1, T, HD), 1.0), orc.E5M2)
+    P = oracle_probabilities(q, orc.E4M3, 1.0, k, 1.0, 0.125, True)
+    mk = lambda x, dt, s: sc.ScaledTensor.make(to_dev(x[0], dt), s)
+    Q, K, V, dO = mk(q, orc.E4M3, 1.0), mk(k, orc.E4M3, 1.0), mk(v, orc.E4M3, 1.0), mk(do, orc.E5M2, 1.0)
+    Pd = sc.ScaledTensor(to_dev(P, orc.E4M3), None)
+    dS = sc.ScaledTensor.empty((1, T, T), torch.float8_e5m2)
+    out2, out3 = [], []
+    for shape, outs in (((T, HD), out2), ((1, T, HD), out3)):
+        dQ, dK, dV = (sc.ScaledTensor.empty(shape, torch.float32) for _ in range(3))
+        a = (Q, K, V, Pd, dO) if len(shape) == 2 else tuple(
+            sc.ScaledTensor(t.data.reshape((1,) + tuple(t.data.shape)), t.scale) if t is not Pd else t
+            for t in (Q, K, V, Pd, dO))
+        sc.scalify_scaled_attention_bwd(*a, dS, dQ, dK, dV, sm_scale=0.125, causal=True)
+        outs.extend(to_bits(t.data, orc.F32).reshape(-1) for t in (dQ, dK, dV))
+    for x, y in zip(out2, out3):
+        assert np.array_equal(x, y)
+
+
 def test_backward_heads_inside_a_token_major_buffer_and_mixed_formats():
     run_case(4, 256, 256, True, merged_layout=True, q_dt=orc.E5M2, do_dt=orc.E4M3, g_dt=orc.F16)
 
