@@ -85,9 +85,9 @@ enum {
 typedef struct scalify_array {
   void* data;        /* device pointer, 16-byte aligned */
   int32_t dtype;     /* scalify_dtype */
-  int32_t ndim;      /* 1..3 */
-  int64_t shape[3];  /* outermost first; unused entries ignored */
-  int64_t stride[3]; /* in elements; stride[ndim-1] must be 1 */
+  int32_t ndim;      /* 1..4 (4: only the attention calls, [batch, heads, T, hd]) */
+  int64_t shape[4];  /* outermost first; unused entries ignored */
+  int64_t stride[4]; /* in elements; stride[ndim-1] must be 1 */
   float* scale;      /* device pointer to one fp32 power of two, or NULL */
 } scalify_array;
 

@@ -40,7 +40,7 @@ class ScalifyError(RuntimeError):
 
 class scalify_array(ctypes.Structure):
     _fields_ = [("data", ctypes.c_void_p), ("dtype", ctypes.c_int32), ("ndim", ctypes.c_int32),
-                ("shape", ctypes.c_int64 * 3), ("stride", ctypes.c_int64 * 3), ("scale", ctypes.c_void_p)]
+                ("shape", ctypes.c_int64 * 4), ("stride", ctypes.c_int64 * 4), ("scale", ctypes.c_void_p)]
 
 
 class scalify_mx_array(ctypes.Structure):
@@ -141,8 +141,8 @@ def _desc(t: Optional[ScaledTensor]):
     cached = t.__dict__.get("_desc_cache")
     if cached is not None and cached[0] == key:
         return cached[1]
-    if d.dim() < 1 or d.dim() > 3:
-        raise ValueError("scalify arrays have 1 to 3 dimensions")
+    if d.dim() < 1 or d.dim() > 4:
+        raise ValueError("scalify arrays have 1 to 4 dimensions")
     a = scalify_array()
     a.data = d.data_ptr()
     a.dtype = _DTYPE_CODE[d.dtype]

@@ -39,14 +39,14 @@ constexpr int kAttTileBytes = kAttK * kAttHd;  // 8 KB: a Q, K or V tile
 constexpr size_t kAttSmem = size_t(kAttTileBytes) * 5 /*Q, 2 x K, 2 x V*/ + kAttQ * kAttK /*P*/ + 1024 + 256;
 
 struct AttParams {
-  int heads, Tq, Tk, q_blocks;
+  int heads, h_inner, Tq, Tk, q_blocks;   // heads = batch x h_inner
   int causal;
   const float* q_scale; const float* k_scale;
   float sc_const;   // kf(hd) c log2(e); times Q_s K_s: scores' data component -> exponent in base 2
   float inv_kf_hd;  // 1 / kf(hd)
   float inv_kf_tk;  // 1 / kf(Tk)
   uint32_t idesc_s, idesc_pv;
-  void* O; long long o_ld, o_hs;
+  void* O; long long o_ld, o_hs, o_bs;
   void* S_dump; void* P_dump;
   const float* v_scale; float kf_tk; float* o_scale;
   uint32_t* status;
@@ -95,6 +95,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   // query blocks in descending order within the launch: with a causal mask the late blocks have the most key
   // blocks, and starting them first leaves the short ones to fill the end of the launch
   const int qb = p.q_blocks - 1 - static_cast<int>(blockIdx.x / p.heads), head = blockIdx.x % p.heads;
+  const int hh = head % p.h_inner, bb = head / p.h_inner;  // head inside its batch element, batch element
   const int q0 = qb * kAttQ;
   const int shift = p.Tk - p.Tq;  // causal: query i sees keys j <= i + shift
   int n_kb = (p.Tk + kAttK - 1) / kAttK;
@@ -137,11 +138,11 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         const int kb = sweep_b ? it - n_kb : it;
         const uint32_t fb = kv_full + 8 * slot;
         mbar_expect_tx(fb, sweep_b ? 2 * kAttTileBytes : kAttTileBytes);
-        tma_load_3d(smem_k + slot * kAttTileBytes, &map_k, fb, 0, kb * kAttK, head);
-        if (sweep_b) tma_load_3d(smem_v + slot * kAttTileBytes, &map_v, fb, 0, kb * kAttK, head);
+        tma_load_4d(smem_k + slot * kAttTileBytes, &map_k, fb, 0, kb * kAttK, hh, bb);
+        if (sweep_b) tma_load_4d(smem_v + slot * kAttTileBytes, &map_v, fb, 0, kb * kAttK, hh, bb);
       };
       mbar_expect_tx(q_full, kAttTileBytes);
-      tma_load_3d(smem_q, &map_q, q_full, 0, q0, head);
+      tma_load_4d(smem_q, &map_q, q_full, 0, q0, hh, bb);
       issue_load(0);
       if (!timed_out && !mbar_wait(q_full, 0u, abort_flag)) timed_out = true;
       const uint64_t q_desc = make_smem_desc_sw64(smem_q, 512u);
@@ -313,7 +314,8 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           uint32_t o[32 * OSZ / 4];
           encode_vec<ODT, 32>(v, o);
           uint4* dst = reinterpret_cast<uint4*>(static_cast<char*>(p.O) +
-                                                (static_cast<long long>(head) * p.o_hs + static_cast<long long>(i) * p.o_ld +
+                                                (static_cast<long long>(bb) * p.o_bs + static_cast<long long>(hh) * p.o_hs +
+                                                 static_cast<long long>(i) * p.o_ld +
                                                  c * 32) * OSZ);
 #pragma unroll
           for (int q = 0; q < 32 * OSZ / 16; ++q) dst[q] = make_uint4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
@@ -335,20 +337,20 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
 
 int launch_attention(const AttentionArgs& a, cudaStream_t st) {
   CUtensorMap map_q, map_k, map_v;
-  int rc = make_byte_map(&map_q, a.Q, a.hd, a.Tq, a.heads, a.q_ld, a.q_hs, kAttHd, kAttQ);
+  int rc = make_byte_map4(&map_q, a.Q, a.hd, a.Tq, a.heads, a.batch, a.q_ld, a.q_hs, a.q_bs, kAttHd, kAttQ);
   if (rc) return rc;
-  rc = make_byte_map(&map_k, a.K, a.hd, a.Tk, a.heads, a.k_ld, a.k_hs, kAttHd, kAttK);
+  rc = make_byte_map4(&map_k, a.K, a.hd, a.Tk, a.heads, a.batch, a.k_ld, a.k_hs, a.k_bs, kAttHd, kAttK);
   if (rc) return rc;
-  rc = make_byte_map(&map_v, a.V, a.hd, a.Tk, a.heads, a.v_ld, a.v_hs, kAttHd, kAttK);
+  rc = make_byte_map4(&map_v, a.V, a.hd, a.Tk, a.heads, a.batch, a.v_ld, a.v_hs, a.v_bs, kAttHd, kAttK);
   if (rc) return rc;
   AttParams p;
-  p.heads = a.heads; p.Tq = a.Tq; p.Tk = a.Tk;
+  p.heads = a.heads * a.batch; p.h_inner = a.heads; p.Tq = a.Tq; p.Tk = a.Tk;
   p.q_blocks = (a.Tq + kAttQ - 1) / kAttQ;
   p.causal = a.causal;
   p.inv_kf_hd = 1.0f / kfactor(a.hd);
   p.kf_tk = kfactor(a.Tk);
   p.inv_kf_tk = 1.0f / p.kf_tk;
-  p.O = a.O; p.o_ld = a.o_ld; p.o_hs = a.o_hs;
+  p.O = a.O; p.o_ld = a.o_ld; p.o_hs = a.o_hs; p.o_bs = a.o_bs;
   p.S_dump = a.S_dump; p.P_dump = a.P_dump;
   p.v_scale = a.v_scale; p.o_scale = a.o_scale;
   p.status = a.status;
@@ -362,7 +364,7 @@ int launch_attention(const AttentionArgs& a, cudaStream_t st) {
   // kf(hd) and a power-of-two c only shift the exponent; the product with log2(e) rounds once, as in the
   // stand-alone softmax kernel
   p.sc_const = kfactor(a.hd) * a.sm_scale * 1.4426950408889634f;
-  const long long ctas = static_cast<long long>(a.heads) * p.q_blocks;
+  const long long ctas = static_cast<long long>(p.heads) * p.q_blocks;
   if (ctas > 0x7FFFFFFF) return SCALIFY_ERR_SHAPE;
   SCALIFY_DISPATCH_WIDE(a.o_dt, ODT, {
     auto kernel = attention_fwd_kernel<ODT>;

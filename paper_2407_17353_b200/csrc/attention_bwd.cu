@@ -42,7 +42,7 @@ constexpr int kBw1TmemCols = 256;
 constexpr uint32_t kBw1DqCol = 128;
 
 struct AttBwdParams {
-  int heads, Tq, Tk, q_blocks, k_blocks;
+  int heads, h_inner, Tq, Tk, q_blocks, k_blocks;   // heads = batch x h_inner
   int causal;
   float inv_kf_hd, inv_kf_tk, inv_kf_tq;
   float kf_hd, kf_tk, kf_tq, sm_scale;
@@ -50,9 +50,9 @@ struct AttBwdParams {
   const float* q_scale; const float* k_scale; const float* v_scale; const float* p_scale; const float* do_scale;
   float* ds_scale; float* dq_scale; float* dk_scale; float* dv_scale;
   void* dS; void* dP_dump;
-  void* dQ; long long dq_ld, dq_hs;
-  void* dK; long long dk_ld, dk_hs;
-  void* dV; long long dv_ld, dv_hs;
+  void* dQ; long long dq_ld, dq_hs, dq_bs;
+  void* dK; long long dk_ld, dk_hs, dk_bs;
+  void* dV; long long dv_ld, dv_hs, dv_bs;
   uint32_t* status;
 };
 
@@ -112,6 +112,7 @@ attention_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_do, const __grid
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // long (late) query blocks first, as in the forward kernel
   const int qb = p.q_blocks - 1 - static_cast<int>(blockIdx.x / p.heads), head = blockIdx.x % p.heads;
+  const int hh = head % p.h_inner, bb = head / p.h_inner;  // head inside its batch element, batch element
   const int q0 = qb * kBwQ;
   const int shift = p.Tk - p.Tq;  // causal: query i sees keys j <= i + shift
   int n_kb = p.k_blocks;
@@ -160,12 +161,12 @@ attention_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_do, const __grid
         const uint32_t fb = kv_full + 8 * slot;
         const uint32_t s0 = smem_slot + slot * kBw1Slot;
         mbar_expect_tx(fb, (sweep_b ? 2 * kBwTile : kBwTile) + kBwPTile);
-        tma_load_3d(s0, &map_v, fb, 0, kb * kBwK, head);
-        if (sweep_b) tma_load_3d(s0 + kBwTile, &map_k, fb, 0, kb * kBwK, head);
+        tma_load_4d(s0, &map_v, fb, 0, kb * kBwK, hh, bb);
+        if (sweep_b) tma_load_4d(s0 + kBwTile, &map_k, fb, 0, kb * kBwK, hh, bb);
         tma_load_3d(s0 + 2 * kBwTile, &map_p, fb, kb * kBwK, q0, head);
       };
       mbar_expect_tx(do_full, kBwTile);
-      tma_load_3d(smem_do, &map_do, do_full, 0, q0, head);
+      tma_load_4d(smem_do, &map_do, do_full, 0, q0, hh, bb);
       issue_load(0);
       if (!timed_out && !mbar_wait(do_full, 0u, abort_flag)) timed_out = true;
       const uint64_t do_desc = bw_desc_sw64(smem_do, 512u);
@@ -330,7 +331,8 @@ attention_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_do, const __grid
         uint32_t o[32 * GSZ / 4];
         encode_vec<GDT, 32>(v, o);
         uint4* dst = reinterpret_cast<uint4*>(static_cast<char*>(p.dQ) +
-                                              (static_cast<long long>(head) * p.dq_hs + static_cast<long long>(i) * p.dq_ld +
+                                              (static_cast<long long>(bb) * p.dq_bs + static_cast<long long>(hh) * p.dq_hs +
+                                               static_cast<long long>(i) * p.dq_ld +
                                                half * 32) * GSZ);
 #pragma unroll
         for (int q = 0; q < 32 * GSZ / 16; ++q) dst[q] = make_uint4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
@@ -380,6 +382,7 @@ attention_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // with a causal mask the early key blocks are seen by the most query blocks: they come first
   const int kb = static_cast<int>(blockIdx.x / p.heads), head = blockIdx.x % p.heads;
+  const int hh = head % p.h_inner, bb = head / p.h_inner;
   const int shift = p.Tk - p.Tq;
   const int i_min = p.causal ? max(0, kb * kBwK - shift) / kBw2Q : 0;  // first 64-query step that sees a key of this block
   const int n_qb = (p.Tq + kBw2Q - 1) / kBw2Q - i_min;
@@ -419,8 +422,8 @@ attention_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
         mbar_expect_tx(fb, kBw2Stage);
         tma_load_3d(s0, &map_p, fb, kb * kBwK, q0, head);
         tma_load_3d(s0 + kBw2PTile, &map_ds, fb, kb * kBwK, q0, head);
-        tma_load_3d(s0 + 2 * kBw2PTile, &map_do, fb, 0, q0, head);
-        tma_load_3d(s0 + 2 * kBw2PTile + kBw2Tile, &map_q, fb, 0, q0, head);
+        tma_load_4d(s0 + 2 * kBw2PTile, &map_do, fb, 0, q0, hh, bb);
+        tma_load_4d(s0 + 2 * kBw2PTile + kBw2Tile, &map_q, fb, 0, q0, hh, bb);
       }
     }
   } else if (warp == 1) {
@@ -469,8 +472,9 @@ attention_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
           uint32_t o[32 * GSZ / 4];
           encode_vec<GDT, 32>(v, o);
           char* out = c < 2 ? static_cast<char*>(p.dV) : static_cast<char*>(p.dK);
-          const long long hs = c < 2 ? p.dv_hs : p.dk_hs, ld = c < 2 ? p.dv_ld : p.dk_ld;
-          uint4* dst = reinterpret_cast<uint4*>(out + (static_cast<long long>(head) * hs + static_cast<long long>(j) * ld +
+          const long long hs = c < 2 ? p.dv_hs : p.dk_hs, ld = c < 2 ? p.dv_ld : p.dk_ld, bs = c < 2 ? p.dv_bs : p.dk_bs;
+          uint4* dst = reinterpret_cast<uint4*>(out + (static_cast<long long>(bb) * bs + static_cast<long long>(hh) * hs +
+                                                       static_cast<long long>(j) * ld +
                                                        (c & 1) * 32) * GSZ);
 #pragma unroll
           for (int q = 0; q < 32 * GSZ / 16; ++q) dst[q] = make_uint4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
@@ -498,19 +502,20 @@ attention_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
 int launch_attention_bwd(const AttentionBwdArgs& a, cudaStream_t st) {
   CUtensorMap map_k, map_v, map_do, map_p;
   int rc;
-  if ((rc = make_byte_map(&map_do, a.dO, a.hd, a.Tq, a.heads, a.do_ld, a.do_hs, kBwHd, kBwQ))) return rc;
-  if ((rc = make_byte_map(&map_k, a.K, a.hd, a.Tk, a.heads, a.k_ld, a.k_hs, kBwHd, kBwK))) return rc;
-  if ((rc = make_byte_map(&map_v, a.V, a.hd, a.Tk, a.heads, a.v_ld, a.v_hs, kBwHd, kBwK))) return rc;
+  const int all_heads = a.heads * a.batch;
+  if ((rc = make_byte_map4(&map_do, a.dO, a.hd, a.Tq, a.heads, a.batch, a.do_ld, a.do_hs, a.do_bs, kBwHd, kBwQ))) return rc;
+  if ((rc = make_byte_map4(&map_k, a.K, a.hd, a.Tk, a.heads, a.batch, a.k_ld, a.k_hs, a.k_bs, kBwHd, kBwK))) return rc;
+  if ((rc = make_byte_map4(&map_v, a.V, a.hd, a.Tk, a.heads, a.batch, a.v_ld, a.v_hs, a.v_bs, kBwHd, kBwK))) return rc;
   const uint64_t plane = static_cast<uint64_t>(a.Tq) * static_cast<uint64_t>(a.Tk);
-  if ((rc = make_byte_map(&map_p, a.P, a.Tk, a.Tq, a.heads, a.Tk, plane, kBwK, kBwQ))) return rc;
+  if ((rc = make_byte_map(&map_p, a.P, a.Tk, a.Tq, all_heads, a.Tk, plane, kBwK, kBwQ))) return rc;
   // launch 2 reads 64 queries per ring slot
   CUtensorMap map_p2, map_ds2, map_do2, map_q2;
-  if ((rc = make_byte_map(&map_p2, a.P, a.Tk, a.Tq, a.heads, a.Tk, plane, kBwK, kBw2Q))) return rc;
-  if ((rc = make_byte_map(&map_ds2, a.dS, a.Tk, a.Tq, a.heads, a.Tk, plane, kBwK, kBw2Q))) return rc;
-  if ((rc = make_byte_map(&map_do2, a.dO, a.hd, a.Tq, a.heads, a.do_ld, a.do_hs, kBwHd, kBw2Q))) return rc;
-  if ((rc = make_byte_map(&map_q2, a.Q, a.hd, a.Tq, a.heads, a.q_ld, a.q_hs, kBwHd, kBw2Q))) return rc;
+  if ((rc = make_byte_map(&map_p2, a.P, a.Tk, a.Tq, all_heads, a.Tk, plane, kBwK, kBw2Q))) return rc;
+  if ((rc = make_byte_map(&map_ds2, a.dS, a.Tk, a.Tq, all_heads, a.Tk, plane, kBwK, kBw2Q))) return rc;
+  if ((rc = make_byte_map4(&map_do2, a.dO, a.hd, a.Tq, a.heads, a.batch, a.do_ld, a.do_hs, a.do_bs, kBwHd, kBw2Q))) return rc;
+  if ((rc = make_byte_map4(&map_q2, a.Q, a.hd, a.Tq, a.heads, a.batch, a.q_ld, a.q_hs, a.q_bs, kBwHd, kBw2Q))) return rc;
   AttBwdParams p;
-  p.heads = a.heads; p.Tq = a.Tq; p.Tk = a.Tk;
+  p.heads = all_heads; p.h_inner = a.heads; p.Tq = a.Tq; p.Tk = a.Tk;
   p.q_blocks = (a.Tq + kBwQ - 1) / kBwQ;
   p.k_blocks = (a.Tk + kBwK - 1) / kBwK;
   p.causal = a.causal;
@@ -531,11 +536,11 @@ int launch_attention_bwd(const AttentionBwdArgs& a, cudaStream_t st) {
   p.q_scale = a.q_scale; p.k_scale = a.k_scale; p.v_scale = a.v_scale; p.p_scale = a.p_scale; p.do_scale = a.do_scale;
   p.ds_scale = a.ds_scale; p.dq_scale = a.dq_scale; p.dk_scale = a.dk_scale; p.dv_scale = a.dv_scale;
   p.dS = a.dS; p.dP_dump = a.dP_dump;
-  p.dQ = a.dQ; p.dq_ld = a.dq_ld; p.dq_hs = a.dq_hs;
-  p.dK = a.dK; p.dk_ld = a.dk_ld; p.dk_hs = a.dk_hs;
-  p.dV = a.dV; p.dv_ld = a.dv_ld; p.dv_hs = a.dv_hs;
+  p.dQ = a.dQ; p.dq_ld = a.dq_ld; p.dq_hs = a.dq_hs; p.dq_bs = a.dq_bs;
+  p.dK = a.dK; p.dk_ld = a.dk_ld; p.dk_hs = a.dk_hs; p.dk_bs = a.dk_bs;
+  p.dV = a.dV; p.dv_ld = a.dv_ld; p.dv_hs = a.dv_hs; p.dv_bs = a.dv_bs;
   p.status = a.status;
-  const long long ctas1 = static_cast<long long>(a.heads) * p.q_blocks, ctas2 = static_cast<long long>(a.heads) * p.k_blocks;
+  const long long ctas1 = static_cast<long long>(p.heads) * p.q_blocks, ctas2 = static_cast<long long>(p.heads) * p.k_blocks;
   if (ctas1 > 0x7FFFFFFF || ctas2 > 0x7FFFFFFF) return SCALIFY_ERR_SHAPE;
   SCALIFY_DISPATCH_WIDE(a.g_dt, GDT, {
     auto k1 = attention_bwd_dq_kernel<GDT>;

@@ -638,6 +638,28 @@ int make_byte_map(CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t ro
   return SCALIFY_OK;
 }
 
+// The same for [batch][heads][rows][inner] views (attention operands): box = one tile of one head
+int make_byte_map4(CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t rows, uint64_t heads, uint64_t batch,
+                   uint64_t ld, uint64_t hs, uint64_t bs, uint32_t box_inner, uint32_t box_rows) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return SCALIFY_ERR_CUDA;
+  cuuint64_t dims[4] = {inner, rows, heads, batch};
+  const uint64_t hs_eff = hs ? hs : ld * rows;
+  cuuint64_t strides[3] = {ld, hs_eff, bs ? bs : hs_eff * heads};
+  cuuint32_t box[4] = {box_inner, box_rows, 1u, 1u};
+  cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+  const CUtensorMapSwizzle sw = box_inner == 32 ? CU_TENSOR_MAP_SWIZZLE_32B
+                              : box_inner == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B;
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    set_last_cuda_error(static_cast<int>(r));
+    return SCALIFY_ERR_CUDA;
+  }
+  return SCALIFY_OK;
+}
+
 // Tensor map of the output [batch][M][N] (row stride ld, batch stride bs, in elements of `es` bytes) for the
 // epilogue's stores: box 32 columns x 32 rows, swizzle equal to the width of a box row (32 / 64 / 128 bytes).
 static int make_map_y(CUtensorMap* map, const void* ptr, int es, uint64_t N, uint64_t M, uint64_t batch, uint64_t ld,

@@ -31,7 +31,7 @@ int sm_count() {
 int check_array(const scalify_array* a) {
   if (!a || !a->data) return SCALIFY_ERR_NULL;
   if (!valid_dtype(a->dtype)) return SCALIFY_ERR_DTYPE;
-  if (a->ndim < 1 || a->ndim > 3) return SCALIFY_ERR_SHAPE;
+  if (a->ndim < 1 || a->ndim > 4) return SCALIFY_ERR_SHAPE;
   for (int i = 0; i < a->ndim; ++i)
     if (a->shape[i] < 0 || a->shape[i] > (int64_t(1) << 40)) return SCALIFY_ERR_SHAPE;
   if (a->stride[a->ndim - 1] != 1) return SCALIFY_ERR_ALIGNMENT;
@@ -400,11 +400,20 @@ int scalify_mx_matmul(const scalify_mx_array* A, const scalify_mx_array* B, scal
   return launch_mx_matmul(a, workspace, static_cast<cudaStream_t>(stream));
 }
 
-// [heads, T, hd] view of a 2-D or 3-D array: head count, rows, row and head strides (elements)
-static int as_heads(const scalify_array* a, int64_t* heads, int64_t* rows, int64_t* cols, int64_t* ld, int64_t* hs) {
-  if (a->ndim == 2) { *heads = 1; *rows = a->shape[0]; *cols = a->shape[1]; *ld = a->stride[0]; *hs = 0; return SCALIFY_OK; }
+// [batch, heads, T, hd] view of a 2-D, 3-D or 4-D array: counts, rows, row / head / batch strides (elements)
+struct HeadsView {
+  int64_t batch, heads, rows, cols, ld, hs, bs;
+};
+static int as_heads(const scalify_array* a, HeadsView* v) {
+  v->batch = 1; v->heads = 1; v->hs = 0; v->bs = 0;
+  if (a->ndim == 2) { v->rows = a->shape[0]; v->cols = a->shape[1]; v->ld = a->stride[0]; return SCALIFY_OK; }
   if (a->ndim == 3) {
-    *heads = a->shape[0]; *rows = a->shape[1]; *cols = a->shape[2]; *ld = a->stride[1]; *hs = a->stride[0];
+    v->heads = a->shape[0]; v->rows = a->shape[1]; v->cols = a->shape[2]; v->ld = a->stride[1]; v->hs = a->stride[0];
+    return SCALIFY_OK;
+  }
+  if (a->ndim == 4) {
+    v->batch = a->shape[0]; v->heads = a->shape[1]; v->rows = a->shape[2]; v->cols = a->shape[3];
+    v->ld = a->stride[2]; v->hs = a->stride[1]; v->bs = a->stride[0];
     return SCALIFY_OK;
   }
   return SCALIFY_ERR_SHAPE;
@@ -418,14 +427,18 @@ int scalify_scaled_attention(const scalify_array* Q, const scalify_array* K, con
   if (is_wide(Q->dtype) || is_wide(K->dtype) || is_wide(V->dtype) || !is_wide(O->dtype)) return SCALIFY_ERR_DTYPE;
   if (!isfinite(sm_scale)) return SCALIFY_ERR_VALUE;
   AttentionArgs a;
-  int64_t hq, hk, hv, ho, tq, tk, tv, to, dq, dk, dv, dout;
-  if ((rc = as_heads(Q, &hq, &tq, &dq, &a.q_ld, &a.q_hs)) || (rc = as_heads(K, &hk, &tk, &dk, &a.k_ld, &a.k_hs)) ||
-      (rc = as_heads(V, &hv, &tv, &dv, &a.v_ld, &a.v_hs)) || (rc = as_heads(O, &ho, &to, &dout, &a.o_ld, &a.o_hs)))
-    return rc;
-  if (hq != hk || hq != hv || hq != ho || tk != tv || tq != to || dq != dk || dq != dv || dq != dout)
+  HeadsView vq, vk, vv, vo;
+  if ((rc = as_heads(Q, &vq)) || (rc = as_heads(K, &vk)) || (rc = as_heads(V, &vv)) || (rc = as_heads(O, &vo))) return rc;
+  if (vq.batch != vk.batch || vq.batch != vv.batch || vq.batch != vo.batch || vq.heads != vk.heads ||
+      vq.heads != vv.heads || vq.heads != vo.heads || vk.rows != vv.rows || vq.rows != vo.rows || vq.cols != vk.cols ||
+      vq.cols != vv.cols || vq.cols != vo.cols)
     return SCALIFY_ERR_SHAPE;
-  if (tq < 1 || tk < 1 || hq < 1 || tq > 0x7FFFFFFF || tk > 0x7FFFFFFF || hq > 0x7FFFFFFF) return SCALIFY_ERR_SHAPE;
-  if (dq != 64 || (causal && tk < tq)) return SCALIFY_ERR_UNSUPPORTED;
+  const int64_t tq = vq.rows, tk = vk.rows, hq = vq.batch * vq.heads;
+  if (tq < 1 || tk < 1 || vq.heads < 1 || vq.batch < 1 || tq > 0x7FFFFFFF || tk > 0x7FFFFFFF || hq > 0x7FFFFFFF)
+    return SCALIFY_ERR_SHAPE;
+  if (vq.cols != 64 || (causal && tk < tq)) return SCALIFY_ERR_UNSUPPORTED;
+  a.q_ld = vq.ld; a.q_hs = vq.hs; a.q_bs = vq.bs; a.k_ld = vk.ld; a.k_hs = vk.hs; a.k_bs = vk.bs;
+  a.v_ld = vv.ld; a.v_hs = vv.hs; a.v_bs = vv.bs; a.o_ld = vo.ld; a.o_hs = vo.hs; a.o_bs = vo.bs;
   if (O->scale && (O->scale == Q->scale || O->scale == K->scale || O->scale == V->scale)) return SCALIFY_ERR_ALIAS;
   a.S_dump = nullptr;
   a.P_dump = nullptr;
@@ -444,7 +457,8 @@ int scalify_scaled_attention(const scalify_array* Q, const scalify_array* K, con
   a.Q = Q->data; a.K = K->data; a.V = V->data;
   a.q_dt = Q->dtype; a.k_dt = K->dtype; a.v_dt = V->dtype;
   a.O = O->data; a.o_dt = O->dtype;
-  a.heads = static_cast<int>(hq); a.Tq = static_cast<int>(tq); a.Tk = static_cast<int>(tk); a.hd = 64;
+  a.batch = static_cast<int>(vq.batch); a.heads = static_cast<int>(vq.heads);
+  a.Tq = static_cast<int>(tq); a.Tk = static_cast<int>(tk); a.hd = 64;
   a.causal = causal ? 1 : 0;
   a.sm_scale = sm_scale;
   a.q_scale = Q->scale; a.k_scale = K->scale; a.v_scale = V->scale; a.o_scale = O->scale;
@@ -468,17 +482,22 @@ int scalify_scaled_attention_bwd(const scalify_array* Q, const scalify_array* K,
   int ex = 0;
   if (!(sm_scale > 0.f) || !isfinite(sm_scale) || frexpf(sm_scale, &ex) != 0.5f) return SCALIFY_ERR_UNSUPPORTED;
   AttentionBwdArgs a;
-  int64_t hq, hk, hv, hdo, h1, h2, h3, tq, tk, tv, tdo, t1, t2, t3, dq, dk, dv, ddo, d1, d2, d3;
-  if ((rc = as_heads(Q, &hq, &tq, &dq, &a.q_ld, &a.q_hs)) || (rc = as_heads(K, &hk, &tk, &dk, &a.k_ld, &a.k_hs)) ||
-      (rc = as_heads(V, &hv, &tv, &dv, &a.v_ld, &a.v_hs)) || (rc = as_heads(dO, &hdo, &tdo, &ddo, &a.do_ld, &a.do_hs)) ||
-      (rc = as_heads(dQ, &h1, &t1, &d1, &a.dq_ld, &a.dq_hs)) || (rc = as_heads(dK, &h2, &t2, &d2, &a.dk_ld, &a.dk_hs)) ||
-      (rc = as_heads(dV, &h3, &t3, &d3, &a.dv_ld, &a.dv_hs)))
+  HeadsView vq, vk, vv, vdo, v1, v2, v3;
+  if ((rc = as_heads(Q, &vq)) || (rc = as_heads(K, &vk)) || (rc = as_heads(V, &vv)) || (rc = as_heads(dO, &vdo)) ||
+      (rc = as_heads(dQ, &v1)) || (rc = as_heads(dK, &v2)) || (rc = as_heads(dV, &v3)))
     return rc;
-  if (hq != hk || hq != hv || hq != hdo || hq != h1 || hq != h2 || hq != h3) return SCALIFY_ERR_SHAPE;
-  if (tk != tv || tq != tdo || tq != t1 || tk != t2 || tk != t3) return SCALIFY_ERR_SHAPE;
-  if (dq != dk || dq != dv || dq != ddo || dq != d1 || dq != d2 || dq != d3) return SCALIFY_ERR_SHAPE;
-  if (tq < 1 || tk < 1 || hq < 1 || tq > 0x7FFFFFFF || tk > 0x7FFFFFFF || hq > 0x7FFFFFFF) return SCALIFY_ERR_SHAPE;
-  if (dq != 64 || (causal && tk < tq)) return SCALIFY_ERR_UNSUPPORTED;
+  const HeadsView* all[7] = {&vq, &vk, &vv, &vdo, &v1, &v2, &v3};
+  for (int i = 1; i < 7; ++i)
+    if (all[i]->batch != vq.batch || all[i]->heads != vq.heads || all[i]->cols != vq.cols) return SCALIFY_ERR_SHAPE;
+  const int64_t tq = vq.rows, tk = vk.rows, hq = vq.batch * vq.heads;
+  if (vv.rows != tk || vdo.rows != tq || v1.rows != tq || v2.rows != tk || v3.rows != tk) return SCALIFY_ERR_SHAPE;
+  if (tq < 1 || tk < 1 || vq.heads < 1 || vq.batch < 1 || tq > 0x7FFFFFFF || tk > 0x7FFFFFFF || hq > 0x7FFFFFFF)
+    return SCALIFY_ERR_SHAPE;
+  if (vq.cols != 64 || (causal && tk < tq)) return SCALIFY_ERR_UNSUPPORTED;
+  a.q_ld = vq.ld; a.q_hs = vq.hs; a.q_bs = vq.bs; a.k_ld = vk.ld; a.k_hs = vk.hs; a.k_bs = vk.bs;
+  a.v_ld = vv.ld; a.v_hs = vv.hs; a.v_bs = vv.bs; a.do_ld = vdo.ld; a.do_hs = vdo.hs; a.do_bs = vdo.bs;
+  a.dq_ld = v1.ld; a.dq_hs = v1.hs; a.dq_bs = v1.bs; a.dk_ld = v2.ld; a.dk_hs = v2.hs; a.dk_bs = v2.bs;
+  a.dv_ld = v3.ld; a.dv_hs = v3.hs; a.dv_bs = v3.bs;
   if (tk % 32 != 0) return SCALIFY_ERR_SHAPE;  // rows of P and dS are read and written in 32-byte pieces
   if (contiguous_numel(P) != hq * tq * tk || contiguous_numel(dS) != hq * tq * tk) return SCALIFY_ERR_SHAPE;
   const float* in_scales[5] = {Q->scale, K->scale, V->scale, P->scale, dO->scale};
@@ -501,7 +520,8 @@ int scalify_scaled_attention_bwd(const scalify_array* Q, const scalify_array* K,
   a.q_dt = Q->dtype; a.k_dt = K->dtype; a.v_dt = V->dtype; a.do_dt = dO->dtype;
   a.P = P->data; a.dS = dS->data;
   a.dQ = dQ->data; a.dK = dK->data; a.dV = dV->data; a.g_dt = dQ->dtype;
-  a.heads = static_cast<int>(hq); a.Tq = static_cast<int>(tq); a.Tk = static_cast<int>(tk); a.hd = 64;
+  a.batch = static_cast<int>(vq.batch); a.heads = static_cast<int>(vq.heads);
+  a.Tq = static_cast<int>(tq); a.Tk = static_cast<int>(tk); a.hd = 64;
   a.causal = causal ? 1 : 0;
   a.sm_scale = sm_scale;
   a.q_scale = Q->scale; a.k_scale = K->scale; a.v_scale = V->scale; a.p_scale = P->scale; a.do_scale = dO->scale;
@@ -597,7 +617,7 @@ static int matmul_impl(const scalify_array* A, int transA, const scalify_array* 
   if (rc) return rc;
   if (!is_fp8(A->dtype) || !is_fp8(B->dtype) || !is_wide(Y->dtype)) return SCALIFY_ERR_DTYPE;
   if (!valid_stat(stat)) return SCALIFY_ERR_VALUE;
-  if (A->ndim < 2 || B->ndim < 2 || Y->ndim != A->ndim || B->ndim > A->ndim) return SCALIFY_ERR_SHAPE;
+  if (A->ndim < 2 || A->ndim > 3 || B->ndim < 2 || Y->ndim != A->ndim || B->ndim > A->ndim) return SCALIFY_ERR_SHAPE;
   const int an = A->ndim, bn = B->ndim, yn = Y->ndim;
   const int64_t batch = an == 3 ? A->shape[0] : 1;
   const int64_t M = transA ? A->shape[an - 1] : A->shape[an - 2];
@@ -688,7 +708,7 @@ int scalify_scaled_matmul_delayed(const scalify_array* A, int transA, const scal
   if (!is_fp8(A->dtype) || !is_fp8(B->dtype)) return SCALIFY_ERR_DTYPE;
   if (!valid_stat(stat)) return SCALIFY_ERR_VALUE;
   if (stat == SCALIFY_STAT_NONE && stat_out) return SCALIFY_ERR_VALUE;
-  if (A->ndim < 2 || B->ndim < 2 || Y->ndim != A->ndim || B->ndim > A->ndim) return SCALIFY_ERR_SHAPE;
+  if (A->ndim < 2 || A->ndim > 3 || B->ndim < 2 || Y->ndim != A->ndim || B->ndim > A->ndim) return SCALIFY_ERR_SHAPE;
   const int an = A->ndim, bn = B->ndim, yn = Y->ndim;
   const int64_t batch = an == 3 ? A->shape[0] : 1;
   const int64_t M = transA ? A->shape[an - 1] : A->shape[an - 2];

@@ -13,6 +13,8 @@ namespace scalify {
 
 int make_byte_map(CUtensorMap_st* map, const void* ptr, uint64_t inner, uint64_t rows, uint64_t batch, uint64_t ld,
                   uint64_t bs, uint32_t box_inner, uint32_t box_rows);
+int make_byte_map4(CUtensorMap_st* map, const void* ptr, uint64_t inner, uint64_t rows, uint64_t heads, uint64_t batch,
+                   uint64_t ld, uint64_t hs, uint64_t bs, uint32_t box_inner, uint32_t box_rows);
 
 enum { kModeCast = 0, kModeDynamic = 1, kModeSet = 2 };
 
@@ -93,8 +95,9 @@ size_t mx_sf_bytes(int64_t rows, int64_t K);
 struct AttentionArgs {
   const void* Q; const void* K; const void* V; int q_dt, k_dt, v_dt;   // FP8 [heads, T, hd] views
   int64_t q_ld, q_hs, k_ld, k_hs, v_ld, v_hs;                         // row and head strides in elements
+  int64_t q_bs, k_bs, v_bs, o_bs;                                     // batch strides in elements
   void* O; int o_dt; int64_t o_ld, o_hs;                              // [heads, Tq, hd], F16 / BF16
-  int heads, Tq, Tk, hd;
+  int batch, heads, Tq, Tk, hd;                                       // heads per batch element
   int causal;
   float sm_scale;
   const float* q_scale; const float* k_scale; const float* v_scale; float* o_scale;
@@ -107,11 +110,12 @@ int launch_attention(const AttentionArgs& a, cudaStream_t st);
 struct AttentionBwdArgs {
   const void* Q; const void* K; const void* V; const void* dO; int q_dt, k_dt, v_dt, do_dt;  // FP8 [heads, T, hd] views
   int64_t q_ld, q_hs, k_ld, k_hs, v_ld, v_hs, do_ld, do_hs;                                  // strides in elements
+  int64_t q_bs, k_bs, v_bs, do_bs, dq_bs, dk_bs, dv_bs;                                      // batch strides
   const void* P;   // E4M3 [heads, Tq, Tk] dense: the probabilities the forward pass used
   void* dS;        // E5M2 [heads, Tq, Tk] dense (output, and operand of the dK product)
   void* dQ; void* dK; void* dV; int g_dt;   // F16 / BF16 / F32 [heads, T, hd] views
   int64_t dq_ld, dq_hs, dk_ld, dk_hs, dv_ld, dv_hs;
-  int heads, Tq, Tk, hd;
+  int batch, heads, Tq, Tk, hd;   // heads per batch element
   int causal;
   float sm_scale;  // a power of two
   const float* q_scale; const float* k_scale; const float* v_scale; const float* p_scale; const float* do_scale;

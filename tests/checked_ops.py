@@ -233,20 +233,23 @@ class Ops:
     def attention(self, Q, K, V, O, sm_scale, causal=True):
         """Fused forward over [heads, T, 64] views; returns the E4M3 probabilities (kept for the backward).
         Checked stage by stage through the kernel's own copies of the scores and probabilities."""
-        H, Tq, _ = Q.data.shape
-        Tk = K.data.shape[1]
-        P = sc.ScaledTensor(torch.zeros((H, Tq, Tk), dtype=torch.uint8, device=Q.data.device).view(torch.float8_e4m3fn),
+        lead, Tq, Tk = tuple(Q.data.shape[:-2]), Q.data.shape[-2], K.data.shape[-2]   # [heads] or [batch, heads]
+        H = int(np.prod(lead))
+        # (the blocks wholly above the diagonal are never written nor read: zeroed only for the checks below)
+        alloc = torch.zeros if self.check else torch.empty
+        P = sc.ScaledTensor(alloc(lead + (Tq, Tk), dtype=torch.uint8, device=Q.data.device).view(torch.float8_e4m3fn),
                             torch.ones(1, dtype=torch.float32, device=Q.data.device))
         Sd = None
         if self.check:
-            Sd = sc.ScaledTensor(torch.zeros((H, Tq, Tk), dtype=torch.bfloat16, device=Q.data.device), None)
+            Sd = sc.ScaledTensor(torch.zeros(lead + (Tq, Tk), dtype=torch.bfloat16, device=Q.data.device), None)
         sc.scalify_scaled_attention(Q, K, V, O, sm_scale=sm_scale, causal=causal, S_dump=Sd, P_dump=P)
         self.calls += 1
         if self.check:
             o = self.orc
             q_dt, k_dt, v_dt, o_dt = code(Q.data), code(K.data), code(V.data), code(O.data)
-            qb, kb, vb = self.bits(Q), self.bits(K), self.bits(V)
-            Sg, Pg, Og = self.bits(Sd), self.bits(P), self.bits(sc.ScaledTensor(O.data.contiguous(), None))
+            flat = lambda a: a.reshape((H,) + a.shape[-2:])
+            qb, kb, vb = flat(self.bits(Q)), flat(self.bits(K)), flat(self.bits(V))
+            Sg, Pg, Og = flat(self.bits(Sd)), flat(self.bits(P)), flat(self.bits(sc.ScaledTensor(O.data.contiguous(), None)))
             ii, jj = np.meshgrid(np.arange(Tq), np.arange(Tk), indexing="ij")
             vis = (jj <= ii + (Tk - Tq)) if causal else np.ones((Tq, Tk), dtype=bool)
             for h in range(H):
@@ -264,22 +267,24 @@ class Ops:
     def attention_bwd(self, Q, K, V, P, dO, dQ, dK, dV, sm_scale, causal=True):
         """Fused backward over [heads, T, 64] views: dQ, dK, dV are written in place (their scale words too).
         Checked stage by stage through the kernel's own dP copy and its dS output."""
-        H, Tq, _ = Q.data.shape
-        Tk = K.data.shape[1]
+        lead, Tq, Tk = tuple(Q.data.shape[:-2]), Q.data.shape[-2], K.data.shape[-2]
+        H = int(np.prod(lead))
         dev = Q.data.device
-        dS = sc.ScaledTensor(torch.zeros((H, Tq, Tk), dtype=torch.uint8, device=dev).view(torch.float8_e5m2),
-                             torch.zeros(1, dtype=torch.float32, device=dev))
+        alloc = torch.zeros if self.check else torch.empty
+        dS = sc.ScaledTensor(alloc(lead + (Tq, Tk), dtype=torch.uint8, device=dev).view(torch.float8_e5m2),
+                             torch.empty(1, dtype=torch.float32, device=dev))
         dPd = None
         if self.check:
-            dPd = sc.ScaledTensor(torch.zeros((H, Tq, Tk), dtype=torch.bfloat16, device=dev), None)
+            dPd = sc.ScaledTensor(torch.zeros(lead + (Tq, Tk), dtype=torch.bfloat16, device=dev), None)
         sc.scalify_scaled_attention_bwd(Q, K, V, P, dO, dS, dQ, dK, dV, sm_scale=sm_scale, causal=causal, dP_dump=dPd)
         self.calls += 1
         if self.check:
             o = self.orc
             q_dt, k_dt, v_dt, g_in, g_dt = code(Q.data), code(K.data), code(V.data), code(dO.data), code(dQ.data)
-            qb, kb, vb, gb, pb = self.bits(Q), self.bits(K), self.bits(V), self.bits(dO), self.bits(P)
-            dPg, dSg = self.bits(dPd), self.bits(dS)
-            dQg, dKg, dVg = (self.bits(sc.ScaledTensor(t.data.contiguous(), None)) for t in (dQ, dK, dV))
+            flat = lambda a: a.reshape((H,) + a.shape[-2:])
+            qb, kb, vb, gb, pb = (flat(self.bits(t)) for t in (Q, K, V, dO, P))
+            dPg, dSg = flat(self.bits(dPd)), flat(self.bits(dS))
+            dQg, dKg, dVg = (flat(self.bits(sc.ScaledTensor(t.data.contiguous(), None))) for t in (dQ, dK, dV))
             ii, jj = np.meshgrid(np.arange(Tq), np.arange(Tk), indexing="ij")
             shift = Tk - Tq
             vis = ((jj // 128) * 128 <= (ii // 128) * 128 + 127 + shift) if causal else np.ones((Tq, Tk), dtype=bool)

@@ -90,6 +90,12 @@ class ScaledGPT:
         t = X.data[b * c.seq:(b + 1) * c.seq].view(c.seq, c.heads, hd).permute(1, 0, 2)
         return sc.ScaledTensor(t, X.scale)
 
+    def _heads4(self, X):
+        """[B, H, T, hd] view of a [n, d] tensor (batch stride T*d, head stride hd, row stride d)."""
+        c = self.cfg
+        hd = c.d // c.heads
+        return sc.ScaledTensor(X.data.view(c.batch, c.seq, c.heads, hd).permute(0, 2, 1, 3), X.scale)
+
     def _linear(self, x8, W8, bias):
         y = self.ops.mm(x8, W8)                       # [n, K] x [K, N], B stored [K, N]
         return self.ops.add(y, self.ops.cast(bias, BF))
@@ -126,19 +132,20 @@ class ScaledGPT:
             att.scale = None
             s["P8"] = []
             att_scale = None
-            for b in range(B):
+            if hd == 64:
+                # Q K^T, 1/sqrt(hd), causal softmax and P V of all sequences and heads in one kernel; the
+                # probabilities it used are kept for the backward pass
+                Oall = sc.ScaledTensor(self._heads4(sc.ScaledTensor(att.data, None)).data,
+                                       torch.empty(1, dtype=torch.float32, device=self.dev))
+                s["P8"] = o.attention(self._heads4(q8), self._heads4(k8), self._heads4(v8), Oall, 1.0 / float(np.sqrt(hd)))
+                att_scale = Oall.scale
+            for b in range(B if hd != 64 else 0):
                 Ob = sc.ScaledTensor(self._heads(sc.ScaledTensor(att.data, None), b).data,
                                      torch.empty(1, dtype=torch.float32, device=self.dev))
-                if hd == 64:
-                    # Q K^T, 1/sqrt(hd), causal softmax and P V in one kernel; the probabilities it used are
-                    # kept for the backward pass
-                    Pb = o.attention(self._heads(q8, b), self._heads(k8, b), self._heads(v8, b), Ob,
-                                     1.0 / float(np.sqrt(hd)))
-                else:
-                    S = o.mm(self._heads(q8, b), self._heads(k8, b), transB=True)    # [H, T, T]
-                    o.scalar_mul(S, 1.0 / float(np.sqrt(hd)))                       # 1/sqrt(hd), a power of two here
-                    Pb = o.softmax(S, True, E4)
-                    o.mm(Pb, self._heads(v8, b), Y=Ob)                               # written into the merged layout
+                S = o.mm(self._heads(q8, b), self._heads(k8, b), transB=True)        # [H, T, T]
+                o.scalar_mul(S, 1.0 / float(np.sqrt(hd)))                           # 1/sqrt(hd), a power of two here
+                Pb = o.softmax(S, True, E4)
+                o.mm(Pb, self._heads(v8, b), Y=Ob)                                   # written into the merged layout
                 s["P8"].append(Pb)
                 att_scale = Ob.scale  # identical for every b: static rule
             att = sc.ScaledTensor(att.data, att_scale)
@@ -176,15 +183,16 @@ class ScaledGPT:
             datt, grads[p + "wo"], grads[p + "bo"] = self._linear_bwd(dx, s["o8"], W8[p + "wo"])
             datt8 = o.cast(datt, E5)
             dq, dk, dv = (o.empty((n, d), BF) for _ in range(3))
-            for b in range(B):
+            if hd == 64:
+                # dO V^T, the softmax backward, 1/sqrt(hd) and the three gradient products of all sequences and
+                # heads in two launches
+                view4 = lambda Tn: sc.ScaledTensor(self._heads4(sc.ScaledTensor(Tn.data, None)).data, Tn.scale)
+                o.attention_bwd(self._heads4(s["q8"]), self._heads4(s["k8"]), self._heads4(s["v8"]), s["P8"],
+                                self._heads4(datt8), view4(dq), view4(dk), view4(dv), 1.0 / float(np.sqrt(hd)))
+            for b in range(B if hd != 64 else 0):
                 Pb = s["P8"][b]
                 dOb = self._heads(datt8, b)
                 view = lambda Tn: sc.ScaledTensor(self._heads(sc.ScaledTensor(Tn.data, None), b).data, Tn.scale)
-                if hd == 64:
-                    # dO V^T, the softmax backward, 1/sqrt(hd) and the three gradient products in two launches
-                    o.attention_bwd(self._heads(s["q8"], b), self._heads(s["k8"], b), self._heads(s["v8"], b), Pb, dOb,
-                                    view(dq), view(dk), view(dv), 1.0 / float(np.sqrt(hd)))
-                    continue
                 dPb = o.mm(dOb, self._heads(s["v8"], b), transB=True)                # dO V^T  [H, T, T]
                 o.mm(Pb, dOb, transA=True, Y=view(dv))                               # P^T dO  [H, T, hd]
                 dSb = o.softmax_bwd(dPb, Pb, E5)

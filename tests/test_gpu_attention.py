@@ -113,3 +113,40 @@ def test_argument_checks():
     O = sc.ScaledTensor.empty((2, 256, 64), torch.bfloat16)
     with pytest.raises(sc.ScalifyError):
         sc.scalify_scaled_attention(Q, K, K, O, sm_scale=0.125, causal=True)   # causal with fewer keys than queries
+
+
+def test_batch_of_sequences_as_a_4d_view_equals_one_call_per_sequence():
+    """[batch, heads, T, 64] views of token-major buffers [batch * T, heads * 64] (the layout the QKV projection
+    writes): one call over the 4-D views must reproduce, bit for bit, one call per sequence; forward and backward."""
+    B, H, T = 3, 4, 256
+    d = H * HD
+    g = torch.Generator(device="cuda").manual_seed(3)
+    rnd = lambda dt: torch.randn((B * T, d), device="cuda", generator=g).to(dt)
+    q, k, v, do = rnd(torch.float8_e4m3fn), rnd(torch.float8_e4m3fn), rnd(torch.float8_e4m3fn), rnd(torch.float8_e5m2)
+    scales = (0.5, 2.0, 0.125, 2.0 ** -9)
+
+    def views(x, b=None):   # [B, H, T, HD] view, or [H, T, HD] of sequence b
+        x4 = x.view(B, T, H, HD).permute(0, 2, 1, 3)
+        return x4 if b is None else x4[b]
+
+    def run(batched):
+        out = {n: torch.zeros((B * T, d), dtype=torch.bfloat16, device="cuda") for n in ("o", "dq", "dk", "dv")}
+        sw = {n: torch.zeros(1, device="cuda") for n in ("o", "ds", "dq", "dk", "dv")}
+        P = torch.zeros((B, H, T, T), dtype=torch.uint8, device="cuda").view(torch.float8_e4m3fn)
+        dS = torch.zeros((B, H, T, T), dtype=torch.uint8, device="cuda").view(torch.float8_e5m2)
+        ones = torch.ones(1, device="cuda")
+        for b in ([None] if batched else range(B)):
+            Q, K, V, dO = (sc.ScaledTensor.make(views(x, b), s) for x, s in zip((q, k, v, do), scales))
+            O, dQ, dK, dV = (sc.ScaledTensor(views(out[n], b), sw[n]) for n in ("o", "dq", "dk", "dv"))
+            Pb = sc.ScaledTensor(P if b is None else P[b], ones)
+            dSb = sc.ScaledTensor(dS if b is None else dS[b], sw["ds"])
+            sc.scalify_scaled_attention(Q, K, V, O, sm_scale=0.125, causal=True, P_dump=Pb)
+            sc.scalify_scaled_attention_bwd(Q, K, V, Pb, dO, dSb, dQ, dK, dV, sm_scale=0.125, causal=True)
+        torch.cuda.synchronize()
+        return ([out[n].view(torch.int16).cpu().numpy() for n in out] + [P.view(torch.uint8).cpu().numpy(),
+                dS.view(torch.uint8).cpu().numpy()], [float(sw[n].item()) for n in sw])
+    one, s_one = run(True)
+    per, s_per = run(False)
+    assert s_one == s_per
+    for a, b in zip(one, per):
+        assert np.array_equal(a, b)
