@@ -98,7 +98,8 @@ enum {
   SCALIFY_OP_LAYERNORM_BWD = 2, /* d0 = rows, d1 = row length */
   SCALIFY_OP_ADAM = 3,          /* d0 = number of tensors, d1 unused */
   SCALIFY_OP_STATISTIC = 4,     /* d0 = number of elements */
-  SCALIFY_OP_CROSS_ENTROPY = 5  /* d0 = number of rows */
+  SCALIFY_OP_CROSS_ENTROPY = 5, /* d0 = number of rows */
+  SCALIFY_OP_COLSUM = 6         /* d0 = rows, d1 = columns */
 };
 
 /* Bytes of workspace the given call needs (an upper bound; always >= 4096).
@@ -445,6 +446,20 @@ int scalify_mx_quantize(const scalify_array* X, scalify_mx_array* Y, uint32_t* s
  */
 int scalify_mx_matmul(const scalify_mx_array* A, const scalify_mx_array* B, scalify_array* Y, int stat,
                       void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Column sums of a scaled matrix: Y[j] = sum over the R rows of X[r, j], by the
+ * rule for a sum of R independent terms (Section 3.2; the same rule as a matmul
+ * with a ones operand and K = R, and as the dbeta of the LayerNorm backward):
+ *   Y_s = X_s kf(R),   Y_d[j] = (sum_r X_d[r, j]) / kf(R)
+ * This is the bias gradient of a linear layer.  X: any dtype, [R, N] (row stride
+ * stride[0]); Y: F16, BF16 or F32, [N] contiguous.  Partial sums are fp32 per slab
+ * of rows, the slabs are added in fp64 in a fixed order (results do not depend on
+ * scheduling).  Workspace: SCALIFY_OP_COLSUM (R, N).
+ * Errors: NULL, DTYPE, SHAPE, ALIGNMENT, WORKSPACE, ALIAS.
+ */
+int scalify_scaled_colsum(const scalify_array* X, scalify_array* Y, void* workspace, size_t workspace_bytes,
+                          void* stream);
 
 /*
  * Fused scaled attention forward: S = Q K^T, P = softmax(S c), O = P V in one

@@ -22,7 +22,7 @@ from . import _build
 
 E4M3, E5M2, F16, BF16, F32 = 0, 1, 2, 3, 4
 STAT_NONE, STAT_AMAX, STAT_L2 = 0, 1, 2
-OP_MATMUL, OP_RESCALE, OP_LAYERNORM_BWD, OP_ADAM, OP_STATISTIC, OP_CROSS_ENTROPY = 0, 1, 2, 3, 4, 5
+OP_MATMUL, OP_RESCALE, OP_LAYERNORM_BWD, OP_ADAM, OP_STATISTIC, OP_CROSS_ENTROPY, OP_COLSUM = 0, 1, 2, 3, 4, 5, 6
 DEV_TIMEOUT, DEV_BAD_SCALE, DEV_NONFINITE_STAT, DEV_BAD_INDEX = 1, 2, 4, 8
 
 _DTYPE_CODE = {torch.float8_e4m3fn: E4M3, torch.float8_e5m2: E5M2, torch.float16: F16,
@@ -82,6 +82,7 @@ def lib() -> ctypes.CDLL:
         L.scalify_scaled_gelu_bwd.argtypes = [P, P, i32, P, vp]
         L.scalify_scaled_adam_step.argtypes = [i32, P, P, P, P, f32, f32, f32, f32, i64, vp, sz, vp]
         L.scalify_scaled_attention.argtypes = [P, P, P, f32, i32, P, P, P, vp, vp]
+        L.scalify_scaled_colsum.argtypes = [P, P, vp, sz, vp]
         L.scalify_scaled_attention_bwd.argtypes = [P, P, P, P, P, f32, i32, P, P, P, P, P, vp, vp]
         L.scalify_mx_sf_bytes.restype = sz
         L.scalify_mx_sf_bytes.argtypes = [i64, i64]
@@ -104,7 +105,7 @@ def lib() -> ctypes.CDLL:
                      "scalify_scaled_embedding_bwd", "scalify_scaled_softmax", "scalify_scaled_softmax_bwd",
                      "scalify_scaled_cross_entropy", "scalify_scalar_mul_pow2", "scalify_debug_expire_wait",
                      "scalify_mx_quantize", "scalify_mx_matmul", "scalify_scaled_attention",
-                     "scalify_scaled_attention_bwd",
+                     "scalify_scaled_attention_bwd", "scalify_scaled_colsum",
                      "scalify_scaled_matmul_speculative"):
             getattr(L, name).restype = i32
         _lib = L
@@ -442,6 +443,12 @@ def scalify_scaled_attention(Q: ScaledTensor, K: ScaledTensor, V: ScaledTensor, 
     _check(lib().scalify_scaled_attention(_ref(q), _ref(k), _ref(v), float(sm_scale), int(bool(causal)), _ref(o),
                                           _ref(sd), _ref(pd), _ptr(status), _stream(stream)),
            "scalify_scaled_attention")
+
+
+def scalify_scaled_colsum(X: ScaledTensor, Y: ScaledTensor, ws: Workspace, stream=None) -> None:
+    """Column sums of a [R, N] matrix into a wide [N] vector (bias gradient): Y_s = X_s kf(R)."""
+    x, y = _desc(X), _desc(Y)
+    _check(lib().scalify_scaled_colsum(_ref(x), _ref(y), ws.ptr, ws.nbytes, _stream(stream)), "scalify_scaled_colsum")
 
 
 def scalify_scaled_attention_bwd(Q: ScaledTensor, K: ScaledTensor, V: ScaledTensor, P: ScaledTensor, dO: ScaledTensor,

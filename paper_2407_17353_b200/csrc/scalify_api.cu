@@ -112,6 +112,7 @@ size_t scalify_workspace_bytes(int op, int64_t d0, int64_t d1) {
     case SCALIFY_OP_LAYERNORM_BWD: n = layernorm_bwd_ws_bytes(d0, d1); break;
     case SCALIFY_OP_ADAM: n = adam_ws_bytes(d0); break;
     case SCALIFY_OP_CROSS_ENTROPY: n = cross_entropy_ws_bytes(d0); break;
+    case SCALIFY_OP_COLSUM: n = colsum_ws_bytes(d1); break;
     default: break;
   }
   if (n < stat_bytes) n = stat_bytes;
@@ -398,6 +399,21 @@ int scalify_mx_matmul(const scalify_mx_array* A, const scalify_mx_array* B, scal
   a.stat = stat;
   a.force_ncta = 0;
   return launch_mx_matmul(a, workspace, static_cast<cudaStream_t>(stream));
+}
+
+int scalify_scaled_colsum(const scalify_array* X, scalify_array* Y, void* workspace, size_t workspace_bytes,
+                          void* stream) {
+  int rc;
+  if ((rc = check_array(X)) || (rc = check_array(Y))) return rc;
+  if (!is_wide(Y->dtype)) return SCALIFY_ERR_DTYPE;
+  if (X->ndim != 2 || Y->ndim != 1 || Y->shape[0] != X->shape[1]) return SCALIFY_ERR_SHAPE;
+  const int64_t R = X->shape[0], N = X->shape[1];
+  if (R < 1 || N < 1 || X->stride[0] < N) return SCALIFY_ERR_SHAPE;
+  if (Y->scale && Y->scale == X->scale) return SCALIFY_ERR_ALIAS;
+  rc = check_ws(workspace, workspace_bytes, scalify_workspace_bytes(SCALIFY_OP_COLSUM, R, N));
+  if (rc) return rc;
+  return launch_colsum(X->data, X->dtype, X->stride[0], R, N, X->scale, Y->data, Y->dtype, Y->scale, workspace,
+                       static_cast<cudaStream_t>(stream));
 }
 
 // [batch, heads, T, hd] view of a 2-D, 3-D or 4-D array: counts, rows, row / head / batch strides (elements)

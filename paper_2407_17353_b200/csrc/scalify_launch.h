@@ -60,6 +60,9 @@ int launch_softmax_fwd(const void* S, int s_dt, void* P, int p_dt, long long row
 int launch_softmax_bwd(const void* dP, int g_dt, const void* P, int p_dt, void* dS, int o_dt, long long rows, int Tk,
                        const float* dp_scale, const float* p_scale, float* ds_scale, cudaStream_t st);
 size_t cross_entropy_ws_bytes(int64_t n);
+size_t colsum_ws_bytes(int64_t N);
+int launch_colsum(const void* X, int x_dt, long long ld, long long R, long long N, const float* x_scale, void* Y, int y_dt,
+                  float* y_scale, void* ws, cudaStream_t st);
 int launch_cross_entropy(const void* logits, int l_dt, long long ld, int n_classes, const long long* targets, long long n,
                          const float* l_scale, float* loss, void* dlogits, int g_dt, float* g_scale, void* ws,
                          cudaStream_t st);

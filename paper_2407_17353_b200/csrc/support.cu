@@ -397,4 +397,109 @@ int launch_cross_entropy(const void* logits, int l_dt, long long ld, int n_class
   return SCALIFY_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// column sums of a scaled matrix (Section 3.2, the rule for a sum of R independent terms: the data
+// component is divided by kf(R), the scale multiplied by it) - the bias gradient of a linear layer
+// ---------------------------------------------------------------------------------------------
+// Launch 1: a block is 32 vectors of columns wide and takes one slab of rows; its eight warps stride over
+// the slab's rows (four rows in flight per thread), are added in warp order through shared memory, and
+// leave one fp32 partial per column and slab.  Launch 2 adds the slabs in index order in fp64.
+constexpr int kColSlabsMax = 64;
+
+template <int DT>
+__global__ void __launch_bounds__(256) colsum_partial_kernel(const void* __restrict__ X, long long ld, long long R,
+                                                             long long N, int slabs, float* __restrict__ part) {
+  constexpr int VEC = 16 / ElemBytes<DT>::v;
+  __shared__ float s_acc[8][32][VEC + 1];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const long long n_vec = N / VEC;
+  const int tail = static_cast<int>(N - n_vec * VEC);
+  const long long vec = static_cast<long long>(blockIdx.x) * 32 + lane;  // vector of columns (n_vec: the ragged end)
+  const long long rows_per_slab = (R + slabs - 1) / slabs;
+  const long long r0 = blockIdx.y * rows_per_slab, r1 = min(R, r0 + rows_per_slab);
+  float acc[VEC];
+#pragma unroll
+  for (int e = 0; e < VEC; ++e) acc[e] = 0.f;
+  if (vec < n_vec) {
+    const char* base = static_cast<const char*>(X) + vec * 16;
+    for (long long r = r0 + warp; r < r1; r += 32) {
+      uint32_t w[4][4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) w[u][q] = 0u;  // zero bits decode to 0.0 in every format
+        if (r + u * 8 < r1) ld_raw_stream<16>(base + (r + u * 8) * ld * ElemBytes<DT>::v, w[u]);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        float f[VEC];
+        decode_vec<DT, VEC>(w[u], f);
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) acc[e] += f[e];
+      }
+    }
+  } else if (vec == n_vec && tail > 0) {
+    for (long long r = r0 + warp; r < r1; r += 8)
+      for (int e = 0; e < tail; ++e) acc[e] += load_elem<DT>(X, r * ld + n_vec * VEC + e);
+  }
+#pragma unroll
+  for (int e = 0; e < VEC; ++e) s_acc[warp][lane][e] = acc[e];
+  __syncthreads();
+  // thread t adds the eight warps' values of (lane t / VEC... ) one column each: 32 * VEC columns per block
+  for (int c = threadIdx.x; c < 32 * VEC; c += 256) {
+    const int l = c / VEC, e = c % VEC;
+    float sum = s_acc[0][l][e];
+#pragma unroll
+    for (int wv = 1; wv < 8; ++wv) sum += s_acc[wv][l][e];
+    const long long col = (static_cast<long long>(blockIdx.x) * 32 + l) * VEC + e;
+    if (col < N) part[static_cast<long long>(blockIdx.y) * N + col] = sum;
+  }
+}
+
+template <int YDT>
+__global__ void __launch_bounds__(256) colsum_finalize_kernel(const float* __restrict__ part, long long N, int slabs,
+                                                              float inv_kf, float kf, void* __restrict__ Y,
+                                                              const float* x_scale, float* y_scale, uint32_t* status) {
+  const long long col = static_cast<long long>(blockIdx.x) * 256 + threadIdx.x;
+  if (col < N) {
+    double sum = 0.0;
+    for (int sIdx = 0; sIdx < slabs; ++sIdx) sum += static_cast<double>(part[static_cast<long long>(sIdx) * N + col]);
+    store_elem<YDT>(Y, col, static_cast<float>(sum * static_cast<double>(inv_kf)));
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    const float xs = load_scale(x_scale);
+    if (y_scale) *y_scale = xs * kf;
+    if (!is_pow2_scale(xs) && status) atomicOr(status, static_cast<uint32_t>(SCALIFY_DEV_BAD_SCALE));
+  }
+}
+
+static int colsum_slabs(long long R, long long N, int elem_bytes) {
+  const long long gx = (N / (16 / elem_bytes) + 1 + 31) / 32;
+  long long s = (static_cast<long long>(sm_count()) * 8 + gx - 1) / gx;   // about eight blocks per SM
+  const long long by_rows = (R + 31) / 32;                                 // at least 32 rows per slab
+  if (s > by_rows) s = by_rows;
+  if (s > kColSlabsMax) s = kColSlabsMax;
+  return static_cast<int>(s < 1 ? 1 : s);
+}
+
+size_t colsum_ws_bytes(int64_t N) { return kWsHeader + static_cast<size_t>(kColSlabsMax) * static_cast<size_t>(N) * sizeof(float) + 256; }
+
+int launch_colsum(const void* X, int x_dt, long long ld, long long R, long long N, const float* x_scale, void* Y, int y_dt,
+                  float* y_scale, void* ws, cudaStream_t st) {
+  WsView v = ws_view(ws);
+  float* part = static_cast<float*>(v.area);
+  const int es = elem_size(x_dt);
+  const int slabs = colsum_slabs(R, N, es);
+  const long long gx = (N / (16 / es) + 1 + 31) / 32;
+  if (gx > 0x7FFFFFFF) return SCALIFY_ERR_SHAPE;
+  const dim3 grid(static_cast<unsigned>(gx), static_cast<unsigned>(slabs));
+  SCALIFY_DISPATCH_DTYPE(x_dt, DT, colsum_partial_kernel<DT><<<grid, 256, 0, st>>>(X, ld, R, N, slabs, part));
+  SCALIFY_CUDA_TRY(cudaGetLastError());
+  const float kf = kfactor(R);
+  SCALIFY_DISPATCH_WIDE(y_dt, YDT, colsum_finalize_kernel<YDT><<<static_cast<unsigned>((N + 255) / 256), 256, 0, st>>>(
+                                       part, N, slabs, 1.0f / kf, kf, Y, x_scale, y_scale, v.status));
+  SCALIFY_CUDA_TRY(cudaGetLastError());
+  return SCALIFY_OK;
+}
+
 }  // namespace scalify

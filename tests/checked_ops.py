@@ -230,6 +230,23 @@ class Ops:
             assert P.scale_value() == ps and self.ulp_diff(self.bits(P), po, p_dt).max() <= 1
         return P
 
+    def colsum(self, X, o_dt=BF):
+        """Column sums of a [R, N] matrix by the reduce-sum rule (the bias gradient)."""
+        R, N = X.data.shape
+        Y = self.empty((N,), o_dt)
+        if not hasattr(self, "ws_col") or self.ws_col.nbytes < sc.scalify_workspace_bytes(sc.OP_COLSUM, R, N):
+            self.ws_col = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_COLSUM, R, N), self.dev)
+        sc.scalify_scaled_colsum(X, Y, self.ws_col)
+        self.calls += 1
+        if self.check:
+            o = self.orc
+            xv = o.decode(self.bits(X), code(X.data))
+            kf = o.kf(R)
+            exact, mag = xv.sum(axis=0) / kf, np.abs(xv).sum(axis=0) / kf
+            assert Y.scale_value() == X.scale_value() * kf
+            assert self.within(self.bits(Y), o.encode(exact, o_dt), o_dt, exact, mag, 1e-5).all()
+        return Y
+
     def attention(self, Q, K, V, O, sm_scale, causal=True):
         """Fused forward over [heads, T, 64] views; returns the E4M3 probabilities (kept for the backward).
         Checked stage by stage through the kernel's own copies of the scores and probabilities."""

@@ -76,7 +76,6 @@ class ScaledGPT:
         self.m = OrderedDict((k, sc.ScaledTensor.make(torch.zeros_like(v.data), 2.0 ** -16)) for k, v in self.params.items())
         self.v = OrderedDict((k, sc.ScaledTensor.make(torch.zeros_like(v.data), 2.0 ** -24)) for k, v in self.params.items())
         n = cfg.batch * cfg.seq
-        self.ones = sc.ScaledTensor.make(torch.ones((1, n), device=device).to(torch.float8_e4m3fn), 1.0)
         self.adam_ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_ADAM, len(self.params)), device)
 
     def n_params(self):
@@ -106,8 +105,8 @@ class ScaledGPT:
         dy8 = o.cast(dy, E5)
         dx = o.mm(dy8, W8, transB=True)               # dy W^T: W stored [K, N] = [N', K'] of this product
         _, dW = o.mm(x8, dy8, transA=True, stat=sc.STAT_AMAX, q_dt=E5)   # x^T dy with fused AMAX rescale
-        _, db = o.mm(self.ones, dy8, stat=sc.STAT_AMAX, q_dt=E5)         # column sum as a contraction
-        return dx, dW, sc.ScaledTensor(db.data.view(-1), db.scale)
+        db = o.rescale(o.colsum(dy8), sc.STAT_AMAX, E5)                    # column sums, then the dynamic rescale
+        return dx, dW, db
 
     # ------------------------------------------------------------------ one training step
     def step(self, ids, targets, t, lr=3e-4, beta1=0.9, beta2=0.999, eps=1e-8):

@@ -125,3 +125,37 @@ def test_cross_entropy_and_gradient(n, V, ld, g_dt):
     bad[1] = V
     sc.scalify_scaled_cross_entropy(L, V, torch.from_numpy(bad).cuda(), loss, None, ws)
     assert ws.check_status() == sc.DEV_BAD_INDEX
+
+
+@pytest.mark.parametrize("R,N,x_dt,y_dt", [(8192, 768, orc.E5M2, orc.BF16), (8192, 3072, orc.E5M2, orc.F32),
+                                          (1000, 50, orc.BF16, orc.BF16), (37, 1030, orc.E4M3, orc.F16),
+                                          (5, 24, orc.F32, orc.F32), (70000, 64, orc.F16, orc.F32)])
+def test_column_sums(R, N, x_dt, y_dt):
+    """The reduce-sum rule is the matmul rule with a ones operand and K = R: the oracle's scaled matmul of
+    [1, R] ones with X is the definition.  Bar: 1 ulp of the output format, or half an ulp plus
+    1e-5 * sum|x| (fp32 partial sums)."""
+    ld = (N // 16 + 2) * 16                                          # a padded, 16-byte-aligned row stride
+    full = si.to_bits(si.normal(91, R, (R, ld), 1.0), x_dt)
+    x = np.ascontiguousarray(full[:, :N])
+    X = sc.ScaledTensor.make(to_dev(full, x_dt)[:, :N], 2.0 ** -7)
+    Y = sc.ScaledTensor.empty((N,), sc.TORCH_DTYPE[y_dt])
+    ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_COLSUM, R, N))
+    sc.scalify_scaled_colsum(X, Y, ws)
+    assert ws.check_status() == 0
+    xv = orc.decode(x, x_dt)
+    kf = orc.kf(R)
+    exact = xv.sum(axis=0) / kf
+    mag = np.abs(xv).sum(axis=0) / kf
+    want = orc.encode(exact, y_dt)
+    assert Y.scale_value() == 2.0 ** -7 * kf
+    ok = within(to_bits(Y.data, y_dt), want, y_dt, exact, mag, 1e-5)
+    assert ok.all(), int((~ok).sum())
+    if x_dt in (orc.E4M3, orc.E5M2) and R <= 8192:
+        # the same numbers from the oracle's matmul with a ones operand
+        ones = si.to_bits(np.ones((1, R), dtype=np.float32), orc.E4M3)
+        yo, ys = orc.scaled_matmul(ones, orc.E4M3, 1.0, x, x_dt, 2.0 ** -7, y_dt)[:2]
+        assert ys == 2.0 ** -7 * kf and np.array_equal(yo.reshape(-1), want)
+    # deterministic: a second call gives the same bits
+    Y2 = sc.ScaledTensor.empty((N,), sc.TORCH_DTYPE[y_dt])
+    sc.scalify_scaled_colsum(X, Y2, ws)
+    assert np.array_equal(to_bits(Y2.data, y_dt), to_bits(Y.data, y_dt))
