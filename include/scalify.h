@@ -474,12 +474,15 @@ int scalify_scaled_colsum(const scalify_array* X, scalify_array* Y, void* worksp
  * scalify_scaled_matmul.  The softmax is the exact two-sweep form (row maximum
  * and sum first, then the normalised probabilities), not an online rescaling.
  *   Q [heads, Tq, hd], K, V [heads, Tk, hd]: E4M3 or E5M2, hd = 64, 3-D views
- *   (row and head strides in stride[1], stride[0]; 2-D arrays are one head);
+ *   (row and head strides in stride[1], stride[0]; 2-D arrays are one head; 4-D
+ *   arrays [batch, heads, T, hd] add a batch stride in front, so that the token-major
+ *   buffers [batch * T, heads * hd] of a transformer are covered by ONE call);
  *   O [heads, Tq, hd]: F16, BF16 or F32, same kind of view; c: any finite
  *   scalar (a power of two only shifts the exponent; otherwise its mantissa is
  *   applied in fp32).  causal needs Tk >= Tq.
  *   S_dump (BF16) and P_dump (E4M3): optional dense [heads, Tq, Tk] DEVICE
- *   copies of S_d and P for checking (Tk % 32 == 0), normally NULL.
+ *   copies of S_d and P for checking (Tk % 32 == 0), normally NULL; with 4-D
+ *   operands the leading dimension counts batch * heads (or is given as two).
  *   status: optional DEVICE word (SCALIFY_DEV_TIMEOUT, SCALIFY_DEV_BAD_SCALE).
  * Errors: NULL, DTYPE, SHAPE, ALIGNMENT, UNSUPPORTED (hd != 64, causal with
  * Tk < Tq), ALIAS (O_s aliasing an input scale word).
