@@ -332,7 +332,7 @@ template <int IN, int OUT>
 __global__ void __launch_bounds__(kThreads) fused_rescale_kernel(const void* x, void* y, int64_t n, int stat,
                                                                  const float* x_scale, float* y_scale,
                                                                  double* partials, float* stat_word,
-                                                                 uint32_t* status) {
+                                                                 uint32_t* status, int one_block) {
   constexpr int VEC = VecElems<IN, OUT>::v;
   constexpr int IB = VEC * ElemBytes<IN>::v, OB = VEC * ElemBytes<OUT>::v;
   constexpr int kTile = kThreads * kUnroll;
@@ -390,7 +390,10 @@ __global__ void __launch_bounds__(kThreads) fused_rescale_kernel(const void* x, 
     }
     partials[blockIdx.x] = tot;
   }
-  grid.sync();
+  // an array of one tile is launched as a single ordinary block (a cooperative launch costs several
+  // microseconds more, which is most of the call for a bias or LayerNorm gradient)
+  if (one_block) __syncthreads();
+  else grid.sync();
 
   // the same fixed-order combination in every block
   double acc = 0.0;
@@ -478,9 +481,15 @@ int launch_fused_rescale(const void* x, int in_dt, void* y, int out_dt, int64_t 
   double* partials = static_cast<double*>(v.area);
   float* stat_word = v.stat;
   uint32_t* status = v.status;
-  void* args[] = {&x, &y, &n, &stat, &x_scale, &y_scale, &partials, &stat_word, &status};
+  int one_block = 0;
+  void* args[] = {&x, &y, &n, &stat, &x_scale, &y_scale, &partials, &stat_word, &status, &one_block};
   int rc = 1;
   SCALIFY_DISPATCH_DTYPE(in_dt, IN, SCALIFY_DISPATCH_DTYPE(out_dt, OUT, {
+    if (grid_for(n_vec, 1) == 1 && room >= 1) {
+      fused_rescale_kernel<IN, OUT><<<1, kThreads, 0, st>>>(x, y, n, stat, x_scale, y_scale, partials, stat_word, status, 1);
+      SCALIFY_CUDA_TRY(cudaGetLastError());
+      return SCALIFY_OK;
+    }
     int per_sm = fused_rescale_blocks_per_sm<IN, OUT>();
     if (per_sm > 0) {
       int grid = grid_for(n_vec, per_sm < 8 ? per_sm : 8);

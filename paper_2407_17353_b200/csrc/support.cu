@@ -463,7 +463,13 @@ __global__ void __launch_bounds__(256) colsum_finalize_kernel(const float* __res
   const long long col = static_cast<long long>(blockIdx.x) * 256 + threadIdx.x;
   if (col < N) {
     double sum = 0.0;
-    for (int sIdx = 0; sIdx < slabs; ++sIdx) sum += static_cast<double>(part[static_cast<long long>(sIdx) * N + col]);
+    for (int s0 = 0; s0 < slabs; s0 += 8) {  // eight loads in flight, added in index order
+      float v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) v[u] = (s0 + u < slabs) ? part[static_cast<long long>(s0 + u) * N + col] : 0.f;
+#pragma unroll
+      for (int u = 0; u < 8; ++u) sum += static_cast<double>(v[u]);
+    }
     store_elem<YDT>(Y, col, static_cast<float>(sum * static_cast<double>(inv_kf)));
   }
   if (blockIdx.x == 0 && threadIdx.x == 0) {
