@@ -358,6 +358,137 @@ __global__ void __launch_bounds__(256) cross_entropy_kernel(const void* __restri
   }
 }
 
+// The same with the row kept in shared memory (rows of up to 110 KB: a 50k-class row of 16-bit logits):
+// one 16-byte-vector sweep over HBM, the other two over shared memory.
+constexpr int kCeSmemMax = 110 * 1024;
+
+// 2^x for x <= 0: the hardware approximation (2 ulp of fp32; results below 2^-126 flush to zero)
+__device__ __forceinline__ float ce_exp2(float x) {
+  float r;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+  return r;
+}
+
+template <int LDT, int GDT>
+__global__ void __launch_bounds__(256, 2) cross_entropy_smem_kernel(const void* __restrict__ logits, long long ld,
+                                                                    int n_classes, const long long* __restrict__ targets,
+                                                                    long long n, const float* l_scale,
+                                                                    void* __restrict__ dlogits, float rem,
+                                                                    float* __restrict__ row_loss, uint32_t* bad_index) {
+  constexpr int VEC = 16 / ElemBytes<LDT>::v;
+  constexpr int GB = VEC * ElemBytes<GDT>::v;
+  extern __shared__ uint4 s_row[];
+  __shared__ float s_red[8];
+  __shared__ float s_bcast;
+  const float ls = load_scale(l_scale) * 1.4426950408889634f;  // positive: the maximum commutes with it
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int nv_full = n_classes / VEC;               // vectors made of classes only
+  const int n_part = n_classes - nv_full * VEC;      // classes in the one partial vector (0: none)
+  const int nv = nv_full + (n_part ? 1 : 0);
+  const int nv_ld = static_cast<int>(ld / VEC);      // vectors of the padded row (the gradient covers them all)
+  for (long long row = blockIdx.x; row < n; row += gridDim.x) {
+    const uint4* lrow = reinterpret_cast<const uint4*>(static_cast<const char*>(logits) + row * ld * ElemBytes<LDT>::v);
+    float mraw = -INFINITY;  // maximum of the data component
+    for (int v0 = threadIdx.x; v0 < nv; v0 += 256 * 8) {  // eight 16-byte loads in flight per thread
+      uint4 w[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        if (v0 + u * 256 < nv) w[u] = __ldcs(lrow + v0 + u * 256);
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int v = v0 + u * 256;
+        if (v < nv) {
+          s_row[v] = w[u];
+          float f[VEC];
+          decode_vec<LDT, VEC>(reinterpret_cast<const uint32_t*>(&w[u]), f);
+          if (v < nv_full) {
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) mraw = fmaxf(mraw, f[e]);
+          } else {
+#pragma unroll
+            for (int e = 0; e < VEC; ++e)
+              if (e < n_part) mraw = fmaxf(mraw, f[e]);
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mraw = fmaxf(mraw, __shfl_xor_sync(0xFFFFFFFFu, mraw, o));
+    __syncthreads();
+    if (lane == 0) s_red[warp] = mraw;
+    __syncthreads();  // also: the row is in shared memory
+    mraw = s_red[0];
+#pragma unroll
+    for (int k = 1; k < 8; ++k) mraw = fmaxf(mraw, s_red[k]);
+    const float mx = mraw * ls;
+    float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int v = threadIdx.x; v < nv; v += 256) {
+      const uint4 w = s_row[v];
+      float f[VEC];
+      decode_vec<LDT, VEC>(reinterpret_cast<const uint32_t*>(&w), f);
+      if (v < nv_full) {
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) sum4[e & 3] += ce_exp2(fmaf(f[e], ls, -mx));
+      } else {
+#pragma unroll
+        for (int e = 0; e < VEC; ++e)
+          if (e < n_part) sum4[e & 3] += ce_exp2(fmaf(f[e], ls, -mx));
+      }
+    }
+    float sum = warp_sum_f32((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
+    __syncthreads();
+    if (lane == 0) s_red[warp] = sum;
+    __syncthreads();
+    sum = 0.f;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) sum += s_red[k];
+    long long t = targets[row];
+    if (t < 0 || t >= n_classes) {
+      if (threadIdx.x == 0 && bad_index) atomicOr(bad_index, static_cast<uint32_t>(SCALIFY_DEV_BAD_INDEX));
+      t = 0;
+    }
+    if (threadIdx.x == 0) {
+      const float zt = load_elem<LDT>(lrow, t) * ls;
+      row_loss[row] = logf(sum) + (mx - zt) * 0.6931471805599453f;
+      s_bcast = rem / sum;
+    }
+    __syncthreads();
+    if (dlogits) {
+      const float k = s_bcast;
+      const int tv = static_cast<int>(t / VEC), te = static_cast<int>(t % VEC);
+      char* grow = static_cast<char*>(dlogits) + row * ld * ElemBytes<GDT>::v;
+      for (int v = threadIdx.x; v < nv_ld; v += 256) {
+        float g[VEC];
+        if (v < nv) {
+          const uint4 w = s_row[v];
+          float f[VEC];
+          decode_vec<LDT, VEC>(reinterpret_cast<const uint32_t*>(&w), f);
+#pragma unroll
+          for (int e = 0; e < VEC; ++e) g[e] = ce_exp2(fmaf(f[e], ls, -mx)) * k;
+          if (v >= nv_full) {
+#pragma unroll
+            for (int e = 0; e < VEC; ++e)
+              if (e >= n_part) g[e] = 0.f;
+          }
+          if (v == tv) {
+#pragma unroll
+            for (int e = 0; e < VEC; ++e)
+              if (e == te) g[e] -= rem;
+          }
+        } else {
+#pragma unroll
+          for (int e = 0; e < VEC; ++e) g[e] = 0.f;
+        }
+        uint32_t o[GB / 4 > 0 ? GB / 4 : 1];
+        encode_vec<GDT, VEC>(g, o);
+        st_raw_stream<GB>(grow + static_cast<long long>(v) * GB, o);
+      }
+      for (long long j = static_cast<long long>(nv_ld) * VEC + threadIdx.x; j < ld; j += 256) store_elem<GDT>(grow, j, 0.f);
+    }
+    __syncthreads();  // the row buffer is rewritten by the next row's first sweep
+  }
+}
+
 __global__ void __launch_bounds__(256) cross_entropy_finalize_kernel(const float* __restrict__ row_loss, long long n,
                                                                      float* loss, float* g_scale, float gs) {
   __shared__ double s[8];
@@ -388,9 +519,30 @@ int launch_cross_entropy(const void* logits, int l_dt, long long ld, int n_class
   const float rem = static_cast<float>((1.0 / static_cast<double>(n)) / gs);
   const long long cap = static_cast<long long>(sm_count()) * 8;
   const int grid = static_cast<int>(n < cap ? n : cap);
-  SCALIFY_DISPATCH_WIDE(l_dt, LDT, SCALIFY_DISPATCH_DTYPE(g_dt, GDT,
-      cross_entropy_kernel<LDT, GDT><<<grid, 256, 0, st>>>(logits, ld, n_classes, targets, n, l_scale, dlogits, rem,
-                                                           row_loss, v.status)));
+  const int les = elem_size(l_dt), lvec = 16 / les;
+  const long long row_smem = static_cast<long long>((n_classes + lvec - 1) / lvec) * 16;
+  // the vector path needs 16-byte-aligned rows on both sides and a gradient vector of at least 4 bytes
+  const bool vec_ok = row_smem <= kCeSmemMax && (ld * les) % 16 == 0 && (!dlogits || (ld * elem_size(g_dt)) % 16 == 0) &&
+                      lvec * elem_size(g_dt) >= 4 && reinterpret_cast<uintptr_t>(logits) % 16 == 0 &&
+                      reinterpret_cast<uintptr_t>(dlogits) % 16 == 0;
+  if (vec_ok) {
+    const long long cap2 = static_cast<long long>(sm_count()) * 2;
+    const int grid2 = static_cast<int>(n < cap2 ? n : cap2);
+    SCALIFY_DISPATCH_WIDE(l_dt, LDT, SCALIFY_DISPATCH_DTYPE(g_dt, GDT, {
+      auto kernel = cross_entropy_smem_kernel<LDT, GDT>;
+      static bool attr_done = false;
+      if (!attr_done) {
+        SCALIFY_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kCeSmemMax));
+        attr_done = true;
+      }
+      kernel<<<grid2, 256, static_cast<size_t>(row_smem), st>>>(logits, ld, n_classes, targets, n, l_scale, dlogits, rem,
+                                                               row_loss, v.status);
+    }));
+  } else {
+    SCALIFY_DISPATCH_WIDE(l_dt, LDT, SCALIFY_DISPATCH_DTYPE(g_dt, GDT,
+        cross_entropy_kernel<LDT, GDT><<<grid, 256, 0, st>>>(logits, ld, n_classes, targets, n, l_scale, dlogits, rem,
+                                                             row_loss, v.status)));
+  }
   SCALIFY_CUDA_TRY(cudaGetLastError());
   cross_entropy_finalize_kernel<<<1, 256, 0, st>>>(row_loss, n, loss, g_scale, static_cast<float>(gs));
   SCALIFY_CUDA_TRY(cudaGetLastError());
