@@ -64,6 +64,7 @@ struct AdamHyper {
 };
 
 __global__ void adam_scales_kernel(AdamScalePtrs sp, AdamHyper h, AdamFactors* __restrict__ fac, uint32_t* status) {
+  asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= sp.count) return;
   const float gs = load_scale(sp.g[i]);
@@ -151,6 +152,7 @@ template <int GDT, int MVDT, int WDT>
 __global__ void __launch_bounds__(kAdamThreads) adam_update_kernel(const __grid_constant__ AdamTable tab,
                                                                    const AdamFactors* __restrict__ fac,
                                                                    AdamHyper h) {
+  asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   constexpr int GB = kAdamVec * ElemBytes<GDT>::v, MB = kAdamVec * ElemBytes<MVDT>::v,
                 WB = kAdamVec * ElemBytes<WDT>::v;
   const int total_chunks = tab.chunk_start[tab.count];

@@ -93,6 +93,7 @@ __global__ void __launch_bounds__(kBw1Threads, 2)
 attention_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_do, const __grid_constant__ CUtensorMap map_v,
                         const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_p,
                         const AttBwdParams p) {
+  asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -369,6 +370,7 @@ __global__ void __launch_bounds__(kBw2Threads, 4)
 attention_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_ds,
                          const __grid_constant__ CUtensorMap map_do, const __grid_constant__ CUtensorMap map_q,
                          const AttBwdParams p) {
+  asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;

@@ -44,6 +44,7 @@ template <int DT>
 __global__ void __launch_bounds__(kThreads) statistic_kernel(const void* __restrict__ x, int64_t n, int stat,
                                                              double* __restrict__ partials, uint32_t* ticket,
                                                              float* stat_word, float* out_stat) {
+  asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   constexpr int VEC = 16 / ElemBytes<DT>::v;
   constexpr int WORDS = 4;
   const int64_t n_vec = n / VEC;
@@ -174,6 +175,7 @@ __global__ void __launch_bounds__(kThreads) rebalance_kernel(const void* __restr
                                                              int64_t n, const float* x_scale, float* y_scale,
                                                              const float* stat, const float* new_scale, int mode,
                                                              uint32_t* status) {
+  asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   constexpr int VEC = VecElems<IN, OUT>::v;
   constexpr int IB = VEC * ElemBytes<IN>::v, OB = VEC * ElemBytes<OUT>::v;
   const float xs = load_scale(x_scale);
@@ -254,6 +256,7 @@ __global__ void __launch_bounds__(kThreads) rebalance_check_kernel(const void* _
                                                                    int64_t n, const float* x_scale, float* y_scale,
                                                                    const float* stat, const float* r_pred,
                                                                    float* hint_out, uint32_t* status) {
+  asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   constexpr int VEC = VecElems<IN, OUT>::v;
   constexpr int IB = VEC * ElemBytes<IN>::v, OB = VEC * ElemBytes<OUT>::v;
   const float xs = load_scale(x_scale);
@@ -333,6 +336,7 @@ __global__ void __launch_bounds__(kThreads) fused_rescale_kernel(const void* x, 
                                                                  const float* x_scale, float* y_scale,
                                                                  double* partials, float* stat_word,
                                                                  uint32_t* status, int one_block) {
+  asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   constexpr int VEC = VecElems<IN, OUT>::v;
   constexpr int IB = VEC * ElemBytes<IN>::v, OB = VEC * ElemBytes<OUT>::v;
   constexpr int kTile = kThreads * kUnroll;
@@ -507,7 +511,10 @@ int launch_fused_rescale(const void* x, int in_dt, void* y, int out_dt, int64_t 
 // multiplication by a scalar constant that is a power of two (Section 3.4: a broadcast scalar
 // splits into mantissa and exponent; with mantissa 1 only the scale word changes)
 // ---------------------------------------------------------------------------------------------
-__global__ void scale_word_mul_kernel(float* scale, float c) { *scale = *scale * c; }
+__global__ void scale_word_mul_kernel(float* scale, float c) {
+  asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
+  *scale = *scale * c;
+}
 
 int launch_scale_word_mul(float* scale, float c, cudaStream_t st) {
   scale_word_mul_kernel<<<1, 1, 0, st>>>(scale, c);
@@ -543,6 +550,7 @@ __global__ void __launch_bounds__(kThreads) add_kernel(const void* __restrict__ 
                                                        void* __restrict__ y, int64_t n, int64_t row_len,
                                                        FastDiv row_vecs, int broadcast, const float* a_scale,
                                                        const float* b_scale, float* y_scale, float sign) {
+  asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   constexpr int VEC = VecElems<AB, OUT>::v;
   constexpr int IB = VEC * ElemBytes<AB>::v, OB = VEC * ElemBytes<OUT>::v;
   const float as = load_scale(a_scale), bs = load_scale(b_scale);
@@ -646,6 +654,7 @@ template <int IN, int OUT, int EXACT, int BWD>
 __global__ void __launch_bounds__(kThreads) gelu_kernel(const void* __restrict__ x, const void* __restrict__ g,
                                                         void* __restrict__ y, int64_t n, const float* x_scale,
                                                         const float* g_scale, float* y_scale) {
+  asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   constexpr int VEC = VecElems<IN, OUT>::v;
   constexpr int IB = VEC * ElemBytes<IN>::v, OB = VEC * ElemBytes<OUT>::v;
   const float xs = load_scale(x_scale);

@@ -107,6 +107,7 @@ __global__ void __launch_bounds__(kLnThreads) layernorm_fwd_kernel(
     const void* __restrict__ gamma, const void* __restrict__ beta, int gb_dt, const float* gamma_scale,
     const float* beta_scale, float* y_scale, float eps, int eps_inside, float* __restrict__ mean_out,
     float* __restrict__ rinv_out, int rows_per_team) {
+  asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   constexpr int VEC = 16 / ElemBytes<XDT>::v;
   constexpr int OB = VEC * ElemBytes<YDT>::v;
   constexpr int TEAM = 32 * TW;
@@ -303,6 +304,7 @@ __global__ void __launch_bounds__(kLnThreads, 2) layernorm_bwd_kernel(
     int64_t dx_ld, int R, int d, const void* __restrict__ gamma, int gb_dt, const float* __restrict__ mean,
     const float* __restrict__ rinv_in, float eps, int eps_inside, int stat, float* __restrict__ dgamma_part,
     float* __restrict__ dbeta_part, double* __restrict__ stat_part) {
+  asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   constexpr int VEC = 16 / ElemBytes<XDT>::v;
   constexpr int OB = VEC * ElemBytes<DXDT>::v;
   constexpr int TEAM = 32 * TW;
@@ -470,6 +472,7 @@ __global__ void __launch_bounds__(1024) layernorm_bwd_finalize_kernel(
     const double* __restrict__ stat_part, int stat, float* stat_word, void* __restrict__ dgamma,
     void* __restrict__ dbeta, const float* g_scale, const float* x_scale, const float* gamma_scale,
     float* dx_scale, float* dgamma_scale, float* dbeta_scale, uint32_t* status) {
+  asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   // block = 8 columns (one 32-byte sector of a partial row) x 128 slices of the block list: 4 x as many
   // blocks as a 32-column layout, so the partials (a few MB in L2) are read by more SMs at once
   __shared__ float s_a[128][9], s_b[128][9];

@@ -123,6 +123,7 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
   using C = GemmCfg<NCTA, MX>;
   constexpr int kStages = C::kStages;
   constexpr int kAcc = C::kAcc;
+  asm volatile("griddepcontrol.launch_dependents;");  // a dependent grid may set up while this one runs
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -157,6 +158,16 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
     mbar_init(drain_bar, 1);
     *abort_flag = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  if constexpr (NCTA == 2) cluster_sync_all();  // the peer's barriers exist before anything signals them
+  tc_fence_after();
+  // Everything above touches no global memory: launched as a programmatic dependent, the grid may set up
+  // while the kernel before it in the stream drains; from here on that kernel's writes are needed.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (threadIdx.x == 0) {
     if (blockIdx.x == 0) {
       float r = 1.0f;
       bool nf = false;
@@ -173,11 +184,6 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
         atomicOr(p.status, static_cast<uint32_t>(SCALIFY_DEV_BAD_SCALE));
     }
   }
-  if (warp == 1) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
-  tc_fence_before();
-  __syncthreads();
-  if constexpr (NCTA == 2) cluster_sync_all();  // the peer's barriers exist before anything signals them
-  tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   bool timed_out = false;
 
@@ -543,6 +549,7 @@ mx_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 // mbarrier that nothing ever arrives at; the wait must give up, record SCALIFY_DEV_TIMEOUT and let
 // the kernel finish normally (this is the path a lost copy or a lost MMA completion would take).
 __global__ void expire_wait_kernel(uint32_t* status, unsigned long long limit_ns, uint32_t* waited_us) {
+  asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   __shared__ uint64_t bar;
   __shared__ uint32_t abort_flag;
   if (threadIdx.x == 0) {
@@ -566,6 +573,7 @@ int launch_expire_wait(void* ws, unsigned long long limit_ns, uint32_t* waited_u
 // Sums the per-warp partial sums of squares in slot order and leaves sqrt(mean) in the statistic word.
 __global__ void __launch_bounds__(256) gemm_l2_finalize_kernel(const double* __restrict__ partials, int n_slots,
                                                                double count, float* stat_word) {
+  asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   __shared__ double s[8];
   double acc = 0.0;
   for (int i = threadIdx.x; i < n_slots; i += 256) acc += partials[i];
@@ -725,18 +733,19 @@ static int launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, co
     attr_done = true;
   }
   cudaLaunchConfig_t cfg = {};
-  cudaLaunchAttribute attrs[1];
+  cudaLaunchAttribute attrs[2];
+  attrs[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // the prologue may overlap the grid before it
+  attrs[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attrs;
+  cfg.numAttrs = 1;
   if (NCTA == 2) {
     const long long units = tiles < max_clusters ? tiles : max_clusters;
     cfg.gridDim = dim3(unsigned(units * 2));
-    attrs[0].id = cudaLaunchAttributeClusterDimension;
-    attrs[0].val.clusterDim.x = 2; attrs[0].val.clusterDim.y = 1; attrs[0].val.clusterDim.z = 1;
-    cfg.attrs = attrs;
-    cfg.numAttrs = 1;
+    attrs[1].id = cudaLaunchAttributeClusterDimension;
+    attrs[1].val.clusterDim.x = 2; attrs[1].val.clusterDim.y = 1; attrs[1].val.clusterDim.z = 1;
+    cfg.numAttrs = 2;
   } else {
     cfg.gridDim = dim3(unsigned(tiles < sm_count() ? tiles : sm_count()));
-    cfg.attrs = nullptr;
-    cfg.numAttrs = 0;
   }
   cfg.blockDim = dim3(kGemmThreads);
   cfg.dynamicSmemBytes = C::kSmem;
@@ -871,13 +880,18 @@ static int launch_mx_variant(const CUtensorMap& map_a, const CUtensorMap& map_b,
     attr_done = true;
   }
   cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute run_attrs[2];
+  run_attrs[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // the prologue may overlap the grid before it
+  run_attrs[0].val.programmaticStreamSerializationAllowed = 1;
+  run_attrs[1] = attrs[0];
+  cfg.attrs = run_attrs;
   if (NCTA == 2) {
     const long long units = tiles < max_clusters ? tiles : max_clusters;
     cfg.gridDim = dim3(unsigned(units * 2));
-    cfg.attrs = attrs;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
   } else {
     cfg.gridDim = dim3(unsigned(tiles < sm_count() ? tiles : sm_count()));
+    cfg.numAttrs = 1;
   }
   cfg.blockDim = dim3(kGemmThreads);
   cfg.dynamicSmemBytes = C::kSmem;

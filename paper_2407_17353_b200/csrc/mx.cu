@@ -44,6 +44,7 @@ __global__ void __launch_bounds__(kMxThreads) mx_quantize_kernel(const void* __r
                                                                  int64_t K, void* __restrict__ data,
                                                                  uint8_t* __restrict__ sf, const float* x_scale,
                                                                  float* y_scale, uint32_t* status) {
+  asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   constexpr int LE = 32 / ElemBytes<IN>::v;       // elements per thread: 16 or 8
   constexpr int kPieces = 128 / LE;               // threads per 128-element row segment: 8 or 16
   constexpr int kLanesPerBlock = kMxBlock / LE;   // 2 or 4

@@ -41,6 +41,14 @@ inline WsView ws_view(void* ws) {
                 reinterpret_cast<uint32_t*>(p + kWsTicket), p + kWsHeader};
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// Every kernel of the library begins with `griddepcontrol.launch_dependents`, so a grid that follows it in
+// the stream AND was launched as a programmatic dependent (the matmul kernels are: their prologue of barrier
+// set-up, TMEM allocation and cluster synchronisation touches no global memory) may be scheduled while it
+// still runs.  Such a dependent executes `griddepcontrol.wait` before its first access to global memory;
+// only from there on are the writes of the grid before it complete and visible.  For an ordinary launch
+// both instructions do nothing.
+
 // ---------------------------------------------------------------- host side helpers
 inline int elem_size(int dt) { return dt <= SCALIFY_E5M2 ? 1 : (dt == SCALIFY_F32 ? 4 : 2); }
 inline bool valid_dtype(int dt) { return dt >= SCALIFY_E4M3 && dt <= SCALIFY_F32; }

@@ -17,6 +17,7 @@ __global__ void __launch_bounds__(256) embedding_fwd_kernel(const long long* __r
                                                             const void* __restrict__ wpe, const float* wte_scale,
                                                             const float* wpe_scale, void* __restrict__ Y, float* y_scale,
                                                             uint32_t* bad_index) {
+  asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   constexpr int VEC = 16 / ElemBytes<WDT>::v;
   constexpr int OB = VEC * ElemBytes<YDT>::v;
   const float ts = load_scale(wte_scale), ps = wpe ? load_scale(wpe_scale) : 0.f;
@@ -58,6 +59,7 @@ template <int GDT>
 __global__ void __launch_bounds__(256) embedding_bwd_scatter_kernel(const long long* __restrict__ ids, long long n, int d,
                                                                     long long vocab, const void* __restrict__ dY,
                                                                     float* __restrict__ dwte) {
+  asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   constexpr int VEC = 16 / ElemBytes<GDT>::v;
   const int n_vec = d / VEC;
   const long long total = n * n_vec;
@@ -82,6 +84,7 @@ __global__ void __launch_bounds__(256) embedding_bwd_pos_kernel(long long n, int
                                                                 const void* __restrict__ dY, float* __restrict__ dwpe,
                                                                 const float* dy_scale, float* dwte_scale,
                                                                 float* dwpe_scale) {
+  asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   constexpr int VEC = 16 / ElemBytes<GDT>::v;
   const int n_vec = d / VEC;
   const int B = static_cast<int>(n / seq_len);
@@ -153,6 +156,7 @@ template <int SDT, int PDT>
 __global__ void __launch_bounds__(128) softmax_fwd_kernel(const void* __restrict__ S, void* __restrict__ P,
                                                           long long rows, int Tq, int Tk, int causal,
                                                           const float* s_scale, float* p_scale) {
+  asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   constexpr int VEC = 16 / ElemBytes<SDT>::v;
   constexpr int OB = VEC * ElemBytes<PDT>::v;
   const int lane = threadIdx.x & 31;
@@ -216,6 +220,7 @@ template <int GDT, int PDT, int ODT>
 __global__ void __launch_bounds__(128) softmax_bwd_kernel(const void* __restrict__ dP, const void* __restrict__ P,
                                                           void* __restrict__ dS, long long rows, int Tk,
                                                           const float* dp_scale, const float* p_scale, float* ds_scale) {
+  asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   constexpr int VEC = 16 / ElemBytes<GDT>::v;            // vector of the gradient dtype
   constexpr int PB = VEC * ElemBytes<PDT>::v, OB = VEC * ElemBytes<ODT>::v;
   const int lane = threadIdx.x & 31;
@@ -306,6 +311,7 @@ __global__ void __launch_bounds__(256) cross_entropy_kernel(const void* __restri
                                                             const float* l_scale, void* __restrict__ dlogits,
                                                             float rem, float* __restrict__ row_loss,
                                                             uint32_t* bad_index) {
+  asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   __shared__ float s_red[8];
   __shared__ float s_bcast;
   const float ls = load_scale(l_scale) * 1.4426950408889634f;
@@ -375,6 +381,7 @@ __global__ void __launch_bounds__(256, 2) cross_entropy_smem_kernel(const void* 
                                                                     long long n, const float* l_scale,
                                                                     void* __restrict__ dlogits, float rem,
                                                                     float* __restrict__ row_loss, uint32_t* bad_index) {
+  asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   constexpr int VEC = 16 / ElemBytes<LDT>::v;
   constexpr int GB = VEC * ElemBytes<GDT>::v;
   extern __shared__ uint4 s_row[];
@@ -491,6 +498,7 @@ __global__ void __launch_bounds__(256, 2) cross_entropy_smem_kernel(const void* 
 
 __global__ void __launch_bounds__(256) cross_entropy_finalize_kernel(const float* __restrict__ row_loss, long long n,
                                                                      float* loss, float* g_scale, float gs) {
+  asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   __shared__ double s[8];
   double acc = 0.0;
   for (long long i = threadIdx.x; i < n; i += 256) acc += static_cast<double>(row_loss[i]);
@@ -561,6 +569,7 @@ constexpr int kColSlabsMax = 64;
 template <int DT>
 __global__ void __launch_bounds__(256) colsum_partial_kernel(const void* __restrict__ X, long long ld, long long R,
                                                              long long N, int slabs, float* __restrict__ part) {
+  asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   constexpr int VEC = 16 / ElemBytes<DT>::v;
   __shared__ float s_acc[8][32][VEC + 1];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -612,6 +621,7 @@ template <int YDT>
 __global__ void __launch_bounds__(256) colsum_finalize_kernel(const float* __restrict__ part, long long N, int slabs,
                                                               float inv_kf, float kf, void* __restrict__ Y,
                                                               const float* x_scale, float* y_scale, uint32_t* status) {
+  asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   const long long col = static_cast<long long>(blockIdx.x) * 256 + threadIdx.x;
   if (col < N) {
     double sum = 0.0;
