@@ -293,6 +293,88 @@ def run_profile_row(args):
     print(json.dumps(out))
 
 
+def run_hbm_sweep(args):
+    """The HBM-bound rows at other sizes: LayerNorm forward / backward + rescale at R in {8192, 131072} and
+    d in {768, 1024, 4096}; stand-alone rescale and add at 2^23, 2^26 and 2^28 elements.  Each case is
+    launched back to back over a rotation of buffer sets larger than L2 in total (the small cases are
+    L2- and launch-bound and say so).  One JSON line per case."""
+    import torch
+
+    import paper_2407_17353_b200 as sc
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    peak = load_peaks()["hbm_gbs"]
+    l2 = 126 * 2 ** 20
+
+    def rnd(shape, dtype, tid):
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(tid)
+        return torch.randn(shape, device=dev, dtype=torch.float32, generator=gen).to(dtype)
+
+    def timed(fns, iters):
+        for f in fns:
+            f()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(iters):
+            fns[i % len(fns)]()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / iters
+
+    def report(name, ms, nbytes, sets, footprint):
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        print(json.dumps({"sweep": name, "ms": round(ms, 4), "GB/s": round(gbs, 1), "frac_of_hbm_peak": round(gbs / peak, 3),
+                          "buffer_sets": sets, "note": "larger than L2 per launch" if footprint > l2 else
+                          "fits L2: rotation over %d sets makes the inputs cold, the launch itself is short" % sets}))
+
+    iters = max(10, args.steps)
+    for R in (8192, 131072):
+        for d in (768, 1024, 4096):
+            per_set = R * d * 2 * 4
+            sets = max(1, min(8, -(-2 * l2 // per_set)))
+            fw, bw = [], []
+            gamma = sc.ScaledTensor.make(torch.ones(d, device=dev).to(torch.bfloat16), 1.0)
+            beta = sc.ScaledTensor.make(torch.zeros(d, device=dev).to(torch.bfloat16), 1.0)
+            ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_LAYERNORM_BWD, R, d), dev)
+            for k in range(sets):
+                X = sc.ScaledTensor.make(rnd((R, d), torch.bfloat16, 10 + k), 1.0)
+                G = sc.ScaledTensor.make(rnd((R, d), torch.bfloat16, 20 + k), 2.0 ** -10)
+                Y = sc.ScaledTensor.empty((R, d), torch.bfloat16, dev)
+                dX = sc.ScaledTensor.empty((R, d), torch.bfloat16, dev)
+                dXq = sc.ScaledTensor.empty((R, d), torch.float8_e5m2, dev)
+                dg = sc.ScaledTensor.empty((d,), torch.float32, dev)
+                db = sc.ScaledTensor.empty((d,), torch.float32, dev)
+                mean = torch.empty(R, dtype=torch.float32, device=dev)
+                rinv = torch.empty(R, dtype=torch.float32, device=dev)
+                fw.append(lambda X=X, Y=Y, mean=mean, rinv=rinv: sc.scalify_scaled_layernorm(
+                    X, gamma, beta, Y, eps=1e-5, mean=mean, rinv=rinv))
+                bw.append(lambda G=G, X=X, mean=mean, rinv=rinv, dX=dX, dXq=dXq, dg=dg, db=db:
+                          sc.scalify_scaled_layernorm_bwd(G, X, gamma, mean, rinv, dX, ws, eps=1e-5, stat_dx=sc.STAT_L2,
+                                                          dXq=dXq, dgamma=dg, dbeta=db))
+            report(f"LayerNorm fwd {R}x{d} BF16->BF16", timed(fw, iters), R * d * 4 + R * 8, sets, R * d * 4)
+            report(f"LayerNorm bwd + L2 rescale to E5M2 {R}x{d}", timed(bw, iters), R * d * 9 + R * 8, sets, R * d * 6)
+            del fw, bw
+            torch.cuda.empty_cache()
+    for lg in (23, 26, 28):
+        n = 1 << lg
+        sets = max(1, min(8, -(-2 * l2 // (n * 3))))
+        rs, ad = [], []
+        ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_RESCALE, n), dev)
+        for k in range(sets):
+            X = sc.ScaledTensor.make(rnd((n,), torch.bfloat16, 30 + k), 1.0)
+            Z = sc.ScaledTensor.make(rnd((n,), torch.bfloat16, 40 + k), 0.25)
+            Yq = sc.ScaledTensor.empty((n,), torch.float8_e4m3fn, dev)
+            S = sc.ScaledTensor.empty((n,), torch.bfloat16, dev)
+            rs.append(lambda X=X, Yq=Yq: sc.scalify_rescale(X, Yq, stat=sc.STAT_AMAX, ws=ws))
+            ad.append(lambda X=X, Z=Z, S=S: sc.scalify_scaled_add(X, Z, S))
+        report(f"stand-alone dynamic rescale BF16->E4M3 2^{lg} elements", timed(rs, iters), 5 * n, sets, 3 * n)
+        report(f"scaled add BF16 2^{lg} elements", timed(ad, iters), 6 * n, sets, 6 * n)
+        del rs, ad
+        torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -304,6 +386,8 @@ def main():
     ap.add_argument("--speculative", action="store_true",
                     help="run rows a1-a3 of the step as ONE call with a predicted statistic "
                          "(scalify_scaled_matmul_speculative; same outputs bit for bit)")
+    ap.add_argument("--hbm-sweep", action="store_true",
+                    help="print one JSON line per size of the HBM-bound rows (LayerNorm, rescale, add) instead of the step")
     ap.add_argument("--no-next", action="store_true",
                     help="skip the separately timed next-row variants f1, f2 (for ncu launch lists of the step)")
     ap.add_argument("--profile-row", default=None, choices=["matmul", "mx", "attention", "attention_bwd", "rescale", "add", "layernorm", "adam"],
@@ -311,6 +395,9 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.hbm_sweep:
+        run_hbm_sweep(args)
         return
     if args.profile_row:
         run_profile_row(args)

@@ -252,10 +252,11 @@ int launch_layernorm_fwd(const void* X, int x_dt, int64_t x_ld, void* Y, int y_d
                          float* rinv, cudaStream_t st) {
   int tw = ln_team_warps(d, x_dt);
   if (tw == 0) return SCALIFY_ERR_UNSUPPORTED;
-  // rows of 65..128 vectors: one warp per row with four vectors per thread (no cross-warp step)
+  // rows of more than 64 vectors: four vectors per thread and a quarter of the warps per row (65..128 vectors:
+  // one warp, no cross-warp step; up to 512 vectors: four warps, so a block works on two rows at a time)
   const int n_vec = d * elem_size(x_dt) / 16;
-  const bool wide = n_vec > 64 && n_vec <= 128;
-  if (wide) tw = 1;
+  const bool wide = n_vec > 64;
+  if (wide) tw = n_vec <= 128 ? 1 : (n_vec <= 256 ? 2 : 4);
   // Blocks are not persistent: each owns a short run of consecutive rows (6 per team) and the
   // hardware scheduler hands out the runs in address order.  Measured on B200 (131072 x 1024 BF16):
   // 90 us, against 104 us for a grid of 3 blocks per SM striding over the rows, and 101 us with 16
@@ -278,7 +279,11 @@ int launch_layernorm_fwd(const void* X, int x_dt, int64_t x_ld, void* Y, int y_d
   } while (0)
   SCALIFY_DISPATCH_WIDE(x_dt, XDT, SCALIFY_DISPATCH_DTYPE(y_dt, YDT, {
     if (wide) {
-      SCALIFY_LN_FWD(1, 4);
+      switch (tw) {
+        case 1: SCALIFY_LN_FWD(1, 4); break;
+        case 2: SCALIFY_LN_FWD(2, 4); break;
+        default: SCALIFY_LN_FWD(4, 4); break;
+      }
     } else {
       switch (tw) {
         case 1: SCALIFY_LN_FWD(1, 2); break;
