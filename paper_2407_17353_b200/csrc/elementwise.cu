@@ -633,7 +633,7 @@ __device__ __forceinline__ float gelu_gate(float x) {
     // logistic of 2u through t = exp(-2|u|) in (0,1]: never overflows, and underflows gradually
     const float u = gelu_u(x);
     const float t = __expf(-2.0f * fabsf(u));
-    const float r = 1.0f / (1.0f + t);
+    const float r = __fdividef(1.0f, 1.0f + t);  // the approximate reciprocal (2 ulp of fp32) is far below the output's ulp
     return u >= 0.f ? r : t * r;
   }
 }
