@@ -564,7 +564,7 @@ int launch_cross_entropy(const void* logits, int l_dt, long long ld, int n_class
 // Launch 1: a block is 32 vectors of columns wide and takes one slab of rows; its eight warps stride over
 // the slab's rows (four rows in flight per thread), are added in warp order through shared memory, and
 // leave one fp32 partial per column and slab.  Launch 2 adds the slabs in index order in fp64.
-constexpr int kColSlabsMax = 64;
+constexpr int kColSlabsMax = 64;  // the finish adds 8 x 8 slabs
 
 template <int DT>
 __global__ void __launch_bounds__(256) colsum_partial_kernel(const void* __restrict__ X, long long ld, long long R,
@@ -617,22 +617,30 @@ __global__ void __launch_bounds__(256) colsum_partial_kernel(const void* __restr
   }
 }
 
+// 32 columns per block; the eight warps each add eight slabs (index order, fp64), warp 0 adds the eight sums
 template <int YDT>
 __global__ void __launch_bounds__(256) colsum_finalize_kernel(const float* __restrict__ part, long long N, int slabs,
                                                               float inv_kf, float kf, void* __restrict__ Y,
                                                               const float* x_scale, float* y_scale, uint32_t* status) {
   asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
-  const long long col = static_cast<long long>(blockIdx.x) * 256 + threadIdx.x;
+  __shared__ double s_sum[8][32];
+  const int lane = threadIdx.x & 31, grp = threadIdx.x >> 5;
+  const long long col = static_cast<long long>(blockIdx.x) * 32 + lane;
+  double sum = 0.0;
   if (col < N) {
-    double sum = 0.0;
-    for (int s0 = 0; s0 < slabs; s0 += 8) {  // eight loads in flight, added in index order
-      float v[8];
+    float v[8];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) v[u] = (s0 + u < slabs) ? part[static_cast<long long>(s0 + u) * N + col] : 0.f;
+    for (int u = 0; u < 8; ++u) v[u] = (grp * 8 + u < slabs) ? part[static_cast<long long>(grp * 8 + u) * N + col] : 0.f;
 #pragma unroll
-      for (int u = 0; u < 8; ++u) sum += static_cast<double>(v[u]);
-    }
-    store_elem<YDT>(Y, col, static_cast<float>(sum * static_cast<double>(inv_kf)));
+    for (int u = 0; u < 8; ++u) sum += static_cast<double>(v[u]);
+  }
+  s_sum[grp][lane] = sum;
+  __syncthreads();
+  if (grp == 0 && col < N) {
+    double tot = s_sum[0][lane];
+#pragma unroll
+    for (int g = 1; g < 8; ++g) tot += s_sum[g][lane];
+    store_elem<YDT>(Y, col, static_cast<float>(tot * static_cast<double>(inv_kf)));
   }
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     const float xs = load_scale(x_scale);
@@ -664,7 +672,7 @@ int launch_colsum(const void* X, int x_dt, long long ld, long long R, long long 
   SCALIFY_DISPATCH_DTYPE(x_dt, DT, colsum_partial_kernel<DT><<<grid, 256, 0, st>>>(X, ld, R, N, slabs, part));
   SCALIFY_CUDA_TRY(cudaGetLastError());
   const float kf = kfactor(R);
-  SCALIFY_DISPATCH_WIDE(y_dt, YDT, colsum_finalize_kernel<YDT><<<static_cast<unsigned>((N + 255) / 256), 256, 0, st>>>(
+  SCALIFY_DISPATCH_WIDE(y_dt, YDT, colsum_finalize_kernel<YDT><<<static_cast<unsigned>((N + 31) / 32), 256, 0, st>>>(
                                        part, N, slabs, 1.0f / kf, kf, Y, x_scale, y_scale, v.status));
   SCALIFY_CUDA_TRY(cudaGetLastError());
   return SCALIFY_OK;
