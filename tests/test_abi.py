@@ -31,7 +31,7 @@ def test_status_strings_and_workspace_sizes():
     assert L.scalify_status_string(0) == b"ok"
     for code in range(-9, 0):
         assert len(L.scalify_status_string(code)) > 3
-    for op in range(5):
+    for op in range(7):
         assert sc.scalify_workspace_bytes(op, 8192, 8192) >= 4096
     assert sc.scalify_workspace_bytes(sc.OP_ADAM, 1000) >= 1000 * 32
 
@@ -92,3 +92,29 @@ def test_validation_rejects_bad_arguments_on_the_host():
     # layernorm row length must be a multiple of 16 bytes
     assert L.scalify_scaled_layernorm(R(_arr(4096, sc.BF16, (4, 60), (64, 1))), None, None, 1e-5, 0,
                                       R(_arr(8192, sc.BF16, (4, 60), (64, 1))), None, None, None) == -3
+    # attention: head dimension, power-of-two scalar, batch views, required scale word of dS
+    Q3 = _arr(4096, sc.E4M3, (2, 128, 64))
+    O3 = _arr(1 << 20, sc.BF16, (2, 128, 64))
+    assert L.scalify_scaled_attention(R(Q3), R(Q3), R(Q3), 0.125, 1, R(_arr(1 << 20, sc.BF16, (2, 128, 32))), None, None,
+                                      None, None) == -3                                      # shapes differ
+    Q32 = _arr(4096, sc.E4M3, (2, 128, 32))
+    assert L.scalify_scaled_attention(R(Q32), R(Q32), R(Q32), 0.125, 1, R(_arr(1 << 20, sc.BF16, (2, 128, 32))), None,
+                                      None, None, None) == -6                                # head dimension 32
+    Q4 = _arr(4096, sc.E4M3, (3, 2, 128, 64))
+    assert L.scalify_scaled_attention(R(Q4), R(Q4), R(Q4), 0.125, 1, R(O3), None, None, None, None) == -3  # batch mismatch
+    P = _arr(1 << 21, sc.E4M3, (2, 128, 128))
+    dS = _arr(1 << 22, sc.E5M2, (2, 128, 128), scale=1024)
+    g = [_arr((3 + i) << 20, sc.BF16, (2, 128, 64)) for i in range(3)]
+    args = lambda c, ds: (R(Q3), R(Q3), R(Q3), R(P), R(Q3), c, 1, R(ds), R(g[0]), R(g[1]), R(g[2]), None, None, None)
+    assert L.scalify_scaled_attention_bwd(*args(0.1, dS)) == -6                              # scalar not a power of two
+    assert L.scalify_scaled_attention_bwd(*args(0.125, _arr(1 << 22, sc.E5M2, (2, 128, 128)))) == -1   # dS without a scale
+    assert L.scalify_scaled_attention_bwd(*args(0.125, _arr(1 << 22, sc.E4M3, (2, 128, 128), scale=1024))) == -2
+    # column sums
+    Xc = _arr(4096, sc.E5M2, (64, 128))
+    assert L.scalify_scaled_colsum(R(Xc), R(_arr(1 << 20, sc.BF16, (64,))), 1 << 21, 1 << 22, None) == -3
+    assert L.scalify_scaled_colsum(R(Xc), R(_arr(1 << 20, sc.E4M3, (128,))), 1 << 21, 1 << 22, None) == -2
+    assert L.scalify_scaled_colsum(R(Xc), R(_arr(1 << 20, sc.BF16, (128,))), 1 << 21, 1024, None) == -5
+    # matmul does not take four-dimensional arrays
+    A4 = _arr(4096, sc.E4M3, (1, 1, 128, 64))
+    assert L.scalify_scaled_matmul(R(A4), 0, R(A4), 1, R(_arr(1 << 20, sc.BF16, (1, 1, 128, 128))), 0, None, 1 << 21,
+                                   1 << 20, None) == -3
