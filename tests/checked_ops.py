@@ -132,9 +132,9 @@ class Ops:
         return Y
 
     # ---------------------------------------------------------------- LayerNorm
-    def ln(self, X, gamma, beta, eps=1e-5):
+    def ln(self, X, gamma, beta, eps=1e-5, out_dt=BF):
         R, d = X.data.shape
-        Y = self.empty((R, d), BF)
+        Y = self.empty((R, d), out_dt)
         mean = torch.empty(R, dtype=torch.float32, device=self.dev)
         rinv = torch.empty(R, dtype=torch.float32, device=self.dev)
         sc.scalify_scaled_layernorm(X, gamma, beta, Y, eps=eps, mean=mean, rinv=rinv)
@@ -144,13 +144,13 @@ class Ops:
             xdt, gdt = code(X.data), code(gamma.data)
             gs, bs = gamma.scale_value(), beta.scale_value()
             yo, ys, _, _ = o.layernorm_fwd(self.bits(X), xdt, self.bits(gamma), gdt, gs, self.bits(beta), gdt, bs, eps,
-                                           False, BF)
+                                           False, out_dt)
             n32, _, _, _ = o.layernorm_fwd(self.bits(X), xdt, None, 0, 1.0, None, 0, 1.0, eps, False, F32)
             nv = o.decode(n32, F32)
             g = o.decode(self.bits(gamma), gdt) * (gs / ys)
             b = o.decode(self.bits(beta), gdt) * (bs / ys)
             assert Y.scale_value() == ys
-            ok = self.within(self.bits(Y), yo, BF, nv * g + b, np.abs(nv * g) + np.abs(b) + 1e-3, 2e-6)
+            ok = self.within(self.bits(Y), yo, out_dt, nv * g + b, np.abs(nv * g) + np.abs(b) + 1e-3, 2e-6)
             assert ok.all(), int((~ok).sum())
         return Y, mean, rinv
 
@@ -193,14 +193,14 @@ class Ops:
         return dXq, dg, db
 
     # ---------------------------------------------------------------- GELU
-    def gelu(self, X):
-        Y = self.empty(X.data.shape, BF)
+    def gelu(self, X, out_dt=BF):
+        Y = self.empty(X.data.shape, out_dt)
         sc.scalify_scaled_gelu(X, Y)
         self.calls += 1
         if self.check:
             o = self.orc
-            yo, ys = o.gelu_fwd(self.bits(X), code(X.data), X.scale_value(), BF)
-            assert Y.scale_value() == ys and self.ulp_diff(self.bits(Y), yo, BF).max() <= 1
+            yo, ys = o.gelu_fwd(self.bits(X), code(X.data), X.scale_value(), out_dt)
+            assert Y.scale_value() == ys and self.ulp_diff(self.bits(Y), yo, out_dt).max() <= 1
         return Y
 
     def gelu_bwd(self, G, X):

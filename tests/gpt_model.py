@@ -95,9 +95,9 @@ class ScaledGPT:
         hd = c.d // c.heads
         return sc.ScaledTensor(X.data.view(c.batch, c.seq, c.heads, hd).permute(0, 2, 1, 3), X.scale)
 
-    def _linear(self, x8, W8, bias):
+    def _linear(self, x8, W8, bias, out_dt=BF):
         y = self.ops.mm(x8, W8)                       # [n, K] x [K, N], B stored [K, N]
-        return self.ops.add(y, self.ops.cast(bias, BF))
+        return self.ops.add(y, self.ops.cast(bias, BF), out_dt=out_dt)   # the bias add may write FP8 directly
 
     def _linear_bwd(self, dy, x8, W8):
         """dy BF16 -> (dx BF16, dW E5M2 rescaled, db E5M2 rescaled)."""
@@ -123,9 +123,10 @@ class ScaledGPT:
         for l in range(c.layers):
             p = f"h{l}."
             s = {"x_in": x}
-            h, s["mean1"], s["rinv1"] = o.ln(x, P[p + "ln1.g"], P[p + "ln1.b"])
-            s["h8"] = h8 = o.cast(h, E4)
-            q8, k8, v8 = (o.cast(self._linear(h8, W8[p + "w" + nm], P[p + "b" + nm]), E4) for nm in ("q", "k", "v"))
+            # producers write the E4M3 operand of the next matmul themselves (cast_on_forward fused in)
+            s["h8"], s["mean1"], s["rinv1"] = o.ln(x, P[p + "ln1.g"], P[p + "ln1.b"], out_dt=E4)
+            h8 = s["h8"]
+            q8, k8, v8 = (self._linear(h8, W8[p + "w" + nm], P[p + "b" + nm], out_dt=E4) for nm in ("q", "k", "v"))
             s["q8"], s["k8"], s["v8"] = q8, k8, v8
             att = o.empty((n, d), BF)
             att.scale = None
@@ -151,14 +152,13 @@ class ScaledGPT:
             s["o8"] = o8 = o.cast(att, E4)
             x = o.add(x, self._linear(o8, W8[p + "wo"], P[p + "bo"]))
             s["x_mid"] = x
-            h2, s["mean2"], s["rinv2"] = o.ln(x, P[p + "ln2.g"], P[p + "ln2.b"])
-            s["h2_8"] = h2_8 = o.cast(h2, E4)
+            s["h2_8"], s["mean2"], s["rinv2"] = o.ln(x, P[p + "ln2.g"], P[p + "ln2.b"], out_dt=E4)
+            h2_8 = s["h2_8"]
             s["a1"] = a1 = self._linear(h2_8, W8[p + "w1"], P[p + "b1"])
-            s["g8"] = g8 = o.cast(o.gelu(a1), E4)
+            s["g8"] = g8 = o.gelu(a1, out_dt=E4)
             x = o.add(x, self._linear(g8, W8[p + "w2"], P[p + "b2"]))
             saved.append(s)
-        hf, meanf, rinvf = o.ln(x, P["lnf.g"], P["lnf.b"])
-        hf8 = o.cast(hf, E4)
+        hf8, meanf, rinvf = o.ln(x, P["lnf.g"], P["lnf.b"], out_dt=E4)
         logits_buf = torch.empty((n, c.vocab_padded), dtype=torch.bfloat16, device=self.dev)
         logits = sc.ScaledTensor(logits_buf[:, :c.vocab], torch.empty(1, dtype=torch.float32, device=self.dev))
         o.mm(hf8, W8["wte"], transB=True, Y=logits)                                  # tied head: wte stored [V, d]
