@@ -99,7 +99,8 @@ enum {
   SCALIFY_OP_ADAM = 3,          /* d0 = number of tensors, d1 unused */
   SCALIFY_OP_STATISTIC = 4,     /* d0 = number of elements */
   SCALIFY_OP_CROSS_ENTROPY = 5, /* d0 = number of rows */
-  SCALIFY_OP_COLSUM = 6         /* d0 = rows, d1 = columns */
+  SCALIFY_OP_COLSUM = 6,        /* d0 = rows, d1 = columns */
+  SCALIFY_OP_MATMUL_SPLITK = 7  /* d0 = M, d1 = N: room for the partial products of a split contraction */
 };
 
 /* Bytes of workspace the given call needs (an upper bound; always >= 4096).
@@ -152,6 +153,14 @@ int scalify_version(void);
  *
  * Accumulation is fp32 on the tensor cores (tcgen05, kind::f8f6f4).  Row
  * strides must be multiples of 16 bytes.  Errors: see scalify_error.
+  *
+ * Split contraction: when the output has few tiles and K >= 2048 (a weight
+ * gradient), and the workspace is at least scalify_workspace_bytes(
+ * SCALIFY_OP_MATMUL_SPLITK, M, N), the K range is cut into up to 16 parts that
+ * run as one batched launch writing fp32 partial products into the workspace; a
+ * second launch adds them in a fixed order, rounds once and takes the statistic.
+ * With the smaller SCALIFY_OP_MATMUL workspace the call never splits.  Results
+ * of the two forms agree within the accumulation bar, not bit for bit.
  */
 int scalify_scaled_matmul(const scalify_array* A, int transA, const scalify_array* B, int transB,
                           scalify_array* Y, int stat, scalify_array* Yq,

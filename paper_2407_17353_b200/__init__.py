@@ -22,7 +22,8 @@ from . import _build
 
 E4M3, E5M2, F16, BF16, F32 = 0, 1, 2, 3, 4
 STAT_NONE, STAT_AMAX, STAT_L2 = 0, 1, 2
-OP_MATMUL, OP_RESCALE, OP_LAYERNORM_BWD, OP_ADAM, OP_STATISTIC, OP_CROSS_ENTROPY, OP_COLSUM = 0, 1, 2, 3, 4, 5, 6
+OP_MATMUL, OP_RESCALE, OP_LAYERNORM_BWD, OP_ADAM, OP_STATISTIC, OP_CROSS_ENTROPY, OP_COLSUM, OP_MATMUL_SPLITK = (
+    0, 1, 2, 3, 4, 5, 6, 7)
 DEV_TIMEOUT, DEV_BAD_SCALE, DEV_NONFINITE_STAT, DEV_BAD_INDEX = 1, 2, 4, 8
 
 _DTYPE_CODE = {torch.float8_e4m3fn: E4M3, torch.float8_e5m2: E5M2, torch.float16: F16,

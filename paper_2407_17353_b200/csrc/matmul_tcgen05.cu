@@ -587,6 +587,93 @@ __global__ void __launch_bounds__(256) gemm_l2_finalize_kernel(const double* __r
   }
 }
 
+// Split contraction: the partial products [splits][M][ldp] (fp32, not yet divided by kf(K)) are added in split
+// order, scaled, rounded once to the output format and written; the statistic of the stored values goes
+// through one partial per block and the block that draws the last ticket (index order: scheduling does not
+// change the result).
+template <int OUT>
+__global__ void __launch_bounds__(256) splitk_reduce_kernel(const float* __restrict__ part, long long ldp, long long plane,
+                                                            int splits, int M, int N, void* __restrict__ Y, long long ldy,
+                                                            float alpha, int stat, const float* a_scale,
+                                                            const float* b_scale, float* y_scale, float kf,
+                                                            double* __restrict__ partials, uint32_t* ticket,
+                                                            float* stat_word) {
+  asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
+  constexpr int OSZ = ElemBytes<OUT>::v;
+  const long long nvr = ldp / 4, total = static_cast<long long>(M) * nvr;
+  const long long idx = static_cast<long long>(blockIdx.x) * 256 + threadIdx.x;
+  uint32_t amax = 0u;
+  float ssq = 0.f;
+  if (idx < total) {
+    const long long row = idx / nvr;
+    const int col = static_cast<int>(idx % nvr) * 4;
+    const float4* src = reinterpret_cast<const float4*>(part + row * ldp + col);
+    float4 acc = __ldcs(src);
+    for (int sIdx = 1; sIdx < splits; ++sIdx) {
+      const float4 t = __ldcs(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(src) + sIdx * plane));
+      acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
+    }
+    float v[4] = {acc.x * alpha, acc.y * alpha, acc.z * alpha, acc.w * alpha};
+    uint32_t o[OSZ];  // 4 elements: 4 * OSZ bytes
+    encode_vec<OUT, 4>(v, o);
+    char* dst = static_cast<char*>(Y) + (row * ldy + col) * OSZ;
+    if (col + 4 <= N) {
+      st_raw<4 * OSZ>(dst, o);
+    } else {
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        if (col + e < N) store_elem<OUT>(Y, row * ldy + col + e, v[e]);
+    }
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      if (col + e < N) {
+        const float sv = round_through<OUT>(v[e]);  // the value as stored
+        amax = max(amax, abs_bits(sv));
+        ssq = fmaf(sv, sv, ssq);
+      }
+    }
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0 && y_scale) *y_scale = load_scale(a_scale) * load_scale(b_scale) * kf;
+  if (stat == SCALIFY_STAT_NONE) return;
+  __shared__ double s_part[8];
+  __shared__ bool s_last;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  double mine = (stat == SCALIFY_STAT_AMAX) ? static_cast<double>(warp_max_u32(amax))
+                                            : warp_sum_f64(static_cast<double>(ssq));
+  if (lane == 0) s_part[warp] = mine;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double tot = 0.0;
+    for (int i = 0; i < 8; ++i) tot = (stat == SCALIFY_STAT_AMAX) ? fmax(tot, s_part[i]) : tot + s_part[i];
+    partials[blockIdx.x] = tot;
+    __threadfence();
+    s_last = atomicAdd(ticket, 1u) == gridDim.x - 1;
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  double acc = 0.0;
+  for (int i = threadIdx.x; i < static_cast<int>(gridDim.x); i += 256) {
+    const double pv = __ldcg(&partials[i]);
+    acc = (stat == SCALIFY_STAT_AMAX) ? fmax(acc, pv) : acc + pv;
+  }
+  acc = (stat == SCALIFY_STAT_AMAX) ? static_cast<double>(warp_max_u32(static_cast<uint32_t>(acc))) : warp_sum_f64(acc);
+  __syncthreads();
+  if (lane == 0) s_part[warp] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double tot = 0.0;
+    for (int i = 0; i < 8; ++i) tot = (stat == SCALIFY_STAT_AMAX) ? fmax(tot, s_part[i]) : tot + s_part[i];
+    *stat_word = (stat == SCALIFY_STAT_AMAX) ? __uint_as_float(static_cast<uint32_t>(tot))
+                                             : static_cast<float>(sqrt(tot / (static_cast<double>(M) * N)));
+    *ticket = 0u;
+  }
+}
+
+// Region of the workspace after the header that is left to per-block statistic partials before the split-K
+// partial products begin
+constexpr size_t kSplitStatBytes = 65536 * sizeof(double);
+
 // ------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -691,6 +778,13 @@ static int make_map_y(CUtensorMap* map, const void* ptr, int es, uint64_t N, uin
   return SCALIFY_OK;
 }
 
+size_t matmul_splitk_ws_bytes(int64_t rows, int64_t cols) {
+  const size_t ldp = static_cast<size_t>((cols + 3) / 4 * 4);
+  const size_t n = kWsHeader + kSplitStatBytes + 16 * static_cast<size_t>(rows) * ldp * sizeof(float) + 256;
+  const size_t base = matmul_ws_bytes(rows, cols);
+  return n > base ? n : base;
+}
+
 size_t matmul_ws_bytes(int64_t rows, int64_t cols) {
   int64_t tiles = ((rows + kBM - 1) / kBM + 8) * ((cols + kBN - 1) / kBN);
   return kWsHeader + size_t(tiles) * 8 * sizeof(double) + 256;
@@ -755,11 +849,48 @@ static int launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, co
   return SCALIFY_OK;
 }
 
-int launch_scaled_matmul(const MatmulArgs& a, void* ws, cudaStream_t st) {
+int launch_scaled_matmul(const MatmulArgs& a, void* ws, size_t ws_bytes, cudaStream_t st) {
   WsView v = ws_view(ws);
   // two-CTA tiles (256 rows) whenever there is more than one 128-row tile of output
   const int ncta = (a.M > kBM && a.force_ncta != 1) ? 2 : 1;
   const int tile_m = kBM * ncta;
+  // A product with few output tiles and a long contraction (a weight gradient) leaves most SMs idle: its K
+  // range is cut into `splits` parts that run as one batched call writing fp32 partial products into the
+  // workspace (when the caller's workspace has the room), and a second launch adds them in split order.
+  if (!a.no_split && a.batch == 1 && !a.stat_in && !a.stat_hint && a.K >= 2048) {
+    const long long out_tiles = static_cast<long long>((a.M + tile_m - 1) / tile_m) * ((a.N + kBN - 1) / kBN);
+    const long long units = ncta == 2 ? sm_count() / 2 : sm_count();
+    int splits = static_cast<int>(units / out_tiles);
+    if (splits > a.K / 512) splits = a.K / 512;
+    if (splits > 16) splits = 16;
+    while (splits >= 3 && a.K % (splits * kBK) != 0) --splits;
+    const long long ldp = (static_cast<long long>(a.N) + 3) / 4 * 4;
+    const size_t need = kWsHeader + kSplitStatBytes + static_cast<size_t>(splits) * a.M * ldp * sizeof(float);
+    const long long red_blocks = (static_cast<long long>(a.M) * (ldp / 4) + 255) / 256;
+    if (splits >= 3 && ws_bytes >= need && red_blocks <= 65536) {  // (two parts measured no faster than one launch)
+      float* part = reinterpret_cast<float*>(static_cast<char*>(v.area) + kSplitStatBytes);
+      MatmulArgs pa = a;
+      const int Kc = a.K / splits;
+      pa.K = Kc;
+      pa.batch = splits;
+      pa.a_bs = a.transA ? static_cast<int64_t>(Kc) * a.lda : Kc;
+      pa.b_bs = a.transB ? Kc : static_cast<int64_t>(Kc) * a.ldb;
+      pa.Y = part; pa.y_dt = SCALIFY_F32; pa.ldy = ldp; pa.y_bs = static_cast<int64_t>(a.M) * ldp;
+      pa.y_scale = nullptr;
+      pa.stat = SCALIFY_STAT_NONE;
+      pa.alpha_override = 1.0f;
+      pa.no_split = 1;
+      int rc2 = launch_scaled_matmul(pa, ws, ws_bytes, st);
+      if (rc2) return rc2;
+      const float kf = kfactor(a.K);
+      SCALIFY_DISPATCH_WIDE(a.y_dt, OUT, splitk_reduce_kernel<OUT><<<static_cast<unsigned>(red_blocks), 256, 0, st>>>(
+                                             part, ldp, static_cast<long long>(a.M) * ldp, splits, a.M, a.N, a.Y, a.ldy,
+                                             1.0f / kf, a.stat, a.a_scale, a.b_scale, a.y_scale, kf,
+                                             static_cast<double*>(v.area), v.ticket, v.stat));
+      SCALIFY_CUDA_TRY(cudaGetLastError());
+      return SCALIFY_OK;
+    }
+  }
   const uint32_t b_box_rows = ncta == 2 ? kBN / 2 : kBN;
   CUtensorMap map_a, map_b, map_y;
   // A is logically [M,K]; stored [M,K] (K-major) or, with transA, [K,M] (MN-major).
@@ -790,7 +921,7 @@ int launch_scaled_matmul(const MatmulArgs& a, void* ws, cudaStream_t st) {
             (uint32_t(p.a_mn_major) << 15) | (uint32_t(p.b_mn_major) << 16) | (uint32_t(kBN >> 3) << 17) |
             (uint32_t(tile_m >> 4) << 24);
   p.kf = kfactor(a.K);
-  p.alpha = 1.0f / p.kf;
+  p.alpha = a.alpha_override != 0.f ? a.alpha_override : 1.0f / p.kf;
   p.Y = a.Y; p.ldy = a.ldy; p.y_batch_stride = a.y_bs;
   p.a_scale = a.a_scale; p.b_scale = a.b_scale; p.y_scale = a.y_scale;
   p.stat = a.stat;

@@ -113,6 +113,7 @@ size_t scalify_workspace_bytes(int op, int64_t d0, int64_t d1) {
     case SCALIFY_OP_ADAM: n = adam_ws_bytes(d0); break;
     case SCALIFY_OP_CROSS_ENTROPY: n = cross_entropy_ws_bytes(d0); break;
     case SCALIFY_OP_COLSUM: n = colsum_ws_bytes(d1); break;
+    case SCALIFY_OP_MATMUL_SPLITK: n = matmul_splitk_ws_bytes(d0, d1); break;
     default: break;
   }
   if (n < stat_bytes) n = stat_bytes;
@@ -671,6 +672,8 @@ static int matmul_impl(const scalify_array* A, int transA, const scalify_array* 
   a.stat = stat;
   a.stat_in = nullptr;
   a.force_ncta = 0;
+  a.alpha_override = 0.f;
+  a.no_split = 0;
   a.stat_hint = nullptr;
   a.Yq = nullptr;
   a.q_dt = SCALIFY_E4M3;
@@ -684,7 +687,7 @@ static int matmul_impl(const scalify_array* A, int transA, const scalify_array* 
     a.q_dt = Yq->dtype;
   }
   if (a.lda < (transA ? M : K) || a.ldb < (transB ? K : N) || a.ldy < N) return SCALIFY_ERR_SHAPE;
-  rc = launch_scaled_matmul(a, workspace, st);
+  rc = launch_scaled_matmul(a, workspace, workspace_bytes, st);
   if (rc) return rc;
   if (Yq) {
     WsView v = ws_view(workspace);
@@ -749,12 +752,14 @@ int scalify_scaled_matmul_delayed(const scalify_array* A, int transA, const scal
   a.stat = stat;
   a.stat_in = stat_in;
   a.force_ncta = 0;
+  a.alpha_override = 0.f;
+  a.no_split = 0;
   a.stat_hint = nullptr;
   a.Yq = nullptr;
   a.q_dt = SCALIFY_E4M3;
   if (a.lda < (transA ? M : K) || a.ldb < (transB ? K : N) || a.ldy < N) return SCALIFY_ERR_SHAPE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  rc = launch_scaled_matmul(a, workspace, st);
+  rc = launch_scaled_matmul(a, workspace, workspace_bytes, st);
   if (rc) return rc;
   // published only after the kernel has finished, so stat_out may be the word stat_in points to
   if (stat_out)

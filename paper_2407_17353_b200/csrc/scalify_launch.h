@@ -79,10 +79,13 @@ struct MatmulArgs {
   // speculative rescale: predicted statistic (device) or NULL; then Yq (FP8, dense like Y) is written by the GEMM
   const float* stat_hint;
   void* Yq; int q_dt;
+  float alpha_override;  // 0: the data component is divided by kf(K); otherwise multiplied by this (split-K partials)
+  int no_split;          // 1: never split the contraction (the partial products of a split call)
 };
 size_t matmul_ws_bytes(int64_t rows, int64_t cols);
+size_t matmul_splitk_ws_bytes(int64_t rows, int64_t cols);
 int launch_expire_wait(void* ws, unsigned long long limit_ns, uint32_t* waited_us, cudaStream_t st);
-int launch_scaled_matmul(const MatmulArgs& a, void* ws, cudaStream_t st);
+int launch_scaled_matmul(const MatmulArgs& a, void* ws, size_t ws_bytes, cudaStream_t st);
 // Block-scaled matmul: A [M,K], B [N,K] FP8 row-major (dense), exponents in 128-row x 4-block tiles.
 struct MxMatmulArgs {
   const void* A; int a_dt; const uint8_t* sfa;

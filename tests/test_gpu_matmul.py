@@ -20,7 +20,7 @@ pytestmark = pytest.mark.gpu
 
 
 def run_matmul(A, a_dt, a_s, B, b_dt, b_s, y_dt, transA=False, transB=False, stat=sc.STAT_NONE, q_dt=None,
-               lda_pad=0, ldb_pad=0):
+               lda_pad=0, ldb_pad=0, splitk=False):
     """A, B: numpy bit arrays as stored (2-D or 3-D). Returns dict of numpy results."""
     def dev(x, dt, pad):
         if pad == 0:
@@ -38,7 +38,7 @@ def run_matmul(A, a_dt, a_s, B, b_dt, b_s, y_dt, transA=False, transB=False, sta
     Y = sc.ScaledTensor.empty(shape, sc.TORCH_DTYPE[y_dt])
     Yq = sc.ScaledTensor.empty(shape, sc.TORCH_DTYPE[q_dt]) if q_dt is not None else None
     rows = M * (A.shape[0] if A.ndim == 3 else 1)
-    ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_MATMUL, rows, N))
+    ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_MATMUL_SPLITK if splitk else sc.OP_MATMUL, rows, N))
     sc.scalify_scaled_matmul(sc.ScaledTensor.make(Ad, a_s), sc.ScaledTensor.make(Bd, b_s), Y, ws, transA=transA,
                              transB=transB, stat=stat, Yq=Yq)
     status = ws.check_status()
@@ -317,3 +317,31 @@ def test_speculative_rescale_is_the_exact_dynamic_rescale(M, N, K, y_dt, q_dt):
         assert Y.scale_value() == plain["y_scale"] and Yq.scale_value() == plain["yq_scale"]
         assert np.array_equal(to_bits(Y.data, y_dt), plain["Y"])
         assert np.array_equal(to_bits(Yq.data, q_dt), plain["Yq"]), hint
+
+
+@pytest.mark.parametrize("M,N,K,transA,transB", [(768, 768, 8192, True, False), (300, 528, 4096, False, True),
+                                                  (144, 272, 2048, True, True), (64, 1040, 6144, False, False)])
+def test_split_contraction_with_a_large_workspace(M, N, K, transA, transB):
+    """Few output tiles and a long K (weight gradients): with the larger workspace the K range is split, the
+    partial products are added in a fixed order by a second launch.  Same bars as the single launch; the fused
+    statistic and the rescaled output are those of the stored result."""
+    a = si.to_bits(si.normal(31, M, (K, M) if transA else (M, K), 1.0), orc.E4M3)
+    b = si.to_bits(si.normal(32, N, (N, K) if transB else (K, N), 1.0), orc.E5M2)
+    check_against_oracle(a, orc.E4M3, 2.0 ** -2, b, orc.E5M2, 2.0 ** -9, transA, transB, splitk=True)
+    for stat in (sc.STAT_AMAX, sc.STAT_L2):
+        g = run_matmul(a, orc.E4M3, 2.0 ** -2, b, orc.E5M2, 2.0 ** -9, orc.BF16, transA, transB, stat=stat, q_dt=orc.E5M2,
+                       splitk=True)
+        assert g["status"] == 0
+        want_stat = orc.statistic(g["Y"], orc.BF16, stat)
+        assert g["stat"] == want_stat if stat == sc.STAT_AMAX else abs(g["stat"] - want_stat) <= 2e-6 * want_stat
+        yq, ys, _ = orc.rescale(g["Y"], orc.BF16, g["y_scale"], stat, orc.E5M2, stat_override=g["stat"])
+        assert g["yq_scale"] == ys and np.array_equal(g["Yq"], yq)
+        # replays give the same bits (fixed summation order)
+        g2 = run_matmul(a, orc.E4M3, 2.0 ** -2, b, orc.E5M2, 2.0 ** -9, orc.BF16, transA, transB, stat=stat, q_dt=orc.E5M2,
+                        splitk=True)
+        assert np.array_equal(g["Y"], g2["Y"]) and g["stat"] == g2["stat"]
+    if K == 8192:
+        # the split did happen: fp32 sums in another order differ somewhere from the single launch's
+        one = run_matmul(a, orc.E4M3, 2.0 ** -2, b, orc.E5M2, 2.0 ** -9, orc.F32, transA, transB)
+        many = run_matmul(a, orc.E4M3, 2.0 ** -2, b, orc.E5M2, 2.0 ** -9, orc.F32, transA, transB, splitk=True)
+        assert not np.array_equal(one["Y"], many["Y"])
