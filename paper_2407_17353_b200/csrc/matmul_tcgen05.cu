@@ -608,10 +608,16 @@ __global__ void __launch_bounds__(256) splitk_reduce_kernel(const float* __restr
     const long long row = idx / nvr;
     const int col = static_cast<int>(idx % nvr) * 4;
     const float4* src = reinterpret_cast<const float4*>(part + row * ldp + col);
-    float4 acc = __ldcs(src);
-    for (int sIdx = 1; sIdx < splits; ++sIdx) {
-      const float4 t = __ldcs(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(src) + sIdx * plane));
-      acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s0 = 0; s0 < splits; s0 += 4) {  // four loads in flight, added in split order
+      float4 t[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        t[u] = (s0 + u < splits)
+                   ? __ldcs(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(src) + (s0 + u) * plane))
+                   : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) { acc.x += t[u].x; acc.y += t[u].y; acc.z += t[u].z; acc.w += t[u].w; }
     }
     float v[4] = {acc.x * alpha, acc.y * alpha, acc.z * alpha, acc.w * alpha};
     uint32_t o[OSZ];  // 4 elements: 4 * OSZ bytes
