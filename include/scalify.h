@@ -167,6 +167,22 @@ int scalify_scaled_matmul(const scalify_array* A, int transA, const scalify_arra
                           void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The same product with a bias vector added in the kernel's epilogue (a linear
+ * layer): the add rule applied to the product and the bias, rounded ONCE:
+ *   Y_s = max(A_s B_s kf(K), bias_s)
+ *   Y_d = (A_d B_d) / kf(K) * (A_s B_s kf(K) / Y_s)  +  bias_d[j] * (bias_s / Y_s)
+ * (both factors are exact powers of two).  bias: [N], F16, BF16 or F32, contiguous.
+ * Y may be F16, BF16, F32 or, as a static cast of the sum, E4M3 / E5M2.  stat, Yq,
+ * workspace as for scalify_scaled_matmul; the contraction is never split.  The
+ * unfused sequence (matmul, then scalify_scaled_add with the bias) rounds twice;
+ * this call is its value with one rounding.
+ * Errors: as scalify_scaled_matmul; NULL (no bias), DTYPE (bias not wide), SHAPE.
+ */
+int scalify_scaled_matmul_bias(const scalify_array* A, int transA, const scalify_array* B, int transB,
+                               const scalify_array* bias, scalify_array* Y, int stat, scalify_array* Yq,
+                               void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * scalify_scaled_matmul with stat = AMAX and a rebalanced FP8 output, made cheaper by a PREDICTION of the
  * statistic (Section 3.3 observes that statistics change slowly, which is what delayed rescaling exploits;
  * here the result stays that of the exact dynamic rescale).  *stat_hint (DEVICE) holds a predicted

@@ -84,6 +84,7 @@ def lib() -> ctypes.CDLL:
         L.scalify_scaled_adam_step.argtypes = [i32, P, P, P, P, f32, f32, f32, f32, i64, vp, sz, vp]
         L.scalify_scaled_attention.argtypes = [P, P, P, f32, i32, P, P, P, vp, vp]
         L.scalify_scaled_colsum.argtypes = [P, P, vp, sz, vp]
+        L.scalify_scaled_matmul_bias.argtypes = [P, i32, P, i32, P, P, i32, P, vp, sz, vp]
         L.scalify_scaled_attention_bwd.argtypes = [P, P, P, P, P, f32, i32, P, P, P, P, P, vp, vp]
         L.scalify_mx_sf_bytes.restype = sz
         L.scalify_mx_sf_bytes.argtypes = [i64, i64]
@@ -106,7 +107,7 @@ def lib() -> ctypes.CDLL:
                      "scalify_scaled_embedding_bwd", "scalify_scaled_softmax", "scalify_scaled_softmax_bwd",
                      "scalify_scaled_cross_entropy", "scalify_scalar_mul_pow2", "scalify_debug_expire_wait",
                      "scalify_mx_quantize", "scalify_mx_matmul", "scalify_scaled_attention",
-                     "scalify_scaled_attention_bwd", "scalify_scaled_colsum",
+                     "scalify_scaled_attention_bwd", "scalify_scaled_colsum", "scalify_scaled_matmul_bias",
                      "scalify_scaled_matmul_speculative"):
             getattr(L, name).restype = i32
         _lib = L
@@ -218,6 +219,15 @@ def scalify_scaled_matmul(A: ScaledTensor, B: ScaledTensor, Y: ScaledTensor, ws:
     a, b, y, yq = _desc(A), _desc(B), _desc(Y), _desc(Yq)
     _check(lib().scalify_scaled_matmul(_ref(a), int(transA), _ref(b), int(transB), _ref(y), stat, _ref(yq),
                                        ws.ptr, ws.nbytes, _stream(stream)), "scalify_scaled_matmul")
+
+
+def scalify_scaled_matmul_bias(A: ScaledTensor, B: ScaledTensor, bias: ScaledTensor, Y: ScaledTensor, ws: Workspace, *,
+                               transA=False, transB=False, stat: int = STAT_NONE, Yq: Optional[ScaledTensor] = None,
+                               stream=None) -> None:
+    """Y = A B + bias (a [N] vector) in the GEMM's epilogue, by the add rule and with one rounding."""
+    a, b, bi, y, yq = _desc(A), _desc(B), _desc(bias), _desc(Y), _desc(Yq)
+    _check(lib().scalify_scaled_matmul_bias(_ref(a), int(transA), _ref(b), int(transB), _ref(bi), _ref(y), stat,
+                                            _ref(yq), ws.ptr, ws.nbytes, _stream(stream)), "scalify_scaled_matmul_bias")
 
 
 def scalify_scaled_matmul_speculative(A: ScaledTensor, B: ScaledTensor, Y: ScaledTensor, Yq: ScaledTensor,

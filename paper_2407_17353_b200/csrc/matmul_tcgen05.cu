@@ -95,6 +95,10 @@ struct GemmParams {
   const float* stat_hint;
   int q_dt;          // SCALIFY_E4M3 or SCALIFY_E5M2
   float* r_pred_out; // the r_pred this launch used (read by the check kernel)
+  // BIAS kernels: Y = A B + bias by the add rule, rounded once: Y_s = max(A_s B_s kf(K), bias_s)
+  const void* bias;  // [N], F16 / BF16 / F32
+  int bias_dt;
+  const float* bias_scale;
   // MX only: block exponents in tiles of 128 rows x 4 K-blocks (512 B each), tile (r, k) at
   // ((r * K/128) + k) * 512, byte (row % 32) * 16 + (row / 32 % 4) * 4 + (block % 4)
   const uint8_t* sfa;
@@ -116,10 +120,11 @@ __device__ __forceinline__ void tile_coords(const GemmParams& p, int tile, int& 
 
 // map_sfa is the exponent map of A in the block-scaled form and the map of the speculative FP8 output in the
 // SPEC form (the two never occur together).
-template <int OUT, int NCTA, bool MX, bool SPEC = false>
+template <int OUT, int NCTA, bool MX, bool SPEC = false, bool BIAS = false>
 __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_y,
                                           const CUtensorMap& map_sfa, const CUtensorMap& map_sfb, const GemmParams& p) {
   static_assert(!SPEC || (!MX && ElemBytes<OUT>::v == 2), "speculative FP8 output: per-tensor kernel, 16-bit Y");
+  static_assert(!BIAS || (!MX && !SPEC), "bias: per-tensor kernel only");
   using C = GemmCfg<NCTA, MX>;
   constexpr int kStages = C::kStages;
   constexpr int kAcc = C::kAcc;
@@ -172,7 +177,9 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
       float r = 1.0f;
       bool nf = false;
       if (p.stat_in) r = rescale_factor(__ldg(p.stat_in), &nf);
-      if (p.y_scale) *p.y_scale = load_scale(p.a_scale) * load_scale(p.b_scale) * p.kf * r;
+      float ys = load_scale(p.a_scale) * load_scale(p.b_scale) * p.kf * r;
+      if constexpr (BIAS) ys = fmaxf(ys, load_scale(p.bias_scale));  // add rule for powers of two
+      if (p.y_scale) *p.y_scale = ys;
       if constexpr (SPEC) {
         bool nf2;
         *p.r_pred_out = rescale_factor(__ldg(p.stat_hint), &nf2);
@@ -180,8 +187,9 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
       if (nf && p.status) atomicOr(p.status, static_cast<uint32_t>(SCALIFY_DEV_NONFINITE_STAT));
     }
     if (blockIdx.x == 0 && p.status) {
-      if (!is_pow2_scale(load_scale(p.a_scale)) || !is_pow2_scale(load_scale(p.b_scale)))
-        atomicOr(p.status, static_cast<uint32_t>(SCALIFY_DEV_BAD_SCALE));
+      bool bad = !is_pow2_scale(load_scale(p.a_scale)) || !is_pow2_scale(load_scale(p.b_scale));
+      if constexpr (BIAS) bad = bad || !is_pow2_scale(load_scale(p.bias_scale));
+      if (bad) atomicOr(p.status, static_cast<uint32_t>(SCALIFY_DEV_BAD_SCALE));
     }
   }
   const uint32_t tmem_base = *tmem_slot;
@@ -344,7 +352,16 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
     // statistic); this step's statistic is taken on the un-rebalanced fp32 values
     float r_prev = 1.0f;
     if (p.stat_in) { bool nf; r_prev = rescale_factor(__ldg(p.stat_in), &nf); }
-    const float alpha = p.alpha * (1.0f / r_prev);  // exact: both are powers of two
+    float alpha = p.alpha * (1.0f / r_prev);  // exact: both are powers of two
+    float beta = 0.f;
+    if constexpr (BIAS) {
+      // both terms are brought to the output scale max(A_s B_s kf(K), bias_s): exact power-of-two factors
+      const float ab_s = load_scale(p.a_scale) * load_scale(p.b_scale) * p.kf;
+      const float b_s = load_scale(p.bias_scale);
+      const float ys = fmaxf(ab_s, b_s);
+      alpha *= ab_s / ys;
+      beta = b_s / ys;
+    }
     for (int tile = unit; tile < num_tiles; tile += num_units) {
       int b, mt, nt;
       tile_coords(p, tile, b, mt, nt);
@@ -356,6 +373,20 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
       const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kBN + c_first * 32;
       // chunks of this warp that lie inside the matrix (warp-uniform)
       const int n_chunks = max(0, min(kChunksPerWarp, (p.N - n0 + 31) / 32 - c_first));
+      float bias_reg[kChunksPerWarp];
+      if constexpr (BIAS) {
+#pragma unroll
+        for (int c = 0; c < kChunksPerWarp; ++c) {
+          const int col = n0 + (c_first + c) * 32 + lane;
+          float bv = 0.f;
+          if (col < p.N) {
+            if (p.bias_dt == SCALIFY_F32) bv = load_elem<SCALIFY_F32>(p.bias, col);
+            else if (p.bias_dt == SCALIFY_BF16) bv = load_elem<SCALIFY_BF16>(p.bias, col);
+            else bv = load_elem<SCALIFY_F16>(p.bias, col);
+          }
+          bias_reg[c] = bv * beta;
+        }
+      }
       // One 32-column chunk of this thread's row in two steps: scale + statistic + round (convert), then store.
       constexpr int CPR = 32 * OSZ / 16;              // 16-byte pieces per row: 2 (FP8), 4 (16-bit), 8 (F32)
       constexpr int kTileBytes = 32 * 32 * OSZ;
@@ -363,12 +394,23 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
       constexpr int NBUF = SPEC ? 2 : (C::kEpiWarpBytes / kTileBytes > 4 ? 4 : C::kEpiWarpBytes / kTileBytes);
       float inv_r_pred = 1.0f;
       if constexpr (SPEC) { bool nf2; inv_r_pred = 1.0f / rescale_factor(__ldg(p.stat_hint), &nf2); }
-      auto convert = [&](const uint32_t* acc_regs, uint32_t* o) {
+      auto convert = [&](const uint32_t* acc_regs, uint32_t* o, int c) {
         float v[32];
+        if constexpr (BIAS) {
+          // lane l holds the (scaled) bias of column l of each of this warp's chunks; every lane needs all 32
+          static_assert(!BIAS || kChunksPerWarp == 4, "four chunks per warp");
+          const float mine = c == 0 ? bias_reg[0] : (c == 1 ? bias_reg[1] : (c == 2 ? bias_reg[2] : bias_reg[3]));
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          v[i] = __uint_as_float(acc_regs[i]) * alpha;
-          amax_bits = max(amax_bits, abs_bits(v[i]));
+          for (int i = 0; i < 32; ++i) {
+            v[i] = fmaf(__uint_as_float(acc_regs[i]), alpha, __shfl_sync(0xFFFFFFFFu, mine, i));
+            amax_bits = max(amax_bits, abs_bits(v[i]));
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            v[i] = __uint_as_float(acc_regs[i]) * alpha;
+            amax_bits = max(amax_bits, abs_bits(v[i]));
+          }
         }
         if (p.stat == SCALIFY_STAT_L2) {
 #pragma unroll
@@ -450,12 +492,12 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
         for (int c = 0; c < n_chunks; c += 2) {
           tmem_ld_wait();
           if (c + 1 < n_chunks) tmem_ld32(t_addr + (c + 1) * 32, rb);
-          convert(ra, o);
+          convert(ra, o, c);
           stage_chunk(o, c);
           if (c + 1 < n_chunks) {
             tmem_ld_wait();
             if (c + 2 < n_chunks) tmem_ld32(t_addr + (c + 2) * 32, ra);
-            convert(rb, o);
+            convert(rb, o, c + 1);
             stage_chunk(o, c + 1);
           }
         }
@@ -474,12 +516,12 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
         for (int c = 0; c < n_chunks; c += 2) {
           tmem_ld_wait();
           if (c + 1 < n_chunks) tmem_ld32(t_addr + (c + 1) * 32, rb);
-          convert(ra, o);
+          convert(ra, o, c);
           store(o, c);
           if (c + 1 < n_chunks) {
             tmem_ld_wait();
             if (c + 2 < n_chunks) tmem_ld32(t_addr + (c + 2) * 32, ra);
-            convert(rb, o);
+            convert(rb, o, c + 1);
             store(o, c + 1);
           }
         }
@@ -525,6 +567,14 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
 scaled_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                      const __grid_constant__ CUtensorMap map_y, const GemmParams p) {
   gemm_body<OUT, NCTA, false>(map_a, map_b, map_y, map_a, map_a, p);
+}
+
+// The same kernel with a bias vector added in the epilogue (add rule, one rounding).
+template <int OUT, int NCTA>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+scaled_matmul_bias_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                          const __grid_constant__ CUtensorMap map_y, const GemmParams p) {
+  gemm_body<OUT, NCTA, false, false, true>(map_a, map_b, map_y, map_a, map_a, p);
 }
 
 // The same kernel that also writes the FP8 output quantised with a PREDICTED rescale factor.
@@ -796,21 +846,25 @@ size_t matmul_ws_bytes(int64_t rows, int64_t cols) {
   return kWsHeader + size_t(tiles) * 8 * sizeof(double) + 256;
 }
 
-template <int OUT, int NCTA, bool SPEC>
+template <int OUT, int NCTA, bool SPEC, bool BIAS>
 struct GemmKernelOf {
   static auto get() { return scaled_matmul_kernel<OUT, NCTA>; }
 };
 template <int OUT, int NCTA>
-struct GemmKernelOf<OUT, NCTA, true> {
+struct GemmKernelOf<OUT, NCTA, true, false> {
   static auto get() { return scaled_matmul_spec_kernel<OUT, NCTA>; }
 };
+template <int OUT, int NCTA>
+struct GemmKernelOf<OUT, NCTA, false, true> {
+  static auto get() { return scaled_matmul_bias_kernel<OUT, NCTA>; }
+};
 
-template <int OUT, int NCTA, bool SPEC = false>
+template <int OUT, int NCTA, bool SPEC = false, bool BIAS = false>
 static int launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_y,
                           const CUtensorMap& map_q, const GemmParams& p, long long tiles,
                           cudaStream_t st) {
   using C = GemmCfg<NCTA>;
-  auto kernel = GemmKernelOf<OUT, NCTA, SPEC>::get();
+  auto kernel = GemmKernelOf<OUT, NCTA, SPEC, BIAS>::get();
   static bool attr_done = false;
   static int max_clusters = 0;
   if (!attr_done) {
@@ -863,7 +917,7 @@ int launch_scaled_matmul(const MatmulArgs& a, void* ws, size_t ws_bytes, cudaStr
   // A product with few output tiles and a long contraction (a weight gradient) leaves most SMs idle: its K
   // range is cut into `splits` parts that run as one batched call writing fp32 partial products into the
   // workspace (when the caller's workspace has the room), and a second launch adds them in split order.
-  if (!a.no_split && a.batch == 1 && !a.stat_in && !a.stat_hint && a.K >= 2048) {
+  if (!a.no_split && a.batch == 1 && !a.stat_in && !a.stat_hint && !a.bias && a.K >= 2048) {
     const long long out_tiles = static_cast<long long>((a.M + tile_m - 1) / tile_m) * ((a.N + kBN - 1) / kBN);
     const long long units = ncta == 2 ? sm_count() / 2 : sm_count();
     int splits = static_cast<int>(units / out_tiles);
@@ -941,6 +995,7 @@ int launch_scaled_matmul(const MatmulArgs& a, void* ws, size_t ws_bytes, cudaStr
   p.sfb = nullptr;
   p.stat_hint = a.stat_hint;
   p.q_dt = a.q_dt;
+  p.bias = a.bias; p.bias_dt = a.bias_dt; p.bias_scale = a.bias_scale;
   p.r_pred_out = reinterpret_cast<float*>(static_cast<char*>(ws) + 52);  // header word read by the check kernel
   const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n * p.batch;
   if (tiles > (1ll << 30)) return SCALIFY_ERR_SHAPE;
@@ -956,6 +1011,11 @@ int launch_scaled_matmul(const MatmulArgs& a, void* ws, size_t ws_bytes, cudaStr
       if (ncta == 2) rc = launch_variant<SCALIFY_F16, 2, true>(map_a, map_b, map_y, map_q, p, tiles, st);
       else rc = launch_variant<SCALIFY_F16, 1, true>(map_a, map_b, map_y, map_q, p, tiles, st);
     }
+  } else if (a.bias) {
+    SCALIFY_DISPATCH_DTYPE(a.y_dt, OUT, {
+      if (ncta == 2) rc = launch_variant<OUT, 2, false, true>(map_a, map_b, map_y, map_a, p, tiles, st);
+      else rc = launch_variant<OUT, 1, false, true>(map_a, map_b, map_y, map_a, p, tiles, st);
+    });
   } else {
     SCALIFY_DISPATCH_DTYPE(a.y_dt, OUT, {
       if (ncta == 2) rc = launch_variant<OUT, 2>(map_a, map_b, map_y, map_a, p, tiles, st);
@@ -1077,6 +1137,7 @@ int launch_mx_matmul(const MxMatmulArgs& a, void* ws, cudaStream_t st) {
   p.l2_partials = static_cast<double*>(v.area);
   p.status = v.status;
   p.sfa = a.sfa;
+  p.bias = nullptr; p.bias_dt = 0; p.bias_scale = nullptr;
   p.sfb = a.sfb;
   p.stat_hint = nullptr;
   p.q_dt = SCALIFY_E4M3;

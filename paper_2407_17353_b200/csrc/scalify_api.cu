@@ -623,16 +623,23 @@ int scalify_scaled_adam_step_cast(int n_tensors, const scalify_array* grads, sca
                         stream);
 }
 
-static int matmul_impl(const scalify_array* A, int transA, const scalify_array* B, int transB, scalify_array* Y,
-                       int stat, scalify_array* Yq, float* stat_hint, void* workspace, size_t workspace_bytes,
-                       void* stream) {
+static int matmul_impl(const scalify_array* A, int transA, const scalify_array* B, int transB,
+                       const scalify_array* bias, scalify_array* Y, int stat, scalify_array* Yq, float* stat_hint,
+                       void* workspace, size_t workspace_bytes, void* stream) {
   int rc = check_array(A);
   if (rc) return rc;
   rc = check_array(B);
   if (rc) return rc;
   rc = check_array(Y);
   if (rc) return rc;
-  if (!is_fp8(A->dtype) || !is_fp8(B->dtype) || !is_wide(Y->dtype)) return SCALIFY_ERR_DTYPE;
+  // the plain call writes a 16- or 32-bit intermediate; with a bias the sum may also be cast straight to FP8
+  if (!is_fp8(A->dtype) || !is_fp8(B->dtype) || (!bias && !is_wide(Y->dtype))) return SCALIFY_ERR_DTYPE;
+  if (bias) {
+    if ((rc = check_array(bias))) return rc;
+    if (!is_wide(bias->dtype)) return SCALIFY_ERR_DTYPE;
+    if (stat_hint) return SCALIFY_ERR_UNSUPPORTED;
+    if (Y->scale && Y->scale == bias->scale) return SCALIFY_ERR_ALIAS;
+  }
   if (!valid_stat(stat)) return SCALIFY_ERR_VALUE;
   if (A->ndim < 2 || A->ndim > 3 || B->ndim < 2 || Y->ndim != A->ndim || B->ndim > A->ndim) return SCALIFY_ERR_SHAPE;
   const int an = A->ndim, bn = B->ndim, yn = Y->ndim;
@@ -643,6 +650,7 @@ static int matmul_impl(const scalify_array* A, int transA, const scalify_array* 
   const int64_t N = transB ? B->shape[bn - 2] : B->shape[bn - 1];
   if (K != Kb || K < 1 || M < 1 || N < 1 || batch < 1) return SCALIFY_ERR_SHAPE;
   if (Y->shape[yn - 2] != M || Y->shape[yn - 1] != N) return SCALIFY_ERR_SHAPE;
+  if (bias && (bias->ndim != 1 || bias->shape[0] != N)) return SCALIFY_ERR_SHAPE;
   if (an == 3 && (Y->shape[0] != batch || (bn == 3 && B->shape[0] != batch))) return SCALIFY_ERR_SHAPE;
   if (M > 0x7FFFFFFF || N > 0x7FFFFFFF || K > 0x7FFFFFFF || batch > 0x7FFFFFFF) return SCALIFY_ERR_SHAPE;
   if (Y->scale && (Y->scale == A->scale || Y->scale == B->scale)) return SCALIFY_ERR_ALIAS;
@@ -674,6 +682,9 @@ static int matmul_impl(const scalify_array* A, int transA, const scalify_array* 
   a.force_ncta = 0;
   a.alpha_override = 0.f;
   a.no_split = 0;
+  a.bias = bias ? bias->data : nullptr;
+  a.bias_dt = bias ? bias->dtype : 0;
+  a.bias_scale = bias ? bias->scale : nullptr;
   a.stat_hint = nullptr;
   a.Yq = nullptr;
   a.q_dt = SCALIFY_E4M3;
@@ -704,14 +715,21 @@ static int matmul_impl(const scalify_array* A, int transA, const scalify_array* 
 
 int scalify_scaled_matmul(const scalify_array* A, int transA, const scalify_array* B, int transB, scalify_array* Y,
                           int stat, scalify_array* Yq, void* workspace, size_t workspace_bytes, void* stream) {
-  return matmul_impl(A, transA, B, transB, Y, stat, Yq, nullptr, workspace, workspace_bytes, stream);
+  return matmul_impl(A, transA, B, transB, nullptr, Y, stat, Yq, nullptr, workspace, workspace_bytes, stream);
+}
+
+int scalify_scaled_matmul_bias(const scalify_array* A, int transA, const scalify_array* B, int transB,
+                               const scalify_array* bias, scalify_array* Y, int stat, scalify_array* Yq,
+                               void* workspace, size_t workspace_bytes, void* stream) {
+  if (!bias) return SCALIFY_ERR_NULL;
+  return matmul_impl(A, transA, B, transB, bias, Y, stat, Yq, nullptr, workspace, workspace_bytes, stream);
 }
 
 int scalify_scaled_matmul_speculative(const scalify_array* A, int transA, const scalify_array* B, int transB,
                                       scalify_array* Y, scalify_array* Yq, float* stat_hint, void* workspace,
                                       size_t workspace_bytes, void* stream) {
   if (!stat_hint || !Yq) return SCALIFY_ERR_NULL;
-  return matmul_impl(A, transA, B, transB, Y, SCALIFY_STAT_AMAX, Yq, stat_hint, workspace, workspace_bytes, stream);
+  return matmul_impl(A, transA, B, transB, nullptr, Y, SCALIFY_STAT_AMAX, Yq, stat_hint, workspace, workspace_bytes, stream);
 }
 
 int scalify_scaled_matmul_delayed(const scalify_array* A, int transA, const scalify_array* B, int transB,
@@ -754,6 +772,7 @@ int scalify_scaled_matmul_delayed(const scalify_array* A, int transA, const scal
   a.force_ncta = 0;
   a.alpha_override = 0.f;
   a.no_split = 0;
+  a.bias = nullptr; a.bias_dt = 0; a.bias_scale = nullptr;
   a.stat_hint = nullptr;
   a.Yq = nullptr;
   a.q_dt = SCALIFY_E4M3;

@@ -79,6 +79,7 @@ struct MatmulArgs {
   // speculative rescale: predicted statistic (device) or NULL; then Yq (FP8, dense like Y) is written by the GEMM
   const float* stat_hint;
   void* Yq; int q_dt;
+  const void* bias; int bias_dt; const float* bias_scale;  // optional [N] vector added in the epilogue (add rule)
   float alpha_override;  // 0: the data component is divided by kf(K); otherwise multiplied by this (split-K partials)
   int no_split;          // 1: never split the contraction (the partial products of a split call)
 };

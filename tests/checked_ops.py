@@ -109,6 +109,27 @@ class Ops:
                     assert np.array_equal(self.bits(Yq).reshape(-1), qo)
         return (Y, Yq) if q_dt is not None else Y
 
+    def linear(self, X, W, bias, out_dt=BF):
+        """Y = X W + bias in one launch: [n, K] x [K, N] + [N], one rounding to out_dt (FP8 allowed)."""
+        n, N = X.data.shape[0], W.data.shape[1]
+        Y = self.empty((n, N), out_dt)
+        sc.scalify_scaled_matmul_bias(X, W, bias, Y, self.ws)
+        self.calls += 1
+        if self.check:
+            o = self.orc
+            self._status_ok()
+            _, ab_s, acc, sab = o.scaled_matmul(self.bits(X), code(X.data), X.scale_value(), self.bits(W), code(W.data),
+                                                W.scale_value(), F32, want_acc=True)
+            bs = bias.scale_value()
+            ys = max(ab_s, bs)
+            assert Y.scale_value() == ys
+            bv = o.decode(self.bits(bias), code(bias.data))
+            exact = acc * (ab_s / ys) + bv[None, :] * (bs / ys)
+            mag = sab * (ab_s / ys) + np.abs(bv)[None, :] * (bs / ys)
+            ok = self.within(self.bits(Y), o.encode(exact, out_dt), out_dt, exact, mag, 1e-5)
+            assert ok.all(), int((~ok).sum())
+        return Y
+
     # ---------------------------------------------------------------- add
     def add(self, A, B, subtract=False, out_dt=None):
         Y = self.empty(A.data.shape, out_dt if out_dt is not None else code(A.data))

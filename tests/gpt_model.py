@@ -96,8 +96,8 @@ class ScaledGPT:
         return sc.ScaledTensor(X.data.view(c.batch, c.seq, c.heads, hd).permute(0, 2, 1, 3), X.scale)
 
     def _linear(self, x8, W8, bias, out_dt=BF):
-        y = self.ops.mm(x8, W8)                       # [n, K] x [K, N], B stored [K, N]
-        return self.ops.add(y, self.ops.cast(bias, BF), out_dt=out_dt)   # the bias add may write FP8 directly
+        # [n, K] x [K, N] (B stored [K, N]) + bias in the matmul's epilogue; the sum may be written as FP8 directly
+        return self.ops.linear(x8, W8, bias, out_dt=out_dt)
 
     def _linear_bwd(self, dy, x8, W8):
         """dy BF16 -> (dx BF16, dW E5M2 rescaled, db E5M2 rescaled)."""

@@ -64,7 +64,7 @@ def test_reduced_gpt_step_every_call_checked_and_model_invariance():
     tgt = torch.from_numpy(si.uniform_int(5, 902, (n,), cfg.vocab))
     ref_loss, ref_grads = torch_reference(model, ids, tgt)
     loss = model.step(ids.cuda(), tgt.cuda(), t=1)
-    assert ops.calls > 200
+    assert ops.calls > 150
     got_loss = float(loss.item())
     assert abs(got_loss - ref_loss) < 0.02 * ref_loss, (got_loss, ref_loss)
     # gradients as handed to the optimizer (E5M2 data x power-of-two scale) against fp64 autograd

@@ -345,3 +345,39 @@ def test_split_contraction_with_a_large_workspace(M, N, K, transA, transB):
         one = run_matmul(a, orc.E4M3, 2.0 ** -2, b, orc.E5M2, 2.0 ** -9, orc.F32, transA, transB)
         many = run_matmul(a, orc.E4M3, 2.0 ** -2, b, orc.E5M2, 2.0 ** -9, orc.F32, transA, transB, splitk=True)
         assert not np.array_equal(one["Y"], many["Y"])
+
+
+@pytest.mark.parametrize("M,N,K,transB", [(256, 256, 256, True), (520, 304, 384, False), (100, 48, 128, True),
+                                          (8192, 768, 768, False)])
+@pytest.mark.parametrize("y_dt,bias_dt", [(orc.BF16, orc.BF16), (orc.F32, orc.F32), (orc.E4M3, orc.F16)])
+def test_matmul_with_bias_in_the_epilogue(M, N, K, transB, y_dt, bias_dt):
+    """Y = A B + bias by the add rule with ONE rounding: Y_s = max(A_s B_s kf(K), bias_s), both terms brought to
+    it by exact powers of two.  The exact value comes from the oracle's exact accumulation; bars as for the
+    plain matmul (1 ulp of the output format, or half an ulp plus 1e-5 of the summed magnitudes)."""
+    a = si.to_bits(si.normal(51, M, (M, K), 1.0), orc.E4M3)
+    b = si.to_bits(si.normal(52, N, (N, K) if transB else (K, N), 1.0), orc.E4M3)
+    for a_s, b_s, bias_s in ((2.0 ** -3, 2.0 ** -6, 2.0 ** -6), (1.0, 2.0 ** -6, 2.0 ** 2)):
+        bias = si.to_bits(si.normal(53, N, (N,), 1.0), bias_dt)
+        A = sc.ScaledTensor.make(to_dev(a, orc.E4M3), a_s)
+        B = sc.ScaledTensor.make(to_dev(b, orc.E4M3), b_s)
+        Bi = sc.ScaledTensor.make(to_dev(bias, bias_dt), bias_s)
+        Y = sc.ScaledTensor.empty((M, N), sc.TORCH_DTYPE[y_dt])
+        ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_MATMUL, M, N))
+        sc.scalify_scaled_matmul_bias(A, B, Bi, Y, ws, transB=transB, stat=sc.STAT_AMAX)
+        assert ws.check_status() == 0
+        rows = np.arange(M) if M <= 520 else np.random.default_rng(1).integers(0, M, 300)
+        _, ab_s, acc, sab = orc.scaled_matmul(a[rows], orc.E4M3, a_s, b, orc.E4M3, b_s, orc.F32, transB=transB,
+                                              want_acc=True)
+        kf = orc.kf(K)
+        assert ab_s == a_s * b_s * kf
+        ys = max(ab_s, bias_s)
+        assert Y.scale_value() == ys
+        fa, fb = ab_s / ys, bias_s / ys
+        bv = orc.decode(bias, bias_dt)
+        exact = acc * fa + bv[None, :] * fb          # acc: the exact data component of the product, (A_d B_d) / kf(K)
+        mag = sab * fa + np.abs(bv)[None, :] * fb
+        got = to_bits(Y.data, y_dt)[rows]
+        ok = within(got, orc.encode(exact, y_dt), y_dt, exact, mag, 1e-5)
+        assert ok.all(), int((~ok).sum())
+        if M <= 520:
+            assert float(ws.statistic().item()) == float(np.abs(orc.decode(got, y_dt)).max())
