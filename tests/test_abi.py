@@ -118,3 +118,10 @@ def test_validation_rejects_bad_arguments_on_the_host():
     A4 = _arr(4096, sc.E4M3, (1, 1, 128, 64))
     assert L.scalify_scaled_matmul(R(A4), 0, R(A4), 1, R(_arr(1 << 20, sc.BF16, (1, 1, 128, 128))), 0, None, 1 << 21,
                                    1 << 20, None) == -3
+    # matmul with a bias: the vector is required, wide and of length N
+    Yb = _arr(1 << 20, sc.BF16, (128, 256))
+    assert L.scalify_scaled_matmul_bias(R(A), 0, R(B), 0, None, R(Yb), 0, None, 1 << 21, 1 << 20, None) == -1
+    assert L.scalify_scaled_matmul_bias(R(A), 0, R(B), 0, R(_arr(1 << 22, sc.BF16, (128,))), R(Yb), 0, None, 1 << 21,
+                                        1 << 20, None) == -3
+    assert L.scalify_scaled_matmul_bias(R(A), 0, R(B), 0, R(_arr(1 << 22, sc.E4M3, (256,))), R(Yb), 0, None, 1 << 21,
+                                        1 << 20, None) == -2
