@@ -104,6 +104,11 @@ class ClockSampler:
                 break
             time.sleep(self.period)
 
+    def mark(self):
+        """Start of the timed region: what was sampled before (NVML start-up, warm-up) is dropped."""
+        self.samples = []
+        self.reasons = set()
+
     def stop(self):
         if self._thread is None:
             return dict(sm_mhz=None, sm_max_mhz=self.max_mhz, reasons=[f"unavailable: {self.err}"])
@@ -517,6 +522,8 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    # the sampler thread starts before the warm-up, so that NVML's start-up is over when the timed region begins
+    sampler = ClockSampler(local_rank) if rank == 0 else None
     for t in range(W):
         step(t, None, args.speculative)
     barrier()
@@ -526,8 +533,9 @@ def main():
             raise SystemExit(f"device status {st} after warm-up")
 
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(n_ev)] for _ in range(K)]
-    sampler = ClockSampler(local_rank) if rank == 0 else None
     barrier()
+    if sampler is not None:
+        sampler.mark()
     t_start = torch.cuda.Event(enable_timing=True)
     t_end = torch.cuda.Event(enable_timing=True)
     t_start.record()
