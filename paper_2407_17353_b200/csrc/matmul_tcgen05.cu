@@ -835,9 +835,15 @@ static int make_map_y(CUtensorMap* map, const void* ptr, int es, uint64_t N, uin
 }
 
 size_t matmul_splitk_ws_bytes(int64_t rows, int64_t cols) {
-  const size_t ldp = static_cast<size_t>((cols + 3) / 4 * 4);
-  const size_t n = kWsHeader + kSplitStatBytes + 16 * static_cast<size_t>(rows) * ldp * sizeof(float) + 256;
   const size_t base = matmul_ws_bytes(rows, cols);
+  // the most parts launch_scaled_matmul would cut a product of this output size into (none for a large output)
+  const int ncta = rows > kBM ? 2 : 1;
+  const int64_t out_tiles = ((rows + kBM * ncta - 1) / (kBM * ncta)) * ((cols + kBN - 1) / kBN);
+  int64_t splits = (ncta == 2 ? sm_count() / 2 : sm_count()) / (out_tiles > 0 ? out_tiles : 1);
+  if (splits > 16) splits = 16;
+  if (splits < 3) return base;
+  const size_t ldp = static_cast<size_t>((cols + 3) / 4 * 4);
+  const size_t n = kWsHeader + kSplitStatBytes + static_cast<size_t>(splits) * static_cast<size_t>(rows) * ldp * sizeof(float) + 256;
   return n > base ? n : base;
 }
 
