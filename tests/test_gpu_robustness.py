@@ -133,3 +133,81 @@ def test_adam_writes_only_its_state(n):
     assert ws.check_status() == 0
     for raw, meta in bufs.values():
         assert_guards_intact(raw, meta)
+
+
+@pytest.mark.parametrize("H,Tq,Tk,causal", [(2, 200, 224, True), (1, 96, 32, False), (3, 129, 160, True)])
+def test_attention_forward_and_backward_write_only_their_outputs(H, Tq, Tk, causal):
+    """Ragged lengths: the last query / key blocks are partial; rows past the end, the padding after
+    each 64-element row and the bytes around the buffers must stay untouched."""
+    HD = 64
+
+    def f8(tid, T, bits_dt, dt):
+        return sc.ScaledTensor.make(to_dev(si.scaled_normal(83, tid, (H, T, HD), bits_dt), bits_dt).view(dt), 1.0)
+
+    Q, K, V = (f8(1, Tq, si.E4M3, torch.float8_e4m3fn), f8(2, Tk, si.E4M3, torch.float8_e4m3fn),
+               f8(3, Tk, si.E4M3, torch.float8_e4m3fn))
+    dO = f8(4, Tq, si.E5M2, torch.float8_e5m2)
+    outs = {}
+    for name, T in (("O", Tq), ("dQ", Tq), ("dK", Tk), ("dV", Tk)):
+        raw, view, meta = guarded((H * T, HD), torch.bfloat16, row_pad=8)
+        ld = view.stride(0)
+        heads = view.as_strided((H, T, HD), (T * ld, ld, 1), view.storage_offset())
+        outs[name] = (raw, meta, sc.ScaledTensor(heads, torch.zeros(1, device="cuda")))
+    rawp, pview, mp = guarded((H * Tq, Tk), torch.float8_e4m3fn)
+    raws, sview, ms = guarded((H * Tq, Tk), torch.float8_e5m2)
+    P = sc.ScaledTensor(pview.view(H, Tq, Tk), None)
+    dS = sc.ScaledTensor(sview.view(H, Tq, Tk), torch.zeros(1, device="cuda"))
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    sc.scalify_scaled_attention(Q, K, V, outs["O"][2], sm_scale=0.125, causal=causal, P_dump=P, status=status)
+    sc.scalify_scaled_attention_bwd(Q, K, V, P, dO, dS, outs["dQ"][2], outs["dK"][2], outs["dV"][2], sm_scale=0.125,
+                                    causal=causal, status=status)
+    assert int(status.item()) == 0
+    for raw, meta, t in outs.values():
+        assert_guards_intact(raw, meta)
+        assert torch.isfinite(t.data.float()).all()
+    assert_guards_intact(rawp, mp)
+    assert_guards_intact(raws, ms)
+
+
+@pytest.mark.parametrize("R,N", [(1, 16), (37, 1030), (300, 48)])
+def test_column_sums_write_only_their_output(R, N):
+    ld = (N // 16 + 2) * 16
+    X = sc.ScaledTensor.make(to_dev(si.scaled_normal(84, 1, (R, ld), si.E5M2), si.E5M2)[:, :N], 1.0)
+    raw, view, meta = guarded((N,), torch.bfloat16)
+    Y = sc.ScaledTensor(view, torch.zeros(1, device="cuda"))
+    ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_COLSUM, R, N))
+    sc.scalify_scaled_colsum(X, Y, ws)
+    assert ws.check_status() == 0
+    assert_guards_intact(raw, meta)
+    assert torch.isfinite(view.float()).all()
+
+
+@pytest.mark.parametrize("M,N,K", [(130, 272, 144), (257, 528, 2048), (64, 48, 4096)])
+def test_bias_and_split_matmul_write_only_their_output(M, N, K):
+    A = sc.ScaledTensor.make(to_dev(si.scaled_normal(85, 1, (M, K), si.E4M3), si.E4M3), 1.0)
+    Bt = sc.ScaledTensor.make(to_dev(si.scaled_normal(85, 2, (N, K), si.E4M3), si.E4M3), 1.0)
+    bias = sc.ScaledTensor.make(torch.ones(N, device="cuda").to(torch.bfloat16), 0.25)
+    for kind in ("bias", "split"):
+        raw, view, meta = guarded((M, N), torch.bfloat16, row_pad=24)
+        Y = sc.ScaledTensor(view, torch.empty(1, dtype=torch.float32, device="cuda"))
+        ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_MATMUL_SPLITK if kind == "split" else sc.OP_MATMUL, M, N))
+        if kind == "bias":
+            sc.scalify_scaled_matmul_bias(A, Bt, bias, Y, ws, transB=True, stat=sc.STAT_AMAX)
+        else:
+            sc.scalify_scaled_matmul(A, Bt, Y, ws, transB=True, stat=sc.STAT_L2)
+        assert ws.check_status() == 0
+        assert_guards_intact(raw, meta)
+        assert torch.isfinite(view.float()).all()
+
+
+@pytest.mark.parametrize("rows,K", [(1, 128), (300, 256)])
+def test_block_quantiser_writes_only_its_data(rows, K):
+    X = sc.ScaledTensor.make(to_dev(si.scaled_normal(86, 1, (rows, K), si.BF16), si.BF16), 1.0)
+    Y = sc.MxTensor(rows, K)
+    raw, view, meta = guarded((rows, K), torch.float8_e4m3fn)
+    Y.data = view
+    Y._d.data = view.data_ptr()
+    sc.scalify_mx_quantize(X, Y)
+    torch.cuda.synchronize()
+    assert_guards_intact(raw, meta)
+    assert torch.isfinite(view.float()).all()
