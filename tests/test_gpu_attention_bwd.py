@@ -32,7 +32,8 @@ def oracle_probabilities(q, q_dt, qs, k, ks, c, causal):
     return np.stack(out)
 
 
-def run_case(H, Tq, Tk, causal, merged_layout=False, q_dt=orc.E4M3, do_dt=orc.E5M2, g_dt=orc.BF16, seed=1):
+def run_case(H, Tq, Tk, causal, merged_layout=False, q_dt=orc.E4M3, do_dt=orc.E5M2, g_dt=orc.BF16, seed=1,
+             check_heads=None):
     qs, ks, vs, dos, c = 2.0 ** -1, 2.0 ** 1, 2.0 ** -3, 2.0 ** -9, 0.125
     q = si.to_bits(si.normal(seed, 1, (H, Tq, HD), 1.0), q_dt)
     k = si.to_bits(si.normal(seed, 2, (H, Tk, HD), 1.0), orc.E4M3)
@@ -86,7 +87,7 @@ def run_case(H, Tq, Tk, causal, merged_layout=False, q_dt=orc.E4M3, do_dt=orc.E5
     else:
         visited = np.ones((Tq, Tk), dtype=bool)
         visible = visited
-    for h in range(H):
+    for h in (range(H) if check_heads is None else check_heads):
         assert np.all(P[h][~visible] == 0)
         # dP
         dPo, dp_scale, acc, sab = orc.scaled_matmul(do[h], do_dt, dos, v[h], orc.E4M3, vs, orc.BF16, transB=True,
@@ -126,6 +127,10 @@ def run_case(H, Tq, Tk, causal, merged_layout=False, q_dt=orc.E4M3, do_dt=orc.E5
 @pytest.mark.parametrize("H,T", [(2, 128), (3, 256), (2, 1024)])
 def test_causal_self_attention_backward(H, T):
     run_case(H, T, T, True)
+
+
+def test_backward_benchmark_shape_96_heads_of_1024_tokens_sampled_heads():
+    run_case(96, 1024, 1024, True, seed=11, check_heads=[0, 1, 37, 73, 94, 95])
 
 
 def test_full_attention_backward_with_more_keys_than_queries():

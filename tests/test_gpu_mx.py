@@ -172,6 +172,35 @@ def test_quantize_then_matmul_matches_the_oracle_pipeline():
     assert rel < 0.05
 
 
+def test_quantize_and_matmul_full_size_8192_sampled():
+    """The benchmark's block-scaled row at its full size: sampled rows of both quantised operands are
+    bit-exact, sampled outputs agree with the oracle, and the statistic word is the AMAX of what was stored."""
+    n = 8192
+    xa = wide_range_input(41, n, n, orc.BF16, spread=8)
+    xb = wide_range_input(42, n, n, orc.BF16, spread=8)
+    A, B = sc.MxTensor(n, n), sc.MxTensor(n, n)
+    sc.scalify_mx_quantize(sc.ScaledTensor.make(to_dev(xa, orc.BF16), 0.5), A)
+    sc.scalify_mx_quantize(sc.ScaledTensor.make(to_dev(xb, orc.BF16), 2.0), B)
+    Y = sc.ScaledTensor.empty((n, n), torch.bfloat16)
+    ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_MATMUL, n, n))
+    sc.scalify_mx_matmul(A, B, Y, ws, stat=sc.STAT_AMAX)
+    assert ws.check_status() == 0
+    rng = np.random.default_rng(9)
+    rows = np.unique(np.concatenate([rng.integers(0, n, 40), [0, 127, 128, 255, 256, n - 129, n - 1]]))
+    cols = np.unique(np.concatenate([rng.integers(0, n, 40), [0, 255, 256, 511, 512, n - 257, n - 1]]))
+    da, ea = orc.mx_quantize(xa[rows], orc.BF16, orc.E4M3)
+    db, eb = orc.mx_quantize(xb[cols], orc.BF16, orc.E4M3)
+    tr, tc = torch.from_numpy(rows).cuda(), torch.from_numpy(cols).cuda()
+    assert np.array_equal(to_bits(A.data[tr], orc.E4M3), da) and np.array_equal(to_bits(B.data[tc], orc.E4M3), db)
+    assert np.array_equal(A.exponents()[tr].cpu().numpy(), ea) and np.array_equal(B.exponents()[tc].cpu().numpy(), eb)
+    Yo, ys, acc, sab = orc.mx_matmul(da, orc.E4M3, ea, 0.5, db, orc.E4M3, eb, 2.0, orc.BF16, want_acc=True)
+    assert Y.scale_value() == ys
+    got = to_bits(Y.data[tr][:, tc], orc.BF16)
+    ok = within(got, Yo, orc.BF16, acc, sab, 1e-5)
+    assert ok.all(), int((~ok).sum())
+    assert float(ws.statistic().item()) == float(Y.data.float().abs().max())
+
+
 def test_mx_argument_checks():
     A = sc.MxTensor(64, 128)
     B = sc.MxTensor(32, 256)
