@@ -375,8 +375,16 @@ __device__ __forceinline__ float ce_exp2(float x) {
   return r;
 }
 
+__device__ __forceinline__ void ce_cp_async16(void* smem_dst, const void* gmem_src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst))),
+               "l"(gmem_src)
+               : "memory");
+}
+
+constexpr int kCeThreads = 512;
+
 template <int LDT, int GDT>
-__global__ void __launch_bounds__(256, 2) cross_entropy_smem_kernel(const void* __restrict__ logits, long long ld,
+__global__ void __launch_bounds__(kCeThreads, 2) cross_entropy_smem_kernel(const void* __restrict__ logits, long long ld,
                                                                     int n_classes, const long long* __restrict__ targets,
                                                                     long long n, const float* l_scale,
                                                                     void* __restrict__ dlogits, float rem,
@@ -385,7 +393,7 @@ __global__ void __launch_bounds__(256, 2) cross_entropy_smem_kernel(const void* 
   constexpr int VEC = 16 / ElemBytes<LDT>::v;
   constexpr int GB = VEC * ElemBytes<GDT>::v;
   extern __shared__ uint4 s_row[];
-  __shared__ float s_red[8];
+  __shared__ float s_red[kCeThreads / 32];
   __shared__ float s_bcast;
   const float ls = load_scale(l_scale) * 1.4426950408889634f;  // positive: the maximum commutes with it
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -393,43 +401,49 @@ __global__ void __launch_bounds__(256, 2) cross_entropy_smem_kernel(const void* 
   const int n_part = n_classes - nv_full * VEC;      // classes in the one partial vector (0: none)
   const int nv = nv_full + (n_part ? 1 : 0);
   const int nv_ld = static_cast<int>(ld / VEC);      // vectors of the padded row (the gradient covers them all)
+  // A row travels as 16-byte asynchronous copies straight into shared memory (about 100 KB in flight per
+  // block for a 50k vocabulary, no registers held) and the three sweeps read it from there.  Every sweep
+  // gives thread t the vectors t, t + 512, ...: a thread reads only what it copied itself, so the copies
+  // need no barrier, and the last sweep refills each slot with the NEXT row's vector as soon as it has
+  // read it - the next row loads behind this row's exponentials.
+  auto row_ptr = [&](long long r) {
+    return reinterpret_cast<const uint4*>(static_cast<const char*>(logits) + r * ld * ElemBytes<LDT>::v);
+  };
+  if (blockIdx.x < n) {
+    const uint4* first = row_ptr(blockIdx.x);
+    for (int v = threadIdx.x; v < nv; v += kCeThreads) ce_cp_async16(&s_row[v], first + v);
+  }
+  asm volatile("cp.async.commit_group;" ::: "memory");
   for (long long row = blockIdx.x; row < n; row += gridDim.x) {
-    const uint4* lrow = reinterpret_cast<const uint4*>(static_cast<const char*>(logits) + row * ld * ElemBytes<LDT>::v);
+    const uint4* lrow = row_ptr(row);
+    const long long next = row + gridDim.x;
+    const uint4* nrow = row_ptr(next < n ? next : row);
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
     float mraw = -INFINITY;  // maximum of the data component
-    for (int v0 = threadIdx.x; v0 < nv; v0 += 256 * 8) {  // eight 16-byte loads in flight per thread
-      uint4 w[8];
+    for (int v = threadIdx.x; v < nv; v += kCeThreads) {
+      const uint4 w = s_row[v];
+      float f[VEC];
+      decode_vec<LDT, VEC>(reinterpret_cast<const uint32_t*>(&w), f);
+      if (v < nv_full) {
 #pragma unroll
-      for (int u = 0; u < 8; ++u)
-        if (v0 + u * 256 < nv) w[u] = __ldcs(lrow + v0 + u * 256);
+        for (int e = 0; e < VEC; ++e) mraw = fmaxf(mraw, f[e]);
+      } else {
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const int v = v0 + u * 256;
-        if (v < nv) {
-          s_row[v] = w[u];
-          float f[VEC];
-          decode_vec<LDT, VEC>(reinterpret_cast<const uint32_t*>(&w[u]), f);
-          if (v < nv_full) {
-#pragma unroll
-            for (int e = 0; e < VEC; ++e) mraw = fmaxf(mraw, f[e]);
-          } else {
-#pragma unroll
-            for (int e = 0; e < VEC; ++e)
-              if (e < n_part) mraw = fmaxf(mraw, f[e]);
-          }
-        }
+        for (int e = 0; e < VEC; ++e)
+          if (e < n_part) mraw = fmaxf(mraw, f[e]);
       }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mraw = fmaxf(mraw, __shfl_xor_sync(0xFFFFFFFFu, mraw, o));
     __syncthreads();
     if (lane == 0) s_red[warp] = mraw;
-    __syncthreads();  // also: the row is in shared memory
+    __syncthreads();
     mraw = s_red[0];
 #pragma unroll
-    for (int k = 1; k < 8; ++k) mraw = fmaxf(mraw, s_red[k]);
+    for (int k = 1; k < kCeThreads / 32; ++k) mraw = fmaxf(mraw, s_red[k]);
     const float mx = mraw * ls;
     float sum4[4] = {0.f, 0.f, 0.f, 0.f};
-    for (int v = threadIdx.x; v < nv; v += 256) {
+    for (int v = threadIdx.x; v < nv; v += kCeThreads) {
       const uint4 w = s_row[v];
       float f[VEC];
       decode_vec<LDT, VEC>(reinterpret_cast<const uint32_t*>(&w), f);
@@ -448,7 +462,7 @@ __global__ void __launch_bounds__(256, 2) cross_entropy_smem_kernel(const void* 
     __syncthreads();
     sum = 0.f;
 #pragma unroll
-    for (int k = 0; k < 8; ++k) sum += s_red[k];
+    for (int k = 0; k < kCeThreads / 32; ++k) sum += s_red[k];
     long long t = targets[row];
     if (t < 0 || t >= n_classes) {
       if (threadIdx.x == 0 && bad_index) atomicOr(bad_index, static_cast<uint32_t>(SCALIFY_DEV_BAD_INDEX));
@@ -464,10 +478,11 @@ __global__ void __launch_bounds__(256, 2) cross_entropy_smem_kernel(const void* 
       const float k = s_bcast;
       const int tv = static_cast<int>(t / VEC), te = static_cast<int>(t % VEC);
       char* grow = static_cast<char*>(dlogits) + row * ld * ElemBytes<GDT>::v;
-      for (int v = threadIdx.x; v < nv_ld; v += 256) {
+      for (int v = threadIdx.x; v < nv_ld; v += kCeThreads) {
         float g[VEC];
         if (v < nv) {
           const uint4 w = s_row[v];
+          if (next < n) ce_cp_async16(&s_row[v], nrow + v);
           float f[VEC];
           decode_vec<LDT, VEC>(reinterpret_cast<const uint32_t*>(&w), f);
 #pragma unroll
@@ -490,9 +505,11 @@ __global__ void __launch_bounds__(256, 2) cross_entropy_smem_kernel(const void* 
         encode_vec<GDT, VEC>(g, o);
         st_raw_stream<GB>(grow + static_cast<long long>(v) * GB, o);
       }
-      for (long long j = static_cast<long long>(nv_ld) * VEC + threadIdx.x; j < ld; j += 256) store_elem<GDT>(grow, j, 0.f);
+      for (long long j = static_cast<long long>(nv_ld) * VEC + threadIdx.x; j < ld; j += kCeThreads) store_elem<GDT>(grow, j, 0.f);
+    } else if (next < n) {
+      for (int v = threadIdx.x; v < nv; v += kCeThreads) ce_cp_async16(&s_row[v], nrow + v);
     }
-    __syncthreads();  // the row buffer is rewritten by the next row's first sweep
+    asm volatile("cp.async.commit_group;" ::: "memory");
   }
 }
 
@@ -543,7 +560,7 @@ int launch_cross_entropy(const void* logits, int l_dt, long long ld, int n_class
         SCALIFY_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kCeSmemMax));
         attr_done = true;
       }
-      kernel<<<grid2, 256, static_cast<size_t>(row_smem), st>>>(logits, ld, n_classes, targets, n, l_scale, dlogits, rem,
+      kernel<<<grid2, kCeThreads, static_cast<size_t>(row_smem), st>>>(logits, ld, n_classes, targets, n, l_scale, dlogits, rem,
                                                                row_loss, v.status);
     }));
   } else {

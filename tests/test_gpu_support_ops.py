@@ -100,9 +100,11 @@ def test_softmax_backward(shape, p_dt, o_dt):
     assert within(to_bits(dS.data, o_dt), so, o_dt, exact, mag, 4e-6).all()
 
 
-@pytest.mark.parametrize("n,V,ld", [(16, 37, 48), (12, 1000, 1008), (64, 50257, 50304)])
+@pytest.mark.parametrize("n,V,ld", [(16, 37, 48), (12, 1000, 1008), (64, 50257, 50304), (700, 1000, 1008),
+                                    (901, 4099, 4112)])
 @pytest.mark.parametrize("g_dt", [orc.BF16, orc.E5M2, orc.F32])
 def test_cross_entropy_and_gradient(n, V, ld, g_dt):
+    # (the last two cases give every block several rows: the next row is copied in behind the current one)
     logits = si.scaled_normal(75, 1, (n, ld), orc.BF16, 3.0)
     tgt = si.uniform_int(75, 2, (n,), V)
     L = ST(logits, orc.BF16, 2.0 ** -1)
@@ -120,6 +122,10 @@ def test_cross_entropy_and_gradient(n, V, ld, g_dt):
     exact = orc.decode(g64, orc.F32)
     assert within(got, go, g_dt, exact, np.abs(exact) + 1e-6, 8e-6).all()
     assert np.all(orc.decode(got, g_dt)[:, V:] == 0.0)
+    # the loss alone (no gradient written) is the same number
+    loss2 = torch.zeros(1, dtype=torch.float32, device="cuda")
+    sc.scalify_scaled_cross_entropy(L, V, torch.from_numpy(tgt).cuda(), loss2, None, ws)
+    assert ws.check_status() == 0 and float(loss2.item()) == float(loss.item())
     # out-of-range target is reported
     bad = tgt.copy()
     bad[1] = V
