@@ -71,3 +71,23 @@ def within(got_bits, want_bits, dtype, exact, err_mag, c):
     err = np.abs(orc.decode(got_bits, dtype) - exact)
     with np.errstate(invalid="ignore"):
         return (d <= 1) | (err <= 0.5 * ulp_of(exact, dtype) + c * err_mag)
+
+
+def layernorm_bwd_delayed(G, gr_dtype, gr_scale, X, x_dtype, x_scale, gamma, g_dtype, g_scale, eps, eps_inside_sqrt,
+                          stat_in, stat, dx_dtype, dg_dtype):
+    """LayerNorm backward with DELAYED rescaling of the input gradient (Section 3.3 applied to the
+    rescale site of Section 4): a composition of the oracle's pieces, no arithmetic of its own beyond
+    the division by r.  The gradient is written already rebalanced by r = p2f(stat_in) (1 if stat_in
+    cannot define a scale), rounded once from the oracle's fp64 derivative, and this step's statistic
+    is taken on the un-rebalanced, unrounded derivative.
+    Returns dict(dX, dX_scale, stat, dgamma, dgamma_scale, dbeta, dbeta_scale, dx_f64, r)."""
+    o = orc.layernorm_bwd(G, gr_dtype, gr_scale, X, x_dtype, x_scale, gamma, g_dtype, g_scale, eps, eps_inside_sqrt,
+                          orc.F32, dg_dtype, want_f64=True)
+    usable = np.isfinite(stat_in) and stat_in >= 2.0 ** -126
+    r = orc.p2f(float(stat_in)) if usable else 1.0
+    dx = o["dx_f64"]
+    o["dX"] = orc.encode(dx / r, dx_dtype)
+    o["dX_scale"] = o["dX_scale"] * r
+    o["stat"] = float(np.abs(dx).max()) if stat == orc.STAT_AMAX else float(np.sqrt(np.mean(dx * dx)))
+    o["r"] = r
+    return o

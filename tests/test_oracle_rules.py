@@ -421,3 +421,32 @@ def test_delayed_matmul_equals_matmul_followed_by_rescale_with_the_old_statistic
         assert s_now == np.abs(acc).max()
     _, _, s_l2 = orc.scaled_matmul_delayed(A, orc.E4M3, 0.5, B, orc.E4M3, 2.0, 1.0, orc.STAT_L2, orc.BF16)
     assert abs(s_l2 - np.sqrt(np.mean(acc ** 2))) < 1e-12
+
+
+def test_delayed_layernorm_bwd_composition_reduces_to_the_plain_call_and_keeps_values():
+    """The composition the GPU tests use for the delayed LayerNorm gradient (tests/helpers.py): with a
+    statistic that cannot define a scale it IS the plain oracle call; with any other the represented
+    values are unchanged up to one rounding of the output format, the scale moves by exactly p2f(stat_in),
+    and the statistic handed on is that of the un-rebalanced derivative."""
+    from helpers import layernorm_bwd_delayed, ulp_of
+    R, d = 12, 48
+    G = si.scaled_normal(33, 1, (R, d), orc.BF16)
+    X = si.scaled_normal(33, 2, (R, d), orc.BF16)
+    gam = si.to_bits(1.0 + 0.1 * si.normal(33, 3, (d,), 1.0), orc.BF16)
+    args = (G, orc.BF16, 2.0 ** -10, X, orc.BF16, 0.5, gam, orc.BF16, 1.0, 1e-5, False)
+    plain = orc.layernorm_bwd(*args, orc.E5M2, orc.F32, want_f64=True)
+    for bad in (0.0, float("inf"), float("nan"), 2.0 ** -130):
+        o = layernorm_bwd_delayed(*args, bad, orc.STAT_AMAX, orc.E5M2, orc.F32)
+        assert o["r"] == 1.0 and o["dX_scale"] == plain["dX_scale"] and np.array_equal(o["dX"], plain["dX"])
+    dx = plain["dx_f64"]
+    for stat_in in (9.0, 0.3, 2.0 ** -7, 1.0):
+        o = layernorm_bwd_delayed(*args, stat_in, orc.STAT_L2, orc.E5M2, orc.F32)
+        m, e = math.frexp(o["r"])
+        assert m == 0.5 and o["r"] <= stat_in < 2 * o["r"]                 # the power of two below the statistic
+        assert o["dX_scale"] == plain["dX_scale"] * o["r"]
+        vals_q = orc.decode(o["dX"], orc.E5M2) * o["r"]                        # back at the static scale
+        assert np.all(np.abs(vals_q - dx) <= 0.5 * ulp_of(dx / o["r"], orc.E5M2) * o["r"])
+        assert abs(o["stat"] - np.sqrt(np.mean(dx * dx))) < 1e-15
+        assert np.array_equal(o["dgamma"], plain["dgamma"]) and o["dgamma_scale"] == plain["dgamma_scale"]
+    o = layernorm_bwd_delayed(*args, 1.0, orc.STAT_AMAX, orc.E5M2, orc.F32)
+    assert o["stat"] == np.abs(dx).max()
