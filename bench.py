@@ -339,7 +339,7 @@ def run_hbm_sweep(args):
         for d in (768, 1024, 4096):
             per_set = R * d * 2 * 4
             sets = max(1, min(8, -(-2 * l2 // per_set)))
-            fw, bw = [], []
+            fw, bw, bwd_delayed = [], [], []
             gamma = sc.ScaledTensor.make(torch.ones(d, device=dev).to(torch.bfloat16), 1.0)
             beta = sc.ScaledTensor.make(torch.zeros(d, device=dev).to(torch.bfloat16), 1.0)
             ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_LAYERNORM_BWD, R, d), dev)
@@ -358,9 +358,15 @@ def run_hbm_sweep(args):
                 bw.append(lambda G=G, X=X, mean=mean, rinv=rinv, dX=dX, dXq=dXq, dg=dg, db=db:
                           sc.scalify_scaled_layernorm_bwd(G, X, gamma, mean, rinv, dX, ws, eps=1e-5, stat_dx=sc.STAT_L2,
                                                           dXq=dXq, dgamma=dg, dbeta=db))
+                bwd_delayed.append(lambda G=G, X=X, mean=mean, rinv=rinv, dXq=dXq, dg=dg, db=db:
+                                   sc.scalify_scaled_layernorm_bwd_delayed(G, X, gamma, mean, rinv, ws.statistic(), dXq, ws,
+                                                                           eps=1e-5, stat_dx=sc.STAT_L2, dgamma=dg,
+                                                                           dbeta=db))
             report(f"LayerNorm fwd {R}x{d} BF16->BF16", timed(fw, iters), R * d * 4 + R * 8, sets, R * d * 4)
             report(f"LayerNorm bwd + L2 rescale to E5M2 {R}x{d}", timed(bw, iters), R * d * 9 + R * 8, sets, R * d * 6)
-            del fw, bw
+            report(f"LayerNorm bwd, delayed L2 rescale, E5M2 out in one pass {R}x{d}", timed(bwd_delayed, iters),
+                   R * d * 5 + R * 8, sets, R * d * 5)
+            del fw, bw, bwd_delayed
             torch.cuda.empty_cache()
     for lg in (23, 26, 28):
         n = 1 << lg
@@ -587,6 +593,25 @@ def main():
     barrier()
     delayed_ms = d0.elapsed_time(d1) / d_iters if d_iters else float("nan")
 
+    # LayerNorm backward with delayed rescale: E5M2 gradient in one pass with the previous step's statistic,
+    # this step's statistic left in the same word (5 B/elem instead of 9)
+    ln_stat = ws_ln.statistic()
+
+    def ln_delayed_step():
+        sc.scalify_scaled_layernorm_bwd_delayed(G, X, gamma, mean, rinv, ln_stat, dXq, ws_ln, eps=1e-5,
+                                                stat_dx=sc.STAT_L2, dgamma=dg, dbeta=db)
+    for _ in range(0 if args.no_next else 3):
+        ln_delayed_step()
+    barrier()
+    l0, l1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    l_iters = 0 if args.no_next else max(3, min(K, 20))
+    l0.record()
+    for _ in range(l_iters):
+        ln_delayed_step()
+    l1.record()
+    barrier()
+    ln_delayed_ms = l0.elapsed_time(l1) / l_iters if l_iters else float("nan")
+
     # Adam that also writes the E4M3 compute copy of the updated weight (1 more byte per parameter)
     awc = sc.ScaledTensor.make(torch.empty(ADAM_N, dtype=torch.float8_e4m3fn, device=dev), 1.0)
 
@@ -768,6 +793,8 @@ def main():
         {"row": "f1 (next, timed outside the step, back to back) delayed-rescale GEMM 8192^3: E4M3 out in one "
                 "kernel, no BF16 intermediate, no pass 2", "ms": round(float(delayed_ms), 4),
          "TFLOP/s": round(flops / (delayed_ms * 1e-3) / 1e12, 1)},
+        row("f1 (next, timed outside the step, back to back) LayerNorm bwd with delayed L2 rescale: E5M2 gradient "
+            "in one pass, no BF16 intermediate, no pass 2 (5 B/elem + 8 B/row)", ln_delayed_ms, 5 * n_ln + 8 * LN_R),
         {"row": "f1b (next, timed in a second pass of the same step) GEMM 8192^3 + EXACT dynamic AMAX rescale to E4M3 "
                 "with a predicted statistic: the GEMM writes BF16 and E4M3, a check launch confirms the prediction "
                 "(bit-identical to a1+a2+a3)",

@@ -303,6 +303,25 @@ int scalify_scaled_layernorm_bwd(const scalify_array* G, const scalify_array* X,
                                  void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The same backward pass with DELAYED rescaling of the input gradient (Section
+ * 3.3: statistic and rebalancing decoupled, the statistic of an earlier step
+ * kept in the caller's state), in ONE pass over G and X:
+ *   r = the power of two at or below *stat_in (1 if *stat_in is zero,
+ *   subnormal, Inf or NaN);  dX_d = cast(dx / r), rounded once from fp32;
+ *   dX_s = G_s*gamma_s / X_s * r.
+ * dX: [R,d] of ANY dtype (E5M2 for the gradient operand of the next matmul).
+ * stat_dx (AMAX or L2; NONE: nothing gathered) is taken on this step's
+ * un-rebalanced, unrounded dx and left at workspace offset 16 for the next
+ * step; stat_in (device, fp32, not NULL) may be that same word.  Everything
+ * else as scalify_scaled_layernorm_bwd.
+ */
+int scalify_scaled_layernorm_bwd_delayed(const scalify_array* G, const scalify_array* X, const scalify_array* gamma,
+                                         const float* mean, const float* rinv, float eps, int eps_inside_sqrt,
+                                         const float* stat_in, int stat_dx, scalify_array* dX,
+                                         scalify_array* dgamma, scalify_array* dbeta,
+                                         void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Scaled GELU forward / backward (Section 3.2.1 and Appendix C.1):
  *   forward  (X_d * g(X_d*X_s), X_s);   backward  dX_d = G_d * f'(X_d*X_s), dX_s = G_s.
  * exact_erf == 0: tanh form; != 0: Gaussian-CDF form.  X, G: F16/BF16/F32

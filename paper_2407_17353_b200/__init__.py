@@ -78,6 +78,7 @@ def lib() -> ctypes.CDLL:
         L.scalify_rescale.argtypes = [P, i32, vp, vp, P, vp, sz, vp]
         L.scalify_scaled_add.argtypes = [P, P, i32, P, vp]
         L.scalify_scaled_layernorm.argtypes = [P, P, P, f32, i32, P, vp, vp, vp]
+        L.scalify_scaled_layernorm_bwd_delayed.argtypes = [P, P, P, vp, vp, f32, i32, vp, i32, P, P, P, vp, sz, vp]
         L.scalify_scaled_layernorm_bwd.argtypes = [P, P, P, vp, vp, f32, i32, i32, P, P, P, P, vp, sz, vp]
         L.scalify_scaled_gelu.argtypes = [P, i32, P, vp]
         L.scalify_scaled_gelu_bwd.argtypes = [P, P, i32, P, vp]
@@ -286,6 +287,19 @@ def scalify_scaled_layernorm_bwd(G: ScaledTensor, X: ScaledTensor, gamma: Option
     _check(lib().scalify_scaled_layernorm_bwd(_ref(g), _ref(x), _ref(gm), _ptr(mean), _ptr(rinv), float(eps),
                                               int(eps_inside_sqrt), stat_dx, _ref(dx), _ref(dxq), _ref(dg), _ref(db),
                                               ws.ptr, ws.nbytes, _stream(stream)), "scalify_scaled_layernorm_bwd")
+
+
+def scalify_scaled_layernorm_bwd_delayed(G: ScaledTensor, X: ScaledTensor, gamma: Optional[ScaledTensor],
+                                         mean: torch.Tensor, rinv: torch.Tensor, stat_in: torch.Tensor, dX: ScaledTensor,
+                                         ws: Workspace, *, eps: float = 1e-5, eps_inside_sqrt=False,
+                                         stat_dx: int = STAT_NONE, dgamma: Optional[ScaledTensor] = None,
+                                         dbeta: Optional[ScaledTensor] = None, stream=None) -> None:
+    """LayerNorm backward writing the gradient already rebalanced by the power of two of an earlier statistic."""
+    g, x, gm, dx, dg, db = (_desc(G), _desc(X), _desc(gamma), _desc(dX), _desc(dgamma), _desc(dbeta))
+    _check(lib().scalify_scaled_layernorm_bwd_delayed(_ref(g), _ref(x), _ref(gm), _ptr(mean), _ptr(rinv), float(eps),
+                                                      int(eps_inside_sqrt), _ptr(stat_in), stat_dx, _ref(dx), _ref(dg),
+                                                      _ref(db), ws.ptr, ws.nbytes, _stream(stream)),
+           "scalify_scaled_layernorm_bwd_delayed")
 
 
 def scalify_scaled_gelu(X: ScaledTensor, Y: ScaledTensor, *, exact_erf=False, stream=None) -> None:

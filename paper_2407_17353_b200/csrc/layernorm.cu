@@ -312,14 +312,18 @@ template <int XDT, int DXDT, int TW, bool STAGED>
 __global__ void __launch_bounds__(kLnThreads, 2) layernorm_bwd_kernel(
     const void* __restrict__ G, int64_t g_ld, const void* __restrict__ X, int64_t x_ld, void* __restrict__ dX,
     int64_t dx_ld, int R, int d, const void* __restrict__ gamma, int gb_dt, const float* __restrict__ mean,
-    const float* __restrict__ rinv_in, float eps, int eps_inside, int stat, float* __restrict__ dgamma_part,
-    float* __restrict__ dbeta_part, double* __restrict__ stat_part) {
+    const float* __restrict__ rinv_in, float eps, int eps_inside, int stat, const float* __restrict__ stat_in,
+    float* __restrict__ dgamma_part, float* __restrict__ dbeta_part, double* __restrict__ stat_part) {
   asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   constexpr int VEC = 16 / ElemBytes<XDT>::v;
   constexpr int OB = VEC * ElemBytes<DXDT>::v;
   constexpr int TEAM = 32 * TW;
   constexpr int TPB = kLnThreads / TEAM;
   __shared__ float smem[2][8][2];
+  // delayed rescale (Section 3.3): the gradient is stored already divided by r = p2_floor(earlier statistic)
+  // and this step's statistic is taken on the un-rebalanced fp32 values
+  float inv_r = 1.0f;
+  if (stat_in) { bool nf; inv_r = 1.0f / rescale_factor(__ldg(stat_in), &nf); }
   const int n_vec = d / VEC;
   const int t = threadIdx.x % TEAM;
   const int team = threadIdx.x / TEAM;
@@ -456,10 +460,20 @@ __global__ void __launch_bounds__(kLnThreads, 2) layernorm_bwd_kernel(
           float o[VEC];
 #pragma unroll
           for (int e = 0; e < VEC; ++e) o[e] = fmaf(g[v][e], rinv, fmaf(x[v][e], -c2, nm1r));
-          uint32_t ow[OB / 4];
-          encode_vec<DXDT, VEC>(o, ow);
+          uint32_t ow[OB / 4 > 0 ? OB / 4 : 1];
+          if (stat_in) {
+            float oq[VEC];
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) oq[e] = o[e] * inv_r;  // exact: a power of two
+            encode_vec<DXDT, VEC>(oq, ow);
+          } else {
+            encode_vec<DXDT, VEC>(o, ow);
+          }
           st_raw<OB>(orow + int64_t(t + v * TEAM) * OB, ow);
-          if (stat == SCALIFY_STAT_AMAX) {
+          if (stat_in && stat == SCALIFY_STAT_L2) {
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) ssq = fmaf(o[e], o[e], ssq);
+          } else if (stat == SCALIFY_STAT_AMAX) {
             // rounding is monotonic: the max of the stored values is the stored value of the max
 #pragma unroll
             for (int e = 0; e < VEC; ++e) amax = max(amax, abs_bits(o[e]));
@@ -512,7 +526,7 @@ __global__ void __launch_bounds__(kLnThreads, 2) layernorm_bwd_kernel(
   if (stat != SCALIFY_STAT_NONE) {
     __shared__ double s_stat[kLnThreads / 32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (stat == SCALIFY_STAT_AMAX) amax = abs_bits(round_through<DXDT>(__uint_as_float(amax)));
+    if (stat == SCALIFY_STAT_AMAX && !stat_in) amax = abs_bits(round_through<DXDT>(__uint_as_float(amax)));
     double mine = (stat == SCALIFY_STAT_AMAX) ? static_cast<double>(warp_max_u32(amax))
                                               : warp_sum_f64(static_cast<double>(ssq));
     if (lane == 0) s_stat[warp] = mine;
@@ -533,7 +547,7 @@ __global__ void __launch_bounds__(1024) layernorm_bwd_finalize_kernel(
     int nblocks, int R, int d, const float* __restrict__ dgamma_part, const float* __restrict__ dbeta_part,
     const double* __restrict__ stat_part, int stat, float* stat_word, void* __restrict__ dgamma,
     void* __restrict__ dbeta, const float* g_scale, const float* x_scale, const float* gamma_scale,
-    float* dx_scale, float* dgamma_scale, float* dbeta_scale, uint32_t* status) {
+    float* dx_scale, float* dgamma_scale, float* dbeta_scale, const float* stat_in, uint32_t* status) {
   asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   // block = 8 columns (one 32-byte sector of a partial row) x 128 slices of the block list: 4 x as many
   // blocks as a 32-column layout, so the partials (a few MB in L2) are read by more SMs at once
@@ -567,6 +581,11 @@ __global__ void __launch_bounds__(1024) layernorm_bwd_finalize_kernel(
     }
   }
   if (blockIdx.x == 0 && warp == 1) {
+    // delayed rescale: the factor the main kernel divided by.  Read before this step's statistic is
+    // written, so the caller may keep both in the same word.
+    float r_prev = 1.0f;
+    if (stat_in) { bool nf; r_prev = rescale_factor(*stat_in, &nf); }
+    __syncwarp();
     if (stat != SCALIFY_STAT_NONE) {
       double tot = 0.0;
       for (int i = cx; i < nblocks; i += 32) {
@@ -589,7 +608,7 @@ __global__ void __launch_bounds__(1024) layernorm_bwd_finalize_kernel(
     if (cx == 0) {
       const float gs = load_scale(g_scale), xs = load_scale(x_scale), gms = load_scale(gamma_scale);
       uint32_t flags = (is_pow2_scale(gs) && is_pow2_scale(xs) && is_pow2_scale(gms)) ? 0u : SCALIFY_DEV_BAD_SCALE;
-      if (dx_scale) *dx_scale = gs * gms / xs;
+      if (dx_scale) *dx_scale = gs * gms / xs * r_prev;
       if (dgamma_scale) *dgamma_scale = gs * kfactor(R);
       if (dbeta_scale) *dbeta_scale = gs * kfactor(R);
       if (flags && status) atomicOr(status, flags);
@@ -609,7 +628,7 @@ int launch_layernorm_bwd(const void* G, int64_t g_ld, const void* X, int x_dt, i
                          int64_t dx_ld, int R, int d, const void* gamma, int gb_dt, const float* mean,
                          const float* rinv, float eps, int eps_inside, int stat, void* dgamma, void* dbeta, int dg_dt,
                          const float* g_scale, const float* x_scale, const float* gamma_scale, float* dx_scale,
-                         float* dgamma_scale, float* dbeta_scale, void* ws, cudaStream_t st) {
+                         float* dgamma_scale, float* dbeta_scale, const float* stat_in, void* ws, cudaStream_t st) {
   const int tw = ln_team_warps(d, x_dt);
   if (tw == 0) return SCALIFY_ERR_UNSUPPORTED;
   const int grid = ln_grid(R, 8 / tw, kLnBwdBlocksPerSm);
@@ -629,9 +648,10 @@ int launch_layernorm_bwd(const void* G, int64_t g_ld, const void* X, int x_dt, i
       attr_done = true;                                                                                          \
     }                                                                                                            \
     layernorm_bwd_kernel<XDT, DXDT, W, STG><<<grid, kLnThreads, STG ? kBwdSmem : 0, st>>>(                       \
-        G, g_ld, X, x_ld, dX, dx_ld, R, d, gamma, gb_dt, mean, rinv, eps, eps_inside, stat, dgp, dbp, st_part);  \
+        G, g_ld, X, x_ld, dX, dx_ld, R, d, gamma, gb_dt, mean, rinv, eps, eps_inside, stat, stat_in, dgp, dbp,   \
+        st_part);                                                                                                \
   } while (0)
-  SCALIFY_DISPATCH_WIDE(x_dt, XDT, SCALIFY_DISPATCH_WIDE(dx_dt, DXDT, {
+  SCALIFY_DISPATCH_WIDE(x_dt, XDT, SCALIFY_DISPATCH_DTYPE(dx_dt, DXDT, {
     switch (tw) {
       case 1: SCALIFY_LN_BWD(1, false); break;
       case 2: SCALIFY_LN_BWD(2, false); break;
@@ -645,7 +665,7 @@ int launch_layernorm_bwd(const void* G, int64_t g_ld, const void* X, int x_dt, i
   SCALIFY_DISPATCH_WIDE(dg_dt, DGDT,
       layernorm_bwd_finalize_kernel<DGDT><<<fgrid, 1024, 0, st>>>(grid, R, d, dgp, dbp, st_part, stat, v.stat, dgamma,
                                                                  dbeta, g_scale, x_scale, gamma_scale, dx_scale,
-                                                                 dgamma_scale, dbeta_scale, v.status));
+                                                                 dgamma_scale, dbeta_scale, stat_in, v.status));
   SCALIFY_CUDA_TRY(cudaGetLastError());
   return SCALIFY_OK;
 }

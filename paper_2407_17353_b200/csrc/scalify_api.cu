@@ -287,10 +287,10 @@ int scalify_scaled_layernorm(const scalify_array* X, const scalify_array* gamma,
                               eps_inside_sqrt ? 1 : 0, mean, rinv, static_cast<cudaStream_t>(stream));
 }
 
-int scalify_scaled_layernorm_bwd(const scalify_array* G, const scalify_array* X, const scalify_array* gamma,
-                                 const float* mean, const float* rinv, float eps, int eps_inside_sqrt, int stat_dx,
-                                 scalify_array* dX, scalify_array* dXq, scalify_array* dgamma, scalify_array* dbeta,
-                                 void* workspace, size_t workspace_bytes, void* stream) {
+static int layernorm_bwd_impl(const scalify_array* G, const scalify_array* X, const scalify_array* gamma,
+                              const float* mean, const float* rinv, float eps, int eps_inside_sqrt, int stat_dx,
+                              const float* stat_in, scalify_array* dX, scalify_array* dXq, scalify_array* dgamma,
+                              scalify_array* dbeta, void* workspace, size_t workspace_bytes, void* stream) {
   int rc = check_array(G);
   if (rc) return rc;
   rc = check_array(X);
@@ -298,7 +298,8 @@ int scalify_scaled_layernorm_bwd(const scalify_array* G, const scalify_array* X,
   rc = check_array(dX);
   if (rc) return rc;
   if (!mean || !rinv) return SCALIFY_ERR_NULL;
-  if (!is_wide(X->dtype) || G->dtype != X->dtype || !is_wide(dX->dtype)) return SCALIFY_ERR_DTYPE;
+  // the plain call keeps the un-rebalanced gradient in a wide format; the delayed one may round it once to FP8
+  if (!is_wide(X->dtype) || G->dtype != X->dtype || (!stat_in && !is_wide(dX->dtype))) return SCALIFY_ERR_DTYPE;
   if (!valid_stat(stat_dx)) return SCALIFY_ERR_VALUE;
   int64_t R, d, x_ld, Rg, dg, g_ld, Rd, dd, dx_ld;
   if (as_rows(X, &R, &d, &x_ld) || as_rows(G, &Rg, &dg, &g_ld) || as_rows(dX, &Rd, &dd, &dx_ld)) return SCALIFY_ERR_SHAPE;
@@ -340,7 +341,8 @@ int scalify_scaled_layernorm_bwd(const scalify_array* G, const scalify_array* X,
                             static_cast<int>(d), gamma ? gamma->data : nullptr, gb_dt, mean, rinv, eps,
                             eps_inside_sqrt ? 1 : 0, stat_dx, dgamma ? dgamma->data : nullptr,
                             dbeta ? dbeta->data : nullptr, dg_dt, G->scale, X->scale, gamma ? gamma->scale : nullptr,
-                            dx_scale, dgamma ? dgamma->scale : nullptr, dbeta ? dbeta->scale : nullptr, workspace, st);
+                            dx_scale, dgamma ? dgamma->scale : nullptr, dbeta ? dbeta->scale : nullptr, stat_in,
+                            workspace, st);
   if (rc) return rc;
   if (dXq) {
     WsView v = ws_view(workspace);
@@ -348,6 +350,23 @@ int scalify_scaled_layernorm_bwd(const scalify_array* G, const scalify_array* X,
                           kModeDynamic, v.status, st);
   }
   return rc;
+}
+
+int scalify_scaled_layernorm_bwd(const scalify_array* G, const scalify_array* X, const scalify_array* gamma,
+                                 const float* mean, const float* rinv, float eps, int eps_inside_sqrt, int stat_dx,
+                                 scalify_array* dX, scalify_array* dXq, scalify_array* dgamma, scalify_array* dbeta,
+                                 void* workspace, size_t workspace_bytes, void* stream) {
+  return layernorm_bwd_impl(G, X, gamma, mean, rinv, eps, eps_inside_sqrt, stat_dx, nullptr, dX, dXq, dgamma, dbeta,
+                            workspace, workspace_bytes, stream);
+}
+
+int scalify_scaled_layernorm_bwd_delayed(const scalify_array* G, const scalify_array* X, const scalify_array* gamma,
+                                         const float* mean, const float* rinv, float eps, int eps_inside_sqrt,
+                                         const float* stat_in, int stat_dx, scalify_array* dX, scalify_array* dgamma,
+                                         scalify_array* dbeta, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!stat_in) return SCALIFY_ERR_NULL;
+  return layernorm_bwd_impl(G, X, gamma, mean, rinv, eps, eps_inside_sqrt, stat_dx, stat_in, dX, nullptr, dgamma, dbeta,
+                            workspace, workspace_bytes, stream);
 }
 
 static int check_mx(const scalify_mx_array* a) {

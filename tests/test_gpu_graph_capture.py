@@ -150,7 +150,12 @@ def test_training_style_chain_with_state_replays_from_a_cuda_graph():
     ws_ln = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_LAYERNORM_BWD, R, D))
     ws_ce = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_CROSS_ENTROPY, R))
     ws_ad = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_ADAM, 1))
-    state = [stat_state, am.data, am.scale, av.data, av.scale, aw.data, aw.scale]
+    # delayed rescale of the LayerNorm gradient: the statistic word of its own workspace IS the state
+    ws_lnd = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_LAYERNORM_BWD, R, D))
+    ln_state = ws_lnd.statistic()
+    ln_state.fill_(2.0 ** -9)
+    dXd = sc.ScaledTensor.empty((R, D), torch.float8_e5m2)
+    state = [stat_state, ln_state, am.data, am.scale, av.data, av.scale, aw.data, aw.scale]
     saved = [x.clone() for x in state]
 
     def reset():
@@ -168,18 +173,20 @@ def test_training_style_chain_with_state_replays_from_a_cuda_graph():
         sc.scalify_scaled_gelu_bwd(dH, X, Ga)
         sc.scalify_scaled_layernorm_bwd(dH, X, gamma, mean, rinv, dX, ws_ln, eps=1e-5, stat_dx=sc.STAT_L2, dXq=dXq,
                                         dgamma=dgam, dbeta=dbet)
+        sc.scalify_scaled_layernorm_bwd_delayed(dH, X, gamma, mean, rinv, ln_state, dXd, ws_lnd, eps=1e-5,
+                                                stat_dx=sc.STAT_L2)
         sc.scalify_scaled_softmax(S, P, causal=True)
         sc.scalify_scaled_softmax_bwd(dP, P, dS)
         sc.scalify_scaled_embedding_bwd(ids, T, dX, dwte, dwpe)
         sc.scalify_scaled_adam_step_cast(adam, wc, ws_ad, lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, step=3)
 
-    outs = [logits, dlogits, dH, act, Ga, dX, dXq, dgam, dbet, P, dS, am, av, aw, awc]
+    outs = [logits, dlogits, dH, act, Ga, dX, dXq, dXd, dgam, dbet, P, dS, am, av, aw, awc]
     atomics = [dwte, dwpe]   # scatter-adds with fp32 atomics: the order of the addends is not fixed
 
     def snapshot():
         torch.cuda.synchronize()
         return [x.data.contiguous().view(torch.uint8).cpu().numpy().copy() for x in outs] + \
-               [np.array([x.scale_value() for x in outs] + [float(loss.item()), float(stat_state.item())])]
+               [np.array([x.scale_value() for x in outs] + [float(loss.item()), float(stat_state.item()), float(ln_state.item())])]
 
     reset()
     step()

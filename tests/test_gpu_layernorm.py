@@ -131,3 +131,65 @@ def test_layernorm_backward_with_gradient_rescale(R, d, eps_inside, stat):
     qo, qs, _ = orc.rescale(got, orc.BF16, o["dX_scale"], stat, orc.E5M2)
     assert dXq.scale_value() == qs
     assert np.array_equal(to_bits(dXq.data, orc.E5M2), qo)
+
+
+@pytest.mark.parametrize("R,d", [(1, 8), (37, 768), (300, 1024), (5, 4096), (1000, 768), (64, 80), (700, 4096)])
+@pytest.mark.parametrize("dx_dt", [orc.E5M2, orc.E4M3, orc.BF16])
+@pytest.mark.parametrize("stat,stat_in", [(sc.STAT_L2, 2.0 ** -7 * 1.3), (sc.STAT_AMAX, 0.011), (sc.STAT_AMAX, 0.0),
+                                          (sc.STAT_L2, float("inf"))])
+def test_layernorm_backward_with_delayed_rescale(R, d, dx_dt, stat, stat_in):
+    """One pass: the gradient is written already divided by the power of two of an EARLIER statistic
+    (Section 3.3), rounded once from fp32, and this step's statistic is that of the un-rebalanced values.
+    Bar: the plain backward's bar (1 ulp of the output format, or half an ulp plus 2^-18 of the row's
+    largest term), scale words exact, statistic 2e-6 relative (L2) or 2^-18 of the largest term (AMAX)."""
+    from helpers import layernorm_bwd_delayed, ulp_of
+    c = si.layernorm_case(R, d, seed=47)
+    x_s, g_s, gam_s = 2.0 ** 2, 2.0 ** -10, 2.0 ** -1
+    X, G, gamma = st(c["X"], orc.BF16, x_s), st(c["G"], orc.BF16, g_s), st(c["gamma"], orc.BF16, gam_s)
+    Y = sc.ScaledTensor.empty((R, d), torch.bfloat16)
+    mean = torch.empty(R, dtype=torch.float32, device="cuda")
+    rinv = torch.empty(R, dtype=torch.float32, device="cuda")
+    sc.scalify_scaled_layernorm(X, gamma, st(c["beta"], orc.BF16, 1.0), Y, eps=1e-5, mean=mean, rinv=rinv)
+    dX = sc.ScaledTensor.empty((R, d), sc.TORCH_DTYPE[dx_dt])
+    dg, db = sc.ScaledTensor.empty((d,), torch.float32), sc.ScaledTensor.empty((d,), torch.float32)
+    ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_LAYERNORM_BWD, R, d))
+    # the earlier statistic sits in the word this call overwrites with its own (the state of a training loop)
+    ws.statistic().fill_(stat_in)
+    sc.scalify_scaled_layernorm_bwd_delayed(G, X, gamma, mean, rinv, ws.statistic(), dX, ws, eps=1e-5, stat_dx=stat,
+                                            dgamma=dg, dbeta=db)
+    assert ws.check_status() == 0
+    o = layernorm_bwd_delayed(c["G"], orc.BF16, g_s, c["X"], orc.BF16, x_s, c["gamma"], orc.BF16, gam_s, 1e-5, False,
+                              stat_in, stat, dx_dt, orc.F32)
+    assert dX.scale_value() == o["dX_scale"]
+    assert dg.scale_value() == o["dgamma_scale"] and db.scale_value() == o["dbeta_scale"]
+    got = to_bits(dX.data, dx_dt)
+    gv = orc.decode(c["G"], orc.BF16) * orc.decode(c["gamma"], orc.BF16)[None, :]
+    _, _, _, ro = orc.layernorm_fwd(c["X"], orc.BF16, None, 0, 1.0, None, 0, 1.0, 1e-5, False, orc.BF16)
+    row_mag = np.abs(gv).max(axis=1) * ro / o["r"]
+    exact = o["dx_f64"] / o["r"]
+    abs_err = np.abs(orc.decode(got, dx_dt) - exact)
+    ok = (ulp_diff(got, o["dX"], dx_dt) <= 1) | (abs_err <= 0.5 * ulp_of(exact, dx_dt) + 2.0 ** -18 * row_mag[:, None])
+    assert ok.all(), int((~ok).sum())
+    gstat = float(ws.statistic().item())
+    if stat == sc.STAT_AMAX:
+        assert abs(gstat - o["stat"]) <= 2.0 ** -18 * (row_mag.max() * o["r"])
+    else:
+        assert abs(gstat - o["stat"]) <= 2e-6 * o["stat"]
+    # dgamma / dbeta do not depend on the rescale
+    plain_dg, plain_db = sc.ScaledTensor.empty((d,), torch.float32), sc.ScaledTensor.empty((d,), torch.float32)
+    dX2 = sc.ScaledTensor.empty((R, d), torch.bfloat16)
+    sc.scalify_scaled_layernorm_bwd(G, X, gamma, mean, rinv, dX2, ws, eps=1e-5, stat_dx=stat, dgamma=plain_dg,
+                                    dbeta=plain_db)
+    assert torch.equal(plain_dg.data, dg.data) and torch.equal(plain_db.data, db.data)
+
+
+def test_layernorm_backward_delayed_argument_checks():
+    R, d = 8, 64
+    X = sc.ScaledTensor.make(torch.zeros((R, d), dtype=torch.bfloat16, device="cuda"), 1.0)
+    dX = sc.ScaledTensor.empty((R, d), torch.float8_e5m2)
+    mean = torch.zeros(R, device="cuda")
+    ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_LAYERNORM_BWD, R, d))
+    with pytest.raises(sc.ScalifyError):   # the plain call keeps a wide gradient
+        sc.scalify_scaled_layernorm_bwd(X, X, None, mean, mean, dX, ws)
+    with pytest.raises(sc.ScalifyError):   # no earlier statistic
+        sc.scalify_scaled_layernorm_bwd_delayed(X, X, None, mean, mean, None, dX, ws)
