@@ -114,6 +114,16 @@ def test_layernorm_writes_only_its_outputs(R, d):
     assert ws.check_status() == 0
     for r_, m_ in ((rawd, md), (rawg, mg), (rawb, mb)):
         assert_guards_intact(r_, m_)
+    # delayed rescale: FP8 rows (8 bytes per vector of a BF16 input) in a padded buffer
+    rawq, qview, mq = guarded((R, d), torch.float8_e5m2, row_pad=16 + (-d) % 16)
+    dXq = sc.ScaledTensor(qview, torch.empty(1, dtype=torch.float32, device="cuda"))
+    ws.statistic().fill_(2.0 ** -9)
+    sc.scalify_scaled_layernorm_bwd_delayed(g, x, gamma, mean, rinv, ws.statistic(), dXq, ws, stat_dx=sc.STAT_AMAX,
+                                            dgamma=dg, dbeta=db)
+    assert ws.check_status() == 0
+    for r_, m_ in ((rawq, mq), (rawg, mg), (rawb, mb)):
+        assert_guards_intact(r_, m_)
+    assert torch.isfinite(qview.float()).all()
 
 
 @pytest.mark.parametrize("n", [1, 9, 8195])
