@@ -92,6 +92,15 @@ def test_validation_rejects_bad_arguments_on_the_host():
     # layernorm row length must be a multiple of 16 bytes
     assert L.scalify_scaled_layernorm(R(_arr(4096, sc.BF16, (4, 60), (64, 1))), None, None, 1e-5, 0,
                                       R(_arr(8192, sc.BF16, (4, 60), (64, 1))), None, None, None) == -3
+    # layernorm backward: the plain call keeps a wide gradient, the delayed one needs the earlier statistic
+    Xl = _arr(4096, sc.BF16, (4, 64))
+    dX8 = _arr(1 << 20, sc.E5M2, (4, 64))
+    assert L.scalify_scaled_layernorm_bwd(R(Xl), R(Xl), None, 64, 128, 1e-5, 0, sc.STAT_L2, R(dX8), None, None, None,
+                                          1 << 21, 1 << 20, None) == -2
+    assert L.scalify_scaled_layernorm_bwd_delayed(R(Xl), R(Xl), None, 64, 128, 1e-5, 0, None, sc.STAT_L2, R(dX8), None,
+                                                  None, 1 << 21, 1 << 20, None) == -1
+    assert L.scalify_scaled_layernorm_bwd_delayed(R(Xl), R(Xl), None, 64, 128, 1e-5, 0, 256, 7, R(dX8), None,
+                                                  None, 1 << 21, 1 << 20, None) == -9
     # attention: head dimension, power-of-two scalar, batch views, required scale word of dS
     Q3 = _arr(4096, sc.E4M3, (2, 128, 64))
     O3 = _arr(1 << 20, sc.BF16, (2, 128, 64))
