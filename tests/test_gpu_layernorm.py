@@ -193,3 +193,37 @@ def test_layernorm_backward_delayed_argument_checks():
         sc.scalify_scaled_layernorm_bwd(X, X, None, mean, mean, dX, ws)
     with pytest.raises(sc.ScalifyError):   # no earlier statistic
         sc.scalify_scaled_layernorm_bwd_delayed(X, X, None, mean, mean, None, dX, ws)
+
+
+@pytest.mark.parametrize("R,d", [(37, 768), (300, 1024), (3, 16)])
+@pytest.mark.parametrize("x_dt,dx_dt", [(orc.F32, orc.E5M2), (orc.F32, orc.F32), (orc.F16, orc.E4M3), (orc.F16, orc.F16)])
+def test_layernorm_backward_delayed_other_input_formats(R, d, x_dt, dx_dt):
+    """fp32 and fp16 inputs (4 or 8 elements per 16-byte vector, so FP8 rows are written 4 or 8 bytes at a time)."""
+    from helpers import layernorm_bwd_delayed, ulp_of
+    Xb = si.scaled_normal(48, 1, (R, d), x_dt)
+    Gb = si.scaled_normal(48, 4, (R, d), x_dt)
+    gam = si.to_bits(1.0 + 0.1 * si.normal(48, 2, (d,)), orc.BF16)
+    x_s, g_s, gam_s, stat_in = 2.0 ** -2, 2.0 ** -10, 1.0, 0.37
+    X, G, gamma = st(Xb, x_dt, x_s), st(Gb, x_dt, g_s), st(gam, orc.BF16, gam_s)
+    Y = sc.ScaledTensor.empty((R, d), torch.float32)
+    mean = torch.empty(R, dtype=torch.float32, device="cuda")
+    rinv = torch.empty(R, dtype=torch.float32, device="cuda")
+    sc.scalify_scaled_layernorm(X, gamma, None, Y, eps=1e-5, eps_inside_sqrt=True, mean=mean, rinv=rinv)
+    dX = sc.ScaledTensor.empty((R, d), sc.TORCH_DTYPE[dx_dt])
+    ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_LAYERNORM_BWD, R, d))
+    state = torch.full((1,), stat_in, dtype=torch.float32, device="cuda")
+    sc.scalify_scaled_layernorm_bwd_delayed(G, X, gamma, mean, rinv, state, dX, ws, eps=1e-5, eps_inside_sqrt=True,
+                                            stat_dx=sc.STAT_AMAX)
+    assert ws.check_status() == 0 and float(state.item()) == np.float32(stat_in)   # a separate state word is only read
+    o = layernorm_bwd_delayed(Gb, x_dt, g_s, Xb, x_dt, x_s, gam, orc.BF16, gam_s, 1e-5, True, stat_in, orc.STAT_AMAX,
+                              dx_dt, orc.F32)
+    assert o["r"] == 0.25 and dX.scale_value() == o["dX_scale"]
+    got = to_bits(dX.data, dx_dt)
+    gv = orc.decode(Gb, x_dt) * orc.decode(gam, orc.BF16)[None, :]
+    _, _, _, ro = orc.layernorm_fwd(Xb, x_dt, None, 0, 1.0, None, 0, 1.0, 1e-5, True, orc.F32)
+    row_mag = np.abs(gv).max(axis=1) * ro / o["r"]
+    exact = o["dx_f64"] / o["r"]
+    abs_err = np.abs(orc.decode(got, dx_dt) - exact)
+    ok = (ulp_diff(got, o["dX"], dx_dt) <= 1) | (abs_err <= 0.5 * ulp_of(exact, dx_dt) + 2.0 ** -18 * row_mag[:, None])
+    assert ok.all(), int((~ok).sum())
+    assert abs(float(ws.statistic().item()) - o["stat"]) <= 2.0 ** -18 * (row_mag.max() * o["r"])
