@@ -221,3 +221,20 @@ def test_block_quantiser_writes_only_its_data(rows, K):
     torch.cuda.synchronize()
     assert_guards_intact(raw, meta)
     assert torch.isfinite(view.float()).all()
+
+
+@pytest.mark.parametrize("n,V,ld", [(700, 1000, 1008), (3, 37, 48)])
+def test_cross_entropy_writes_only_its_gradient(n, V, ld):
+    """Several rows per block: the kernel copies the next row in while it writes the current gradient row."""
+    logits = sc.ScaledTensor.make(to_dev(si.scaled_normal(87, 1, (n, ld), si.BF16, 3.0), si.BF16), 0.5)
+    tgt = torch.from_numpy(si.uniform_int(87, 2, (n,), V)).cuda()
+    raw, view, meta = guarded((n, ld), torch.float8_e5m2)
+    G = sc.ScaledTensor(view, torch.empty(1, dtype=torch.float32, device="cuda"))
+    rawl, lview, ml = guarded((1,), torch.float32)
+    ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_CROSS_ENTROPY, n))
+    sc.scalify_scaled_cross_entropy(logits, V, tgt, lview, G, ws)
+    assert ws.check_status() == 0
+    assert_guards_intact(raw, meta)
+    assert_guards_intact(rawl, ml)
+    assert torch.isfinite(view.float()).all() and bool(torch.isfinite(lview).all())
+    assert bool((view.float()[:, V:] == 0).all())
