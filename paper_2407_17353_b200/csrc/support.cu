@@ -393,7 +393,9 @@ __global__ void __launch_bounds__(kCeThreads, 2) cross_entropy_smem_kernel(const
   constexpr int VEC = 16 / ElemBytes<LDT>::v;
   constexpr int GB = VEC * ElemBytes<GDT>::v;
   extern __shared__ uint4 s_row[];
-  __shared__ float s_red[kCeThreads / 32];
+  // one array per reduction: a write is separated from the previous row's reads of the same array by the
+  // barriers of the other reduction, so no barrier is needed in front of it
+  __shared__ float s_max[kCeThreads / 32], s_sum[kCeThreads / 32];
   __shared__ float s_bcast;
   const float ls = load_scale(l_scale) * 1.4426950408889634f;  // positive: the maximum commutes with it
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -435,12 +437,11 @@ __global__ void __launch_bounds__(kCeThreads, 2) cross_entropy_smem_kernel(const
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mraw = fmaxf(mraw, __shfl_xor_sync(0xFFFFFFFFu, mraw, o));
+    if (lane == 0) s_max[warp] = mraw;
     __syncthreads();
-    if (lane == 0) s_red[warp] = mraw;
-    __syncthreads();
-    mraw = s_red[0];
+    mraw = s_max[0];
 #pragma unroll
-    for (int k = 1; k < kCeThreads / 32; ++k) mraw = fmaxf(mraw, s_red[k]);
+    for (int k = 1; k < kCeThreads / 32; ++k) mraw = fmaxf(mraw, s_max[k]);
     const float mx = mraw * ls;
     float sum4[4] = {0.f, 0.f, 0.f, 0.f};
     for (int v = threadIdx.x; v < nv; v += kCeThreads) {
@@ -457,12 +458,11 @@ __global__ void __launch_bounds__(kCeThreads, 2) cross_entropy_smem_kernel(const
       }
     }
     float sum = warp_sum_f32((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
-    __syncthreads();
-    if (lane == 0) s_red[warp] = sum;
+    if (lane == 0) s_sum[warp] = sum;
     __syncthreads();
     sum = 0.f;
 #pragma unroll
-    for (int k = 0; k < kCeThreads / 32; ++k) sum += s_red[k];
+    for (int k = 0; k < kCeThreads / 32; ++k) sum += s_sum[k];
     long long t = targets[row];
     if (t < 0 || t >= n_classes) {
       if (threadIdx.x == 0 && bad_index) atomicOr(bad_index, static_cast<uint32_t>(SCALIFY_DEV_BAD_INDEX));
