@@ -343,6 +343,16 @@ int scalify_debug_expire_wait(void* workspace, size_t workspace_bytes, uint32_t 
                               void* stream);
 
 /*
+ * Diagnostic (no counterpart in the paper): the launch shape the LayerNorm kernels would use for an
+ * [R,d] input of dtype x_dtype on the current device, so that a test can state which code path it
+ * exercised.  Host only, launches nothing.  plan[0] = thread blocks; plan[1] = rows every team of
+ * warps walks one after another (forward: consecutive rows of its block's run; backward: the
+ * persistent grid's stride loop); plan[2] = warps per row; plan[3] = rows kept in flight through
+ * shared memory (0: the backward kernel prefetches one row in registers instead).
+ */
+int scalify_debug_layernorm_plan(int64_t R, int64_t d, int x_dtype, int backward, int32_t plan[4]);
+
+/*
  * Multiply a ScaledArray by a scalar constant c that is a positive power of two (Section 3.4: a
  * broadcast scalar contributes the scale "c rounded down to a power of two" and its mantissa stays
  * in the data; for a power of two the mantissa is 1, so only the scale word changes: X_s *= c).

@@ -94,6 +94,7 @@ def lib() -> ctypes.CDLL:
         L.scalify_scaled_adam_step_cast.argtypes = [i32, P, P, P, P, P, f32, f32, f32, f32, i64, vp, sz, vp]
         L.scalify_debug_expire_wait.argtypes = [vp, sz, c.c_uint32, vp, vp]
         L.scalify_scalar_mul_pow2.argtypes = [P, f32, vp]
+        L.scalify_debug_layernorm_plan.argtypes = [i64, i64, i32, i32, vp]
         L.scalify_scaled_embedding.argtypes = [vp, i64, i64, P, P, P, vp, vp]
         L.scalify_scaled_embedding_bwd.argtypes = [vp, i64, i64, P, P, P, vp]
         L.scalify_scaled_softmax.argtypes = [P, i32, P, vp]
@@ -107,6 +108,7 @@ def lib() -> ctypes.CDLL:
                      "scalify_scaled_adam_step", "scalify_scaled_adam_step_cast", "scalify_scaled_adam_step_static", "scalify_scaled_embedding",
                      "scalify_scaled_embedding_bwd", "scalify_scaled_softmax", "scalify_scaled_softmax_bwd",
                      "scalify_scaled_cross_entropy", "scalify_scalar_mul_pow2", "scalify_debug_expire_wait",
+                     "scalify_debug_layernorm_plan",
                      "scalify_mx_quantize", "scalify_mx_matmul", "scalify_scaled_attention",
                      "scalify_scaled_attention_bwd", "scalify_scaled_colsum", "scalify_scaled_matmul_bias",
                      "scalify_scaled_matmul_speculative"):
@@ -406,6 +408,14 @@ def scalify_scalar_mul_pow2(X: ScaledTensor, c: float, *, stream=None) -> None:
 def scalify_debug_expire_wait(ws: Workspace, limit_us: int, waited_us: Optional[torch.Tensor] = None, *, stream=None) -> None:
     _check(lib().scalify_debug_expire_wait(ws.ptr, ws.nbytes, int(limit_us), _ptr(waited_us), _stream(stream)),
            "scalify_debug_expire_wait")
+
+
+def scalify_debug_layernorm_plan(R: int, d: int, x_dtype: int, backward: bool) -> dict:
+    """Launch shape of the LayerNorm kernels for an [R, d] input (host only, launches nothing)."""
+    out = (ctypes.c_int32 * 4)()
+    _check(lib().scalify_debug_layernorm_plan(int(R), int(d), int(x_dtype), int(bool(backward)),
+                                              ctypes.cast(out, ctypes.c_void_p)), "scalify_debug_layernorm_plan")
+    return dict(grid=out[0], rows_per_team=out[1], team_warps=out[2], stages=out[3])
 
 
 class MxTensor:

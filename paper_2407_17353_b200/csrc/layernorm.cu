@@ -251,25 +251,38 @@ static int ln_team_warps(int d, int x_dt) {
   return 0;
 }
 
-int launch_layernorm_fwd(const void* X, int x_dt, int64_t x_ld, void* Y, int y_dt, int64_t y_ld, int R, int d,
-                         const void* gamma, const void* beta, int gb_dt, const float* gamma_scale,
-                         const float* beta_scale, float* y_scale, float eps, int eps_inside, float* mean,
-                         float* rinv, cudaStream_t st) {
-  int tw = ln_team_warps(d, x_dt);
-  if (tw == 0) return SCALIFY_ERR_UNSUPPORTED;
+// Launch shape of the forward kernel: team width, vectors per thread, rows each team walks, grid.
+struct LnFwdPlan { int tw, vpt, rpt, grid; bool ok; };
+static LnFwdPlan ln_fwd_plan(int R, int d, int x_dt) {
+  LnFwdPlan p{};
+  p.tw = ln_team_warps(d, x_dt);
+  p.ok = p.tw != 0;
+  if (!p.ok) return p;
   // rows of more than 64 vectors: four vectors per thread and a quarter of the warps per row (65..128 vectors:
   // one warp, no cross-warp step; up to 512 vectors: four warps, so a block works on two rows at a time)
   const int n_vec = d * elem_size(x_dt) / 16;
   const bool wide = n_vec > 64;
-  if (wide) tw = n_vec <= 128 ? 1 : (n_vec <= 256 ? 2 : 4);
+  if (wide) p.tw = n_vec <= 128 ? 1 : (n_vec <= 256 ? 2 : 4);
+  p.vpt = wide ? 4 : 2;
   // Blocks are not persistent: each owns a short run of consecutive rows (6 per team) and the
   // hardware scheduler hands out the runs in address order.  Measured on B200 (131072 x 1024 BF16):
   // 90 us, against 104 us for a grid of 3 blocks per SM striding over the rows, and 101 us with 16
   // rows per team (fewer, longer blocks leave a larger partial last wave).
-  const int tpb = 8 / tw;
-  int rpt = 6;
-  while (rpt > 1 && (int64_t(R) + tpb * rpt - 1) / (tpb * rpt) < 4 * int64_t(sm_count())) --rpt;
-  const int grid = static_cast<int>((int64_t(R) + tpb * rpt - 1) / (tpb * rpt));
+  const int tpb = 8 / p.tw;
+  p.rpt = 6;
+  while (p.rpt > 1 && (int64_t(R) + tpb * p.rpt - 1) / (tpb * p.rpt) < 4 * int64_t(sm_count())) --p.rpt;
+  p.grid = static_cast<int>((int64_t(R) + tpb * p.rpt - 1) / (tpb * p.rpt));
+  return p;
+}
+
+int launch_layernorm_fwd(const void* X, int x_dt, int64_t x_ld, void* Y, int y_dt, int64_t y_ld, int R, int d,
+                         const void* gamma, const void* beta, int gb_dt, const float* gamma_scale,
+                         const float* beta_scale, float* y_scale, float eps, int eps_inside, float* mean,
+                         float* rinv, cudaStream_t st) {
+  const LnFwdPlan plan = ln_fwd_plan(R, d, x_dt);
+  if (!plan.ok) return SCALIFY_ERR_UNSUPPORTED;
+  const int tw = plan.tw, rpt = plan.rpt, grid = plan.grid;
+  const bool wide = plan.vpt == 4;
 #define SCALIFY_LN_FWD(W, V)                                                                                   \
   do {                                                                                                         \
     /* row staging + gamma and beta (up to 4 bytes per element each) */                                       \
@@ -624,14 +637,42 @@ size_t layernorm_bwd_ws_bytes(int64_t R, int64_t d) {
   return kWsHeader + size_t(grid) * size_t(d) * 8 + size_t(grid) * 8 + 256;
 }
 
+// Launch shape of the backward kernel: team width, whether rows are staged through shared memory, grid
+// (persistent) and the number of rows each team walks.
+struct LnBwdPlan { int tw, staged, grid, iters; bool ok; };
+static LnBwdPlan ln_bwd_plan(int R, int d, int x_dt) {
+  LnBwdPlan p{};
+  p.tw = ln_team_warps(d, x_dt);
+  p.ok = p.tw != 0;
+  if (!p.ok) return p;
+  p.staged = p.tw >= 4;
+  p.grid = ln_grid(R, 8 / p.tw, kLnBwdBlocksPerSm);
+  const int64_t rows_per_iter = int64_t(p.grid) * (8 / p.tw);
+  p.iters = static_cast<int>((R + rows_per_iter - 1) / rows_per_iter);
+  return p;
+}
+
+int layernorm_plan(int64_t R, int64_t d, int x_dt, int backward, int32_t out[4]) {
+  if (backward) {
+    const LnBwdPlan p = ln_bwd_plan(static_cast<int>(R), static_cast<int>(d), x_dt);
+    if (!p.ok) return SCALIFY_ERR_UNSUPPORTED;
+    out[0] = p.grid; out[1] = p.iters; out[2] = p.tw; out[3] = p.staged ? kLnBwdStages : 0;
+  } else {
+    const LnFwdPlan p = ln_fwd_plan(static_cast<int>(R), static_cast<int>(d), x_dt);
+    if (!p.ok) return SCALIFY_ERR_UNSUPPORTED;
+    out[0] = p.grid; out[1] = p.rpt; out[2] = p.tw; out[3] = kLnFwdStages;
+  }
+  return SCALIFY_OK;
+}
+
 int launch_layernorm_bwd(const void* G, int64_t g_ld, const void* X, int x_dt, int64_t x_ld, void* dX, int dx_dt,
                          int64_t dx_ld, int R, int d, const void* gamma, int gb_dt, const float* mean,
                          const float* rinv, float eps, int eps_inside, int stat, void* dgamma, void* dbeta, int dg_dt,
                          const float* g_scale, const float* x_scale, const float* gamma_scale, float* dx_scale,
                          float* dgamma_scale, float* dbeta_scale, const float* stat_in, void* ws, cudaStream_t st) {
-  const int tw = ln_team_warps(d, x_dt);
-  if (tw == 0) return SCALIFY_ERR_UNSUPPORTED;
-  const int grid = ln_grid(R, 8 / tw, kLnBwdBlocksPerSm);
+  const LnBwdPlan plan = ln_bwd_plan(R, d, x_dt);
+  if (!plan.ok) return SCALIFY_ERR_UNSUPPORTED;
+  const int tw = plan.tw, grid = plan.grid;
   WsView v = ws_view(ws);
   float* dg_part = static_cast<float*>(v.area);
   float* db_part = dg_part + size_t(grid) * d;

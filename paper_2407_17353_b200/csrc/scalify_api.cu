@@ -814,6 +814,13 @@ int scalify_debug_expire_wait(void* workspace, size_t workspace_bytes, uint32_t 
                             static_cast<cudaStream_t>(stream));
 }
 
+int scalify_debug_layernorm_plan(int64_t R, int64_t d, int x_dtype, int backward, int32_t plan[4]) {
+  if (!plan) return SCALIFY_ERR_NULL;
+  if (!is_wide(x_dtype)) return SCALIFY_ERR_DTYPE;
+  if (R < 1 || d < 1 || R > 0x7FFFFFFF || d > 0x7FFFFFFF || (d * elem_size(x_dtype)) % 16 != 0) return SCALIFY_ERR_SHAPE;
+  return layernorm_plan(R, d, x_dtype, backward, plan);
+}
+
 int scalify_scalar_mul_pow2(scalify_array* X, float c, void* stream) {
   if (!X || !X->scale) return SCALIFY_ERR_NULL;
   int ex;

@@ -38,6 +38,7 @@ int launch_layernorm_fwd(const void* X, int x_dt, int64_t x_ld, void* Y, int y_d
                          const float* beta_scale, float* y_scale, float eps, int eps_inside, float* mean,
                          float* rinv, cudaStream_t st);
 size_t layernorm_bwd_ws_bytes(int64_t R, int64_t d);
+int layernorm_plan(int64_t R, int64_t d, int x_dt, int backward, int32_t out[4]);
 int launch_layernorm_bwd(const void* G, int64_t g_ld, const void* X, int x_dt, int64_t x_ld, void* dX, int dx_dt,
                          int64_t dx_ld, int R, int d, const void* gamma, int gb_dt, const float* mean,
                          const float* rinv, float eps, int eps_inside, int stat, void* dgamma, void* dbeta, int dg_dt,

@@ -196,9 +196,7 @@ class Ops:
             ghat = o.decode(gb, xdt) * gv[None, :]
             row_mag = np.abs(ghat).max(axis=1) * ro
             got = self.bits(dX)
-            err = np.abs(o.decode(got, BF) - r["dx_f64"])
-            ok = (self.ulp_diff(got, r["dX"], BF) <= 1) | (err <= 0.5 * np.abs(r["dx_f64"]) * 2.0 ** -8 +
-                                                           2.0 ** -18 * row_mag[:, None])
+            ok = self.within(got, r["dX"], BF, r["dx_f64"], row_mag[:, None], 2.0 ** -18)
             assert ok.all(), int((~ok).sum())
             n32, _, _, _ = o.layernorm_fwd(xb, xdt, None, 0, 1.0, None, 0, 1.0, eps, False, F32)
             nv, Gd, f = o.decode(n32, F32), o.decode(gb, xdt), o.kf(R)

@@ -62,15 +62,49 @@ def ulp_of(x: np.ndarray, dtype: int) -> np.ndarray:
     return np.exp2(e - _MBITS[dtype])
 
 
-def within(got_bits, want_bits, dtype, exact, err_mag, c):
+# Every call of within() leaves a record here: (label, elements, elements accepted ONLY by the
+# cancellation clause).  conftest.py writes the totals per label at the end of a session when
+# SCALIFY_TOLERANCE_LOG names a file, so the share of outputs that lean on the wider clause is a
+# measured number and not an assumption.
+LOOSE_LOG = []
+_DT_NAME = {orc.E4M3: "e4m3", orc.E5M2: "e5m2", orc.F16: "f16", orc.BF16: "bf16", orc.F32: "f32"}
+
+# An output may need the cancellation clause only when the fp32 rounding error of the sum (a few
+# 2^-24 of its largest terms) exceeds an ulp of the RESULT, i.e. when |result| is below about
+# 2^(mantissa bits) * 2^-22 of its terms: 2^-15 of them for BF16, 2^-19 / 2^-20 for FP8.  For the
+# Gaussian workloads here that is far below one output in a hundred, so a kernel that is more than
+# 1 ulp off on ordinary outputs exceeds the cap and fails, whatever c and err_mag are.
+LOOSE_CAP = 0.01
+LOOSE_FLOOR = 2   # tiny arrays: a couple of outputs near a zero crossing are not a share
+
+
+def _caller_label():
+    import inspect
+    for fr in inspect.stack()[2:8]:
+        if fr.function.startswith("test_") or fr.function in ("smoke",):
+            return fr.function
+    return inspect.stack()[2].function
+
+
+def within(got_bits, want_bits, dtype, exact, err_mag, c, loose_cap=LOOSE_CAP, label=None):
     """Mask of acceptable outputs for a result computed in fp32 and rounded once to `dtype`:
     within 1 ulp of the oracle's encoding, or |value - exact| <= ulp(exact)/2 + c * err_mag, where
     err_mag is the magnitude of the terms that were added (a sum that cancels has an error
-    relative to its terms, not to its result)."""
+    relative to its terms, not to its result).  The second clause may carry at most `loose_cap` of
+    the outputs (plus LOOSE_FLOOR of them): beyond that the outputs it alone accepted count as
+    failures.  The number it carried is recorded in LOOSE_LOG.  An fp32 OUTPUT is the exception: it comes
+    out of several fp32 operations, so it is a few fp32 ulp from the fp64 result on every element and the
+    second clause (c * err_mag, a few 2^-24 of the terms) is its bar; no cap applies."""
     d = ulp_diff(got_bits, want_bits, dtype)
     err = np.abs(orc.decode(got_bits, dtype) - exact)
+    tight = d <= 1
     with np.errstate(invalid="ignore"):
-        return (d <= 1) | (err <= 0.5 * ulp_of(exact, dtype) + c * err_mag)
+        loose = ~tight & (err <= 0.5 * ulp_of(exact, dtype) + c * err_mag)
+    n, n_loose = int(tight.size), int(loose.sum())
+    LOOSE_LOG.append(((label or _caller_label()) + ":" + _DT_NAME[dtype], n, n_loose))
+    if dtype != orc.F32 and n_loose > loose_cap * n + LOOSE_FLOOR:
+        return tight
+    return tight | loose
 
 
 def layernorm_bwd_delayed(G, gr_dtype, gr_scale, X, x_dtype, x_scale, gamma, g_dtype, g_scale, eps, eps_inside_sqrt,

@@ -173,8 +173,7 @@ def test_mlp_block_forward_and_backward():
     ghat = orc.decode(bits(dH0, BF), BF) * gv[None, :]
     row_mag = np.abs(ghat).max(axis=1) * ro
     got = bits(dX, BF)
-    err = np.abs(orc.decode(got, BF) - o["dx_f64"])
-    ok = (ulp_diff(got, o["dX"], BF) <= 1) | (err <= 0.5 * np.abs(o["dx_f64"]) * 2.0 ** -8 + 2.0 ** -18 * row_mag[:, None])
+    ok = within(got, o["dX"], BF, o["dx_f64"], row_mag[:, None], 2.0 ** -18)
     assert ok.all(), int((~ok).sum())
     so = orc.statistic(got, BF, orc.STAT_L2)
     assert abs(float(L.ws.statistic().item()) - so) <= 2e-6 * so
