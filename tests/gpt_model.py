@@ -109,7 +109,9 @@ class ScaledGPT:
         return dx, dW, db
 
     # ------------------------------------------------------------------ one training step
-    def step(self, ids, targets, t, lr=3e-4, beta1=0.9, beta2=0.999, eps=1e-8):
+    def step(self, ids, targets, t, lr=3e-4, beta1=0.9, beta2=0.999, eps=1e-8, check_layers=None):
+        """One training step.  check_layers: the transformer layers whose calls the Ops object checks (None: all);
+        embedding, head, loss, the parameter-gradient rescales and the optimizer are always checked."""
         c, o, P = self.cfg, self.ops, self.params
         d, H, T, B = c.d, c.heads, c.seq, c.batch
         hd = d // H
@@ -122,6 +124,7 @@ class ScaledGPT:
         x = o.embedding(ids, T, P["wte"], P["wpe"])
         for l in range(c.layers):
             p = f"h{l}."
+            o.active = check_layers is None or l in check_layers
             s = {"x_in": x}
             # producers write the E4M3 operand of the next matmul themselves (cast_on_forward fused in)
             s["h8"], s["mean1"], s["rinv1"] = o.ln(x, P[p + "ln1.g"], P[p + "ln1.b"], out_dt=E4)
@@ -158,6 +161,7 @@ class ScaledGPT:
             s["g8"] = g8 = o.gelu(a1, out_dt=E4)
             x = o.add(x, self._linear(g8, W8[p + "w2"], P[p + "b2"]))
             saved.append(s)
+        o.active = True
         hf8, meanf, rinvf = o.ln(x, P["lnf.g"], P["lnf.b"], out_dt=E4)
         logits_buf = torch.empty((n, c.vocab_padded), dtype=torch.bfloat16, device=self.dev)
         logits = sc.ScaledTensor(logits_buf[:, :c.vocab], torch.empty(1, dtype=torch.float32, device=self.dev))
@@ -171,6 +175,7 @@ class ScaledGPT:
         dx, grads["lnf.g"], grads["lnf.b"] = o.ln_bwd(dhf, x, P["lnf.g"], meanf, rinvf)
         for l in reversed(range(c.layers)):
             p = f"h{l}."
+            o.active = check_layers is None or l in check_layers
             s = saved[l]
             # MLP
             dg, grads[p + "w2"], grads[p + "b2"] = self._linear_bwd(dx, s["g8"], W8[p + "w2"])
@@ -204,6 +209,7 @@ class ScaledGPT:
                 dh = dxx if dh is None else o.add(dh, dxx)
             dln, grads[p + "ln1.g"], grads[p + "ln1.b"] = o.ln_bwd(dh, s["x_in"], P[p + "ln1.g"], s["mean1"], s["rinv1"])
             dx = o.add(dx, dln)
+        o.active = True
         dwte_emb, dwpe = o.embedding_bwd(ids, T, dx, c.vocab)
         grads["wte"] = o.rescale(o.add(dwte_head, dwte_emb), sc.STAT_AMAX, E5)
         grads["wpe"] = o.rescale(dwpe, sc.STAT_AMAX, E5)

@@ -5,9 +5,17 @@ Reduced shapes (vocab 1000 padded to 1024, seq 128, d 128, 2 heads, 2 layers, ba
 fp64 oracle can follow every one of the ~250 kernel launches of the step: each call is checked
 stage-isolated against the oracle on the library's own inputs (see checked_ops.Ops).  Then model
 invariance (Section 1): the loss and the gradients agree with an unscaled fp64 PyTorch evaluation
-of the same network to FP8 quantisation noise.  The GPT-2-small shapes themselves (12 layers,
-d 768, 12 heads, seq 1024, batch 8, vocab 50257) run through the same code unchecked in
-`test_full_size_step_runs`."""
+of the same network to FP8 quantisation noise.
+
+The GPT-2-small shapes themselves (12 layers, d 768, 12 heads, seq 1024, batch 8, vocab 50257) run
+through the same code in `test_full_size_step_checked_against_the_oracle_on_samples`: every call of
+the embedding, of three of the twelve layers (forward and backward), of the head, the loss, the
+parameter-gradient rescales and the optimizer is compared with the oracle on that call's own inputs:
+scale, statistic and status words exactly; matmul outputs on sampled positions; large row-wise
+arrays on sampled rows in full; LayerNorm, the residual adds, the parameter gradients and all 148
+tensors of the optimizer step in full."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -83,9 +91,23 @@ def test_reduced_gpt_step_every_call_checked_and_model_invariance():
     assert np.median(list(worst.values())) < 0.15
 
 
+def test_full_size_step_checked_against_the_oracle_on_samples():
+    cfg = GPTConfig()
+    ops = Ops(check="sampled")
+    model = ScaledGPT(cfg, ops, seed=6)
+    n = cfg.batch * cfg.seq
+    ids = torch.from_numpy(si.uniform_int(6, 901, (n,), cfg.vocab)).cuda()
+    tgt = torch.from_numpy(si.uniform_int(6, 902, (n,), cfg.vocab)).cuda()
+    # three layers keep the test under two minutes; SCALIFY_CHECK_ALL_LAYERS=1 checks all twelve
+    layers = None if os.environ.get("SCALIFY_CHECK_ALL_LAYERS") == "1" else (0, 5, 11)
+    loss = float(model.step(ids, tgt, t=1, check_layers=layers).item())
+    assert np.isfinite(loss) and abs(loss - np.log(cfg.vocab)) < 1.0, loss
+    assert ops.checked_calls > 300, ops.checked_calls
+
+
 def test_full_size_step_runs():
-    """GPT-2-small shapes, unchecked (the oracle cannot follow 7e12 flop): two steps run, the loss is finite
-    and near ln(vocab) for random weights, every scale stays a power of two, no status bit is raised."""
+    """GPT-2-small shapes, two consecutive steps without checks: the loss is finite and near ln(vocab) for
+    random weights, every scale stays a power of two, no status bit is raised."""
     cfg = GPTConfig()
     ops = Ops(check=False)
     model = ScaledGPT(cfg, ops, seed=6)
