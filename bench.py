@@ -298,6 +298,54 @@ def run_profile_row(args):
     print(json.dumps(out))
 
 
+def run_gpt_step(args):
+    """Config 5: the GPT-2-small-shaped training step (12 layers, d 768, 12 heads, 8 x 1024 tokens, vocab 50257)
+    composed from the C-ABI calls by the test harness (tests/gpt_model.py, unchecked here), launched call by
+    call from Python or, with --graph, recorded once into a CUDA graph and replayed.  One JSON line."""
+    import torch
+
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    import scalify_inputs as si
+    from checked_ops import Ops
+    from gpt_model import GPTConfig, ScaledGPT
+    torch.cuda.set_device(0)
+    cfg = GPTConfig()
+    ops = Ops(check=False)
+    model = ScaledGPT(cfg, ops, seed=6)
+    n = cfg.batch * cfg.seq
+    ids = torch.from_numpy(si.uniform_int(6, 901, (n,), cfg.vocab)).cuda()
+    tgt = torch.from_numpy(si.uniform_int(6, 902, (n,), cfg.vocab)).cuda()
+    for t in range(1, 1 + max(args.warmup, 1)):
+        model.step(ids, tgt, t=t)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    calls = ops.calls
+    if args.graph:
+        stream = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(stream):
+            with torch.cuda.graph(graph, stream=stream):
+                model.step(ids, tgt, t=10)
+        calls = ops.calls - calls
+        graph.replay()
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(args.steps):
+            graph.replay()
+        e1.record()
+    else:
+        e0.record()
+        for t in range(10, 10 + args.steps):
+            model.step(ids, tgt, t=t)
+        e1.record()
+        calls = (ops.calls - calls) // max(args.steps, 1)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / max(args.steps, 1)
+    print(json.dumps({"row": "config 5: GPT-2-small-shaped training step, all matmuls scaled FP8, FP16 scaled "
+                             "optimizer state", "launch": "CUDA graph replay" if args.graph else "call by call from Python",
+                      "ms_per_step": round(ms, 3), "tokens/s": round(n / ms * 1e3), "library_calls_per_step": calls}))
+
+
 def run_hbm_sweep(args):
     """The HBM-bound rows at other sizes: LayerNorm forward / backward + rescale at R in {8192, 131072} and
     d in {768, 1024, 4096}; stand-alone rescale and add at 2^23, 2^26 and 2^28 elements.  Each case is
@@ -403,7 +451,13 @@ def main():
                     help="skip the separately timed next-row variants f1, f2 (for ncu launch lists of the step)")
     ap.add_argument("--profile-row", default=None, choices=["matmul", "mx", "attention", "attention_bwd", "rescale", "add", "layernorm", "adam"],
                     help="run only this row on a reduced, still larger-than-L2 case (for ncu captures)")
+    ap.add_argument("--gpt-step", action="store_true",
+                    help="time the config-5 step (GPT-2-small shapes) instead; with --graph replayed from a CUDA graph")
+    ap.add_argument("--graph", action="store_true")
     args = ap.parse_args()
+    if args.gpt_step:
+        run_gpt_step(args)
+        return
     if args.impl == "reference":
         run_reference(args)
         return

@@ -421,6 +421,10 @@ int scalify_scaled_cross_entropy(const scalify_array* logits, int64_t n_classes,
  *   grads[i]: any dtype (E5M2 typical); m[i], v[i]: F16 or F32 (same);
  *   w[i]: F16, BF16 or F32.  All four have the same element count, are
  *   contiguous, and m, v, w (data and scale words) are updated in place.
+ *   Every m, v and w scale word of the whole list must be a word of its own
+ *   (the kernels read the old scales while the new ones are written) and none
+ *   of them a gradient's scale word; gradients may share one.  A repeated word
+ *   returns SCALIFY_ERR_ALIAS and enqueues nothing.
  *   step >= 1 is t.  Needs a workspace (SCALIFY_OP_ADAM, n_tensors).
  */
 int scalify_scaled_adam_step(int n_tensors, const scalify_array* grads, scalify_array* m, scalify_array* v,

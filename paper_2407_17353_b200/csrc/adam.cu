@@ -9,6 +9,8 @@
 //      kAdamChunk elements, finds the owning tensor by binary search in a prefix table passed
 //      by value, and moves 8 elements per thread access (8 B of FP8 gradient, 16 B of each
 //      16-bit state, 32 B of fp32 master weight).
+#include <algorithm>
+
 #include "scalify_common.cuh"
 #include "scalify_launch.h"
 
@@ -287,6 +289,24 @@ int launch_adam(int n_tensors, const scalify_array* grads, scalify_array* m, sca
 #undef SCALIFY_ADAM_LAUNCH
     SCALIFY_CUDA_TRY(cudaGetLastError());
   }
+  return SCALIFY_OK;
+}
+
+int check_adam_scale_words(int n_tensors, const scalify_array* grads, const scalify_array* m, const scalify_array* v,
+                           const scalify_array* w, const scalify_array* w_cast, const void** scratch) {
+  int k = 0;
+  for (int i = 0; i < n_tensors; ++i) {
+    scratch[k++] = m[i].scale;
+    scratch[k++] = v[i].scale;
+    scratch[k++] = w[i].scale;
+    if (w_cast) scratch[k++] = w_cast[i].scale;
+  }
+  std::sort(scratch, scratch + k);
+  for (int i = 1; i < k; ++i)
+    if (scratch[i] == scratch[i - 1]) return SCALIFY_ERR_ALIAS;
+  for (int i = 0; i < n_tensors; ++i)
+    if (grads[i].scale && std::binary_search(scratch, scratch + k, static_cast<const void*>(grads[i].scale)))
+      return SCALIFY_ERR_ALIAS;
   return SCALIFY_OK;
 }
 

@@ -76,8 +76,11 @@ extern "C" int scalify_scaled_adam_step_static(int n_tensors, const scalify_arra
       return SCALIFY_ERR_ALIAS;
     numel[i] = n;
   }
+  const void* words[kStaticAdamMaxTensors * 4];  // (on the stack: this call allocates nothing, on the host either)
+  int rc = check_adam_scale_words(n_tensors, grads, m, v, w, nullptr, words);
+  if (rc) return rc;
   void* scratch = nullptr;
-  int rc = static_scratch_ptr(&scratch);
+  rc = static_scratch_ptr(&scratch);
   if (rc) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // the array keeps whatever the previous call left: the status word has to start at zero

@@ -3,6 +3,8 @@
 #include <math.h>
 #include <string.h>
 
+#include <algorithm>
+
 #include "scalify_common.cuh"
 #include "scalify_launch.h"
 #include <new>
@@ -619,6 +621,12 @@ static int adam_step_impl(int n_tensors, const scalify_array* grads, scalify_arr
       }
     }
     numel[i] = n;
+  }
+  if (rc == SCALIFY_OK) {
+    const void** words = new (std::nothrow) const void*[size_t(n_tensors) * 4];
+    if (!words) rc = SCALIFY_ERR_VALUE;
+    else rc = check_adam_scale_words(n_tensors, grads, m, v, w, w_cast, words);
+    delete[] words;
   }
   if (rc == SCALIFY_OK)
     rc = launch_adam(n_tensors, grads, m, v, w, w_cast, numel, lr, beta1, beta2, eps, step, workspace,

@@ -45,6 +45,10 @@ int launch_layernorm_bwd(const void* G, int64_t g_ld, const void* X, int x_dt, i
                          const float* g_scale, const float* x_scale, const float* gamma_scale, float* dx_scale,
                          float* dgamma_scale, float* dbeta_scale, const float* stat_in, void* ws, cudaStream_t st);
 size_t adam_ws_bytes(int64_t n_tensors);
+// Every scale word the step WRITES (m, v, w, w_cast of every tensor) must be a different word, and none of them a
+// gradient's scale word: the kernels read and write them concurrently.  `scratch` holds 4 * n_tensors pointers.
+int check_adam_scale_words(int n_tensors, const scalify_array* grads, const scalify_array* m, const scalify_array* v,
+                           const scalify_array* w, const scalify_array* w_cast, const void** scratch);
 int launch_adam(int n_tensors, const scalify_array* grads, scalify_array* m, scalify_array* v, scalify_array* w,
                 const scalify_array* w_cast,
                 const int64_t* numel, float lr, float beta1, float beta2, float eps, int64_t step, void* ws,

@@ -4,16 +4,18 @@
 memory pool already holds the whole device, or they must avoid cudaMalloc's synchronisation);
 its scratch is a fixed array inside the library.  It runs the same kernels, so its results
 must be identical, bit for bit, to those of `scalify_scaled_adam_step` - on a first call and on
-a second call that finds the first call's leftovers in the shared array.  This file is
-collected last on purpose: a failure here stops a `-x` run only after every other test ran.
+a second call that finds the first call's leftovers in the shared array - and, like them, within
+one FP16 ulp of the oracle's step with exactly the oracle's scale words.  This file is collected
+last on purpose: a failure here stops a `-x` run only after every other test ran.
 """
 import numpy as np
 import pytest
 import torch
 
+import oracle as orc
 import paper_2407_17353_b200 as sc
 import scalify_inputs as si
-from helpers import to_dev, to_bits
+from helpers import to_dev, to_bits, ulp_diff
 
 pytestmark = pytest.mark.gpu
 
@@ -43,6 +45,9 @@ def test_static_adam_matches_workspace_adam_on_two_calls_in_a_row():
     ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_ADAM, len(sizes)))
     status = torch.full((1,), 77, dtype=torch.int32, device="cuda")
     for step in (1000, 1001):  # the second call meets the scratch contents of the first
+        before = [(to_bits(g.data, si.E5M2), g.scale_value(), to_bits(m.data, si.F16), m.scale_value(),
+                   to_bits(v.data, si.F16), v.scale_value(), to_bits(w.data, si.F16), w.scale_value())
+                  for g, m, v, w in zip(*new.keep)]
         sc.scalify_scaled_adam_step(ref, ws, step=step, **hyper)
         sc.scalify_scaled_adam_step_static(new, step=step, status_out=status, **hyper)
         torch.cuda.synchronize()
@@ -50,6 +55,14 @@ def test_static_adam_matches_workspace_adam_on_two_calls_in_a_row():
         for (a, sa), (b, sb) in zip(snapshot(ref), snapshot(new)):
             assert sa == sb
             assert np.array_equal(a, b)
+        # ... and against the oracle's step on the same inputs
+        for (g, gs, m0, ms0, v0, vs0, w0, ws0), m, v, w in zip(before, new.keep[1], new.keep[2], new.keep[3]):
+            mo, vo, wo, ms, vs, wsn = orc.adam_step(g, orc.E5M2, gs, m0, v0, orc.F16, ms0, vs0, w0, orc.F16, ws0,
+                                                    hyper["lr"], hyper["beta1"], hyper["beta2"], hyper["eps"], step)
+            assert (m.scale_value(), v.scale_value(), w.scale_value()) == (ms, vs, wsn)
+            assert ulp_diff(to_bits(m.data, si.F16), mo, orc.F16).max() <= 1
+            assert ulp_diff(to_bits(v.data, si.F16), vo, orc.F16).max() <= 1
+            assert ulp_diff(to_bits(w.data, si.F16), wo, orc.F16).max() <= 1
 
 
 def test_static_adam_reports_bad_scale_and_then_starts_clean():
@@ -61,6 +74,18 @@ def test_static_adam_reports_bad_scale_and_then_starts_clean():
     good = make_state([256], 93)
     sc.scalify_scaled_adam_step_static(good, lr=1e-3, beta1=0.9, beta2=0.99, eps=1e-8, step=1, status_out=status)
     assert int(status.item()) == 0  # the status word of the previous call was cleared
+
+
+def test_a_scale_word_shared_by_two_tensors_is_rejected_by_both_calls():
+    two = make_state([64, 64], 95)
+    two.keep[2][1].scale = two.keep[2][0].scale      # both v tensors point at one scale word
+    shared = sc.AdamTensors(*two.keep)
+    ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_ADAM, 2))
+    for call in (lambda: sc.scalify_scaled_adam_step(shared, ws, lr=1e-3, beta1=0.9, beta2=0.99, eps=1e-8, step=1),
+                 lambda: sc.scalify_scaled_adam_step_static(shared, lr=1e-3, beta1=0.9, beta2=0.99, eps=1e-8, step=1)):
+        with pytest.raises(sc.ScalifyError) as e:
+            call()
+        assert e.value.code == -8      # SCALIFY_ERR_ALIAS: nothing was enqueued
 
 
 def test_static_adam_rejects_more_tensors_than_its_scratch_holds():
