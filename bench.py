@@ -4,7 +4,9 @@
 One step = one pass over every row of the hot path on synthetic, seeded inputs
 shaped like GPT-style training tensors:
   1. scaled FP8 matmul 8192^3 (E4M3 x E4M3, fp32 accumulate) with fused AMAX, BF16 intermediate
-  2. dynamic rescale pass 2: BF16 -> E4M3 with power-of-two rebalance          (headline = 1 + 2)
+  2. dynamic rescale pass 2: BF16 -> E4M3 with power-of-two rebalance
+  H. the headline: 1 + 2 as ONE call, scalify_scaled_matmul(A, B, Y, AMAX, Yq): BF16 intermediate, fused AMAX and
+     the E4M3 output written by the GEMM with the predicted power of two, confirmed (or rebuilt) by a check launch
   3. stand-alone dynamic rescale (statistic pass + cast pass) of a BF16 tensor
   4. scaled add of two BF16 tensors
   5. scaled LayerNorm forward  [131072, 1024] BF16
@@ -13,7 +15,7 @@ shaped like GPT-style training tensors:
 Outside the step (own timed loop) the next-row variant is reported too: the same GEMM with delayed
 rescaling - one kernel, E4M3 written directly with the previous step's statistic while this step's AMAX
 is gathered, no BF16 intermediate, no pass 2.
-`value` is the headline metric: 2*M*N*K / (time of rows 1+2), measured with CUDA events inside
+`value` is the headline metric: 2*M*N*K / (time of call H), measured with CUDA events inside
 the step.  Rows 3-7 are reported as GB/s of algorithmic bytes in `rows`.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
@@ -39,11 +41,23 @@ LN_R, LN_D = 131072, 1024
 ADAM_N = 125_000_000
 ADD_SHAPE = (8192, 8192)
 ORACLE_SAMPLE_ROWS = 1024     # cpu_baseline leg: one sample (10-30 s of CPU work)
-REFERENCE_ROWS_PER_STEP = 32  # --impl reference: rows per timed step
+# --impl reference: the same 1024-row sample per timed step while the whole run stays within a few minutes
+# (about 7 s per sample on 16 cores), fewer rows per step for longer runs
+REFERENCE_ROWS_BUDGET = 24 * 1024
 
-# DRAM traffic of one 8192^3 GEMM launch (dram__bytes_read.sum + dram__bytes_write.sum), from the ncu
-# capture summarised in profiles/ (algorithmic bytes: 268 MB).
-GEMM_DRAM_TRAFFIC_BYTES = 358_119_424  # profiles/matmul_8192_e4m3_two_cta_ncu.md: 240.0 MB read + 118.1 MB written
+def gemm_dram_traffic():
+    """DRAM bytes of one 8192^3 GEMM launch (dram__bytes_read.sum + dram__bytes_write.sum of an ncu capture) from
+    the small record kept beside the profile summaries, or None when the kernel's source has changed since the
+    capture was taken (the record carries a hash of the source files)."""
+    import hashlib
+    rec = os.path.join(ROOT, "profiles", "matmul_8192_dram_traffic.json")
+    if not os.path.exists(rec):
+        return None
+    d = json.load(open(rec))
+    h = hashlib.sha256()
+    for f in d.get("sources", []):
+        h.update(open(os.path.join(ROOT, f), "rb").read())
+    return int(d["dram_bytes_per_launch"]) if h.hexdigest() == d.get("sources_sha256") else None
 
 
 def load_peaks():
@@ -145,7 +159,7 @@ def run_reference(args):
     if rank != 0:
         return
     import oracle as orc
-    rows = REFERENCE_ROWS_PER_STEP
+    rows = max(32, min(ORACLE_SAMPLE_ROWS, REFERENCE_ROWS_BUDGET // max(args.steps + min(args.warmup, 1), 1)))
     for _ in range(min(args.warmup, 1)):
         oracle_sample(rows)
     vals, times = [], []
@@ -442,9 +456,6 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (for ncu launch lists)")
-    ap.add_argument("--speculative", action="store_true",
-                    help="run rows a1-a3 of the step as ONE call with a predicted statistic "
-                         "(scalify_scaled_matmul_speculative; same outputs bit for bit)")
     ap.add_argument("--hbm-sweep", action="store_true",
                     help="print one JSON line per size of the HBM-bound rows (LayerNorm, rescale, add) instead of the step")
     ap.add_argument("--no-next", action="store_true",
@@ -544,38 +555,39 @@ def main():
     Yd = sc.ScaledTensor.empty((N_GEMM, N_GEMM), torch.float8_e4m3fn, dev)
     stat_state = torch.full((1,), 4.0, dtype=torch.float32, device=dev)
 
-    spec_hint = torch.zeros(1, dtype=torch.float32, device=dev)
-    n_ev = 8
-    # kernels of this library per step: matmul + pass 2, one-launch rescale, add, LayerNorm fwd,
-    # LayerNorm bwd + finalize + pass 2, Adam scales + update
-    launches_per_step = 2 + 1 + 1 + 1 + 3 + 2
+    Yq2 = sc.ScaledTensor.empty((N_GEMM, N_GEMM), torch.float8_e4m3fn, dev)
+    ws_head = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_MATMUL, N_GEMM, N_GEMM), dev)   # keeps the prediction
+    n_ev = 9
+    # kernels of this library per step: matmul + pass 2, headline call (matmul + check launch), one-launch rescale,
+    # add, LayerNorm fwd, LayerNorm bwd + finalize + pass 2, Adam scales + update
+    launches_per_step = 2 + 2 + 1 + 1 + 1 + 3 + 2
 
-    def step(t, evs=None, speculative=False):
+    def step(t, evs=None, fp8_only=False):
         def mark(i):
             if evs is not None:
                 evs[i].record()
+        # Each of the two GEMMs follows memory-bound rows: a GEMM that follows another one finds the clocks the
+        # power limit left behind (measured: the same call is 4 % slower there).
         mark(0)
-        if speculative:
-            # GEMM writes BF16 and E4M3 (predicted factor), then the check launch: segment a1+a2 holds both,
-            # segment a3 is empty
-            sc.scalify_scaled_matmul_speculative(A, Bt, Y, Yq, spec_hint, ws_mm, transB=True)
-            mark(1)
-        else:
-            sc.scalify_scaled_matmul(A, Bt, Y, ws_mm, transB=True, stat=sc.STAT_AMAX, Yq=None)
-            mark(1)
-            sc.scalify_rescale(Y, Yq, stat=sc.STAT_AMAX, stat_in=ws_mm.statistic())
-        mark(2)
+        # the headline: GEMM + fused AMAX + rescale to E4M3 as ONE call of the library's main entry point
+        sc.scalify_scaled_matmul(A, Bt, None if fp8_only else Y, ws_head, transB=True, stat=sc.STAT_AMAX, Yq=Yq2)
+        mark(1)
         sc.scalify_rescale(P, Rq, stat=sc.STAT_AMAX, ws=ws_rs)
-        mark(3)
+        mark(2)
         sc.scalify_scaled_add(P, Q, S)
-        mark(4)
+        mark(3)
         sc.scalify_scaled_layernorm(X, gamma, beta, LY, eps=1e-5, mean=mean, rinv=rinv)
+        mark(4)
+        # rows a1+a2 and a3 as two calls, so that the dominant kernel has a time of its own
+        sc.scalify_scaled_matmul(A, Bt, Y, ws_mm, transB=True, stat=sc.STAT_AMAX, Yq=None)
         mark(5)
+        sc.scalify_rescale(Y, Yq, stat=sc.STAT_AMAX, stat_in=ws_mm.statistic())
+        mark(6)
         sc.scalify_scaled_layernorm_bwd(G, X, gamma, mean, rinv, dX, ws_ln, eps=1e-5, stat_dx=sc.STAT_L2, dXq=dXq,
                                         dgamma=dg, dbeta=db)
-        mark(6)
-        sc.scalify_scaled_adam_step(adam, ws_ad, lr=3e-4, beta1=0.9, beta2=0.999, eps=1e-8, step=1000 + t)
         mark(7)
+        sc.scalify_scaled_adam_step(adam, ws_ad, lr=3e-4, beta1=0.9, beta2=0.999, eps=1e-8, step=1000 + t)
+        mark(8)
 
     def barrier():
         if dist is not None:
@@ -585,9 +597,9 @@ def main():
     # the sampler thread starts before the warm-up, so that NVML's start-up is over when the timed region begins
     sampler = ClockSampler(local_rank) if rank == 0 else None
     for t in range(W):
-        step(t, None, args.speculative)
+        step(t, None)
     barrier()
-    for w in (ws_mm, ws_rs, ws_ln, ws_ad):
+    for w in (ws_mm, ws_head, ws_rs, ws_ln, ws_ad):
         st = w.check_status()
         if st != 0:
             raise SystemExit(f"device status {st} after warm-up")
@@ -600,23 +612,29 @@ def main():
     t_end = torch.cuda.Event(enable_timing=True)
     t_start.record()
     for t in range(K):
-        step(W + t, evs[t], args.speculative)
+        step(W + t, evs[t])
     t_end.record()
     barrier()
     clocks = sampler.stop() if sampler is not None else None
     total_ms = t_start.elapsed_time(t_end)
     seg = np.array([[evs[t][i].elapsed_time(evs[t][i + 1]) for i in range(n_ev - 1)] for t in range(K)])
     seg_ms = seg.mean(axis=0)
-    for w in (ws_mm, ws_rs, ws_ln, ws_ad):
+    for w in (ws_mm, ws_head, ws_rs, ws_ln, ws_ad):
         st = w.check_status()
         if st & sc.DEV_TIMEOUT:
             raise SystemExit(f"device status {st} in the timed region")
 
-    # The same step once more with rows a1-a3 as ONE speculative call (same outputs bit for bit): its first
-    # segment is the whole GEMM + rescale.  Timed in the step, like the headline, because a loop of GEMMs alone
-    # runs at other clocks.
-    spec_ms = float("nan")
-    if not args.no_next and not args.speculative:
+    # The headline's outputs must be those of the two-call form, bit for bit
+    torch.cuda.synchronize()
+    if not (torch.equal(Yq.data.view(torch.uint8), Yq2.data.view(torch.uint8)) and
+            float(Yq.scale.item()) == float(Yq2.scale.item())):
+        raise SystemExit("the one-call headline and the two-call form disagree")
+
+    # The same step once more with the headline call in its FP8-only form (Y = NULL: the BF16 intermediate is not
+    # stored; same Yq, scale and statistic bit for bit).  Timed in the step, like the headline, because a loop of
+    # GEMMs alone runs at other clocks.
+    fp8_only_ms = float("nan")
+    if not args.no_next:
         for t in range(3):
             step(W + K + t, None, True)
         barrier()
@@ -624,10 +642,12 @@ def main():
         for t in range(K):
             step(W + K + 3 + t, evs2[t], True)
         barrier()
-        spec_ms = float(np.mean([evs2[t][0].elapsed_time(evs2[t][2]) for t in range(K)]))
+        fp8_only_ms = float(np.mean([evs2[t][0].elapsed_time(evs2[t][1]) for t in range(K)]))
+        if not torch.equal(Yq.data.view(torch.uint8), Yq2.data.view(torch.uint8)):
+            raise SystemExit("the FP8-only headline form and the two-call form disagree")
 
     flops = 2.0 * N_GEMM ** 3
-    head_ms = float(seg_ms[0] + seg_ms[1])
+    head_ms = float(seg_ms[0])
     value_local = flops / (head_ms * 1e-3) / 1e12
     ms_per_step = total_ms / K
 
@@ -754,6 +774,45 @@ def main():
         att_bwd_ms = a0.elapsed_time(a1) / a_iters
         del Qa, Ka, Va, Oa, Pa, dOa, dSa, dQa, dKa, dVa
 
+    # ------------------------------------------------------------------ configs[1]: the other sizes and formats
+    # M = N = K in {1024, 4096, 8192}, forward E4M3 x E4M3 and gradient E5M2 x E4M3, each as the one-call form
+    # (BF16 intermediate + fused AMAX + E4M3 output), back to back over a rotation of buffer sets that together
+    # exceed twice the L2 (one workspace per set, so that every set keeps its own prediction)
+    sweep_rows = []
+    if not args.no_next:
+        l2 = 126 * 2 ** 20
+        for n in (1024, 4096, N_GEMM):
+            for kind, a_dt, a_s in (("forward E4M3 x E4M3", torch.float8_e4m3fn, 1.0),
+                                    ("gradient E5M2 x E4M3", torch.float8_e5m2, 2.0 ** -10)):
+                per_set = n * n * 5
+                sets = max(2, min(64, -(-2 * l2 // per_set)))
+                calls = []
+                for k in range(sets):
+                    As = sc.ScaledTensor.make(rnd((n, n), a_dt, 50 + 2 * k), a_s)
+                    Bs = sc.ScaledTensor.make(rnd((n, n), torch.float8_e4m3fn, 51 + 2 * k), 2.0 ** -6)
+                    Ys = sc.ScaledTensor.empty((n, n), torch.bfloat16, dev)
+                    Yqs_ = sc.ScaledTensor.empty((n, n), torch.float8_e4m3fn, dev)
+                    wss = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_MATMUL, n, n), dev)
+                    calls.append(lambda As=As, Bs=Bs, Ys=Ys, Yqs_=Yqs_, wss=wss: sc.scalify_scaled_matmul(
+                        As, Bs, Ys, wss, transB=True, stat=sc.STAT_AMAX, Yq=Yqs_))
+                for _ in range(2):
+                    for f in calls:
+                        f()
+                barrier()
+                g_iters = max(len(calls), min(K, 20)) if n == N_GEMM else 4 * len(calls)
+                g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                g0.record()
+                for i in range(g_iters):
+                    calls[i % len(calls)]()
+                g1.record()
+                barrier()
+                g_ms = g0.elapsed_time(g1) / g_iters
+                sweep_rows.append({"row": f"configs[1] {kind}, M=N=K={n}: GEMM + fused AMAX + rescale to E4M3, one call "
+                                          f"(own loop, back to back over {sets} buffer sets)",
+                                   "ms": round(g_ms, 4), "TFLOP/s": round(2.0 * n ** 3 / (g_ms * 1e-3) / 1e12, 1)})
+                del calls
+                torch.cuda.empty_cache()
+
     # ------------------------------------------------------------------ end to end through host buffers
     hY = torch.empty((N_GEMM, N_GEMM), dtype=torch.int8).pin_memory()
     hscale = torch.empty(1, dtype=torch.float32).pin_memory()
@@ -836,23 +895,28 @@ def main():
         return {"row": name, "ms": round(float(ms), 4), "GB/s": round(gbs, 1), "frac_of_hbm_peak": round(gbs / hbm, 3)}
 
     rows = [
-        {"row": "a1+a2 scaled FP8 matmul 8192^3 + fused AMAX", "ms": round(float(seg_ms[0]), 4),
-         "TFLOP/s": round(flops / (seg_ms[0] * 1e-3) / 1e12, 1)},
-        row("a3 rescale pass 2 BF16->E4M3 (3 B/elem)", seg_ms[1], 3 * N_GEMM * N_GEMM),
-        row("a3'+a3 stand-alone dynamic rescale BF16->E4M3 (5 B/elem)", seg_ms[2], 5 * n_add),
-        row("a4 scaled add BF16 (6 B/elem)", seg_ms[3], 6 * n_add),
-        row("a5 scaled LayerNorm fwd BF16->BF16 (4 B/elem + 8 B/row)", seg_ms[4], 4 * n_ln + 8 * LN_R),
-        row("a6 scaled LayerNorm bwd + L2 rescale to E5M2 (9 B/elem + 8 B/row)", seg_ms[5], 9 * n_ln + 8 * LN_R),
-        row("a7 scaled Adam, E5M2 grads, FP16 m/v/w (13 B/param)", seg_ms[6], 13 * ADAM_N),
+        {"row": "a1+a2 scaled FP8 matmul 8192^3 + fused AMAX", "ms": round(float(seg_ms[4]), 4),
+         "TFLOP/s": round(flops / (seg_ms[4] * 1e-3) / 1e12, 1)},
+        row("a3 rescale pass 2 BF16->E4M3 (3 B/elem)", seg_ms[5], 3 * N_GEMM * N_GEMM),
+        {"row": "a1+a2+a3 as two calls (GEMM + AMAX, then pass 2)", "ms": round(float(seg_ms[4] + seg_ms[5]), 4),
+         "TFLOP/s": round(flops / ((seg_ms[4] + seg_ms[5]) * 1e-3) / 1e12, 1)},
+        {"row": "HEADLINE a1+a2+a3 as one call: scalify_scaled_matmul(A, B, Y, AMAX, Yq) - BF16 intermediate, fused "
+                "AMAX, E4M3 written by the GEMM with the predicted power of two, check launch (bit-identical to the "
+                "two calls)", "ms": round(float(seg_ms[0]), 4), "TFLOP/s": round(flops / (seg_ms[0] * 1e-3) / 1e12, 1)},
+        row("a3'+a3 stand-alone dynamic rescale BF16->E4M3 (5 B/elem)", seg_ms[1], 5 * n_add),
+        row("a4 scaled add BF16 (6 B/elem)", seg_ms[2], 6 * n_add),
+        row("a5 scaled LayerNorm fwd BF16->BF16 (4 B/elem + 8 B/row)", seg_ms[3], 4 * n_ln + 8 * LN_R),
+        row("a6 scaled LayerNorm bwd + L2 rescale to E5M2 (9 B/elem + 8 B/row)", seg_ms[6], 9 * n_ln + 8 * LN_R),
+        row("a7 scaled Adam, E5M2 grads, FP16 m/v/w (13 B/param)", seg_ms[7], 13 * ADAM_N),
         {"row": "f1 (next, timed outside the step, back to back) delayed-rescale GEMM 8192^3: E4M3 out in one "
                 "kernel, no BF16 intermediate, no pass 2", "ms": round(float(delayed_ms), 4),
          "TFLOP/s": round(flops / (delayed_ms * 1e-3) / 1e12, 1)},
         row("f1 (next, timed outside the step, back to back) LayerNorm bwd with delayed L2 rescale: E5M2 gradient "
             "in one pass, no BF16 intermediate, no pass 2 (5 B/elem + 8 B/row)", ln_delayed_ms, 5 * n_ln + 8 * LN_R),
-        {"row": "f1b (next, timed in a second pass of the same step) GEMM 8192^3 + EXACT dynamic AMAX rescale to E4M3 "
-                "with a predicted statistic: the GEMM writes BF16 and E4M3, a check launch confirms the prediction "
-                "(bit-identical to a1+a2+a3)",
-         "ms": round(float(spec_ms), 4), "TFLOP/s": round(flops / (spec_ms * 1e-3) / 1e12, 1)},
+        {"row": "f1b (next, timed in a second pass of the same step) the headline call with Y = NULL: only the E4M3 "
+                "output is stored (values still rounded through BF16, AMAX of the BF16 values; a repair launch of the "
+                "same kernel returns at once when the prediction held); Yq, scale and statistic bit-identical",
+         "ms": round(float(fp8_only_ms), 4), "TFLOP/s": round(flops / (fp8_only_ms * 1e-3) / 1e12, 1)},
         row("f2 (next, timed outside the step, back to back) scaled Adam that also writes the E4M3 compute copy "
             "of the weight (14 B/param)", adam_cast_ms, 14 * ADAM_N),
         row("f3 (next, own loop) block-scale quantisation of two 8192^2 BF16 operands to E4M3 + E8M0 per 32 "
@@ -869,24 +933,35 @@ def main():
          "ms": round(float(att_bwd_ms), 4),
          "TFLOP/s": round(4.0 * ATT_H * ATT_T * ATT_T * ATT_HD / (att_bwd_ms * 1e-3) / 1e12, 1),
          "note": "flop counted for the causal half of dO V^T, dS K, dS^T Q and P^T dO"},
-    ]
-    fp8_peak = 2.0 * peaks["bf16_sustained"]
-    gemm_tflops = flops / (float(seg_ms[0]) * 1e-3) / 1e12
+    ] + sweep_rows
+    # Which of the two measured bf16 rates is the denominator: the sustained one holds for a GEMM that runs for
+    # seconds under the power cap; a timed region under a second, or a GEMM that is less than half of the step's
+    # duty cycle, runs at burst clocks.
+    gemm_share = float(seg_ms[0] + seg_ms[4]) / float(np.sum(seg_ms))
+    burst = total_ms < 1000.0 or gemm_share < 0.5
+    gemm_tflops = flops / (float(seg_ms[4]) * 1e-3) / 1e12
+    peak_burst, peak_sust = 2.0 * peaks["bf16_burst"], 2.0 * peaks["bf16_sustained"]
+    fp8_peak = peak_burst if burst else peak_sust
     roofline = {
         "bound": "tensor", "kernel": "scaled_matmul_kernel<BF16> (tcgen05 kind::f8f6f4)",
         "achieved": round(gemm_tflops, 1), "peak": round(fp8_peak, 1), "unit": "TFLOP/s",
         "frac": round(gemm_tflops / fp8_peak, 4),
-        "peak_source": f"{peaks['source']}: 2 x sustained bf16 cuBLAS ({peaks['bf16_sustained']} TFLOP/s), "
-                       f"fp8:bf16 nominal ratio 2; burst would be {2 * peaks['bf16_burst']:.0f}; nominal dense fp8 4500",
+        "frac_vs_burst": round(gemm_tflops / peak_burst, 4), "frac_vs_sustained": round(gemm_tflops / peak_sust, 4),
+        "peak_source": f"{peaks['source']}: 2 x {'burst' if burst else 'sustained'} bf16 cuBLAS "
+                       f"({peaks['bf16_burst'] if burst else peaks['bf16_sustained']} TFLOP/s), fp8:bf16 nominal ratio 2 "
+                       f"(timed region {total_ms:.0f} ms, GEMMs {100 * gemm_share:.0f} % of it); nominal dense fp8 4500",
         "frac_of_nominal_4500": round(gemm_tflops / 4500.0, 4),
-        "traffic": GEMM_DRAM_TRAFFIC_BYTES,
+        "headline_frac_of_peak": round(value_local / fp8_peak, 4),
+        "headline_frac_of_nominal_4500": round(value_local / 4500.0, 4),
+        "traffic": gemm_dram_traffic(),
     }
     line = {
         "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "fp8 (e4m3 x e4m3, fp32 accumulate)", "data": "synthetic",
         "config": {"workload": f"configs[1]: scaled GEMM M=N=K={N_GEMM} forward E4M3xE4M3, BF16 intermediate + fused "
-                               "AMAX, pass 2 to E4M3; the step also runs rows a3'-a7 (see rows)",
+                               "AMAX + rescale to E4M3 in one call; the step also runs the two-call form and rows "
+                               "a3'-a7, and the other sizes and the gradient formats of configs[1] follow in rows",
                    "l2": "inputs larger than L2: every step streams > 5 GB, so no operand survives in L2 between "
                          "iterations", "replicas": world},
         "headline_ms": round(head_ms_max, 4),

@@ -151,6 +151,25 @@ int scalify_version(void);
  *       rescale of Y: r = statistic rounded down to a power of two,
  *       Yq_d = cast(Y_d / r), Yq_s = Y_s * r.  Any dtype; same shape as Y.
  *
+ * Predicted rescale (Section 3.3: statistic and rebalancing are separate
+ * primitives).  With stat = AMAX, a BF16/F16 Y, an FP8 Yq of its own and rows
+ * of a multiple of 16 elements, the GEMM's epilogue already writes Yq with
+ * the power of two of the statistic this workspace saw last (fp32 word at
+ * byte offset 56 of the workspace), and the launch that follows rebuilds Yq
+ * from Y only if this call's statistic has another power of two.  Y, Yq, both
+ * scale words and the statistic word are the same bits either way and for any
+ * content of that word; the call leaves its own statistic there.  Keep one
+ * workspace per matmul of a training step for the prediction to hold.
+ *
+ * Y == NULL (FP8 output only): allowed with stat = AMAX and an FP8, contiguous
+ * Yq with its own scale word and rows of a multiple of 16 elements.  The
+ * values are still rounded to BF16 first and the statistic is still that of
+ * the BF16 values, so Yq, Yq_s and the statistic word equal those of the call
+ * with a BF16 Y bit for bit, but the intermediate is not stored: the epilogue
+ * writes Yq with the predicted power of two, and a second launch of the same
+ * kernel, whose thread blocks return at once when the prediction held,
+ * computes the product again otherwise.  Never splits the contraction.
+ *
  * Accumulation is fp32 on the tensor cores (tcgen05, kind::f8f6f4).  Row
  * strides must be multiples of 16 bytes.  Errors: see scalify_error.
   *

@@ -202,6 +202,11 @@ class Workspace:
         """The fp32 statistic word (byte offset 16) as a 1-element tensor view."""
         return self.buf[16:20].view(torch.float32)
 
+    def prediction(self) -> torch.Tensor:
+        """The AMAX statistic of the last matmul + FP8 rescale on this workspace (byte offset 56), which the next
+        such call uses as its prediction; a 1-element tensor view."""
+        return self.buf[56:60].view(torch.float32)
+
     def check_status(self, stream=None) -> int:
         return scalify_check_status(self, stream)
 
@@ -217,8 +222,9 @@ def scalify_check_status(ws: Workspace, stream=None) -> int:
     return rc
 
 
-def scalify_scaled_matmul(A: ScaledTensor, B: ScaledTensor, Y: ScaledTensor, ws: Workspace, *, transA=False,
+def scalify_scaled_matmul(A: ScaledTensor, B: ScaledTensor, Y: Optional[ScaledTensor], ws: Workspace, *, transA=False,
                           transB=False, stat: int = STAT_NONE, Yq: Optional[ScaledTensor] = None, stream=None) -> None:
+    """Y may be None with stat=STAT_AMAX and an FP8 Yq: only the rescaled output is stored."""
     a, b, y, yq = _desc(A), _desc(B), _desc(Y), _desc(Yq)
     _check(lib().scalify_scaled_matmul(_ref(a), int(transA), _ref(b), int(transB), _ref(y), stat, _ref(yq),
                                        ws.ptr, ws.nbytes, _stream(stream)), "scalify_scaled_matmul")

@@ -257,6 +257,8 @@ __global__ void __launch_bounds__(kThreads) rebalance_check_kernel(const void* _
                                                                    const float* stat, const float* r_pred,
                                                                    float* hint_out, uint32_t* status) {
   asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
+  // launched as a programmatic dependent of the GEMM: its blocks are resident when the GEMM ends and start here
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   constexpr int VEC = VecElems<IN, OUT>::v;
   constexpr int IB = VEC * ElemBytes<IN>::v, OB = VEC * ElemBytes<OUT>::v;
   const float xs = load_scale(x_scale);
@@ -311,8 +313,18 @@ int launch_rebalance_check(const void* x, int in_dt, void* y, int out_dt, int64_
                            uint32_t* status, cudaStream_t st) {
   const int64_t n_vec = n / (16 / 2);
   const int grid = grid_for(n_vec, 8);  // small grid: in the expected case every block returns at once
-#define SCALIFY_RBC(IN, OUT) \
-  rebalance_check_kernel<IN, OUT><<<grid, kThreads, 0, st>>>(x, y, n, x_scale, y_scale, stat, r_pred, hint_out, status)
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cfg.gridDim = dim3(unsigned(grid));
+  cfg.blockDim = dim3(kThreads);
+  cfg.stream = st;
+#define SCALIFY_RBC(IN, OUT)                                                                                     \
+  SCALIFY_CUDA_TRY(cudaLaunchKernelEx(&cfg, rebalance_check_kernel<IN, OUT>, x, y, n, x_scale, y_scale, stat, r_pred, \
+                                      hint_out, status))
   if (in_dt == SCALIFY_BF16) {
     if (out_dt == SCALIFY_E4M3) SCALIFY_RBC(SCALIFY_BF16, SCALIFY_E4M3); else SCALIFY_RBC(SCALIFY_BF16, SCALIFY_E5M2);
   } else {

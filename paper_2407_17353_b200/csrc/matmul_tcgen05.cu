@@ -95,6 +95,14 @@ struct GemmParams {
   const float* stat_hint;
   int q_dt;          // SCALIFY_E4M3 or SCALIFY_E5M2
   float* r_pred_out; // the r_pred this launch used (read by the check kernel)
+  // FP8-only form (NOY kernels: no 16-bit intermediate is stored).  The CTA that draws the last ticket also
+  // publishes what the check launch publishes otherwise: the FP8 output's scale word and the prediction for the
+  // next call.  redo != 0 marks the repair launch that follows every such GEMM: its CTAs return at once when
+  // the power of two of the statistic equals the predicted one, and otherwise compute the product again with
+  // the statistic itself as the "prediction".
+  float* yq_scale;
+  float* hint_out;
+  int redo;
   // BIAS kernels: Y = A B + bias by the add rule, rounded once: Y_s = max(A_s B_s kf(K), bias_s)
   const void* bias;  // [N], F16 / BF16 / F32
   int bias_dt;
@@ -120,14 +128,24 @@ __device__ __forceinline__ void tile_coords(const GemmParams& p, int tile, int& 
 
 // map_sfa is the exponent map of A in the block-scaled form and the map of the speculative FP8 output in the
 // SPEC form (the two never occur together).
-template <int OUT, int NCTA, bool MX, bool SPEC = false, bool BIAS = false>
+template <int OUT, int NCTA, bool MX, bool SPEC = false, bool BIAS = false, bool NOY = false>
 __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_y,
                                           const CUtensorMap& map_sfa, const CUtensorMap& map_sfb, const GemmParams& p) {
   static_assert(!SPEC || (!MX && ElemBytes<OUT>::v == 2), "speculative FP8 output: per-tensor kernel, 16-bit Y");
   static_assert(!BIAS || (!MX && !SPEC), "bias: per-tensor kernel only");
+  static_assert(!NOY || SPEC, "the FP8-only form is a speculative form");
   using C = GemmCfg<NCTA, MX>;
   constexpr int kStages = C::kStages;
   constexpr int kAcc = C::kAcc;
+  if constexpr (NOY) {
+    if (p.redo) {
+      // repair launch: the GEMM before it has finished (and so has everything it wrote) once this returns
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      bool nf0;
+      const float r_true = rescale_factor(*reinterpret_cast<const volatile float*>(p.stat_word), &nf0);
+      if (r_true == *reinterpret_cast<const volatile float*>(p.r_pred_out)) return;  // the same words for every thread
+    }
+  }
   asm volatile("griddepcontrol.launch_dependents;");  // a dependent grid may set up while this one runs
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -182,7 +200,7 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
       if (p.y_scale) *p.y_scale = ys;
       if constexpr (SPEC) {
         bool nf2;
-        *p.r_pred_out = rescale_factor(__ldg(p.stat_hint), &nf2);
+        if (!(NOY && p.redo)) *p.r_pred_out = rescale_factor(*reinterpret_cast<const volatile float*>(p.stat_hint), &nf2);
       }
       if (nf && p.status) atomicOr(p.status, static_cast<uint32_t>(SCALIFY_DEV_NONFINITE_STAT));
     }
@@ -391,9 +409,11 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
       constexpr int CPR = 32 * OSZ / 16;              // 16-byte pieces per row: 2 (FP8), 4 (16-bit), 8 (F32)
       constexpr int kTileBytes = 32 * 32 * OSZ;
       // staging tiles per warp: 4, 4 or 2; with the speculative output 2 of Y (4 KB) and 2 FP8 tiles behind them
-      constexpr int NBUF = SPEC ? 2 : (C::kEpiWarpBytes / kTileBytes > 4 ? 4 : C::kEpiWarpBytes / kTileBytes);
+      // (the FP8-only form stages no 16-bit tile and uses four FP8 tiles)
+      constexpr int NBUF = NOY ? 4 : SPEC ? 2 : (C::kEpiWarpBytes / kTileBytes > 4 ? 4 : C::kEpiWarpBytes / kTileBytes);
       float inv_r_pred = 1.0f;
-      if constexpr (SPEC) { bool nf2; inv_r_pred = 1.0f / rescale_factor(__ldg(p.stat_hint), &nf2); }
+      // (a plain load: in the FP8-only form the word is rewritten at the end of this very kernel)
+      if constexpr (SPEC) { bool nf2; inv_r_pred = 1.0f / rescale_factor(*reinterpret_cast<const volatile float*>(p.stat_hint), &nf2); }
       auto convert = [&](const uint32_t* acc_regs, uint32_t* o, int c) {
         float v[32];
         if constexpr (BIAS) {
@@ -435,11 +455,13 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
       // the tile to a TMA store, which writes whole row segments and clips rows >= M and columns >= N.
       // (stage_chunk fills the tile; issue_chunk hands it to TMA)
       auto stage_chunk = [&](const uint32_t* o, int c) {
-        uint8_t* tile_b = epi_mem + (warp - 2) * C::kEpiWarpBytes + (c % NBUF) * kTileBytes;
-        uint4* tile = reinterpret_cast<uint4*>(tile_b);
+        if constexpr (!NOY) {
+          uint8_t* tile_b = epi_mem + (warp - 2) * C::kEpiWarpBytes + (c % NBUF) * kTileBytes;
+          uint4* tile = reinterpret_cast<uint4*>(tile_b);
 #pragma unroll
-        for (int j = 0; j < CPR; ++j)
-          tile[lane * CPR + (j ^ ((lane / (8 / CPR)) % CPR))] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+          for (int j = 0; j < CPR; ++j)
+            tile[lane * CPR + (j ^ ((lane / (8 / CPR)) % CPR))] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+        }
         if constexpr (SPEC) {
           uint8_t* tile_q = epi_mem + (warp - 2) * C::kEpiWarpBytes + 4096 + (c % NBUF) * 1024;
           uint32_t oq[8];
@@ -452,8 +474,10 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
       auto issue_chunk = [&](int c) {  // lane 0, after fence_async_smem + __syncwarp
         const int col0 = n0 + (c_first + c) * 32;
         const int row0 = mt * C::kTileM + static_cast<int>(rank) * kBM + q * 32;
-        uint8_t* tile_b = epi_mem + (warp - 2) * C::kEpiWarpBytes + (c % NBUF) * kTileBytes;
-        tma_store_3d(&map_y, smem_u32(tile_b), col0, row0, b);
+        if constexpr (!NOY) {
+          uint8_t* tile_b = epi_mem + (warp - 2) * C::kEpiWarpBytes + (c % NBUF) * kTileBytes;
+          tma_store_3d(&map_y, smem_u32(tile_b), col0, row0, b);
+        }
         if constexpr (SPEC) {
           uint8_t* tile_q = epi_mem + (warp - 2) * C::kEpiWarpBytes + 4096 + (c % NBUF) * 1024;
           tma_store_3d(&map_sfa, smem_u32(tile_q), col0, row0, b);
@@ -551,8 +575,17 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
     __threadfence();
     if (atomicAdd(p.ticket, 1u) == gridDim.x - 1) {
       __threadfence();
-      *p.stat_word = __uint_as_float(atomicExch(p.amax_scratch, 0u));
+      const float stat_now = __uint_as_float(atomicExch(p.amax_scratch, 0u));
+      *p.stat_word = stat_now;
       *p.ticket = 0u;
+      if constexpr (NOY) {
+        bool nfq;
+        const float r_true = rescale_factor(stat_now, &nfq);
+        const float ys = load_scale(p.a_scale) * load_scale(p.b_scale) * p.kf;
+        if (p.yq_scale) *p.yq_scale = ys * r_true;
+        if (p.hint_out) *p.hint_out = stat_now;  // every CTA has read the old prediction: all passed the ticket
+        if (nfq && p.status) atomicOr(p.status, static_cast<uint32_t>(SCALIFY_DEV_NONFINITE_STAT));
+      }
     }
   }
   if constexpr (NCTA == 2) cluster_sync_all();  // neither CTA leaves while the other may still touch its memory
@@ -584,6 +617,14 @@ scaled_matmul_spec_kernel(const __grid_constant__ CUtensorMap map_a, const __gri
                           const __grid_constant__ CUtensorMap map_y, const __grid_constant__ CUtensorMap map_q,
                           const GemmParams p) {
   gemm_body<OUT, NCTA, false, true>(map_a, map_b, map_y, map_q, map_q, p);
+}
+
+// The speculative kernel without the 16-bit intermediate: only the FP8 output is stored (map_y is not used).
+template <int OUT, int NCTA>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+scaled_matmul_fp8only_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                             const __grid_constant__ CUtensorMap map_q, const GemmParams p) {
+  gemm_body<OUT, NCTA, false, true, false, true>(map_a, map_b, map_q, map_q, map_q, p);
 }
 
 // Block-scaled operands (E8M0 exponent per 32 elements of K), K-major A [M,K] and B [N,K].
@@ -852,25 +893,29 @@ size_t matmul_ws_bytes(int64_t rows, int64_t cols) {
   return kWsHeader + size_t(tiles) * 8 * sizeof(double) + 256;
 }
 
-template <int OUT, int NCTA, bool SPEC, bool BIAS>
+template <int OUT, int NCTA, bool SPEC, bool BIAS, bool NOY = false>
 struct GemmKernelOf {
   static auto get() { return scaled_matmul_kernel<OUT, NCTA>; }
 };
 template <int OUT, int NCTA>
-struct GemmKernelOf<OUT, NCTA, true, false> {
+struct GemmKernelOf<OUT, NCTA, true, false, true> {
+  static auto get() { return scaled_matmul_fp8only_kernel<OUT, NCTA>; }
+};
+template <int OUT, int NCTA>
+struct GemmKernelOf<OUT, NCTA, true, false, false> {
   static auto get() { return scaled_matmul_spec_kernel<OUT, NCTA>; }
 };
 template <int OUT, int NCTA>
-struct GemmKernelOf<OUT, NCTA, false, true> {
+struct GemmKernelOf<OUT, NCTA, false, true, false> {
   static auto get() { return scaled_matmul_bias_kernel<OUT, NCTA>; }
 };
 
-template <int OUT, int NCTA, bool SPEC = false, bool BIAS = false>
+template <int OUT, int NCTA, bool SPEC = false, bool BIAS = false, bool NOY = false>
 static int launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_y,
                           const CUtensorMap& map_q, const GemmParams& p, long long tiles,
                           cudaStream_t st) {
   using C = GemmCfg<NCTA>;
-  auto kernel = GemmKernelOf<OUT, NCTA, SPEC, BIAS>::get();
+  auto kernel = GemmKernelOf<OUT, NCTA, SPEC, BIAS, NOY>::get();
   static bool attr_done = false;
   static int max_clusters = 0;
   if (!attr_done) {
@@ -910,7 +955,8 @@ static int launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, co
   cfg.blockDim = dim3(kGemmThreads);
   cfg.dynamicSmemBytes = C::kSmem;
   cfg.stream = st;
-  if constexpr (SPEC) SCALIFY_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, map_a, map_b, map_y, map_q, p));
+  if constexpr (NOY) SCALIFY_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, map_a, map_b, map_q, p));
+  else if constexpr (SPEC) SCALIFY_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, map_a, map_b, map_y, map_q, p));
   else SCALIFY_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, map_a, map_b, map_y, p));
   return SCALIFY_OK;
 }
@@ -923,7 +969,9 @@ int launch_scaled_matmul(const MatmulArgs& a, void* ws, size_t ws_bytes, cudaStr
   // A product with few output tiles and a long contraction (a weight gradient) leaves most SMs idle: its K
   // range is cut into `splits` parts that run as one batched call writing fp32 partial products into the
   // workspace (when the caller's workspace has the room), and a second launch adds them in split order.
-  if (!a.no_split && a.batch == 1 && !a.stat_in && !a.stat_hint && !a.bias && a.K >= 2048) {
+  if (a.took_spec) *a.took_spec = 0;
+  if (!a.no_split && a.batch == 1 && !a.stat_in && (!a.stat_hint || a.hint_optional) && !a.noy && !a.bias &&
+      a.K >= 2048) {
     const long long out_tiles = static_cast<long long>((a.M + tile_m - 1) / tile_m) * ((a.N + kBN - 1) / kBN);
     const long long units = ncta == 2 ? sm_count() / 2 : sm_count();
     int splits = static_cast<int>(units / out_tiles);
@@ -936,6 +984,7 @@ int launch_scaled_matmul(const MatmulArgs& a, void* ws, size_t ws_bytes, cudaStr
     if (splits >= 3 && ws_bytes >= need && red_blocks <= 65536) {  // (two parts measured no faster than one launch)
       float* part = reinterpret_cast<float*>(static_cast<char*>(v.area) + kSplitStatBytes);
       MatmulArgs pa = a;
+      pa.stat_hint = nullptr; pa.Yq = nullptr; pa.hint_optional = 0; pa.took_spec = nullptr;
       const int Kc = a.K / splits;
       pa.K = Kc;
       pa.batch = splits;
@@ -971,8 +1020,10 @@ int launch_scaled_matmul(const MatmulArgs& a, void* ws, size_t ws_bytes, cudaStr
   else rc = make_map(&map_b, a.B, a.N, a.K, b_batch, a.ldb, a.b_bs, kBK);
   if (rc) return rc;
 
-  rc = make_map_y(&map_y, a.Y, elem_size(a.y_dt), a.N, a.M, a.batch, a.ldy, a.y_bs);
-  if (rc) return rc;
+  if (!a.noy) {
+    rc = make_map_y(&map_y, a.Y, elem_size(a.y_dt), a.N, a.M, a.batch, a.ldy, a.y_bs);
+    if (rc) return rc;
+  }
 
   GemmParams p;
   p.M = a.M; p.N = a.N; p.K = a.K; p.batch = a.batch;
@@ -1003,9 +1054,28 @@ int launch_scaled_matmul(const MatmulArgs& a, void* ws, size_t ws_bytes, cudaStr
   p.q_dt = a.q_dt;
   p.bias = a.bias; p.bias_dt = a.bias_dt; p.bias_scale = a.bias_scale;
   p.r_pred_out = reinterpret_cast<float*>(static_cast<char*>(ws) + 52);  // header word read by the check kernel
+  p.yq_scale = a.yq_scale; p.hint_out = a.hint_out; p.redo = 0;
   const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n * p.batch;
   if (tiles > (1ll << 30)) return SCALIFY_ERR_SHAPE;
-  if (a.stat_hint) {
+  if (a.stat_hint && a.noy) {
+    // FP8 output only, then the repair launch (its CTAs return at once when the prediction held)
+    CUtensorMap map_q;
+    rc = make_map_y(&map_q, a.Yq, 1, a.N, a.M, a.batch, a.ldy, a.y_bs);
+    if (rc) return rc;
+    for (int pass = 0; pass < 2 && !rc; ++pass) {
+      p.redo = pass;
+      if (pass) p.stat_hint = v.stat;  // the statistic the first launch left is the exact "prediction"
+      if (a.y_dt == SCALIFY_BF16) {
+        if (ncta == 2) rc = launch_variant<SCALIFY_BF16, 2, true, false, true>(map_a, map_b, map_q, map_q, p, tiles, st);
+        else rc = launch_variant<SCALIFY_BF16, 1, true, false, true>(map_a, map_b, map_q, map_q, p, tiles, st);
+      } else {
+        if (ncta == 2) rc = launch_variant<SCALIFY_F16, 2, true, false, true>(map_a, map_b, map_q, map_q, p, tiles, st);
+        else rc = launch_variant<SCALIFY_F16, 1, true, false, true>(map_a, map_b, map_q, map_q, p, tiles, st);
+      }
+    }
+    if (a.took_spec) *a.took_spec = 1;
+  } else if (a.stat_hint) {
+    if (a.took_spec) *a.took_spec = 1;
     // speculative FP8 output next to the 16-bit intermediate
     CUtensorMap map_q;
     rc = make_map_y(&map_q, a.Yq, 1, a.N, a.M, a.batch, a.ldy, a.y_bs);
@@ -1148,6 +1218,7 @@ int launch_mx_matmul(const MxMatmulArgs& a, void* ws, cudaStream_t st) {
   p.stat_hint = nullptr;
   p.q_dt = SCALIFY_E4M3;
   p.r_pred_out = nullptr;
+  p.yq_scale = nullptr; p.hint_out = nullptr; p.redo = 0;
   const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n;
   if (tiles > (1ll << 30)) return SCALIFY_ERR_SHAPE;
   SCALIFY_DISPATCH_WIDE(a.y_dt, OUT, {

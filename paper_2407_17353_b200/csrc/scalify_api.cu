@@ -692,7 +692,7 @@ static int matmul_impl(const scalify_array* A, int transA, const scalify_array* 
     if (Yq->data == Y->data && elem_size(Yq->dtype) != elem_size(Y->dtype)) return SCALIFY_ERR_ALIAS;
     if (Yq->scale && (Yq->scale == A->scale || Yq->scale == B->scale)) return SCALIFY_ERR_ALIAS;
   }
-  MatmulArgs a;
+  MatmulArgs a{};
   a.A = A->data; a.a_dt = A->dtype; a.transA = transA ? 1 : 0; a.lda = A->stride[an - 2];
   a.a_bs = an == 3 ? A->stride[0] : 0;
   a.B = B->data; a.b_dt = B->dtype; a.transB = transB ? 1 : 0; a.ldb = B->stride[bn - 2];
@@ -715,6 +715,16 @@ static int matmul_impl(const scalify_array* A, int transA, const scalify_array* 
   a.stat_hint = nullptr;
   a.Yq = nullptr;
   a.q_dt = SCALIFY_E4M3;
+  int took_spec = 0;
+  a.took_spec = &took_spec;
+  if (!stat_hint && !bias && Yq && stat == SCALIFY_STAT_AMAX && is_fp8(Yq->dtype) && Yq->data != Y->data &&
+      (Y->dtype == SCALIFY_BF16 || Y->dtype == SCALIFY_F16) && N % 16 == 0) {
+    // The exact dynamic rescale, predicted: the GEMM already writes Yq with the power of two of the statistic
+    // this workspace saw last (header word at byte 56) and the check launch rebuilds Yq from Y only when this
+    // call's statistic has another power of two.  Same bits as statistic + second pass, whatever the word holds.
+    stat_hint = reinterpret_cast<float*>(static_cast<char*>(workspace) + 56);
+    a.hint_optional = 1;
+  }
   if (stat_hint) {
     // speculative rescale: 16-bit intermediate, FP8 result, AMAX (the statistic the GEMM gathers exactly)
     if (!Yq || stat != SCALIFY_STAT_AMAX) return SCALIFY_ERR_VALUE;
@@ -729,7 +739,7 @@ static int matmul_impl(const scalify_array* A, int transA, const scalify_array* 
   if (rc) return rc;
   if (Yq) {
     WsView v = ws_view(workspace);
-    if (stat_hint)
+    if (took_spec)
       rc = launch_rebalance_check(Y->data, Y->dtype, Yq->data, Yq->dtype, batch * M * N, y_scale, Yq->scale, v.stat,
                                   reinterpret_cast<const float*>(static_cast<char*>(workspace) + 52), stat_hint,
                                   v.status, st);
@@ -740,8 +750,54 @@ static int matmul_impl(const scalify_array* A, int transA, const scalify_array* 
   return rc;
 }
 
+// Y == NULL: only the rescaled FP8 output is stored (see the header).
+static int matmul_fp8only_impl(const scalify_array* A, int transA, const scalify_array* B, int transB, int stat,
+                               scalify_array* Yq, void* workspace, size_t workspace_bytes, void* stream) {
+  int rc = check_array(A);
+  if (rc) return rc;
+  if ((rc = check_array(B))) return rc;
+  if (!Yq) return SCALIFY_ERR_NULL;
+  if ((rc = check_array(Yq))) return rc;
+  if (!is_fp8(A->dtype) || !is_fp8(B->dtype) || !is_fp8(Yq->dtype)) return SCALIFY_ERR_DTYPE;
+  if (stat != SCALIFY_STAT_AMAX) return SCALIFY_ERR_VALUE;
+  if (A->ndim < 2 || A->ndim > 3 || B->ndim < 2 || Yq->ndim != A->ndim || B->ndim > A->ndim) return SCALIFY_ERR_SHAPE;
+  const int an = A->ndim, bn = B->ndim, yn = Yq->ndim;
+  const int64_t batch = an == 3 ? A->shape[0] : 1;
+  const int64_t M = transA ? A->shape[an - 1] : A->shape[an - 2];
+  const int64_t K = transA ? A->shape[an - 2] : A->shape[an - 1];
+  const int64_t Kb = transB ? B->shape[bn - 1] : B->shape[bn - 2];
+  const int64_t N = transB ? B->shape[bn - 2] : B->shape[bn - 1];
+  if (K != Kb || K < 1 || M < 1 || N < 1 || batch < 1) return SCALIFY_ERR_SHAPE;
+  if (Yq->shape[yn - 2] != M || Yq->shape[yn - 1] != N || contiguous_numel(Yq) != batch * M * N) return SCALIFY_ERR_SHAPE;
+  if (an == 3 && (Yq->shape[0] != batch || (bn == 3 && B->shape[0] != batch))) return SCALIFY_ERR_SHAPE;
+  if (M > 0x7FFFFFFF || N > 0x7FFFFFFF || K > 0x7FFFFFFF || batch > 0x7FFFFFFF) return SCALIFY_ERR_SHAPE;
+  if (N % 16 != 0) return SCALIFY_ERR_ALIGNMENT;  // rows of the FP8 output are written by TMA: 16-byte row stride
+  if (!Yq->scale) return SCALIFY_ERR_NULL;
+  if (Yq->scale == A->scale || Yq->scale == B->scale) return SCALIFY_ERR_ALIAS;
+  rc = check_ws(workspace, workspace_bytes, scalify_workspace_bytes(SCALIFY_OP_MATMUL, batch * M, N));
+  if (rc) return rc;
+  MatmulArgs a{};
+  a.A = A->data; a.a_dt = A->dtype; a.transA = transA ? 1 : 0; a.lda = A->stride[an - 2];
+  a.a_bs = an == 3 ? A->stride[0] : 0;
+  a.B = B->data; a.b_dt = B->dtype; a.transB = transB ? 1 : 0; a.ldb = B->stride[bn - 2];
+  a.b_bs = bn == 3 ? B->stride[0] : 0;
+  a.Y = nullptr; a.y_dt = SCALIFY_BF16; a.ldy = N; a.y_bs = yn == 3 ? M * N : 0;
+  a.M = static_cast<int>(M); a.N = static_cast<int>(N); a.K = static_cast<int>(K); a.batch = static_cast<int>(batch);
+  a.a_scale = A->scale; a.b_scale = B->scale;
+  a.y_scale = reinterpret_cast<float*>(static_cast<char*>(workspace) + 48);  // scale of the intermediate that is not stored
+  a.stat = SCALIFY_STAT_AMAX;
+  a.no_split = 1;
+  float* hint = reinterpret_cast<float*>(static_cast<char*>(workspace) + 56);
+  a.stat_hint = hint; a.hint_out = hint;
+  a.Yq = Yq->data; a.q_dt = Yq->dtype; a.yq_scale = Yq->scale;
+  a.noy = 1;
+  if (a.lda < (transA ? M : K) || a.ldb < (transB ? K : N)) return SCALIFY_ERR_SHAPE;
+  return launch_scaled_matmul(a, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
+}
+
 int scalify_scaled_matmul(const scalify_array* A, int transA, const scalify_array* B, int transB, scalify_array* Y,
                           int stat, scalify_array* Yq, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!Y) return matmul_fp8only_impl(A, transA, B, transB, stat, Yq, workspace, workspace_bytes, stream);
   return matmul_impl(A, transA, B, transB, nullptr, Y, stat, Yq, nullptr, workspace, workspace_bytes, stream);
 }
 
@@ -786,7 +842,7 @@ int scalify_scaled_matmul_delayed(const scalify_array* A, int transA, const scal
   if (Y->scale && (Y->scale == A->scale || Y->scale == B->scale)) return SCALIFY_ERR_ALIAS;
   rc = check_ws(workspace, workspace_bytes, scalify_workspace_bytes(SCALIFY_OP_MATMUL, batch * M, N));
   if (rc) return rc;
-  MatmulArgs a;
+  MatmulArgs a{};
   a.A = A->data; a.a_dt = A->dtype; a.transA = transA ? 1 : 0; a.lda = A->stride[an - 2];
   a.a_bs = an == 3 ? A->stride[0] : 0;
   a.B = B->data; a.b_dt = B->dtype; a.transB = transB ? 1 : 0; a.ldb = B->stride[bn - 2];

@@ -20,6 +20,7 @@ namespace scalify {
 // byte 32  : uint32 ticket of the "last block finishes" reductions (self-resetting)
 // byte 48  : fp32 scale word of an output whose caller passed no scale pointer
 // byte 52  : fp32 rescale factor a speculative matmul predicted
+// byte 56  : fp32 AMAX of the last matmul + FP8 rescale on this workspace (the next call's prediction)
 // byte 64  : (Adam) not used
 // byte 256 : operation-specific area
 constexpr size_t kWsStatus = 0;

@@ -84,6 +84,15 @@ struct MatmulArgs {
   // speculative rescale: predicted statistic (device) or NULL; then Yq (FP8, dense like Y) is written by the GEMM
   const float* stat_hint;
   void* Yq; int q_dt;
+  // stat_hint came from the library itself (the workspace header), not from the caller: a product that is better
+  // split over K ignores it.  *took_spec (optional) reports whether the speculative kernel ran.
+  int hint_optional;
+  int* took_spec;
+  // FP8-only form: Y is not stored (y_dt still names the 16-bit format the values are rounded through); the GEMM
+  // publishes Yq's scale word and the next prediction itself, and a repair launch of the same kernel follows.
+  int noy;
+  float* yq_scale;
+  float* hint_out;
   const void* bias; int bias_dt; const float* bias_scale;  // optional [N] vector added in the epilogue (add rule)
   float alpha_override;  // 0: the data component is divided by kf(K); otherwise multiplied by this (split-K partials)
   int no_split;          // 1: never split the contraction (the partial products of a split call)

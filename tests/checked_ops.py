@@ -130,7 +130,9 @@ class Ops:
         return X
 
     # ---------------------------------------------------------------- matmul
-    def mm(self, A, B, *, transA=False, transB=False, out_dt=BF, Y=None, stat=sc.STAT_NONE, q_dt=None):
+    def mm(self, A, B, *, transA=False, transB=False, out_dt=BF, Y=None, stat=sc.STAT_NONE, q_dt=None, key=None):
+        """key: a name for this call site.  A matmul with a fused rescale to FP8 predicts its rescale factor from the
+        statistic its workspace saw last, so such a call keeps a workspace of its own from step to step."""
         a, b = A.data, B.data
         M = a.shape[-1] if transA else a.shape[-2]
         N = b.shape[-2] if transB else b.shape[-1]
@@ -138,11 +140,18 @@ class Ops:
         if Y is None:
             Y = self.empty(shape, out_dt)
         Yq = self.empty(shape, q_dt) if q_dt is not None else None
-        sc.scalify_scaled_matmul(A, B, Y, self.ws, transA=transA, transB=transB, stat=stat, Yq=Yq)
+        ws = self.ws
+        if key is not None:
+            if not hasattr(self, "ws_keyed"):
+                self.ws_keyed = {}
+            if key not in self.ws_keyed:
+                self.ws_keyed[key] = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_MATMUL_SPLITK, M, N), self.dev)
+            ws = self.ws_keyed[key]
+        sc.scalify_scaled_matmul(A, B, Y, ws, transA=transA, transB=transB, stat=stat, Yq=Yq)
         self.calls += 1 + (1 if Yq is not None else 0)
         if self.check:
             o = self.orc
-            self._status_ok()
+            assert ws.check_status() == 0
             a_dt, b_dt, y_dt = code(a), code(b), code(Y.data)
             K = a.shape[-2] if transA else a.shape[-1]
             if self.mode == "sampled" and a.dim() == 2 and 2.0 * M * N * K > 4e9:
@@ -168,7 +177,7 @@ class Ops:
                     assert ok.all(), int((~ok).sum())
             if Yq is not None:
                 so = o.statistic(self.bits(Y).reshape(-1), y_dt, stat)
-                got = float(self.ws.statistic().item())
+                got = float(ws.statistic().item())
                 assert got == so if stat == sc.STAT_AMAX else abs(got - so) <= 2e-6 * so
                 qo, qs, _ = o.rescale(self.bits(Y).reshape(-1), y_dt, Y.scale_value(), stat, q_dt)
                 if not (stat == sc.STAT_L2 and abs(np.log2(so) - round(np.log2(so))) < 1e-5):

@@ -99,12 +99,13 @@ class ScaledGPT:
         # [n, K] x [K, N] (B stored [K, N]) + bias in the matmul's epilogue; the sum may be written as FP8 directly
         return self.ops.linear(x8, W8, bias, out_dt=out_dt)
 
-    def _linear_bwd(self, dy, x8, W8):
+    def _linear_bwd(self, dy, x8, W8, name):
         """dy BF16 -> (dx BF16, dW E5M2 rescaled, db E5M2 rescaled)."""
         o = self.ops
         dy8 = o.cast(dy, E5)
         dx = o.mm(dy8, W8, transB=True)               # dy W^T: W stored [K, N] = [N', K'] of this product
-        _, dW = o.mm(x8, dy8, transA=True, stat=sc.STAT_AMAX, q_dt=E5)   # x^T dy with fused AMAX rescale
+        # x^T dy with fused AMAX rescale; a workspace per weight, so that the predicted rescale holds step after step
+        _, dW = o.mm(x8, dy8, transA=True, stat=sc.STAT_AMAX, q_dt=E5, key=name)
         db = o.rescale(o.colsum(dy8), sc.STAT_AMAX, E5)                    # column sums, then the dynamic rescale
         return dx, dW, db
 
@@ -178,13 +179,13 @@ class ScaledGPT:
             o.active = check_layers is None or l in check_layers
             s = saved[l]
             # MLP
-            dg, grads[p + "w2"], grads[p + "b2"] = self._linear_bwd(dx, s["g8"], W8[p + "w2"])
+            dg, grads[p + "w2"], grads[p + "b2"] = self._linear_bwd(dx, s["g8"], W8[p + "w2"], p + "w2")
             da1 = o.gelu_bwd(dg, s["a1"])
-            dh2, grads[p + "w1"], grads[p + "b1"] = self._linear_bwd(da1, s["h2_8"], W8[p + "w1"])
+            dh2, grads[p + "w1"], grads[p + "b1"] = self._linear_bwd(da1, s["h2_8"], W8[p + "w1"], p + "w1")
             dln, grads[p + "ln2.g"], grads[p + "ln2.b"] = o.ln_bwd(dh2, s["x_mid"], P[p + "ln2.g"], s["mean2"], s["rinv2"])
             dx = o.add(dx, dln)
             # attention
-            datt, grads[p + "wo"], grads[p + "bo"] = self._linear_bwd(dx, s["o8"], W8[p + "wo"])
+            datt, grads[p + "wo"], grads[p + "bo"] = self._linear_bwd(dx, s["o8"], W8[p + "wo"], p + "wo")
             datt8 = o.cast(datt, E5)
             dq, dk, dv = (o.empty((n, d), BF) for _ in range(3))
             if hd == 64:
@@ -205,7 +206,7 @@ class ScaledGPT:
                 o.mm(dSb, self._heads(s["q8"], b), transA=True, Y=view(dk))          # dS^T Q
             dh = None
             for nm, dy in (("q", dq), ("k", dk), ("v", dv)):
-                dxx, grads[p + "w" + nm], grads[p + "b" + nm] = self._linear_bwd(dy, s["h8"], W8[p + "w" + nm])
+                dxx, grads[p + "w" + nm], grads[p + "b" + nm] = self._linear_bwd(dy, s["h8"], W8[p + "w" + nm], p + "w" + nm)
                 dh = dxx if dh is None else o.add(dh, dxx)
             dln, grads[p + "ln1.g"], grads[p + "ln1.b"] = o.ln_bwd(dh, s["x_in"], P[p + "ln1.g"], s["mean1"], s["rinv1"])
             dx = o.add(dx, dln)

@@ -381,3 +381,69 @@ def test_matmul_with_bias_in_the_epilogue(M, N, K, transB, y_dt, bias_dt):
         assert ok.all(), int((~ok).sum())
         if M <= 520:
             assert float(ws.statistic().item()) == float(np.abs(orc.decode(got, y_dt)).max())
+
+
+def _two_pass_reference(Ad, Bd, shape, y_dt, q_dt, **kw):
+    """The unpredicted path: GEMM with fused AMAX into the 16-bit intermediate, then the rebalance pass."""
+    Y = sc.ScaledTensor.empty(shape, sc.TORCH_DTYPE[y_dt])
+    Yq = sc.ScaledTensor.empty(shape, sc.TORCH_DTYPE[q_dt])
+    ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_MATMUL, shape[-2] * (shape[0] if len(shape) == 3 else 1), shape[-1]))
+    sc.scalify_scaled_matmul(Ad, Bd, Y, ws, stat=sc.STAT_AMAX, **kw)
+    sc.scalify_rescale(Y, Yq, stat=sc.STAT_AMAX, stat_in=ws.statistic())
+    assert ws.check_status() == 0
+    return dict(Y=to_bits(Y.data, y_dt), Yq=to_bits(Yq.data, q_dt), y_scale=Y.scale_value(), yq_scale=Yq.scale_value(),
+                stat=float(ws.statistic().item()))
+
+
+@pytest.mark.parametrize("shape_a,shape_b,transB", [((256, 256), (256, 256), True), ((520, 384), (384, 304), False),
+                                                     ((100, 128), (48, 128), True), ((3, 300, 192), (3, 272, 192), True),
+                                                     ((1024, 512), (768, 512), True)])
+@pytest.mark.parametrize("q_dt", [orc.E4M3, orc.E5M2])
+def test_main_call_predicts_the_rescale_and_the_fp8_only_form_is_bit_identical(shape_a, shape_b, transB, q_dt):
+    """scalify_scaled_matmul(..., AMAX, Yq) lets the GEMM write the FP8 output with the power of two of the
+    statistic its workspace saw last, and with Y = None stores nothing else.  For a fresh workspace, a right, a
+    wrong and a degenerate prediction alike: Y, Yq, both scale words and the statistic word are those of the
+    two-pass path (GEMM + AMAX, then the rebalance pass) bit for bit, and the prediction word leaves as this
+    call's statistic."""
+    A = si.to_bits(si.normal(91, 1, shape_a, 1.0), orc.E4M3)
+    B = si.to_bits(si.normal(92, 2, shape_b, 1.0), orc.E5M2)
+    Ad = sc.ScaledTensor.make(to_dev(A, orc.E4M3), 2.0 ** -2)
+    Bd = sc.ScaledTensor.make(to_dev(B, orc.E5M2), 2.0 ** 3)
+    M, N = shape_a[-2], (shape_b[-2] if transB else shape_b[-1])
+    shape = (M, N) if len(shape_a) == 2 else (shape_a[0], M, N)
+    ref = _two_pass_reference(Ad, Bd, shape, orc.BF16, q_dt, transB=transB)
+    qo, qs, _ = orc.rescale(ref["Y"].reshape(-1), orc.BF16, ref["y_scale"], orc.STAT_AMAX, q_dt)
+    assert ref["yq_scale"] == qs and np.array_equal(ref["Yq"].reshape(-1), qo)
+    stat = ref["stat"]
+    rows = M * (shape[0] if len(shape) == 3 else 1)
+    for fp8_only in (False, True):
+        ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_MATMUL, rows, N))
+        for k, hint in enumerate((None, None, stat * 1.3, stat * 64.0, stat / 1000.0, float("nan"), float("inf"), stat)):
+            if hint is not None:
+                ws.prediction().fill_(hint)      # (None: what the workspace holds: zero at first, then the statistic)
+            Y = None if fp8_only else sc.ScaledTensor.empty(shape, torch.bfloat16)
+            Yq = sc.ScaledTensor.empty(shape, sc.TORCH_DTYPE[q_dt])
+            Yq.data.view(torch.uint8).fill_(0x55)
+            sc.scalify_scaled_matmul(Ad, Bd, Y, ws, transB=transB, stat=sc.STAT_AMAX, Yq=Yq)
+            assert ws.check_status() == 0
+            assert float(ws.statistic().item()) == stat and float(ws.prediction().item()) == stat, (fp8_only, k)
+            assert Yq.scale_value() == ref["yq_scale"]
+            assert np.array_equal(to_bits(Yq.data, q_dt), ref["Yq"]), (fp8_only, k, hint)
+            if Y is not None:
+                assert Y.scale_value() == ref["y_scale"] and np.array_equal(to_bits(Y.data, orc.BF16), ref["Y"])
+
+
+def test_fp8_only_form_argument_checks():
+    A = sc.ScaledTensor.make(to_dev(si.to_bits(si.normal(93, 1, (64, 128), 1.0), orc.E4M3), orc.E4M3), 1.0)
+    B = sc.ScaledTensor.make(to_dev(si.to_bits(si.normal(93, 2, (40, 128), 1.0), orc.E4M3), orc.E4M3), 1.0)
+    ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_MATMUL, 64, 40))
+    Yq = sc.ScaledTensor.empty((64, 40), torch.float8_e4m3fn)
+    with pytest.raises(sc.ScalifyError) as e:      # rows of 40 bytes: not a multiple of 16
+        sc.scalify_scaled_matmul(A, B, None, ws, transB=True, stat=sc.STAT_AMAX, Yq=Yq)
+    assert e.value.code == -4
+    B16 = sc.ScaledTensor.make(to_dev(si.to_bits(si.normal(93, 3, (48, 128), 1.0), orc.E4M3), orc.E4M3), 1.0)
+    Yq16 = sc.ScaledTensor.empty((64, 48), torch.float8_e4m3fn)
+    for bad in (dict(stat=sc.STAT_L2, Yq=Yq16), dict(stat=sc.STAT_NONE, Yq=Yq16), dict(stat=sc.STAT_AMAX, Yq=None),
+                dict(stat=sc.STAT_AMAX, Yq=sc.ScaledTensor.empty((64, 48), torch.bfloat16))):
+        with pytest.raises(sc.ScalifyError):
+            sc.scalify_scaled_matmul(A, B16, None, ws, transB=True, **bad)
