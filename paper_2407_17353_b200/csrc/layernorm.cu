@@ -138,10 +138,11 @@ __global__ void __launch_bounds__(kLnThreads) layernorm_fwd_kernel(
   const int iters = rows_per_team;
   int buf = 0;
   extern __shared__ uint4 ln_stage[];  // [stage][v][thread]
-  auto issue = [&](int row, int slot) {
+  // (only rows of this block's own run are fetched: `mine` is false for the stages beyond it)
+  auto issue = [&](int row, int slot, bool mine) {
 #pragma unroll
     for (int v = 0; v < VPT; ++v) {
-      if (has[v] && row < R)
+      if (mine && has[v] && row < R)
         cp_async16(&ln_stage[(slot * VPT + v) * kLnThreads + threadIdx.x],
                    static_cast<const char*>(X) + (int64_t(row) * x_ld) * ElemBytes<XDT>::v + int64_t(t + v * TEAM) * 16);
     }
@@ -160,7 +161,7 @@ __global__ void __launch_bounds__(kLnThreads) layernorm_fwd_kernel(
   }
   cp_async_commit();
 #pragma unroll
-  for (int st = 0; st < kLnFwdStages; ++st) issue(first_row + st * rows_per_iter, st);
+  for (int st = 0; st < kLnFwdStages; ++st) issue(first_row + st * rows_per_iter, st, st < iters);
   cp_async_wait<kLnFwdStages>();  // the parameter group has landed (this thread's part) ...
   __syncthreads();                // ... and everybody else's
   const void* gamma_s = gb_stage;
@@ -195,7 +196,7 @@ __global__ void __launch_bounds__(kLnThreads) layernorm_fwd_kernel(
       }
       decode_vec<XDT, VEC>(w, x[v]);
     }
-    issue(row + kLnFwdStages * rows_per_iter, slot);  // refill the slot just read
+    issue(row + kLnFwdStages * rows_per_iter, slot, it + kLnFwdStages < iters);  // refill the slot just read
     if (++slot == kLnFwdStages) slot = 0;
     float s = 0.f;
 #pragma unroll
@@ -321,7 +322,80 @@ int launch_layernorm_fwd(const void* X, int x_dt, int64_t x_ld, void* Y, int y_d
 // ---------------------------------------------------------------------------------------------
 // ws layout (after the header): float dgamma_part[grid][d]; float dbeta_part[grid][d];
 // double stat_part[grid].
-template <int XDT, int DXDT, int TW, bool STAGED>
+// Packed two-wide fp32 arithmetic (one instruction for two lanes): the backward kernel is bound by instruction
+// issue, not by bytes, so its per-element arithmetic runs on float2 pairs.
+__device__ __forceinline__ float2 f2(float a, float b) { return make_float2(a, b); }
+__device__ __forceinline__ float2 f2(float a) { return make_float2(a, a); }
+
+// N elements of dtype DT held in raw words -> N/2 float2 pairs (element 2i in .x, 2i+1 in .y)
+template <int DT, int N>
+__device__ __forceinline__ void decode_pairs(const uint32_t* w, float2* f) {
+  if constexpr (DT == SCALIFY_F32) {
+#pragma unroll
+    for (int i = 0; i < N / 2; ++i) f[i] = f2(__uint_as_float(w[2 * i]), __uint_as_float(w[2 * i + 1]));
+  } else if constexpr (DT == SCALIFY_BF16) {
+#pragma unroll
+    for (int i = 0; i < N / 2; ++i) f[i] = f2(__uint_as_float(w[i] << 16), __uint_as_float(w[i] & 0xFFFF0000u));
+  } else if constexpr (DT == SCALIFY_F16) {
+#pragma unroll
+    for (int i = 0; i < N / 2; ++i) f[i] = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+  } else {
+#pragma unroll
+    for (int i = 0; i < N / 4; ++i) {
+      f[2 * i] = fp8x2_to_float2(w[i], DT == SCALIFY_E5M2);
+      f[2 * i + 1] = fp8x2_to_float2(w[i] >> 16, DT == SCALIFY_E5M2);
+    }
+  }
+}
+
+// N/2 float2 pairs -> N elements of dtype DT (round to nearest even; FP8 saturates)
+template <int DT, int N>
+__device__ __forceinline__ void encode_pairs(const float2* f, uint32_t* w) {
+  if constexpr (DT == SCALIFY_F32) {
+#pragma unroll
+    for (int i = 0; i < N / 2; ++i) { w[2 * i] = __float_as_uint(f[i].x); w[2 * i + 1] = __float_as_uint(f[i].y); }
+  } else if constexpr (DT == SCALIFY_BF16) {
+#pragma unroll
+    for (int i = 0; i < N / 2; ++i) {
+      __nv_bfloat162 t = __float22bfloat162_rn(f[i]);
+      w[i] = *reinterpret_cast<uint32_t*>(&t);
+    }
+  } else if constexpr (DT == SCALIFY_F16) {
+#pragma unroll
+    for (int i = 0; i < N / 2; ++i) {
+      __half2 t = __float22half2_rn(f[i]);
+      w[i] = *reinterpret_cast<uint32_t*>(&t);
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < N / 4; ++i) {
+      const uint32_t lo = __nv_cvt_float2_to_fp8x2(f[2 * i], __NV_SATFINITE, DT == SCALIFY_E5M2 ? __NV_E5M2 : __NV_E4M3);
+      const uint32_t hi = __nv_cvt_float2_to_fp8x2(f[2 * i + 1], __NV_SATFINITE, DT == SCALIFY_E5M2 ? __NV_E5M2 : __NV_E4M3);
+      w[i] = (lo & 0xFFFFu) | (hi << 16);
+    }
+  }
+}
+
+// Sum of a pair (a.x, a.y are two independent quantities) over the team; same buffer discipline as team_sum2.
+template <int TW>
+__device__ __forceinline__ float2 team_sum_pair(float2 a, float (*smem)[8][2], int team, int& buf) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1)
+    a = __fadd2_rn(a, f2(__shfl_xor_sync(0xFFFFFFFFu, a.x, o), __shfl_xor_sync(0xFFFFFFFFu, a.y, o)));
+  if constexpr (TW > 1) {
+    const int lane = threadIdx.x & 31, wit = (threadIdx.x >> 5) % TW;
+    float2* s = reinterpret_cast<float2*>(smem[buf] + team * TW);
+    if (lane == 0) s[wit] = a;
+    team_barrier<TW>(team);
+    a = s[0];
+#pragma unroll
+    for (int w = 1; w < TW; ++w) a = __fadd2_rn(a, s[w]);
+    buf ^= 1;
+  }
+  return a;
+}
+
+template <int XDT, int DXDT, int TW>
 __global__ void __launch_bounds__(kLnThreads, 2) layernorm_bwd_kernel(
     const void* __restrict__ G, int64_t g_ld, const void* __restrict__ X, int64_t x_ld, void* __restrict__ dX,
     int64_t dx_ld, int R, int d, const void* __restrict__ gamma, int gb_dt, const float* __restrict__ mean,
@@ -329,132 +403,114 @@ __global__ void __launch_bounds__(kLnThreads, 2) layernorm_bwd_kernel(
     float* __restrict__ dgamma_part, float* __restrict__ dbeta_part, double* __restrict__ stat_part) {
   asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   constexpr int VEC = 16 / ElemBytes<XDT>::v;
+  constexpr int HP = VEC / 2;  // float2 pairs per vector
   constexpr int OB = VEC * ElemBytes<DXDT>::v;
   constexpr int TEAM = 32 * TW;
   constexpr int TPB = kLnThreads / TEAM;
-  __shared__ float smem[2][8][2];
+  __shared__ __align__(16) float smem[2][8][2];
   // delayed rescale (Section 3.3): the gradient is stored already divided by r = p2_floor(earlier statistic)
-  // and this step's statistic is taken on the un-rebalanced fp32 values
-  float inv_r = 1.0f;
-  if (stat_in) { bool nf; inv_r = 1.0f / rescale_factor(__ldg(stat_in), &nf); }
+  // and this step's statistic is that of the un-rebalanced fp32 values.  r is a power of two, so dividing the
+  // three coefficients of the output expression by it gives the same bits as dividing the result, and the
+  // statistic of the un-rebalanced values is the statistic of the stored-scale values times r (exactly).
+  float inv_r = 1.0f, r_prev = 1.0f;
+  if (stat_in) { bool nf; r_prev = rescale_factor(__ldg(stat_in), &nf); inv_r = 1.0f / r_prev; }
   const int n_vec = d / VEC;
   const int t = threadIdx.x % TEAM;
   const int team = threadIdx.x / TEAM;
   const float inv_d = 1.0f / static_cast<float>(d);
   bool has[kLnVpt];
-  float gam[kLnVpt][VEC], acc_dg[kLnVpt][VEC], acc_db[kLnVpt][VEC];
+  float2 gam[kLnVpt][HP], acc_dg[kLnVpt][HP], acc_db[kLnVpt][HP];
 #pragma unroll
   for (int v = 0; v < kLnVpt; ++v) {
     has[v] = (t + v * TEAM) < n_vec;
+    float gf[VEC];
 #pragma unroll
-    for (int e = 0; e < VEC; ++e) { gam[v][e] = 1.0f; acc_dg[v][e] = 0.f; acc_db[v][e] = 0.f; }
-    if (has[v] && gamma) load_param_vec<VEC>(gamma, gb_dt, (t + v * TEAM) * VEC, gam[v]);
+    for (int e = 0; e < VEC; ++e) gf[e] = 1.0f;
+    if (has[v] && gamma) load_param_vec<VEC>(gamma, gb_dt, (t + v * TEAM) * VEC, gf);
+#pragma unroll
+    for (int h = 0; h < HP; ++h) { gam[v][h] = f2(gf[2 * h], gf[2 * h + 1]); acc_dg[v][h] = f2(0.f); acc_db[v][h] = f2(0.f); }
   }
   uint32_t amax = 0u;
-  float ssq = 0.f;
+  float2 ssq2 = f2(0.f);
+  // the grid strides over the rows: at any moment its teams work on one dense stretch of X, G and dX (teams that
+  // each walk their own contiguous run of rows measured 5 % slower)
   const int rows_per_iter = gridDim.x * TPB;
   const int iters = (R + rows_per_iter - 1) / rows_per_iter;
   int buf = 0;
-  // Rows in flight.  Short rows (several teams per block): the raw words of the team's next row are fetched
-  // into registers before the current row is processed.  Long rows (STAGED: one or two teams per block): one
-  // row ahead leaves too few bytes in flight per SM to cover the DRAM latency, so the next kLnBwdStages rows
-  // of X and G (and their mean / 1/sigma) travel as cp.async copies into shared memory, every thread copying
-  // and later reading only its own vectors.  (For short rows the staging costs more instructions than it
-  // saves: 131072 x 1024 went from 0.89 to 0.84 of the copy rate with it, 131072 x 4096 from 0.72 to 0.86.)
-  extern __shared__ uint4 ln_bstage[];  // STAGED: [stage][x | g][v][thread], then [stage][thread] {mean, rinv}
-  float2* ms_stage = reinterpret_cast<float2*>(ln_bstage + kLnBwdStages * 2 * kLnVpt * kLnThreads);
-  uint32_t nx[kLnVpt][4] = {}, ng[kLnVpt][4] = {};  // (zeroed once: words of absent vectors are decoded, never used)
+  // Rows in flight: the next kLnBwdStages rows of X and G travel as cp.async copies into shared memory, every
+  // thread copying and later reading only its own vectors (no barrier involved), so that enough bytes are in
+  // flight per SM to cover the DRAM latency whatever the arithmetic of the current row is waiting for; the
+  // row's mean and 1/sigma are fetched one row ahead into registers.  (Measured, 131072 x 1024 BF16: 139 us
+  // against 150 us with one row prefetched in registers.  An earlier form that also staged mean and 1/sigma with
+  // two 4-byte copies per thread was slower than either: 158 us.)
+  extern __shared__ uint4 ln_bstage[];  // [stage][x | g][v][thread]
   float nmu = 0.f, nrinv = 0.f;
-  auto fetch = [&](int row) {
-#pragma unroll
-    for (int v = 0; v < kLnVpt; ++v) {
-      if (has[v] && row < R) {
-        ld_raw_stream<16>(static_cast<const char*>(X) + (int64_t(row) * x_ld) * ElemBytes<XDT>::v +
-                              int64_t(t + v * TEAM) * 16, nx[v]);
-        ld_raw_stream<16>(static_cast<const char*>(G) + (int64_t(row) * g_ld) * ElemBytes<XDT>::v +
-                              int64_t(t + v * TEAM) * 16, ng[v]);
-      }
-    }
-    if (row < R) { nmu = __ldg(&mean[row]); nrinv = __ldg(&rinv_in[row]); }
-  };
+  const char* xcol = static_cast<const char*>(X) + int64_t(t) * 16;
+  const char* gcol = static_cast<const char*>(G) + int64_t(t) * 16;
+  const int64_t x_row_bytes = x_ld * ElemBytes<XDT>::v, g_row_bytes = g_ld * ElemBytes<XDT>::v;
+  const int first_row = blockIdx.x * TPB + team;
+  const int row_end = R;
   auto issue = [&](int row, int slot) {
-    if (row < R) {
+    if (row < row_end) {
 #pragma unroll
       for (int v = 0; v < kLnVpt; ++v) {
         if (has[v]) {
           cp_async16(&ln_bstage[((slot * 2 + 0) * kLnVpt + v) * kLnThreads + threadIdx.x],
-                     static_cast<const char*>(X) + (int64_t(row) * x_ld) * ElemBytes<XDT>::v + int64_t(t + v * TEAM) * 16);
+                     xcol + row * x_row_bytes + v * (TEAM * 16));
           cp_async16(&ln_bstage[((slot * 2 + 1) * kLnVpt + v) * kLnThreads + threadIdx.x],
-                     static_cast<const char*>(G) + (int64_t(row) * g_ld) * ElemBytes<XDT>::v + int64_t(t + v * TEAM) * 16);
+                     gcol + row * g_row_bytes + v * (TEAM * 16));
         }
       }
-      cp_async4(&ms_stage[slot * kLnThreads + threadIdx.x].x, &mean[row]);
-      cp_async4(&ms_stage[slot * kLnThreads + threadIdx.x].y, &rinv_in[row]);
     }
     cp_async_commit();  // one group per row, even when empty, so that the group count stays uniform
   };
-  const int first_row = blockIdx.x * TPB + team;
-  if constexpr (STAGED) {
 #pragma unroll
-    for (int st = 0; st < kLnBwdStages; ++st) issue(first_row + st * rows_per_iter, st);
-  } else {
-    fetch(first_row);
-  }
+  for (int st = 0; st < kLnBwdStages; ++st) issue(first_row + st * rows_per_iter, st);
+  if (first_row < row_end) { nmu = __ldg(&mean[first_row]); nrinv = __ldg(&rinv_in[first_row]); }
   int slot = 0;
   for (int it = 0; it < iters; ++it) {
     const int row = it * rows_per_iter + first_row;
-    const bool live = row < R;
-    float x[kLnVpt][VEC], g[kLnVpt][VEC];
+    const bool live = row < row_end;
+    float2 x[kLnVpt][HP], g[kLnVpt][HP];
     float mu = 0.f, rinv = 0.f;
-    if constexpr (STAGED) {
-      cp_async_wait<kLnBwdStages - 1>();  // the oldest row in flight has landed
-      if (live) {
-        const float2 ms = ms_stage[slot * kLnThreads + threadIdx.x];
-        mu = ms.x; rinv = ms.y;
-      }
-#pragma unroll
-      for (int v = 0; v < kLnVpt; ++v) {
-        uint32_t wx[4] = {0u, 0u, 0u, 0u}, wg[4] = {0u, 0u, 0u, 0u};
-        if (has[v] && live) {
-          const uint4 qx = ln_bstage[((slot * 2 + 0) * kLnVpt + v) * kLnThreads + threadIdx.x];
-          const uint4 qg = ln_bstage[((slot * 2 + 1) * kLnVpt + v) * kLnThreads + threadIdx.x];
-          wx[0] = qx.x; wx[1] = qx.y; wx[2] = qx.z; wx[3] = qx.w;
-          wg[0] = qg.x; wg[1] = qg.y; wg[2] = qg.z; wg[3] = qg.w;
-        }
-        decode_vec<XDT, VEC>(wx, x[v]);
-        decode_vec<XDT, VEC>(wg, g[v]);
-      }
-      issue(row + kLnBwdStages * rows_per_iter, slot);  // refill the slot just read
-      if (++slot == kLnBwdStages) slot = 0;
-    } else {
-#pragma unroll
-      for (int v = 0; v < kLnVpt; ++v) {
-        decode_vec<XDT, VEC>(nx[v], x[v]);
-        decode_vec<XDT, VEC>(ng[v], g[v]);
-      }
-      mu = nmu; rinv = nrinv;
-      fetch(row + rows_per_iter);
-    }
-    float m1 = 0.f, m2 = 0.f;
+    cp_async_wait<kLnBwdStages - 1>();  // the oldest row in flight has landed
+    mu = live ? nmu : 0.f;
+    rinv = live ? nrinv : 0.f;
+    if (row + rows_per_iter < row_end) { nmu = __ldg(&mean[row + rows_per_iter]); nrinv = __ldg(&rinv_in[row + rows_per_iter]); }
 #pragma unroll
     for (int v = 0; v < kLnVpt; ++v) {
+      uint32_t wx[4] = {0u, 0u, 0u, 0u}, wg[4] = {0u, 0u, 0u, 0u};
       if (has[v] && live) {
+        const uint4 qx = ln_bstage[((slot * 2 + 0) * kLnVpt + v) * kLnThreads + threadIdx.x];
+        const uint4 qg = ln_bstage[((slot * 2 + 1) * kLnVpt + v) * kLnThreads + threadIdx.x];
+        wx[0] = qx.x; wx[1] = qx.y; wx[2] = qx.z; wx[3] = qx.w;
+        wg[0] = qg.x; wg[1] = qg.y; wg[2] = qg.z; wg[3] = qg.w;
+      }
+      decode_pairs<XDT, VEC>(wx, x[v]);
+      decode_pairs<XDT, VEC>(wg, g[v]);
+    }
+    issue(row + kLnBwdStages * rows_per_iter, slot);  // refill the slot just read
+    if (++slot == kLnBwdStages) slot = 0;
+    // A row past the end (or an absent vector) holds zeros with rinv = 0: it adds exact zeros everywhere below,
+    // so the arithmetic needs no predicates; only the stores are guarded.
+    const float2 nmu2 = f2(-mu), rinv2 = f2(rinv);
+    float2 m12 = f2(0.f), m22 = f2(0.f);
 #pragma unroll
-        for (int e = 0; e < VEC; ++e) {
-          const float n = (x[v][e] - mu) * rinv;
-          acc_dg[v][e] = fmaf(g[v][e], n, acc_dg[v][e]);
-          acc_db[v][e] += g[v][e];
-          const float gh = g[v][e] * gam[v][e];
-          x[v][e] = n;   // keep n
-          g[v][e] = gh;  // keep ghat
-          m1 += gh;
-          m2 = fmaf(gh, n, m2);
-        }
+    for (int v = 0; v < kLnVpt; ++v) {
+#pragma unroll
+      for (int h = 0; h < HP; ++h) {
+        const float2 n = __fmul2_rn(__fadd2_rn(x[v][h], nmu2), rinv2);
+        acc_dg[v][h] = __ffma2_rn(g[v][h], n, acc_dg[v][h]);
+        acc_db[v][h] = __fadd2_rn(acc_db[v][h], g[v][h]);
+        const float2 gh = __fmul2_rn(g[v][h], gam[v][h]);
+        x[v][h] = n;   // keep n
+        g[v][h] = gh;  // keep ghat
+        m12 = __fadd2_rn(m12, gh);
+        m22 = __ffma2_rn(gh, n, m22);
       }
     }
-    team_sum2<TW>(m1, m2, smem, team, buf);
-    m1 *= inv_d;
-    m2 *= inv_d;
+    const float2 m = team_sum_pair<TW>(f2(m12.x + m12.y, m22.x + m22.y), smem, team, buf);
+    const float m1 = m.x * inv_d, m2 = m.y * inv_d;
     // eps outside the root: dx = (ghat-m1)*rinv - n*m2/s with s = 1/rinv - eps (0 if s == 0)
     // eps inside the root:  dx = rinv*(ghat - m1 - n*m2)
     float c2;
@@ -464,42 +520,39 @@ __global__ void __launch_bounds__(kLnThreads, 2) layernorm_bwd_kernel(
       const float s = __fdividef(1.0f, rinv) - eps;
       c2 = (s > 0.f) ? __fdividef(m2, s) : 0.f;
     }
-    const float nm1r = -m1 * rinv;
+    // coefficients at the stored scale (inv_r is 1 unless the rescale is delayed)
+    const float2 k_g = f2(rinv * inv_r), k_n = f2(-c2 * inv_r), k_0 = f2(-m1 * rinv * inv_r);
     if (live) {
-      char* orow = static_cast<char*>(dX) + int64_t(row) * dx_ld * ElemBytes<DXDT>::v;
+      char* orow = static_cast<char*>(dX) + int64_t(row) * dx_ld * ElemBytes<DXDT>::v + int64_t(t) * OB;
 #pragma unroll
       for (int v = 0; v < kLnVpt; ++v) {
         if (has[v]) {
-          float o[VEC];
+          float2 o[HP];
 #pragma unroll
-          for (int e = 0; e < VEC; ++e) o[e] = fmaf(g[v][e], rinv, fmaf(x[v][e], -c2, nm1r));
+          for (int h = 0; h < HP; ++h) o[h] = __ffma2_rn(g[v][h], k_g, __ffma2_rn(x[v][h], k_n, k_0));
           uint32_t ow[OB / 4 > 0 ? OB / 4 : 1];
-          if (stat_in) {
-            float oq[VEC];
-#pragma unroll
-            for (int e = 0; e < VEC; ++e) oq[e] = o[e] * inv_r;  // exact: a power of two
-            encode_vec<DXDT, VEC>(oq, ow);
-          } else {
-            encode_vec<DXDT, VEC>(o, ow);
-          }
-          st_raw<OB>(orow + int64_t(t + v * TEAM) * OB, ow);
-          if (stat_in && stat == SCALIFY_STAT_L2) {
-#pragma unroll
-            for (int e = 0; e < VEC; ++e) ssq = fmaf(o[e], o[e], ssq);
-          } else if (stat == SCALIFY_STAT_AMAX) {
+          encode_pairs<DXDT, VEC>(o, ow);
+          st_raw<OB>(orow + v * (TEAM * OB), ow);
+          if (stat == SCALIFY_STAT_AMAX) {
             // rounding is monotonic: the max of the stored values is the stored value of the max
 #pragma unroll
-            for (int e = 0; e < VEC; ++e) amax = max(amax, abs_bits(o[e]));
+            for (int h = 0; h < HP; ++h) amax = __vimax3_u32(amax, abs_bits(o[h].x), abs_bits(o[h].y));
           } else if (stat == SCALIFY_STAT_L2) {
-            float sv[VEC];
-            decode_vec<DXDT, VEC>(ow, sv);  // the values as stored
+            if (stat_in) {  // the unrounded values
 #pragma unroll
-            for (int e = 0; e < VEC; ++e) ssq = fmaf(sv[e], sv[e], ssq);
+              for (int h = 0; h < HP; ++h) ssq2 = __ffma2_rn(o[h], o[h], ssq2);
+            } else {        // the values as stored
+              float2 sv[HP];
+              decode_pairs<DXDT, VEC>(ow, sv);
+#pragma unroll
+              for (int h = 0; h < HP; ++h) ssq2 = __ffma2_rn(sv[h], sv[h], ssq2);
+            }
           }
         }
       }
     }
   }
+  const float ssq = ssq2.x + ssq2.y;
   // per-block column partials of dgamma / dbeta: teams of a block own the same columns
   if (dgamma_part) {
     if constexpr (TPB > 1) {
@@ -510,7 +563,11 @@ __global__ void __launch_bounds__(kLnThreads, 2) layernorm_bwd_kernel(
         for (int v = 0; v < kLnVpt; ++v) {
           __syncthreads();
 #pragma unroll
-          for (int e = 0; e < VEC; ++e) s_col[team][t][e] = pass ? acc_db[v][e] : acc_dg[v][e];
+          for (int h = 0; h < HP; ++h) {
+            const float2 a = pass ? acc_db[v][h] : acc_dg[v][h];
+            s_col[team][t][2 * h] = a.x;
+            s_col[team][t][2 * h + 1] = a.y;
+          }
           __syncthreads();
           if (team == 0 && has[v]) {
             float* dst = (pass ? dbeta_part : dgamma_part) + int64_t(blockIdx.x) * d + (t + v * TEAM) * VEC;
@@ -528,10 +585,10 @@ __global__ void __launch_bounds__(kLnThreads, 2) layernorm_bwd_kernel(
 #pragma unroll
       for (int v = 0; v < kLnVpt; ++v) {
         if (has[v]) {
-          float* dg = dgamma_part + int64_t(blockIdx.x) * d + (t + v * TEAM) * VEC;
-          float* db = dbeta_part + int64_t(blockIdx.x) * d + (t + v * TEAM) * VEC;
+          float2* dg = reinterpret_cast<float2*>(dgamma_part + int64_t(blockIdx.x) * d + (t + v * TEAM) * VEC);
+          float2* db = reinterpret_cast<float2*>(dbeta_part + int64_t(blockIdx.x) * d + (t + v * TEAM) * VEC);
 #pragma unroll
-          for (int e = 0; e < VEC; ++e) { dg[e] = acc_dg[v][e]; db[e] = acc_db[v][e]; }
+          for (int h = 0; h < HP; ++h) { dg[h] = acc_dg[v][h]; db[h] = acc_db[v][h]; }
         }
       }
     }
@@ -539,9 +596,12 @@ __global__ void __launch_bounds__(kLnThreads, 2) layernorm_bwd_kernel(
   if (stat != SCALIFY_STAT_NONE) {
     __shared__ double s_stat[kLnThreads / 32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (stat == SCALIFY_STAT_AMAX && !stat_in) amax = abs_bits(round_through<DXDT>(__uint_as_float(amax)));
-    double mine = (stat == SCALIFY_STAT_AMAX) ? static_cast<double>(warp_max_u32(amax))
-                                              : warp_sum_f64(static_cast<double>(ssq));
+    // AMAX: of the stored values (plain call) or of the un-rebalanced, unrounded ones (delayed: times r, exact)
+    if (stat == SCALIFY_STAT_AMAX)
+      amax = stat_in ? abs_bits(__uint_as_float(amax) * r_prev) : abs_bits(round_through<DXDT>(__uint_as_float(amax)));
+    double mine = (stat == SCALIFY_STAT_AMAX)
+                      ? static_cast<double>(warp_max_u32(amax))
+                      : warp_sum_f64(static_cast<double>(ssq)) * (static_cast<double>(r_prev) * static_cast<double>(r_prev));
     if (lane == 0) s_stat[warp] = mine;
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -637,15 +697,13 @@ size_t layernorm_bwd_ws_bytes(int64_t R, int64_t d) {
   return kWsHeader + size_t(grid) * size_t(d) * 8 + size_t(grid) * 8 + 256;
 }
 
-// Launch shape of the backward kernel: team width, whether rows are staged through shared memory, grid
-// (persistent) and the number of rows each team walks.
-struct LnBwdPlan { int tw, staged, grid, iters; bool ok; };
+// Launch shape of the backward kernel: team width, grid (persistent) and the number of rows each team walks.
+struct LnBwdPlan { int tw, grid, iters; bool ok; };
 static LnBwdPlan ln_bwd_plan(int R, int d, int x_dt) {
   LnBwdPlan p{};
   p.tw = ln_team_warps(d, x_dt);
   p.ok = p.tw != 0;
   if (!p.ok) return p;
-  p.staged = p.tw >= 4;
   p.grid = ln_grid(R, 8 / p.tw, kLnBwdBlocksPerSm);
   const int64_t rows_per_iter = int64_t(p.grid) * (8 / p.tw);
   p.iters = static_cast<int>((R + rows_per_iter - 1) / rows_per_iter);
@@ -656,7 +714,7 @@ int layernorm_plan(int64_t R, int64_t d, int x_dt, int backward, int32_t out[4])
   if (backward) {
     const LnBwdPlan p = ln_bwd_plan(static_cast<int>(R), static_cast<int>(d), x_dt);
     if (!p.ok) return SCALIFY_ERR_UNSUPPORTED;
-    out[0] = p.grid; out[1] = p.iters; out[2] = p.tw; out[3] = p.staged ? kLnBwdStages : 0;
+    out[0] = p.grid; out[1] = p.iters; out[2] = p.tw; out[3] = kLnBwdStages;
   } else {
     const LnFwdPlan p = ln_fwd_plan(static_cast<int>(R), static_cast<int>(d), x_dt);
     if (!p.ok) return SCALIFY_ERR_UNSUPPORTED;
@@ -679,25 +737,21 @@ int launch_layernorm_bwd(const void* G, int64_t g_ld, const void* X, int x_dt, i
   double* st_part = reinterpret_cast<double*>(db_part + size_t(grid) * d);
   float* dgp = dgamma ? dg_part : nullptr;
   float* dbp = dgamma ? db_part : nullptr;
-  constexpr int kBwdSmem = kLnBwdStages * (2 * kLnVpt * kLnThreads * 16 + kLnThreads * 8);
-#define SCALIFY_LN_BWD(W, STG)                                                                                   \
+  constexpr int kBwdSmem = kLnBwdStages * 2 * kLnVpt * kLnThreads * 16;
+#define SCALIFY_LN_BWD(W)                                                                                        \
   do {                                                                                                           \
-    static bool attr_done = false;                                                                               \
-    if (STG && !attr_done) {                                                                                     \
-      SCALIFY_CUDA_TRY(cudaFuncSetAttribute(layernorm_bwd_kernel<XDT, DXDT, W, STG>,                             \
-                                            cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmem));             \
-      attr_done = true;                                                                                          \
-    }                                                                                                            \
-    layernorm_bwd_kernel<XDT, DXDT, W, STG><<<grid, kLnThreads, STG ? kBwdSmem : 0, st>>>(                       \
+    SCALIFY_CUDA_TRY(cudaFuncSetAttribute(layernorm_bwd_kernel<XDT, DXDT, W>,                                    \
+                                          cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmem));               \
+    layernorm_bwd_kernel<XDT, DXDT, W><<<grid, kLnThreads, kBwdSmem, st>>>(                                      \
         G, g_ld, X, x_ld, dX, dx_ld, R, d, gamma, gb_dt, mean, rinv, eps, eps_inside, stat, stat_in, dgp, dbp,   \
         st_part);                                                                                                \
   } while (0)
   SCALIFY_DISPATCH_WIDE(x_dt, XDT, SCALIFY_DISPATCH_DTYPE(dx_dt, DXDT, {
     switch (tw) {
-      case 1: SCALIFY_LN_BWD(1, false); break;
-      case 2: SCALIFY_LN_BWD(2, false); break;
-      case 4: SCALIFY_LN_BWD(4, true); break;
-      default: SCALIFY_LN_BWD(8, true); break;
+      case 1: SCALIFY_LN_BWD(1); break;
+      case 2: SCALIFY_LN_BWD(2); break;
+      case 4: SCALIFY_LN_BWD(4); break;
+      default: SCALIFY_LN_BWD(8); break;
     }
   }));
 #undef SCALIFY_LN_BWD
