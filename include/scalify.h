@@ -362,6 +362,18 @@ int scalify_debug_expire_wait(void* workspace, size_t workspace_bytes, uint32_t 
                               void* stream);
 
 /*
+ * Diagnostics of the library's host-side state (no counterpart in the paper; host only, no GPU needed).
+ * The library keeps two things between calls: the one-time set-up of each kernel PER DEVICE (dynamic
+ * shared-memory limit, co-resident cluster count) and a cache of encoded TMA tensor maps keyed by pointer,
+ * extents, strides and box.  scalify_debug_host_state_selftest drives both with made-up device numbers and a
+ * stand-in encoder and returns 0 if each device was set up exactly once and the cache returned the right map
+ * for every key; scalify_debug_tensor_map_cache reports how many encodes the real cache has saved (hits) and
+ * made (misses) so far in this process.
+ */
+int scalify_debug_host_state_selftest(void);
+int scalify_debug_tensor_map_cache(uint64_t* hits, uint64_t* misses);
+
+/*
  * Diagnostic (no counterpart in the paper): the launch shape the LayerNorm kernels would use for an
  * [R,d] input of dtype x_dtype on the current device, so that a test can state which code path it
  * exercised.  Host only, launches nothing.  plan[0] = thread blocks; plan[1] = rows every team of

@@ -95,6 +95,9 @@ def lib() -> ctypes.CDLL:
         L.scalify_debug_expire_wait.argtypes = [vp, sz, c.c_uint32, vp, vp]
         L.scalify_scalar_mul_pow2.argtypes = [P, f32, vp]
         L.scalify_debug_layernorm_plan.argtypes = [i64, i64, i32, i32, vp]
+        L.scalify_debug_host_state_selftest.restype = i32
+        L.scalify_debug_tensor_map_cache.argtypes = [vp, vp]
+        L.scalify_debug_tensor_map_cache.restype = i32
         L.scalify_scaled_embedding.argtypes = [vp, i64, i64, P, P, P, vp, vp]
         L.scalify_scaled_embedding_bwd.argtypes = [vp, i64, i64, P, P, P, vp]
         L.scalify_scaled_softmax.argtypes = [P, i32, P, vp]
@@ -414,6 +417,13 @@ def scalify_scalar_mul_pow2(X: ScaledTensor, c: float, *, stream=None) -> None:
 def scalify_debug_expire_wait(ws: Workspace, limit_us: int, waited_us: Optional[torch.Tensor] = None, *, stream=None) -> None:
     _check(lib().scalify_debug_expire_wait(ws.ptr, ws.nbytes, int(limit_us), _ptr(waited_us), _stream(stream)),
            "scalify_debug_expire_wait")
+
+
+def scalify_debug_tensor_map_cache() -> dict:
+    """Encodes saved (hits) and made (misses) by the library's tensor-map cache in this process."""
+    h, m = ctypes.c_uint64(0), ctypes.c_uint64(0)
+    _check(lib().scalify_debug_tensor_map_cache(ctypes.byref(h), ctypes.byref(m)), "scalify_debug_tensor_map_cache")
+    return dict(hits=int(h.value), misses=int(m.value))
 
 
 def scalify_debug_layernorm_plan(R: int, d: int, x_dtype: int, backward: bool) -> dict:

@@ -369,11 +369,12 @@ int launch_attention(const AttentionArgs& a, cudaStream_t st) {
   if (ctas > 0x7FFFFFFF) return SCALIFY_ERR_SHAPE;
   SCALIFY_DISPATCH_WIDE(a.o_dt, ODT, {
     auto kernel = attention_fwd_kernel<ODT>;
-    static bool attr_done = false;
-    if (!attr_done) {
+    static DeviceOnce once;  // (one per instantiation: the attribute belongs to this kernel on this device)
+    int rc_once = device_once(once, nullptr, [&](int*) {
       SCALIFY_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kAttSmem)));
-      attr_done = true;
-    }
+      return int(SCALIFY_OK);
+    });
+    if (rc_once) return rc_once;
     kernel<<<static_cast<unsigned>(ctas), kAttThreads, kAttSmem, st>>>(map_q, map_k, map_v, p);
   });
   SCALIFY_CUDA_TRY(cudaGetLastError());

@@ -547,12 +547,13 @@ int launch_attention_bwd(const AttentionBwdArgs& a, cudaStream_t st) {
   SCALIFY_DISPATCH_WIDE(a.g_dt, GDT, {
     auto k1 = attention_bwd_dq_kernel<GDT>;
     auto k2 = attention_bwd_dkv_kernel<GDT>;
-    static bool attr_done = false;
-    if (!attr_done) {
+    static DeviceOnce once;  // (one per instantiation: the attributes belong to these kernels on this device)
+    int rc_once = device_once(once, nullptr, [&](int*) {
       SCALIFY_CUDA_TRY(cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kBw1Smem)));
       SCALIFY_CUDA_TRY(cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kBw2Smem)));
-      attr_done = true;
-    }
+      return int(SCALIFY_OK);
+    });
+    if (rc_once) return rc_once;
     k1<<<static_cast<unsigned>(ctas1), kBw1Threads, kBw1Smem, st>>>(map_do, map_v, map_k, map_p, p);
     SCALIFY_CUDA_TRY(cudaGetLastError());
     k2<<<static_cast<unsigned>(ctas2), kBw2Threads, kBw2Smem, st>>>(map_p2, map_ds2, map_do2, map_q2, p);

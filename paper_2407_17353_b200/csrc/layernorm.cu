@@ -289,9 +289,15 @@ int launch_layernorm_fwd(const void* X, int x_dt, int64_t x_ld, void* Y, int y_d
     /* row staging + gamma and beta (up to 4 bytes per element each) */                                       \
     constexpr int kSmemMax = kLnFwdStages * V * kLnThreads * 16 + 2 * (32 * W * V * 16 / 2) * 4;               \
     const int smem_bytes = kLnFwdStages * V * kLnThreads * 16 + 2 * d * 4;                                     \
-    if (kSmemMax > 40 * 1024) /* the kernel also has a little static shared memory */                         \
-      SCALIFY_CUDA_TRY(cudaFuncSetAttribute(layernorm_fwd_kernel<XDT, YDT, W, V>,                              \
-                                            cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax));           \
+    if (kSmemMax > 40 * 1024) { /* the kernel also has a little static shared memory */                       \
+      static DeviceOnce once; /* per instantiation and device */                                               \
+      int rc_once = device_once(once, nullptr, [&](int*) {                                                     \
+        SCALIFY_CUDA_TRY(cudaFuncSetAttribute(layernorm_fwd_kernel<XDT, YDT, W, V>,                            \
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax));         \
+        return int(SCALIFY_OK);                                                                                \
+      });                                                                                                      \
+      if (rc_once) return rc_once;                                                                             \
+    }                                                                                                          \
     layernorm_fwd_kernel<XDT, YDT, W, V><<<grid, kLnThreads, smem_bytes, st>>>(                                     \
         X, x_ld, Y, y_ld, R, d, gamma, beta, gb_dt, gamma_scale, beta_scale, y_scale, eps, eps_inside, mean,   \
         rinv, rpt);                                                                                                \
@@ -740,8 +746,13 @@ int launch_layernorm_bwd(const void* G, int64_t g_ld, const void* X, int x_dt, i
   constexpr int kBwdSmem = kLnBwdStages * 2 * kLnVpt * kLnThreads * 16;
 #define SCALIFY_LN_BWD(W)                                                                                        \
   do {                                                                                                           \
-    SCALIFY_CUDA_TRY(cudaFuncSetAttribute(layernorm_bwd_kernel<XDT, DXDT, W>,                                    \
-                                          cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmem));               \
+    static DeviceOnce once; /* per instantiation and device */                                                   \
+    int rc_once = device_once(once, nullptr, [&](int*) {                                                         \
+      SCALIFY_CUDA_TRY(cudaFuncSetAttribute(layernorm_bwd_kernel<XDT, DXDT, W>,                                  \
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmem));             \
+      return int(SCALIFY_OK);                                                                                    \
+    });                                                                                                          \
+    if (rc_once) return rc_once;                                                                                 \
     layernorm_bwd_kernel<XDT, DXDT, W><<<grid, kLnThreads, kBwdSmem, st>>>(                                      \
         G, g_ld, X, x_ld, dX, dx_ld, R, d, gamma, gb_dt, mean, rinv, eps, eps_inside, stat, stat_in, dgp, dbp,   \
         st_part);                                                                                                \

@@ -18,6 +18,9 @@
 // Every wait on an mbarrier is bounded; on expiry the CTA records SCALIFY_DEV_TIMEOUT, drains
 // its own copies in flight, frees its TMEM and returns.
 #include <cuda.h>
+#include <string.h>
+
+#include <mutex>
 
 #include "scalify_common.cuh"
 #include "scalify_launch.h"
@@ -788,6 +791,119 @@ static EncodeTiledFn get_encode_fn() {
   return fn;
 }
 
+// Encoded tensor maps are kept: a training step calls the same matmuls on the same buffers over and over, and
+// encoding is host work (about a microsecond per map, three to five maps per call).  The key is everything the
+// encoder is given; a tensor map describes addresses and a layout, not the memory's contents, so it stays valid
+// for as long as that key describes what the caller passes.  256 entries, hashed, overwritten on collision.
+struct MapKey {
+  uint64_t ptr, dims[5], strides[4];
+  uint32_t box[5], estr[5], dtype, rank, interleave, swizzle, promo, oob;
+};
+struct MapCache {
+  static constexpr int kEntries = 256;
+  std::mutex mu;
+  bool used[kEntries] = {};
+  MapKey keys[kEntries];
+  CUtensorMap maps[kEntries];
+  unsigned long long hits = 0, misses = 0;
+};
+static MapCache g_map_cache;
+
+int encode_tiled_cached(MapCache& cache, EncodeTiledFn fn, CUtensorMap* map, CUtensorMapDataType dt, cuuint32_t rank,
+                        void* ptr, const cuuint64_t* dims, const cuuint64_t* strides, const cuuint32_t* box,
+                        const cuuint32_t* estr, CUtensorMapInterleave il, CUtensorMapSwizzle sw,
+                        CUtensorMapL2promotion promo, CUtensorMapFloatOOBfill oob) {
+  MapKey k;
+  memset(&k, 0, sizeof(k));
+  k.ptr = reinterpret_cast<uint64_t>(ptr);
+  for (cuuint32_t i = 0; i < rank; ++i) { k.dims[i] = dims[i]; k.box[i] = box[i]; k.estr[i] = estr[i]; }
+  for (cuuint32_t i = 0; i + 1 < rank; ++i) k.strides[i] = strides[i];
+  k.dtype = static_cast<uint32_t>(dt); k.rank = rank; k.interleave = static_cast<uint32_t>(il);
+  k.swizzle = static_cast<uint32_t>(sw); k.promo = static_cast<uint32_t>(promo); k.oob = static_cast<uint32_t>(oob);
+  uint64_t h = 1469598103934665603ull;  // FNV-1a over the key
+  const unsigned char* b = reinterpret_cast<const unsigned char*>(&k);
+  for (size_t i = 0; i < sizeof(k); ++i) { h ^= b[i]; h *= 1099511628211ull; }
+  const int slot = static_cast<int>((h ^ (h >> 29)) % MapCache::kEntries);
+  std::lock_guard<std::mutex> lock(cache.mu);
+  if (cache.used[slot] && memcmp(&cache.keys[slot], &k, sizeof(k)) == 0) {
+    *map = cache.maps[slot];
+    ++cache.hits;
+    return SCALIFY_OK;
+  }
+  CUresult r = fn(map, dt, rank, ptr, dims, strides, box, estr, il, sw, promo, oob);
+  if (r != CUDA_SUCCESS) {
+    set_last_cuda_error(static_cast<int>(r));
+    return SCALIFY_ERR_CUDA;
+  }
+  cache.keys[slot] = k;
+  cache.maps[slot] = *map;
+  cache.used[slot] = true;
+  ++cache.misses;
+  return SCALIFY_OK;
+}
+
+// Self-test of the two pieces of host state above, without a GPU: the per-device one-time set-up is driven with
+// made-up device numbers, the tensor-map cache with a stand-in for the driver's encoder that counts its calls.
+static int g_fake_encodes = 0;
+static CUresult fake_encode(CUtensorMap* m, CUtensorMapDataType, cuuint32_t rank, void* p, const cuuint64_t* dims,
+                            const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                            CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill) {
+  ++g_fake_encodes;
+  memset(m, 0, sizeof(*m));
+  uint64_t tag = reinterpret_cast<uint64_t>(p) ^ (dims[0] << 20) ^ rank;
+  memcpy(m, &tag, sizeof(tag));
+  return CUDA_SUCCESS;
+}
+int host_state_selftest() {
+  // (1) per-device once: devices 0, 1, 0, 2, 1, 63 -> four set-ups, each device keeps its own value
+  DeviceOnce once;
+  int runs = 0, v = -1;
+  const int order[6] = {0, 1, 0, 2, 1, 63};
+  for (int i = 0; i < 6; ++i) {
+    const int dev = order[i];
+    if (device_once_at(once, dev, &v, [&](int* val) { ++runs; *val = 100 + dev; return int(SCALIFY_OK); })) return 1;
+    if (v != 100 + dev) return 2;
+  }
+  if (runs != 4) return 3;
+  if (device_once_at(once, 64, &v, [&](int*) { return int(SCALIFY_OK); }) != SCALIFY_ERR_UNSUPPORTED) return 4;
+  // a set-up that fails is not remembered as done
+  int tries = 0;
+  if (device_once_at(once, 5, &v, [&](int*) { ++tries; return int(SCALIFY_ERR_CUDA); }) != SCALIFY_ERR_CUDA) return 5;
+  if (device_once_at(once, 5, &v, [&](int* val) { ++tries; *val = 7; return int(SCALIFY_OK); }) || v != 7 || tries != 2) return 6;
+  // (2) tensor-map cache
+  MapCache* cache = new MapCache();
+  g_fake_encodes = 0;
+  cuuint64_t dims[3] = {4096, 128, 1}, strides[2] = {4096, 4096 * 128};
+  cuuint32_t box[3] = {128, 128, 1}, estr[3] = {1, 1, 1};
+  CUtensorMap a, b, c;
+  char* base = reinterpret_cast<char*>(0x100000);
+  int bad = 0;
+  auto enc = [&](CUtensorMap* m, void* p, cuuint64_t d0) {
+    dims[0] = d0;
+    return encode_tiled_cached(*cache, fake_encode, m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, p, dims, strides, box, estr,
+                               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  };
+  bad |= enc(&a, base, 4096);             // miss
+  bad |= enc(&b, base, 4096);             // hit: same bytes, no second encode
+  if (bad || g_fake_encodes != 1 || memcmp(&a, &b, sizeof(a)) != 0) { delete cache; return 7; }
+  bad |= enc(&c, base + 4096, 4096);      // another pointer: miss
+  bad |= enc(&c, base, 8192);             // another extent: miss
+  if (bad || g_fake_encodes != 3 || memcmp(&a, &c, sizeof(a)) == 0) { delete cache; return 8; }
+  for (int i = 0; i < 2000; ++i) bad |= enc(&c, base + 16 * i, 4096);   // more keys than entries: still correct
+  bad |= enc(&b, base, 4096);
+  if (bad || memcmp(&a, &b, sizeof(a)) != 0) { delete cache; return 9; }
+  const bool counted = cache->hits + cache->misses == 2005 && cache->misses == static_cast<unsigned long long>(g_fake_encodes);
+  delete cache;
+  return counted ? 0 : 10;
+}
+
+void map_cache_counters(unsigned long long* hits, unsigned long long* misses) {
+  std::lock_guard<std::mutex> lock(g_map_cache.mu);
+  *hits = g_map_cache.hits;
+  *misses = g_map_cache.misses;
+}
+
 // Tensor map over a row-major byte matrix [batch][rows][inner] with row stride ld and batch
 // stride bs (bytes); box = [1][box_rows][128].
 static int make_map(CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t rows, uint64_t batch, uint64_t ld,
@@ -798,14 +914,9 @@ static int make_map(CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t 
   cuuint64_t strides[2] = {ld, bs ? bs : ld * rows};
   cuuint32_t box[3] = {128u, box_rows, 1u};
   cuuint32_t estr[3] = {1u, 1u, 1u};
-  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(ptr), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) {
-    set_last_cuda_error(static_cast<int>(r));
-    return SCALIFY_ERR_CUDA;
-  }
-  return SCALIFY_OK;
+  return encode_tiled_cached(g_map_cache, fn, map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(ptr), dims, strides,
+                             box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
 }
 
 // Tensor map over a row-major byte matrix [batch][rows][inner] with a box of [1][box_rows][box_inner]
@@ -820,14 +931,9 @@ int make_byte_map(CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t ro
   cuuint32_t estr[3] = {1u, 1u, 1u};
   const CUtensorMapSwizzle sw = box_inner == 32 ? CU_TENSOR_MAP_SWIZZLE_32B
                               : box_inner == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B;
-  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(ptr), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) {
-    set_last_cuda_error(static_cast<int>(r));
-    return SCALIFY_ERR_CUDA;
-  }
-  return SCALIFY_OK;
+  return encode_tiled_cached(g_map_cache, fn, map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(ptr), dims, strides,
+                             box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
 }
 
 // The same for [batch][heads][rows][inner] views (attention operands): box = one tile of one head
@@ -842,14 +948,9 @@ int make_byte_map4(CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t r
   cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
   const CUtensorMapSwizzle sw = box_inner == 32 ? CU_TENSOR_MAP_SWIZZLE_32B
                               : box_inner == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B;
-  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(ptr), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) {
-    set_last_cuda_error(static_cast<int>(r));
-    return SCALIFY_ERR_CUDA;
-  }
-  return SCALIFY_OK;
+  return encode_tiled_cached(g_map_cache, fn, map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(ptr), dims, strides,
+                             box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
 }
 
 // Tensor map of the output [batch][M][N] (row stride ld, batch stride bs, in elements of `es` bytes) for the
@@ -866,13 +967,9 @@ static int make_map_y(CUtensorMap* map, const void* ptr, int es, uint64_t N, uin
                                : es == 2 ? CU_TENSOR_MAP_DATA_TYPE_UINT16 : CU_TENSOR_MAP_DATA_TYPE_UINT32;
   const CUtensorMapSwizzle sw = es == 1 ? CU_TENSOR_MAP_SWIZZLE_32B
                               : es == 2 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B;
-  CUresult r = fn(map, dt, 3, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
-                  CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) {
-    set_last_cuda_error(static_cast<int>(r));
-    return SCALIFY_ERR_CUDA;
-  }
-  return SCALIFY_OK;
+  return encode_tiled_cached(g_map_cache, fn, map, dt, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+                             CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
 }
 
 size_t matmul_splitk_ws_bytes(int64_t rows, int64_t cols) {
@@ -916,9 +1013,10 @@ static int launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, co
                           cudaStream_t st) {
   using C = GemmCfg<NCTA>;
   auto kernel = GemmKernelOf<OUT, NCTA, SPEC, BIAS, NOY>::get();
-  static bool attr_done = false;
-  static int max_clusters = 0;
-  if (!attr_done) {
+  // per device: the dynamic shared-memory limit of this kernel and the number of CTA pairs that fit the GPU
+  static DeviceOnce once;
+  int max_clusters = 0;
+  int rc_once = device_once(once, &max_clusters, [&](int* clusters) {
     SCALIFY_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(C::kSmem)));
     if (NCTA == 2) {
       cudaLaunchConfig_t qc = {};
@@ -932,11 +1030,12 @@ static int launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, co
       qc.numAttrs = 1;
       int n = 0;
       SCALIFY_CUDA_TRY(cudaOccupancyMaxActiveClusters(&n, kernel, &qc));
-      if (n < 1) return SCALIFY_ERR_UNSUPPORTED;
-      max_clusters = n;
+      if (n < 1) return int(SCALIFY_ERR_UNSUPPORTED);
+      *clusters = n;
     }
-    attr_done = true;
-  }
+    return int(SCALIFY_OK);
+  });
+  if (rc_once) return rc_once;
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attrs[2];
   attrs[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // the prologue may overlap the grid before it
@@ -1115,14 +1214,9 @@ static int make_map_sf(CUtensorMap* map, const void* ptr, uint64_t n_tiles) {
   cuuint64_t strides[2] = {512, 512 * n_tiles};
   cuuint32_t box[3] = {128u, 1u, 1u};
   cuuint32_t estr[3] = {1u, 1u, 1u};
-  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<void*>(ptr), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) {
-    set_last_cuda_error(static_cast<int>(r));
-    return SCALIFY_ERR_CUDA;
-  }
-  return SCALIFY_OK;
+  return encode_tiled_cached(g_map_cache, fn, map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<void*>(ptr), dims, strides,
+                             box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                             CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
 }
 
 template <int OUT, int NCTA>
@@ -1131,12 +1225,12 @@ static int launch_mx_variant(const CUtensorMap& map_a, const CUtensorMap& map_b,
                              long long tiles, cudaStream_t st) {
   using C = GemmCfg<NCTA, true>;
   auto kernel = mx_matmul_kernel<OUT, NCTA>;
-  static bool attr_done = false;
-  static int max_clusters = 0;
   cudaLaunchAttribute attrs[1];
   attrs[0].id = cudaLaunchAttributeClusterDimension;
   attrs[0].val.clusterDim.x = 2; attrs[0].val.clusterDim.y = 1; attrs[0].val.clusterDim.z = 1;
-  if (!attr_done) {
+  static DeviceOnce once;  // per device, like the per-tensor kernel
+  int max_clusters = 0;
+  int rc_once = device_once(once, &max_clusters, [&](int* clusters) {
     SCALIFY_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(C::kSmem)));
     if (NCTA == 2) {
       cudaLaunchConfig_t qc = {};
@@ -1147,11 +1241,12 @@ static int launch_mx_variant(const CUtensorMap& map_a, const CUtensorMap& map_b,
       qc.numAttrs = 1;
       int n = 0;
       SCALIFY_CUDA_TRY(cudaOccupancyMaxActiveClusters(&n, kernel, &qc));
-      if (n < 1) return SCALIFY_ERR_UNSUPPORTED;
-      max_clusters = n;
+      if (n < 1) return int(SCALIFY_ERR_UNSUPPORTED);
+      *clusters = n;
     }
-    attr_done = true;
-  }
+    return int(SCALIFY_OK);
+  });
+  if (rc_once) return rc_once;
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute run_attrs[2];
   run_attrs[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // the prologue may overlap the grid before it

@@ -878,6 +878,17 @@ int scalify_debug_expire_wait(void* workspace, size_t workspace_bytes, uint32_t 
                             static_cast<cudaStream_t>(stream));
 }
 
+int scalify_debug_host_state_selftest(void) { return host_state_selftest(); }
+
+int scalify_debug_tensor_map_cache(uint64_t* hits, uint64_t* misses) {
+  if (!hits || !misses) return SCALIFY_ERR_NULL;
+  unsigned long long h = 0, m = 0;
+  map_cache_counters(&h, &m);
+  *hits = h;
+  *misses = m;
+  return SCALIFY_OK;
+}
+
 int scalify_debug_layernorm_plan(int64_t R, int64_t d, int x_dtype, int backward, int32_t plan[4]) {
   if (!plan) return SCALIFY_ERR_NULL;
   if (!is_wide(x_dtype)) return SCALIFY_ERR_DTYPE;

@@ -9,6 +9,8 @@
 #include <cuda_fp8.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "scalify.h"
 
 namespace scalify {
@@ -63,6 +65,36 @@ int check_array(const scalify_array* a);
 int sm_count();
 void set_last_cuda_error(int e);
 int cuda_fail(cudaError_t e);
+
+// One-time set-up of a kernel PER DEVICE.  Function attributes (the dynamic shared-memory limit) and occupancy
+// figures belong to a device, not to the process: a process that uses the library on a second GPU has to set
+// them again there.  `fn(int* value)` runs once per device, with that device current, under a lock (so two host
+// threads cannot both believe the other did it); `value` is what it computed for that device (e.g. the number
+// of co-resident clusters), handed back on every later call.
+constexpr int kMaxDevices = 64;
+struct DeviceOnce {
+  std::mutex mu;
+  bool done[kMaxDevices] = {};
+  int value[kMaxDevices] = {};
+};
+template <class Fn>
+inline int device_once_at(DeviceOnce& o, int dev, int* value_out, Fn fn) {
+  if (dev < 0 || dev >= kMaxDevices) return SCALIFY_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(o.mu);
+  if (!o.done[dev]) {
+    int rc = fn(&o.value[dev]);
+    if (rc) return rc;
+    o.done[dev] = true;
+  }
+  if (value_out) *value_out = o.value[dev];
+  return SCALIFY_OK;
+}
+template <class Fn>
+inline int device_once(DeviceOnce& o, int* value_out, Fn fn) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return SCALIFY_ERR_CUDA;
+  return device_once_at(o, dev, value_out, fn);
+}
 
 #define SCALIFY_CUDA_TRY(expr)                               \
   do {                                                       \

@@ -99,6 +99,8 @@ struct MatmulArgs {
 };
 size_t matmul_ws_bytes(int64_t rows, int64_t cols);
 size_t matmul_splitk_ws_bytes(int64_t rows, int64_t cols);
+int host_state_selftest();
+void map_cache_counters(unsigned long long* hits, unsigned long long* misses);
 int launch_expire_wait(void* ws, unsigned long long limit_ns, uint32_t* waited_us, cudaStream_t st);
 int launch_scaled_matmul(const MatmulArgs& a, void* ws, size_t ws_bytes, cudaStream_t st);
 // Block-scaled matmul: A [M,K], B [N,K] FP8 row-major (dense), exponents in 128-row x 4-block tiles.

@@ -555,11 +555,12 @@ int launch_cross_entropy(const void* logits, int l_dt, long long ld, int n_class
     const int grid2 = static_cast<int>(n < cap2 ? n : cap2);
     SCALIFY_DISPATCH_WIDE(l_dt, LDT, SCALIFY_DISPATCH_DTYPE(g_dt, GDT, {
       auto kernel = cross_entropy_smem_kernel<LDT, GDT>;
-      static bool attr_done = false;
-      if (!attr_done) {
+      static DeviceOnce once;  // (one per instantiation: the attribute belongs to this kernel on this device)
+      int rc_once = device_once(once, nullptr, [&](int*) {
         SCALIFY_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kCeSmemMax));
-        attr_done = true;
-      }
+        return int(SCALIFY_OK);
+      });
+      if (rc_once) return rc_once;
       kernel<<<grid2, kCeThreads, static_cast<size_t>(row_smem), st>>>(logits, ld, n_classes, targets, n, l_scale, dlogits, rem,
                                                                row_loss, v.status);
     }));

@@ -134,3 +134,12 @@ def test_validation_rejects_bad_arguments_on_the_host():
                                         1 << 20, None) == -3
     assert L.scalify_scaled_matmul_bias(R(A), 0, R(B), 0, R(_arr(1 << 22, sc.E4M3, (256,))), R(Yb), 0, None, 1 << 21,
                                         1 << 20, None) == -2
+
+
+def test_per_device_set_up_and_tensor_map_cache_selftest():
+    """Host-side state: every kernel's one-time set-up is kept per device (a second GPU in the same process gets
+    its own), and encoded tensor maps are cached by pointer / extents / strides / box.  The library's self-test
+    drives both with made-up device numbers and a stand-in encoder; 0 means every check held."""
+    assert sc.lib().scalify_debug_host_state_selftest() == 0
+    c = sc.scalify_debug_tensor_map_cache()
+    assert c["hits"] >= 0 and c["misses"] >= 0
