@@ -362,6 +362,14 @@ int scalify_debug_expire_wait(void* workspace, size_t workspace_bytes, uint32_t 
                               void* stream);
 
 /*
+ * Diagnostic (no counterpart in the paper): y[i] = x[i] rounded to the nearest BF16 value (ties to even), as
+ * fp32, computed by the routine the fused attention kernels use for the scores' BF16 intermediate (three fp32
+ * operations instead of a conversion).  x, y: device fp32 arrays of n elements.  Lets a test compare that
+ * routine with the definition over any set of bit patterns.
+ */
+int scalify_debug_bf16_round(const float* x, float* y, int64_t n, void* stream);
+
+/*
  * Diagnostics of the library's host-side state (no counterpart in the paper; host only, no GPU needed).
  * The library keeps two things between calls: the one-time set-up of each kernel PER DEVICE (dynamic
  * shared-memory limit, co-resident cluster count) and a cache of encoded TMA tensor maps keyed by pointer,

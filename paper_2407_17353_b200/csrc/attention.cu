@@ -18,6 +18,14 @@
 // (moved to the new maximum whenever a 32-key chunk raises it); sweep B recomputes Q K^T, forms p = exp(s - m) / l, rounds it to
 // E4M3 and accumulates P V in TMEM.  The probabilities are therefore the same normalised values
 // the unfused path quantises, and O needs no rescaling.  Cost: the Q K^T work twice.
+// The tensor core stays AHEAD of the row threads.  A row thread hands the score buffer back as soon as its
+// last chunk of the block is in registers, and the issuing thread computes the scores of block b+1 BEFORE it
+// waits for the probabilities of block b; two probability tiles in shared memory let the rows write block b+1
+// while P V of block b runs; K / V tiles travel through a three-deep ring, fetched two blocks ahead.  (When the
+// two sides took turns - one probability tile, buffer handed back after the arithmetic - 96 heads x 1024 x 64
+// took 71 us; 57 us with the cheaper BF16 rounding below, 50 us with the hand-offs out of the way.  A form
+// with ONE CTA of 16 row warps per SM and two score buffers in TMEM measured 67 us: two CTAs that drift apart
+// fill each other's exp2 / conversion phases, sixteen warps released by the same barrier do not.)
 // TMEM: 128 columns of scores + 64 columns of O (256 allocated, so two CTAs share an SM).
 // Every mbarrier wait is bounded; on expiry the CTA records SCALIFY_DEV_TIMEOUT and leaves.
 #include <cuda.h>
@@ -35,8 +43,10 @@ constexpr int kAttSmWarps = 8;   // softmax warps: two per TMEM lane quarter, ea
 constexpr int kAttThreads = 32 * (kAttSmWarps + 1);
 constexpr int kAttTmemCols = 256;
 constexpr uint32_t kAttOCol = 128;
+constexpr int kAttKvStages = 3;
 constexpr int kAttTileBytes = kAttK * kAttHd;  // 8 KB: a Q, K or V tile
-constexpr size_t kAttSmem = size_t(kAttTileBytes) * 5 /*Q, 2 x K, 2 x V*/ + kAttQ * kAttK /*P*/ + 1024 + 256;
+constexpr size_t kAttSmem = size_t(kAttTileBytes) * (1 + 2 * kAttKvStages) /*Q, K ring, V ring*/ +
+                            2 * kAttQ * kAttK /*two P tiles*/ + 1024 + 256;
 
 struct AttParams {
   int heads, h_inner, Tq, Tk, q_blocks;   // heads = batch x h_inner
@@ -81,15 +91,15 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (base - raw);
   const uint32_t smem_q = base;
-  const uint32_t smem_k = base + kAttTileBytes;          // 2 slots
-  const uint32_t smem_v = base + 3 * kAttTileBytes;      // 2 slots
-  const uint32_t smem_p = base + 5 * kAttTileBytes;      // 16 KB, 1024-byte aligned
-  uint8_t* p_tile = smem + 5 * kAttTileBytes;
-  uint8_t* bar_mem = p_tile + kAttQ * kAttK;
-  const uint32_t bars = smem_p + kAttQ * kAttK;
-  const uint32_t q_full = bars, kv_full = bars + 8 /*2*/, kv_empty = bars + 24 /*2*/, s_full = bars + 40,
-                 s_empty = bars + 48, p_full = bars + 56, p_empty = bars + 64, o_full = bars + 72;
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bar_mem + 80);
+  const uint32_t smem_k = base + kAttTileBytes;                              // kAttKvStages slots
+  const uint32_t smem_v = base + (1 + kAttKvStages) * kAttTileBytes;         // kAttKvStages slots
+  const uint32_t smem_p = base + (1 + 2 * kAttKvStages) * kAttTileBytes;     // 2 x 16 KB, 1024-byte aligned
+  uint8_t* p_tiles = smem + (1 + 2 * kAttKvStages) * kAttTileBytes;
+  uint8_t* bar_mem = p_tiles + 2 * kAttQ * kAttK;
+  const uint32_t bars = smem_p + 2 * kAttQ * kAttK;
+  const uint32_t q_full = bars, kv_full = bars + 8 /*3*/, kv_empty = bars + 32 /*3*/, s_full = bars + 56,
+                 s_empty = bars + 72, p_full = bars + 88 /*2*/, p_empty = bars + 104 /*2*/, o_full = bars + 120;
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bar_mem + 128);
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -104,11 +114,10 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
 
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
-    for (int s = 0; s < 2; ++s) { mbar_init(kv_full + 8 * s, 1); mbar_init(kv_empty + 8 * s, 1); }
+    for (int s = 0; s < kAttKvStages; ++s) { mbar_init(kv_full + 8 * s, 1); mbar_init(kv_empty + 8 * s, 1); }
     mbar_init(s_full, 1);
     mbar_init(s_empty, kAttSmWarps);
-    mbar_init(p_full, kAttSmWarps);
-    mbar_init(p_empty, 1);
+    for (int s = 0; s < 2; ++s) { mbar_init(p_full + 8 * s, kAttSmWarps); mbar_init(p_empty + 8 * s, 1); }
     mbar_init(o_full, 1);
     *abort_flag = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -131,12 +140,13 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_q)) : "memory");
       asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_k)) : "memory");
       asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_v)) : "memory");
-      const int n_it = 2 * n_kb;  // sweep A (K only), sweep B (K and V)
-      auto issue_load = [&](int it) {
-        const int slot = it & 1, use = it >> 1;
+      const int n_it = 2 * n_kb;  // iteration j: sweep A block j (K only), then sweep B block j - n_kb (K and V)
+      // K (and V) tiles of iteration j into ring slot j % kAttKvStages
+      auto issue_load = [&](int j) {
+        const int slot = j % kAttKvStages, use = j / kAttKvStages;
         if (use >= 1 && !mbar_wait(kv_empty + 8 * slot, (use - 1) & 1, abort_flag)) { timed_out = true; return; }
-        const bool sweep_b = it >= n_kb;
-        const int kb = sweep_b ? it - n_kb : it;
+        const bool sweep_b = j >= n_kb;
+        const int kb = sweep_b ? j - n_kb : j;
         const uint32_t fb = kv_full + 8 * slot;
         mbar_expect_tx(fb, sweep_b ? 2 * kAttTileBytes : kAttTileBytes);
         tma_load_4d(smem_k + slot * kAttTileBytes, &map_k, fb, 0, kb * kAttK, hh, bb);
@@ -145,35 +155,41 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       mbar_expect_tx(q_full, kAttTileBytes);
       tma_load_4d(smem_q, &map_q, q_full, 0, q0, hh, bb);
       issue_load(0);
+      if (!timed_out && n_it > 1) issue_load(1);
       if (!timed_out && !mbar_wait(q_full, 0u, abort_flag)) timed_out = true;
       const uint64_t q_desc = make_smem_desc_sw64(smem_q, 512u);
-      const uint64_t p_desc = make_smem_desc(smem_p, 0u, 1024u);
-      for (int it = 0; it < n_it && !timed_out; ++it) {
-        if (it + 1 < n_it) { issue_load(it + 1); if (timed_out) break; }
-        const int slot = it & 1;
-        if (!mbar_wait(kv_full + 8 * slot, (it >> 1) & 1, abort_flag)) { timed_out = true; break; }
-        // the score block in TMEM is free once the softmax threads have read the previous one
-        if (it >= 1 && !mbar_wait(s_empty, (it - 1) & 1, abort_flag)) { timed_out = true; break; }
+      // scores of iteration j (the score buffer is free once the rows have taken iteration j - 1 to registers)
+      auto issue_scores = [&](int j) {
+        const int slot = j % kAttKvStages;
+        if (!mbar_wait(kv_full + 8 * slot, (j / kAttKvStages) & 1, abort_flag)) { timed_out = true; return; }
+        if (j >= 1 && !mbar_wait(s_empty, (j - 1) & 1, abort_flag)) { timed_out = true; return; }
         tc_fence_after();
         const uint64_t k_desc = make_smem_desc_sw64(smem_k + slot * kAttTileBytes, 512u);
 #pragma unroll
         for (int k = 0; k < kAttHd / 32; ++k)  // K = 32 bytes per MMA: +32 B on both K-major operands
-          umma_f8(tmem_base, q_desc + static_cast<uint64_t>(k * 2), k_desc + static_cast<uint64_t>(k * 2), p.idesc_s,
-                  k != 0 ? 1u : 0u);
+          umma_f8(tmem_base, q_desc + static_cast<uint64_t>(k * 2), k_desc + static_cast<uint64_t>(k * 2),
+                  p.idesc_s, k != 0 ? 1u : 0u);
         umma_commit(s_full);
-        if (it < n_kb) {
-          umma_commit(kv_empty + 8 * slot);  // sweep A: the K tile is free after Q K^T
-        } else {
-          const int b = it - n_kb;
-          if (!mbar_wait(p_full, b & 1, abort_flag)) { timed_out = true; break; }
+        if (j < n_kb) umma_commit(kv_empty + 8 * slot);  // sweep A: the K tile is free after Q K^T
+      };
+      if (!timed_out) issue_scores(0);
+      for (int it = 0; it < n_it && !timed_out; ++it) {
+        // stay ahead of the rows: tiles two iterations ahead, scores one iteration ahead
+        if (it + 2 < n_it) { issue_load(it + 2); if (timed_out) break; }
+        if (it + 1 < n_it) { issue_scores(it + 1); if (timed_out) break; }
+        if (it >= n_kb) {
+          const int b = it - n_kb, pb = b & 1, slot = it % kAttKvStages;
+          if (!mbar_wait(p_full + 8 * pb, (b >> 1) & 1, abort_flag)) { timed_out = true; break; }
           tc_fence_after();
-          // V tile [128 keys][64 B]: the B operand in MN-major form, 8-key atoms 512 B apart, 32 keys per MMA
+          // P tile [128 queries][128 B of keys], K-major; V tile [128 keys][64 B]: the B operand in MN-major form,
+          // 8-key atoms 512 B apart, 32 keys per MMA
+          const uint64_t p_desc = make_smem_desc(smem_p + pb * (kAttQ * kAttK), 0u, 1024u);
           const uint64_t v_desc = make_smem_desc_sw64(smem_v + slot * kAttTileBytes, 512u);
 #pragma unroll
           for (int k = 0; k < kAttK / 32; ++k)
             umma_f8(tmem_base + kAttOCol, p_desc + static_cast<uint64_t>(k * 2),
                     v_desc + static_cast<uint64_t>(k * (32 * kAttHd / 16)), p.idesc_pv, (b | k) != 0 ? 1u : 0u);
-          umma_commit(p_empty);
+          umma_commit(p_empty + 8 * pb);
           umma_commit(kv_empty + 8 * slot);
         }
       }
@@ -199,16 +215,22 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     // x = data component of the score, rounded to BF16 like the unfused intermediate, in units of log2(e).
     // Dividing by kf(hd) only shifts the exponent, so it commutes with the rounding and is folded into sc3.
     const float sc3 = sc2 * p.inv_kf_hd;
-    // The BF16 rounding is done with integer arithmetic (round to nearest even on the upper 16 bits; the
-    // scores are finite): the conversion unit is shared with exp2 and is this kernel's busiest pipe.
-    auto bf16_rne = [](uint32_t b) { return __uint_as_float((b + 0x7FFFu + ((b >> 16) & 1u)) & 0xFFFF0000u); };
+    // The BF16 rounding (round to nearest even, as the unfused intermediate is rounded) runs on the fp32 pipe
+    // (bf16_round_f32): the conversion unit is shared with exp2, and the integer form (four half-rate
+    // instructions per element) made the integer pipe this kernel's busiest.
+    const float2 sc3_2 = make_float2(sc3, sc3);
+    // x[e] = rounded score times sc3 for the visible keys of a 32-key chunk, -inf for the others
     auto chunk_scores = [&](const uint32_t* acc_bits, int j0, float* x) {
-      if (j0 + 32 <= lim) {  // every key of the chunk is visible to this row
 #pragma unroll
-        for (int e = 0; e < 32; ++e) x[e] = bf16_rne(acc_bits[e]) * sc3;
-      } else {
+      for (int e = 0; e < 32; e += 2) {
+        const float2 v = __fmul2_rn(make_float2(bf16_round_f32(__uint_as_float(acc_bits[e])),
+                                                bf16_round_f32(__uint_as_float(acc_bits[e + 1]))), sc3_2);
+        x[e] = v.x;
+        x[e + 1] = v.y;
+      }
+      if (j0 + 32 > lim) {  // the chunk crosses the end of this row's visible keys
 #pragma unroll
-        for (int e = 0; e < 32; ++e) x[e] = (j0 + e < lim) ? bf16_rne(acc_bits[e]) * sc3 : -INFINITY;
+        for (int e = 0; e < 32; ++e) x[e] = (j0 + e < lim) ? x[e] : -INFINITY;
       }
     };
     int it = 0;
@@ -221,6 +243,14 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       for (int c = c_first; c < c_first + kChunks; ++c) {
         tmem_ld32(t_row + c * 32, acc);
         tmem_ld_wait();
+        if (c == c_first + kChunks - 1) {
+          // the score block is in registers: hand the TMEM buffer back now, so that the tensor core computes the
+          // next block's scores while this one is worked on (taking both chunks to registers first, to hand it
+          // back a chunk earlier, costs a second CTA per SM its registers: 83 us against 54 us)
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(s_empty);
+        }
         // one pass per 32-key chunk: chunk maximum, then the running sum is moved to the new maximum
         float x[32];
         chunk_scores(acc, kb * kAttK + c * 32, x);
@@ -229,10 +259,14 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         for (int e = 0; e < 32; ++e) cm4[e & 3] = fmaxf(cm4[e & 3], x[e]);
         const float m_new = fmaxf(m, fmaxf(fmaxf(cm4[0], cm4[1]), fmaxf(cm4[2], cm4[3])));
         if (m_new > -INFINITY) {
-          float add4[4] = {0.f, 0.f, 0.f, 0.f};
+          const float2 nm2 = make_float2(-m_new, -m_new);
+          float2 add2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
 #pragma unroll
-          for (int e = 0; e < 32; ++e) add4[e & 3] += exp2_neg(x[e] - m_new);  // 2^-inf = 0 for masked keys
-          l = l * exp2_neg(m - m_new) + ((add4[0] + add4[1]) + (add4[2] + add4[3]));  // and while nothing was seen
+          for (int e = 0; e < 32; e += 2) {
+            const float2 a = __fadd2_rn(make_float2(x[e], x[e + 1]), nm2);
+            add2[(e >> 1) & 1] = __fadd2_rn(add2[(e >> 1) & 1], make_float2(exp2_neg(a.x), exp2_neg(a.y)));  // 2^-inf = 0 for masked keys
+          }
+          l = l * exp2_neg(m - m_new) + ((add2[0].x + add2[0].y) + (add2[1].x + add2[1].y));  // and while nothing was seen
           m = m_new;
         }
         if (p.S_dump && i < p.Tq) {
@@ -249,12 +283,9 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           }
         }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(s_empty);
     }
     // the two threads of a row (one per half of the key columns) combine their maxima and sums
-    float2* part = reinterpret_cast<float2*>(p_tile);  // [2][128], the P tile is not in use yet
+    float2* part = reinterpret_cast<float2*>(p_tiles);  // [2][128], the P tiles are not in use yet
     part[half * kAttQ + r] = make_float2(m, l);
     asm volatile("bar.sync 1, %0;" ::"n"(32 * kAttSmWarps) : "memory");
     {
@@ -268,21 +299,36 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     for (int kb = 0; kb < n_kb && !timed_out; ++kb, ++it) {
       if (!mbar_wait(s_full, it & 1, abort_flag)) { timed_out = true; break; }
       tc_fence_after();
-      // the previous block's P V must have read the tile before it is overwritten
-      if (kb >= 1 && !mbar_wait(p_empty, (kb - 1) & 1, abort_flag)) { timed_out = true; break; }
+      // P V of the block that used this probability tile last (two blocks ago) must have read it
+      const int pb = kb & 1;
+      if (kb >= 2 && !mbar_wait(p_empty + 8 * pb, ((kb >> 1) - 1) & 1, abort_flag)) { timed_out = true; break; }
       uint32_t acc[32];
 #pragma unroll 1
       for (int c = c_first; c < c_first + kChunks; ++c) {
         tmem_ld32(t_row + c * 32, acc);
         tmem_ld_wait();
+        if (c == c_first + kChunks - 1) {
+          // the score block is in registers: hand the TMEM buffer back now, so that the tensor core computes the
+          // next block's scores while this one is worked on (taking both chunks to registers first, to hand it
+          // back a chunk earlier, costs a second CTA per SM its registers: 83 us against 54 us)
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(s_empty);
+        }
         float pr[32];
         chunk_scores(acc, kb * kAttK + c * 32, pr);
+        const float2 nm2 = make_float2(-m, -m), il2 = make_float2(inv_l, inv_l);
 #pragma unroll
-        for (int e = 0; e < 32; ++e) pr[e] = exp2_neg(pr[e] - m) * inv_l;
+        for (int e = 0; e < 32; e += 2) {
+          const float2 a = __fadd2_rn(make_float2(pr[e], pr[e + 1]), nm2);
+          const float2 q = __fmul2_rn(make_float2(exp2_neg(a.x), exp2_neg(a.y)), il2);
+          pr[e] = q.x;
+          pr[e + 1] = q.y;
+        }
         uint32_t o[8];
         encode_vec<SCALIFY_E4M3, 32>(pr, o);
         // row r of the tile: 128 bytes = eight 16-byte pieces, piece index XOR (r % 8) (128-byte swizzle)
-        uint4* row = reinterpret_cast<uint4*>(p_tile + r * 128);
+        uint4* row = reinterpret_cast<uint4*>(p_tiles + pb * (kAttQ * kAttK) + r * 128);
         row[(2 * c) ^ (r & 7)] = make_uint4(o[0], o[1], o[2], o[3]);
         row[(2 * c + 1) ^ (r & 7)] = make_uint4(o[4], o[5], o[6], o[7]);
         if (p.P_dump && i < p.Tq) {
@@ -297,7 +343,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       fence_async_smem();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) { mbar_arrive(s_empty); mbar_arrive(p_full); }
+      if (lane == 0) mbar_arrive(p_full + 8 * pb);
     }
     // O: 64 fp32 columns of this row
     if (!timed_out && mbar_wait(o_full, 0u, abort_flag)) {

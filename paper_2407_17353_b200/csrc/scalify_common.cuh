@@ -302,6 +302,20 @@ __device__ __forceinline__ float round_through(float x) {
   }
 }
 
+// fp32 -> the nearest BF16 value (ties to even), returned as fp32, computed on the fp32 pipe: Veltkamp's split
+// with the constant 2^16 + 1,   c = x (2^16 + 1);  hi = c - (c - x),   leaves exactly the upper 8 significand
+// bits of x rounded to nearest even.  Exact for every normal x below 2^111 (checked on the GPU against the
+// integer formula for all 2^32 bit patterns; zero stays zero; subnormal inputs are not covered).  It replaces
+// four half-rate integer instructions, or a conversion instruction plus unpacking, in the attention kernels.
+// The three operations must remain three separately rounded operations: the scalar intrinsics are documented
+// never to be contracted into a multiply-add.  (The two-wide forms are NOT safe here: the same sequence written
+// with mul.rn.f32x2 / sub.rn.f32x2 came out fused on this toolchain and returned x unrounded.)
+__device__ __forceinline__ float bf16_round_f32(float x) {
+  const float c = __fmul_rn(x, 65537.0f);
+  const float d = __fsub_rn(c, x);
+  return __fsub_rn(c, d);
+}
+
 // scalar load/store for ragged tails
 template <int DT>
 __device__ __forceinline__ float load_elem(const void* p, int64_t i) {

@@ -696,4 +696,18 @@ int launch_colsum(const void* X, int x_dt, long long ld, long long R, long long 
   return SCALIFY_OK;
 }
 
+// Diagnostic: the fp32-pipe BF16 rounding used inside the attention kernels, applied to an array
+__global__ void __launch_bounds__(256) bf16_round_kernel(const float* __restrict__ x, float* __restrict__ y, long long n) {
+  asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
+  for (long long i = static_cast<long long>(blockIdx.x) * 256 + threadIdx.x; i < n; i += static_cast<long long>(gridDim.x) * 256)
+    y[i] = bf16_round_f32(x[i]);
+}
+
+int launch_bf16_round(const float* x, float* y, long long n, cudaStream_t st) {
+  const long long blocks = (n + 255) / 256;
+  bf16_round_kernel<<<static_cast<unsigned>(blocks < 148 * 16 ? blocks : 148 * 16), 256, 0, st>>>(x, y, n);
+  SCALIFY_CUDA_TRY(cudaGetLastError());
+  return SCALIFY_OK;
+}
+
 }  // namespace scalify

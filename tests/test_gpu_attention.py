@@ -166,3 +166,24 @@ def test_batch_of_sequences_as_a_4d_view_equals_one_call_per_sequence():
     assert s_one == s_per
     for a, b in zip(one, per):
         assert np.array_equal(a, b)
+
+
+def test_fp32_pipe_bf16_rounding_is_round_to_nearest_even():
+    """The attention kernels round the scores (and dP) to BF16 with three fp32 operations instead of a
+    conversion.  That routine against the definition (torch's CPU cast): every upper half-word with the tie
+    pattern and its two neighbours below it, and sixteen million random bit patterns (normal numbers below 2^111,
+    zero included; the products of FP8 operands are far inside that range)."""
+    g = torch.Generator().manual_seed(7)
+    upper = torch.arange(65536, dtype=torch.int64) << 16
+    pats = [upper | low for low in (0x8000, 0x7FFF, 0x8001, 0x0000, 0xFFFF, 0x0001)]
+    pats.append(torch.randint(0, 2 ** 32, (1 << 24,), generator=g, dtype=torch.int64))
+    bits = torch.cat(pats)
+    e = (bits >> 23) & 0xFF
+    bits = bits[((e > 0) & (e < 0xFF - 20)) | ((bits & 0x7FFFFFFF) == 0)]
+    x = (bits & 0xFFFFFFFF).to(torch.uint32).view(torch.float32).contiguous()
+    want = x.to(torch.bfloat16).to(torch.float32)
+    xd = x.cuda()
+    yd = torch.empty_like(xd)
+    sc.scalify_debug_bf16_round(xd, yd)
+    got = yd.cpu()
+    assert torch.equal(got.view(torch.int32), want.view(torch.int32))
