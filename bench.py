@@ -723,7 +723,7 @@ def main():
 
     # Block-scaled variant (E8M0 exponent per 32 elements of K): quantise both BF16 operands, then the
     # block-scaled GEMM with fused AMAX, BF16 out
-    mx_q_ms = mx_mm_ms = float("nan")
+    mx_q_ms = mx_mm_ms = mx_qt_ms = mx_mmt_ms = float("nan")
     if not args.no_next:
         Xa = sc.ScaledTensor.make(rnd((N_GEMM, N_GEMM), torch.bfloat16, 21), 1.0)
         Xb = sc.ScaledTensor.make(rnd((N_GEMM, N_GEMM), torch.bfloat16, 22), 1.0)
@@ -735,9 +735,19 @@ def main():
 
         def mx_mm():
             sc.scalify_mx_matmul(Am, Bm, Y, ws_mm, stat=sc.STAT_AMAX)
+
+        # the weight-gradient form: both operands stored with the contraction axis slow ([K, rows])
+        Amt, Bmt = (sc.MxTensor(N_GEMM, N_GEMM, device=dev, transposed=True) for _ in range(2))
+
+        def mx_quant_t():
+            sc.scalify_mx_quantize(Xa, Amt)
+            sc.scalify_mx_quantize(Xb, Bmt)
+
+        def mx_mm_t():
+            sc.scalify_mx_matmul(Amt, Bmt, Y, ws_mm, stat=sc.STAT_AMAX)
         x_iters = max(3, min(K, 20))
         times = []
-        for fn in (mx_quant, mx_mm):
+        for fn in (mx_quant, mx_mm, mx_quant_t, mx_mm_t):
             for _ in range(3):
                 fn()
             barrier()
@@ -748,8 +758,8 @@ def main():
             x1.record()
             barrier()
             times.append(x0.elapsed_time(x1) / x_iters)
-        mx_q_ms, mx_mm_ms = times
-        del Xa, Xb, Am, Bm
+        mx_q_ms, mx_mm_ms, mx_qt_ms, mx_mmt_ms = times
+        del Xa, Xb, Am, Bm, Amt, Bmt
 
     # Fused attention forward on the config-5 shape: 8 sequences x 12 heads, 1024 tokens, head dimension 64
     att_ms = att_bwd_ms = float("nan")
@@ -940,6 +950,11 @@ def main():
         {"row": "f3 (next, own loop) block-scaled GEMM 8192^3 (tcgen05 kind::mxf8f6f4.block_scale, two-CTA tiles), "
                 "BF16 out + fused AMAX", "ms": round(float(mx_mm_ms), 4),
          "TFLOP/s": round(flops / (mx_mm_ms * 1e-3) / 1e12, 1)},
+        row("f3 (next, own loop) block-scale quantisation, transposed form: operands stored [K, rows], blocks of 32 "
+            "down the columns (3.03 B/elem)", mx_qt_ms, 2 * (3 * N_GEMM * N_GEMM + N_GEMM * N_GEMM // 32)),
+        {"row": "f3 (next, own loop) block-scaled GEMM 8192^3, both operands in the transposed (MN-major) form of "
+                "the gradient products", "ms": round(float(mx_mmt_ms), 4),
+         "TFLOP/s": round(flops / (mx_mmt_ms * 1e-3) / 1e12, 1)},
         {"row": "f4 (next, own loop) fused causal attention forward, 96 heads x 1024 tokens x 64 (scores and "
                 "probabilities never leave the chip)", "ms": round(float(att_ms), 4),
          "TFLOP/s": round(2.0 * ATT_H * ATT_T * ATT_T * ATT_HD / (att_ms * 1e-3) / 1e12, 1),

@@ -515,6 +515,10 @@ typedef struct scalify_mx_array {
   int64_t K;
   uint8_t* sf;    /* E8M0 exponents, tiled as described above */
   float* scale;   /* one fp32 power of two, or NULL (scale 1) */
+  int32_t transposed; /* 0: data [rows, K].  1: data stored [K, rows] (row-major, `rows` contiguous, rows a
+                         multiple of 16): the form of an operand whose contraction dimension is the slow one
+                         of the forward tensor (weight and activation gradients); a block is then 32
+                         consecutive ROWS of the storage at one column.  The exponent tiles are the same. */
 } scalify_mx_array;
 
 size_t scalify_mx_sf_bytes(int64_t rows, int64_t K);
@@ -528,6 +532,9 @@ size_t scalify_mx_sf_bytes(int64_t rows, int64_t K);
  * x * 2^-e, saturating.  A block whose maximum is zero, infinite or NaN gets
  * e = 0.  Y_s = X_s.  `status`: optional DEVICE word that receives
  * SCALIFY_DEV_BAD_SCALE.  Errors: NULL, DTYPE, SHAPE (K % 128), ALIGNMENT.
+ * With Y->transposed, X is [K, rows] like the data it is quantised into, and
+ * the blocks run down the columns; the values and exponents are those of the
+ * plain form applied to the transposed matrix.
  */
 int scalify_mx_quantize(const scalify_array* X, scalify_mx_array* Y, uint32_t* status, void* stream);
 
@@ -536,7 +543,9 @@ int scalify_mx_quantize(const scalify_array* X, scalify_mx_array* Y, uint32_t* s
  * tensor-wide scales:  Y_s = A_s * B_s * kf(K),
  *   Y_d[i,j] = (sum_k A_d[i,k] 2^(Ea[i,k/32]-127) * B_d[j,k] 2^(Eb[j,k/32]-127)) / kf(K)
  * with fp32 accumulation on the tensor cores (tcgen05 kind::mxf8f6f4 with the
- * exponents in tensor memory).  A is [M,K], B is [N,K]; Y [M,N] is F16, BF16
+ * exponents in tensor memory).  A is [M,K], B is [N,K] (either may be stored
+ * transposed, see scalify_mx_array: the tensor cores then read it MN-major and
+ * no transposed copy is made); Y [M,N] is F16, BF16
  * or F32 (row stride stride[0]).  stat: NONE, AMAX or L2 of the stored Y, left
  * in the workspace's statistic word as by scalify_scaled_matmul.  Workspace:
  * SCALIFY_OP_MATMUL (M, N).

@@ -46,7 +46,7 @@ class scalify_array(ctypes.Structure):
 
 class scalify_mx_array(ctypes.Structure):
     _fields_ = [("data", ctypes.c_void_p), ("dtype", ctypes.c_int32), ("rows", ctypes.c_int64), ("K", ctypes.c_int64),
-                ("sf", ctypes.c_void_p), ("scale", ctypes.c_void_p)]
+                ("sf", ctypes.c_void_p), ("scale", ctypes.c_void_p), ("transposed", ctypes.c_int32)]
 
 
 _lib = None
@@ -447,14 +447,16 @@ class MxTensor:
     """Block-scaled array: FP8 data [rows, K], E8M0 exponents per 32 elements of K in the tile order the
     tensor cores consume (see ``include/scalify.h``), and the tensor-wide fp32 power-of-two scale."""
 
-    def __init__(self, rows: int, K: int, dtype: torch.dtype = torch.float8_e4m3fn, device="cuda"):
+    def __init__(self, rows: int, K: int, dtype: torch.dtype = torch.float8_e4m3fn, device="cuda", transposed=False):
+        """transposed: the data are stored [K, rows] (blocks of 32 run down the columns); rows % 16 == 0."""
         assert dtype in (torch.float8_e4m3fn, torch.float8_e5m2) and K % 128 == 0 and rows >= 1
-        self.rows, self.K = int(rows), int(K)
-        self.data = torch.empty((rows, K), dtype=dtype, device=device)
+        assert not transposed or rows % 16 == 0
+        self.rows, self.K, self.transposed = int(rows), int(K), bool(transposed)
+        self.data = torch.empty((K, rows) if transposed else (rows, K), dtype=dtype, device=device)
         self.sf = torch.empty(scalify_mx_sf_bytes(rows, K), dtype=torch.uint8, device=device)
         self.scale = torch.ones(1, dtype=torch.float32, device=device)
         self._d = scalify_mx_array(self.data.data_ptr(), _DTYPE_CODE[dtype], self.rows, self.K, self.sf.data_ptr(),
-                                   self.scale.data_ptr())
+                                   self.scale.data_ptr(), int(self.transposed))
 
     def scale_value(self) -> float:
         return float(self.scale.item())

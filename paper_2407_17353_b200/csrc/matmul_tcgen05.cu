@@ -1273,9 +1273,14 @@ int launch_mx_matmul(const MxMatmulArgs& a, void* ws, cudaStream_t st) {
   const int ncta = (a.M > kBM && a.force_ncta != 1) ? 2 : 1;
   const int tile_m = kBM * ncta;
   CUtensorMap map_a, map_b, map_y, map_sfa, map_sfb;
-  int rc = make_map(&map_a, a.A, a.K, a.M, 1, a.K, 0, kBM);
+  // K-major operand [rows, K]: box of 128 (or 256) rows x 128 bytes of K; transposed operand [K, rows]: box of
+  // 128 K-rows x 128 bytes of rows, consumed MN-major (as the per-tensor kernel does for transA / plain B)
+  int rc;
+  if (!a.transA) rc = make_map(&map_a, a.A, a.K, a.M, 1, a.K, 0, kBM);
+  else rc = make_map(&map_a, a.A, a.M, a.K, 1, a.M, 0, kBK);
   if (rc) return rc;
-  rc = make_map(&map_b, a.B, a.K, a.N, 1, a.K, 0, ncta == 2 ? kBN / 2 : kBN);
+  if (!a.transB) rc = make_map(&map_b, a.B, a.K, a.N, 1, a.K, 0, ncta == 2 ? kBN / 2 : kBN);
+  else rc = make_map(&map_b, a.B, a.N, a.K, 1, a.N, 0, kBK);
   if (rc) return rc;
   rc = make_map_y(&map_y, a.Y, elem_size(a.y_dt), a.N, a.M, 1, a.ldy, 0);
   if (rc) return rc;
@@ -1288,13 +1293,14 @@ int launch_mx_matmul(const MxMatmulArgs& a, void* ws, cudaStream_t st) {
   p.M = a.M; p.N = a.N; p.K = a.K; p.batch = 1;
   p.tiles_m = (a.M + tile_m - 1) / tile_m;
   p.tiles_n = (a.N + kBN - 1) / kBN;
-  p.a_mn_major = 0;
-  p.b_mn_major = 0;
+  p.a_mn_major = a.transA ? 1 : 0;
+  p.b_mn_major = a.transB ? 1 : 0;
   p.b_batched = 0;
   // block-scaled instruction descriptor (kind::mxf8f6f4): scale-factor ids in bits 4-5 (B) and 29-30 (A)
-  // are filled in per MMA; A/B formats, K-major operands, N >> 3, E8M0 exponents (bit 23), M >> 4 (M counts
-  // the rows of the whole CTA pair)
+  // are filled in per MMA; A/B formats, operand majorness (0 = K-major), N >> 3, E8M0 exponents (bit 23),
+  // M >> 4 (M counts the rows of the whole CTA pair)
   p.idesc = (uint32_t(a.a_dt == SCALIFY_E5M2) << 7) | (uint32_t(a.b_dt == SCALIFY_E5M2) << 10) |
+            (uint32_t(p.a_mn_major) << 15) | (uint32_t(p.b_mn_major) << 16) |
             (uint32_t(kBN >> 3) << 17) | (1u << 23) | (uint32_t(tile_m >> 4) << 24);
   p.kf = kfactor(a.K);
   p.alpha = 1.0f / p.kf;

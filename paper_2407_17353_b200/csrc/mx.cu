@@ -125,6 +125,116 @@ __global__ void __launch_bounds__(kMxThreads) mx_quantize_kernel(const void* __r
   }
 }
 
+// The same quantisation for an operand stored TRANSPOSED: X and the data are [K, rows] (row-major, `rows`
+// contiguous), and a block is 32 consecutive elements of K = 32 consecutive ROWS of the storage at one column.
+// This is the form a backward matmul needs (the contraction runs over the dimension that is not contiguous in the
+// forward tensors); the matmul then consumes the data MN-major, so no transposed copy exists.  The exponent tiles
+// are the same as for the plain form: tile (r, k) holds operand rows r*128..+127 (columns of the storage here)
+// and the four blocks of K-rows k*128..+127.
+// One thread block quantises 128 K-rows x 128 columns (one exponent tile).  Warp w takes the 32 K-rows of block
+// w / 2 and the 64 columns of half w % 2; a lane takes 8 rows x 8 columns (eight loads in flight), the column
+// maxima of the four lanes that share a column come from two shuffles.
+template <int IN, int ELEM>
+__global__ void __launch_bounds__(kMxThreads) mx_quantize_t_kernel(const void* __restrict__ X, int64_t ldx, int64_t rows,
+                                                                   int64_t K, void* __restrict__ data, int64_t ldd,
+                                                                   uint8_t* __restrict__ sf, const float* x_scale,
+                                                                   float* y_scale, uint32_t* status) {
+  asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
+  constexpr int ES = ElemBytes<IN>::v;
+  constexpr int kEmax = ELEM == SCALIFY_E4M3 ? 8 : 15;
+  __shared__ __align__(16) uint8_t s_sf[512];
+  const int64_t k_tile = blockIdx.x, r_tile = blockIdx.y;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int blk = warp >> 1, half = warp & 1;
+  const int cg = lane & 7, rq = lane >> 3;
+  const int64_t col0 = r_tile * 128 + half * 64 + cg * 8;            // first of this lane's 8 columns (operand rows)
+  const int64_t krow0 = k_tile * 128 + blk * 32 + rq * 8;            // first of this lane's 8 K-rows
+  const bool in_cols = col0 < rows;                                   // rows is a multiple of 8: whole vector or nothing
+  float f[8][8];
+  uint32_t cmax[8];
+#pragma unroll
+  for (int c = 0; c < 8; ++c) cmax[c] = 0u;
+  uint32_t w[8][8 * ES / 4];
+#pragma unroll
+  for (int r = 0; r < 8; ++r) {
+#pragma unroll
+    for (int q = 0; q < 8 * ES / 4; ++q) w[r][q] = 0u;
+    if (in_cols) ld_raw_stream<8 * ES>(static_cast<const char*>(X) + ((krow0 + r) * ldx + col0) * ES, w[r]);
+  }
+#pragma unroll
+  for (int r = 0; r < 8; ++r) {
+    decode_vec<IN, 8>(w[r], f[r]);
+#pragma unroll
+    for (int c = 0; c < 8; ++c) cmax[c] = max(cmax[c], abs_bits(f[r][c]));
+  }
+#pragma unroll
+  for (int c = 0; c < 8; ++c) {
+    cmax[c] = max(cmax[c], __shfl_xor_sync(0xFFFFFFFFu, cmax[c], 8));
+    cmax[c] = max(cmax[c], __shfl_xor_sync(0xFFFFFFFFu, cmax[c], 16));
+  }
+  float sc[8];
+  uint32_t ebytes[2] = {0u, 0u};
+#pragma unroll
+  for (int c = 0; c < 8; ++c) {
+    // shared exponent: floor(log2(amax)) - emax of the element format; 0 for a block whose maximum is zero,
+    // infinite or NaN
+    const uint32_t amax = cmax[c];
+    int e = 0;
+    if (amax != 0u && amax < 0x7F800000u) {
+      int ex = static_cast<int>(amax >> 23) - 127;
+      if ((amax >> 23) == 0u) ex = -127 - __clz(amax << 9);
+      e = max(-127, min(127, ex - kEmax));
+    }
+    const uint32_t field = static_cast<uint32_t>(127 - e);
+    sc[c] = __uint_as_float(field ? field << 23 : 0x00400000u);  // 2^-e, exactly (2^-127 as a subnormal)
+    ebytes[c >> 2] |= static_cast<uint32_t>(e + 127) << (8 * (c & 3));
+  }
+  if (in_cols) {
+#pragma unroll
+    for (int r = 0; r < 8; ++r) {
+      float g[8];
+#pragma unroll
+      for (int c = 0; c < 8; ++c) g[c] = f[r][c] * sc[c];
+      uint32_t o[2];
+      encode_vec<ELEM, 8>(g, o);
+      st_raw<8>(static_cast<char*>(data) + (krow0 + r) * ldd + col0, o);
+    }
+  }
+  if (rq == 0) {
+    // operand row m = half*64 + cg*8 + c of the tile, block blk: byte (m % 32) * 16 + (m / 32) * 4 + blk
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+      const int m = half * 64 + cg * 8 + c;
+      s_sf[(m & 31) * 16 + (m >> 5) * 4 + blk] = static_cast<uint8_t>((ebytes[c >> 2] >> (8 * (c & 3))) & 0xFFu);
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x < 32)
+    reinterpret_cast<uint4*>(sf + (r_tile * gridDim.x + k_tile) * 512)[threadIdx.x] =
+        reinterpret_cast<const uint4*>(s_sf)[threadIdx.x];
+  if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
+    const float xs = load_scale(x_scale);
+    if (y_scale) *y_scale = xs;
+    if (!is_pow2_scale(xs) && status) atomicOr(status, static_cast<uint32_t>(SCALIFY_DEV_BAD_SCALE));
+  }
+}
+
+int launch_mx_quantize_t(const void* X, int x_dt, int64_t rows, int64_t K, int64_t ldx, void* data, int elem_dt,
+                         uint8_t* sf, const float* x_scale, float* y_scale, uint32_t* status, cudaStream_t st) {
+  const int64_t r_tiles = (rows + 255) / 256 * 2;  // 128-row tiles of the operand, padding rows included
+  if (r_tiles > 65535) return SCALIFY_ERR_SHAPE;
+  const dim3 grid(static_cast<unsigned>(K / 128), static_cast<unsigned>(r_tiles));
+#define SCALIFY_MXT_LAUNCH(ELEM) \
+  mx_quantize_t_kernel<IN, ELEM><<<grid, kMxThreads, 0, st>>>(X, ldx, rows, K, data, rows, sf, x_scale, y_scale, status)
+  SCALIFY_DISPATCH_WIDE(x_dt, IN, {
+    if (elem_dt == SCALIFY_E4M3) SCALIFY_MXT_LAUNCH(SCALIFY_E4M3);
+    else SCALIFY_MXT_LAUNCH(SCALIFY_E5M2);
+  });
+#undef SCALIFY_MXT_LAUNCH
+  SCALIFY_CUDA_TRY(cudaGetLastError());
+  return SCALIFY_OK;
+}
+
 int launch_mx_quantize(const void* X, int x_dt, int64_t rows, int64_t K, int64_t ldx, void* data, int elem_dt,
                        uint8_t* sf, const float* x_scale, float* y_scale, uint32_t* status, cudaStream_t st) {
   const int64_t r_tiles = (rows + 255) / 256 * 2;  // 128-row tiles, padding rows included

@@ -378,6 +378,8 @@ static int check_mx(const scalify_mx_array* a) {
     return SCALIFY_ERR_SHAPE;
   if (reinterpret_cast<uintptr_t>(a->data) % 16 != 0 || reinterpret_cast<uintptr_t>(a->sf) % 16 != 0)
     return SCALIFY_ERR_ALIGNMENT;
+  if (a->transposed != 0 && a->transposed != 1) return SCALIFY_ERR_VALUE;
+  if (a->transposed && a->rows % 16 != 0) return SCALIFY_ERR_ALIGNMENT;  // rows of the storage are `rows` bytes long
   return SCALIFY_OK;
 }
 
@@ -392,8 +394,13 @@ int scalify_mx_quantize(const scalify_array* X, scalify_mx_array* Y, uint32_t* s
   rc = check_mx(Y);
   if (rc) return rc;
   if (!is_wide(X->dtype)) return SCALIFY_ERR_DTYPE;
-  if (X->ndim != 2 || X->shape[0] != Y->rows || X->shape[1] != Y->K) return SCALIFY_ERR_SHAPE;
   if (Y->scale && Y->scale == X->scale) return SCALIFY_ERR_ALIAS;
+  if (Y->transposed) {
+    if (X->ndim != 2 || X->shape[0] != Y->K || X->shape[1] != Y->rows) return SCALIFY_ERR_SHAPE;
+    return launch_mx_quantize_t(X->data, X->dtype, Y->rows, Y->K, X->stride[0], Y->data, Y->dtype, Y->sf, X->scale,
+                                Y->scale, status, static_cast<cudaStream_t>(stream));
+  }
+  if (X->ndim != 2 || X->shape[0] != Y->rows || X->shape[1] != Y->K) return SCALIFY_ERR_SHAPE;
   return launch_mx_quantize(X->data, X->dtype, Y->rows, Y->K, X->stride[0], Y->data, Y->dtype, Y->sf, X->scale,
                             Y->scale, status, static_cast<cudaStream_t>(stream));
 }
@@ -420,6 +427,8 @@ int scalify_mx_matmul(const scalify_mx_array* A, const scalify_mx_array* B, scal
   a.a_scale = A->scale; a.b_scale = B->scale; a.y_scale = Y->scale;
   a.stat = stat;
   a.force_ncta = 0;
+  a.transA = A->transposed;
+  a.transB = B->transposed;
   return launch_mx_matmul(a, workspace, static_cast<cudaStream_t>(stream));
 }
 

@@ -113,6 +113,7 @@ struct MxMatmulArgs {
   const float* a_scale; const float* b_scale; float* y_scale;
   int stat;
   int force_ncta;  // 0: choose; 1: force the one-CTA kernel
+  int transA, transB;  // operand stored [K, rows]: consumed MN-major
 };
 int launch_mx_matmul(const MxMatmulArgs& a, void* ws, cudaStream_t st);
 size_t mx_sf_bytes(int64_t rows, int64_t K);
@@ -148,6 +149,8 @@ struct AttentionBwdArgs {
   uint32_t* status;
 };
 int launch_attention_bwd(const AttentionBwdArgs& a, cudaStream_t st);
+int launch_mx_quantize_t(const void* X, int x_dt, int64_t rows, int64_t K, int64_t ldx, void* data, int elem_dt,
+                         uint8_t* sf, const float* x_scale, float* y_scale, uint32_t* status, cudaStream_t st);
 int launch_mx_quantize(const void* X, int x_dt, int64_t rows, int64_t K, int64_t ldx, void* data, int elem_dt,
                        uint8_t* sf, const float* x_scale, float* y_scale, uint32_t* status, cudaStream_t st);
 
