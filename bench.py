@@ -605,6 +605,32 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    def graph_ms(calls, n_calls):
+        """Average device time per call of `n_calls` library calls (round robin over `calls`) recorded once
+        into a CUDA graph and replayed: what a launch-bound call costs on the device once Python and the
+        driver's launch path are out of the way."""
+        side = torch.cuda.Stream(dev)
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for f in calls:
+                f()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                for i in range(n_calls):
+                    calls[i % len(calls)]()
+        torch.cuda.current_stream().wait_stream(side)
+        g.replay()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(3):
+            g.replay()
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1) / (3 * n_calls)
+        del g
+        return ms
+
     # the sampler thread starts before the warm-up, so that NVML's start-up is over when the timed region begins
     sampler = ClockSampler(local_rank) if rank == 0 else None
     for t in range(W):
@@ -762,23 +788,30 @@ def main():
         del Xa, Xb, Am, Bm, Amt, Bmt
 
     # Fused attention forward on the config-5 shape: 8 sequences x 12 heads, 1024 tokens, head dimension 64
-    att_ms = att_bwd_ms = float("nan")
+    att_ms = att_bwd_ms = att_graph_ms = att_bwd_graph_ms = float("nan")
     ATT_H, ATT_T, ATT_HD = 96, 1024, 64
+    ATT_SETS = 9   # 9 x 31 MB of Q, K, V, O: twice the L2, so no call finds its inputs there
     if not args.no_next:
-        Qa, Ka, Va = (sc.ScaledTensor.make(rnd((ATT_H, ATT_T, ATT_HD), torch.float8_e4m3fn, 30 + i), 1.0)
-                      for i in range(3))
-        Oa = sc.ScaledTensor.empty((ATT_H, ATT_T, ATT_HD), torch.bfloat16, dev)
-        for _ in range(3):
-            sc.scalify_scaled_attention(Qa, Ka, Va, Oa, sm_scale=0.125, causal=True)
+        att_sets = []
+        for k in range(ATT_SETS):
+            q_, k_, v_ = (sc.ScaledTensor.make(rnd((ATT_H, ATT_T, ATT_HD), torch.float8_e4m3fn, 30 + i + 3 * k), 1.0)
+                          for i in range(3))
+            att_sets.append((q_, k_, v_, sc.ScaledTensor.empty((ATT_H, ATT_T, ATT_HD), torch.bfloat16, dev)))
+        att_calls = [lambda t=t: sc.scalify_scaled_attention(t[0], t[1], t[2], t[3], sm_scale=0.125, causal=True)
+                     for t in att_sets]
+        Qa, Ka, Va, Oa = att_sets[0]
+        for f in att_calls:
+            f()
         barrier()
         a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a_iters = max(3, min(K, 20))
+        a_iters = max(ATT_SETS, min(K, 2 * ATT_SETS))
         a0.record()
-        for _ in range(a_iters):
-            sc.scalify_scaled_attention(Qa, Ka, Va, Oa, sm_scale=0.125, causal=True)
+        for i in range(a_iters):
+            att_calls[i % ATT_SETS]()
         a1.record()
         barrier()
         att_ms = a0.elapsed_time(a1) / a_iters
+        att_graph_ms = graph_ms(att_calls, 2 * ATT_SETS)
         # ... and its backward (two launches): P from the forward's copy, dO as E5M2
         Pa = sc.ScaledTensor(torch.zeros((ATT_H, ATT_T, ATT_T), dtype=torch.uint8, device=dev).view(torch.float8_e4m3fn),
                              torch.ones(1, dtype=torch.float32, device=dev))
@@ -797,7 +830,8 @@ def main():
         a1.record()
         barrier()
         att_bwd_ms = a0.elapsed_time(a1) / a_iters
-        del Qa, Ka, Va, Oa, Pa, dOa, dSa, dQa, dKa, dVa
+        att_bwd_graph_ms = graph_ms([att_bwd], 10)   # P and dS are 100 MB each: larger than the L2 by themselves
+        del Qa, Ka, Va, Oa, Pa, dOa, dSa, dQa, dKa, dVa, att_sets, att_calls
 
     # ------------------------------------------------------------------ configs[1]: the other sizes and formats
     # M = N = K in {1024, 4096, 8192}, forward E4M3 x E4M3 and gradient E5M2 x E4M3, each as the one-call form
@@ -832,9 +866,15 @@ def main():
                 g1.record()
                 barrier()
                 g_ms = g0.elapsed_time(g1) / g_iters
-                sweep_rows.append({"row": f"configs[1] {kind}, M=N=K={n}: GEMM + fused AMAX + rescale to E4M3, one call "
-                                          f"(own loop, back to back over {sets} buffer sets)",
-                                   "ms": round(g_ms, 4), "TFLOP/s": round(2.0 * n ** 3 / (g_ms * 1e-3) / 1e12, 1)})
+                sweep = {"row": f"configs[1] {kind}, M=N=K={n}: GEMM + fused AMAX + rescale to E4M3, one call "
+                                f"(own loop, back to back over {sets} buffer sets)",
+                         "ms": round(g_ms, 4), "TFLOP/s": round(2.0 * n ** 3 / (g_ms * 1e-3) / 1e12, 1)}
+                if n < N_GEMM:
+                    # a call this short is bound by the launch path from Python; the same calls replayed from a CUDA graph
+                    gg_ms = graph_ms(calls, 2 * len(calls))
+                    sweep["ms_cuda_graph"] = round(gg_ms, 4)
+                    sweep["TFLOP/s_cuda_graph"] = round(2.0 * n ** 3 / (gg_ms * 1e-3) / 1e12, 1)
+                sweep_rows.append(sweep)
                 del calls
                 torch.cuda.empty_cache()
 
@@ -955,15 +995,18 @@ def main():
         {"row": "f3 (next, own loop) block-scaled GEMM 8192^3, both operands in the transposed (MN-major) form of "
                 "the gradient products", "ms": round(float(mx_mmt_ms), 4),
          "TFLOP/s": round(flops / (mx_mmt_ms * 1e-3) / 1e12, 1)},
-        {"row": "f4 (next, own loop) fused causal attention forward, 96 heads x 1024 tokens x 64 (scores and "
-                "probabilities never leave the chip)", "ms": round(float(att_ms), 4),
+        {"row": f"f4 (next, own loop over {ATT_SETS} buffer sets) fused causal attention forward, 96 heads x 1024 tokens "
+                "x 64 (scores and probabilities never leave the chip)", "ms": round(float(att_ms), 4),
          "TFLOP/s": round(2.0 * ATT_H * ATT_T * ATT_T * ATT_HD / (att_ms * 1e-3) / 1e12, 1),
-         "note": "flop counted for the causal half of Q K^T and P V"},
+         "ms_cuda_graph": round(float(att_graph_ms), 4),
+         "note": "flop counted for the causal half of Q K^T and P V; ms_cuda_graph: the same calls replayed from a "
+                 "CUDA graph (the call from Python takes longer than the kernel runs)"},
         {"row": "f4 (next, own loop) fused causal attention backward, same shape: dQ, dK, dV from dO and the "
                 "forward's E4M3 probabilities in two launches (dP never leaves the chip, dS is written once)",
          "ms": round(float(att_bwd_ms), 4),
          "TFLOP/s": round(4.0 * ATT_H * ATT_T * ATT_T * ATT_HD / (att_bwd_ms * 1e-3) / 1e12, 1),
-         "note": "flop counted for the causal half of dO V^T, dS K, dS^T Q and P^T dO"},
+         "ms_cuda_graph": round(float(att_bwd_graph_ms), 4),
+         "note": "flop counted for the causal half of dO V^T, dS K, dS^T Q and P^T dO; ms_cuda_graph as above"},
     ] + sweep_rows
     # Which of the two measured bf16 rates is the denominator: the sustained one holds for a GEMM that runs for
     # seconds under the power cap; a timed region under a second, or a GEMM that is less than half of the step's
