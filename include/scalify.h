@@ -364,10 +364,11 @@ int scalify_debug_expire_wait(void* workspace, size_t workspace_bytes, uint32_t 
 /*
  * Diagnostic (no counterpart in the paper): y[i] = x[i] rounded to the nearest BF16 value (ties to even), as
  * fp32, computed by the routine the fused attention kernels use for the scores' BF16 intermediate (three fp32
- * operations instead of a conversion).  x, y: device fp32 arrays of n elements.  Lets a test compare that
- * routine with the definition over any set of bit patterns.
+ * operations instead of a conversion).  x, y: device fp32 arrays of n elements.  two_wide = 0: the scalar
+ * form; 1: the form on two-wide fp32 instructions, which takes the elements in pairs (x[0], x[1]), ...
+ * Lets a test compare both with the definition over any set of bit patterns.
  */
-int scalify_debug_bf16_round(const float* x, float* y, int64_t n, void* stream);
+int scalify_debug_bf16_round(const float* x, float* y, int64_t n, int two_wide, void* stream);
 
 /*
  * Diagnostics of the library's host-side state (no counterpart in the paper; host only, no GPU needed).

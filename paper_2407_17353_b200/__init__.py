@@ -96,7 +96,7 @@ def lib() -> ctypes.CDLL:
         L.scalify_scalar_mul_pow2.argtypes = [P, f32, vp]
         L.scalify_debug_layernorm_plan.argtypes = [i64, i64, i32, i32, vp]
         L.scalify_debug_host_state_selftest.restype = i32
-        L.scalify_debug_bf16_round.argtypes = [vp, vp, i64, vp]
+        L.scalify_debug_bf16_round.argtypes = [vp, vp, i64, i32, vp]
         L.scalify_debug_bf16_round.restype = i32
         L.scalify_debug_tensor_map_cache.argtypes = [vp, vp]
         L.scalify_debug_tensor_map_cache.restype = i32
@@ -421,10 +421,11 @@ def scalify_debug_expire_wait(ws: Workspace, limit_us: int, waited_us: Optional[
            "scalify_debug_expire_wait")
 
 
-def scalify_debug_bf16_round(x: torch.Tensor, y: torch.Tensor, stream=None) -> None:
-    """y = x rounded to the nearest BF16 value (as fp32) by the routine the attention kernels use."""
+def scalify_debug_bf16_round(x: torch.Tensor, y: torch.Tensor, two_wide: bool = False, stream=None) -> None:
+    """y = x rounded to the nearest BF16 value (as fp32) by the routine the attention kernels use (scalar form,
+    or the two-wide form that takes the elements in pairs)."""
     assert x.dtype == y.dtype == torch.float32 and x.is_contiguous() and y.is_contiguous() and x.numel() == y.numel()
-    _check(lib().scalify_debug_bf16_round(x.data_ptr(), y.data_ptr(), x.numel(), _stream(stream)),
+    _check(lib().scalify_debug_bf16_round(x.data_ptr(), y.data_ptr(), x.numel(), int(bool(two_wide)), _stream(stream)),
            "scalify_debug_bf16_round")
 
 

@@ -75,6 +75,13 @@ __device__ __forceinline__ uint64_t make_smem_desc_sw64(uint32_t saddr, uint32_t
 
 // 2^x for x <= 0 (and -inf): the hardware approximation (2 ulp of fp32, results below 2^-126 flush to 0),
 // far finer than the E4M3 probabilities it feeds
+// three-input maximum (one instruction on sm_100)
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+
 __device__ __forceinline__ float exp2_neg(float x) {
   float r;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
@@ -233,6 +240,23 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         for (int e = 0; e < 32; ++e) x[e] = (j0 + e < lim) ? x[e] : -INFINITY;
       }
     };
+    // Fast form for a positive scale (every real use): r[k] = the two rounded scores 2k, 2k+1 in accumulator
+    // units (two-wide rounding, 1.5 instructions per element), -inf for hidden keys.  The scale is applied
+    // inside the multiply-add that also subtracts the row maximum, and the row maximum is taken on the unscaled
+    // values (scaling by a positive constant is monotone, so fl(max r * sc3) is the maximum of fl(r * sc3)).
+    const bool pos_scale = sc3 > 0.f;
+    auto chunk_rounded = [&](const uint32_t* acc_bits, int j0, float2* r2) {
+#pragma unroll
+      for (int k = 0; k < 16; ++k)
+        r2[k] = bf16_round_f32x2(make_float2(__uint_as_float(acc_bits[2 * k]), __uint_as_float(acc_bits[2 * k + 1])));
+      if (j0 + 32 > lim) {
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+          r2[k].x = (j0 + 2 * k < lim) ? r2[k].x : -INFINITY;
+          r2[k].y = (j0 + 2 * k + 1 < lim) ? r2[k].y : -INFINITY;
+        }
+      }
+    };
     int it = 0;
     // sweep A: row maximum and sum of exponentials
     for (int kb = 0; kb < n_kb; ++kb, ++it) {
@@ -246,28 +270,49 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         if (c == c_first + kChunks - 1) {
           // the score block is in registers: hand the TMEM buffer back now, so that the tensor core computes the
           // next block's scores while this one is worked on (taking both chunks to registers first, to hand it
-          // back a chunk earlier, costs a second CTA per SM its registers: 83 us against 54 us)
+          // back a chunk earlier, costs a second CTA per SM its registers: 83 us against 54 us; issuing the next
+          // chunk's read under this chunk's arithmetic changed nothing: 51.5 against 50.6 us)
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(s_empty);
         }
         // one pass per 32-key chunk: chunk maximum, then the running sum is moved to the new maximum
-        float x[32];
-        chunk_scores(acc, kb * kAttK + c * 32, x);
-        float cm4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // four independent chains
+        if (pos_scale) {
+          float2 r2[16];
+          chunk_rounded(acc, kb * kAttK + c * 32, r2);
+          float cm4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // four independent chains
 #pragma unroll
-        for (int e = 0; e < 32; ++e) cm4[e & 3] = fmaxf(cm4[e & 3], x[e]);
-        const float m_new = fmaxf(m, fmaxf(fmaxf(cm4[0], cm4[1]), fmaxf(cm4[2], cm4[3])));
-        if (m_new > -INFINITY) {
-          const float2 nm2 = make_float2(-m_new, -m_new);
-          float2 add2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+          for (int k = 0; k < 16; ++k) cm4[k & 3] = fmax3(cm4[k & 3], r2[k].x, r2[k].y);
+          const float m_new = fmaxf(m, fmaxf(fmaxf(cm4[0], cm4[1]), fmaxf(cm4[2], cm4[3])) * sc3);
+          if (m_new > -INFINITY) {
+            const float2 nm2 = make_float2(-m_new, -m_new);
+            float2 add2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
 #pragma unroll
-          for (int e = 0; e < 32; e += 2) {
-            const float2 a = __fadd2_rn(make_float2(x[e], x[e + 1]), nm2);
-            add2[(e >> 1) & 1] = __fadd2_rn(add2[(e >> 1) & 1], make_float2(exp2_neg(a.x), exp2_neg(a.y)));  // 2^-inf = 0 for masked keys
+            for (int k = 0; k < 16; ++k) {
+              const float2 a = __ffma2_rn(r2[k], sc3_2, nm2);  // -inf for hidden keys: 2^-inf = 0
+              add2[k & 1] = __fadd2_rn(add2[k & 1], make_float2(exp2_neg(a.x), exp2_neg(a.y)));
+            }
+            l = l * exp2_neg(m - m_new) + ((add2[0].x + add2[0].y) + (add2[1].x + add2[1].y));  // and while nothing was seen
+            m = m_new;
           }
-          l = l * exp2_neg(m - m_new) + ((add2[0].x + add2[0].y) + (add2[1].x + add2[1].y));  // and while nothing was seen
-          m = m_new;
+        } else {
+          float x[32];
+          chunk_scores(acc, kb * kAttK + c * 32, x);
+          float cm4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+          for (int e = 0; e < 32; ++e) cm4[e & 3] = fmaxf(cm4[e & 3], x[e]);
+          const float m_new = fmaxf(m, fmaxf(fmaxf(cm4[0], cm4[1]), fmaxf(cm4[2], cm4[3])));
+          if (m_new > -INFINITY) {
+            const float2 nm2 = make_float2(-m_new, -m_new);
+            float2 add2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+#pragma unroll
+            for (int e = 0; e < 32; e += 2) {
+              const float2 a = __fadd2_rn(make_float2(x[e], x[e + 1]), nm2);
+              add2[(e >> 1) & 1] = __fadd2_rn(add2[(e >> 1) & 1], make_float2(exp2_neg(a.x), exp2_neg(a.y)));
+            }
+            l = l * exp2_neg(m - m_new) + ((add2[0].x + add2[0].y) + (add2[1].x + add2[1].y));
+            m = m_new;
+          }
         }
         if (p.S_dump && i < p.Tq) {
           const int j0 = kb * kAttK + c * 32;
@@ -295,6 +340,9 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     }
     asm volatile("bar.sync 1, %0;" ::"n"(32 * kAttSmWarps) : "memory");  // the tile may be overwritten from here on
     const float inv_l = 1.0f / l;
+    // positive scale: the division by l moves into the exponent, p = 2^(r * sc3 - (m + log2 l)) in one
+    // multiply-add and one exp2 per element (log2 to 2^-22 absolute: far finer than the E4M3 result)
+    const float m_l = m + __log2f(l);
     // sweep B: probabilities -> E4M3 -> shared memory (A operand of P V)
     for (int kb = 0; kb < n_kb && !timed_out; ++kb, ++it) {
       if (!mbar_wait(s_full, it & 1, abort_flag)) { timed_out = true; break; }
@@ -308,22 +356,32 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         tmem_ld32(t_row + c * 32, acc);
         tmem_ld_wait();
         if (c == c_first + kChunks - 1) {
-          // the score block is in registers: hand the TMEM buffer back now, so that the tensor core computes the
-          // next block's scores while this one is worked on (taking both chunks to registers first, to hand it
-          // back a chunk earlier, costs a second CTA per SM its registers: 83 us against 54 us)
+          // the score block is in registers: hand the TMEM buffer back now (as in sweep A)
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(s_empty);
         }
         float pr[32];
-        chunk_scores(acc, kb * kAttK + c * 32, pr);
-        const float2 nm2 = make_float2(-m, -m), il2 = make_float2(inv_l, inv_l);
+        if (pos_scale) {
+          float2 r2[16];
+          chunk_rounded(acc, kb * kAttK + c * 32, r2);
+          const float2 nml2 = make_float2(-m_l, -m_l);
 #pragma unroll
-        for (int e = 0; e < 32; e += 2) {
-          const float2 a = __fadd2_rn(make_float2(pr[e], pr[e + 1]), nm2);
-          const float2 q = __fmul2_rn(make_float2(exp2_neg(a.x), exp2_neg(a.y)), il2);
-          pr[e] = q.x;
-          pr[e + 1] = q.y;
+          for (int k = 0; k < 16; ++k) {
+            const float2 a = __ffma2_rn(r2[k], sc3_2, nml2);
+            pr[2 * k] = exp2_neg(a.x);
+            pr[2 * k + 1] = exp2_neg(a.y);
+          }
+        } else {
+          chunk_scores(acc, kb * kAttK + c * 32, pr);
+          const float2 nm2 = make_float2(-m, -m), il2 = make_float2(inv_l, inv_l);
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            const float2 a = __fadd2_rn(make_float2(pr[e], pr[e + 1]), nm2);
+            const float2 q = __fmul2_rn(make_float2(exp2_neg(a.x), exp2_neg(a.y)), il2);
+            pr[e] = q.x;
+            pr[e + 1] = q.y;
+          }
         }
         uint32_t o[8];
         encode_vec<SCALIFY_E4M3, 32>(pr, o);

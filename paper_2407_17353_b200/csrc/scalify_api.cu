@@ -887,10 +887,10 @@ int scalify_debug_expire_wait(void* workspace, size_t workspace_bytes, uint32_t 
                             static_cast<cudaStream_t>(stream));
 }
 
-int scalify_debug_bf16_round(const float* x, float* y, int64_t n, void* stream) {
+int scalify_debug_bf16_round(const float* x, float* y, int64_t n, int two_wide, void* stream) {
   if (!x || !y) return SCALIFY_ERR_NULL;
   if (n < 1) return SCALIFY_ERR_SHAPE;
-  return launch_bf16_round(x, y, n, static_cast<cudaStream_t>(stream));
+  return launch_bf16_round(x, y, n, two_wide ? 1 : 0, static_cast<cudaStream_t>(stream));
 }
 
 int scalify_debug_host_state_selftest(void) { return host_state_selftest(); }

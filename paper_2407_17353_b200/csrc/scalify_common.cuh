@@ -316,6 +316,17 @@ __device__ __forceinline__ float bf16_round_f32(float x) {
   return __fsub_rn(c, d);
 }
 
+// The same rounding for two values at once on the two-wide fp32 instructions.  Each of the three steps is
+// written as a fused multiply-add with a non-trivial addend (65536 x + x = 65537 x rounded once; c - x and
+// c - d as (-1) * v + c), so that there is no separate multiply for the toolchain to contract into the
+// subtraction that follows: a multiply-add cannot be merged with another operation.
+__device__ __forceinline__ float2 bf16_round_f32x2(float2 x) {
+  const float2 k = make_float2(65536.0f, 65536.0f), neg = make_float2(-1.0f, -1.0f);
+  const float2 c = __ffma2_rn(x, k, x);
+  const float2 d = __ffma2_rn(x, neg, c);
+  return __ffma2_rn(d, neg, c);
+}
+
 // scalar load/store for ragged tails
 template <int DT>
 __device__ __forceinline__ float load_elem(const void* p, int64_t i) {

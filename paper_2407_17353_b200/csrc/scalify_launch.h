@@ -99,7 +99,7 @@ struct MatmulArgs {
 };
 size_t matmul_ws_bytes(int64_t rows, int64_t cols);
 size_t matmul_splitk_ws_bytes(int64_t rows, int64_t cols);
-int launch_bf16_round(const float* x, float* y, long long n, cudaStream_t st);
+int launch_bf16_round(const float* x, float* y, long long n, int two_wide, cudaStream_t st);
 int host_state_selftest();
 void map_cache_counters(unsigned long long* hits, unsigned long long* misses);
 int launch_expire_wait(void* ws, unsigned long long limit_ns, uint32_t* waited_us, cudaStream_t st);

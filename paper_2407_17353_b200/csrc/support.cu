@@ -696,16 +696,29 @@ int launch_colsum(const void* X, int x_dt, long long ld, long long R, long long 
   return SCALIFY_OK;
 }
 
-// Diagnostic: the fp32-pipe BF16 rounding used inside the attention kernels, applied to an array
+// Diagnostic: the fp32-pipe BF16 rounding used inside the attention kernels, applied to an array; the
+// two-wide form takes the elements in pairs (a last odd element goes through the scalar form)
+template <bool TWO_WIDE>
 __global__ void __launch_bounds__(256) bf16_round_kernel(const float* __restrict__ x, float* __restrict__ y, long long n) {
   asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
-  for (long long i = static_cast<long long>(blockIdx.x) * 256 + threadIdx.x; i < n; i += static_cast<long long>(gridDim.x) * 256)
-    y[i] = bf16_round_f32(x[i]);
+  const long long t0 = static_cast<long long>(blockIdx.x) * 256 + threadIdx.x, step = static_cast<long long>(gridDim.x) * 256;
+  if constexpr (TWO_WIDE) {
+    for (long long i = t0; i < n / 2; i += step) {
+      const float2 r = bf16_round_f32x2(make_float2(x[2 * i], x[2 * i + 1]));
+      y[2 * i] = r.x;
+      y[2 * i + 1] = r.y;
+    }
+    if ((n & 1) && t0 == 0) y[n - 1] = bf16_round_f32(x[n - 1]);
+  } else {
+    for (long long i = t0; i < n; i += step) y[i] = bf16_round_f32(x[i]);
+  }
 }
 
-int launch_bf16_round(const float* x, float* y, long long n, cudaStream_t st) {
+int launch_bf16_round(const float* x, float* y, long long n, int two_wide, cudaStream_t st) {
   const long long blocks = (n + 255) / 256;
-  bf16_round_kernel<<<static_cast<unsigned>(blocks < 148 * 16 ? blocks : 148 * 16), 256, 0, st>>>(x, y, n);
+  const unsigned grid = static_cast<unsigned>(blocks < 148 * 16 ? blocks : 148 * 16);
+  if (two_wide) bf16_round_kernel<true><<<grid, 256, 0, st>>>(x, y, n);
+  else bf16_round_kernel<false><<<grid, 256, 0, st>>>(x, y, n);
   SCALIFY_CUDA_TRY(cudaGetLastError());
   return SCALIFY_OK;
 }

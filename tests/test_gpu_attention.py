@@ -20,8 +20,8 @@ HD = 64
 
 
 def run_case(H, Tq, Tk, causal, merged_layout=False, q_dt=orc.E4M3, v_dt=orc.E4M3, o_dt=orc.BF16, seed=1,
-             check_heads=None):
-    qs, ks, vs, c = 2.0 ** -1, 2.0 ** 1, 2.0 ** -3, 0.125
+             check_heads=None, c=0.125):
+    qs, ks, vs = 2.0 ** -1, 2.0 ** 1, 2.0 ** -3
     q = si.to_bits(si.normal(seed, 1, (H, Tq, HD), 1.0), q_dt)
     k = si.to_bits(si.normal(seed, 2, (H, Tk, HD), 1.0), orc.E4M3)
     v = si.to_bits(si.normal(seed, 3, (H, Tk, HD), 1.0), v_dt)
@@ -85,6 +85,15 @@ def test_full_attention_with_more_keys_than_queries():
 
 def test_ragged_lengths_and_shifted_causal_mask():
     run_case(2, 200, 224, True)
+
+
+@pytest.mark.parametrize("c", [-0.125, 0.3, 1.0])
+def test_other_softmax_scales(c):
+    """A positive scale takes the kernel's short form (scale folded into the multiply-add that subtracts the row
+    maximum, 1/l folded into the exponent); a negative one the general form, in which the largest score is not
+    the largest scaled score."""
+    run_case(2, 200, 224, True, c=c)
+    run_case(1, 128, 256, False, c=c, seed=5)
 
 
 def test_heads_inside_a_token_major_buffer_and_mixed_formats():
@@ -183,7 +192,8 @@ def test_fp32_pipe_bf16_rounding_is_round_to_nearest_even():
     x = (bits & 0xFFFFFFFF).to(torch.uint32).view(torch.float32).contiguous()
     want = x.to(torch.bfloat16).to(torch.float32)
     xd = x.cuda()
-    yd = torch.empty_like(xd)
-    sc.scalify_debug_bf16_round(xd, yd)
-    got = yd.cpu()
-    assert torch.equal(got.view(torch.int32), want.view(torch.int32))
+    for two_wide in (False, True):   # the scalar routine and the one on two-wide instructions (elements in pairs)
+        yd = torch.empty_like(xd)
+        sc.scalify_debug_bf16_round(xd, yd, two_wide=two_wide)
+        got = yd.cpu()
+        assert torch.equal(got.view(torch.int32), want.view(torch.int32)), two_wide
