@@ -77,8 +77,8 @@ __device__ __forceinline__ void e4m3x4_to_float(uint32_t w, float* f) {
 }
 
 // Two fp32 accumulators -> their BF16 roundings (round to nearest even, one conversion instruction for
-// the pair: that pipe is idle in these kernels, and the three-operation fp32 form of the forward kernel measured
-// 90 us against 86 us here), widened back to fp32
+// the pair: that pipe is idle in these kernels; the forward kernel's fp32 forms measured 90 us (scalar) and
+// 86.6 us (two-wide), alternating the two 85.1 us, against 84.7 us here), widened back to fp32
 __device__ __forceinline__ void bf16_round_pair(uint32_t a_bits, uint32_t b_bits, float& a, float& b) {
   uint32_t packed;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(packed) : "f"(__uint_as_float(b_bits)), "f"(__uint_as_float(a_bits)));
@@ -241,16 +241,15 @@ attention_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_do, const __grid
         float pf[32];
         load_p(p_tile, c, pf);
         tmem_ld_wait();
-        float d4[4] = {0.f, 0.f, 0.f, 0.f};  // four independent chains
+        float2 d2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};  // four independent chains, two per instruction
 #pragma unroll
         for (int e = 0; e < 32; e += 2) {
           float x0, x1;
           bf16_round_pair(acc[e], acc[e + 1], x0, x1);
-          d4[e & 3] = fmaf(x0, pf[e], d4[e & 3]);
-          d4[(e + 1) & 3] = fmaf(x1, pf[e + 1], d4[(e + 1) & 3]);
+          d2[(e >> 1) & 1] = __ffma2_rn(make_float2(x0, x1), make_float2(pf[e], pf[e + 1]), d2[(e >> 1) & 1]);
         }
         // (the division by kf(hd), a power of two, commutes with every rounding above: applied once per chunk)
-        delta += ((d4[0] + d4[1]) + (d4[2] + d4[3])) * p.inv_kf_hd;
+        delta += ((d2[0].x + d2[0].y) + (d2[1].x + d2[1].y)) * p.inv_kf_hd;
         if (p.dP_dump && i < p.Tq) {
           const int j0 = kb * kBwK + c * 32;
           if (j0 < p.Tk) {  // Tk is a multiple of 32
@@ -291,12 +290,14 @@ attention_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_do, const __grid
         float pf[32];
         load_p(p_tile, c, pf);
         tmem_ld_wait();
+        const float2 ik2 = make_float2(p.inv_kf_hd, p.inv_kf_hd), nd2 = make_float2(-delta, -delta);
 #pragma unroll
         for (int e = 0; e < 32; e += 2) {
           float x0, x1;
           bf16_round_pair(acc[e], acc[e + 1], x0, x1);
-          pf[e] *= fmaf(x0, p.inv_kf_hd, -delta);
-          pf[e + 1] *= fmaf(x1, p.inv_kf_hd, -delta);
+          const float2 q = __fmul2_rn(make_float2(pf[e], pf[e + 1]), __ffma2_rn(make_float2(x0, x1), ik2, nd2));
+          pf[e] = q.x;
+          pf[e + 1] = q.y;
         }
         uint32_t o[8];
         encode_vec<SCALIFY_E5M2, 32>(pf, o);
