@@ -314,6 +314,18 @@ int scalify_scaled_layernorm(const scalify_array* X, const scalify_array* gamma,
  * stat_dx: statistic of the stored dX data, left at workspace offset 16.
  * dXq: optional rescaled gradient (any dtype), as Yq of the matmul.
  * dgamma, dbeta: optional [d] outputs, F32/BF16/F16 (both or neither).
+ *
+ * dX == NULL (one pass, the un-rebalanced gradient is not stored): allowed with
+ * stat_dx != NONE and a contiguous FP8 dXq.  The values are still rounded to
+ * the dtype of X first and the statistic is still that of those rounded values,
+ * so dXq, dXq_s, the statistic word, dgamma and dbeta equal those of the call
+ * with a dX of X's dtype bit for bit; the gradient is written with the power
+ * of two of the statistic this workspace saw last (fp32 word at byte offset 56
+ * of the workspace, any content) and a second launch of the same kernel, whose
+ * thread blocks return at once when that prediction held, writes it again
+ * otherwise.  The call leaves its own statistic in that word: keep one
+ * workspace per LayerNorm of a training step for the prediction to hold.
+ * (Section 3.3: statistic and rebalancing are separate primitives.)
  */
 int scalify_scaled_layernorm_bwd(const scalify_array* G, const scalify_array* X, const scalify_array* gamma,
                                  const float* mean, const float* rinv, float eps, int eps_inside_sqrt,

@@ -292,7 +292,7 @@ def scalify_scaled_layernorm(X: ScaledTensor, gamma: Optional[ScaledTensor], bet
 
 
 def scalify_scaled_layernorm_bwd(G: ScaledTensor, X: ScaledTensor, gamma: Optional[ScaledTensor], mean: torch.Tensor,
-                                 rinv: torch.Tensor, dX: ScaledTensor, ws: Workspace, *, eps: float = 1e-5,
+                                 rinv: torch.Tensor, dX: Optional[ScaledTensor], ws: Workspace, *, eps: float = 1e-5,
                                  eps_inside_sqrt=False, stat_dx: int = STAT_NONE, dXq: Optional[ScaledTensor] = None,
                                  dgamma: Optional[ScaledTensor] = None, dbeta: Optional[ScaledTensor] = None,
                                  stream=None) -> None:

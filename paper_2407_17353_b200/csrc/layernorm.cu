@@ -401,12 +401,42 @@ __device__ __forceinline__ float2 team_sum_pair(float2 a, float (*smem)[8][2], i
   return a;
 }
 
-template <int XDT, int DXDT, int TW>
+// EXACT: the dynamic rescale of the plain call (values rounded through the intermediate format XDT, statistic of
+// those rounded values, rebalanced output in DXDT) in ONE pass over the data: the output is written with a
+// predicted power of two (that of the statistic word `pred.hint`, the statistic this workspace saw last), and a
+// second launch of the same kernel (`pred.redo`) returns at once if this call's statistic has the same power of
+// two and otherwise writes the output again with the right one.  The intermediate is never stored.
+struct LnBwdPredict {
+  const float* hint;       // statistic of the previous call (any content: a wrong prediction only costs the second pass)
+  float* r_used;           // power of two the first launch divided by
+  const float* stat_word;  // this call's statistic (read by the second launch)
+  int redo;                // 0: first launch, 1: second launch
+};
+
+template <int XDT, int DXDT, int TW, bool EXACT>
 __global__ void __launch_bounds__(kLnThreads, 2) layernorm_bwd_kernel(
     const void* __restrict__ G, int64_t g_ld, const void* __restrict__ X, int64_t x_ld, void* __restrict__ dX,
     int64_t dx_ld, int R, int d, const void* __restrict__ gamma, int gb_dt, const float* __restrict__ mean,
-    const float* __restrict__ rinv_in, float eps, int eps_inside, int stat, const float* __restrict__ stat_in,
-    float* __restrict__ dgamma_part, float* __restrict__ dbeta_part, double* __restrict__ stat_part) {
+    const float* __restrict__ rinv_in, float eps, int eps_inside, int stat_arg, const float* __restrict__ stat_in,
+    float* __restrict__ dgamma_part_arg, float* __restrict__ dbeta_part, double* __restrict__ stat_part,
+    const LnBwdPredict pred) {
+  int stat = stat_arg;
+  float* dgamma_part = dgamma_part_arg;
+  float exact_r = 1.0f;
+  if constexpr (EXACT) {
+    bool nf;
+    if (pred.redo) {
+      // everything this launch reads was written by the launches before it
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      exact_r = rescale_factor(*reinterpret_cast<const volatile float*>(pred.stat_word), &nf);
+      if (exact_r == *reinterpret_cast<const volatile float*>(pred.r_used)) return;  // the prediction held
+      stat = SCALIFY_STAT_NONE;   // statistic and column sums are already final
+      dgamma_part = nullptr;
+    } else {
+      exact_r = rescale_factor(*reinterpret_cast<const volatile float*>(pred.hint), &nf);
+      if (blockIdx.x == 0 && threadIdx.x == 0) *pred.r_used = exact_r;
+    }
+  }
   asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   constexpr int VEC = 16 / ElemBytes<XDT>::v;
   constexpr int HP = VEC / 2;  // float2 pairs per vector
@@ -419,7 +449,8 @@ __global__ void __launch_bounds__(kLnThreads, 2) layernorm_bwd_kernel(
   // three coefficients of the output expression by it gives the same bits as dividing the result, and the
   // statistic of the un-rebalanced values is the statistic of the stored-scale values times r (exactly).
   float inv_r = 1.0f, r_prev = 1.0f;
-  if (stat_in) { bool nf; r_prev = rescale_factor(__ldg(stat_in), &nf); inv_r = 1.0f / r_prev; }
+  if (!EXACT && stat_in) { bool nf; r_prev = rescale_factor(__ldg(stat_in), &nf); inv_r = 1.0f / r_prev; }
+  const float2 exact_inv_r = f2(1.0f / exact_r);
   const int n_vec = d / VEC;
   const int t = threadIdx.x % TEAM;
   const int team = threadIdx.x / TEAM;
@@ -537,6 +568,28 @@ __global__ void __launch_bounds__(kLnThreads, 2) layernorm_bwd_kernel(
 #pragma unroll
           for (int h = 0; h < HP; ++h) o[h] = __ffma2_rn(g[v][h], k_g, __ffma2_rn(x[v][h], k_n, k_0));
           uint32_t ow[OB / 4 > 0 ? OB / 4 : 1];
+          if constexpr (EXACT) {
+            // the value the plain call would have stored in the intermediate (one rounding to XDT), its
+            // statistic, and the rebalanced output: an exact division by a power of two, then one rounding
+            if constexpr (XDT != SCALIFY_F32) {
+              uint32_t iw[4];
+              encode_pairs<XDT, VEC>(o, iw);
+              decode_pairs<XDT, VEC>(iw, o);
+            }
+            if (stat == SCALIFY_STAT_AMAX) {
+#pragma unroll
+              for (int h = 0; h < HP; ++h) amax = __vimax3_u32(amax, abs_bits(o[h].x), abs_bits(o[h].y));
+            } else if (stat == SCALIFY_STAT_L2) {
+#pragma unroll
+              for (int h = 0; h < HP; ++h) ssq2 = __ffma2_rn(o[h], o[h], ssq2);
+            }
+            float2 q[HP];
+#pragma unroll
+            for (int h = 0; h < HP; ++h) q[h] = __fmul2_rn(o[h], exact_inv_r);
+            encode_pairs<DXDT, VEC>(q, ow);
+            st_raw<OB>(orow + v * (TEAM * OB), ow);
+            continue;
+          }
           encode_pairs<DXDT, VEC>(o, ow);
           st_raw<OB>(orow + v * (TEAM * OB), ow);
           if (stat == SCALIFY_STAT_AMAX) {
@@ -603,7 +656,7 @@ __global__ void __launch_bounds__(kLnThreads, 2) layernorm_bwd_kernel(
     __shared__ double s_stat[kLnThreads / 32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     // AMAX: of the stored values (plain call) or of the un-rebalanced, unrounded ones (delayed: times r, exact)
-    if (stat == SCALIFY_STAT_AMAX)
+    if (stat == SCALIFY_STAT_AMAX && !EXACT)  // (EXACT: the maximum is already that of the rounded intermediate values)
       amax = stat_in ? abs_bits(__uint_as_float(amax) * r_prev) : abs_bits(round_through<DXDT>(__uint_as_float(amax)));
     double mine = (stat == SCALIFY_STAT_AMAX)
                       ? static_cast<double>(warp_max_u32(amax))
@@ -626,8 +679,12 @@ __global__ void __launch_bounds__(1024) layernorm_bwd_finalize_kernel(
     int nblocks, int R, int d, const float* __restrict__ dgamma_part, const float* __restrict__ dbeta_part,
     const double* __restrict__ stat_part, int stat, float* stat_word, void* __restrict__ dgamma,
     void* __restrict__ dbeta, const float* g_scale, const float* x_scale, const float* gamma_scale,
-    float* dx_scale, float* dgamma_scale, float* dbeta_scale, const float* stat_in, uint32_t* status) {
+    float* dx_scale, float* dgamma_scale, float* dbeta_scale, const float* stat_in, uint32_t* status,
+    float* exact_hint) {
   asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
+  // exact_hint != nullptr: the one-pass dynamic rescale.  The output scale carries the power of two of THIS
+  // call's statistic (the second launch of the main kernel makes the data agree with it), and the statistic is
+  // left in *exact_hint as the next call's prediction.
   // block = 8 columns (one 32-byte sector of a partial row) x 128 slices of the block list: 4 x as many
   // blocks as a 32-column layout, so the partials (a few MB in L2) are read by more SMs at once
   __shared__ float s_a[128][9], s_b[128][9];
@@ -665,6 +722,7 @@ __global__ void __launch_bounds__(1024) layernorm_bwd_finalize_kernel(
     float r_prev = 1.0f;
     if (stat_in) { bool nf; r_prev = rescale_factor(*stat_in, &nf); }
     __syncwarp();
+    float result = 0.f;
     if (stat != SCALIFY_STAT_NONE) {
       double tot = 0.0;
       for (int i = cx; i < nblocks; i += 32) {
@@ -678,7 +736,6 @@ __global__ void __launch_bounds__(1024) layernorm_bwd_finalize_kernel(
         tot = warp_sum_f64(tot);
       }
       if (cx == 0) {
-        float result;
         if (stat == SCALIFY_STAT_AMAX) result = __uint_as_float(static_cast<uint32_t>(tot));
         else result = static_cast<float>(sqrt(tot / (static_cast<double>(R) * static_cast<double>(d))));
         *stat_word = result;
@@ -687,6 +744,12 @@ __global__ void __launch_bounds__(1024) layernorm_bwd_finalize_kernel(
     if (cx == 0) {
       const float gs = load_scale(g_scale), xs = load_scale(x_scale), gms = load_scale(gamma_scale);
       uint32_t flags = (is_pow2_scale(gs) && is_pow2_scale(xs) && is_pow2_scale(gms)) ? 0u : SCALIFY_DEV_BAD_SCALE;
+      if (exact_hint) {
+        bool nonfinite;
+        r_prev = rescale_factor(result, &nonfinite);
+        if (nonfinite) flags |= SCALIFY_DEV_NONFINITE_STAT;
+        *exact_hint = result;
+      }
       if (dx_scale) *dx_scale = gs * gms / xs * r_prev;
       if (dgamma_scale) *dgamma_scale = gs * kfactor(R);
       if (dbeta_scale) *dbeta_scale = gs * kfactor(R);
@@ -733,7 +796,8 @@ int launch_layernorm_bwd(const void* G, int64_t g_ld, const void* X, int x_dt, i
                          int64_t dx_ld, int R, int d, const void* gamma, int gb_dt, const float* mean,
                          const float* rinv, float eps, int eps_inside, int stat, void* dgamma, void* dbeta, int dg_dt,
                          const float* g_scale, const float* x_scale, const float* gamma_scale, float* dx_scale,
-                         float* dgamma_scale, float* dbeta_scale, const float* stat_in, void* ws, cudaStream_t st) {
+                         float* dgamma_scale, float* dbeta_scale, const float* stat_in, int exact, void* ws,
+                         cudaStream_t st) {
   const LnBwdPlan plan = ln_bwd_plan(R, d, x_dt);
   if (!plan.ok) return SCALIFY_ERR_UNSUPPORTED;
   const int tw = plan.tw, grid = plan.grid;
@@ -744,18 +808,78 @@ int launch_layernorm_bwd(const void* G, int64_t g_ld, const void* X, int x_dt, i
   float* dgp = dgamma ? dg_part : nullptr;
   float* dbp = dgamma ? db_part : nullptr;
   constexpr int kBwdSmem = kLnBwdStages * 2 * kLnVpt * kLnThreads * 16;
+  if (exact) {
+    // one-pass dynamic rescale: first launch with the predicted power of two, finalize (statistic, scale words,
+    // next prediction), second launch as a programmatic dependent that returns at once if the prediction held
+    if (dx_dt != SCALIFY_E4M3 && dx_dt != SCALIFY_E5M2) return SCALIFY_ERR_UNSUPPORTED;
+    LnBwdPredict pred;
+    pred.hint = reinterpret_cast<const float*>(static_cast<char*>(ws) + 56);
+    pred.r_used = reinterpret_cast<float*>(static_cast<char*>(ws) + 52);
+    pred.stat_word = v.stat;
+    const int fgrid = dgamma ? (d + 7) / 8 : 1;
+#define SCALIFY_LN_BWD_EXACT(W)                                                                                  \
+  do {                                                                                                           \
+    auto kernel = layernorm_bwd_kernel<XDT, DXDT, W, true>;                                                      \
+    static DeviceOnce once; /* per instantiation and device */                                                   \
+    int rc_once = device_once(once, nullptr, [&](int*) {                                                         \
+      SCALIFY_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmem));     \
+      return int(SCALIFY_OK);                                                                                    \
+    });                                                                                                          \
+    if (rc_once) return rc_once;                                                                                 \
+    pred.redo = 0;                                                                                               \
+    kernel<<<grid, kLnThreads, kBwdSmem, st>>>(G, g_ld, X, x_ld, dX, dx_ld, R, d, gamma, gb_dt, mean, rinv, eps, \
+                                               eps_inside, stat, nullptr, dgp, dbp, st_part, pred);              \
+    SCALIFY_CUDA_TRY(cudaGetLastError());                                                                        \
+    SCALIFY_DISPATCH_WIDE(dg_dt, DGDT,                                                                           \
+        layernorm_bwd_finalize_kernel<DGDT><<<fgrid, 1024, 0, st>>>(grid, R, d, dgp, dbp, st_part, stat, v.stat, \
+            dgamma, dbeta, g_scale, x_scale, gamma_scale, dx_scale, dgamma_scale, dbeta_scale, nullptr, v.status, \
+            reinterpret_cast<float*>(static_cast<char*>(ws) + 56)));                                             \
+    SCALIFY_CUDA_TRY(cudaGetLastError());                                                                        \
+    pred.redo = 1;                                                                                               \
+    cudaLaunchConfig_t cfg = {};                                                                                 \
+    cudaLaunchAttribute attr[1];                                                                                 \
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;                                             \
+    attr[0].val.programmaticStreamSerializationAllowed = 1;                                                      \
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(kLnThreads); cfg.dynamicSmemBytes = kBwdSmem; cfg.stream = st; \
+    cfg.attrs = attr; cfg.numAttrs = 1;                                                                          \
+    SCALIFY_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, G, g_ld, X, x_ld, dX, dx_ld, R, d, gamma, gb_dt, mean,     \
+                                        rinv, eps, eps_inside, stat, static_cast<const float*>(nullptr), dgp,   \
+                                        dbp, st_part, pred));                                                    \
+  } while (0)
+    SCALIFY_DISPATCH_WIDE(x_dt, XDT, {
+      if (dx_dt == SCALIFY_E4M3) {
+        constexpr int DXDT = SCALIFY_E4M3;
+        switch (tw) {
+          case 1: SCALIFY_LN_BWD_EXACT(1); break;
+          case 2: SCALIFY_LN_BWD_EXACT(2); break;
+          case 4: SCALIFY_LN_BWD_EXACT(4); break;
+          default: SCALIFY_LN_BWD_EXACT(8); break;
+        }
+      } else {
+        constexpr int DXDT = SCALIFY_E5M2;
+        switch (tw) {
+          case 1: SCALIFY_LN_BWD_EXACT(1); break;
+          case 2: SCALIFY_LN_BWD_EXACT(2); break;
+          case 4: SCALIFY_LN_BWD_EXACT(4); break;
+          default: SCALIFY_LN_BWD_EXACT(8); break;
+        }
+      }
+    });
+#undef SCALIFY_LN_BWD_EXACT
+    return SCALIFY_OK;
+  }
 #define SCALIFY_LN_BWD(W)                                                                                        \
   do {                                                                                                           \
     static DeviceOnce once; /* per instantiation and device */                                                   \
     int rc_once = device_once(once, nullptr, [&](int*) {                                                         \
-      SCALIFY_CUDA_TRY(cudaFuncSetAttribute(layernorm_bwd_kernel<XDT, DXDT, W>,                                  \
+      SCALIFY_CUDA_TRY(cudaFuncSetAttribute(layernorm_bwd_kernel<XDT, DXDT, W, false>,                           \
                                             cudaFuncAttributeMaxDynamicSharedMemorySize, kBwdSmem));             \
       return int(SCALIFY_OK);                                                                                    \
     });                                                                                                          \
     if (rc_once) return rc_once;                                                                                 \
-    layernorm_bwd_kernel<XDT, DXDT, W><<<grid, kLnThreads, kBwdSmem, st>>>(                                      \
+    layernorm_bwd_kernel<XDT, DXDT, W, false><<<grid, kLnThreads, kBwdSmem, st>>>(                               \
         G, g_ld, X, x_ld, dX, dx_ld, R, d, gamma, gb_dt, mean, rinv, eps, eps_inside, stat, stat_in, dgp, dbp,   \
-        st_part);                                                                                                \
+        st_part, LnBwdPredict{});                                                                                \
   } while (0)
   SCALIFY_DISPATCH_WIDE(x_dt, XDT, SCALIFY_DISPATCH_DTYPE(dx_dt, DXDT, {
     switch (tw) {
@@ -771,7 +895,7 @@ int launch_layernorm_bwd(const void* G, int64_t g_ld, const void* X, int x_dt, i
   SCALIFY_DISPATCH_WIDE(dg_dt, DGDT,
       layernorm_bwd_finalize_kernel<DGDT><<<fgrid, 1024, 0, st>>>(grid, R, d, dgp, dbp, st_part, stat, v.stat, dgamma,
                                                                  dbeta, g_scale, x_scale, gamma_scale, dx_scale,
-                                                                 dgamma_scale, dbeta_scale, stat_in, v.status));
+                                                                 dgamma_scale, dbeta_scale, stat_in, v.status, nullptr));
   SCALIFY_CUDA_TRY(cudaGetLastError());
   return SCALIFY_OK;
 }

@@ -297,11 +297,19 @@ static int layernorm_bwd_impl(const scalify_array* G, const scalify_array* X, co
   if (rc) return rc;
   rc = check_array(X);
   if (rc) return rc;
+  // dX == NULL with an FP8 dXq: the one-pass form of the dynamic rescale (the intermediate is not stored)
+  const bool one_pass = dX == nullptr && dXq != nullptr && !stat_in;
+  if (one_pass) {
+    rc = check_array(dXq);
+    if (rc) return rc;
+    if (is_wide(dXq->dtype)) return SCALIFY_ERR_DTYPE;
+    dX = dXq;  // shape, layout and scale word checks below apply to the array that is written
+  }
   rc = check_array(dX);
   if (rc) return rc;
   if (!mean || !rinv) return SCALIFY_ERR_NULL;
   // the plain call keeps the un-rebalanced gradient in a wide format; the delayed one may round it once to FP8
-  if (!is_wide(X->dtype) || G->dtype != X->dtype || (!stat_in && !is_wide(dX->dtype))) return SCALIFY_ERR_DTYPE;
+  if (!is_wide(X->dtype) || G->dtype != X->dtype || (!stat_in && !one_pass && !is_wide(dX->dtype))) return SCALIFY_ERR_DTYPE;
   if (!valid_stat(stat_dx)) return SCALIFY_ERR_VALUE;
   int64_t R, d, x_ld, Rg, dg, g_ld, Rd, dd, dx_ld;
   if (as_rows(X, &R, &d, &x_ld) || as_rows(G, &Rg, &dg, &g_ld) || as_rows(dX, &Rd, &dd, &dx_ld)) return SCALIFY_ERR_SHAPE;
@@ -325,7 +333,10 @@ static int layernorm_bwd_impl(const scalify_array* G, const scalify_array* X, co
     if (dgamma->ndim != 1 || dgamma->shape[0] != d || dbeta->ndim != 1 || dbeta->shape[0] != d) return SCALIFY_ERR_SHAPE;
     dg_dt = dgamma->dtype;
   }
-  if (dXq) {
+  if (one_pass) {
+    if (stat_dx == SCALIFY_STAT_NONE) return SCALIFY_ERR_VALUE;
+    if (contiguous_numel(dXq) != R * d) return SCALIFY_ERR_SHAPE;
+  } else if (dXq) {
     rc = check_array(dXq);
     if (rc) return rc;
     if (stat_dx == SCALIFY_STAT_NONE) return SCALIFY_ERR_VALUE;
@@ -344,9 +355,9 @@ static int layernorm_bwd_impl(const scalify_array* G, const scalify_array* X, co
                             eps_inside_sqrt ? 1 : 0, stat_dx, dgamma ? dgamma->data : nullptr,
                             dbeta ? dbeta->data : nullptr, dg_dt, G->scale, X->scale, gamma ? gamma->scale : nullptr,
                             dx_scale, dgamma ? dgamma->scale : nullptr, dbeta ? dbeta->scale : nullptr, stat_in,
-                            workspace, st);
+                            one_pass ? 1 : 0, workspace, st);
   if (rc) return rc;
-  if (dXq) {
+  if (dXq && !one_pass) {
     WsView v = ws_view(workspace);
     rc = launch_rebalance(dX->data, dX->dtype, dXq->data, dXq->dtype, R * d, dx_scale, dXq->scale, v.stat, nullptr,
                           kModeDynamic, v.status, st);

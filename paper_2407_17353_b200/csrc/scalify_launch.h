@@ -43,7 +43,8 @@ int launch_layernorm_bwd(const void* G, int64_t g_ld, const void* X, int x_dt, i
                          int64_t dx_ld, int R, int d, const void* gamma, int gb_dt, const float* mean,
                          const float* rinv, float eps, int eps_inside, int stat, void* dgamma, void* dbeta, int dg_dt,
                          const float* g_scale, const float* x_scale, const float* gamma_scale, float* dx_scale,
-                         float* dgamma_scale, float* dbeta_scale, const float* stat_in, void* ws, cudaStream_t st);
+                         float* dgamma_scale, float* dbeta_scale, const float* stat_in, int exact, void* ws,
+                         cudaStream_t st);
 size_t adam_ws_bytes(int64_t n_tensors);
 // Every scale word the step WRITES (m, v, w, w_cast of every tensor) must be a different word, and none of them a
 // gradient's scale word: the kernels read and write them concurrently.  `scratch` holds 4 * n_tensors pointers.

@@ -165,6 +165,20 @@ def test_layernorm_backward_with_gradient_rescale_on_benchmarked_launch_shapes(R
     qo, qs, _ = orc.rescale(got, BF, dx_scale, stat, orc.E5M2)
     assert dXq.scale_value() == qs
     assert np.array_equal(to_bits(dXq.data, orc.E5M2), qo)
+    # the one-pass form (dX = None) on the same launch shape: first with nothing to predict from (its second
+    # launch writes the gradient again), then with the right prediction; the same bits as above both times
+    ws1 = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_LAYERNORM_BWD, R, d))
+    for _ in range(2):
+        q1 = sc.ScaledTensor.empty((R, d), torch.float8_e5m2)
+        dg1, db1 = sc.ScaledTensor.empty((d,), torch.float32), sc.ScaledTensor.empty((d,), torch.float32)
+        sc.scalify_scaled_layernorm_bwd(G, X, gamma, mean, rinv, None, ws1, eps=EPS, stat_dx=stat, dXq=q1, dgamma=dg1,
+                                        dbeta=db1)
+        assert ws1.check_status() == 0
+        assert torch.equal(ws1.statistic().view(torch.int32), ws.statistic().view(torch.int32))
+        assert q1.scale_value() == qs
+        assert torch.equal(q1.data.view(torch.uint8), dXq.data.view(torch.uint8))
+        assert torch.equal(dg1.data.view(torch.int32), dg.data.view(torch.int32))
+        assert torch.equal(db1.data.view(torch.int32), db.data.view(torch.int32))
 
 
 DELAYED_CASES = [
