@@ -269,6 +269,13 @@ int scalify_statistic(const scalify_array* X, int stat, float* out_stat,
  *
  * Y->scale may alias X->scale for the dynamic and delayed forms (in-place
  * rebalance of a state tensor).
+ *
+ * The dynamic form with an output buffer of its own reads X once when the power
+ * of two can be predicted: while the statistic is gathered, Y is already written
+ * with the power of two of the statistic this workspace saw last (fp32 word at
+ * byte offset 56 of the workspace, any content), and X is read a second time
+ * only if this call's statistic has another power of two.  Y, Y_s and the
+ * statistic word do not depend on that word; the call leaves its statistic there.
  */
 int scalify_rescale(const scalify_array* X, int stat, const float* new_scale, const float* stat_in,
                     scalify_array* Y, void* workspace, size_t workspace_bytes, void* stream);

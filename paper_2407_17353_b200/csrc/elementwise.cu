@@ -336,6 +336,154 @@ int launch_rebalance_check(const void* x, int in_dt, void* y, int out_dt, int64_
 }
 
 // ---------------------------------------------------------------------------------------------
+// dynamic rescale with a predicted power of two (Section 3.3: statistic and rebalancing are separate
+// primitives): the array is read ONCE
+// ---------------------------------------------------------------------------------------------
+// While the statistic is gathered (as statistic_kernel does: one partial per block, the block that draws the
+// last ticket combines them in index order), the output is already written with the power of two of the
+// statistic the workspace saw last (*hint, any content).  rebalance_check_kernel follows as a programmatic
+// dependent: it writes the scale word and the next prediction and returns at once when this call's statistic
+// has the predicted power of two; otherwise it rebalances from x as usual.  Either way every element is
+// computed as cast(x / r) with the same r, so the result does not depend on the prediction.
+template <int IN, int OUT>
+__global__ void __launch_bounds__(kThreads) rescale_predict_kernel(const void* __restrict__ x, void* __restrict__ y,
+                                                                   int64_t n, int stat, const float* hint,
+                                                                   float* r_used, double* __restrict__ partials,
+                                                                   uint32_t* ticket, float* stat_word) {
+  bool nf;
+  const float pred_r = rescale_factor(*reinterpret_cast<const volatile float*>(hint), &nf);
+  if (blockIdx.x == 0 && threadIdx.x == 0) *r_used = pred_r;
+  asm volatile("griddepcontrol.launch_dependents;");  // the dependent sets up while this grid runs
+  const float factor = 1.0f / pred_r;  // exact: a power of two
+  constexpr int VEC = VecElems<IN, OUT>::v;
+  constexpr int IB = VEC * ElemBytes<IN>::v, OB = VEC * ElemBytes<OUT>::v;
+  const int64_t n_vec = n / VEC;
+  uint32_t amax = 0u;
+  float ssq = 0.f;
+  // every block takes one contiguous run of vectors; the runs differ by at most one vector
+  const int64_t v0 = n_vec / gridDim.x * blockIdx.x + min(int64_t(blockIdx.x), int64_t(n_vec % gridDim.x));
+  const int64_t v1 = v0 + n_vec / gridDim.x + (blockIdx.x < n_vec % gridDim.x ? 1 : 0);
+  for (int64_t base = v0; base < v1; base += kThreads * kUnroll) {
+    uint32_t w[kUnroll][IB / 4];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const int64_t i = base + u * kThreads + threadIdx.x;
+      if (i < v1) {
+        ld_raw_stream<IB>(static_cast<const char*>(x) + i * IB, w[u]);
+      } else {
+#pragma unroll
+        for (int q = 0; q < IB / 4; ++q) w[u][q] = 0u;
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const int64_t i = base + u * kThreads + threadIdx.x;
+      float f[VEC];
+      decode_vec<IN, VEC>(w[u], f);
+      if (stat == SCALIFY_STAT_AMAX) {
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) amax = max(amax, abs_bits(f[e]));
+      } else {
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) ssq = fmaf(f[e], f[e], ssq);
+      }
+      if (i < v1) {
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) f[e] *= factor;
+        uint32_t o[OB / 4];
+        encode_vec<OUT, VEC>(f, o);
+        st_raw_stream<OB>(static_cast<char*>(y) + i * OB, o);
+      }
+    }
+  }
+  if (blockIdx.x == 0 && threadIdx.x < static_cast<int>(n - n_vec * VEC)) {
+    const int64_t i = n_vec * VEC + threadIdx.x;
+    const float f = load_elem<IN>(x, i);
+    amax = max(amax, abs_bits(f));
+    ssq = fmaf(f, f, ssq);
+    store_elem<OUT>(y, i, f * factor);
+  }
+  __shared__ double s_part[kThreads / 32];
+  __shared__ bool s_last;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  double mine;
+  if (stat == SCALIFY_STAT_AMAX) mine = static_cast<double>(warp_max_u32(amax));
+  else mine = warp_sum_f64(static_cast<double>(ssq));
+  if (lane == 0) s_part[warp] = mine;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double tot;
+    if (stat == SCALIFY_STAT_AMAX) {
+      uint32_t m = 0u;
+      for (int i = 0; i < kThreads / 32; ++i) m = max(m, static_cast<uint32_t>(s_part[i]));
+      tot = static_cast<double>(m);
+    } else {
+      tot = 0.0;
+      for (int i = 0; i < kThreads / 32; ++i) tot += s_part[i];
+    }
+    partials[blockIdx.x] = tot;
+    __threadfence();
+    const uint32_t t = atomicAdd(ticket, 1u);
+    s_last = (t == gridDim.x - 1);
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  // fixed-order combination of the per-block partials
+  double acc = 0.0;
+  uint32_t accm = 0u;
+  for (int i = threadIdx.x; i < static_cast<int>(gridDim.x); i += kThreads) {
+    const double p = __ldcg(&partials[i]);
+    if (stat == SCALIFY_STAT_AMAX) accm = max(accm, static_cast<uint32_t>(p));
+    else acc += p;
+  }
+  if (stat == SCALIFY_STAT_AMAX) acc = static_cast<double>(warp_max_u32(accm));
+  else acc = warp_sum_f64(acc);
+  __syncthreads();
+  if (lane == 0) s_part[warp] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float result;
+    if (stat == SCALIFY_STAT_AMAX) {
+      uint32_t m = 0u;
+      for (int i = 0; i < kThreads / 32; ++i) m = max(m, static_cast<uint32_t>(s_part[i]));
+      result = __uint_as_float(m);
+    } else {
+      double tot = 0.0;
+      for (int i = 0; i < kThreads / 32; ++i) tot += s_part[i];
+      result = static_cast<float>(sqrt(tot / static_cast<double>(n)));
+    }
+    *stat_word = result;
+    *ticket = 0u;
+  }
+}
+
+// Returns SCALIFY_OK after the two launches, or 1 if this pair of formats has no predicted form.
+int launch_rescale_predicted(const void* x, int in_dt, void* y, int out_dt, int64_t n, int stat, const float* x_scale,
+                             float* y_scale, void* ws, size_t ws_bytes, cudaStream_t st) {
+  if ((in_dt != SCALIFY_BF16 && in_dt != SCALIFY_F16) || (out_dt != SCALIFY_E4M3 && out_dt != SCALIFY_E5M2)) return 1;
+  WsView v = ws_view(ws);
+  int64_t grid = statistic_blocks_wanted(n, elem_size(in_dt));
+  const int64_t room = static_cast<int64_t>((ws_bytes - kWsHeader) / sizeof(double));
+  if (grid > room) grid = room;
+  if (grid < 1) grid = 1;
+  float* hint = reinterpret_cast<float*>(static_cast<char*>(ws) + 56);
+  float* r_used = reinterpret_cast<float*>(static_cast<char*>(ws) + 52);
+#define SCALIFY_RP(IN, OUT)                                                                                     \
+  rescale_predict_kernel<IN, OUT><<<static_cast<int>(grid), kThreads, 0, st>>>(x, y, n, stat, hint, r_used,     \
+                                                                              static_cast<double*>(v.area),     \
+                                                                              v.ticket, v.stat)
+  if (in_dt == SCALIFY_BF16) {
+    if (out_dt == SCALIFY_E4M3) SCALIFY_RP(SCALIFY_BF16, SCALIFY_E4M3); else SCALIFY_RP(SCALIFY_BF16, SCALIFY_E5M2);
+  } else {
+    if (out_dt == SCALIFY_E4M3) SCALIFY_RP(SCALIFY_F16, SCALIFY_E4M3); else SCALIFY_RP(SCALIFY_F16, SCALIFY_E5M2);
+  }
+#undef SCALIFY_RP
+  SCALIFY_CUDA_TRY(cudaGetLastError());
+  return launch_rebalance_check(x, in_dt, y, out_dt, n, x_scale, y_scale, v.stat, r_used, hint, v.status, st);
+}
+
+// ---------------------------------------------------------------------------------------------
 // dynamic rescale in one cooperative launch (Section 3.3): statistic, grid barrier, rebalance
 // ---------------------------------------------------------------------------------------------
 // Every block owns one contiguous run of vectors.  Phase 1 reads the run front to back with the

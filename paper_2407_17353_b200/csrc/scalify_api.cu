@@ -192,6 +192,18 @@ int scalify_rescale(const scalify_array* X, int stat, const float* new_scale, co
   }
   rc = check_ws(workspace, workspace_bytes, kWsMin);
   if (rc) return rc;
+  // BF16 / F16 into an FP8 buffer of its own: the array is read once, the output written with the predicted
+  // power of two, and a check launch repairs it if the prediction failed
+  {
+    const char* xb = static_cast<const char*>(X->data);
+    const char* yb = static_cast<const char*>(Y->data);
+    const bool disjoint = yb + n * elem_size(Y->dtype) <= xb || xb + n * elem_size(X->dtype) <= yb;
+    if (disjoint && !(Y->scale && Y->scale == X->scale)) {
+      rc = launch_rescale_predicted(X->data, X->dtype, Y->data, Y->dtype, n, stat, X->scale, Y->scale, workspace,
+                                    workspace_bytes, st);
+      if (rc <= 0) return rc;
+    }
+  }
   // one cooperative launch (statistic, grid barrier, rebalance); two launches where the device
   // cannot run a cooperative grid
   rc = launch_fused_rescale(X->data, X->dtype, Y->data, Y->dtype, n, stat, X->scale, Y->scale, workspace,

@@ -21,6 +21,8 @@ enum { kModeCast = 0, kModeDynamic = 1, kModeSet = 2 };
 int64_t statistic_blocks_wanted(int64_t n, int elem_bytes);
 int launch_statistic(const void* x, int dtype, int64_t n, int stat, void* ws, size_t ws_bytes, float* out_stat,
                      cudaStream_t st);
+int launch_rescale_predicted(const void* x, int in_dt, void* y, int out_dt, int64_t n, int stat, const float* x_scale,
+                             float* y_scale, void* ws, size_t ws_bytes, cudaStream_t st);
 int launch_fused_rescale(const void* x, int in_dt, void* y, int out_dt, int64_t n, int stat, const float* x_scale,
                          float* y_scale, void* ws, size_t ws_bytes, cudaStream_t st);
 int launch_rebalance(const void* x, int in_dt, void* y, int out_dt, int64_t n, const float* x_scale, float* y_scale,

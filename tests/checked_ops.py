@@ -103,14 +103,22 @@ class Ops:
             assert np.array_equal(self.take(Y, rows), o.encode(o.decode(self.take(X, rows), code(X.data)), dt))
         return Y
 
-    def rescale(self, X, stat, dt):
-        """Dynamic rescale (statistic -> power of two -> rebalance)."""
+    def rescale(self, X, stat, dt, key=None):
+        """Dynamic rescale (statistic -> power of two -> rebalance).  key: a workspace of its own for this call
+        site, so that the power of two predicted from the site's previous statistic holds step after step."""
         Y = self.empty(X.data.shape, dt)
-        sc.scalify_rescale(X, Y, stat=stat, ws=self.ws)
+        ws = self.ws
+        if key is not None:
+            if not hasattr(self, "ws_rescale"):
+                self.ws_rescale = {}
+            if key not in self.ws_rescale:
+                self.ws_rescale[key] = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_RESCALE, X.data.numel(), 0), self.dev)
+            ws = self.ws_rescale[key]
+        sc.scalify_rescale(X, Y, stat=stat, ws=ws)
         self.calls += 2
         if self.check:
             o = self.orc
-            self._status_ok()
+            assert ws.check_status() == 0
             so = o.statistic(self.bits(X).reshape(-1), code(X.data), stat)      # always over the whole array
             if stat == sc.STAT_L2 and abs(np.log2(so) - round(np.log2(so))) < 1e-5:
                 return Y  # binade edge: either neighbouring scale is correct

@@ -106,7 +106,7 @@ class ScaledGPT:
         dx = o.mm(dy8, W8, transB=True)               # dy W^T: W stored [K, N] = [N', K'] of this product
         # x^T dy with fused AMAX rescale; a workspace per weight, so that the predicted rescale holds step after step
         _, dW = o.mm(x8, dy8, transA=True, stat=sc.STAT_AMAX, q_dt=E5, key=name)
-        db = o.rescale(o.colsum(dy8), sc.STAT_AMAX, E5)                    # column sums, then the dynamic rescale
+        db = o.rescale(o.colsum(dy8), sc.STAT_AMAX, E5, key=name + ".bias")   # column sums, then the dynamic rescale
         return dx, dW, db
 
     # ------------------------------------------------------------------ one training step
@@ -212,11 +212,11 @@ class ScaledGPT:
             dx = o.add(dx, dln)
         o.active = True
         dwte_emb, dwpe = o.embedding_bwd(ids, T, dx, c.vocab)
-        grads["wte"] = o.rescale(o.add(dwte_head, dwte_emb), sc.STAT_AMAX, E5)
-        grads["wpe"] = o.rescale(dwpe, sc.STAT_AMAX, E5)
+        grads["wte"] = o.rescale(o.add(dwte_head, dwte_emb), sc.STAT_AMAX, E5, key="wte")
+        grads["wpe"] = o.rescale(dwpe, sc.STAT_AMAX, E5, key="wpe")
         for k in list(grads):
             if grads[k].data.dtype != torch.float8_e5m2:                              # LayerNorm dgamma / dbeta (F32)
-                grads[k] = o.rescale(grads[k], sc.STAT_AMAX, E5)
+                grads[k] = o.rescale(grads[k], sc.STAT_AMAX, E5, key=k)
         self.last_grads = grads
 
         # ---------------- optimizer

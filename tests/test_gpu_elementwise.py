@@ -74,6 +74,39 @@ def test_dynamic_rescale_many_tiles_per_block(stat, in_dt, out_dt, in_place):
     assert np.array_equal(to_bits(Y.data, out_dt), yo)
 
 
+@pytest.mark.parametrize("n", [1000, 70001, 8 * 1024 * 700 + 13])
+@pytest.mark.parametrize("stat", [sc.STAT_AMAX, sc.STAT_L2])
+@pytest.mark.parametrize("in_dt,out_dt", [(orc.BF16, orc.E4M3), (orc.F32, orc.E5M2), (orc.BF16, orc.BF16)])
+def test_dynamic_rescale_does_not_depend_on_the_prediction(n, stat, in_dt, out_dt):
+    """The one-launch dynamic rescale writes its output while it gathers the statistic, with the power of two of
+    the statistic the workspace saw last, and reads the input again only if that was wrong.  Whatever the word
+    holds - nothing, the right statistic, another binade, infinity, NaN, a negative number - output, scale and
+    statistic are the oracle's."""
+    base = si.normal(36, n, (n,), 5.0).astype(np.float32)
+    ws = new_ws()
+    for mult, hint in [(1.0, None), (1.0, None), (64.0, None), (1.0 / 4096, None), (1.0, float("inf")),
+                       (1.0, float("nan")), (1.0, -3.0), (1.7, None), (1.7, 0.0)]:
+        x = si.to_bits(base * np.float32(mult), in_dt)
+        X = st(x, in_dt, 2.0 ** -5)
+        Y = sc.ScaledTensor.empty((n,), sc.TORCH_DTYPE[out_dt])
+        Y.data.view(torch.uint8).fill_(0x55)
+        if hint is not None:
+            ws.prediction().fill_(hint)
+        sc.scalify_rescale(X, Y, stat=stat, ws=ws)
+        assert ws.check_status() == 0
+        yo, ys, so = orc.rescale(x, in_dt, 2.0 ** -5, stat, out_dt)
+        got_stat = float(ws.statistic().item())
+        if stat == sc.STAT_AMAX:
+            assert got_stat == so
+        else:
+            assert abs(got_stat - so) <= 2e-6 * so
+            assert abs(math.log2(so) - round(math.log2(so))) > 1e-5, "seed lands on a binade edge: pick another"
+        assert Y.scale_value() == ys, (mult, hint)
+        assert np.array_equal(to_bits(Y.data, out_dt), yo), (mult, hint)
+        if in_dt != orc.F32 and out_dt != orc.BF16:   # the pairs of formats that have the predicted form
+            assert float(ws.prediction().item()) == got_stat
+
+
 @pytest.mark.parametrize("in_dt", [orc.E4M3, orc.E5M2, orc.F16, orc.BF16, orc.F32])
 def test_statistic_kernel(in_dt):
     n = 3 * 256 * 64 + 11
