@@ -230,6 +230,12 @@ def run_profile_row(args):
         ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_MATMUL, n, n), dev)
         fn = lambda t: sc.scalify_scaled_matmul(A, Bt, Y, ws, transB=True, stat=sc.STAT_AMAX, Yq=Yq)
         work = {"flop": 2.0 * n ** 3}
+    elif row == "mx_quantize_t":
+        n = N_GEMM
+        Xa = sc.ScaledTensor.make(rnd((n, n), torch.bfloat16, 1), 1.0)
+        Amt = sc.MxTensor(n, n, device=dev, transposed=True)
+        fn = lambda t: sc.scalify_mx_quantize(Xa, Amt)
+        work = {"bytes": n * n * (3.0 + 1.0 / 32)}
     elif row == "mx":
         n = N_GEMM
         Xa = sc.ScaledTensor.make(rnd((n, n), torch.bfloat16, 1), 1.0)
@@ -268,7 +274,7 @@ def run_profile_row(args):
         Yq = sc.ScaledTensor.empty((n,), torch.float8_e4m3fn, dev)
         ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_RESCALE, n), dev)
         fn = lambda t: sc.scalify_rescale(X, Yq, stat=sc.STAT_AMAX, ws=ws)
-        work = {"bytes": 5.0 * n}
+        work = {"bytes": 3.0 * n}   # read once, written once
     elif row == "add":
         n = 8192 * 8192
         P = sc.ScaledTensor.make(rnd((n,), torch.bfloat16, 1), 1.0)
@@ -276,7 +282,7 @@ def run_profile_row(args):
         S = sc.ScaledTensor.empty((n,), torch.bfloat16, dev)
         fn = lambda t: sc.scalify_scaled_add(P, Q, S)
         work = {"bytes": 6.0 * n}
-    elif row == "layernorm":
+    elif row in ("layernorm", "layernorm_onepass"):
         R, d = 65536, 1024
         X = sc.ScaledTensor.make(rnd((R, d), torch.bfloat16, 3), 1.0)
         G = sc.ScaledTensor.make(rnd((R, d), torch.bfloat16, 4), 2.0 ** -10)
@@ -291,11 +297,19 @@ def run_profile_row(args):
         db = sc.ScaledTensor.empty((d,), torch.float32, dev)
         ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_LAYERNORM_BWD, R, d), dev)
 
-        def fn(t):
+        if row == "layernorm":
+            def fn(t):
+                sc.scalify_scaled_layernorm(X, gamma, beta, LY, eps=1e-5, mean=mean, rinv=rinv)
+                sc.scalify_scaled_layernorm_bwd(G, X, gamma, mean, rinv, dX, ws, eps=1e-5, stat_dx=sc.STAT_L2, dXq=dXq,
+                                                dgamma=dg, dbeta=db)
+            work = {"bytes": 13.0 * R * d}
+        else:   # the backward with the exact rescale in one pass (dX = None)
             sc.scalify_scaled_layernorm(X, gamma, beta, LY, eps=1e-5, mean=mean, rinv=rinv)
-            sc.scalify_scaled_layernorm_bwd(G, X, gamma, mean, rinv, dX, ws, eps=1e-5, stat_dx=sc.STAT_L2, dXq=dXq,
-                                            dgamma=dg, dbeta=db)
-        work = {"bytes": 13.0 * R * d}
+
+            def fn(t):
+                sc.scalify_scaled_layernorm_bwd(G, X, gamma, mean, rinv, None, ws, eps=1e-5, stat_dx=sc.STAT_L2,
+                                                dXq=dXq, dgamma=dg, dbeta=db)
+            work = {"bytes": 5.0 * R * d}
     else:
         n = 64 * 1024 * 1024
         ag = sc.ScaledTensor.make(rnd((n,), torch.float8_e5m2, 7), 2.0 ** -12)
@@ -473,7 +487,8 @@ def main():
                     help="print one JSON line per size of the HBM-bound rows (LayerNorm, rescale, add) instead of the step")
     ap.add_argument("--no-next", action="store_true",
                     help="skip the separately timed next-row variants f1, f2 (for ncu launch lists of the step)")
-    ap.add_argument("--profile-row", default=None, choices=["matmul", "headline", "mx", "attention", "attention_bwd", "rescale", "add", "layernorm", "adam"],
+    ap.add_argument("--profile-row", default=None, choices=["matmul", "headline", "mx", "mx_quantize_t", "attention", "attention_bwd", "rescale", "add", "layernorm",
+                             "layernorm_onepass", "adam"],
                     help="run only this row on a reduced, still larger-than-L2 case (for ncu captures)")
     ap.add_argument("--gpt-step", action="store_true",
                     help="time the config-5 step (GPT-2-small shapes) instead; with --graph replayed from a CUDA graph")
