@@ -357,8 +357,9 @@ __global__ void __launch_bounds__(kThreads) rescale_predict_kernel(const void* _
   const float factor = 1.0f / pred_r;  // exact: a power of two
   constexpr int VEC = VecElems<IN, OUT>::v;
   constexpr int IB = VEC * ElemBytes<IN>::v, OB = VEC * ElemBytes<OUT>::v;
+  static_assert(ElemBytes<IN>::v == 2, "the packed maximum below is for 16-bit inputs");
   const int64_t n_vec = n / VEC;
-  uint32_t amax = 0u;
+  uint32_t amax = 0u, pmax = 0u;
   float ssq = 0.f;
   // every block takes one contiguous run of vectors; the runs differ by at most one vector
   const int64_t v0 = n_vec / gridDim.x * blockIdx.x + min(int64_t(blockIdx.x), int64_t(n_vec % gridDim.x));
@@ -381,8 +382,9 @@ __global__ void __launch_bounds__(kThreads) rescale_predict_kernel(const void* _
       float f[VEC];
       decode_vec<IN, VEC>(w[u], f);
       if (stat == SCALIFY_STAT_AMAX) {
+        // magnitudes compare as unsigned integers on the raw 16-bit patterns, two elements per instruction
 #pragma unroll
-        for (int e = 0; e < VEC; ++e) amax = max(amax, abs_bits(f[e]));
+        for (int q = 0; q < IB / 4; ++q) pmax = __vmaxu2(pmax, w[u][q] & 0x7FFF7FFFu);
       } else {
 #pragma unroll
         for (int e = 0; e < VEC; ++e) ssq = fmaf(f[e], f[e], ssq);
@@ -402,6 +404,13 @@ __global__ void __launch_bounds__(kThreads) rescale_predict_kernel(const void* _
     amax = max(amax, abs_bits(f));
     ssq = fmaf(f, f, ssq);
     store_elem<OUT>(y, i, f * factor);
+  }
+  {
+    // the larger 16-bit pattern, widened to the fp32 bit pattern of the same value
+    const uint32_t h = max(pmax & 0xFFFFu, pmax >> 16);
+    const uint32_t wide = IN == SCALIFY_BF16 ? h << 16
+                                             : __float_as_uint(__half2float(__ushort_as_half(static_cast<unsigned short>(h))));
+    amax = max(amax, wide);
   }
   __shared__ double s_part[kThreads / 32];
   __shared__ bool s_last;
