@@ -38,15 +38,18 @@ namespace scalify {
 
 constexpr int kAttQ = 128;     // queries per CTA
 constexpr int kAttK = 128;     // keys per block
-constexpr int kAttHd = 64;     // head dimension (bytes per row of Q, K, V)
+constexpr int kAttHd = 64;     // bytes per row of a Q, K or V tile: a head dimension of 128 travels as two such tiles
 constexpr int kAttSmWarps = 8;   // softmax warps: two per TMEM lane quarter, each taking half of the key columns
 constexpr int kAttThreads = 32 * (kAttSmWarps + 1);
 constexpr int kAttTmemCols = 256;
 constexpr uint32_t kAttOCol = 128;
 constexpr int kAttKvStages = 3;
 constexpr int kAttTileBytes = kAttK * kAttHd;  // 8 KB: a Q, K or V tile
-constexpr size_t kAttSmem = size_t(kAttTileBytes) * (1 + 2 * kAttKvStages) /*Q, K ring, V ring*/ +
-                            2 * kAttQ * kAttK /*two P tiles*/ + 1024 + 256;
+// NH = head dimension / 64: every Q, K, V tile is NH column halves of 8 KB, one after the other
+constexpr size_t att_smem(int nh) {
+  return size_t(kAttTileBytes) * nh * (1 + 2 * kAttKvStages) /*Q, K ring, V ring*/ + 2 * kAttQ * kAttK /*two P tiles*/ +
+         1024 + 256;
+}
 
 struct AttParams {
   int heads, h_inner, Tq, Tk, q_blocks;   // heads = batch x h_inner
@@ -88,7 +91,7 @@ __device__ __forceinline__ float exp2_neg(float x) {
   return r;
 }
 
-template <int ODT>
+template <int ODT, int NH>
 __global__ void __launch_bounds__(kAttThreads, 2)
 attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                      const __grid_constant__ CUtensorMap map_v, const AttParams p) {
@@ -97,11 +100,12 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (base - raw);
+  constexpr int kTile = NH * kAttTileBytes;  // a Q, K or V tile: NH column halves of [128 rows][64 B]
   const uint32_t smem_q = base;
-  const uint32_t smem_k = base + kAttTileBytes;                              // kAttKvStages slots
-  const uint32_t smem_v = base + (1 + kAttKvStages) * kAttTileBytes;         // kAttKvStages slots
-  const uint32_t smem_p = base + (1 + 2 * kAttKvStages) * kAttTileBytes;     // 2 x 16 KB, 1024-byte aligned
-  uint8_t* p_tiles = smem + (1 + 2 * kAttKvStages) * kAttTileBytes;
+  const uint32_t smem_k = base + kTile;                              // kAttKvStages slots
+  const uint32_t smem_v = base + (1 + kAttKvStages) * kTile;         // kAttKvStages slots
+  const uint32_t smem_p = base + (1 + 2 * kAttKvStages) * kTile;     // 2 x 16 KB, 1024-byte aligned
+  uint8_t* p_tiles = smem + (1 + 2 * kAttKvStages) * kTile;
   uint8_t* bar_mem = p_tiles + 2 * kAttQ * kAttK;
   const uint32_t bars = smem_p + 2 * kAttQ * kAttK;
   const uint32_t q_full = bars, kv_full = bars + 8 /*3*/, kv_empty = bars + 32 /*3*/, s_full = bars + 56,
@@ -155,12 +159,16 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         const bool sweep_b = j >= n_kb;
         const int kb = sweep_b ? j - n_kb : j;
         const uint32_t fb = kv_full + 8 * slot;
-        mbar_expect_tx(fb, sweep_b ? 2 * kAttTileBytes : kAttTileBytes);
-        tma_load_4d(smem_k + slot * kAttTileBytes, &map_k, fb, 0, kb * kAttK, hh, bb);
-        if (sweep_b) tma_load_4d(smem_v + slot * kAttTileBytes, &map_v, fb, 0, kb * kAttK, hh, bb);
+        mbar_expect_tx(fb, sweep_b ? 2 * kTile : kTile);
+#pragma unroll
+        for (int h = 0; h < NH; ++h) {
+          tma_load_4d(smem_k + slot * kTile + h * kAttTileBytes, &map_k, fb, h * kAttHd, kb * kAttK, hh, bb);
+          if (sweep_b) tma_load_4d(smem_v + slot * kTile + h * kAttTileBytes, &map_v, fb, h * kAttHd, kb * kAttK, hh, bb);
+        }
       };
-      mbar_expect_tx(q_full, kAttTileBytes);
-      tma_load_4d(smem_q, &map_q, q_full, 0, q0, hh, bb);
+      mbar_expect_tx(q_full, kTile);
+#pragma unroll
+      for (int h = 0; h < NH; ++h) tma_load_4d(smem_q + h * kAttTileBytes, &map_q, q_full, h * kAttHd, q0, hh, bb);
       issue_load(0);
       if (!timed_out && n_it > 1) issue_load(1);
       if (!timed_out && !mbar_wait(q_full, 0u, abort_flag)) timed_out = true;
@@ -171,11 +179,13 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         if (!mbar_wait(kv_full + 8 * slot, (j / kAttKvStages) & 1, abort_flag)) { timed_out = true; return; }
         if (j >= 1 && !mbar_wait(s_empty, (j - 1) & 1, abort_flag)) { timed_out = true; return; }
         tc_fence_after();
-        const uint64_t k_desc = make_smem_desc_sw64(smem_k + slot * kAttTileBytes, 512u);
+        const uint64_t k_desc = make_smem_desc_sw64(smem_k + slot * kTile, 512u);
 #pragma unroll
-        for (int k = 0; k < kAttHd / 32; ++k)  // K = 32 bytes per MMA: +32 B on both K-major operands
-          umma_f8(tmem_base, q_desc + static_cast<uint64_t>(k * 2), k_desc + static_cast<uint64_t>(k * 2),
-                  p.idesc_s, k != 0 ? 1u : 0u);
+        for (int h = 0; h < NH; ++h)  // the contraction runs over the column halves ...
+#pragma unroll
+          for (int k = 0; k < kAttHd / 32; ++k)  // ... K = 32 bytes per MMA: +32 B on both K-major operands
+            umma_f8(tmem_base, q_desc + static_cast<uint64_t>(h * (kAttTileBytes >> 4) + k * 2),
+                    k_desc + static_cast<uint64_t>(h * (kAttTileBytes >> 4) + k * 2), p.idesc_s, (h | k) != 0 ? 1u : 0u);
         umma_commit(s_full);
         if (j < n_kb) umma_commit(kv_empty + 8 * slot);  // sweep A: the K tile is free after Q K^T
       };
@@ -191,11 +201,14 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           // P tile [128 queries][128 B of keys], K-major; V tile [128 keys][64 B]: the B operand in MN-major form,
           // 8-key atoms 512 B apart, 32 keys per MMA
           const uint64_t p_desc = make_smem_desc(smem_p + pb * (kAttQ * kAttK), 0u, 1024u);
-          const uint64_t v_desc = make_smem_desc_sw64(smem_v + slot * kAttTileBytes, 512u);
+          const uint64_t v_desc = make_smem_desc_sw64(smem_v + slot * kTile, 512u);
 #pragma unroll
-          for (int k = 0; k < kAttK / 32; ++k)
-            umma_f8(tmem_base + kAttOCol, p_desc + static_cast<uint64_t>(k * 2),
-                    v_desc + static_cast<uint64_t>(k * (32 * kAttHd / 16)), p.idesc_pv, (b | k) != 0 ? 1u : 0u);
+          for (int h = 0; h < NH; ++h)  // 64 columns of O per column half of V
+#pragma unroll
+            for (int k = 0; k < kAttK / 32; ++k)
+              umma_f8(tmem_base + kAttOCol + h * kAttHd, p_desc + static_cast<uint64_t>(k * 2),
+                      v_desc + static_cast<uint64_t>(h * (kAttTileBytes >> 4) + k * (32 * kAttHd / 16)), p.idesc_pv,
+                      (b | k) != 0 ? 1u : 0u);
           umma_commit(p_empty + 8 * pb);
           umma_commit(kv_empty + 8 * slot);
         }
@@ -408,7 +421,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       tc_fence_after();
       constexpr int OSZ = ElemBytes<ODT>::v;
 #pragma unroll 1
-      for (int c = half; c < half + 1; ++c) {
+      for (int c = half; c < 2 * NH; c += 2) {  // 32 of the row's 64 * NH columns at a time
         uint32_t acc[32];
         tmem_ld32(t_row + kAttOCol + c * 32, acc);
         tmem_ld_wait();
@@ -471,16 +484,23 @@ int launch_attention(const AttentionArgs& a, cudaStream_t st) {
   p.sc_const = kfactor(a.hd) * a.sm_scale * 1.4426950408889634f;
   const long long ctas = static_cast<long long>(p.heads) * p.q_blocks;
   if (ctas > 0x7FFFFFFF) return SCALIFY_ERR_SHAPE;
+#define SCALIFY_ATT_LAUNCH(NH)                                                                                   \
+  do {                                                                                                           \
+    auto kernel = attention_fwd_kernel<ODT, NH>;                                                                 \
+    static DeviceOnce once; /* one per instantiation: the attribute belongs to this kernel on this device */     \
+    int rc_once = device_once(once, nullptr, [&](int*) {                                                         \
+      SCALIFY_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,                 \
+                                            int(att_smem(NH))));                                                 \
+      return int(SCALIFY_OK);                                                                                    \
+    });                                                                                                          \
+    if (rc_once) return rc_once;                                                                                 \
+    kernel<<<static_cast<unsigned>(ctas), kAttThreads, att_smem(NH), st>>>(map_q, map_k, map_v, p);              \
+  } while (0)
   SCALIFY_DISPATCH_WIDE(a.o_dt, ODT, {
-    auto kernel = attention_fwd_kernel<ODT>;
-    static DeviceOnce once;  // (one per instantiation: the attribute belongs to this kernel on this device)
-    int rc_once = device_once(once, nullptr, [&](int*) {
-      SCALIFY_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kAttSmem)));
-      return int(SCALIFY_OK);
-    });
-    if (rc_once) return rc_once;
-    kernel<<<static_cast<unsigned>(ctas), kAttThreads, kAttSmem, st>>>(map_q, map_k, map_v, p);
+    if (a.hd == 64) SCALIFY_ATT_LAUNCH(1);
+    else SCALIFY_ATT_LAUNCH(2);
   });
+#undef SCALIFY_ATT_LAUNCH
   SCALIFY_CUDA_TRY(cudaGetLastError());
   return SCALIFY_OK;
 }

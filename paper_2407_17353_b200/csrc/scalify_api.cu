@@ -506,7 +506,7 @@ int scalify_scaled_attention(const scalify_array* Q, const scalify_array* K, con
   const int64_t tq = vq.rows, tk = vk.rows, hq = vq.batch * vq.heads;
   if (tq < 1 || tk < 1 || vq.heads < 1 || vq.batch < 1 || tq > 0x7FFFFFFF || tk > 0x7FFFFFFF || hq > 0x7FFFFFFF)
     return SCALIFY_ERR_SHAPE;
-  if (vq.cols != 64 || (causal && tk < tq)) return SCALIFY_ERR_UNSUPPORTED;
+  if ((vq.cols != 64 && vq.cols != 128) || (causal && tk < tq)) return SCALIFY_ERR_UNSUPPORTED;
   a.q_ld = vq.ld; a.q_hs = vq.hs; a.q_bs = vq.bs; a.k_ld = vk.ld; a.k_hs = vk.hs; a.k_bs = vk.bs;
   a.v_ld = vv.ld; a.v_hs = vv.hs; a.v_bs = vv.bs; a.o_ld = vo.ld; a.o_hs = vo.hs; a.o_bs = vo.bs;
   if (O->scale && (O->scale == Q->scale || O->scale == K->scale || O->scale == V->scale)) return SCALIFY_ERR_ALIAS;
@@ -528,7 +528,7 @@ int scalify_scaled_attention(const scalify_array* Q, const scalify_array* K, con
   a.q_dt = Q->dtype; a.k_dt = K->dtype; a.v_dt = V->dtype;
   a.O = O->data; a.o_dt = O->dtype;
   a.batch = static_cast<int>(vq.batch); a.heads = static_cast<int>(vq.heads);
-  a.Tq = static_cast<int>(tq); a.Tk = static_cast<int>(tk); a.hd = 64;
+  a.Tq = static_cast<int>(tq); a.Tk = static_cast<int>(tk); a.hd = static_cast<int>(vq.cols);
   a.causal = causal ? 1 : 0;
   a.sm_scale = sm_scale;
   a.q_scale = Q->scale; a.k_scale = K->scale; a.v_scale = V->scale; a.o_scale = O->scale;

@@ -20,7 +20,7 @@ HD = 64
 
 
 def run_case(H, Tq, Tk, causal, merged_layout=False, q_dt=orc.E4M3, v_dt=orc.E4M3, o_dt=orc.BF16, seed=1,
-             check_heads=None, c=0.125):
+             check_heads=None, c=0.125, HD=HD):
     qs, ks, vs = 2.0 ** -1, 2.0 ** 1, 2.0 ** -3
     q = si.to_bits(si.normal(seed, 1, (H, Tq, HD), 1.0), q_dt)
     k = si.to_bits(si.normal(seed, 2, (H, Tk, HD), 1.0), orc.E4M3)
@@ -98,6 +98,18 @@ def test_other_softmax_scales(c):
 
 def test_heads_inside_a_token_major_buffer_and_mixed_formats():
     run_case(4, 256, 256, True, merged_layout=True, q_dt=orc.E5M2, v_dt=orc.E5M2, o_dt=orc.F16)
+
+
+@pytest.mark.parametrize("H,Tq,Tk,causal", [(2, 128, 128, True), (3, 384, 384, True), (2, 200, 224, True),
+                                            (2, 128, 384, False), (1, 1024, 1024, True)])
+def test_head_dimension_128(H, Tq, Tk, causal):
+    """Rows of 128 elements travel as two 64-byte column halves per tile: the scores accumulate over both, the
+    output has 64 columns per half."""
+    run_case(H, Tq, Tk, causal, HD=128, c=2.0 ** -3.5 if Tq == 200 else 0.125)
+
+
+def test_head_dimension_128_inside_a_token_major_buffer_and_mixed_formats():
+    run_case(3, 256, 256, True, merged_layout=True, q_dt=orc.E5M2, v_dt=orc.E5M2, o_dt=orc.F16, HD=128)
 
 
 def test_benchmark_shape_96_heads_of_1024_tokens_sampled_heads():
