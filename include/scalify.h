@@ -599,7 +599,7 @@ int scalify_scaled_colsum(const scalify_array* X, scalify_array* Y, void* worksp
  * i.e. scalify_scaled_matmul, scalify_scalar_mul_pow2, scalify_scaled_softmax,
  * scalify_scaled_matmul.  The softmax is the exact two-sweep form (row maximum
  * and sum first, then the normalised probabilities), not an online rescaling.
- *   Q [heads, Tq, hd], K, V [heads, Tk, hd]: E4M3 or E5M2, hd = 64, 3-D views
+ *   Q [heads, Tq, hd], K, V [heads, Tk, hd]: E4M3 or E5M2, hd = 64 or 128, 3-D views
  *   (row and head strides in stride[1], stride[0]; 2-D arrays are one head; 4-D
  *   arrays [batch, heads, T, hd] add a batch stride in front, so that the token-major
  *   buffers [batch * T, heads * hd] of a transformer are covered by ONE call);
@@ -632,7 +632,7 @@ int scalify_scaled_attention(const scalify_array* Q, const scalify_array* K, con
  * and three more scalify_scaled_matmul.  Two launches: one CTA per (head, 128
  * queries) forms dP (twice, it never reaches memory), dS and dQ; one CTA per
  * (head, 128 keys) contracts P and dS over the queries into dV and dK.
- *   Q, dO [heads, Tq, hd], K, V [heads, Tk, hd]: E4M3 or E5M2, hd = 64, 3-D views
+ *   Q, dO [heads, Tq, hd], K, V [heads, Tk, hd]: E4M3 or E5M2, hd = 64 or 128, 3-D views
  *   as for the forward call.  P: E4M3, dense [heads, Tq, Tk], non-negative (the
  *   sign bit is ignored), exact zeros where the mask hides a key.  dS (output): E5M2, dense [heads, Tq, Tk], scale word
  *   required; with causal != 0 the 128 x 128 blocks wholly above the diagonal are

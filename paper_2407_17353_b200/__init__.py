@@ -501,7 +501,7 @@ def scalify_scaled_attention(Q: ScaledTensor, K: ScaledTensor, V: ScaledTensor, 
                              causal: bool = True, S_dump: Optional[ScaledTensor] = None,
                              P_dump: Optional[ScaledTensor] = None, status: Optional[torch.Tensor] = None,
                              stream=None) -> None:
-    """Fused attention forward over [heads, T, 64] FP8 views; S_dump / P_dump are optional debug copies."""
+    """Fused attention forward over [heads, T, hd] FP8 views (hd = 64 or 128); S_dump / P_dump are optional debug copies."""
     q, k, v, o, sd, pd = _desc(Q), _desc(K), _desc(V), _desc(O), _desc(S_dump), _desc(P_dump)
     _check(lib().scalify_scaled_attention(_ref(q), _ref(k), _ref(v), float(sm_scale), int(bool(causal)), _ref(o),
                                           _ref(sd), _ref(pd), _ptr(status), _stream(stream)),

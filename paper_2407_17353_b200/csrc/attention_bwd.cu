@@ -31,13 +31,14 @@ namespace scalify {
 
 constexpr int kBwQ = 128;      // queries per block
 constexpr int kBwK = 128;      // keys per block
-constexpr int kBwHd = 64;      // head dimension
-constexpr int kBwTile = kBwK * kBwHd;        // 8 KB: a Q, K, V or dO tile
+constexpr int kBwHd = 64;      // bytes per row of a Q, K, V or dO tile: a head dimension of 128 travels as two such tiles
+constexpr int kBwTile = kBwK * kBwHd;        // 8 KB: one column half of a Q, K, V or dO tile
 constexpr int kBwPTile = kBwQ * kBwK;        // 16 KB: a P or dS tile
 constexpr int kBwSmWarps = 8;
 constexpr int kBw1Threads = 32 * (kBwSmWarps + 1);
-constexpr int kBw1Slot = 2 * kBwTile + kBwPTile;  // V, K, P of one key block
-constexpr size_t kBw1Smem = size_t(kBwTile) + 2 * kBw1Slot + kBwPTile + 1024 + 256;
+// NH = head dimension / 64 column halves per tile
+__host__ __device__ constexpr int bw1_slot(int nh) { return 2 * nh * kBwTile + kBwPTile; }  // V, K, P of one key block
+__host__ __device__ constexpr size_t bw1_smem(int nh) { return size_t(nh) * kBwTile + 2 * bw1_slot(nh) + kBwPTile + 1024 + 256; }
 constexpr int kBw1TmemCols = 256;
 constexpr uint32_t kBw1DqCol = 128;
 
@@ -86,7 +87,7 @@ __device__ __forceinline__ void bf16_round_pair(uint32_t a_bits, uint32_t b_bits
   b = __uint_as_float(packed & 0xFFFF0000u);
 }
 
-template <int GDT>
+template <int GDT, int NH>
 __global__ void __launch_bounds__(kBw1Threads, 2)
 attention_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_do, const __grid_constant__ CUtensorMap map_v,
                         const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_p,
@@ -96,11 +97,13 @@ attention_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_do, const __grid
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (base - raw);
+  constexpr int kTile = NH * kBwTile;         // a dO, V or K tile: NH column halves of [128 rows][64 B]
+  constexpr int kBw1Slot = bw1_slot(NH);
   const uint32_t smem_do = base;
-  const uint32_t smem_slot = base + kBwTile;                       // 2 slots: [V 8 KB | K 8 KB | P 16 KB]
-  const uint32_t smem_ds = base + kBwTile + 2 * kBw1Slot;          // 16 KB, 1024-byte aligned
-  uint8_t* slot_mem = smem + kBwTile;
-  uint8_t* ds_tile = smem + kBwTile + 2 * kBw1Slot;
+  const uint32_t smem_slot = base + kTile;                       // 2 slots: [V | K | P 16 KB]
+  const uint32_t smem_ds = base + kTile + 2 * kBw1Slot;          // 16 KB, 1024-byte aligned
+  uint8_t* slot_mem = smem + kTile;
+  uint8_t* ds_tile = smem + kTile + 2 * kBw1Slot;
   uint8_t* bar_mem = ds_tile + kBwPTile;
   const uint32_t bars = smem_ds + kBwPTile;
   const uint32_t do_full = bars, kv_full = bars + 8 /*2*/, kv_empty = bars + 24 /*2*/, s_full = bars + 40,
@@ -159,13 +162,17 @@ attention_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_do, const __grid
         const int kb = sweep_b ? it - n_kb : it;
         const uint32_t fb = kv_full + 8 * slot;
         const uint32_t s0 = smem_slot + slot * kBw1Slot;
-        mbar_expect_tx(fb, (sweep_b ? 2 * kBwTile : kBwTile) + kBwPTile);
-        tma_load_4d(s0, &map_v, fb, 0, kb * kBwK, hh, bb);
-        if (sweep_b) tma_load_4d(s0 + kBwTile, &map_k, fb, 0, kb * kBwK, hh, bb);
-        tma_load_3d(s0 + 2 * kBwTile, &map_p, fb, kb * kBwK, q0, head);
+        mbar_expect_tx(fb, (sweep_b ? 2 * kTile : kTile) + kBwPTile);
+#pragma unroll
+        for (int h = 0; h < NH; ++h) {
+          tma_load_4d(s0 + h * kBwTile, &map_v, fb, h * kBwHd, kb * kBwK, hh, bb);
+          if (sweep_b) tma_load_4d(s0 + kTile + h * kBwTile, &map_k, fb, h * kBwHd, kb * kBwK, hh, bb);
+        }
+        tma_load_3d(s0 + 2 * kTile, &map_p, fb, kb * kBwK, q0, head);
       };
-      mbar_expect_tx(do_full, kBwTile);
-      tma_load_4d(smem_do, &map_do, do_full, 0, q0, hh, bb);
+      mbar_expect_tx(do_full, kTile);
+#pragma unroll
+      for (int h = 0; h < NH; ++h) tma_load_4d(smem_do + h * kBwTile, &map_do, do_full, h * kBwHd, q0, hh, bb);
       issue_load(0);
       if (!timed_out && !mbar_wait(do_full, 0u, abort_flag)) timed_out = true;
       const uint64_t do_desc = bw_desc_sw64(smem_do, 512u);
@@ -180,9 +187,11 @@ attention_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_do, const __grid
         const uint32_t s0 = smem_slot + slot * kBw1Slot;
         const uint64_t v_desc = bw_desc_sw64(s0, 512u);
 #pragma unroll
-        for (int k = 0; k < kBwHd / 32; ++k)  // dP = dO V^T: both operands K-major, 32 bytes of hd per MMA
-          umma_f8(tmem_base, do_desc + static_cast<uint64_t>(k * 2), v_desc + static_cast<uint64_t>(k * 2), p.idesc_dp,
-                  k != 0 ? 1u : 0u);
+        for (int h = 0; h < NH; ++h)  // dP = dO V^T over the column halves ...
+#pragma unroll
+          for (int k = 0; k < kBwHd / 32; ++k)  // ... both operands K-major, 32 bytes of hd per MMA
+            umma_f8(tmem_base, do_desc + static_cast<uint64_t>(h * (kBwTile >> 4) + k * 2),
+                    v_desc + static_cast<uint64_t>(h * (kBwTile >> 4) + k * 2), p.idesc_dp, (h | k) != 0 ? 1u : 0u);
         umma_commit(s_full);
         if (it < n_kb) {
           umma_commit(kv_empty + 8 * slot);  // sweep A: V is free after dO V^T (P: the row threads arrive)
@@ -191,11 +200,14 @@ attention_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_do, const __grid
           if (!mbar_wait(p_full, b & 1, abort_flag)) { timed_out = true; break; }
           tc_fence_after();
           // K tile [128 keys][64 B]: the B operand in MN-major form (keys are the contraction), 32 keys per MMA
-          const uint64_t k_desc = bw_desc_sw64(s0 + kBwTile, 512u);
+          const uint64_t k_desc = bw_desc_sw64(s0 + kTile, 512u);
 #pragma unroll
-          for (int k = 0; k < kBwK / 32; ++k)
-            umma_f8(tmem_base + kBw1DqCol, ds_desc + static_cast<uint64_t>(k * 2),
-                    k_desc + static_cast<uint64_t>(k * (32 * kBwHd / 16)), p.idesc_dq, (b | k) != 0 ? 1u : 0u);
+          for (int h = 0; h < NH; ++h)  // 64 columns of dQ per column half of K
+#pragma unroll
+            for (int k = 0; k < kBwK / 32; ++k)
+              umma_f8(tmem_base + kBw1DqCol + h * kBwHd, ds_desc + static_cast<uint64_t>(k * 2),
+                      k_desc + static_cast<uint64_t>(h * (kBwTile >> 4) + k * (32 * kBwHd / 16)), p.idesc_dq,
+                      (b | k) != 0 ? 1u : 0u);
           umma_commit(p_empty);
           umma_commit(kv_empty + 8 * slot);
         }
@@ -233,7 +245,7 @@ attention_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_do, const __grid
       if (!mbar_wait(s_full, it & 1, abort_flag)) { timed_out = true; break; }
       if (!mbar_wait(kv_full + 8 * slot, (it >> 1) & 1, abort_flag)) { timed_out = true; break; }  // the P tile
       tc_fence_after();
-      const uint8_t* p_tile = slot_mem + slot * kBw1Slot + 2 * kBwTile;
+      const uint8_t* p_tile = slot_mem + slot * kBw1Slot + 2 * kTile;
       uint32_t acc[32];
 #pragma unroll 1
       for (int c = c_first; c < c_first + kChunks; ++c) {
@@ -282,7 +294,7 @@ attention_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_do, const __grid
       tc_fence_after();
       // the previous block's dS K must have read the tile before it is overwritten
       if (kb >= 1 && !mbar_wait(p_empty, (kb - 1) & 1, abort_flag)) { timed_out = true; break; }
-      const uint8_t* p_tile = slot_mem + slot * kBw1Slot + 2 * kBwTile;
+      const uint8_t* p_tile = slot_mem + slot * kBw1Slot + 2 * kTile;
       uint32_t acc[32];
 #pragma unroll 1
       for (int c = c_first; c < c_first + kChunks; ++c) {
@@ -322,21 +334,24 @@ attention_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_do, const __grid
     if (!timed_out && mbar_wait(o_full, 0u, abort_flag)) {
       tc_fence_after();
       constexpr int GSZ = ElemBytes<GDT>::v;
-      uint32_t acc[32];
-      tmem_ld32(t_row + kBw1DqCol + half * 32, acc);
-      tmem_ld_wait();
-      if (i < p.Tq) {
-        float v[32];
+#pragma unroll 1
+      for (int c = half; c < 2 * NH; c += 2) {  // 32 of the row's 64 * NH columns at a time
+        uint32_t acc[32];
+        tmem_ld32(t_row + kBw1DqCol + c * 32, acc);
+        tmem_ld_wait();
+        if (i < p.Tq) {
+          float v[32];
 #pragma unroll
-        for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(acc[e]) * p.inv_kf_tk;
-        uint32_t o[32 * GSZ / 4];
-        encode_vec<GDT, 32>(v, o);
-        uint4* dst = reinterpret_cast<uint4*>(static_cast<char*>(p.dQ) +
-                                              (static_cast<long long>(bb) * p.dq_bs + static_cast<long long>(hh) * p.dq_hs +
-                                               static_cast<long long>(i) * p.dq_ld +
-                                               half * 32) * GSZ);
+          for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(acc[e]) * p.inv_kf_tk;
+          uint32_t o[32 * GSZ / 4];
+          encode_vec<GDT, 32>(v, o);
+          uint4* dst = reinterpret_cast<uint4*>(static_cast<char*>(p.dQ) +
+                                                (static_cast<long long>(bb) * p.dq_bs + static_cast<long long>(hh) * p.dq_hs +
+                                                 static_cast<long long>(i) * p.dq_ld +
+                                                 c * 32) * GSZ);
 #pragma unroll
-        for (int q = 0; q < 32 * GSZ / 16; ++q) dst[q] = make_uint4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
+          for (int q = 0; q < 32 * GSZ / 16; ++q) dst[q] = make_uint4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
+        }
       }
     } else {
       timed_out = true;
@@ -356,16 +371,17 @@ attention_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_do, const __grid
 // launch 2: dV = P^T dO and dK = dS^T Q for one (head, block of 128 keys)
 // ---------------------------------------------------------------------------------------------
 constexpr int kBw2Threads = 192;   // warp 0: TMA, warp 1: MMA, warps 2-5: read-out
-constexpr int kBw2Stages = 2;
+__host__ __device__ constexpr int bw2_stages(int nh) { return nh == 1 ? 2 : 3; }  // (a third slot for 128: at most two CTAs fit an SM then,
+                                                              // as many as the 256 accumulator columns each allow)
 constexpr int kBw2Q = 64;          // queries per ring slot: short slots, so that four CTAs fit an SM and their
                                    // prologues and read-outs overlap the others' loads
 constexpr int kBw2PTile = kBw2Q * kBwK;    // 8 KB: 64 queries x 128 keys of P or dS
-constexpr int kBw2Tile = kBw2Q * kBwHd;    // 4 KB: 64 rows of dO or Q
-constexpr int kBw2Stage = 2 * kBw2PTile + 2 * kBw2Tile;  // 24 KB
-constexpr size_t kBw2Smem = size_t(kBw2Stages) * kBw2Stage + 1024 + 256;
-constexpr int kBw2TmemCols = 128;  // dV: columns 0-63, dK: columns 64-127
+constexpr int kBw2Tile = kBw2Q * kBwHd;    // 4 KB: one column half of 64 rows of dO or Q
+__host__ __device__ constexpr int bw2_stage(int nh) { return 2 * kBw2PTile + 2 * nh * kBw2Tile; }  // 24 KB / 32 KB
+__host__ __device__ constexpr size_t bw2_smem(int nh) { return size_t(bw2_stages(nh)) * bw2_stage(nh) + 1024 + 256; }
+// TMEM: dV in columns [0, 64 NH), dK in [64 NH, 128 NH)
 
-template <int GDT>
+template <int GDT, int NH>
 __global__ void __launch_bounds__(kBw2Threads, 4)
 attention_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_ds,
                          const __grid_constant__ CUtensorMap map_do, const __grid_constant__ CUtensorMap map_q,
@@ -375,6 +391,8 @@ attention_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (base - raw);
+  constexpr int kBw2Stages = bw2_stages(NH), kBw2Stage = bw2_stage(NH), kBw2TmemCols = 128 * NH;
+  constexpr int kTile2 = NH * kBw2Tile;  // a dO or Q tile of 64 rows: NH column halves
   uint8_t* bar_mem = smem + kBw2Stages * kBw2Stage;
   const uint32_t bars = base + kBw2Stages * kBw2Stage;
   const uint32_t full_bar = bars, empty_bar = bars + 8 * kBw2Stages, acc_full = bars + 16 * kBw2Stages;
@@ -424,8 +442,11 @@ attention_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
         mbar_expect_tx(fb, kBw2Stage);
         tma_load_3d(s0, &map_p, fb, kb * kBwK, q0, head);
         tma_load_3d(s0 + kBw2PTile, &map_ds, fb, kb * kBwK, q0, head);
-        tma_load_4d(s0 + 2 * kBw2PTile, &map_do, fb, 0, q0, hh, bb);
-        tma_load_4d(s0 + 2 * kBw2PTile + kBw2Tile, &map_q, fb, 0, q0, hh, bb);
+#pragma unroll
+        for (int h = 0; h < NH; ++h) {
+          tma_load_4d(s0 + 2 * kBw2PTile + h * kBw2Tile, &map_do, fb, h * kBwHd, q0, hh, bb);
+          tma_load_4d(s0 + 2 * kBw2PTile + kTile2 + h * kBw2Tile, &map_q, fb, h * kBwHd, q0, hh, bb);
+        }
       }
     }
   } else if (warp == 1) {
@@ -441,15 +462,21 @@ attention_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
         const uint64_t p_desc = make_smem_desc(s0, 0u, 1024u);
         const uint64_t ds_desc = make_smem_desc(s0 + kBw2PTile, 0u, 1024u);
         const uint64_t do_desc = bw_desc_sw64(s0 + 2 * kBw2PTile, 512u);
-        const uint64_t q_desc = bw_desc_sw64(s0 + 2 * kBw2PTile + kBw2Tile, 512u);
+        const uint64_t q_desc = bw_desc_sw64(s0 + 2 * kBw2PTile + kTile2, 512u);
 #pragma unroll
-        for (int k = 0; k < kBw2Q / 32; ++k)
-          umma_f8(tmem_base, p_desc + static_cast<uint64_t>(k * (32 * 128 / 16)),
-                  do_desc + static_cast<uint64_t>(k * (32 * kBwHd / 16)), p.idesc_dv, (t | k) != 0 ? 1u : 0u);
+        for (int h = 0; h < NH; ++h)  // 64 columns of dV per column half of dO
 #pragma unroll
-        for (int k = 0; k < kBw2Q / 32; ++k)
-          umma_f8(tmem_base + 64, ds_desc + static_cast<uint64_t>(k * (32 * 128 / 16)),
-                  q_desc + static_cast<uint64_t>(k * (32 * kBwHd / 16)), p.idesc_dk, (t | k) != 0 ? 1u : 0u);
+          for (int k = 0; k < kBw2Q / 32; ++k)
+            umma_f8(tmem_base + h * kBwHd, p_desc + static_cast<uint64_t>(k * (32 * 128 / 16)),
+                    do_desc + static_cast<uint64_t>(h * (kBw2Tile >> 4) + k * (32 * kBwHd / 16)), p.idesc_dv,
+                    (t | k) != 0 ? 1u : 0u);
+#pragma unroll
+        for (int h = 0; h < NH; ++h)  // 64 columns of dK per column half of Q
+#pragma unroll
+          for (int k = 0; k < kBw2Q / 32; ++k)
+            umma_f8(tmem_base + (NH + h) * kBwHd, ds_desc + static_cast<uint64_t>(k * (32 * 128 / 16)),
+                    q_desc + static_cast<uint64_t>(h * (kBw2Tile >> 4) + k * (32 * kBwHd / 16)), p.idesc_dk,
+                    (t | k) != 0 ? 1u : 0u);
         umma_commit(empty_bar + 8 * stage);
       }
       if (!timed_out) umma_commit(acc_full);
@@ -463,7 +490,7 @@ attention_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
       tc_fence_after();
       constexpr int GSZ = ElemBytes<GDT>::v;
 #pragma unroll 1
-      for (int c = 0; c < 4; ++c) {  // dV: columns 0-63, dK: columns 64-127
+      for (int c = 0; c < 4 * NH; ++c) {  // dV: the first 64 NH columns, dK: the next 64 NH
         uint32_t acc[32];
         tmem_ld32(t_row + c * 32, acc);
         tmem_ld_wait();
@@ -473,11 +500,12 @@ attention_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_p, const __grid
           for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(acc[e]) * p.inv_kf_tq;
           uint32_t o[32 * GSZ / 4];
           encode_vec<GDT, 32>(v, o);
-          char* out = c < 2 ? static_cast<char*>(p.dV) : static_cast<char*>(p.dK);
-          const long long hs = c < 2 ? p.dv_hs : p.dk_hs, ld = c < 2 ? p.dv_ld : p.dk_ld, bs = c < 2 ? p.dv_bs : p.dk_bs;
+          const bool is_dv = c < 2 * NH;
+          char* out = is_dv ? static_cast<char*>(p.dV) : static_cast<char*>(p.dK);
+          const long long hs = is_dv ? p.dv_hs : p.dk_hs, ld = is_dv ? p.dv_ld : p.dk_ld, bs = is_dv ? p.dv_bs : p.dk_bs;
           uint4* dst = reinterpret_cast<uint4*>(out + (static_cast<long long>(bb) * bs + static_cast<long long>(hh) * hs +
                                                        static_cast<long long>(j) * ld +
-                                                       (c & 1) * 32) * GSZ);
+                                                       (c % (2 * NH)) * 32) * GSZ);
 #pragma unroll
           for (int q = 0; q < 32 * GSZ / 16; ++q) dst[q] = make_uint4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
         }
@@ -544,20 +572,26 @@ int launch_attention_bwd(const AttentionBwdArgs& a, cudaStream_t st) {
   p.status = a.status;
   const long long ctas1 = static_cast<long long>(p.heads) * p.q_blocks, ctas2 = static_cast<long long>(p.heads) * p.k_blocks;
   if (ctas1 > 0x7FFFFFFF || ctas2 > 0x7FFFFFFF) return SCALIFY_ERR_SHAPE;
+#define SCALIFY_ATT_BWD_LAUNCH(NH)                                                                               \
+  do {                                                                                                           \
+    auto k1 = attention_bwd_dq_kernel<GDT, NH>;                                                                  \
+    auto k2 = attention_bwd_dkv_kernel<GDT, NH>;                                                                 \
+    static DeviceOnce once; /* one per instantiation: the attributes belong to these kernels on this device */   \
+    int rc_once = device_once(once, nullptr, [&](int*) {                                                         \
+      SCALIFY_CUDA_TRY(cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, int(bw1_smem(NH)))); \
+      SCALIFY_CUDA_TRY(cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, int(bw2_smem(NH)))); \
+      return int(SCALIFY_OK);                                                                                    \
+    });                                                                                                          \
+    if (rc_once) return rc_once;                                                                                 \
+    k1<<<static_cast<unsigned>(ctas1), kBw1Threads, bw1_smem(NH), st>>>(map_do, map_v, map_k, map_p, p);         \
+    SCALIFY_CUDA_TRY(cudaGetLastError());                                                                        \
+    k2<<<static_cast<unsigned>(ctas2), kBw2Threads, bw2_smem(NH), st>>>(map_p2, map_ds2, map_do2, map_q2, p);    \
+  } while (0)
   SCALIFY_DISPATCH_WIDE(a.g_dt, GDT, {
-    auto k1 = attention_bwd_dq_kernel<GDT>;
-    auto k2 = attention_bwd_dkv_kernel<GDT>;
-    static DeviceOnce once;  // (one per instantiation: the attributes belong to these kernels on this device)
-    int rc_once = device_once(once, nullptr, [&](int*) {
-      SCALIFY_CUDA_TRY(cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kBw1Smem)));
-      SCALIFY_CUDA_TRY(cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kBw2Smem)));
-      return int(SCALIFY_OK);
-    });
-    if (rc_once) return rc_once;
-    k1<<<static_cast<unsigned>(ctas1), kBw1Threads, kBw1Smem, st>>>(map_do, map_v, map_k, map_p, p);
-    SCALIFY_CUDA_TRY(cudaGetLastError());
-    k2<<<static_cast<unsigned>(ctas2), kBw2Threads, kBw2Smem, st>>>(map_p2, map_ds2, map_do2, map_q2, p);
+    if (a.hd == 64) SCALIFY_ATT_BWD_LAUNCH(1);
+    else SCALIFY_ATT_BWD_LAUNCH(2);
   });
+#undef SCALIFY_ATT_BWD_LAUNCH
   SCALIFY_CUDA_TRY(cudaGetLastError());
   return SCALIFY_OK;
 }

@@ -563,7 +563,7 @@ int scalify_scaled_attention_bwd(const scalify_array* Q, const scalify_array* K,
   if (vv.rows != tk || vdo.rows != tq || v1.rows != tq || v2.rows != tk || v3.rows != tk) return SCALIFY_ERR_SHAPE;
   if (tq < 1 || tk < 1 || vq.heads < 1 || vq.batch < 1 || tq > 0x7FFFFFFF || tk > 0x7FFFFFFF || hq > 0x7FFFFFFF)
     return SCALIFY_ERR_SHAPE;
-  if (vq.cols != 64 || (causal && tk < tq)) return SCALIFY_ERR_UNSUPPORTED;
+  if ((vq.cols != 64 && vq.cols != 128) || (causal && tk < tq)) return SCALIFY_ERR_UNSUPPORTED;
   a.q_ld = vq.ld; a.q_hs = vq.hs; a.q_bs = vq.bs; a.k_ld = vk.ld; a.k_hs = vk.hs; a.k_bs = vk.bs;
   a.v_ld = vv.ld; a.v_hs = vv.hs; a.v_bs = vv.bs; a.do_ld = vdo.ld; a.do_hs = vdo.hs; a.do_bs = vdo.bs;
   a.dq_ld = v1.ld; a.dq_hs = v1.hs; a.dq_bs = v1.bs; a.dk_ld = v2.ld; a.dk_hs = v2.hs; a.dk_bs = v2.bs;
@@ -591,7 +591,7 @@ int scalify_scaled_attention_bwd(const scalify_array* Q, const scalify_array* K,
   a.P = P->data; a.dS = dS->data;
   a.dQ = dQ->data; a.dK = dK->data; a.dV = dV->data; a.g_dt = dQ->dtype;
   a.batch = static_cast<int>(vq.batch); a.heads = static_cast<int>(vq.heads);
-  a.Tq = static_cast<int>(tq); a.Tk = static_cast<int>(tk); a.hd = 64;
+  a.Tq = static_cast<int>(tq); a.Tk = static_cast<int>(tk); a.hd = static_cast<int>(vq.cols);
   a.causal = causal ? 1 : 0;
   a.sm_scale = sm_scale;
   a.q_scale = Q->scale; a.k_scale = K->scale; a.v_scale = V->scale; a.p_scale = P->scale; a.do_scale = dO->scale;

@@ -33,7 +33,7 @@ def oracle_probabilities(q, q_dt, qs, k, ks, c, causal):
 
 
 def run_case(H, Tq, Tk, causal, merged_layout=False, q_dt=orc.E4M3, do_dt=orc.E5M2, g_dt=orc.BF16, seed=1,
-             check_heads=None):
+             check_heads=None, HD=HD):
     qs, ks, vs, dos, c = 2.0 ** -1, 2.0 ** 1, 2.0 ** -3, 2.0 ** -9, 0.125
     q = si.to_bits(si.normal(seed, 1, (H, Tq, HD), 1.0), q_dt)
     k = si.to_bits(si.normal(seed, 2, (H, Tk, HD), 1.0), orc.E4M3)
@@ -147,6 +147,18 @@ def test_backward_edge_shapes(H, Tq, Tk, causal):
     # a single partial key block; a length that ends in the middle of a 128-query block (one 64-query ring
     # slot of the dK/dV launch is empty past the end); few queries against many keys; 16 key blocks
     run_case(H, Tq, Tk, causal, seed=7)
+
+
+@pytest.mark.parametrize("H,Tq,Tk,causal", [(2, 128, 128, True), (3, 384, 384, True), (2, 200, 224, True),
+                                            (2, 128, 384, False), (1, 1024, 1024, True), (1, 96, 32, False)])
+def test_backward_head_dimension_128(H, Tq, Tk, causal):
+    """Rows of 128 elements travel as two 64-byte column halves per tile: dP accumulates over both, dQ, dK and dV
+    have 64 columns per half."""
+    run_case(H, Tq, Tk, causal, HD=128)
+
+
+def test_backward_head_dimension_128_inside_a_token_major_buffer_and_mixed_formats():
+    run_case(3, 256, 256, True, merged_layout=True, q_dt=orc.E5M2, do_dt=orc.E4M3, g_dt=orc.F16, HD=128)
 
 
 def test_backward_of_a_single_head_given_as_2d_arrays():
