@@ -399,6 +399,24 @@ int scalify_debug_bf16_round(const float* x, float* y, int64_t n, int two_wide, 
  * made (misses) so far in this process.
  */
 int scalify_debug_host_state_selftest(void);
+
+/*
+ * Bounds-checking build (no counterpart in the paper).  The library built with -DSCALIFY_DEBUG
+ * (`libscalify_debug.so`) checks every global access of its memory-bound kernels that goes through their vector,
+ * row-copy and scalar-tail helpers (the element-wise, LayerNorm, Adam, block-scale quantisation and support
+ * kernels, and the split-K reduction; the tensor-core kernels move their tiles with TMA, which the hardware
+ * bounds by the tensor map) against the byte spans of the arrays and workspaces its entry points have validated
+ * so far.  An access outside all of them is counted, its address kept, and skipped (a load yields zeros), so
+ * nothing faults.  Registration copies a table to the device synchronously: this build is for tests, not for
+ * timing or stream capture.  Spans that touch are merged, and spans are never forgotten until reset.
+ *
+ * scalify_debug_bounds_report: synchronises the device; out[0] = accesses refused since the last report, out[1]
+ * = address of the first, out[2] = its width in bytes; clears the counters.  reset_ranges != 0 also forgets every
+ * registered span.  range_limit >= 0 caps the length of every span registered from now on (a self-test: accesses
+ * past the cap, still inside the caller's buffers, are then refused and reported); -1 lifts the cap.
+ * Returns SCALIFY_ERR_UNSUPPORTED in the ordinary build.
+ */
+int scalify_debug_bounds_report(uint64_t out[3], int reset_ranges, int64_t range_limit);
 int scalify_debug_tensor_map_cache(uint64_t* hits, uint64_t* misses);
 
 /*

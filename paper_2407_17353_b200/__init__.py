@@ -53,12 +53,15 @@ _lib = None
 
 
 def lib() -> ctypes.CDLL:
-    """Load ``libscalify.so`` (building it with nvcc if it is not there).  Raises if neither works."""
+    """Load ``libscalify.so`` (building it with nvcc if it is not there).  Raises if neither works.
+    With ``SCALIFY_DEBUG_BUILD=1`` in the environment the bounds-checking build ``libscalify_debug.so`` is loaded
+    instead (see ``scalify_debug_bounds_report`` in ``include/scalify.h``)."""
     global _lib
     if _lib is None:
-        path = _build.LIB
+        debug = os.environ.get("SCALIFY_DEBUG_BUILD", "") == "1"
+        path = _build.LIB_DEBUG if debug else _build.LIB
         if not os.path.exists(path):
-            path = _build.build()
+            path = _build.build(debug=debug)
         L = ctypes.CDLL(path)
         c = ctypes
         P = c.POINTER(scalify_array)
@@ -96,6 +99,8 @@ def lib() -> ctypes.CDLL:
         L.scalify_scalar_mul_pow2.argtypes = [P, f32, vp]
         L.scalify_debug_layernorm_plan.argtypes = [i64, i64, i32, i32, vp]
         L.scalify_debug_host_state_selftest.restype = i32
+        L.scalify_debug_bounds_report.argtypes = [vp, i32, i64]
+        L.scalify_debug_bounds_report.restype = i32
         L.scalify_debug_bf16_round.argtypes = [vp, vp, i64, i32, vp]
         L.scalify_debug_bf16_round.restype = i32
         L.scalify_debug_tensor_map_cache.argtypes = [vp, vp]
@@ -427,6 +432,14 @@ def scalify_debug_bf16_round(x: torch.Tensor, y: torch.Tensor, two_wide: bool = 
     assert x.dtype == y.dtype == torch.float32 and x.is_contiguous() and y.is_contiguous() and x.numel() == y.numel()
     _check(lib().scalify_debug_bf16_round(x.data_ptr(), y.data_ptr(), x.numel(), int(bool(two_wide)), _stream(stream)),
            "scalify_debug_bf16_round")
+
+
+def scalify_debug_bounds_report(reset_ranges: bool = False, range_limit: int = -1) -> dict:
+    """Bounds-checking build only: accesses refused since the last report (and where the first one was)."""
+    out = (ctypes.c_uint64 * 3)()
+    _check(lib().scalify_debug_bounds_report(ctypes.cast(out, ctypes.c_void_p), int(bool(reset_ranges)), int(range_limit)),
+           "scalify_debug_bounds_report")
+    return dict(violations=int(out[0]), first_address=int(out[1]), first_bytes=int(out[2]))
 
 
 def scalify_debug_tensor_map_cache() -> dict:

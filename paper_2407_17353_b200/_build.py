@@ -14,8 +14,11 @@ from concurrent.futures import ThreadPoolExecutor
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
-OBJ = os.path.join(_HERE, "build")
-LIB = os.path.join(_HERE, "libscalify.so")
+OBJ_RELEASE = os.path.join(_HERE, "build")
+LIB_RELEASE = os.path.join(_HERE, "libscalify.so")
+OBJ_DEBUG = os.path.join(_HERE, "build_debug")
+LIB_DEBUG = os.path.join(_HERE, "libscalify_debug.so")
+OBJ, LIB = OBJ_RELEASE, LIB_RELEASE
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -40,7 +43,9 @@ def _newest_header() -> float:
     return max(os.path.getmtime(h) for h in hs)
 
 
-def build(force: bool = False, verbose: bool = False, ptxas_info: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, ptxas_info: bool = False, debug: bool = False) -> str:
+    """debug: the bounds-checking build (-DSCALIFY_DEBUG, see include/scalify.h), a library of its own."""
+    OBJ, LIB = (OBJ_DEBUG, LIB_DEBUG) if debug else (OBJ_RELEASE, LIB_RELEASE)
     os.makedirs(OBJ, exist_ok=True)
     nvcc = _nvcc()
     hdr = _newest_header()
@@ -51,7 +56,8 @@ def build(force: bool = False, verbose: bool = False, ptxas_info: bool = False) 
         objs.append(obj)
         stale = force or not os.path.exists(obj) or os.path.getmtime(obj) < max(os.path.getmtime(src), hdr)
         if stale:
-            cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if ptxas_info else []) + ["-c", src, "-o", obj]
+            cmd = ([nvcc] + NVCC_FLAGS + (["-DSCALIFY_DEBUG"] if debug else []) +
+                   (["-Xptxas", "-v"] if ptxas_info else []) + ["-c", src, "-o", obj])
             jobs.append(cmd)
 
     def run(cmd):
@@ -73,4 +79,4 @@ def build(force: bool = False, verbose: bool = False, ptxas_info: bool = False) 
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose=True, ptxas_info="--ptxas" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose=True, ptxas_info="--ptxas" in sys.argv, debug="--debug" in sys.argv))

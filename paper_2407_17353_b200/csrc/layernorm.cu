@@ -22,6 +22,9 @@ constexpr int kLnBwdStages = 3;  // rows (of X and G) in flight per team, backwa
 // barrier is involved; cp.async.wait_group is a hardware wait, not a spin.  This keeps several rows
 // per thread in flight without holding them in registers.
 __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+#ifdef SCALIFY_DEBUG
+  if (!dbg_ok(gmem_src, 16)) { *static_cast<uint4*>(smem_dst) = make_uint4(0u, 0u, 0u, 0u); return; }
+#endif
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst))),
                "l"(gmem_src) : "memory");
 }

@@ -43,6 +43,18 @@ int check_array(const scalify_array* a) {
     if (a->stride[i] < 0) return SCALIFY_ERR_ALIGNMENT;
     if (a->shape[i] > 1 && (a->stride[i] * es) % 16 != 0) return SCALIFY_ERR_ALIGNMENT;
   }
+#ifdef SCALIFY_DEBUG
+  {
+    // the bytes this array spans: every kernel access through the checked helpers must fall inside a registered span
+    int64_t last = 0;
+    bool empty = false;
+    for (int i = 0; i < a->ndim; ++i) {
+      if (a->shape[i] == 0) empty = true;
+      else last += (a->shape[i] - 1) * a->stride[i];
+    }
+    if (!empty) dbg_register_range(a->data, static_cast<unsigned long long>(last + 1) * es);
+  }
+#endif
   return SCALIFY_OK;
 }
 
@@ -146,6 +158,9 @@ static int check_ws(void* ws, size_t bytes, size_t need) {
   if (!ws) return SCALIFY_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(ws) % 256 != 0) return SCALIFY_ERR_WORKSPACE;
   if (bytes < need) return SCALIFY_ERR_WORKSPACE;
+#ifdef SCALIFY_DEBUG
+  dbg_register_range(ws, bytes);
+#endif
   return SCALIFY_OK;
 }
 
@@ -403,6 +418,10 @@ static int check_mx(const scalify_mx_array* a) {
     return SCALIFY_ERR_ALIGNMENT;
   if (a->transposed != 0 && a->transposed != 1) return SCALIFY_ERR_VALUE;
   if (a->transposed && a->rows % 16 != 0) return SCALIFY_ERR_ALIGNMENT;  // rows of the storage are `rows` bytes long
+#ifdef SCALIFY_DEBUG
+  dbg_register_range(a->data, static_cast<unsigned long long>(a->rows) * a->K);
+  dbg_register_range(a->sf, mx_sf_bytes(a->rows, a->K));
+#endif
   return SCALIFY_OK;
 }
 
@@ -917,6 +936,13 @@ int scalify_debug_bf16_round(const float* x, float* y, int64_t n, int two_wide, 
 }
 
 int scalify_debug_host_state_selftest(void) { return host_state_selftest(); }
+
+int scalify_debug_bounds_report(uint64_t out[3], int reset_ranges, int64_t range_limit) {
+  unsigned long long v[3] = {0, 0, 0};
+  const int rc = debug_bounds_report(v, reset_ranges, range_limit);
+  if (rc == SCALIFY_OK && out) { out[0] = v[0]; out[1] = v[1]; out[2] = v[2]; }
+  return rc;
+}
 
 int scalify_debug_tensor_map_cache(uint64_t* hits, uint64_t* misses) {
   if (!hits || !misses) return SCALIFY_ERR_NULL;

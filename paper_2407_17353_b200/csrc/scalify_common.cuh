@@ -147,6 +147,58 @@ __device__ __forceinline__ float p2_sqrt_floor(float s) {
 template <int DT> struct ElemBytes { static constexpr int v = (DT <= SCALIFY_E5M2) ? 1 : (DT == SCALIFY_F32 ? 4 : 2); };
 
 // ---- vector load of N consecutive elements (N*size bytes, naturally aligned) into fp32
+// ---------------------------------------------------------------------------------------------
+// Debug build (-DSCALIFY_DEBUG): every global access that goes through the helpers below (vector loads and
+// stores, the asynchronous row copies, the scalar tail accesses) is checked against the byte ranges of the
+// arrays the host has registered (every scalify_array an entry point validates).  An access outside all of
+// them is counted, its address recorded, and SKIPPED (a load yields zeros), so nothing faults.  The table
+// lives in one translation unit; every other one holds a pointer to it that the host sets before first use.
+// ---------------------------------------------------------------------------------------------
+#ifdef SCALIFY_DEBUG
+constexpr int kDbgMaxRanges = 4096;
+struct DbgTable {
+  unsigned long long lo[kDbgMaxRanges], hi[kDbgMaxRanges];  // sorted by lo, disjoint
+  int n;
+  unsigned long long violations, first_addr, first_bytes;
+};
+static __device__ DbgTable* g_dbg_table = nullptr;
+__device__ __forceinline__ bool dbg_ok(const void* p, int bytes) {
+  const DbgTable* t = g_dbg_table;
+  if (!t || !__isGlobal(p)) return true;  // (the helpers also read parameters staged in shared memory)
+  const unsigned long long a = reinterpret_cast<unsigned long long>(p);
+  int l = 0, r = t->n;  // last range whose lo <= a
+  while (l < r) {
+    const int m = (l + r) >> 1;
+    if (t->lo[m] <= a) l = m + 1; else r = m;
+  }
+  if (l > 0 && a + static_cast<unsigned long long>(bytes) <= t->hi[l - 1]) return true;
+  DbgTable* w = g_dbg_table;
+  if (atomicAdd(&w->violations, 1ull) == 0ull) { w->first_addr = a; w->first_bytes = static_cast<unsigned long long>(bytes); }
+  return false;
+}
+// host side (support.cu): registration of a translation unit's pointer, of an array's byte range, report
+typedef cudaError_t (*DbgSetPointerFn)(DbgTable*);
+void dbg_add_translation_unit(DbgSetPointerFn fn);
+void dbg_register_range(const void* base, unsigned long long bytes);
+namespace {
+struct DbgTranslationUnit {
+  DbgTranslationUnit() {
+    dbg_add_translation_unit([](DbgTable* t) { return cudaMemcpyToSymbol(g_dbg_table, &t, sizeof(t)); });
+  }
+} g_dbg_translation_unit;
+}  // namespace
+#define SCALIFY_DBG_CHECK_LOAD(p, bytes, words)                      \
+  if (!dbg_ok(p, bytes)) {                                          \
+    for (int dbg_i = 0; dbg_i < (words); ++dbg_i) w[dbg_i] = 0u;    \
+    return;                                                         \
+  }
+#define SCALIFY_DBG_CHECK_STORE(p, bytes) \
+  if (!dbg_ok(p, bytes)) return;
+#else
+#define SCALIFY_DBG_CHECK_LOAD(p, bytes, words)
+#define SCALIFY_DBG_CHECK_STORE(p, bytes)
+#endif
+
 template <int BYTES> struct RawVec;
 template <> struct RawVec<4> { uint32_t w[1]; };
 template <> struct RawVec<8> { uint32_t w[2]; };
@@ -156,6 +208,7 @@ template <> struct RawVec<2> { uint16_t h; };
 
 template <int BYTES>
 __device__ __forceinline__ void ld_raw(const void* p, uint32_t* w) {
+  SCALIFY_DBG_CHECK_LOAD(p, BYTES, BYTES / 4)
   if constexpr (BYTES == 16) {
     uint4 v = *reinterpret_cast<const uint4*>(p);
     w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
@@ -175,6 +228,7 @@ __device__ __forceinline__ void ld_raw(const void* p, uint32_t* w) {
 
 template <int BYTES>
 __device__ __forceinline__ void st_raw(void* p, const uint32_t* w) {
+  SCALIFY_DBG_CHECK_STORE(p, BYTES)
   if constexpr (BYTES == 16) {
     *reinterpret_cast<uint4*>(p) = make_uint4(w[0], w[1], w[2], w[3]);
   } else if constexpr (BYTES == 32) {
@@ -191,6 +245,7 @@ __device__ __forceinline__ void st_raw(void* p, const uint32_t* w) {
 // streaming variants (read-once / write-once data: do not keep in L1)
 template <int BYTES>
 __device__ __forceinline__ void ld_raw_stream(const void* p, uint32_t* w) {
+  SCALIFY_DBG_CHECK_LOAD(p, BYTES, BYTES / 4)
   if constexpr (BYTES == 16) {
     uint4 v = __ldcs(reinterpret_cast<const uint4*>(p));
     w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
@@ -209,6 +264,7 @@ __device__ __forceinline__ void ld_raw_stream(const void* p, uint32_t* w) {
 
 template <int BYTES>
 __device__ __forceinline__ void st_raw_stream(void* p, const uint32_t* w) {
+  SCALIFY_DBG_CHECK_STORE(p, BYTES)
   if constexpr (BYTES == 16) {
     __stcs(reinterpret_cast<uint4*>(p), make_uint4(w[0], w[1], w[2], w[3]));
   } else if constexpr (BYTES == 32) {
@@ -330,6 +386,9 @@ __device__ __forceinline__ float2 bf16_round_f32x2(float2 x) {
 // scalar load/store for ragged tails
 template <int DT>
 __device__ __forceinline__ float load_elem(const void* p, int64_t i) {
+#ifdef SCALIFY_DEBUG
+  if (!dbg_ok(static_cast<const char*>(p) + i * ElemBytes<DT>::v, ElemBytes<DT>::v)) return 0.f;
+#endif
   if constexpr (DT == SCALIFY_F32) return static_cast<const float*>(p)[i];
   else if constexpr (DT == SCALIFY_BF16) return bf16_bits_to_float(static_cast<const uint16_t*>(p)[i]);
   else if constexpr (DT == SCALIFY_F16) return __half2float(static_cast<const __half*>(p)[i]);
@@ -338,6 +397,9 @@ __device__ __forceinline__ float load_elem(const void* p, int64_t i) {
 
 template <int DT>
 __device__ __forceinline__ void store_elem(void* p, int64_t i, float x) {
+#ifdef SCALIFY_DEBUG
+  if (!dbg_ok(static_cast<char*>(p) + i * ElemBytes<DT>::v, ElemBytes<DT>::v)) return;
+#endif
   if constexpr (DT == SCALIFY_F32) static_cast<float*>(p)[i] = x;
   else if constexpr (DT == SCALIFY_BF16) static_cast<__nv_bfloat16*>(p)[i] = __float2bfloat16_rn(x);
   else if constexpr (DT == SCALIFY_F16) static_cast<__half*>(p)[i] = __float2half_rn(x);

@@ -104,6 +104,8 @@ size_t matmul_ws_bytes(int64_t rows, int64_t cols);
 size_t matmul_splitk_ws_bytes(int64_t rows, int64_t cols);
 int launch_bf16_round(const float* x, float* y, long long n, int two_wide, cudaStream_t st);
 int host_state_selftest();
+// debug build only (SCALIFY_ERR_UNSUPPORTED otherwise): violations seen since the last report
+int debug_bounds_report(unsigned long long out[3], int reset_ranges, long long limit);
 void map_cache_counters(unsigned long long* hits, unsigned long long* misses);
 int launch_expire_wait(void* ws, unsigned long long limit_ns, uint32_t* waited_us, cudaStream_t st);
 int launch_scaled_matmul(const MatmulArgs& a, void* ws, size_t ws_bytes, cudaStream_t st);

@@ -723,4 +723,86 @@ int launch_bf16_round(const float* x, float* y, long long n, int two_wide, cudaS
   return SCALIFY_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// debug build: the table of registered byte ranges (host shadow, device copy) and its report
+// ---------------------------------------------------------------------------------------------
+#ifdef SCALIFY_DEBUG
+}  // namespace scalify
+#include <algorithm>
+#include <mutex>
+#include <vector>
+namespace scalify {
+static __device__ DbgTable g_dbg_storage;
+namespace {
+std::mutex g_dbg_mu;
+std::vector<DbgSetPointerFn>& dbg_units() { static std::vector<DbgSetPointerFn> v; return v; }
+std::vector<std::pair<unsigned long long, unsigned long long>> g_dbg_ranges;  // sorted, disjoint
+bool g_dbg_pointers_set[64] = {};
+long long g_dbg_limit = -1;  // self-test: cap on the length of every range registered from now on
+}  // namespace
+
+void dbg_add_translation_unit(DbgSetPointerFn fn) { dbg_units().push_back(fn); }
+
+static cudaError_t dbg_upload() {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  DbgTable* dptr = nullptr;
+  if ((e = cudaGetSymbolAddress(reinterpret_cast<void**>(&dptr), g_dbg_storage)) != cudaSuccess) return e;
+  if (dev >= 0 && dev < 64 && !g_dbg_pointers_set[dev]) {
+    for (DbgSetPointerFn fn : dbg_units())
+      if ((e = fn(dptr)) != cudaSuccess) return e;
+    g_dbg_pointers_set[dev] = true;
+  }
+  const int n = static_cast<int>(g_dbg_ranges.size());
+  std::vector<unsigned long long> lo(n), hi(n);
+  for (int i = 0; i < n; ++i) { lo[i] = g_dbg_ranges[i].first; hi[i] = g_dbg_ranges[i].second; }
+  // synchronous copies: the debug build is not meant for stream capture or for timing
+  if (n && (e = cudaMemcpy(dptr->lo, lo.data(), n * sizeof(unsigned long long), cudaMemcpyHostToDevice)) != cudaSuccess) return e;
+  if (n && (e = cudaMemcpy(dptr->hi, hi.data(), n * sizeof(unsigned long long), cudaMemcpyHostToDevice)) != cudaSuccess) return e;
+  return cudaMemcpy(&dptr->n, &n, sizeof(int), cudaMemcpyHostToDevice);
+}
+
+void dbg_register_range(const void* base, unsigned long long bytes) {
+  if (!base || bytes == 0) return;
+  std::lock_guard<std::mutex> lock(g_dbg_mu);
+  if (g_dbg_limit >= 0 && bytes > static_cast<unsigned long long>(g_dbg_limit)) bytes = static_cast<unsigned long long>(g_dbg_limit);
+  unsigned long long lo = reinterpret_cast<unsigned long long>(base), hi = lo + bytes;
+  // already covered: nothing to do (the common case: the same buffers call after call)
+  for (const auto& r : g_dbg_ranges)
+    if (r.first <= lo && hi <= r.second) return;
+  // merge with every range it touches, keep the list sorted and disjoint
+  std::vector<std::pair<unsigned long long, unsigned long long>> out;
+  for (const auto& r : g_dbg_ranges) {
+    if (r.second < lo || hi < r.first) out.push_back(r);
+    else { lo = std::min(lo, r.first); hi = std::max(hi, r.second); }
+  }
+  out.emplace_back(lo, hi);
+  std::sort(out.begin(), out.end());
+  if (static_cast<int>(out.size()) > kDbgMaxRanges) out.erase(out.begin(), out.begin() + (out.size() - kDbgMaxRanges));
+  g_dbg_ranges.swap(out);
+  (void)dbg_upload();
+}
+
+int debug_bounds_report(unsigned long long out[3], int reset_ranges, long long limit) {
+  std::lock_guard<std::mutex> lock(g_dbg_mu);
+  DbgTable* dptr = nullptr;
+  SCALIFY_CUDA_TRY(cudaDeviceSynchronize());
+  SCALIFY_CUDA_TRY(cudaGetSymbolAddress(reinterpret_cast<void**>(&dptr), g_dbg_storage));
+  unsigned long long v[3] = {0, 0, 0};
+  SCALIFY_CUDA_TRY(cudaMemcpy(v, &dptr->violations, sizeof(v), cudaMemcpyDeviceToHost));
+  if (out) { out[0] = v[0]; out[1] = v[1]; out[2] = v[2]; }
+  const unsigned long long zero[3] = {0, 0, 0};
+  SCALIFY_CUDA_TRY(cudaMemcpy(&dptr->violations, zero, sizeof(zero), cudaMemcpyHostToDevice));
+  g_dbg_limit = limit;
+  if (reset_ranges) {
+    g_dbg_ranges.clear();
+    SCALIFY_CUDA_TRY(dbg_upload());
+  }
+  return SCALIFY_OK;
+}
+#else
+int debug_bounds_report(unsigned long long*, int, long long) { return SCALIFY_ERR_UNSUPPORTED; }
+#endif
+
 }  // namespace scalify

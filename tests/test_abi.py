@@ -26,6 +26,20 @@ def test_library_exports_every_declared_function():
     assert L.scalify_version() >= 100
 
 
+def test_bounds_checking_build_exports_the_same_functions():
+    """libscalify_debug.so (-DSCALIFY_DEBUG) is a drop-in for the ordinary library; the ordinary one answers the
+    checker's report call with 'not supported'."""
+    import ctypes
+    from paper_2407_17353_b200 import _build
+    D = ctypes.CDLL(_build.build(debug=True))
+    for n in declared_functions():
+        assert hasattr(D, n), n
+    assert D.scalify_version() == sc.lib().scalify_version()
+    if os.environ.get("SCALIFY_DEBUG_BUILD", "") != "1":
+        sc.lib().scalify_debug_bounds_report.restype = ctypes.c_int
+        assert sc.lib().scalify_debug_bounds_report(None, 0, -1) == -6
+
+
 def test_status_strings_and_workspace_sizes():
     L = sc.lib()
     assert L.scalify_status_string(0) == b"ok"
