@@ -262,10 +262,12 @@ __global__ void __launch_bounds__(kThreads) rebalance_check_kernel(const void* _
   constexpr int VEC = VecElems<IN, OUT>::v;
   constexpr int IB = VEC * ElemBytes<IN>::v, OB = VEC * ElemBytes<OUT>::v;
   const float xs = load_scale(x_scale);
-  const float s = __ldg(stat);
+  // (volatile: these two words are written by the grid this one depends on; a read-only-path load may be
+  // scheduled above the wait, and then sees what the words held before)
+  const float s = *reinterpret_cast<const volatile float*>(stat);
   bool nonfinite;
   const float r = rescale_factor(s, &nonfinite);
-  const float rp = __ldg(r_pred);
+  const float rp = *reinterpret_cast<const volatile float*>(r_pred);
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     uint32_t flags = is_pow2_scale(xs) ? 0u : SCALIFY_DEV_BAD_SCALE;
     if (nonfinite) flags |= SCALIFY_DEV_NONFINITE_STAT;

@@ -197,7 +197,9 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
     if (blockIdx.x == 0) {
       float r = 1.0f;
       bool nf = false;
-      if (p.stat_in) r = rescale_factor(__ldg(p.stat_in), &nf);
+      // (volatile: the word may have been written by the grid this one depends on; a read-only-path load could be
+      // scheduled above the wait)
+      if (p.stat_in) r = rescale_factor(*reinterpret_cast<const volatile float*>(p.stat_in), &nf);
       float ys = load_scale(p.a_scale) * load_scale(p.b_scale) * p.kf * r;
       if constexpr (BIAS) ys = fmaxf(ys, load_scale(p.bias_scale));  // add rule for powers of two
       if (p.y_scale) *p.y_scale = ys;
@@ -372,7 +374,7 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
     // delayed rescale (Section 3.3): the data are written already divided by r = p2_floor(earlier
     // statistic); this step's statistic is taken on the un-rebalanced fp32 values
     float r_prev = 1.0f;
-    if (p.stat_in) { bool nf; r_prev = rescale_factor(__ldg(p.stat_in), &nf); }
+    if (p.stat_in) { bool nf; r_prev = rescale_factor(*reinterpret_cast<const volatile float*>(p.stat_in), &nf); }
     float alpha = p.alpha * (1.0f / r_prev);  // exact: both are powers of two
     float beta = 0.f;
     if constexpr (BIAS) {

@@ -106,7 +106,12 @@ inline int device_once(DeviceOnce& o, int* value_out, Fn fn) {
 #ifdef __CUDACC__
 
 // scale word or 1 (Section 3.1: an unscaled array unbundles to (x, 1))
-__device__ __forceinline__ float load_scale(const float* s) { return s ? __ldg(s) : 1.0f; }
+// A scale word is usually written by the kernel just before this one.  The load is a volatile one on purpose:
+// a load through the read-only path (__ldg) is treated as invariant and may be scheduled above the
+// `griddepcontrol.wait` of a programmatic dependent, where it would see the word's previous content.
+__device__ __forceinline__ float load_scale(const float* s) {
+  return s ? *reinterpret_cast<const volatile float*>(s) : 1.0f;
+}
 
 __device__ __forceinline__ bool is_pow2_scale(float s) {
   uint32_t b = __float_as_uint(s);

@@ -26,6 +26,20 @@ def pytest_collection_modifyitems(config, items):
             item.add_marker(skip)
 
 
+@pytest.fixture(autouse=True)
+def _bounds_checked(request):
+    """With SCALIFY_DEBUG_BUILD=1 (the bounds-checking build of the library is loaded): every GPU test starts with
+    an empty table of registered arrays and fails if the checker refused an access while it ran."""
+    if os.environ.get("SCALIFY_DEBUG_BUILD", "") != "1" or "gpu" not in request.keywords:
+        yield
+        return
+    import paper_2407_17353_b200 as sc
+    sc.scalify_debug_bounds_report(reset_ranges=True)
+    yield
+    rep = sc.scalify_debug_bounds_report(reset_ranges=True)
+    assert rep["violations"] == 0, rep
+
+
 def pytest_sessionfinish(session, exitstatus):
     """With SCALIFY_TOLERANCE_LOG=<file>: per test function, how many outputs were compared by
     helpers.within() and how many of them only its cancellation clause accepted."""
