@@ -11,7 +11,8 @@ shaped like GPT-style training tensors:
      two while the statistic is gathered; a check launch repairs it if the prediction failed)
   4. scaled add of two BF16 tensors
   5. scaled LayerNorm forward  [131072, 1024] BF16
-  6. scaled LayerNorm backward + L2 dynamic rescale of the input gradient to E5M2
+  6. scaled LayerNorm backward + L2 dynamic rescale of the input gradient to E5M2 (exact, in one pass: the
+     gradient is written with the predicted power of two; a repair launch returns at once when it held)
   7. scaled Adam step over 125M parameters (E5M2 grads, FP16 scaled m/v/w)
 Outside the step (own timed loop) the next-row variant is reported too: the same GEMM with delayed
 rescaling - one kernel, E4M3 written directly with the previous step's statistic while this step's AMAX
@@ -595,12 +596,16 @@ def main():
     ws_head = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_MATMUL, N_GEMM, N_GEMM), dev)   # keeps the prediction
     n_ev = 9
     # kernels of this library per step: headline call (matmul + check launch), one-read rescale (statistic with the
-    # predicted output + check launch), add, LayerNorm fwd, LayerNorm bwd + finalize + pass 2, Adam scales + update
+    # predicted output + check launch), add, LayerNorm fwd, LayerNorm bwd + finalize + repair launch, Adam scales +
+    # update
     launches_per_step = 2 + 2 + 1 + 1 + 3 + 2
+    ws_ln1 = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_LAYERNORM_BWD, LN_R, LN_D), dev)   # keeps the prediction
+    dXq1 = sc.ScaledTensor.empty((LN_R, LN_D), torch.float8_e5m2, dev)
 
     def step(t, evs=None, form=0):
-        """form 0: the headline as one call; 1: the same work as two calls (GEMM + AMAX, then pass 2), each with a
-        time of its own; 2: the one call without the BF16 intermediate (Y = NULL)."""
+        """form 0: the headline as one call and the LayerNorm gradient's rescale in one pass; 1: the same work as two
+        calls (GEMM + AMAX, then pass 2, each with a time of its own) and the LayerNorm backward with its stored BF16
+        intermediate and a second pass; 2: the one call without the BF16 intermediate (Y = NULL)."""
         def mark(i):
             if evs is not None:
                 evs[i].record()
@@ -620,8 +625,13 @@ def main():
         mark(4)
         sc.scalify_scaled_layernorm(X, gamma, beta, LY, eps=1e-5, mean=mean, rinv=rinv)
         mark(5)
-        sc.scalify_scaled_layernorm_bwd(G, X, gamma, mean, rinv, dX, ws_ln, eps=1e-5, stat_dx=sc.STAT_L2, dXq=dXq,
-                                        dgamma=dg, dbeta=db)
+        if form == 1:
+            sc.scalify_scaled_layernorm_bwd(G, X, gamma, mean, rinv, dX, ws_ln, eps=1e-5, stat_dx=sc.STAT_L2, dXq=dXq,
+                                            dgamma=dg, dbeta=db)
+        else:
+            # a6 in ONE pass (dX = None): the exact dynamic rescale with the predicted power of two
+            sc.scalify_scaled_layernorm_bwd(G, X, gamma, mean, rinv, None, ws_ln1, eps=1e-5, stat_dx=sc.STAT_L2,
+                                            dXq=dXq1, dgamma=dg, dbeta=db)
         mark(6)
         sc.scalify_scaled_adam_step(adam, ws_ad, lr=3e-4, beta1=0.9, beta2=0.999, eps=1e-8, step=1000 + t)
         mark(7)
@@ -663,7 +673,7 @@ def main():
     for t in range(W):
         step(t, None)
     barrier()
-    for w in (ws_mm, ws_head, ws_rs, ws_ln, ws_ad):
+    for w in (ws_mm, ws_head, ws_rs, ws_ln, ws_ln1, ws_ad):
         st = w.check_status()
         if st != 0:
             raise SystemExit(f"device status {st} after warm-up")
@@ -683,7 +693,7 @@ def main():
     total_ms = t_start.elapsed_time(t_end)
     seg = np.array([[evs[t][i].elapsed_time(evs[t][i + 1]) for i in range(n_ev - 1)] for t in range(K)])
     seg_ms = seg.mean(axis=0)
-    for w in (ws_mm, ws_head, ws_rs, ws_ln, ws_ad):
+    for w in (ws_mm, ws_head, ws_rs, ws_ln, ws_ln1, ws_ad):
         st = w.check_status()
         if st & sc.DEV_TIMEOUT:
             raise SystemExit(f"device status {st} in the timed region")
@@ -692,6 +702,7 @@ def main():
     # pass each get a time of their own, in the same surroundings), and with the one call in its FP8-only form
     # (Y = NULL).  All three forms must leave the same E4M3 output and scale, bit for bit.
     two_call_ms = [float("nan"), float("nan")]
+    ln_two_pass_ms = float("nan")
     fp8_only_ms = float("nan")
     if not args.no_next:
         for form in (1, 2):
@@ -705,10 +716,16 @@ def main():
             if form == 1:
                 two_call_ms = [float(np.mean([evs2[t][0].elapsed_time(evs2[t][1]) for t in range(K)])),
                                float(np.mean([evs2[t][1].elapsed_time(evs2[t][2]) for t in range(K)]))]
+                ln_two_pass_ms = float(np.mean([evs2[t][5].elapsed_time(evs2[t][6]) for t in range(K)]))
                 same = torch.equal(Yq.data.view(torch.uint8), Yq2.data.view(torch.uint8)) and \
                     float(Yq.scale.item()) == float(Yq2.scale.item())
                 if not same:
                     raise SystemExit("the one-call headline and the two-call form disagree")
+                same_ln = torch.equal(dXq.data.view(torch.uint8), dXq1.data.view(torch.uint8)) and \
+                    dXq.scale_value() == dXq1.scale_value() and \
+                    torch.equal(ws_ln.statistic().view(torch.int32), ws_ln1.statistic().view(torch.int32))
+                if not same_ln:
+                    raise SystemExit("the one-pass LayerNorm gradient rescale and the two-pass form disagree")
             else:
                 fp8_only_ms = float(np.mean([evs2[t][0].elapsed_time(evs2[t][2]) for t in range(K)]))
                 if not torch.equal(Yq.data.view(torch.uint8), Yq2.data.view(torch.uint8)):
@@ -753,35 +770,6 @@ def main():
     l1.record()
     barrier()
     ln_delayed_ms = l0.elapsed_time(l1) / l_iters if l_iters else float("nan")
-
-    # LayerNorm backward + EXACT dynamic rescale in one pass (dX = None): the same bits as segment a6 (checked
-    # here), with the un-rebalanced BF16 gradient never stored and the output written with the predicted power of
-    # two; a second launch of the kernel returns at once when the prediction held (5 B/elem instead of 9)
-    ln_onepass_ms = float("nan")
-    ln_onepass_same = None
-    if not args.no_next:
-        ws_ln1 = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_LAYERNORM_BWD, LN_R, LN_D), dev)
-        dXq1 = sc.ScaledTensor.empty((LN_R, LN_D), torch.float8_e5m2, dev)
-
-        def ln_onepass_step():
-            sc.scalify_scaled_layernorm_bwd(G, X, gamma, mean, rinv, None, ws_ln1, eps=1e-5, stat_dx=sc.STAT_L2,
-                                            dXq=dXq1, dgamma=dg, dbeta=db)
-        for _ in range(3):
-            ln_onepass_step()
-        barrier()
-        l0.record()
-        for _ in range(l_iters):
-            ln_onepass_step()
-        l1.record()
-        barrier()
-        ln_onepass_ms = l0.elapsed_time(l1) / l_iters
-        # against the two-pass call of segment a6 on the same inputs
-        sc.scalify_scaled_layernorm_bwd(G, X, gamma, mean, rinv, dX, ws_ln, eps=1e-5, stat_dx=sc.STAT_L2, dXq=dXq,
-                                        dgamma=dg, dbeta=db)
-        ln_onepass_same = bool(torch.equal(dXq1.data.view(torch.uint8), dXq.data.view(torch.uint8)) and
-                               dXq1.scale_value() == dXq.scale_value() and
-                               torch.equal(ws_ln1.statistic().view(torch.int32), ws_ln.statistic().view(torch.int32)))
-        del dXq1, ws_ln1
 
     # Adam that also writes the E4M3 compute copy of the updated weight (1 more byte per parameter)
     awc = sc.ScaledTensor.make(torch.empty(ADAM_N, dtype=torch.float8_e4m3fn, device=dev), 1.0)
@@ -1030,17 +1018,17 @@ def main():
                  3 * n_add), GBps_at_5_bytes_per_elem=round(5 * n_add / (seg_ms[2] * 1e-3) / 1e9, 1)),
         row("a4 scaled add BF16 (6 B/elem)", seg_ms[3], 6 * n_add),
         row("a5 scaled LayerNorm fwd BF16->BF16 (4 B/elem + 8 B/row)", seg_ms[4], 4 * n_ln + 8 * LN_R),
-        row("a6 scaled LayerNorm bwd + L2 rescale to E5M2 (9 B/elem + 8 B/row)", seg_ms[5], 9 * n_ln + 8 * LN_R),
+        row("a6 scaled LayerNorm bwd + exact dynamic L2 rescale to E5M2 in ONE pass (dX = NULL: rebalanced with the "
+            "predicted power of two, repair launch returns at once when it held; 5 B/elem + 8 B/row; bit-identical to "
+            "the two-pass row below, checked)", seg_ms[5], 5 * n_ln + 8 * LN_R),
+        row("a6 as two passes with the BF16 intermediate stored (second pass of the same step, 9 B/elem + 8 B/row)",
+            ln_two_pass_ms, 9 * n_ln + 8 * LN_R),
         row("a7 scaled Adam, E5M2 grads, FP16 m/v/w (13 B/param)", seg_ms[6], 13 * ADAM_N),
         {"row": "f1 (next, timed outside the step, back to back) delayed-rescale GEMM 8192^3: E4M3 out in one "
                 "kernel, no BF16 intermediate, no pass 2", "ms": round(float(delayed_ms), 4),
          "TFLOP/s": round(flops / (delayed_ms * 1e-3) / 1e12, 1)},
         row("f1 (next, timed outside the step, back to back) LayerNorm bwd with delayed L2 rescale: E5M2 gradient "
             "in one pass, no BF16 intermediate, no pass 2 (5 B/elem + 8 B/row)", ln_delayed_ms, 5 * n_ln + 8 * LN_R),
-        dict(row("a6 as ONE pass (timed outside the step, back to back): LayerNorm bwd + exact dynamic L2 rescale to "
-                 "E5M2 with dX = NULL - rebalanced with the predicted power of two, repair launch returns at once "
-                 "when it held (5 B/elem + 8 B/row)", ln_onepass_ms, 5 * n_ln + 8 * LN_R),
-             bit_identical_to_a6=ln_onepass_same),
         {"row": "f1b (next, timed in a third pass of the same step) the headline call with Y = NULL: only the E4M3 "
                 "output is stored (values still rounded through BF16, AMAX of the BF16 values; a repair launch of the "
                 "same kernel returns at once when the prediction held); Yq, scale and statistic bit-identical",

@@ -261,13 +261,21 @@ __global__ void __launch_bounds__(kThreads) rebalance_check_kernel(const void* _
   asm volatile("griddepcontrol.wait;" ::: "memory");
   constexpr int VEC = VecElems<IN, OUT>::v;
   constexpr int IB = VEC * ElemBytes<IN>::v, OB = VEC * ElemBytes<OUT>::v;
-  const float xs = load_scale(x_scale);
-  // (volatile: these two words are written by the grid this one depends on; a read-only-path load may be
-  // scheduled above the wait, and then sees what the words held before)
-  const float s = *reinterpret_cast<const volatile float*>(stat);
+  // One thread per block reads the three words the grid before this one wrote (input scale, statistic, the power
+  // of two it divided by) and hands them to the others: the loads are volatile, because a load through the
+  // read-only path may be scheduled above the wait and then sees what the words held before.
+  __shared__ float s_words[3];
+  if (threadIdx.x == 0) {
+    s_words[0] = load_scale_after_wait(x_scale);
+    s_words[1] = *reinterpret_cast<const volatile float*>(stat);
+    s_words[2] = *reinterpret_cast<const volatile float*>(r_pred);
+  }
+  __syncthreads();
+  const float xs = s_words[0];
+  const float s = s_words[1];
   bool nonfinite;
   const float r = rescale_factor(s, &nonfinite);
-  const float rp = *reinterpret_cast<const volatile float*>(r_pred);
+  const float rp = s_words[2];
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     uint32_t flags = is_pow2_scale(xs) ? 0u : SCALIFY_DEV_BAD_SCALE;
     if (nonfinite) flags |= SCALIFY_DEV_NONFINITE_STAT;

@@ -200,8 +200,8 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
       // (volatile: the word may have been written by the grid this one depends on; a read-only-path load could be
       // scheduled above the wait)
       if (p.stat_in) r = rescale_factor(*reinterpret_cast<const volatile float*>(p.stat_in), &nf);
-      float ys = load_scale(p.a_scale) * load_scale(p.b_scale) * p.kf * r;
-      if constexpr (BIAS) ys = fmaxf(ys, load_scale(p.bias_scale));  // add rule for powers of two
+      float ys = load_scale_after_wait(p.a_scale) * load_scale_after_wait(p.b_scale) * p.kf * r;
+      if constexpr (BIAS) ys = fmaxf(ys, load_scale_after_wait(p.bias_scale));  // add rule for powers of two
       if (p.y_scale) *p.y_scale = ys;
       if constexpr (SPEC) {
         bool nf2;
@@ -210,8 +210,8 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
       if (nf && p.status) atomicOr(p.status, static_cast<uint32_t>(SCALIFY_DEV_NONFINITE_STAT));
     }
     if (blockIdx.x == 0 && p.status) {
-      bool bad = !is_pow2_scale(load_scale(p.a_scale)) || !is_pow2_scale(load_scale(p.b_scale));
-      if constexpr (BIAS) bad = bad || !is_pow2_scale(load_scale(p.bias_scale));
+      bool bad = !is_pow2_scale(load_scale_after_wait(p.a_scale)) || !is_pow2_scale(load_scale_after_wait(p.b_scale));
+      if constexpr (BIAS) bad = bad || !is_pow2_scale(load_scale_after_wait(p.bias_scale));
       if (bad) atomicOr(p.status, static_cast<uint32_t>(SCALIFY_DEV_BAD_SCALE));
     }
   }
@@ -379,8 +379,8 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
     float beta = 0.f;
     if constexpr (BIAS) {
       // both terms are brought to the output scale max(A_s B_s kf(K), bias_s): exact power-of-two factors
-      const float ab_s = load_scale(p.a_scale) * load_scale(p.b_scale) * p.kf;
-      const float b_s = load_scale(p.bias_scale);
+      const float ab_s = load_scale_after_wait(p.a_scale) * load_scale_after_wait(p.b_scale) * p.kf;
+      const float b_s = load_scale_after_wait(p.bias_scale);
       const float ys = fmaxf(ab_s, b_s);
       alpha *= ab_s / ys;
       beta = b_s / ys;
@@ -586,7 +586,7 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
       if constexpr (NOY) {
         bool nfq;
         const float r_true = rescale_factor(stat_now, &nfq);
-        const float ys = load_scale(p.a_scale) * load_scale(p.b_scale) * p.kf;
+        const float ys = load_scale_after_wait(p.a_scale) * load_scale_after_wait(p.b_scale) * p.kf;
         if (p.yq_scale) *p.yq_scale = ys * r_true;
         if (p.hint_out) *p.hint_out = stat_now;  // every CTA has read the old prediction: all passed the ticket
         if (nfq && p.status) atomicOr(p.status, static_cast<uint32_t>(SCALIFY_DEV_NONFINITE_STAT));

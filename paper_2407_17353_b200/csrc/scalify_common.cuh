@@ -106,10 +106,13 @@ inline int device_once(DeviceOnce& o, int* value_out, Fn fn) {
 #ifdef __CUDACC__
 
 // scale word or 1 (Section 3.1: an unscaled array unbundles to (x, 1))
-// A scale word is usually written by the kernel just before this one.  The load is a volatile one on purpose:
-// a load through the read-only path (__ldg) is treated as invariant and may be scheduled above the
-// `griddepcontrol.wait` of a programmatic dependent, where it would see the word's previous content.
-__device__ __forceinline__ float load_scale(const float* s) {
+// A scale word is usually written by the kernel just before this one.  In an ordinary launch the read-only path
+// is right for it (every thread of thousands of blocks reads the same word: it has to be served by the L1s).
+__device__ __forceinline__ float load_scale(const float* s) { return s ? __ldg(s) : 1.0f; }
+// In a kernel launched as a PROGRAMMATIC DEPENDENT, after its `griddepcontrol.wait`: a load through the read-only
+// path counts as invariant and may be scheduled above the wait, where it would see the word's previous content;
+// this one is volatile (use it from few threads: it goes to the L2 every time).
+__device__ __forceinline__ float load_scale_after_wait(const float* s) {
   return s ? *reinterpret_cast<const volatile float*>(s) : 1.0f;
 }
 
