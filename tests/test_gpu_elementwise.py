@@ -76,7 +76,8 @@ def test_dynamic_rescale_many_tiles_per_block(stat, in_dt, out_dt, in_place):
 
 @pytest.mark.parametrize("n", [1000, 70001, 8 * 1024 * 700 + 13])
 @pytest.mark.parametrize("stat", [sc.STAT_AMAX, sc.STAT_L2])
-@pytest.mark.parametrize("in_dt,out_dt", [(orc.BF16, orc.E4M3), (orc.F32, orc.E5M2), (orc.BF16, orc.BF16)])
+@pytest.mark.parametrize("in_dt,out_dt", [(orc.BF16, orc.E4M3), (orc.F16, orc.E5M2), (orc.F16, orc.E4M3),
+                                          (orc.F32, orc.E5M2), (orc.BF16, orc.BF16)])
 def test_dynamic_rescale_does_not_depend_on_the_prediction(n, stat, in_dt, out_dt):
     """The one-launch dynamic rescale writes its output while it gathers the statistic, with the power of two of
     the statistic the workspace saw last, and reads the input again only if that was wrong.  Whatever the word

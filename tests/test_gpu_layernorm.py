@@ -277,6 +277,34 @@ def test_one_pass_gradient_rescale_is_bit_identical_to_the_two_pass_call(R, d, s
         assert torch.equal(ws1.prediction().view(torch.int32), ws1.statistic().view(torch.int32)), tag
 
 
+@pytest.mark.parametrize("with_gamma,with_dgamma", [(False, False), (True, False), (False, True)])
+def test_one_pass_gradient_rescale_without_gamma_or_column_sums(with_gamma, with_dgamma):
+    R, d = 77, 512
+    c = si.layernorm_case(R, d, seed=49)
+    X, G = st(c["X"], orc.BF16, 2.0), st(c["G"], orc.BF16, 2.0 ** -7)
+    gamma = st(c["gamma"], orc.BF16, 0.5) if with_gamma else None
+    Y = sc.ScaledTensor.empty((R, d), torch.bfloat16)
+    mean = torch.empty(R, dtype=torch.float32, device="cuda")
+    rinv = torch.empty(R, dtype=torch.float32, device="cuda")
+    sc.scalify_scaled_layernorm(X, gamma, st(c["beta"], orc.BF16, 1.0) if with_gamma else None, Y, mean=mean, rinv=rinv)
+    outs = []
+    for one_pass in (False, True):
+        ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_LAYERNORM_BWD, R, d))
+        dX = None if one_pass else sc.ScaledTensor.empty((R, d), torch.bfloat16)
+        q = sc.ScaledTensor.empty((R, d), torch.float8_e5m2)
+        dg = sc.ScaledTensor.empty((d,), torch.float32) if with_dgamma else None
+        db = sc.ScaledTensor.empty((d,), torch.float32) if with_dgamma else None
+        for _ in range(2):   # without and with a prediction
+            sc.scalify_scaled_layernorm_bwd(G, X, gamma, mean, rinv, dX, ws, stat_dx=sc.STAT_AMAX, dXq=q, dgamma=dg, dbeta=db)
+        assert ws.check_status() == 0
+        outs.append((q.data.view(torch.uint8).clone(), q.scale_value(), float(ws.statistic().item()),
+                     None if dg is None else dg.data.clone(), None if db is None else db.data.clone()))
+    a, b = outs
+    assert torch.equal(a[0], b[0]) and a[1] == b[1] and a[2] == b[2]
+    if with_dgamma:
+        assert torch.equal(a[3], b[3]) and torch.equal(a[4], b[4])
+
+
 def test_one_pass_gradient_rescale_argument_checks():
     R, d = 16, 256
     z = lambda dt: sc.ScaledTensor.make(torch.zeros((R, d), device="cuda").to(dt), 1.0)
