@@ -108,6 +108,11 @@ def test_head_dimension_128(H, Tq, Tk, causal):
     run_case(H, Tq, Tk, causal, HD=128, c=2.0 ** -3.5 if Tq == 200 else 0.125)
 
 
+def test_head_dimension_128_at_48_heads_of_1024_tokens_sampled_heads():
+    """8 sequences x 6 heads of 128: the model width of the benchmark's shape with the wider heads."""
+    run_case(48, 1024, 1024, True, seed=13, check_heads=[0, 17, 47], HD=128)
+
+
 def test_head_dimension_128_inside_a_token_major_buffer_and_mixed_formats():
     run_case(3, 256, 256, True, merged_layout=True, q_dt=orc.E5M2, v_dt=orc.E5M2, o_dt=orc.F16, HD=128)
 

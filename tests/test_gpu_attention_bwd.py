@@ -157,6 +157,10 @@ def test_backward_head_dimension_128(H, Tq, Tk, causal):
     run_case(H, Tq, Tk, causal, HD=128)
 
 
+def test_backward_head_dimension_128_at_48_heads_of_1024_tokens_sampled_heads():
+    run_case(48, 1024, 1024, True, seed=13, check_heads=[0, 17, 47], HD=128)
+
+
 def test_backward_head_dimension_128_inside_a_token_major_buffer_and_mixed_formats():
     run_case(3, 256, 256, True, merged_layout=True, q_dt=orc.E5M2, do_dt=orc.E4M3, g_dt=orc.F16, HD=128)
 
