@@ -606,6 +606,18 @@ int scalify_scaled_colsum(const scalify_array* X, scalify_array* Y, void* worksp
                           void* stream);
 
 /*
+ * The static cast of a gradient to FP8 (Appendix A: cast_on_backward) fused with the column sums of the cast
+ * values: C = cast(X) with C_s = X_s, and Y = the column sums of C by the rule above, in one pass over X.  C, its
+ * scale and Y are the bits scalify_rescale (plain cast) followed by scalify_scaled_colsum of its output give.
+ * This is what the backward of a linear layer needs of the output gradient: its E5M2 copy for the two gradient
+ * matmuls and the bias gradient.  X: BF16 or F16 [R, N]; C: E4M3 or E5M2 [R, N] (row stride a multiple of 16
+ * bytes); Y: F16, BF16 or F32 [N].  Workspace: SCALIFY_OP_COLSUM (R, N).
+ * Errors: NULL, DTYPE, SHAPE, ALIGNMENT, WORKSPACE, ALIAS.
+ */
+int scalify_scaled_cast_colsum(const scalify_array* X, scalify_array* C, scalify_array* Y, void* workspace,
+                               size_t workspace_bytes, void* stream);
+
+/*
  * Fused scaled attention forward: S = Q K^T, P = softmax(S c), O = P V in one
  * kernel per (head, 128 queries); the scores and the probabilities stay on chip.
  * The paper names attention as a place for a custom scale rule (Section 3.2.1)

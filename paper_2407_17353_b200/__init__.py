@@ -88,6 +88,7 @@ def lib() -> ctypes.CDLL:
         L.scalify_scaled_adam_step.argtypes = [i32, P, P, P, P, f32, f32, f32, f32, i64, vp, sz, vp]
         L.scalify_scaled_attention.argtypes = [P, P, P, f32, i32, P, P, P, vp, vp]
         L.scalify_scaled_colsum.argtypes = [P, P, vp, sz, vp]
+        L.scalify_scaled_cast_colsum.argtypes = [P, P, P, vp, sz, vp]
         L.scalify_scaled_matmul_bias.argtypes = [P, i32, P, i32, P, P, i32, P, vp, sz, vp]
         L.scalify_scaled_attention_bwd.argtypes = [P, P, P, P, P, f32, i32, P, P, P, P, P, vp, vp]
         L.scalify_mx_sf_bytes.restype = sz
@@ -120,7 +121,7 @@ def lib() -> ctypes.CDLL:
                      "scalify_scaled_cross_entropy", "scalify_scalar_mul_pow2", "scalify_debug_expire_wait",
                      "scalify_debug_layernorm_plan",
                      "scalify_mx_quantize", "scalify_mx_matmul", "scalify_scaled_attention",
-                     "scalify_scaled_attention_bwd", "scalify_scaled_colsum", "scalify_scaled_matmul_bias",
+                     "scalify_scaled_attention_bwd", "scalify_scaled_colsum", "scalify_scaled_cast_colsum", "scalify_scaled_matmul_bias",
                      "scalify_scaled_matmul_speculative"):
             getattr(L, name).restype = i32
         _lib = L
@@ -519,6 +520,13 @@ def scalify_scaled_attention(Q: ScaledTensor, K: ScaledTensor, V: ScaledTensor, 
     _check(lib().scalify_scaled_attention(_ref(q), _ref(k), _ref(v), float(sm_scale), int(bool(causal)), _ref(o),
                                           _ref(sd), _ref(pd), _ptr(status), _stream(stream)),
            "scalify_scaled_attention")
+
+
+def scalify_scaled_cast_colsum(X: ScaledTensor, C: ScaledTensor, Y: ScaledTensor, ws: Workspace, stream=None) -> None:
+    """C = static cast of X to FP8, Y = column sums of C (the bias gradient), in one pass over X."""
+    x, c, y = _desc(X), _desc(C), _desc(Y)
+    _check(lib().scalify_scaled_cast_colsum(_ref(x), _ref(c), _ref(y), ws.ptr, ws.nbytes, _stream(stream)),
+           "scalify_scaled_cast_colsum")
 
 
 def scalify_scaled_colsum(X: ScaledTensor, Y: ScaledTensor, ws: Workspace, stream=None) -> None:

@@ -489,6 +489,24 @@ int scalify_scaled_colsum(const scalify_array* X, scalify_array* Y, void* worksp
                        static_cast<cudaStream_t>(stream));
 }
 
+int scalify_scaled_cast_colsum(const scalify_array* X, scalify_array* C, scalify_array* Y, void* workspace,
+                               size_t workspace_bytes, void* stream) {
+  int rc;
+  if ((rc = check_array(X)) || (rc = check_array(C)) || (rc = check_array(Y))) return rc;
+  if ((X->dtype != SCALIFY_BF16 && X->dtype != SCALIFY_F16) || is_wide(C->dtype) || !is_wide(Y->dtype)) return SCALIFY_ERR_DTYPE;
+  if (X->ndim != 2 || C->ndim != 2 || Y->ndim != 1 || Y->shape[0] != X->shape[1] || C->shape[0] != X->shape[0] ||
+      C->shape[1] != X->shape[1])
+    return SCALIFY_ERR_SHAPE;
+  const int64_t R = X->shape[0], N = X->shape[1];
+  if (R < 1 || N < 1 || X->stride[0] < N || C->stride[0] < N) return SCALIFY_ERR_SHAPE;
+  if (C->data == X->data) return SCALIFY_ERR_ALIAS;
+  if ((Y->scale && (Y->scale == X->scale || Y->scale == C->scale)) || (C->scale && C->scale == X->scale)) return SCALIFY_ERR_ALIAS;
+  rc = check_ws(workspace, workspace_bytes, scalify_workspace_bytes(SCALIFY_OP_COLSUM, R, N));
+  if (rc) return rc;
+  return launch_cast_colsum(X->data, X->dtype, X->stride[0], R, N, X->scale, C->data, C->dtype, C->stride[0], C->scale,
+                            Y->data, Y->dtype, Y->scale, workspace, static_cast<cudaStream_t>(stream));
+}
+
 // [batch, heads, T, hd] view of a 2-D, 3-D or 4-D array: counts, rows, row / head / batch strides (elements)
 struct HeadsView {
   int64_t batch, heads, rows, cols, ld, hs, bs;

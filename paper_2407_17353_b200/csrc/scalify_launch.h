@@ -69,6 +69,9 @@ int launch_softmax_bwd(const void* dP, int g_dt, const void* P, int p_dt, void* 
                        const float* dp_scale, const float* p_scale, float* ds_scale, cudaStream_t st);
 size_t cross_entropy_ws_bytes(int64_t n);
 size_t colsum_ws_bytes(int64_t N);
+int launch_cast_colsum(const void* X, int x_dt, long long ld, long long R, long long N, const float* x_scale, void* C,
+                       int c_dt, long long ldc, float* c_scale, void* Y, int y_dt, float* y_scale, void* ws,
+                       cudaStream_t st);
 int launch_colsum(const void* X, int x_dt, long long ld, long long R, long long N, const float* x_scale, void* Y, int y_dt,
                   float* y_scale, void* ws, cudaStream_t st);
 int launch_cross_entropy(const void* logits, int l_dt, long long ld, int n_classes, const long long* targets, long long n,

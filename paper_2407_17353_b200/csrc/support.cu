@@ -584,9 +584,13 @@ int launch_cross_entropy(const void* logits, int l_dt, long long ld, int n_class
 // leave one fp32 partial per column and slab.  Launch 2 adds the slabs in index order in fp64.
 constexpr int kColSlabsMax = 64;  // the finish adds 8 x 8 slabs
 
-template <int DT>
+// CDT >= 0: the fused cast (Appendix A: cast_on_backward of a gradient) - the input is also written to C in
+// format CDT, and the sums are those of the values AS CAST, so that the result is what the cast followed by
+// the column sums of its output gives.
+template <int DT, int CDT = -1>
 __global__ void __launch_bounds__(256) colsum_partial_kernel(const void* __restrict__ X, long long ld, long long R,
-                                                             long long N, int slabs, float* __restrict__ part) {
+                                                             long long N, int slabs, float* __restrict__ part,
+                                                             void* __restrict__ C = nullptr, long long ldc = 0) {
   asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   constexpr int VEC = 16 / ElemBytes<DT>::v;
   __shared__ float s_acc[8][32][VEC + 1];
@@ -613,13 +617,29 @@ __global__ void __launch_bounds__(256) colsum_partial_kernel(const void* __restr
       for (int u = 0; u < 4; ++u) {
         float f[VEC];
         decode_vec<DT, VEC>(w[u], f);
+        if constexpr (CDT >= 0) {
+          if (r + u * 8 < r1) {
+            constexpr int CB = VEC * ElemBytes<CDT>::v;
+            uint32_t cw[CB / 4];
+            encode_vec<CDT, VEC>(f, cw);
+            st_raw_stream<CB>(static_cast<char*>(C) + ((r + u * 8) * ldc + vec * VEC) * ElemBytes<CDT>::v, cw);
+            decode_vec<CDT, VEC>(cw, f);   // the values as cast
+          }
+        }
 #pragma unroll
         for (int e = 0; e < VEC; ++e) acc[e] += f[e];
       }
     }
   } else if (vec == n_vec && tail > 0) {
     for (long long r = r0 + warp; r < r1; r += 8)
-      for (int e = 0; e < tail; ++e) acc[e] += load_elem<DT>(X, r * ld + n_vec * VEC + e);
+      for (int e = 0; e < tail; ++e) {
+        float f = load_elem<DT>(X, r * ld + n_vec * VEC + e);
+        if constexpr (CDT >= 0) {
+          store_elem<CDT>(C, r * ldc + n_vec * VEC + e, f);
+          f = round_through<CDT>(f);
+        }
+        acc[e] += f;
+      }
   }
 #pragma unroll
   for (int e = 0; e < VEC; ++e) s_acc[warp][lane][e] = acc[e];
@@ -639,7 +659,8 @@ __global__ void __launch_bounds__(256) colsum_partial_kernel(const void* __restr
 template <int YDT>
 __global__ void __launch_bounds__(256) colsum_finalize_kernel(const float* __restrict__ part, long long N, int slabs,
                                                               float inv_kf, float kf, void* __restrict__ Y,
-                                                              const float* x_scale, float* y_scale, uint32_t* status) {
+                                                              const float* x_scale, float* y_scale, uint32_t* status,
+                                                              float* c_scale = nullptr) {
   asm volatile("griddepcontrol.launch_dependents;");  // a programmatic dependent may set up while this grid runs
   __shared__ double s_sum[8][32];
   const int lane = threadIdx.x & 31, grp = threadIdx.x >> 5;
@@ -663,6 +684,7 @@ __global__ void __launch_bounds__(256) colsum_finalize_kernel(const float* __res
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     const float xs = load_scale(x_scale);
     if (y_scale) *y_scale = xs * kf;
+    if (c_scale) *c_scale = xs;   // fused cast: the scale is unchanged
     if (!is_pow2_scale(xs) && status) atomicOr(status, static_cast<uint32_t>(SCALIFY_DEV_BAD_SCALE));
   }
 }
@@ -692,6 +714,34 @@ int launch_colsum(const void* X, int x_dt, long long ld, long long R, long long 
   const float kf = kfactor(R);
   SCALIFY_DISPATCH_WIDE(y_dt, YDT, colsum_finalize_kernel<YDT><<<static_cast<unsigned>((N + 31) / 32), 256, 0, st>>>(
                                        part, N, slabs, 1.0f / kf, kf, Y, x_scale, y_scale, v.status));
+  SCALIFY_CUDA_TRY(cudaGetLastError());
+  return SCALIFY_OK;
+}
+
+// Cast of a 16-bit matrix to FP8 fused with the column sums of the cast values (the bias gradient of a linear
+// layer is the column sum of the E5M2 copy of the output gradient that the weight-gradient matmul reads).  The
+// slabs are those the column sums of an FP8 matrix would get, and every column is added in the same order, so
+// the sums equal those of scalify_scaled_colsum applied to the cast output bit for bit.
+int launch_cast_colsum(const void* X, int x_dt, long long ld, long long R, long long N, const float* x_scale, void* C,
+                       int c_dt, long long ldc, float* c_scale, void* Y, int y_dt, float* y_scale, void* ws,
+                       cudaStream_t st) {
+  WsView v = ws_view(ws);
+  float* part = static_cast<float*>(v.area);
+  const int slabs = colsum_slabs(R, N, 1);
+  const long long gx = (N / 8 + 1 + 31) / 32;   // vectors of eight 16-bit columns
+  if (gx > 0x7FFFFFFF) return SCALIFY_ERR_SHAPE;
+  const dim3 grid(static_cast<unsigned>(gx), static_cast<unsigned>(slabs));
+#define SCALIFY_CCS(DT, CDT) colsum_partial_kernel<DT, CDT><<<grid, 256, 0, st>>>(X, ld, R, N, slabs, part, C, ldc)
+  if (x_dt == SCALIFY_BF16) {
+    if (c_dt == SCALIFY_E4M3) SCALIFY_CCS(SCALIFY_BF16, SCALIFY_E4M3); else SCALIFY_CCS(SCALIFY_BF16, SCALIFY_E5M2);
+  } else {
+    if (c_dt == SCALIFY_E4M3) SCALIFY_CCS(SCALIFY_F16, SCALIFY_E4M3); else SCALIFY_CCS(SCALIFY_F16, SCALIFY_E5M2);
+  }
+#undef SCALIFY_CCS
+  SCALIFY_CUDA_TRY(cudaGetLastError());
+  const float kf = kfactor(R);
+  SCALIFY_DISPATCH_WIDE(y_dt, YDT, colsum_finalize_kernel<YDT><<<static_cast<unsigned>((N + 31) / 32), 256, 0, st>>>(
+                                       part, N, slabs, 1.0f / kf, kf, Y, x_scale, y_scale, v.status, c_scale));
   SCALIFY_CUDA_TRY(cudaGetLastError());
   return SCALIFY_OK;
 }

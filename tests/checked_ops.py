@@ -365,6 +365,28 @@ class Ops:
             assert self.within(self.bits(Y), o.encode(exact, o_dt), o_dt, exact, mag, 1e-5).all()
         return Y
 
+    def cast_colsum(self, X, dt, o_dt=BF):
+        """The FP8 copy of a gradient and the column sums of that copy (the bias gradient) in one pass."""
+        R, N = X.data.shape
+        C = self.empty((R, N), dt)
+        Y = self.empty((N,), o_dt)
+        if not hasattr(self, "ws_col") or self.ws_col.nbytes < sc.scalify_workspace_bytes(sc.OP_COLSUM, R, N):
+            self.ws_col = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_COLSUM, R, N), self.dev)
+        sc.scalify_scaled_cast_colsum(X, C, Y, self.ws_col)
+        self.calls += 1
+        if self.check:
+            o = self.orc
+            assert self.ws_col.check_status() == 0
+            assert C.scale_value() == X.scale_value()
+            rows = self._rows(R, X.data.numel())
+            assert np.array_equal(self.take(C, rows), o.encode(o.decode(self.take(X, rows), code(X.data)), dt))
+            cv = o.decode(self.bits(C), dt)                       # the sums are those of the library's own cast
+            kf = o.kf(R)
+            exact, mag = cv.sum(axis=0) / kf, np.abs(cv).sum(axis=0) / kf
+            assert Y.scale_value() == X.scale_value() * kf
+            assert self.within(self.bits(Y), o.encode(exact, o_dt), o_dt, exact, mag, 1e-5).all()
+        return C, Y
+
     def attention(self, Q, K, V, O, sm_scale, causal=True):
         """Fused forward over [heads, T, 64] views; returns the E4M3 probabilities (kept for the backward).
         Checked stage by stage through the kernel's own copies of the scores and probabilities."""

@@ -102,11 +102,11 @@ class ScaledGPT:
     def _linear_bwd(self, dy, x8, W8, name):
         """dy BF16 -> (dx BF16, dW E5M2 rescaled, db E5M2 rescaled)."""
         o = self.ops
-        dy8 = o.cast(dy, E5)
+        dy8, colsums = o.cast_colsum(dy, E5)          # the E5M2 copy and its column sums in one pass over dy
         dx = o.mm(dy8, W8, transB=True)               # dy W^T: W stored [K, N] = [N', K'] of this product
         # x^T dy with fused AMAX rescale; a workspace per weight, so that the predicted rescale holds step after step
         _, dW = o.mm(x8, dy8, transA=True, stat=sc.STAT_AMAX, q_dt=E5, key=name)
-        db = o.rescale(o.colsum(dy8), sc.STAT_AMAX, E5, key=name + ".bias")   # column sums, then the dynamic rescale
+        db = o.rescale(colsums, sc.STAT_AMAX, E5, key=name + ".bias")          # the bias gradient's dynamic rescale
         return dx, dW, db
 
     # ------------------------------------------------------------------ one training step

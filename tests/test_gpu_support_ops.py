@@ -165,3 +165,63 @@ def test_column_sums(R, N, x_dt, y_dt):
     Y2 = sc.ScaledTensor.empty((N,), sc.TORCH_DTYPE[y_dt])
     sc.scalify_scaled_colsum(X, Y2, ws)
     assert np.array_equal(to_bits(Y2.data, y_dt), to_bits(Y.data, y_dt))
+
+
+@pytest.mark.parametrize("R,N,x_dt,c_dt,y_dt", [(8192, 768, orc.BF16, orc.E5M2, orc.BF16), (8192, 3072, orc.BF16, orc.E5M2, orc.F32),
+                                               (1000, 50, orc.F16, orc.E4M3, orc.BF16), (37, 1030, orc.BF16, orc.E4M3, orc.F16),
+                                               (5, 24, orc.BF16, orc.E5M2, orc.F32), (70000, 64, orc.F16, orc.E5M2, orc.F32)])
+def test_cast_fused_with_column_sums(R, N, x_dt, c_dt, y_dt):
+    """One pass over a 16-bit gradient: its FP8 cast (the oracle's encoding of every element, scale unchanged)
+    and the column sums of the CAST values by the reduce-sum rule - against the oracle, and bit for bit what the
+    plain cast followed by the column sums of its output gives."""
+    ld = (N // 16 + 2) * 16
+    spread = 40.0 if c_dt == orc.E5M2 else 4.0
+    full = si.to_bits(si.normal(93, R, (R, ld), spread), x_dt)
+    x = np.ascontiguousarray(full[:, :N])
+    X = sc.ScaledTensor.make(to_dev(full, x_dt)[:, :N], 2.0 ** -9)
+    cbuf = torch.zeros((R, ld), dtype=torch.uint8, device="cuda").view(sc.TORCH_DTYPE[c_dt])
+    cbuf.view(torch.uint8).fill_(0x55)
+    C = sc.ScaledTensor(cbuf[:, :N], torch.zeros(1, device="cuda"))
+    Y = sc.ScaledTensor.empty((N,), sc.TORCH_DTYPE[y_dt])
+    ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_COLSUM, R, N))
+    sc.scalify_scaled_cast_colsum(X, C, Y, ws)
+    assert ws.check_status() == 0
+    # the cast: every element the oracle's encoding, the padding columns untouched
+    want_c = orc.encode(orc.decode(x, x_dt), c_dt)
+    got_c = to_bits(cbuf, c_dt)
+    assert np.array_equal(got_c[:, :N], want_c) and np.all(got_c[:, N:] == 0x55)
+    assert C.scale_value() == 2.0 ** -9
+    # the sums: of the cast values
+    cv = orc.decode(want_c, c_dt)
+    kf = orc.kf(R)
+    exact, mag = cv.sum(axis=0) / kf, np.abs(cv).sum(axis=0) / kf
+    assert Y.scale_value() == 2.0 ** -9 * kf
+    ok = within(to_bits(Y.data, y_dt), orc.encode(exact, y_dt), y_dt, exact, mag, 1e-5)
+    assert ok.all(), int((~ok).sum())
+    # the same bits as the two separate calls
+    Xc = sc.ScaledTensor.make(to_dev(x, x_dt), 2.0 ** -9)
+    Cc = sc.ScaledTensor.empty((R, N), sc.TORCH_DTYPE[c_dt]) if N % 16 == 0 else None
+    if Cc is not None:
+        sc.scalify_rescale(Xc, Cc)
+        Y2 = sc.ScaledTensor.empty((N,), sc.TORCH_DTYPE[y_dt])
+        sc.scalify_scaled_colsum(Cc, Y2, ws)
+        assert np.array_equal(to_bits(Cc.data, c_dt), want_c)
+        assert Y2.scale_value() == Y.scale_value()
+        assert np.array_equal(to_bits(Y2.data, y_dt), to_bits(Y.data, y_dt))
+
+
+def test_cast_colsum_argument_checks():
+    R, N = 64, 128
+    X = sc.ScaledTensor.make(torch.zeros((R, N), dtype=torch.bfloat16, device="cuda"), 1.0)
+    C = sc.ScaledTensor.empty((R, N), torch.float8_e5m2)
+    Y = sc.ScaledTensor.empty((N,), torch.float32)
+    ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_COLSUM, R, N))
+    sc.scalify_scaled_cast_colsum(X, C, Y, ws)
+    with pytest.raises(sc.ScalifyError):   # the input is a 16-bit gradient
+        sc.scalify_scaled_cast_colsum(sc.ScaledTensor.make(torch.zeros((R, N), device="cuda"), 1.0), C, Y, ws)
+    with pytest.raises(sc.ScalifyError):   # the cast goes to FP8
+        sc.scalify_scaled_cast_colsum(X, sc.ScaledTensor.empty((R, N), torch.bfloat16), Y, ws)
+    with pytest.raises(sc.ScalifyError):   # shapes
+        sc.scalify_scaled_cast_colsum(X, sc.ScaledTensor.empty((R, N + 16), torch.float8_e5m2), Y, ws)
+    with pytest.raises(sc.ScalifyError):   # a scale word of its own
+        sc.scalify_scaled_cast_colsum(X, sc.ScaledTensor(C.data, X.scale), Y, ws)
