@@ -42,7 +42,7 @@ N_GEMM = 8192
 LN_R, LN_D = 131072, 1024
 ADAM_N = 125_000_000
 ADD_SHAPE = (8192, 8192)
-ORACLE_SAMPLE_ROWS = 1024     # cpu_baseline leg: one sample (10-30 s of CPU work)
+ORACLE_SAMPLE_ROWS = 2048     # cpu_baseline leg: one sample (10-30 s of CPU work)
 # --impl reference: the same 1024-row sample per timed step while the whole run stays within a few minutes
 # (about 7 s per sample on 16 cores), fewer rows per step for longer runs
 REFERENCE_ROWS_BUDGET = 24 * 1024
