@@ -37,6 +37,8 @@ constexpr int kEpiWarps = 8;                 // two warps per TMEM lane quarter,
 constexpr int kGemmThreads = 64 + 32 * kEpiWarps;
 constexpr int kTmemCols = kAccStages * kBN;  // 512
 constexpr int kGroupM = 16;                  // m-tiles per rasterisation group
+constexpr int kMxSfWarps = 4;                // block-scaled kernel: one warp per TMEM lane quarter writes the exponents
+constexpr int kMxGemmThreads = kGemmThreads + 32 * kMxSfWarps;
 
 // NCTA = 1: one CTA computes a 128 x 256 tile (tcgen05 cta_group::1).
 // NCTA = 2: a cluster of two CTAs on an SM pair computes a 256 x 256 tile (cta_group::2): each
@@ -44,19 +46,22 @@ constexpr int kGroupM = 16;                  // m-tiles per rasterisation group
 //           issues the MMAs, which read both CTAs' shared memory and write both CTAs' TMEM.
 //           Per SM this halves the shared-memory traffic of B, the limiter of the 1-CTA form.
 // MX: block-scaled operands (one E8M0 exponent per 32 elements of K, Section 2's block-scale
-//     generalisation): each ring slot also holds the exponent tiles of its K block (512 B for the
-//     128 rows of A, 2 x 512 B for the 256 rows of B), which the MMA warp copies into TMEM before
-//     the block's four MMAs.  TMEM then holds ONE 256-column accumulator plus 12 exponent columns.
-//     In the two-CTA form every CTA stages the exponents of its own 128 rows of A and of ALL 256
-//     rows of B (each CTA multiplies its rows of A with the whole B tile).
+//     generalisation).  The MMAs read the exponents from tensor memory: TMEM holds ONE 256-column
+//     accumulator and, behind it, one 16-column exponent buffer per ring slot (A: 4 columns, B: 8).
+//     Four extra warps, one per TMEM lane quarter, read the exponent tiles of a K block (512 B for
+//     the 128 rows of A, 2 x 512 B for the 256 rows of B) from L2, 16 bytes per lane, and write
+//     them into the slot's buffer with tcgen05.st; they wait for the slot on the same "empty"
+//     barrier as the TMA producer and arrive on the same "full" barrier as the TMA bytes, so the
+//     MMA thread issues exactly what the per-tensor kernel's does.  In the two-CTA form every CTA
+//     holds the exponents of its own 128 rows of A and of ALL 256 rows of B (each CTA multiplies
+//     its rows of A with the whole B tile).
 template <int NCTA, bool MX = false> struct GemmCfg {
   static constexpr int kTileM = kBM * NCTA;
   static constexpr int kBRows = kBN / NCTA;          // B rows (columns of the output) staged per CTA
   static constexpr int kABytes = kBM * kBK;          // 16 KB
   static constexpr int kBBytes = kBRows * kBK;       // 32 KB / 16 KB
-  static constexpr int kSfBytes = MX ? 2048 : 0;     // exponent tiles of one K block (1536 B used)
-  static constexpr int kStageBytes = kABytes + kBBytes + kSfBytes;
-  static constexpr int kStages = MX ? (NCTA == 1 ? 3 : 4) : (NCTA == 1 ? 3 : 5);
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kStages = NCTA == 1 ? 3 : 5;
   static constexpr int kAcc = MX ? 1 : kAccStages;   // accumulators in TMEM
   // Epilogue staging: 8 KB per warp = one tile (32 rows x 32 columns) per chunk of a 16-bit output, so that a
   // warp never waits for the TMA store of an earlier chunk of the same accumulator (two tiles for fp32 output).
@@ -64,10 +69,9 @@ template <int NCTA, bool MX = false> struct GemmCfg {
   static constexpr int kEpiBytes = kEpiWarps * kEpiWarpBytes;
   static constexpr size_t kSmem = size_t(kStages) * kStageBytes + kEpiBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
-// MX: TMEM columns of the exponents, two buffers 64 columns apart (A: 4 columns at +0, B: 8 columns at +32)
-// used by alternate K blocks so that the copy for one block does not have to wait for the MMAs of the block
-// before it
+// MX: TMEM columns of the exponents: one buffer of 16 columns per ring slot (A: 4 columns at +0, B: 8 columns at +4)
 constexpr uint32_t kSfaTmemCol = 256;
+constexpr uint32_t kMxSfCols = 16;
 
 struct GemmParams {
   int M, N, K, batch;
@@ -129,8 +133,7 @@ __device__ __forceinline__ void tile_coords(const GemmParams& p, int tile, int& 
   nt = r / gm;
 }
 
-// map_sfa is the exponent map of A in the block-scaled form and the map of the speculative FP8 output in the
-// SPEC form (the two never occur together).
+// map_sfa is the map of the speculative FP8 output in the SPEC form (map_sfb is not used).
 template <int OUT, int NCTA, bool MX, bool SPEC = false, bool BIAS = false, bool NOY = false>
 __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_y,
                                           const CUtensorMap& map_sfa, const CUtensorMap& map_sfb, const GemmParams& p) {
@@ -156,7 +159,6 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
   uint8_t* smem = smem_raw + (base - raw);
   const uint32_t smem_a = base;
   const uint32_t smem_b = base + kStages * C::kABytes;
-  const uint32_t smem_sf = smem_b + kStages * C::kBBytes;  // MX: [stage][A exponents 512 B | B exponents 2 x 512 B | pad]
   uint8_t* epi_mem = smem + kStages * C::kStageBytes;  // 8 KB per epilogue warp, 1024-byte aligned
   uint8_t* bar_mem = epi_mem + C::kEpiBytes;
   const uint32_t bars = base + kStages * C::kStageBytes + C::kEpiBytes;
@@ -176,7 +178,8 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
   const int num_tiles = p.tiles_m * p.tiles_n * p.batch;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(full_bar + 8 * s, 1); mbar_init(empty_bar + 8 * s, 1); }
+    // MX: besides the producer's arrival (with the byte count), one arrival per exponent warp of every CTA of the pair
+    for (int s = 0; s < kStages; ++s) { mbar_init(full_bar + 8 * s, MX ? 1 + kMxSfWarps * NCTA : 1); mbar_init(empty_bar + 8 * s, 1); }
     for (int s = 0; s < kAccStages; ++s) {
       mbar_init(acc_full_bar + 8 * s, 1);
       mbar_init(acc_empty_bar + 8 * s, kEpiWarps * NCTA);  // one arrival per epilogue warp of every CTA of the pair
@@ -238,13 +241,7 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
           const int bb = p.b_batched ? b : 0;
           if constexpr (NCTA == 1) {
             const uint32_t fb = full_bar + 8 * stage;
-            mbar_expect_tx(fb, C::kABytes + C::kBBytes + (MX ? 1536 : 0));
-            if constexpr (MX) {
-              const uint32_t ssf = smem_sf + stage * C::kSfBytes;
-              bulk_load(ssf, p.sfa + (static_cast<size_t>(mt) * num_kb + kb) * 512, 512, fb);
-              bulk_load(ssf + 512, p.sfb + (static_cast<size_t>(2 * nt) * num_kb + kb) * 512, 512, fb);
-              bulk_load(ssf + 1024, p.sfb + (static_cast<size_t>(2 * nt + 1) * num_kb + kb) * 512, 512, fb);
-            }
+            mbar_expect_tx(fb, C::kABytes + C::kBBytes);
             if (p.a_mn_major) tma_load_3d(sa, &map_a, fb, m0, k0, b);
             else tma_load_3d(sa, &map_a, fb, k0, m0, b);
             if (p.b_mn_major) {
@@ -256,18 +253,11 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
           } else {
             // both CTAs' copies are counted on the LEADER's full barrier, which expects the bytes of the pair
             const uint32_t fb = map_to_cta(full_bar + 8 * stage, 0u);
-            if (rank == 0u) mbar_expect_tx(full_bar + 8 * stage, 2 * (C::kABytes + C::kBBytes + (MX ? 1536 : 0)));
+            if (rank == 0u) mbar_expect_tx(full_bar + 8 * stage, 2 * (C::kABytes + C::kBBytes));
             if (p.a_mn_major) tma_load_3d_pair(sa, &map_a, fb, m0, k0, b);
             else tma_load_3d_pair(sa, &map_a, fb, k0, m0, b);
             if (p.b_mn_major) tma_load_3d_pair(sb, &map_b, fb, n0, k0, bb);
             else tma_load_3d_pair(sb, &map_b, fb, k0, n0, bb);
-            if constexpr (MX) {
-              // exponent tiles (rows of 512 bytes in the tile list): own half of A, both halves of B
-              const uint32_t ssf = smem_sf + stage * C::kSfBytes;
-              tma_load_3d_pair(ssf, &map_sfa, fb, 0, (2 * mt + static_cast<int>(rank)) * num_kb + kb, 0);
-              tma_load_3d_pair(ssf + 512, &map_sfb, fb, 0, (2 * nt) * num_kb + kb, 0);
-              tma_load_3d_pair(ssf + 1024, &map_sfb, fb, 0, (2 * nt + 1) * num_kb + kb, 0);
-            }
           }
           ++issued;
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
@@ -299,8 +289,7 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
       // 2^18 bytes), and the four instruction descriptors of a K block.
       const uint64_t a_desc0 = make_smem_desc(smem_a, a_lbo, a_sbo);
       const uint64_t b_desc0 = make_smem_desc(smem_b, b_lbo, b_sbo);
-      const uint64_t sf_desc0 = make_smem_desc_noswizzle(smem_sf, 512u, 128u);
-      constexpr uint32_t kAStageInc = C::kABytes >> 4, kBStageInc = C::kBBytes >> 4, kSfStageInc = C::kSfBytes >> 4;
+      constexpr uint32_t kAStageInc = C::kABytes >> 4, kBStageInc = C::kBBytes >> 4;
       const uint32_t a_k_inc = a_step >> 4, b_k_inc = b_step >> 4;
       uint32_t idesc_k[kBK / kUmmaK];
 #pragma unroll
@@ -315,29 +304,16 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
           tc_fence_after();
           const uint64_t ad0 = a_desc0 + static_cast<uint64_t>(stage * kAStageInc);
           const uint64_t bd0 = b_desc0 + static_cast<uint64_t>(stage * kBStageInc);
-          const uint32_t sf_col = tmem_base + kSfaTmemCol + static_cast<uint32_t>(kb & 1) * 64u;
-          if constexpr (MX) {
-            // this K block's exponents: shared memory -> TMEM (executes in order with the MMAs of this thread);
-            // A's tile, then the two tiles of B, 512 bytes apart in the slot
-            const uint64_t sfd = sf_desc0 + static_cast<uint64_t>(stage * kSfStageInc);
-            if constexpr (NCTA == 1) {
-              tmem_cp_32x128b_warpx4(sf_col, sfd);
-              tmem_cp_32x128b_warpx4(sf_col + 32, sfd + 32);
-              tmem_cp_32x128b_warpx4(sf_col + 36, sfd + 64);
-            } else {
-              tmem_cp_32x128b_warpx4_pair(sf_col, sfd);
-              tmem_cp_32x128b_warpx4_pair(sf_col + 32, sfd + 32);
-              tmem_cp_32x128b_warpx4_pair(sf_col + 36, sfd + 64);
-            }
-          }
+          // MX: the slot's exponents are in tensor memory (the "full" barrier also counts the exponent warps)
+          const uint32_t sf_col = tmem_base + kSfaTmemCol + stage * kMxSfCols;
 #pragma unroll
           for (int k = 0; k < kBK / kUmmaK; ++k) {
             const uint64_t ad = ad0 + static_cast<uint64_t>(k * a_k_inc);
             const uint64_t bd = bd0 + static_cast<uint64_t>(k * b_k_inc);
             const uint32_t accumulate = (kb | k) != 0 ? 1u : 0u;
             if constexpr (MX) {
-              if constexpr (NCTA == 1) umma_mxf8(d_tmem, ad, bd, idesc_k[k], accumulate, sf_col, sf_col + 32);
-              else umma_mxf8_pair(d_tmem, ad, bd, idesc_k[k], accumulate, sf_col, sf_col + 32);
+              if constexpr (NCTA == 1) umma_mxf8(d_tmem, ad, bd, idesc_k[k], accumulate, sf_col, sf_col + 4);
+              else umma_mxf8_pair(d_tmem, ad, bd, idesc_k[k], accumulate, sf_col, sf_col + 4);
             } else if constexpr (NCTA == 1) {
               umma_f8(d_tmem, ad, bd, idesc_k[k], accumulate);
             } else {
@@ -363,8 +339,67 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap& map_a, const CUtens
         while (!mbar_try_wait(drain_bar, 0u) && global_timer_ns() - t0 < kWaitLimitNs) {}
       }
     }
+  } else if (MX && warp >= 2 + kEpiWarps) {
+    // ---------------------------------------------------------------- exponent warps (block-scaled kernel)
+    // One warp per TMEM lane quarter.  A 512-byte exponent tile is 16 bytes per row % 32 (byte (row / 32) * 4 +
+    // block), which is what lane (row % 32) of EVERY quarter must hold in four consecutive columns: each warp
+    // reads the tile with one 16-byte load per lane (from L2: the four warps and the peer CTA read the same
+    // bytes) and stores it into its own quarter of the ring slot's exponent buffer.  The loads of the next three
+    // K blocks are in flight while the current three are stored.
+    const int q = warp & 3;
+    const uint32_t t_sf = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + kSfaTmemCol;
+    uint32_t stage = 0, phase = 0;
+    for (int tile = unit; tile < num_tiles && !timed_out; tile += num_units) {
+      int b, mt, nt;
+      tile_coords(p, tile, b, mt, nt);
+      const uint4* ta = reinterpret_cast<const uint4*>(p.sfa) +
+                        (static_cast<size_t>(NCTA == 2 ? 2 * mt + static_cast<int>(rank) : mt) * num_kb) * 32 + lane;
+      const uint4* tb0 = reinterpret_cast<const uint4*>(p.sfb) + (static_cast<size_t>(2 * nt) * num_kb) * 32 + lane;
+      const uint4* tb1 = reinterpret_cast<const uint4*>(p.sfb) + (static_cast<size_t>(2 * nt + 1) * num_kb) * 32 + lane;
+      constexpr int kG = 3;  // K blocks per group of loads (registers: two groups of 12 per block)
+      uint4 va[kG], vb0[kG], vb1[kG], na[kG], nb0[kG], nb1[kG];
+      auto load_group = [&](int kb0, uint4 (&xa)[kG], uint4 (&xb0)[kG], uint4 (&xb1)[kG]) {
+#pragma unroll
+        for (int j = 0; j < kG; ++j) {
+          if (kb0 + j < num_kb) {
+            ld_raw<16>(ta + (kb0 + j) * 32, reinterpret_cast<uint32_t*>(&xa[j]));
+            ld_raw<16>(tb0 + (kb0 + j) * 32, reinterpret_cast<uint32_t*>(&xb0[j]));
+            ld_raw<16>(tb1 + (kb0 + j) * 32, reinterpret_cast<uint32_t*>(&xb1[j]));
+          }
+        }
+      };
+      load_group(0, va, vb0, vb1);
+      for (int kb0 = 0; kb0 < num_kb && !timed_out; kb0 += kG) {
+        if (kb0 + kG < num_kb) load_group(kb0 + kG, na, nb0, nb1);
+#pragma unroll
+        for (int j = 0; j < kG; ++j) {
+          if (kb0 + j < num_kb && !timed_out) {
+            // the MMAs that read this slot (operands and exponents) one ring revolution ago have completed
+            if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag)) {
+              timed_out = true;
+            } else {
+              tc_fence_after();
+              const uint32_t col = t_sf + stage * kMxSfCols;
+              tmem_st4(col, va[j]);
+              tmem_st4(col + 4u, vb0[j]);
+              tmem_st4(col + 8u, vb1[j]);
+              tmem_st_wait();
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0) {
+                if constexpr (NCTA == 1) mbar_arrive(full_bar + 8 * stage);
+                else mbar_arrive_cluster(map_to_cta(full_bar + 8 * stage, 0u));  // the leader issues the MMAs
+              }
+              if (++stage == kStages) { stage = 0; phase ^= 1u; }
+            }
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < kG; ++j) { va[j] = na[j]; vb0[j] = nb0[j]; vb1[j] = nb1[j]; }
+      }
+    }
   } else {
-    // ---------------------------------------------------------------- epilogue (warps 2..5)
+    // ---------------------------------------------------------------- epilogue (warps 2..9)
     const int q = warp & 3;                       // TMEM lane quarter this warp may read
     const int half = (warp - 2) / 4;              // which half of the tile's columns this warp handles
     constexpr int kChunksPerWarp = (kBN / 32) / (kEpiWarps / 4);
@@ -634,11 +669,10 @@ scaled_matmul_fp8only_kernel(const __grid_constant__ CUtensorMap map_a, const __
 
 // Block-scaled operands (E8M0 exponent per 32 elements of K), K-major A [M,K] and B [N,K].
 template <int OUT, int NCTA>
-__global__ void __launch_bounds__(kGemmThreads, 1)
+__global__ void __launch_bounds__(kMxGemmThreads, 1)
 mx_matmul_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                 const __grid_constant__ CUtensorMap map_y, const __grid_constant__ CUtensorMap map_sfa,
-                 const __grid_constant__ CUtensorMap map_sfb, const GemmParams p) {
-  gemm_body<OUT, NCTA, true>(map_a, map_b, map_y, map_sfa, map_sfb, p);
+                 const __grid_constant__ CUtensorMap map_y, const GemmParams p) {
+  gemm_body<OUT, NCTA, true>(map_a, map_b, map_y, map_a, map_a, p);
 }
 
 // Diagnostic: one thread waits, with the GEMM's bounded-wait routine and a short limit, on an
@@ -1208,23 +1242,9 @@ int launch_scaled_matmul(const MatmulArgs& a, void* ws, size_t ws_bytes, cudaStr
   return SCALIFY_OK;
 }
 
-// Tensor map over the exponent tiles of a block-scaled operand: a list of 512-byte tiles, one per box.
-static int make_map_sf(CUtensorMap* map, const void* ptr, uint64_t n_tiles) {
-  EncodeTiledFn fn = get_encode_fn();
-  if (!fn) return SCALIFY_ERR_CUDA;
-  cuuint64_t dims[3] = {128, n_tiles, 1};  // 128 32-bit words = 512 bytes per tile
-  cuuint64_t strides[2] = {512, 512 * n_tiles};
-  cuuint32_t box[3] = {128u, 1u, 1u};
-  cuuint32_t estr[3] = {1u, 1u, 1u};
-  return encode_tiled_cached(g_map_cache, fn, map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<void*>(ptr), dims, strides,
-                             box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
-                             CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-}
-
 template <int OUT, int NCTA>
 static int launch_mx_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_y,
-                             const CUtensorMap& map_sfa, const CUtensorMap& map_sfb, const GemmParams& p,
-                             long long tiles, cudaStream_t st) {
+                             const GemmParams& p, long long tiles, cudaStream_t st) {
   using C = GemmCfg<NCTA, true>;
   auto kernel = mx_matmul_kernel<OUT, NCTA>;
   cudaLaunchAttribute attrs[1];
@@ -1237,7 +1257,7 @@ static int launch_mx_variant(const CUtensorMap& map_a, const CUtensorMap& map_b,
     if (NCTA == 2) {
       cudaLaunchConfig_t qc = {};
       qc.gridDim = dim3(unsigned(sm_count() / 2 * 2));
-      qc.blockDim = dim3(kGemmThreads);
+      qc.blockDim = dim3(kMxGemmThreads);
       qc.dynamicSmemBytes = C::kSmem;
       qc.attrs = attrs;
       qc.numAttrs = 1;
@@ -1263,10 +1283,10 @@ static int launch_mx_variant(const CUtensorMap& map_a, const CUtensorMap& map_b,
     cfg.gridDim = dim3(unsigned(tiles < sm_count() ? tiles : sm_count()));
     cfg.numAttrs = 1;
   }
-  cfg.blockDim = dim3(kGemmThreads);
+  cfg.blockDim = dim3(kMxGemmThreads);
   cfg.dynamicSmemBytes = C::kSmem;
   cfg.stream = st;
-  SCALIFY_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, map_a, map_b, map_y, map_sfa, map_sfb, p));
+  SCALIFY_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, map_a, map_b, map_y, p));
   return SCALIFY_OK;
 }
 
@@ -1274,7 +1294,7 @@ int launch_mx_matmul(const MxMatmulArgs& a, void* ws, cudaStream_t st) {
   WsView v = ws_view(ws);
   const int ncta = (a.M > kBM && a.force_ncta != 1) ? 2 : 1;
   const int tile_m = kBM * ncta;
-  CUtensorMap map_a, map_b, map_y, map_sfa, map_sfb;
+  CUtensorMap map_a, map_b, map_y;
   // K-major operand [rows, K]: box of 128 (or 256) rows x 128 bytes of K; transposed operand [K, rows]: box of
   // 128 K-rows x 128 bytes of rows, consumed MN-major (as the per-tensor kernel does for transA / plain B)
   int rc;
@@ -1285,11 +1305,6 @@ int launch_mx_matmul(const MxMatmulArgs& a, void* ws, cudaStream_t st) {
   else rc = make_map(&map_b, a.B, a.N, a.K, 1, a.N, 0, kBK);
   if (rc) return rc;
   rc = make_map_y(&map_y, a.Y, elem_size(a.y_dt), a.N, a.M, 1, a.ldy, 0);
-  if (rc) return rc;
-  const uint64_t k_tiles = uint64_t(a.K) / 128;
-  rc = make_map_sf(&map_sfa, a.sfa, uint64_t((a.M + 255) / 256 * 2) * k_tiles);
-  if (rc) return rc;
-  rc = make_map_sf(&map_sfb, a.sfb, uint64_t((a.N + 255) / 256 * 2) * k_tiles);
   if (rc) return rc;
   GemmParams p;
   p.M = a.M; p.N = a.N; p.K = a.K; p.batch = 1;
@@ -1325,8 +1340,8 @@ int launch_mx_matmul(const MxMatmulArgs& a, void* ws, cudaStream_t st) {
   const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n;
   if (tiles > (1ll << 30)) return SCALIFY_ERR_SHAPE;
   SCALIFY_DISPATCH_WIDE(a.y_dt, OUT, {
-    if (ncta == 2) rc = launch_mx_variant<OUT, 2>(map_a, map_b, map_y, map_sfa, map_sfb, p, tiles, st);
-    else rc = launch_mx_variant<OUT, 1>(map_a, map_b, map_y, map_sfa, map_sfb, p, tiles, st);
+    if (ncta == 2) rc = launch_mx_variant<OUT, 2>(map_a, map_b, map_y, p, tiles, st);
+    else rc = launch_mx_variant<OUT, 1>(map_a, map_b, map_y, p, tiles, st);
   });
   if (rc) return rc;
   if (a.stat == SCALIFY_STAT_L2) {
