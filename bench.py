@@ -250,6 +250,19 @@ def run_profile_row(args):
             sc.scalify_mx_quantize(Xb, Bm)
             sc.scalify_mx_matmul(Am, Bm, Y, ws, stat=sc.STAT_AMAX)
         work = {"flop": 2.0 * n ** 3}
+    elif row == "mx_gemm":
+        # the block-scaled GEMM alone (operands quantised once, outside the timed calls); --zero-operands as above
+        n = N_GEMM
+        std = 0.0 if args.zero_operands else 1.0
+        Xa = sc.ScaledTensor.make(rnd((n, n), torch.bfloat16, 1, std), 1.0)
+        Xb = sc.ScaledTensor.make(rnd((n, n), torch.bfloat16, 2, std), 1.0)
+        Am, Bm = sc.MxTensor(n, n, device=dev), sc.MxTensor(n, n, device=dev)
+        sc.scalify_mx_quantize(Xa, Am)
+        sc.scalify_mx_quantize(Xb, Bm)
+        Y = sc.ScaledTensor.empty((n, n), torch.bfloat16, dev)
+        ws = sc.Workspace(sc.scalify_workspace_bytes(sc.OP_MATMUL, n, n), dev)
+        fn = lambda t: sc.scalify_mx_matmul(Am, Bm, Y, ws, stat=sc.STAT_AMAX)
+        work = {"flop": 2.0 * n ** 3}
     elif row == "attention":
         H, T, HD = 96, 1024, 64
         Qa, Ka, Va = (sc.ScaledTensor.make(rnd((H, T, HD), torch.float8_e4m3fn, 30 + i), 1.0) for i in range(3))
@@ -494,14 +507,14 @@ def main():
                     help="print one JSON line per size of the HBM-bound rows (LayerNorm, rescale, add) instead of the step")
     ap.add_argument("--no-next", action="store_true",
                     help="skip the separately timed next-row variants f1, f2 (for ncu launch lists of the step)")
-    ap.add_argument("--profile-row", default=None, choices=["matmul", "headline", "mx", "mx_quantize_t", "attention", "attention_bwd", "rescale", "add", "layernorm",
+    ap.add_argument("--profile-row", default=None, choices=["matmul", "headline", "mx", "mx_gemm", "mx_quantize_t", "attention", "attention_bwd", "rescale", "add", "layernorm",
                              "layernorm_onepass", "adam"],
                     help="run only this row on a reduced, still larger-than-L2 case (for ncu captures)")
     ap.add_argument("--gpt-step", action="store_true",
                     help="time the config-5 step (GPT-2-small shapes) instead; with --graph replayed from a CUDA graph")
     ap.add_argument("--graph", action="store_true")
     ap.add_argument("--zero-operands", action="store_true",
-                    help="with --profile-row matmul: all-zero operands (the kernel without the power cap binding)")
+                    help="with --profile-row matmul or mx_gemm: all-zero operands (the kernel without the power cap binding)")
     args = ap.parse_args()
     if args.gpt_step:
         run_gpt_step(args)
