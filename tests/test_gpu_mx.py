@@ -114,6 +114,25 @@ def test_mx_matmul_against_oracle(M, N, K, a_dt, b_dt):
     assert stat == float(np.abs(orc.decode(gb, orc.BF16)).max())
 
 
+@pytest.mark.parametrize("M,N,K", [(2304, 2560, 640), (1280, 4864, 128)])
+def test_mx_matmul_more_tiles_than_ctas(M, N, K):
+    """90 and 95 output tiles of 256 x 256 on 74 CTA pairs: some pairs compute two tiles, so the ring of
+    operand slots and exponent buffers runs on across a tile boundary at a K-block count (5, 1) that is neither
+    a multiple of the ring depth nor of the exponent warps' load group.  Every element against the oracle."""
+    a_dt = b_dt = orc.E4M3
+    a = si.to_bits(si.normal(31, M + K, (M, K), 1.0), a_dt)
+    b = si.to_bits(si.normal(32, N + K, (N, K), 1.0), b_dt)
+    rng = np.random.default_rng(M + 3 * N + K)
+    ea = rng.integers(117, 138, size=(M, K // 32)).astype(np.uint8)
+    eb = rng.integers(117, 138, size=(N, K // 32)).astype(np.uint8)
+    Yo, ys, acc, sab = orc.mx_matmul(a, a_dt, ea, 0.5, b, b_dt, eb, 2.0, orc.BF16, want_acc=True)
+    gb, sb, stat = run_mx_matmul(a, a_dt, ea, 0.5, b, b_dt, eb, 2.0, orc.BF16, stat=sc.STAT_AMAX)
+    assert sb == ys
+    ok = within(gb, Yo, orc.BF16, acc, sab, 1e-5)
+    assert ok.all(), int((~ok).sum())
+    assert stat == float(np.abs(orc.decode(gb, orc.BF16)).max())
+
+
 @pytest.mark.parametrize("M", [128, 256])
 def test_mx_matmul_distinguishes_every_exponent_byte(M):
     """One block of A and one block of B get a large exponent each, at every position in turn: a kernel
